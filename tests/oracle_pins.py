@@ -1,0 +1,410 @@
+"""Pins that tie the CPU oracle to the paper and to plain mathematics.
+
+Every function takes the loaded oracle library (so that the very same checks can be
+run against deliberately broken copies of the oracle, see test_oracle_mutants.py)
+and raises AssertionError when the oracle disagrees with
+
+  * hand-worked iterations of Algorithm 1 (tests/golden/*.txt),
+  * exact rational arithmetic (fractions.Fraction) for the mean of |x| (Def. 4),
+  * brute-force Python loops for bit packing and for sorting by magnitude (Def. 2),
+  * the contraction property of Def. 1 and the identities that follow from Def. 4,
+  * the error recursion e_{t+1} = v_t - p_t and Lemma 3,
+  * plain SGD for the identity operator with one worker.
+"""
+from __future__ import annotations
+
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+
+import oracle
+from oracle import IDENTITY, SIGN, TOPK
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+
+
+# ----------------------------------------------------------------------------- helpers
+
+def read_golden(name):
+    out = {}
+    with open(os.path.join(GOLDEN, name)) as fh:
+        for line in fh:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            key, vals = line.split(":")
+            out[key.strip()] = [float(v) for v in vals.split()]
+    return out
+
+
+def decode_sign(words, scales, off):
+    off = np.asarray(off, dtype=np.int64)
+    d = int(off[-1])
+    out = np.zeros(d, np.float32)
+    woff = 0
+    for t in range(len(off) - 1):
+        n = int(off[t + 1] - off[t])
+        for j in range(n):
+            bit = (int(words[woff + j // 32]) >> (j % 32)) & 1
+            out[off[t] + j] = -scales[t] if bit else scales[t]
+        woff += (n + 31) // 32
+    return out
+
+
+def decode_topk(idx, val, d):
+    out = np.zeros(d, np.float32)
+    out[np.asarray(idx, dtype=np.int64)] = val
+    return out
+
+
+def brute_topk(x, k):
+    """Indices of the k largest |x| (ties to the lower index), ascending.  Pure Python."""
+    order = sorted(range(len(x)), key=lambda j: (-abs(float(x[j])), j))
+    return sorted(order[:k])
+
+
+def exact_mean_abs_f32(x):
+    """float32 nearest to the exact rational mean of |x|."""
+    total = sum((Fraction(abs(float(v))) for v in x), Fraction(0))
+    mean = total / len(x)
+    f = np.float32(float(mean))           # Fraction -> double is correctly rounded
+    # resolve double rounding: pick the float32 neighbour closest to the exact mean
+    cands = [f, np.nextafter(f, np.float32(np.inf)), np.nextafter(f, np.float32(-np.inf))]
+    return min(cands, key=lambda c: abs(Fraction(float(c)) - mean))
+
+
+# ----------------------------------------------------------------------------- golden
+
+def _run_golden(L, name, up, down):
+    g = read_golden(name)
+    N, d = int(g["N"][0]), int(g["d"][0])
+    off = np.asarray(g["off"], dtype=np.int64)
+    k = np.asarray(g["k"], dtype=np.int64) if "k" in g else None
+    lr = g["lr"][0]
+    X = np.tile(np.asarray(g["x0"], np.float32), (N, 1)).copy()
+    e = np.zeros(d, np.float32)
+    step = 1
+    while f"g.{step}.0" in g:
+        G = np.asarray([g[f"g.{step}.{i}"] for i in range(N)], np.float32)
+        r = oracle.step(X, e, G, lr, off, up, down, k=k, _lib=L)
+        for i in range(N):
+            if up == SIGN:
+                assert r.up_scales[i].tolist() == g[f"up_scales.{step}.{i}"], (name, step, i, "up_scales")
+                assert r.up_words[i].tolist() == g[f"up_words.{step}.{i}"], (name, step, i, "up_words")
+            if up == TOPK:
+                assert r.up_idx[i].tolist() == g[f"up_idx.{step}.{i}"], (name, step, i, "up_idx")
+                assert r.up_val[i].tolist() == g[f"up_val.{step}.{i}"], (name, step, i, "up_val")
+            assert X[i].tolist() == g[f"x.{step}.{i}"], (name, step, i, "x", X[i])
+        assert r.v.tolist() == g[f"v.{step}"], (name, step, "v", r.v)
+        if down == SIGN:
+            assert r.down_scales.tolist() == g[f"down_scales.{step}"], (name, step, "down_scales")
+            assert r.down_words.tolist() == g[f"down_words.{step}"], (name, step, "down_words")
+        if down == TOPK:
+            assert r.down_idx.tolist() == g[f"down_idx.{step}"], (name, step, "down_idx")
+            assert r.down_val.tolist() == g[f"down_val.{step}"], (name, step, "down_val")
+        assert e.tolist() == g[f"e.{step}"], (name, step, "e", e)
+        step += 1
+    assert step > 1
+
+
+def pin_golden_sign(L):
+    _run_golden(L, "sign_two_steps.txt", SIGN, SIGN)
+
+
+def pin_golden_blockwise(L):
+    _run_golden(L, "blockwise_one_step.txt", SIGN, SIGN)
+
+
+def pin_golden_topk(L):
+    _run_golden(L, "topk_one_step.txt", TOPK, TOPK)
+
+
+# ----------------------------------------------------------------------------- scaled sign
+
+def pin_scale_is_exact_mean(L):
+    """Def. 4: the scale is ||x||_1 / d.  Compared with exact rational arithmetic."""
+    rng = np.random.default_rng(11)
+    for n in (1, 2, 3, 5, 31, 32, 33, 100, 257, 1000, 4097):
+        x = rng.standard_normal(n).astype(np.float32)
+        assert oracle.scale(x, _lib=L) == exact_mean_abs_f32(x), n
+        x = (rng.standard_normal(n) * np.exp(rng.uniform(-20, 20, n))).astype(np.float32)
+        assert oracle.scale(x, _lib=L) == exact_mean_abs_f32(x), ("wide", n)
+    # closed forms
+    assert oracle.scale(np.full(64, -0.75, np.float32), _lib=L) == np.float32(0.75)
+    assert oracle.scale(np.asarray([1, -2, 3, -4], np.float32), _lib=L) == np.float32(2.5)
+    assert oracle.scale(np.asarray([0.0, -0.0, 0.0], np.float32), _lib=L) == np.float32(0.0)
+    assert oracle.scale(np.asarray([3.0, 0.0, 0.0], np.float32), _lib=L) == np.float32(1.0)
+
+
+def pin_tree_shape(L):
+    """The binary64 sum follows the balanced tree over the zero-padded power of two.
+
+    Expected values derived by hand from IEEE round-to-nearest-even:
+    2^53 + 1 rounds back to 2^53, while 1 + 1 = 2 is added exactly.
+    """
+    big = float(2 ** 53)
+    t = lambda v: oracle.tree_abs_sum(np.asarray(v, np.float32), _lib=L)
+    assert t([big, 1, 1, 1]) == big + 2          # (big+1) + (1+1); a running sum gives big
+    assert t([1, 1, 1, big]) == big + 2          # (1+1) + (1+big)
+    assert t([big, 1, 1]) == big                 # (big+1) + (1+0) = big + 1 -> ties to even
+    assert t([1, big, 1, 1, 1, 1, 1, 1]) == big + 6   # ((1+big)+(1+1)) + ((1+1)+(1+1))
+    assert t([big, 1, 1, 1, 1]) == big + 4       # padded to 8: ((big+1)+(1+1)) + ((1+0)+0) = (big+2)+1 -> ties to even
+    assert t([-1.5, 2.5]) == 4.0
+    x = np.random.default_rng(5).standard_normal(1000).astype(np.float32)
+    assert abs(t(x) - math.fsum(abs(float(v)) for v in x)) <= 1e-12 * 1000
+
+
+def pin_sign_bits_bruteforce(L):
+    """Bit b of word w of segment t is set iff element off[t]+32w+b < 0; padding bits 0."""
+    rng = np.random.default_rng(3)
+    sizes = [1, 7, 32, 33, 64, 95, 1, 130]
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    x = rng.standard_normal(int(off[-1])).astype(np.float32)
+    x[::11] = 0.0
+    x[5::13] = -0.0
+    words, scales, dec = oracle.sign_compress(x, off, _lib=L)
+    assert len(words) == sum((n + 31) // 32 for n in sizes)
+    woff = 0
+    negatives = 0
+    for t, n in enumerate(sizes):
+        seg = x[off[t]:off[t + 1]]
+        expect = [0] * ((n + 31) // 32)
+        for j in range(n):
+            if float(seg[j]) < 0.0:
+                expect[j // 32] |= 1 << (j % 32)
+                negatives += 1
+        assert [int(w) for w in words[woff:woff + len(expect)]] == expect, t
+        assert scales[t] == exact_mean_abs_f32(seg), t
+        for j in range(n):
+            want = -scales[t] if float(seg[j]) < 0.0 else scales[t]
+            assert dec[off[t] + j] == want
+        woff += len(expect)
+    assert sum(bin(int(w)).count("1") for w in words) == negatives
+    assert np.array_equal(decode_sign(words, scales, off), dec)
+
+
+def pin_sign_contraction(L):
+    """Def. 1 with Def. 4: ||x - C(x)||^2 = ||x||^2 - d s^2 <= (1 - delta)||x||^2, delta -> 2/pi on Gaussians."""
+    rng = np.random.default_rng(7)
+    n = 200_000
+    x = rng.standard_normal(n).astype(np.float32)
+    _, scales, dec = oracle.sign_compress(x, [0, n], _lib=L)
+    x64, c64 = x.astype(np.float64), dec.astype(np.float64)
+    lhs = np.sum((x64 - c64) ** 2)
+    rhs = np.sum(x64 ** 2) - n * float(scales[0]) ** 2
+    assert abs(lhs - rhs) <= 1e-6 * rhs
+    delta = 1.0 - lhs / np.sum(x64 ** 2)
+    assert abs(delta - 2.0 / math.pi) < 0.01
+    assert abs(float(scales[0]) - math.sqrt(2.0 / math.pi)) < 0.01
+
+
+def pin_blockwise_reduces_to_sign(L):
+    """Def. 5 with one block is Def. 4; with several blocks it is Def. 4 per block."""
+    rng = np.random.default_rng(9)
+    x = rng.standard_normal(300).astype(np.float32)
+    w1, s1, d1 = oracle.sign_compress(x, [0, 300], _lib=L)
+    assert s1[0] == exact_mean_abs_f32(x)
+    off = [0, 64, 96, 300]
+    w, s, d = oracle.sign_compress(x, off, _lib=L)
+    wcat, dcat = [], []
+    for t in range(3):
+        wt, st, dt = oracle.sign_compress(x[off[t]:off[t + 1]], [0, off[t + 1] - off[t]], _lib=L)
+        assert st[0] == s[t]
+        wcat.append(wt)
+        dcat.append(dt)
+    assert np.array_equal(np.concatenate(wcat), w) and np.array_equal(np.concatenate(dcat), d)
+    # idempotence when the block length is a power of two (n * s / n is exact)
+    x = rng.standard_normal(256).astype(np.float32)
+    _, s_a, d_a = oracle.sign_compress(x, [0, 256], _lib=L)
+    w_b, s_b, d_b = oracle.sign_compress(d_a, [0, 256], _lib=L)
+    assert s_a[0] == s_b[0] and np.array_equal(d_a, d_b)
+
+
+# ----------------------------------------------------------------------------- top-k
+
+def pin_topk_bruteforce(L):
+    """Def. 2 against a full Python sort, with heavy ties, zeros and +-pairs."""
+    rng = np.random.default_rng(13)
+    cases = []
+    cases.append((rng.integers(-3, 4, 200).astype(np.float32), 17))          # many ties
+    cases.append((np.zeros(50, np.float32), 5))                               # all equal (zeros)
+    cases.append((np.full(40, -2.0, np.float32), 7))                          # all equal, negative
+    cases.append((np.asarray([1, -1, 1, -1, 1, -1], np.float32), 3))          # +- pairs
+    cases.append((rng.standard_normal(1000).astype(np.float32), 1))           # k = 1
+    cases.append((rng.standard_normal(64).astype(np.float32), 64))            # k = n
+    cases.append((np.asarray([0.0, -0.0, 1e-40, -1e-40, 0.0], np.float32), 3))  # denormals, signed zeros
+    cases.append((rng.standard_normal(3000).astype(np.float32), 30))
+    for x, k in cases:
+        idx, val, dec = oracle.topk_compress(x, [0, len(x)], [k], _lib=L)
+        want = brute_topk(x, k)
+        assert idx.tolist() == want, (k, idx[:8], want[:8])
+        assert np.array_equal(val.view(np.uint32), x[want].view(np.uint32))
+        expect_dec = np.zeros_like(x)
+        expect_dec[want] = x[want]
+        assert np.array_equal(dec, expect_dec)
+        x64 = x.astype(np.float64)
+        assert np.sum((x64 - dec) ** 2) <= (1 - k / len(x)) * np.sum(x64 ** 2) + 1e-12
+    # segment-wise: flat indices, each segment independent
+    x = rng.integers(-5, 6, 150).astype(np.float32)
+    off, k = [0, 10, 11, 80, 150], [3, 1, 7, 70]
+    idx, val, dec = oracle.topk_compress(x, off, k, _lib=L)
+    want = []
+    for t in range(4):
+        want += [off[t] + j for j in brute_topk(x[off[t]:off[t + 1]], k[t])]
+    assert idx.tolist() == want and np.array_equal(val, x[want])
+
+
+def pin_topk_quantile(L):
+    """On Gaussians the 1 % magnitude threshold is the textbook two-sided quantile 2.576 sigma."""
+    n = 400_000
+    x = np.random.default_rng(17).standard_normal(n).astype(np.float32)
+    k = n // 100
+    idx, val, _ = oracle.topk_compress(x, [0, n], [k], _lib=L)
+    assert len(idx) == k and np.all(np.diff(idx.astype(np.int64)) > 0)
+    assert abs(np.min(np.abs(val)) - 2.5758) < 0.03
+    mask = np.ones(n, bool)
+    mask[idx] = False
+    assert np.max(np.abs(x[mask])) <= np.min(np.abs(val))
+
+
+# ----------------------------------------------------------------------------- whole step
+
+def _random_problem(rng, N, off, integer=False):
+    d = int(off[-1])
+    if integer:
+        G = rng.integers(-8, 9, (N, d)).astype(np.float32)
+    else:
+        G = rng.standard_normal((N, d)).astype(np.float32)
+    return G
+
+
+def pin_error_recursion(L):
+    """e_{t+1} = v_t - p_t: decoded message plus new error gives back v
+    (exactly for top-k and identity, within one rounding for scaled sign)."""
+    rng = np.random.default_rng(21)
+    off = np.asarray([0, 5, 37, 100, 164], np.int64)
+    d, N = 164, 3
+    k = np.asarray([2, 4, 9, 1], np.int64)
+    for up, down in ((SIGN, SIGN), (TOPK, TOPK), (IDENTITY, IDENTITY), (SIGN, TOPK), (TOPK, SIGN),
+                     (IDENTITY, SIGN), (SIGN, IDENTITY)):
+        X = rng.standard_normal((N, d)).astype(np.float32)
+        e = rng.standard_normal(d).astype(np.float32) * np.float32(0.1)
+        e0 = e.copy()
+        G = _random_problem(rng, N, off)
+        r = oracle.step(X, e, G, 0.1, off, up, down, k=k, _lib=L)
+        # v from its definition, evaluated independently in float32 numpy
+        if up == SIGN:
+            P = np.stack([decode_sign(r.up_words[i], r.up_scales[i], off) for i in range(N)])
+        elif up == TOPK:
+            P = np.stack([decode_topk(r.up_idx[i], r.up_val[i], d) for i in range(N)])
+        else:
+            P = G
+        acc = np.zeros(d, np.float32)
+        for i in range(N):
+            acc = acc + P[i]
+        v = e0 + acc / np.float32(N)
+        assert np.array_equal(v, r.v), (up, down)
+        if down == SIGN:
+            p = decode_sign(r.down_words, r.down_scales, off)
+            # e' = fl(v - p): off from the exact difference by at most half a unit in its own last place
+            assert np.all(np.abs((p.astype(np.float64) + e) - r.v) <= 0.5 * np.spacing(np.abs(e)).astype(np.float64))
+        elif down == TOPK:
+            p = decode_topk(r.down_idx, r.down_val, d)
+            assert np.array_equal(p + e, r.v)
+            assert np.all(e[r.down_idx.astype(np.int64)] == 0.0)
+        else:
+            assert np.all(e == 0.0)
+
+
+def pin_identity_one_worker_is_sgd(L):
+    """Algorithm 1 with C = identity and N = 1 is x <- x - eta g."""
+    rng = np.random.default_rng(23)
+    d = 257
+    X = rng.standard_normal((1, d)).astype(np.float32)
+    e = np.zeros(d, np.float32)
+    ref = X.copy()
+    for step in range(5):
+        G = rng.standard_normal((1, d)).astype(np.float32)
+        oracle.step(X, e, G, 0.05, [0, 100, d], IDENTITY, IDENTITY, _lib=L)
+        ref = ref - np.float32(0.05) * G
+        assert np.array_equal(X, ref) and np.all(e == 0.0)
+
+
+def pin_identical_workers(L):
+    """Equal gradients on N = 2^m workers with e = 0: v = p^i, C(v) = v, e' = 0, x <- x - eta g."""
+    rng = np.random.default_rng(29)
+    d, N = 128, 4
+    g = rng.integers(-8, 9, d).astype(np.float32)      # scales are exact binary fractions
+    G = np.tile(g, (N, 1))
+    X = np.tile(rng.standard_normal(d).astype(np.float32), (N, 1)).copy()
+    x0 = X[0].copy()
+    e = np.zeros(d, np.float32)
+    r = oracle.step(X, e, G, 0.5, [0, 64, 128], SIGN, SIGN, _lib=L)
+    assert np.array_equal(r.v, decode_sign(r.up_words[0], r.up_scales[0], [0, 64, 128]))
+    assert np.array_equal(r.down_words, r.up_words[0]) and np.array_equal(r.down_scales, r.up_scales[0])
+    assert np.all(e == 0.0)
+    for i in range(N):
+        assert np.array_equal(X[i], x0 - np.float32(0.5) * g)
+
+
+def pin_lemma3_exact(L):
+    """Lemma 3: mean_i x_t^i - (x_0 - eta sum_tau mean_i g_tau^i) = eta e_t.
+
+    Small integers, power-of-two sizes and eta = 1/2 keep every operation exact, so
+    the identity has to hold to the last bit over several iterations.
+    """
+    rng = np.random.default_rng(31)
+    for up, down, off, k, N in ((SIGN, SIGN, [0, 4, 8], None, 2),
+                                (TOPK, TOPK, [0, 16, 24], [3, 2], 4),
+                                (SIGN, TOPK, [0, 4, 8], [1, 2], 2),
+                                (IDENTITY, SIGN, [0, 4, 8], None, 2)):
+        off = np.asarray(off, np.int64)
+        d = int(off[-1])
+        x0 = rng.integers(-4, 5, d).astype(np.float32)
+        X = np.tile(x0, (N, 1)).copy()
+        e = np.zeros(d, np.float32)
+        gsum = np.zeros(d, np.float64)
+        for step in range(4):
+            G = _random_problem(rng, N, off, integer=True)
+            oracle.step(X, e, G, 0.5, off, up, down, k=k, _lib=L)
+            gsum += G.astype(np.float64).mean(axis=0)
+            xbar = X.astype(np.float64).mean(axis=0)
+            xhat = x0.astype(np.float64) - 0.5 * gsum
+            assert np.array_equal(xbar - xhat, 0.5 * e.astype(np.float64)), (up, down, step)
+        assert np.any(e != 0.0)
+
+
+def pin_lemma3_float(L):
+    """Lemma 3 on Gaussian data holds up to binary32 rounding accumulated over the steps."""
+    rng = np.random.default_rng(37)
+    off = np.asarray([0, 100, 130, 400], np.int64)
+    d, N, lr = 400, 5, 0.1
+    for up, down, k in ((SIGN, SIGN, None), (TOPK, TOPK, [5, 2, 20])):
+        X = np.zeros((N, d), np.float32)
+        e = np.zeros(d, np.float32)
+        gsum = np.zeros(d, np.float64)
+        for step in range(20):
+            G = _random_problem(rng, N, off)
+            oracle.step(X, e, G, lr, off, up, down, k=k, _lib=L)
+            gsum += G.astype(np.float64).mean(axis=0)
+        lhs = X.astype(np.float64).mean(axis=0) + lr * gsum
+        assert np.max(np.abs(lhs - lr * e.astype(np.float64))) < 2e-5
+        assert np.max(np.abs(e)) > 0.1
+
+
+def pin_bf16_widening(L):
+    bits = np.asarray([0x3F80, 0xBF80, 0x0000, 0x8000, 0x3DCD, 0x7F7F, 0x0001], np.uint16)
+    out = oracle.widen_bf16(bits)
+    assert out.view(np.uint32).tolist() == [int(b) << 16 for b in bits]
+    assert out[0] == 1.0 and out[1] == -1.0
+
+
+ALL_PINS = [
+    pin_golden_sign, pin_golden_blockwise, pin_golden_topk,
+    pin_scale_is_exact_mean, pin_tree_shape, pin_sign_bits_bruteforce, pin_sign_contraction,
+    pin_blockwise_reduces_to_sign, pin_topk_bruteforce, pin_topk_quantile,
+    pin_error_recursion, pin_identity_one_worker_is_sgd, pin_identical_workers,
+    pin_lemma3_exact, pin_lemma3_float, pin_bf16_widening,
+]

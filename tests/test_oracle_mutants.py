@@ -1,0 +1,69 @@
+"""Each plausible mistake, planted in a copy of the oracle on the CPU, must trip a pin.
+
+The copies are made by editing the oracle's C text, compiled to a temporary shared
+object and run through the same pins as the real oracle.  A mutant that survives
+means the pins would not have noticed that mistake in the real oracle either.
+"""
+import os
+
+import pytest
+
+import oracle
+import oracle_pins
+from oracle import liec_oracle as wrapper
+
+MUTANTS = {
+    "sign_of_zero_negative": ("int neg = xs[j] < 0.0f;", "int neg = xs[j] <= 0.0f;"),
+    "bit_order_reversed": ("(uint32_t)1 << (j % 32)", "(uint32_t)1 << (31 - j % 32)"),
+    "segment_word_offset_dropped": ("words[woff + j / 32] |=", "words[j / 32] |="),
+    "scale_not_divided": ("double mean = S / (double)n;", "double mean = S;"),
+    "scale_without_abs": ("if (a < 0.0f) a = -a;", ""),
+    "scale_summed_in_binary32": ("double left = tree_node", "float left = tree_node"),
+    "scale_running_sum": ("double left = tree_node(x, n, lo, len / 2);\n    double right = tree_node(x, n, lo + len / 2, len / 2);\n    return left + right;",
+                          "double s = 0.0; for (int64_t q = lo; q < lo + len && q < n; ++q) s += (double)(x[q] < 0 ? -x[q] : x[q]);\n    return s;"),
+    "decoded_sign_flipped": ("dec[off[t] + j] = neg ? -s : s;", "dec[off[t] + j] = neg ? s : -s;"),
+    "topk_smallest_first": ("return p->key > q->key ? -1 : 1;", "return p->key > q->key ? 1 : -1;"),
+    "topk_tie_higher_index": ("return p->pos < q->pos ? -1 : 1;", "return p->pos < q->pos ? 1 : -1;"),
+    "topk_signed_key": ("& 0x7fffffffu", "& 0xffffffffu"),
+    "topk_segment_relative_index": ("idx[out] = (uint32_t)(off[t] + j);", "idx[out] = (uint32_t)j;"),
+    "mean_not_divided": ("float mean = acc / (float)N;", "float mean = acc;"),
+    "global_error_not_added": ("v[j] = e[j] + mean;", "v[j] = mean;"),
+    "global_error_subtracted": ("v[j] = e[j] + mean;", "v[j] = e[j] - mean;"),
+    "workers_summed_backwards": ("acc = acc + P[(size_t)i * d + j];", "acc = acc + P[(size_t)(N - 1 - i) * d + j];"),
+    "downlink_compresses_error": ("rc = compress(down, v, d, T, off, k,", "rc = compress(down, e, d, T, off, k,"),
+    "error_update_sign": ("e[j] = v[j] - p[j];", "e[j] = p[j] - v[j];"),
+    "compensation_sign": ("float diff = p[j] - pi[j];", "float diff = pi[j] - p[j];"),
+    "compensation_dropped": ("const float *pi = P + (size_t)i * d;", "const float *pi = g;"),
+    "gradient_subtracted": ("float u = diff + g[j];", "float u = diff - g[j];"),
+    "learning_rate_dropped": ("float step = lr * u;", "float step = u;"),
+    "ascent_instead_of_descent": ("x[j] = x[j] - step;", "x[j] = x[j] + step;"),
+}
+
+
+def _failures(L):
+    failed = []
+    for pin in oracle_pins.ALL_PINS:
+        try:
+            pin(L)
+        except AssertionError:
+            failed.append(pin.__name__)
+    return failed
+
+
+@pytest.mark.parametrize("name", sorted(MUTANTS))
+def test_mutant_is_caught(name, tmp_path):
+    old, new = MUTANTS[name]
+    with open(wrapper._SRC) as fh:
+        text = fh.read()
+    assert text.count(old) == 1, f"mutation site for {name} not found exactly once"
+    src = tmp_path / "mutant.c"
+    src.write_text(text.replace(old, new))
+    out = str(tmp_path / "libmutant.so")
+    import subprocess
+    subprocess.run(["gcc", *wrapper.CFLAGS, "-w", str(src), "-o", out], check=True)
+    failed = _failures(oracle.lib(out))
+    assert failed, f"mutant {name} passed every pin"
+
+
+def test_real_oracle_passes_every_pin():
+    assert _failures(oracle.lib()) == []
