@@ -1,0 +1,163 @@
+/*
+ * liec.h - C ABI of the LIEC-SGD compression-step library for NVIDIA B200 (sm_100a).
+ *
+ * The library runs, on one GPU, the per-iteration bidirectional compression step of
+ * LIEC-SGD (Algorithm 1, the branch with compression, i.e. every iteration that is not
+ * a model-averaging iteration).  N workers minimise f(x) = 1/N sum_i E f_i(x, xi_i),
+ * x in R^d (Eq. 1); they are simulated as the N rows of device tensors:
+ *
+ *   uplink    p^i = C(g^i)                          worker compress step of Algorithm 1
+ *   server    v   = e + (1/N) sum_i p^i             server compensate step
+ *   downlink  p   = C(v),  e <- v - p               server compress step, global error update
+ *   update    x^i <- x^i - eta (p - p^i + g^i)      local immediate error compensation
+ *
+ * C is applied per segment (a contiguous block of the flattened model, e.g. one
+ * parameter tensor) and is one of: scaled sign  C(x)_j = (||x||_1/n) sign(x_j)
+ * (Def. 4; with several segments Def. 5, Blockwise-SignSGD), top-k (Def. 2), identity.
+ *
+ * Arithmetic contract (the paper does not fix one; results are reproducible bit for bit):
+ *   - state and messages are IEEE binary32, every written operation rounded once to
+ *     nearest-even, no fused multiply-add; gradients may be binary32 or bfloat16
+ *     (bfloat16 is widened exactly before use);
+ *   - sign(x) is negative iff x < 0 (zeros decode to +scale);
+ *   - ||x||_1 of a segment is accumulated in binary64 over a balanced binary tree on
+ *     the segment zero-padded to a power of two, divided by n in binary64 and rounded
+ *     once to binary32;
+ *   - top-k orders by |x| (binary32 magnitude), ties go to the lower index;
+ *   - the server adds the N decoded messages in worker order starting from +0,
+ *     divides by (float)N and then adds e;
+ *   - the update is evaluated as x - eta*((p - p^i) + g).
+ *
+ * Message ("wire") layouts, all in the caller's workspace:
+ *   sign   : words[W] + scales[T].  Segment t owns ceil(n_t/32) consecutive 32-bit
+ *            words starting at sum_{u<t} ceil(n_u/32); bit b (LSB = 0) of its word w is
+ *            1 iff element seg_offsets[t]+32w+b is negative; padding bits are 0.
+ *   top-k  : idx[K] (uint32 flat index into [0,d)) + val[K] (binary32 copy of the kept
+ *            entry), K = sum_t k_t; segment t owns [sum_{u<t} k_u, +k_t), ascending index.
+ *   identity: no message buffer; the dense vector itself.
+ *
+ * Ownership: the caller owns every device buffer (params, error, gradients, workspace).
+ * The library owns only the host-side context.  The hot calls allocate nothing, never
+ * synchronise the device and only enqueue work on the given stream.
+ *
+ * Errors: every call returns a liec_status; nothing throws, aborts or traps the GPU.
+ * liec_last_error() gives a message for the last failing call on that context.
+ */
+#ifndef LIEC_H
+#define LIEC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct liec_ctx liec_ctx; /* opaque, lives in host memory */
+
+typedef enum {
+    LIEC_OK = 0,
+    LIEC_ERR_INVALID_ARG = 1,  /* NULL / misaligned pointer, bad sizes, bad segment table, bad k */
+    LIEC_ERR_UNSUPPORTED = 2,  /* d >= 2^32, too many workers or segments for the launch grid */
+    LIEC_ERR_WORKSPACE = 3,    /* workspace smaller than liec_workspace_bytes() */
+    LIEC_ERR_STATE = 4,        /* staged calls made out of order */
+    LIEC_ERR_CUDA = 5,         /* a CUDA runtime call failed; see liec_last_error() */
+    LIEC_ERR_DEVICE_CHECK = 6  /* a kernel recorded an internal inconsistency in the status word */
+} liec_status;
+
+typedef enum { LIEC_COMP_IDENTITY = 0, LIEC_COMP_SCALED_SIGN = 1, LIEC_COMP_TOPK = 2 } liec_comp;
+typedef enum { LIEC_F32 = 0, LIEC_BF16 = 1 } liec_dtype;
+
+typedef struct {
+    int32_t num_workers;        /* N >= 1 (Eq. 1) */
+    int64_t dim;                /* d, 1 <= d < 2^32; N*d may exceed 2^32 */
+    int32_t num_segments;       /* T >= 1.  T = 1: whole-vector operator (Def. 4); T > 1: blockwise (Def. 5) */
+    const int64_t *seg_offsets; /* host, T+1 entries, [0] = 0, [T] = d, strictly increasing; copied */
+    int32_t uplink;             /* liec_comp used by the workers  (C in the worker compress step) */
+    int32_t downlink;           /* liec_comp used by the server   (C in the server compress step) */
+    const int64_t *topk_k;      /* host, T entries, 1 <= k_t <= n_t; needed iff a side is TOPK; copied */
+    int32_t grad_dtype;         /* liec_dtype of the gradient rows; params, error, messages are binary32 */
+} liec_config;
+
+/* Device pointers into the workspace (NULL for parts the configuration does not use). */
+typedef struct {
+    const uint32_t *up_words;    /* [N][W]   sign uplink */
+    const float *up_scales;      /* [N][T] */
+    const uint32_t *up_idx;      /* [N][K]   top-k uplink */
+    const float *up_val;         /* [N][K] */
+    const uint32_t *down_words;  /* [W]      sign downlink */
+    const float *down_scales;    /* [T] */
+    const uint32_t *down_idx;    /* [K]      top-k downlink */
+    const float *down_val;       /* [K] */
+    const float *v;              /* [d] v_t; valid between liec_server_aggregate and
+                                    liec_downlink_compress (it aliases the error buffer) */
+    int64_t num_words;           /* W */
+    int64_t num_topk;            /* K (0 when no side is top-k) */
+} liec_messages;
+
+/*
+ * Bytes of device workspace needed for this configuration (message buffers, per-tile
+ * partial sums, selection scratch).  Pure host arithmetic; returns 0 for an invalid
+ * configuration.
+ */
+size_t liec_workspace_bytes(const liec_config *cfg);
+
+/* Bytes of the downlink message as copied out by liec_step_host (0 for identity/invalid). */
+size_t liec_down_message_bytes(const liec_config *cfg);
+
+/*
+ * Creates a context (Algorithm 1, initialisation line: x_0^i = x_0, e_0 = 0 are the
+ * caller's job - the buffers are used as they are, which is also how a run is resumed).
+ *   params    device, [N][d] binary32, row stride d, 16-byte aligned: the local models x^i.
+ *   error     device, [d] binary32, 16-byte aligned: the server's global error e.
+ *   workspace device, 256-byte aligned, at least liec_workspace_bytes(cfg) bytes.
+ * Copies the segment tables to the workspace with synchronous copies on the current
+ * device; the workspace must not be touched by the caller until liec_destroy.
+ */
+liec_status liec_init(const liec_config *cfg, float *params, float *error,
+                      void *workspace, size_t workspace_bytes, liec_ctx **out);
+
+/*
+ * The four stages of one iteration.  They must be called in this order (LIEC_ERR_STATE
+ * otherwise), all on streams that order them one after another.  `stream` is a
+ * cudaStream_t passed as void* (NULL = legacy default stream).
+ *   grads  device, [N][d] of cfg.grad_dtype, row stride d, 16-byte aligned; read-only; the
+ *          same pointer and contents must be given to liec_worker_update of the same step.
+ */
+liec_status liec_uplink_compress(liec_ctx *ctx, const void *grads, void *stream);   /* p^i = C(g^i) */
+liec_status liec_server_aggregate(liec_ctx *ctx, void *stream);                      /* v = e + mean_i p^i (into error) */
+liec_status liec_downlink_compress(liec_ctx *ctx, void *stream);                     /* p = C(v); error <- v - p */
+liec_status liec_worker_update(liec_ctx *ctx, const void *grads, float lr, void *stream); /* x^i -= lr (p - p^i + g^i) */
+
+/* The four stages in sequence; produces the same bytes as calling them one by one. */
+liec_status liec_step(liec_ctx *ctx, const void *grads, float lr, void *stream);
+
+/*
+ * One iteration fed from host memory: copies grads_host ([N][d] of cfg.grad_dtype, pinned
+ * memory recommended) into grads_dev (device staging buffer of the same size, caller
+ * owned), runs liec_step, copies the downlink message (sign: words then scales; top-k:
+ * idx then val; liec_down_message_bytes() bytes) to down_msg_host, all on `stream`.
+ * down_msg_host may be NULL to skip the read-back.  Does not synchronise.
+ */
+liec_status liec_step_host(liec_ctx *ctx, const void *grads_host, void *grads_dev, float lr,
+                           void *down_msg_host, void *stream);
+
+/* Device pointers of the current messages (valid until the next stage overwrites them). */
+liec_status liec_get_messages(const liec_ctx *ctx, liec_messages *out);
+
+/*
+ * Synchronises `stream` and reads the device status word: 0 = clean; non-zero bits name an
+ * internal check that failed.  Returns LIEC_ERR_DEVICE_CHECK when non-zero.
+ */
+liec_status liec_device_status(liec_ctx *ctx, void *stream, int32_t *out);
+
+/* Number of kernel launches enqueued by this context so far (host-side counter). */
+int64_t liec_launch_count(const liec_ctx *ctx);
+
+const char *liec_last_error(const liec_ctx *ctx); /* never NULL; ctx may be NULL */
+void liec_destroy(liec_ctx *ctx);                  /* frees host memory only */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LIEC_H */
