@@ -1,0 +1,147 @@
+// Device helpers shared by the tile kernels: tile lookup, 4-wide loads, the balanced
+// binary64 tree over a warp's 1024 elements, sign-word packing.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "plan.h"
+
+namespace liec {
+
+struct TileInfo {
+    int t;            // segment
+    int64_t seg_beg;  // first element of the segment within a row
+    int64_t n;        // segment length
+    int64_t rel;      // first element of the tile, relative to the segment
+    int len;          // valid elements in the tile (1..TILE)
+    int tile_in_seg;  // tile index inside the segment
+};
+
+// Segment owning tile `tile`: largest t with tile_prefix[t] <= tile.
+__device__ __forceinline__ TileInfo locate_tile(const Params &p, int tile) {
+    int lo = 0, hi = p.T;  // invariant: prefix[lo] <= tile < prefix[hi]
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (__ldg(p.tile_prefix + mid) <= tile) lo = mid; else hi = mid;
+    }
+    TileInfo ti;
+    ti.t = lo;
+    ti.seg_beg = __ldg(p.seg_off + lo);
+    ti.n = __ldg(p.seg_off + lo + 1) - ti.seg_beg;
+    ti.tile_in_seg = tile - __ldg(p.tile_prefix + lo);
+    ti.rel = (int64_t)ti.tile_in_seg * TILE;
+    int64_t left = ti.n - ti.rel;
+    ti.len = left < TILE ? (int)left : TILE;
+    return ti;
+}
+
+// ---- 4 consecutive gradient elements, widened to binary32 --------------------------------
+
+__device__ __forceinline__ void load4_stream(const float *ptr, float (&v)[4]) {
+    float4 q = __ldcs(reinterpret_cast<const float4 *>(ptr));
+    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+}
+__device__ __forceinline__ void load4_stream(const __nv_bfloat16 *ptr, float (&v)[4]) {
+    uint2 q = __ldcs(reinterpret_cast<const uint2 *>(ptr));
+    v[0] = __uint_as_float(q.x << 16);
+    v[1] = __uint_as_float(q.x & 0xffff0000u);
+    v[2] = __uint_as_float(q.y << 16);
+    v[3] = __uint_as_float(q.y & 0xffff0000u);
+}
+__device__ __forceinline__ float load1(const float *ptr) { return *ptr; }
+__device__ __forceinline__ float load1(const __nv_bfloat16 *ptr) {
+    return __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short *>(ptr)) << 16);
+}
+// Guarded scalar version: elements at or beyond `len` read as +0.
+template <typename GT>
+__device__ __forceinline__ void load4_guarded(const GT *tile_ptr, int pos, int len, float (&v)[4]) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) v[c] = (pos + c < len) ? load1(tile_ptr + pos + c) : 0.0f;
+}
+
+// Position (relative to the tile) of the 4 elements a thread owns in row j of its warp.
+__device__ __forceinline__ int tile_pos(int warp, int lane, int j) { return warp * 1024 + j * 128 + lane * 4; }
+
+// ---- balanced binary64 tree -----------------------------------------------------------------
+//
+// A warp owns 1024 consecutive elements as 8 rows of 128; lane l of row j owns elements
+// 4l..4l+3 of that row.  leaf4 sums a lane's 4 magnitudes (two tree levels).  The warp
+// reduction then follows the tree upwards: lanes xor 1,2,4,8,16 inside each row, then rows
+// pairwise.  Rows are folded across lanes while reducing ("transposed" butterfly) so that
+// each level costs one shuffle+add per surviving value instead of one per row.
+
+__device__ __forceinline__ double leaf4(const float (&v)[4]) {
+    double a0 = (double)fabsf(v[0]), a1 = (double)fabsf(v[1]);
+    double a2 = (double)fabsf(v[2]), a3 = (double)fabsf(v[3]);
+    return __dadd_rn(__dadd_rn(a0, a1), __dadd_rn(a2, a3));
+}
+
+__device__ __forceinline__ double shfl_xor_f64(double x, int mask) {
+    return __shfl_xor_sync(0xffffffffu, x, mask);
+}
+
+// a[j] = this lane's leaf sum in row j.  Returns, in every lane, the tree sum of the warp's
+// 1024 elements.
+__device__ __forceinline__ double warp_tree_reduce8(double (&a)[8], int lane) {
+    // lane levels 1,2,4 while folding 8 rows -> 1 value per lane
+#pragma unroll
+    for (int step = 0; step < 3; ++step) {
+        const int m = 1 << step;
+        const int half = 4 >> step;
+        const bool upper = (lane & m) != 0;
+#pragma unroll
+        for (int r = 0; r < half; ++r) {
+            double send = upper ? a[r] : a[r + half];
+            double keep = upper ? a[r + half] : a[r];
+            double recv = shfl_xor_f64(send, m);
+            a[r] = __dadd_rn(keep, recv);
+        }
+    }
+    double s = a[0];
+    // remaining lane levels of the row this lane now represents
+    s = __dadd_rn(s, shfl_xor_f64(s, 8));
+    s = __dadd_rn(s, shfl_xor_f64(s, 16));
+    // row levels: row bit 0 lives in lane bit 2, row bit 1 in lane bit 1, row bit 2 in lane bit 0
+    s = __dadd_rn(s, shfl_xor_f64(s, 4));
+    s = __dadd_rn(s, shfl_xor_f64(s, 2));
+    s = __dadd_rn(s, shfl_xor_f64(s, 1));
+    return s;
+}
+
+// Combine the 8 warp sums of a CTA (tile of 8192 elements) in tree order; result in thread 0.
+__device__ __forceinline__ double cta_tree_reduce(double warp_sum, double *smem8) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) smem8[warp] = warp_sum;
+    __syncthreads();
+    double s = 0.0;
+    if (threadIdx.x == 0) {
+        double s01 = __dadd_rn(smem8[0], smem8[1]), s23 = __dadd_rn(smem8[2], smem8[3]);
+        double s45 = __dadd_rn(smem8[4], smem8[5]), s67 = __dadd_rn(smem8[6], smem8[7]);
+        s = __dadd_rn(__dadd_rn(s01, s23), __dadd_rn(s45, s67));
+    }
+    return s;
+}
+
+// ---- sign words -------------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t sign_nibble(const float (&v)[4]) {
+    return (v[0] < 0.0f ? 1u : 0u) | (v[1] < 0.0f ? 2u : 0u) | (v[2] < 0.0f ? 4u : 0u) | (v[3] < 0.0f ? 8u : 0u);
+}
+
+// The 8 lanes that share a 32-element word OR their nibbles together; every lane of the
+// group gets the word.
+__device__ __forceinline__ uint32_t pack_word(uint32_t nibble, int lane) {
+    uint32_t w = nibble << (4 * (lane & 7));
+    w |= __shfl_xor_sync(0xffffffffu, w, 1);
+    w |= __shfl_xor_sync(0xffffffffu, w, 2);
+    w |= __shfl_xor_sync(0xffffffffu, w, 4);
+    return w;
+}
+
+// Nibble of this lane's 4 elements in row j, taken from the warp's 32 words (lane l holds word l).
+__device__ __forceinline__ uint32_t nibble_from_words(uint32_t my_word, int lane, int j) {
+    uint32_t w = __shfl_sync(0xffffffffu, my_word, 4 * j + (lane >> 3));
+    return (w >> (4 * (lane & 7))) & 0xfu;
+}
+
+}  // namespace liec

@@ -1,0 +1,20 @@
+// Launchers of the CUDA kernels (one translation unit per kernel family).
+#pragma once
+#include <cuda_runtime.h>
+
+#include "plan.h"
+
+namespace liec {
+
+// scaled sign
+cudaError_t launch_sign_uplink(const Params &p, cudaStream_t st);
+cudaError_t launch_scale_finalize(const Params &p, bool uplink, cudaStream_t st);
+cudaError_t launch_server_dense(const Params &p, cudaStream_t st);
+cudaError_t launch_sign_downlink(const Params &p, cudaStream_t st);
+cudaError_t launch_sign_error(const Params &p, cudaStream_t st);
+cudaError_t launch_identity_downlink(const Params &p, cudaStream_t st);
+
+// worker update
+cudaError_t launch_worker_update(const Params &p, float lr, cudaStream_t st);
+
+}  // namespace liec

@@ -1,0 +1,436 @@
+// C ABI of the library: configuration checks, workspace plan, stage sequencing.
+// Every numeric step runs in the kernels launched from here.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/liec.h"
+#include "kernels.h"
+#include "plan.h"
+
+using namespace liec;
+
+namespace {
+
+thread_local char g_no_ctx_error[256] = "";
+
+struct Region {
+    size_t off = 0, bytes = 0;
+};
+
+struct Plan {
+    int32_t N = 0, T = 0, TT = 0;
+    int64_t d = 0, W = 0, K = 0, CAP = 0;
+    std::vector<int64_t> seg_off, word_off, k_off, cap_off, topk_k;
+    std::vector<int32_t> tile_prefix;
+    Region r_seg_off, r_word_off, r_k_off, r_cap_off, r_tile_prefix, r_status;
+    Region r_up_words, r_up_scales, r_up_partials, r_down_words, r_down_scales, r_down_partials, r_vbuf;
+    Region r_up_idx, r_up_val, r_down_idx, r_down_val;
+    Region r_up_hist, r_down_hist, r_up_hist2, r_down_hist2, r_up_sel, r_down_sel;
+    Region r_up_cand_idx, r_up_cand_val, r_down_cand_idx, r_down_cand_val;
+    Region r_up_tile_meta, r_down_tile_meta, r_up_outbase, r_down_outbase;
+    size_t total = 0;
+};
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Carver {
+    size_t cursor = 0;
+    Region take(size_t bytes, size_t align = 256) {
+        Region r;
+        cursor = align_up(cursor, align);
+        r.off = cursor;
+        r.bytes = bytes;
+        cursor += bytes;
+        return r;
+    }
+};
+
+liec_status fail(std::string *msg, liec_status st, const char *text) {
+    if (msg) *msg = text;
+    return st;
+}
+
+liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
+    if (!cfg) return fail(msg, LIEC_ERR_INVALID_ARG, "config is NULL");
+    if (cfg->num_workers < 1) return fail(msg, LIEC_ERR_INVALID_ARG, "num_workers must be >= 1");
+    if (cfg->num_workers > 65535) return fail(msg, LIEC_ERR_UNSUPPORTED, "num_workers above 65535 (grid y limit)");
+    if (cfg->dim < 1) return fail(msg, LIEC_ERR_INVALID_ARG, "dim must be >= 1");
+    if (cfg->dim >= (int64_t(1) << 32)) return fail(msg, LIEC_ERR_UNSUPPORTED, "dim must be below 2^32 (32-bit indices)");
+    if (cfg->num_segments < 1) return fail(msg, LIEC_ERR_INVALID_ARG, "num_segments must be >= 1");
+    if (cfg->num_segments > 65535) return fail(msg, LIEC_ERR_UNSUPPORTED, "num_segments above 65535 (grid limit)");
+    if (!cfg->seg_offsets) return fail(msg, LIEC_ERR_INVALID_ARG, "seg_offsets is NULL");
+    auto comp_ok = [](int32_t c) { return c == LIEC_COMP_IDENTITY || c == LIEC_COMP_SCALED_SIGN || c == LIEC_COMP_TOPK; };
+    if (!comp_ok(cfg->uplink) || !comp_ok(cfg->downlink)) return fail(msg, LIEC_ERR_INVALID_ARG, "unknown compressor");
+    if (cfg->grad_dtype != LIEC_F32 && cfg->grad_dtype != LIEC_BF16) return fail(msg, LIEC_ERR_INVALID_ARG, "unknown grad_dtype");
+    const int T = cfg->num_segments;
+    if (cfg->seg_offsets[0] != 0 || cfg->seg_offsets[T] != cfg->dim)
+        return fail(msg, LIEC_ERR_INVALID_ARG, "seg_offsets must start at 0 and end at dim");
+    for (int t = 0; t < T; ++t)
+        if (cfg->seg_offsets[t + 1] <= cfg->seg_offsets[t])
+            return fail(msg, LIEC_ERR_INVALID_ARG, "seg_offsets must be strictly increasing");
+    const bool any_topk = cfg->uplink == LIEC_COMP_TOPK || cfg->downlink == LIEC_COMP_TOPK;
+    if (any_topk) {
+        if (!cfg->topk_k) return fail(msg, LIEC_ERR_INVALID_ARG, "topk_k is NULL but a side uses top-k");
+        for (int t = 0; t < T; ++t) {
+            int64_t n = cfg->seg_offsets[t + 1] - cfg->seg_offsets[t];
+            if (cfg->topk_k[t] < 1 || cfg->topk_k[t] > n)
+                return fail(msg, LIEC_ERR_INVALID_ARG, "topk_k[t] must satisfy 1 <= k_t <= n_t");
+        }
+    }
+
+    pl.N = cfg->num_workers;
+    pl.T = T;
+    pl.d = cfg->dim;
+    pl.seg_off.assign(cfg->seg_offsets, cfg->seg_offsets + T + 1);
+    pl.word_off.assign(T + 1, 0);
+    pl.k_off.assign(T + 1, 0);
+    pl.cap_off.assign(T + 1, 0);
+    pl.tile_prefix.assign(T + 1, 0);
+    pl.topk_k.assign(T, 0);
+    int64_t tiles = 0;
+    for (int t = 0; t < T; ++t) {
+        int64_t n = pl.seg_off[t + 1] - pl.seg_off[t];
+        pl.word_off[t + 1] = pl.word_off[t] + (n + 31) / 32;
+        tiles += (n + TILE - 1) / TILE;
+        if (tiles > 0x7fffffff) return fail(msg, LIEC_ERR_UNSUPPORTED, "too many tiles");
+        pl.tile_prefix[t + 1] = (int32_t)tiles;
+        if (any_topk) {
+            int64_t k = cfg->topk_k[t];
+            pl.topk_k[t] = k;
+            pl.k_off[t + 1] = pl.k_off[t] + k;
+            int64_t cap = 2 * k + 2048;  // room for the entries sharing the threshold's first digit
+            if (cap > n) cap = n;
+            pl.cap_off[t + 1] = pl.cap_off[t] + cap;
+        }
+    }
+    pl.W = pl.word_off[T];
+    pl.K = pl.k_off[T];
+    pl.CAP = pl.cap_off[T];
+    pl.TT = (int32_t)tiles;
+
+    Carver c;
+    pl.r_seg_off = c.take(sizeof(int64_t) * (T + 1));
+    pl.r_word_off = c.take(sizeof(int64_t) * (T + 1));
+    pl.r_k_off = c.take(sizeof(int64_t) * (T + 1));
+    pl.r_cap_off = c.take(sizeof(int64_t) * (T + 1));
+    pl.r_tile_prefix = c.take(sizeof(int32_t) * (T + 1));
+    pl.r_status = c.take(256);
+    const size_t N = pl.N;
+    if (cfg->uplink == LIEC_COMP_SCALED_SIGN) {
+        pl.r_up_words = c.take(sizeof(uint32_t) * N * pl.W);
+        pl.r_up_scales = c.take(sizeof(float) * N * T);
+        pl.r_up_partials = c.take(sizeof(double) * N * pl.TT);
+    }
+    if (cfg->downlink == LIEC_COMP_SCALED_SIGN) {
+        // words and scales are adjacent: together they are the downlink message
+        pl.r_down_words = c.take(sizeof(uint32_t) * pl.W + sizeof(float) * T);
+        pl.r_down_words.bytes = sizeof(uint32_t) * pl.W;
+        pl.r_down_scales.off = pl.r_down_words.off + pl.r_down_words.bytes;
+        pl.r_down_scales.bytes = sizeof(float) * T;
+        pl.r_down_partials = c.take(sizeof(double) * pl.TT);
+    }
+    if (cfg->downlink == LIEC_COMP_IDENTITY) pl.r_vbuf = c.take(sizeof(float) * pl.d);
+    auto topk_regions = [&](size_t rows, Region &idx, Region &val, Region &hist, Region &hist2, Region &sel,
+                            Region &cidx, Region &cval, Region &meta, Region &outbase) {
+        idx = c.take(sizeof(uint32_t) * rows * pl.K * 2);  // idx then val, adjacent
+        idx.bytes = sizeof(uint32_t) * rows * pl.K;
+        val.off = idx.off + idx.bytes;
+        val.bytes = sizeof(float) * rows * pl.K;
+        hist = c.take(sizeof(uint32_t) * rows * T * DIGIT1_BINS);
+        hist2 = c.take(sizeof(uint32_t) * rows * T * DIGIT1_BINS);
+        sel = c.take(sizeof(uint32_t) * rows * T * SEL_WORDS);
+        cidx = c.take(sizeof(uint32_t) * rows * pl.CAP);
+        cval = c.take(sizeof(float) * rows * pl.CAP);
+        meta = c.take(sizeof(uint32_t) * rows * pl.TT * 4);
+        outbase = c.take(sizeof(uint32_t) * rows * (pl.TT + 1));
+    };
+    if (cfg->uplink == LIEC_COMP_TOPK)
+        topk_regions(N, pl.r_up_idx, pl.r_up_val, pl.r_up_hist, pl.r_up_hist2, pl.r_up_sel, pl.r_up_cand_idx,
+                     pl.r_up_cand_val, pl.r_up_tile_meta, pl.r_up_outbase);
+    if (cfg->downlink == LIEC_COMP_TOPK)
+        topk_regions(1, pl.r_down_idx, pl.r_down_val, pl.r_down_hist, pl.r_down_hist2, pl.r_down_sel,
+                     pl.r_down_cand_idx, pl.r_down_cand_val, pl.r_down_tile_meta, pl.r_down_outbase);
+    pl.total = align_up(c.cursor, 256);
+    return LIEC_OK;
+}
+
+}  // namespace
+
+struct liec_ctx {
+    Plan plan;
+    Params p;
+    liec_config cfg;
+    char *ws = nullptr;
+    int stage = 0;  // 0 idle, 1 after uplink, 2 after aggregate, 3 after downlink
+    int64_t launches = 0;
+    std::string err;
+};
+
+namespace {
+
+template <typename Tp>
+Tp *at(liec_ctx *c, const Region &r) {
+    return r.bytes ? reinterpret_cast<Tp *>(c->ws + r.off) : nullptr;
+}
+
+liec_status cuda_fail(liec_ctx *c, cudaError_t e, const char *what) {
+    c->err = std::string(what) + ": " + cudaGetErrorString(e);
+    return LIEC_ERR_CUDA;
+}
+
+#define LIEC_LAUNCH(ctx, call)                                        \
+    do {                                                              \
+        cudaError_t e__ = (call);                                     \
+        if (e__ != cudaSuccess) return cuda_fail(ctx, e__, #call);    \
+        ++(ctx)->launches;                                            \
+    } while (0)
+
+bool aligned16(const void *ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+size_t liec_workspace_bytes(const liec_config *cfg) {
+    Plan pl;
+    if (make_plan(cfg, pl, nullptr) != LIEC_OK) return 0;
+    return pl.total;
+}
+
+size_t liec_down_message_bytes(const liec_config *cfg) {
+    Plan pl;
+    if (make_plan(cfg, pl, nullptr) != LIEC_OK) return 0;
+    if (cfg->downlink == LIEC_COMP_SCALED_SIGN) return sizeof(uint32_t) * pl.W + sizeof(float) * pl.T;
+    if (cfg->downlink == LIEC_COMP_TOPK) return (sizeof(uint32_t) + sizeof(float)) * pl.K;
+    return 0;
+}
+
+liec_status liec_init(const liec_config *cfg, float *params, float *error, void *workspace,
+                      size_t workspace_bytes, liec_ctx **out) {
+    std::string msg;
+    auto bail = [&](liec_status st, const char *text) {
+        snprintf(g_no_ctx_error, sizeof(g_no_ctx_error), "%s", text);
+        return st;
+    };
+    if (!out) return bail(LIEC_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    liec_ctx *c = new (std::nothrow) liec_ctx();
+    if (!c) return bail(LIEC_ERR_INVALID_ARG, "out of host memory");
+    liec_status st = make_plan(cfg, c->plan, &msg);
+    if (st != LIEC_OK) { delete c; return bail(st, msg.c_str()); }
+    if (!params || !error || !workspace) { delete c; return bail(LIEC_ERR_INVALID_ARG, "params, error and workspace must be non-NULL"); }
+    if (!aligned16(params) || !aligned16(error)) { delete c; return bail(LIEC_ERR_INVALID_ARG, "params and error must be 16-byte aligned"); }
+    if (reinterpret_cast<uintptr_t>(workspace) & 255u) { delete c; return bail(LIEC_ERR_INVALID_ARG, "workspace must be 256-byte aligned"); }
+    if (workspace_bytes < c->plan.total) { delete c; return bail(LIEC_ERR_WORKSPACE, "workspace smaller than liec_workspace_bytes()"); }
+
+    const Plan &pl = c->plan;
+    c->cfg = *cfg;
+    c->cfg.seg_offsets = nullptr;
+    c->cfg.topk_k = nullptr;
+    c->ws = static_cast<char *>(workspace);
+    Params &p = c->p;
+    memset(&p, 0, sizeof(p));
+    p.N = pl.N; p.T = pl.T; p.TT = pl.TT; p.d = pl.d; p.W = pl.W; p.K = pl.K; p.CAP = pl.CAP;
+    p.up = cfg->uplink; p.down = cfg->downlink; p.gdt = cfg->grad_dtype;
+    p.seg_off = at<int64_t>(c, pl.r_seg_off);
+    p.word_off = at<int64_t>(c, pl.r_word_off);
+    p.k_off = at<int64_t>(c, pl.r_k_off);
+    p.cap_off = at<int64_t>(c, pl.r_cap_off);
+    p.tile_prefix = at<int32_t>(c, pl.r_tile_prefix);
+    p.status = at<int32_t>(c, pl.r_status);
+    p.X = params;
+    p.e = error;
+    p.up_words = at<uint32_t>(c, pl.r_up_words);
+    p.up_scales = at<float>(c, pl.r_up_scales);
+    p.up_partials = at<double>(c, pl.r_up_partials);
+    p.down_words = at<uint32_t>(c, pl.r_down_words);
+    p.down_scales = at<float>(c, pl.r_down_scales);
+    p.down_partials = at<double>(c, pl.r_down_partials);
+    p.vbuf = at<float>(c, pl.r_vbuf);
+    p.up_idx = at<uint32_t>(c, pl.r_up_idx);       p.up_val = at<float>(c, pl.r_up_val);
+    p.down_idx = at<uint32_t>(c, pl.r_down_idx);   p.down_val = at<float>(c, pl.r_down_val);
+    p.up_hist = at<uint32_t>(c, pl.r_up_hist);     p.down_hist = at<uint32_t>(c, pl.r_down_hist);
+    p.up_hist2 = at<uint32_t>(c, pl.r_up_hist2);   p.down_hist2 = at<uint32_t>(c, pl.r_down_hist2);
+    p.up_sel = at<uint32_t>(c, pl.r_up_sel);       p.down_sel = at<uint32_t>(c, pl.r_down_sel);
+    p.up_cand_idx = at<uint32_t>(c, pl.r_up_cand_idx);   p.down_cand_idx = at<uint32_t>(c, pl.r_down_cand_idx);
+    p.up_cand_val = at<float>(c, pl.r_up_cand_val);      p.down_cand_val = at<float>(c, pl.r_down_cand_val);
+    p.up_tile_meta = at<uint32_t>(c, pl.r_up_tile_meta); p.down_tile_meta = at<uint32_t>(c, pl.r_down_tile_meta);
+    p.up_outbase = at<uint32_t>(c, pl.r_up_outbase);     p.down_outbase = at<uint32_t>(c, pl.r_down_outbase);
+
+    struct Up { const Region *r; const void *src; };
+    const Up ups[] = {
+        {&pl.r_seg_off, pl.seg_off.data()}, {&pl.r_word_off, pl.word_off.data()}, {&pl.r_k_off, pl.k_off.data()},
+        {&pl.r_cap_off, pl.cap_off.data()}, {&pl.r_tile_prefix, pl.tile_prefix.data()},
+    };
+    for (const Up &u : ups) {
+        cudaError_t e = cudaMemcpy(c->ws + u.r->off, u.src, u.r->bytes, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            snprintf(g_no_ctx_error, sizeof(g_no_ctx_error), "cudaMemcpy of tables failed: %s", cudaGetErrorString(e));
+            delete c;
+            return LIEC_ERR_CUDA;
+        }
+    }
+    // status word and every selection scratch region start at zero
+    auto zero = [&](const Region &r) { return r.bytes ? cudaMemset(c->ws + r.off, 0, r.bytes) : cudaSuccess; };
+    const Region *zs[] = {&pl.r_status, &pl.r_up_hist, &pl.r_down_hist, &pl.r_up_hist2, &pl.r_down_hist2,
+                          &pl.r_up_sel, &pl.r_down_sel, &pl.r_up_tile_meta, &pl.r_down_tile_meta,
+                          &pl.r_up_outbase, &pl.r_down_outbase};
+    for (const Region *r : zs) {
+        cudaError_t e = zero(*r);
+        if (e != cudaSuccess) {
+            snprintf(g_no_ctx_error, sizeof(g_no_ctx_error), "cudaMemset of scratch failed: %s", cudaGetErrorString(e));
+            delete c;
+            return LIEC_ERR_CUDA;
+        }
+    }
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        snprintf(g_no_ctx_error, sizeof(g_no_ctx_error), "cudaDeviceSynchronize failed: %s", cudaGetErrorString(e));
+        delete c;
+        return LIEC_ERR_CUDA;
+    }
+    *out = c;
+    return LIEC_OK;
+}
+
+static liec_status check_stage(liec_ctx *c, int want, const char *name) {
+    if (!c) return LIEC_ERR_INVALID_ARG;
+    if (c->stage != want) {
+        c->err = std::string(name) + " called out of order (stages: uplink, aggregate, downlink, update)";
+        return LIEC_ERR_STATE;
+    }
+    return LIEC_OK;
+}
+
+liec_status liec_uplink_compress(liec_ctx *c, const void *grads, void *stream) {
+    liec_status st = check_stage(c, 0, "liec_uplink_compress");
+    if (st != LIEC_OK) return st;
+    if (!grads || !aligned16(grads)) { c->err = "grads must be non-NULL and 16-byte aligned"; return LIEC_ERR_INVALID_ARG; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    c->p.G = grads;
+    if (c->p.up == COMP_SIGN) {
+        LIEC_LAUNCH(c, launch_sign_uplink(c->p, s));
+        LIEC_LAUNCH(c, launch_scale_finalize(c->p, true, s));
+    } else if (c->p.up == COMP_TOPK) {
+        c->err = "top-k uplink not built";
+        return LIEC_ERR_UNSUPPORTED;
+    }
+    c->stage = 1;
+    return LIEC_OK;
+}
+
+liec_status liec_server_aggregate(liec_ctx *c, void *stream) {
+    liec_status st = check_stage(c, 1, "liec_server_aggregate");
+    if (st != LIEC_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (c->p.up == COMP_TOPK) {
+        c->err = "top-k uplink not built";
+        return LIEC_ERR_UNSUPPORTED;
+    }
+    LIEC_LAUNCH(c, launch_server_dense(c->p, s));
+    c->stage = 2;
+    return LIEC_OK;
+}
+
+liec_status liec_downlink_compress(liec_ctx *c, void *stream) {
+    liec_status st = check_stage(c, 2, "liec_downlink_compress");
+    if (st != LIEC_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (c->p.down == COMP_SIGN) {
+        LIEC_LAUNCH(c, launch_scale_finalize(c->p, false, s));
+        LIEC_LAUNCH(c, launch_sign_error(c->p, s));
+    } else if (c->p.down == COMP_IDENTITY) {
+        LIEC_LAUNCH(c, launch_identity_downlink(c->p, s));
+    } else {
+        c->err = "top-k downlink not built";
+        return LIEC_ERR_UNSUPPORTED;
+    }
+    c->stage = 3;
+    return LIEC_OK;
+}
+
+liec_status liec_worker_update(liec_ctx *c, const void *grads, float lr, void *stream) {
+    liec_status st = check_stage(c, 3, "liec_worker_update");
+    if (st != LIEC_OK) return st;
+    if (grads != c->p.G) { c->err = "liec_worker_update needs the gradient pointer given to liec_uplink_compress"; return LIEC_ERR_INVALID_ARG; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    LIEC_LAUNCH(c, launch_worker_update(c->p, lr, s));
+    c->stage = 0;
+    return LIEC_OK;
+}
+
+liec_status liec_step(liec_ctx *c, const void *grads, float lr, void *stream) {
+    liec_status st = liec_uplink_compress(c, grads, stream);
+    if (st != LIEC_OK) return st;
+    if ((st = liec_server_aggregate(c, stream)) != LIEC_OK) return st;
+    if ((st = liec_downlink_compress(c, stream)) != LIEC_OK) return st;
+    return liec_worker_update(c, grads, lr, stream);
+}
+
+liec_status liec_step_host(liec_ctx *c, const void *grads_host, void *grads_dev, float lr, void *down_msg_host,
+                           void *stream) {
+    if (!c) return LIEC_ERR_INVALID_ARG;
+    if (!grads_host || !grads_dev) { c->err = "grads_host and grads_dev must be non-NULL"; return LIEC_ERR_INVALID_ARG; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t esz = c->p.gdt == DT_BF16 ? 2 : 4;
+    const size_t row_bytes = esz * (size_t)c->p.d;
+    for (int i = 0; i < c->p.N; ++i) {
+        cudaError_t e = cudaMemcpyAsync(static_cast<char *>(grads_dev) + i * row_bytes,
+                                        static_cast<const char *>(grads_host) + i * row_bytes, row_bytes,
+                                        cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpyAsync(grads)");
+    }
+    liec_status st = liec_step(c, grads_dev, lr, stream);
+    if (st != LIEC_OK) return st;
+    if (down_msg_host) {
+        const void *src = nullptr;
+        size_t bytes = 0;
+        if (c->p.down == COMP_SIGN) { src = c->p.down_words; bytes = sizeof(uint32_t) * c->p.W + sizeof(float) * c->p.T; }
+        else if (c->p.down == COMP_TOPK) { src = c->p.down_idx; bytes = 2 * sizeof(uint32_t) * c->p.K; }
+        if (bytes) {
+            cudaError_t e = cudaMemcpyAsync(down_msg_host, src, bytes, cudaMemcpyDeviceToHost, s);
+            if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpyAsync(down message)");
+        }
+    }
+    return LIEC_OK;
+}
+
+liec_status liec_get_messages(const liec_ctx *c, liec_messages *out) {
+    if (!c || !out) return LIEC_ERR_INVALID_ARG;
+    out->up_words = c->p.up_words;
+    out->up_scales = c->p.up_scales;
+    out->up_idx = c->p.up_idx;
+    out->up_val = c->p.up_val;
+    out->down_words = c->p.down_words;
+    out->down_scales = c->p.down_scales;
+    out->down_idx = c->p.down_idx;
+    out->down_val = c->p.down_val;
+    out->v = c->p.e;
+    out->num_words = c->p.W;
+    out->num_topk = c->p.K;
+    return LIEC_OK;
+}
+
+liec_status liec_device_status(liec_ctx *c, void *stream, int32_t *out) {
+    if (!c || !out) return LIEC_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(out, c->p.status, sizeof(int32_t), cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpyAsync(status)");
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaStreamSynchronize");
+    if (*out != 0) { c->err = "a kernel recorded a failed internal check"; return LIEC_ERR_DEVICE_CHECK; }
+    return LIEC_OK;
+}
+
+int64_t liec_launch_count(const liec_ctx *c) { return c ? c->launches : 0; }
+
+const char *liec_last_error(const liec_ctx *c) { return c ? c->err.c_str() : g_no_ctx_error; }
+
+void liec_destroy(liec_ctx *c) { delete c; }
+
+}  // extern "C"

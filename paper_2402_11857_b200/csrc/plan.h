@@ -1,0 +1,76 @@
+// Host-side plan (workspace layout, tile tables) and the parameter block handed to kernels.
+//
+// Work decomposition: every segment t is cut into tiles of TILE consecutive elements
+// counted from the segment's own start, so that a tile is always an aligned subtree of
+// the segment's balanced summation tree and owns whole 32-bit sign words.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+
+namespace liec {
+
+constexpr int TILE = 8192;             // elements per tile
+constexpr int TILE_WORDS = TILE / 32;  // sign words per tile
+constexpr int THREADS = 256;           // threads per CTA in the tile kernels (8 warps x 1024 elements)
+
+constexpr int COMP_IDENTITY = 0, COMP_SIGN = 1, COMP_TOPK = 2;
+constexpr int DT_F32 = 0, DT_BF16 = 1;
+
+// top-k selection constants
+constexpr int DIGIT1_BITS = 12;                 // first radix digit: key bits 30..19
+constexpr int DIGIT1_BINS = 1 << DIGIT1_BITS;
+constexpr int DIGIT1_SHIFT = 31 - DIGIT1_BITS;  // 19
+
+struct Params {
+    int32_t N, T, TT;      // workers, segments, tiles per row
+    int64_t d, W, K;       // dimension, words per row, top-k entries per row
+    int32_t up, down, gdt;
+
+    // tables (device, in the workspace)
+    const int64_t *seg_off;      // [T+1]
+    const int64_t *word_off;     // [T+1]
+    const int64_t *k_off;        // [T+1] (top-k only)
+    const int64_t *cap_off;      // [T+1] candidate capacity prefix (top-k only)
+    const int32_t *tile_prefix;  // [T+1] tiles before segment t
+
+    // state
+    float *X;         // [N][d]
+    float *e;         // [d]
+    const void *G;    // [N][d] current gradients
+
+    // sign messages
+    uint32_t *up_words;    // [N][W]
+    float *up_scales;      // [N][T]
+    double *up_partials;   // [N][TT]
+    uint32_t *down_words;  // [W]
+    float *down_scales;    // [T]
+    double *down_partials; // [TT]
+
+    // top-k messages and scratch (row count R = N for uplink, 1 for downlink)
+    uint32_t *up_idx;  float *up_val;    // [N][K]
+    uint32_t *down_idx; float *down_val; // [K]
+    uint32_t *up_hist, *down_hist;       // [R][T][DIGIT1_BINS]
+    uint32_t *up_hist2, *down_hist2;     // [R][T][DIGIT1_BINS] second / third digit
+    uint32_t *up_sel, *down_sel;         // [R][T][SEL_WORDS] per-problem selection state
+    uint32_t *up_cand_idx, *down_cand_idx;   // [R][CAP] candidate entries
+    float *up_cand_val, *down_cand_val;      // [R][CAP]
+    uint32_t *up_tile_meta, *down_tile_meta; // [R][TT][4] pos, cnt, n_greater, n_ties
+    uint32_t *up_outbase, *down_outbase;     // [R][TT+1] first output slot of each tile
+    int64_t CAP;                              // candidate capacity per row
+
+    float *vbuf;      // [d] identity downlink copy of v
+    int32_t *status;  // device status word
+};
+
+// per-problem selection state words
+constexpr int SEL_WORDS = 8;
+constexpr int SEL_PREFIX = 0;     // key prefix fixed so far (aligned to its bit position)
+constexpr int SEL_REMAIN = 1;     // rank still to find inside the prefix bin (1-based)
+constexpr int SEL_CAND_COUNT = 2; // atomic cursor: candidates appended so far
+constexpr int SEL_THRESH = 3;     // final threshold key T
+constexpr int SEL_TIES = 4;       // number of entries equal to T to accept, lowest index first
+constexpr int SEL_CUT = 5;        // flat index of the last accepted tie
+constexpr int SEL_FLAGS = 6;      // bit0: candidate buffer overflow -> slow path
+constexpr int SEL_NCAND = 7;      // exact number of candidates (elements with digit1 >= bin1)
+
+}  // namespace liec

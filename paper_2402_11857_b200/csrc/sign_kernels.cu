@@ -1,0 +1,311 @@
+// Scaled-sign operator (Def. 4 / Def. 5) and the server pass that consumes sign messages.
+//
+//   sign_uplink_kernel     p^i = C(g^i): sign words + per-tile binary64 partial of ||g||_1
+//   scale_finalize_kernel  combines tile partials in tree order, scale = ||x||_1 / n
+//   server_dense_kernel    v = e + (1/N) sum_i p^i for sign / identity uplinks, fused with
+//                          the first half of a sign downlink (words of v, partials of ||v||_1)
+//   sign_error_kernel      e <- v - p for a sign downlink
+#include "device_common.cuh"
+#include "kernels.h"
+
+namespace liec {
+
+// ------------------------------------------------------------------------------------------------
+// Uplink: one CTA per (tile, worker).  Reads g once; writes 1 bit per element and one double.
+// ------------------------------------------------------------------------------------------------
+template <typename GT>
+__global__ void __launch_bounds__(THREADS) sign_uplink_kernel(const __grid_constant__ Params p) {
+    __shared__ double warp_sums[8];
+    const int worker = blockIdx.y;
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t row_beg = (int64_t)worker * p.d + ti.seg_beg;  // segment start in the [N][d] array
+    const GT *tile_ptr = reinterpret_cast<const GT *>(p.G) + row_beg + ti.rel;
+    const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+
+    float v[8][4];
+    if (fast) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) load4_stream(tile_ptr + tile_pos(warp, lane, j), v[j]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v[j]);
+    }
+
+    uint32_t *words = p.up_words + (int64_t)worker * p.W + __ldg(p.word_off + ti.t) + ti.rel / 32;
+    const int nwords = (ti.len + 31) >> 5;
+    double a[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        a[j] = leaf4(v[j]);
+        uint32_t w = pack_word(sign_nibble(v[j]), lane);
+        int widx = warp * 32 + j * 4 + (lane >> 3);
+        if ((lane & 7) == 0 && widx < nwords) words[widx] = w;
+    }
+    double s = cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
+    if (threadIdx.x == 0) p.up_partials[(int64_t)worker * p.TT + blockIdx.x] = s;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Scale: one CTA per (segment, row).  Tile partials are combined pairwise, level by level,
+// over the tile count zero-padded to a power of two (adding +0 is exact), which continues the
+// segment's balanced tree above the tile level.
+// ------------------------------------------------------------------------------------------------
+constexpr int FIN_CHUNK = 2048;
+
+__global__ void __launch_bounds__(THREADS) scale_finalize_kernel(const __grid_constant__ Params p,
+                                                                  const double *partials, float *scales) {
+    __shared__ double buf[FIN_CHUNK];
+    __shared__ double chunk_sums[512];  // 2^32 / TILE / FIN_CHUNK = 256 chunks at most
+    const int t = blockIdx.x, row = blockIdx.y;
+    const int first = __ldg(p.tile_prefix + t);
+    const int ntiles = __ldg(p.tile_prefix + t + 1) - first;
+    const double *src = partials + (int64_t)row * p.TT + first;
+    const int nchunks = (ntiles + FIN_CHUNK - 1) / FIN_CHUNK;
+
+    for (int c = 0; c < nchunks; ++c) {
+        for (int q = threadIdx.x; q < FIN_CHUNK; q += THREADS) {
+            int idx = c * FIN_CHUNK + q;
+            buf[q] = idx < ntiles ? src[idx] : 0.0;
+        }
+        __syncthreads();
+        for (int width = FIN_CHUNK / 2; width >= 1; width >>= 1) {
+            // pairwise: new[q] = old[2q] + old[2q+1]; done in two phases to avoid overwrite hazards
+            double vals[FIN_CHUNK / 2 / THREADS];
+#pragma unroll
+            for (int r = 0; r < FIN_CHUNK / 2 / THREADS; ++r) {
+                int q = threadIdx.x + r * THREADS;
+                vals[r] = q < width ? __dadd_rn(buf[2 * q], buf[2 * q + 1]) : 0.0;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int r = 0; r < FIN_CHUNK / 2 / THREADS; ++r) {
+                int q = threadIdx.x + r * THREADS;
+                if (q < width) buf[q] = vals[r];
+            }
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) chunk_sums[c] = buf[0];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        int L = 1;
+        while (L < nchunks) L <<= 1;
+        for (int c = nchunks; c < L; ++c) chunk_sums[c] = 0.0;
+        for (int width = L / 2; width >= 1; width >>= 1)
+            for (int q = 0; q < width; ++q) chunk_sums[q] = __dadd_rn(chunk_sums[2 * q], chunk_sums[2 * q + 1]);
+        const int64_t n = __ldg(p.seg_off + t + 1) - __ldg(p.seg_off + t);
+        double mean = __ddiv_rn(chunk_sums[0], (double)n);
+        scales[(int64_t)row * p.T + t] = __double2float_rn(mean);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Server pass for dense uplink messages (sign words or raw gradients): one CTA per tile.
+//   acc = +0; for i = 0..N-1: acc = acc + p^i_j;   v_j = e_j + acc / N        (written over e)
+// and, when the downlink is scaled sign, the words of v and the tile partial of ||v||_1.
+// ------------------------------------------------------------------------------------------------
+template <int UP, bool DOWN_SIGN, typename GT>
+__global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_constant__ Params p) {
+    __shared__ double warp_sums[8];
+    extern __shared__ float up_scale_smem[];  // [N] scales of this segment (sign uplink)
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
+    const int64_t wbase = __ldg(p.word_off + ti.t) + ti.rel / 32;
+    const int nwords = (ti.len + 31) >> 5;
+
+    if (UP == COMP_SIGN) {
+        for (int i = threadIdx.x; i < p.N; i += THREADS) up_scale_smem[i] = p.up_scales[(int64_t)i * p.T + ti.t];
+        __syncthreads();
+    }
+
+    float acc[8][4];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[j][c] = 0.0f;
+
+    if (UP == COMP_SIGN) {
+        const int my_widx = warp * 32 + lane;
+        for (int i = 0; i < p.N; ++i) {
+            const uint32_t sbits = __float_as_uint(up_scale_smem[i]);
+            uint32_t my_word = my_widx < nwords ? __ldg(p.up_words + (int64_t)i * p.W + wbase + my_widx) : 0u;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                uint32_t nib = nibble_from_words(my_word, lane, j);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    float pij = __uint_as_float(sbits ^ ((nib << (31 - c)) & 0x80000000u));
+                    acc[j][c] = __fadd_rn(acc[j][c], pij);
+                }
+            }
+        }
+    } else {  // identity uplink: the message is the gradient itself
+        for (int i = 0; i < p.N; ++i) {
+            const int64_t row_beg = (int64_t)i * p.d + ti.seg_beg;
+            const GT *tile_ptr = reinterpret_cast<const GT *>(p.G) + row_beg + ti.rel;
+            const bool gfast = (ti.len == TILE) && ((row_beg & 3) == 0);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                float g[4];
+                if (gfast) load4_stream(tile_ptr + tile_pos(warp, lane, j), g);
+                else load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, g);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) acc[j][c] = __fadd_rn(acc[j][c], g[c]);
+            }
+        }
+    }
+
+    const float nf = (float)p.N;
+    float *e_tile = p.e + ti.seg_beg + ti.rel;
+    double a[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pos = tile_pos(warp, lane, j);
+        float ev[4], v[4];
+        if (fast) load4_stream(e_tile + pos, ev);
+        else load4_guarded(e_tile, pos, ti.len, ev);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) v[c] = __fadd_rn(ev[c], __fdiv_rn(acc[j][c], nf));
+        if (fast) {
+            *reinterpret_cast<float4 *>(e_tile + pos) = make_float4(v[0], v[1], v[2], v[3]);
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                if (pos + c < ti.len) e_tile[pos + c] = v[c]; else v[c] = 0.0f;  // padding: +0, bit 0
+            }
+        }
+        if (DOWN_SIGN) {
+            a[j] = leaf4(v);
+            uint32_t w = pack_word(sign_nibble(v), lane);
+            int widx = warp * 32 + j * 4 + (lane >> 3);
+            if ((lane & 7) == 0 && widx < nwords) p.down_words[wbase + widx] = w;
+        }
+    }
+    if (DOWN_SIGN) {
+        double s = cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
+        if (threadIdx.x == 0) p.down_partials[blockIdx.x] = s;
+    }
+}
+
+// First half of a sign downlink on a v that is already in the error buffer (used when the
+// aggregation kernel could not fuse it, i.e. after a top-k uplink).
+__global__ void __launch_bounds__(THREADS) sign_downlink_kernel(const __grid_constant__ Params p) {
+    __shared__ double warp_sums[8];
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
+    const int64_t wbase = __ldg(p.word_off + ti.t) + ti.rel / 32;
+    const int nwords = (ti.len + 31) >> 5;
+    const float *v_tile = p.e + ti.seg_beg + ti.rel;
+    double a[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pos = tile_pos(warp, lane, j);
+        float v[4];
+        if (fast) load4_stream(v_tile + pos, v);
+        else load4_guarded(v_tile, pos, ti.len, v);
+        a[j] = leaf4(v);
+        uint32_t w = pack_word(sign_nibble(v), lane);
+        int widx = warp * 32 + j * 4 + (lane >> 3);
+        if ((lane & 7) == 0 && widx < nwords) p.down_words[wbase + widx] = w;
+    }
+    double s = cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
+    if (threadIdx.x == 0) p.down_partials[blockIdx.x] = s;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Global error for a sign downlink: e_j <- v_j - p_j with p_j = -s or +s by the sign word.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(THREADS) sign_error_kernel(const __grid_constant__ Params p) {
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
+    const int64_t wbase = __ldg(p.word_off + ti.t) + ti.rel / 32;
+    const int nwords = (ti.len + 31) >> 5;
+    const float s = p.down_scales[ti.t];
+    const uint32_t sbits = __float_as_uint(s);
+    float *e_tile = p.e + ti.seg_beg + ti.rel;
+    const int my_widx = warp * 32 + lane;
+    const uint32_t my_word = my_widx < nwords ? p.down_words[wbase + my_widx] : 0u;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pos = tile_pos(warp, lane, j);
+        uint32_t nib = nibble_from_words(my_word, lane, j);
+        float v[4];
+        if (fast) load4_stream(e_tile + pos, v);
+        else load4_guarded(e_tile, pos, ti.len, v);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            float pj = __uint_as_float(sbits ^ ((nib << (31 - c)) & 0x80000000u));
+            v[c] = __fsub_rn(v[c], pj);
+        }
+        if (fast) {
+            *reinterpret_cast<float4 *>(e_tile + pos) = make_float4(v[0], v[1], v[2], v[3]);
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (pos + c < ti.len) e_tile[pos + c] = v[c];
+        }
+    }
+}
+
+// Identity downlink: p = v, so the workers read v from a copy and the error becomes +0.
+__global__ void __launch_bounds__(THREADS) identity_downlink_kernel(const __grid_constant__ Params p) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < p.d; j += stride) {
+        p.vbuf[j] = p.e[j];
+        p.e[j] = 0.0f;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// launchers
+// ------------------------------------------------------------------------------------------------
+cudaError_t launch_sign_uplink(const Params &p, cudaStream_t st) {
+    dim3 grid(p.TT, p.N);
+    if (p.gdt == DT_F32) sign_uplink_kernel<float><<<grid, THREADS, 0, st>>>(p);
+    else sign_uplink_kernel<__nv_bfloat16><<<grid, THREADS, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scale_finalize(const Params &p, bool uplink, cudaStream_t st) {
+    dim3 grid(p.T, uplink ? p.N : 1);
+    scale_finalize_kernel<<<grid, THREADS, 0, st>>>(p, uplink ? p.up_partials : p.down_partials,
+                                                    uplink ? p.up_scales : p.down_scales);
+    return cudaGetLastError();
+}
+
+template <int UP, typename GT>
+static cudaError_t launch_server_dense_t(const Params &p, cudaStream_t st) {
+    size_t smem = UP == COMP_SIGN ? sizeof(float) * (size_t)p.N : 0;
+    if (p.down == COMP_SIGN) server_dense_kernel<UP, true, GT><<<p.TT, THREADS, smem, st>>>(p);
+    else server_dense_kernel<UP, false, GT><<<p.TT, THREADS, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_server_dense(const Params &p, cudaStream_t st) {
+    if (p.up == COMP_SIGN) return launch_server_dense_t<COMP_SIGN, float>(p, st);
+    if (p.gdt == DT_F32) return launch_server_dense_t<COMP_IDENTITY, float>(p, st);
+    return launch_server_dense_t<COMP_IDENTITY, __nv_bfloat16>(p, st);
+}
+
+cudaError_t launch_sign_downlink(const Params &p, cudaStream_t st) {
+    sign_downlink_kernel<<<p.TT, THREADS, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sign_error(const Params &p, cudaStream_t st) {
+    sign_error_kernel<<<p.TT, THREADS, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_identity_downlink(const Params &p, cudaStream_t st) {
+    int64_t blocks = (p.d + THREADS - 1) / THREADS;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    identity_downlink_kernel<<<(int)blocks, THREADS, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace liec

@@ -1,0 +1,93 @@
+// Local immediate error compensation and model update (last worker step of Algorithm 1):
+//   x^i_j <- x^i_j - eta * ((p_j - p^i_j) + g^i_j)
+// p^i is not stored: it is recomputed from g^i and the worker's own scale (sign), its
+// selection threshold (top-k) or taken as g^i itself (identity).  p is decoded from the
+// downlink message.
+#include "device_common.cuh"
+#include "kernels.h"
+
+namespace liec {
+
+template <int UP, int DOWN, typename GT>
+__global__ void __launch_bounds__(THREADS) worker_update_kernel(const __grid_constant__ Params p, const float lr) {
+    const int worker = blockIdx.y;
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t row_beg = (int64_t)worker * p.d + ti.seg_beg;
+    const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+    const GT *g_tile = reinterpret_cast<const GT *>(p.G) + row_beg + ti.rel;
+    float *x_tile = p.X + row_beg + ti.rel;
+
+    float su = 0.0f, sd = 0.0f;
+    uint32_t my_word = 0u;
+    if (UP == COMP_SIGN) su = p.up_scales[(int64_t)worker * p.T + ti.t];
+    if (DOWN == COMP_SIGN) {
+        sd = p.down_scales[ti.t];
+        const int nwords = (ti.len + 31) >> 5;
+        const int my_widx = warp * 32 + lane;
+        if (my_widx < nwords) my_word = __ldg(p.down_words + __ldg(p.word_off + ti.t) + ti.rel / 32 + my_widx);
+    }
+    const uint32_t su_bits = __float_as_uint(su), sd_bits = __float_as_uint(sd);
+    const float *v_tile = DOWN == COMP_IDENTITY ? p.vbuf + ti.seg_beg + ti.rel : nullptr;
+
+    float g[8][4], x[8][4];
+    if (fast) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) load4_stream(g_tile + tile_pos(warp, lane, j), g[j]);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) load4_stream(x_tile + tile_pos(warp, lane, j), x[j]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            load4_guarded(g_tile, tile_pos(warp, lane, j), ti.len, g[j]);
+            load4_guarded(x_tile, tile_pos(warp, lane, j), ti.len, x[j]);
+        }
+    }
+
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pos = tile_pos(warp, lane, j);
+        float pd[4];
+        if (DOWN == COMP_SIGN) {
+            uint32_t nib = nibble_from_words(my_word, lane, j);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) pd[c] = __uint_as_float(sd_bits ^ ((nib << (31 - c)) & 0x80000000u));
+        } else if (DOWN == COMP_IDENTITY) {
+            load4_guarded(v_tile, pos, ti.len, pd);
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            float pi;
+            if (UP == COMP_SIGN) pi = __uint_as_float(su_bits ^ (g[j][c] < 0.0f ? 0x80000000u : 0u));
+            else pi = g[j][c];
+            float diff = __fsub_rn(pd[c], pi);
+            float u = __fadd_rn(diff, g[j][c]);
+            x[j][c] = __fsub_rn(x[j][c], __fmul_rn(lr, u));
+        }
+        if (fast) {
+            __stcs(reinterpret_cast<float4 *>(x_tile + pos), make_float4(x[j][0], x[j][1], x[j][2], x[j][3]));
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (pos + c < ti.len) x_tile[pos + c] = x[j][c];
+        }
+    }
+}
+
+template <int UP, int DOWN>
+static cudaError_t launch_t(const Params &p, float lr, cudaStream_t st) {
+    dim3 grid(p.TT, p.N);
+    if (p.gdt == DT_F32) worker_update_kernel<UP, DOWN, float><<<grid, THREADS, 0, st>>>(p, lr);
+    else worker_update_kernel<UP, DOWN, __nv_bfloat16><<<grid, THREADS, 0, st>>>(p, lr);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_worker_update(const Params &p, float lr, cudaStream_t st) {
+    if (p.up == COMP_SIGN && p.down == COMP_SIGN) return launch_t<COMP_SIGN, COMP_SIGN>(p, lr, st);
+    if (p.up == COMP_SIGN && p.down == COMP_IDENTITY) return launch_t<COMP_SIGN, COMP_IDENTITY>(p, lr, st);
+    if (p.up == COMP_IDENTITY && p.down == COMP_SIGN) return launch_t<COMP_IDENTITY, COMP_SIGN>(p, lr, st);
+    if (p.up == COMP_IDENTITY && p.down == COMP_IDENTITY) return launch_t<COMP_IDENTITY, COMP_IDENTITY>(p, lr, st);
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace liec
