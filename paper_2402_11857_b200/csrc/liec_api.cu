@@ -190,6 +190,12 @@ liec_status cuda_fail(liec_ctx *c, cudaError_t e, const char *what) {
         ++(ctx)->launches;                                            \
     } while (0)
 
+#define LIEC_CALL(ctx, call)                                          \
+    do {                                                              \
+        cudaError_t e__ = (call);                                     \
+        if (e__ != cudaSuccess) return cuda_fail(ctx, e__, #call);    \
+    } while (0)
+
 bool aligned16(const void *ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
 
 }  // namespace
@@ -288,9 +294,10 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
             return LIEC_ERR_CUDA;
         }
     }
-    cudaError_t e = cudaDeviceSynchronize();
+    cudaError_t e = configure_topk_kernels();
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
-        snprintf(g_no_ctx_error, sizeof(g_no_ctx_error), "cudaDeviceSynchronize failed: %s", cudaGetErrorString(e));
+        snprintf(g_no_ctx_error, sizeof(g_no_ctx_error), "kernel configuration / synchronize failed: %s", cudaGetErrorString(e));
         delete c;
         return LIEC_ERR_CUDA;
     }
@@ -317,8 +324,8 @@ liec_status liec_uplink_compress(liec_ctx *c, const void *grads, void *stream) {
         LIEC_LAUNCH(c, launch_sign_uplink(c->p, s));
         LIEC_LAUNCH(c, launch_scale_finalize(c->p, true, s));
     } else if (c->p.up == COMP_TOPK) {
-        c->err = "top-k uplink not built";
-        return LIEC_ERR_UNSUPPORTED;
+        LIEC_CALL(c, launch_topk_hist1(c->p, true, s, &c->launches));
+        LIEC_CALL(c, launch_topk_select(c->p, true, s, &c->launches));
     }
     c->stage = 1;
     return LIEC_OK;
@@ -329,10 +336,10 @@ liec_status liec_server_aggregate(liec_ctx *c, void *stream) {
     if (st != LIEC_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (c->p.up == COMP_TOPK) {
-        c->err = "top-k uplink not built";
-        return LIEC_ERR_UNSUPPORTED;
+        LIEC_CALL(c, launch_server_topk(c->p, s, &c->launches));
+    } else {
+        LIEC_LAUNCH(c, launch_server_dense(c->p, s));
     }
-    LIEC_LAUNCH(c, launch_server_dense(c->p, s));
     c->stage = 2;
     return LIEC_OK;
 }
@@ -347,8 +354,9 @@ liec_status liec_downlink_compress(liec_ctx *c, void *stream) {
     } else if (c->p.down == COMP_IDENTITY) {
         LIEC_LAUNCH(c, launch_identity_downlink(c->p, s));
     } else {
-        c->err = "top-k downlink not built";
-        return LIEC_ERR_UNSUPPORTED;
+        // the first-digit histogram of v is fused into the server pass after a top-k uplink
+        if (c->p.up != COMP_TOPK) LIEC_CALL(c, launch_topk_hist1(c->p, false, s, &c->launches));
+        LIEC_CALL(c, launch_topk_select(c->p, false, s, &c->launches));
     }
     c->stage = 3;
     return LIEC_OK;

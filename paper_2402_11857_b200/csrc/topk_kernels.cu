@@ -1,0 +1,638 @@
+// Deterministic top-k (Def. 2) per segment: exact radix select on the 31-bit magnitude key,
+// ties broken toward the lower index, output (index, value) compacted in ascending index.
+//
+// One selection "problem" is a (row, segment) pair; the uplink has N rows (the workers'
+// gradients), the downlink one row (v, held in the error buffer).  Pipeline per side:
+//
+//   hist1   dense pass 1: histogram of the first key digit (bits 30..19) per problem
+//   pick1   bin b1 holding the k-th largest key, rank left inside it, exact candidate count
+//   filter  dense pass 2: entries with digit >= b1 appended (in index order inside each tile)
+//           to the problem's candidate buffer; histogram of the second digit (bits 18..7)
+//           over the entries whose first digit equals b1
+//   pick2   second digit
+//   hist3   candidates only: histogram of the last 7 key bits under the 24-bit prefix
+//   pick3   threshold key and number of ties to accept
+//   count   candidates only: per tile, entries above the threshold and entries equal to it
+//   scan    per problem: first output slot and accepted ties of every tile
+//   write   candidates only: ordered compaction into (idx, val); records the last accepted tie
+//   slow    one CTA per problem, only for problems whose candidates exceed the buffer
+//           (huge groups of equal magnitudes, e.g. mostly-zero rows): same result, dense passes
+//
+// Nothing waits on another CTA; cross-CTA order comes from kernel boundaries.
+#include "device_common.cuh"
+#include "kernels.h"
+
+namespace liec {
+
+struct TopkSide {
+    const void *src;      // rows of the vector being compressed
+    int64_t row_stride;   // elements between rows (d for the uplink, 0 for the single downlink row)
+    int R;                // rows
+    uint32_t *idx; float *val;            // [R][K] output message
+    uint32_t *hist, *hist2, *sel;         // [R][T][...]
+    uint32_t *cand_idx; float *cand_val;  // [R][CAP]
+    uint32_t *meta;                        // [R][TT][4]: pos, cnt, n_greater -> unused, ties allowed
+    uint32_t *outbase;                     // [R][TT+1]
+    float *zero_out;                       // downlink: error buffer, selected entries become +0
+};
+
+static TopkSide make_side(const Params &p, bool uplink) {
+    TopkSide s;
+    if (uplink) {
+        s.src = p.G; s.row_stride = p.d; s.R = p.N;
+        s.idx = p.up_idx; s.val = p.up_val; s.hist = p.up_hist; s.hist2 = p.up_hist2; s.sel = p.up_sel;
+        s.cand_idx = p.up_cand_idx; s.cand_val = p.up_cand_val; s.meta = p.up_tile_meta; s.outbase = p.up_outbase;
+        s.zero_out = nullptr;
+    } else {
+        s.src = p.e; s.row_stride = 0; s.R = 1;
+        s.idx = p.down_idx; s.val = p.down_val; s.hist = p.down_hist; s.hist2 = p.down_hist2; s.sel = p.down_sel;
+        s.cand_idx = p.down_cand_idx; s.cand_val = p.down_cand_val; s.meta = p.down_tile_meta; s.outbase = p.down_outbase;
+        s.zero_out = p.e;
+    }
+    return s;
+}
+
+__device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) & 0x7fffffffu; }
+
+enum { STATUS_PICK_RANK = 1, STATUS_CAND_OVERFLOW = 2, STATUS_COUNT_MISMATCH = 4 };
+
+// ------------------------------------------------------------------------------------------------
+// Block helper: bins[0..nbins) in shared memory, find the bin that holds the rank-th largest
+// entry counting from the top bin down.  All threads get (bin, rank inside bin, count above+bin).
+// ------------------------------------------------------------------------------------------------
+struct PickResult { uint32_t bin, rank_in_bin, count_ge; bool ok; };
+
+__device__ PickResult block_pick(const uint32_t *bins, int nbins, uint32_t rank, uint32_t *scratch /*[THREADS+4]*/) {
+    const int tid = threadIdx.x;
+    const int per = nbins >= THREADS ? nbins / THREADS : 1;
+    const int active = nbins / per;
+    uint32_t mine = 0;
+    if (tid < active)
+        for (int q = 0; q < per; ++q) mine += bins[tid * per + q];
+    // inclusive suffix sum over threads: suf[i] = sum_{i' >= i} mine[i']
+    scratch[tid] = mine;
+    __syncthreads();
+    for (int offs = 1; offs < THREADS; offs <<= 1) {
+        uint32_t add = (tid + offs < THREADS) ? scratch[tid + offs] : 0u;
+        __syncthreads();
+        scratch[tid] += add;
+        __syncthreads();
+    }
+    const uint32_t suf_incl = scratch[tid];
+    const uint32_t suf_excl = suf_incl - mine;
+    if (tid == 0) scratch[THREADS + 3] = 0u;  // found flag
+    __syncthreads();
+    if (tid < active && suf_excl < rank && rank <= suf_incl) {
+        uint32_t above = suf_excl;
+        for (int q = per - 1; q >= 0; --q) {
+            uint32_t c = bins[tid * per + q];
+            if (above + c >= rank) {
+                scratch[THREADS + 0] = (uint32_t)(tid * per + q);
+                scratch[THREADS + 1] = rank - above;
+                scratch[THREADS + 2] = above + c;
+                scratch[THREADS + 3] = 1u;
+                break;
+            }
+            above += c;
+        }
+    }
+    __syncthreads();
+    PickResult r;
+    r.bin = scratch[THREADS + 0];
+    r.rank_in_bin = scratch[THREADS + 1];
+    r.count_ge = scratch[THREADS + 2];
+    r.ok = scratch[THREADS + 3] != 0u;
+    __syncthreads();
+    return r;
+}
+
+// ------------------------------------------------------------------------------------------------
+// hist1: one CTA per (tile, row)
+// ------------------------------------------------------------------------------------------------
+template <typename GT>
+__global__ void __launch_bounds__(THREADS) topk_hist1_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    __shared__ uint32_t h[DIGIT1_BINS];
+    const int row = blockIdx.y;
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) h[b] = 0u;
+    __syncthreads();
+    const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
+    const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
+    const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+    float v[8][4];
+    if (fast) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) load4_stream(tile_ptr + tile_pos(warp, lane, j), v[j]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v[j]);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pos = tile_pos(warp, lane, j);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if (fast || pos + c < ti.len) atomicAdd(&h[key_of(v[j][c]) >> DIGIT1_SHIFT], 1u);
+    }
+    __syncthreads();
+    uint32_t *gh = s.hist + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS;
+    for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) {
+        uint32_t c = h[b];
+        if (c) atomicAdd(gh + b, c);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// pick: one CTA per (segment, row).  level 1: first digit; 2: second digit; 3: last 7 bits.
+// The histogram is cleared for the next use.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constant__ Params p, const TopkSide s,
+                                                             const int level) {
+    __shared__ uint32_t bins[DIGIT1_BINS];
+    __shared__ uint32_t scratch[THREADS + 4];
+    const int t = blockIdx.x, row = blockIdx.y;
+    uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
+    if (level > 1 && (sel[SEL_FLAGS] & 1u)) return;  // handled by the slow path
+    const int nbins = level == 3 ? 128 : DIGIT1_BINS;
+    uint32_t *gh = (level == 1 ? s.hist : s.hist2) + ((int64_t)row * p.T + t) * DIGIT1_BINS;
+    for (int b = threadIdx.x; b < nbins; b += THREADS) {
+        bins[b] = gh[b];
+        gh[b] = 0u;
+    }
+    __syncthreads();
+    const uint32_t k = (uint32_t)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
+    const uint32_t rank = level == 1 ? k : sel[SEL_REMAIN];
+    const PickResult r = block_pick(bins, nbins, rank, scratch);
+    if (threadIdx.x == 0) {
+        if (!r.ok) { atomicOr(p.status, STATUS_PICK_RANK); return; }
+        if (level == 1) {
+            const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
+            sel[SEL_PREFIX] = r.bin;
+            sel[SEL_REMAIN] = r.rank_in_bin;
+            sel[SEL_NCAND] = r.count_ge;
+            sel[SEL_CAND_COUNT] = 0u;
+            sel[SEL_FLAGS] = r.count_ge > cap ? 1u : 0u;
+        } else if (level == 2) {
+            sel[SEL_PREFIX] = (sel[SEL_PREFIX] << 12) | r.bin;
+            sel[SEL_REMAIN] = r.rank_in_bin;
+        } else {
+            sel[SEL_THRESH] = (sel[SEL_PREFIX] << 7) | r.bin;
+            sel[SEL_TIES] = r.rank_in_bin;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// filter: one CTA per (tile, row); ordered append of candidates
+// ------------------------------------------------------------------------------------------------
+template <typename GT>
+__global__ void __launch_bounds__(THREADS) topk_filter_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    __shared__ uint32_t warp_tot[8];
+    __shared__ uint32_t tile_base;
+    const int row = blockIdx.y;
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
+    if (sel[SEL_FLAGS] & 1u) return;
+    const uint32_t b1 = sel[SEL_PREFIX];
+    const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
+    const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
+    const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+    float v[8][4];
+    if (fast) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) load4_stream(tile_ptr + tile_pos(warp, lane, j), v[j]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v[j]);
+    }
+    uint32_t *gh2 = s.hist2 + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    uint32_t nib[8], rowoff[8];
+    uint32_t running = 0;  // candidates of this warp before the current row
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pos = tile_pos(warp, lane, j);
+        uint32_t f = 0, before = 0, total = 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint32_t key = key_of(v[j][c]);
+            const uint32_t d1 = key >> DIGIT1_SHIFT;
+            const bool valid = fast || pos + c < ti.len;
+            const bool cand = valid && d1 >= b1;
+            if (valid && d1 == b1) atomicAdd(gh2 + ((key >> 7) & 0xfffu), 1u);
+            const uint32_t bal = __ballot_sync(0xffffffffu, cand);
+            before += __popc(bal & lt_mask);
+            total += __popc(bal);
+            f |= cand ? (1u << c) : 0u;
+        }
+        nib[j] = f;
+        rowoff[j] = running + before;
+        running += total;
+    }
+    if (lane == 0) warp_tot[warp] = running;
+    __syncthreads();
+    uint32_t warp_off = 0, tile_cnt = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) {
+        if (w < warp) warp_off += warp_tot[w];
+        tile_cnt += warp_tot[w];
+    }
+    const uint32_t cap = (uint32_t)(__ldg(p.cap_off + ti.t + 1) - __ldg(p.cap_off + ti.t));
+    if (threadIdx.x == 0) {
+        uint32_t pos0 = tile_cnt ? atomicAdd(&sel[SEL_CAND_COUNT], tile_cnt) : 0u;
+        if (pos0 + tile_cnt > cap) { atomicOr(p.status, STATUS_CAND_OVERFLOW); pos0 = 0xffffffffu; }
+        tile_base = pos0;
+        uint32_t *m = s.meta + ((int64_t)row * p.TT + blockIdx.x) * 4;
+        m[0] = pos0 == 0xffffffffu ? 0u : pos0;
+        m[1] = pos0 == 0xffffffffu ? 0u : tile_cnt;
+    }
+    __syncthreads();
+    if (tile_base == 0xffffffffu) return;
+    const int64_t cbase = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + tile_base + warp_off;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        uint32_t o = rowoff[j];
+        const uint32_t flat = (uint32_t)(ti.seg_beg + ti.rel) + tile_pos(warp, lane, j);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            if (nib[j] & (1u << c)) {
+                s.cand_idx[cbase + o] = flat + c;
+                s.cand_val[cbase + o] = v[j][c];
+                ++o;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// candidate passes: one CTA per (tile, row) walks that tile's block of the candidate buffer
+// ------------------------------------------------------------------------------------------------
+struct CandBlock { int64_t base; uint32_t cnt; int t; uint32_t *sel; uint32_t *meta; bool skip; };
+
+__device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide &s, int tile, int row) {
+    CandBlock cb;
+    const TileInfo ti = locate_tile(p, tile);
+    cb.t = ti.t;
+    cb.sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
+    cb.meta = s.meta + ((int64_t)row * p.TT + tile) * 4;
+    cb.skip = (cb.sel[SEL_FLAGS] & 1u) != 0u;
+    cb.cnt = cb.skip ? 0u : cb.meta[1];
+    cb.base = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + cb.meta[0];
+    return cb;
+}
+
+__global__ void __launch_bounds__(THREADS) topk_hist3_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    const int row = blockIdx.y;
+    const CandBlock cb = cand_block(p, s, blockIdx.x, row);
+    if (cb.skip) return;
+    const uint32_t prefix24 = cb.sel[SEL_PREFIX];
+    uint32_t *gh = s.hist2 + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
+    for (uint32_t q = threadIdx.x; q < cb.cnt; q += THREADS) {
+        const uint32_t key = key_of(s.cand_val[cb.base + q]);
+        if ((key >> 7) == prefix24) atomicAdd(gh + (key & 0x7fu), 1u);
+    }
+}
+
+__global__ void __launch_bounds__(THREADS) topk_count_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    __shared__ uint32_t cnt_g, cnt_t;
+    const int row = blockIdx.y;
+    const CandBlock cb = cand_block(p, s, blockIdx.x, row);
+    if (cb.skip) return;
+    if (threadIdx.x == 0) { cnt_g = 0u; cnt_t = 0u; }
+    __syncthreads();
+    const uint32_t T = cb.sel[SEL_THRESH];
+    uint32_t g = 0, e = 0;
+    for (uint32_t q = threadIdx.x; q < cb.cnt; q += THREADS) {
+        const uint32_t key = key_of(s.cand_val[cb.base + q]);
+        g += key > T ? 1u : 0u;
+        e += key == T ? 1u : 0u;
+    }
+    g = __reduce_add_sync(0xffffffffu, g);
+    e = __reduce_add_sync(0xffffffffu, e);
+    if ((threadIdx.x & 31) == 0) { if (g) atomicAdd(&cnt_g, g); if (e) atomicAdd(&cnt_t, e); }
+    __syncthreads();
+    if (threadIdx.x == 0) { cb.meta[2] = cnt_g; cb.meta[3] = cnt_t; }
+}
+
+// scan: one CTA per (segment, row); tiles of the segment in order
+__global__ void __launch_bounds__(THREADS) topk_scan_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    __shared__ uint32_t sg[THREADS], st[THREADS];
+    __shared__ uint32_t carry_sel, carry_ties;
+    const int t = blockIdx.x, row = blockIdx.y;
+    uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
+    if (sel[SEL_FLAGS] & 1u) return;
+    const int first = __ldg(p.tile_prefix + t), ntiles = __ldg(p.tile_prefix + t + 1) - first;
+    const uint32_t ties_wanted = sel[SEL_TIES];
+    const uint32_t kbeg = (uint32_t)__ldg(p.k_off + t), k = (uint32_t)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
+    if (threadIdx.x == 0) { carry_sel = 0u; carry_ties = 0u; }
+    __syncthreads();
+    for (int c0 = 0; c0 < ntiles; c0 += THREADS) {
+        const int q = c0 + threadIdx.x;
+        uint32_t *m = s.meta + ((int64_t)row * p.TT + first + (q < ntiles ? q : 0)) * 4;
+        const uint32_t g = q < ntiles ? m[2] : 0u, e = q < ntiles ? m[3] : 0u;
+        // exclusive prefix of the tie counts inside the chunk
+        st[threadIdx.x] = e;
+        __syncthreads();
+        for (int offs = 1; offs < THREADS; offs <<= 1) {
+            uint32_t add = threadIdx.x >= offs ? st[threadIdx.x - offs] : 0u;
+            __syncthreads();
+            st[threadIdx.x] += add;
+            __syncthreads();
+        }
+        const uint32_t ties_before = carry_ties + st[threadIdx.x] - e;
+        uint32_t allowed = 0;
+        if (ties_before < ties_wanted) allowed = min(e, ties_wanted - ties_before);
+        const uint32_t mine = g + allowed;
+        sg[threadIdx.x] = mine;
+        __syncthreads();
+        for (int offs = 1; offs < THREADS; offs <<= 1) {
+            uint32_t add = threadIdx.x >= offs ? sg[threadIdx.x - offs] : 0u;
+            __syncthreads();
+            sg[threadIdx.x] += add;
+            __syncthreads();
+        }
+        if (q < ntiles) {
+            s.outbase[(int64_t)row * (p.TT + 1) + first + q] = kbeg + carry_sel + sg[threadIdx.x] - mine;
+            m[3] = allowed;
+            m[2] = (ties_before + allowed == ties_wanted && allowed > 0) ? 1u : 0u;  // holds the last accepted tie
+        }
+        __syncthreads();
+        if (threadIdx.x == THREADS - 1) { carry_sel += sg[THREADS - 1]; carry_ties += st[THREADS - 1]; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0 && carry_sel != k) atomicOr(p.status, STATUS_COUNT_MISMATCH);
+}
+
+// write: ordered compaction of a tile's candidate block into the message
+__global__ void __launch_bounds__(THREADS) topk_write_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    __shared__ uint32_t wsel[8], wtie[8];
+    const int row = blockIdx.y;
+    const CandBlock cb = cand_block(p, s, blockIdx.x, row);
+    if (cb.skip || cb.cnt == 0) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t T = cb.sel[SEL_THRESH];
+    const uint32_t allowed = cb.meta[3];
+    const bool has_last = cb.meta[2] != 0u;
+    const int64_t obase = (int64_t)row * p.K + s.outbase[(int64_t)row * (p.TT + 1) + blockIdx.x];
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    uint32_t run_sel = 0, run_tie = 0;
+    for (uint32_t c0 = 0; c0 < cb.cnt; c0 += THREADS) {
+        const uint32_t q = c0 + threadIdx.x;
+        const bool in = q < cb.cnt;
+        const float val = in ? s.cand_val[cb.base + q] : 0.0f;
+        const uint32_t idx = in ? s.cand_idx[cb.base + q] : 0u;
+        const uint32_t key = key_of(val);
+        const bool tie = in && key == T;
+        const uint32_t tb = __ballot_sync(0xffffffffu, tie);
+        if (lane == 0) wtie[warp] = __popc(tb);
+        __syncthreads();
+        uint32_t tie_rank = run_tie + __popc(tb & lt_mask), tie_tot = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) { if (w < warp) tie_rank += wtie[w]; tie_tot += wtie[w]; }
+        const bool take = in && (key > T || (tie && tie_rank < allowed));
+        const uint32_t sb = __ballot_sync(0xffffffffu, take);
+        if (lane == 0) wsel[warp] = __popc(sb);
+        __syncthreads();
+        uint32_t out = run_sel + __popc(sb & lt_mask), sel_tot = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) { if (w < warp) out += wsel[w]; sel_tot += wsel[w]; }
+        if (take) {
+            s.idx[obase + out] = idx;
+            s.val[obase + out] = val;
+            if (s.zero_out) s.zero_out[idx] = 0.0f;
+            if (has_last && tie && tie_rank == allowed - 1) cb.sel[SEL_CUT] = idx;
+        }
+        run_sel += sel_tot;
+        run_tie += tie_tot;
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// slow path: one CTA per problem whose candidates did not fit.  Dense passes over the segment.
+// ------------------------------------------------------------------------------------------------
+template <typename GT>
+__global__ void __launch_bounds__(THREADS) topk_slow_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    __shared__ uint32_t bins[DIGIT1_BINS];
+    __shared__ uint32_t scratch[THREADS + 4];
+    __shared__ uint32_t wa[8], wb[8];
+    const int t = blockIdx.x, row = blockIdx.y;
+    uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
+    if (!(sel[SEL_FLAGS] & 1u)) return;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t seg_beg = __ldg(p.seg_off + t);
+    const int64_t n = __ldg(p.seg_off + t + 1) - seg_beg;
+    const GT *src = reinterpret_cast<const GT *>(s.src) + (int64_t)row * s.row_stride + seg_beg;
+    const uint32_t b1 = sel[SEL_PREFIX];
+    uint32_t rank = sel[SEL_REMAIN];
+    // second digit
+    for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) bins[b] = 0u;
+    __syncthreads();
+    for (int64_t j = threadIdx.x; j < n; j += THREADS) {
+        const uint32_t key = key_of(load1(src + j));
+        if ((key >> DIGIT1_SHIFT) == b1) atomicAdd(&bins[(key >> 7) & 0xfffu], 1u);
+    }
+    __syncthreads();
+    PickResult r = block_pick(bins, DIGIT1_BINS, rank, scratch);
+    if (!r.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
+    const uint32_t prefix24 = (b1 << 12) | r.bin;
+    rank = r.rank_in_bin;
+    // last 7 bits
+    for (int b = threadIdx.x; b < 128; b += THREADS) bins[b] = 0u;
+    __syncthreads();
+    for (int64_t j = threadIdx.x; j < n; j += THREADS) {
+        const uint32_t key = key_of(load1(src + j));
+        if ((key >> 7) == prefix24) atomicAdd(&bins[key & 0x7fu], 1u);
+    }
+    __syncthreads();
+    r = block_pick(bins, 128, rank, scratch);
+    if (!r.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
+    const uint32_t T = (prefix24 << 7) | r.bin;
+    const uint32_t ties_wanted = r.rank_in_bin;
+    if (threadIdx.x == 0) { sel[SEL_THRESH] = T; sel[SEL_TIES] = ties_wanted; }
+    // ordered compaction over the dense segment
+    const int first_tile = __ldg(p.tile_prefix + t);
+    const uint32_t kbeg = (uint32_t)__ldg(p.k_off + t), k = (uint32_t)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
+    const int64_t obase = (int64_t)row * p.K + kbeg;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    uint32_t run_sel = 0, run_tie = 0;
+    for (int64_t j0 = 0; j0 < n; j0 += THREADS) {
+        if ((j0 % TILE) == 0 && threadIdx.x == 0)
+            s.outbase[(int64_t)row * (p.TT + 1) + first_tile + (int)(j0 / TILE)] = kbeg + run_sel;
+        const int64_t j = j0 + threadIdx.x;
+        const bool in = j < n;
+        const float val = in ? load1(src + j) : 0.0f;
+        const uint32_t key = key_of(val);
+        const bool tie = in && key == T;
+        const uint32_t tb = __ballot_sync(0xffffffffu, tie);
+        if (lane == 0) wa[warp] = __popc(tb);
+        __syncthreads();
+        uint32_t tie_rank = run_tie + __popc(tb & lt_mask), tie_tot = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) { if (w < warp) tie_rank += wa[w]; tie_tot += wa[w]; }
+        const bool take = in && (key > T || (tie && tie_rank < ties_wanted));
+        const uint32_t sb = __ballot_sync(0xffffffffu, take);
+        if (lane == 0) wb[warp] = __popc(sb);
+        __syncthreads();
+        uint32_t out = run_sel + __popc(sb & lt_mask), sel_tot = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) { if (w < warp) out += wb[w]; sel_tot += wb[w]; }
+        if (take) {
+            const uint32_t flat = (uint32_t)(seg_beg + j);
+            s.idx[obase + out] = flat;
+            s.val[obase + out] = val;
+            if (tie && tie_rank == ties_wanted - 1) sel[SEL_CUT] = flat;
+        }
+        run_sel += sel_tot;
+        run_tie += tie_tot;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0 && run_sel != k) atomicOr(p.status, STATUS_COUNT_MISMATCH);
+    // downlink: selected entries of the error become +0 (after every read of the segment is done)
+    if (s.zero_out) {
+        __syncthreads();
+        for (uint32_t q = threadIdx.x; q < k; q += THREADS) s.zero_out[s.idx[obase + q]] = 0.0f;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Server pass for top-k uplink messages: one CTA per tile.
+//   acc_j = sum over workers, in worker order, of the entries that hit j (absent entries add +0)
+//   v_j   = e_j + acc_j / N   (written over e where it changes)
+// fused with the first step of the downlink: first-digit histogram (top-k) or sign words and
+// ||v||_1 partial (scaled sign).
+// ------------------------------------------------------------------------------------------------
+template <int DOWN>
+__global__ void __launch_bounds__(THREADS) server_topk_kernel(const __grid_constant__ Params p) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *acc = reinterpret_cast<float *>(smem_raw);                       // [TILE]
+    uint32_t *h = reinterpret_cast<uint32_t *>(smem_raw + sizeof(float) * TILE);  // [DIGIT1_BINS] (top-k downlink)
+    __shared__ double warp_sums[8];
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int q = threadIdx.x; q < TILE; q += THREADS) acc[q] = 0.0f;
+    if (DOWN == COMP_TOPK)
+        for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) h[b] = 0u;
+    __syncthreads();
+    const bool last_tile = (blockIdx.x + 1 == __ldg(p.tile_prefix + ti.t + 1));
+    const uint32_t tile_first = (uint32_t)(ti.seg_beg + ti.rel);
+    for (int i = 0; i < p.N; ++i) {
+        const uint32_t *ob = p.up_outbase + (int64_t)i * (p.TT + 1) + blockIdx.x;
+        const uint32_t beg = ob[0];
+        const uint32_t end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : ob[1];
+        const uint32_t *idx = p.up_idx + (int64_t)i * p.K;
+        const float *val = p.up_val + (int64_t)i * p.K;
+        for (uint32_t q = beg + threadIdx.x; q < end; q += THREADS) {
+            const uint32_t o = idx[q] - tile_first;
+            acc[o] = __fadd_rn(acc[o], val[q]);
+        }
+        __syncthreads();
+    }
+    const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
+    const float nf = (float)p.N;
+    float *e_tile = p.e + ti.seg_beg + ti.rel;
+    const int64_t wbase = __ldg(p.word_off + ti.t) + ti.rel / 32;
+    const int nwords = (ti.len + 31) >> 5;
+    double a[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pos = tile_pos(warp, lane, j);
+        float ev[4], v[4];
+        if (fast) load4_stream(e_tile + pos, ev);
+        else load4_guarded(e_tile, pos, ti.len, ev);
+        const float4 a4 = *reinterpret_cast<const float4 *>(&acc[pos]);
+        const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const bool valid = fast || pos + c < ti.len;
+            v[c] = __fadd_rn(ev[c], __fdiv_rn(av[c], nf));
+            if (!valid) v[c] = 0.0f;
+            if (valid && __float_as_uint(v[c]) != __float_as_uint(ev[c])) e_tile[pos + c] = v[c];
+            if (DOWN == COMP_TOPK && valid) atomicAdd(&h[key_of(v[c]) >> DIGIT1_SHIFT], 1u);
+        }
+        if (DOWN == COMP_SIGN) {
+            a[j] = leaf4(v);
+            uint32_t w = pack_word(sign_nibble(v), lane);
+            int widx = warp * 32 + j * 4 + (lane >> 3);
+            if ((lane & 7) == 0 && widx < nwords) p.down_words[wbase + widx] = w;
+        }
+    }
+    if (DOWN == COMP_SIGN) {
+        double sum = cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
+        if (threadIdx.x == 0) p.down_partials[blockIdx.x] = sum;
+    }
+    if (DOWN == COMP_TOPK) {
+        __syncthreads();
+        uint32_t *gh = p.down_hist + (int64_t)ti.t * DIGIT1_BINS;
+        for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) {
+            uint32_t c = h[b];
+            if (c) atomicAdd(gh + b, c);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// launchers
+// ------------------------------------------------------------------------------------------------
+#define CHECK_LAUNCH()                                   \
+    do {                                                 \
+        cudaError_t e__ = cudaGetLastError();            \
+        if (e__ != cudaSuccess) return e__;              \
+        ++*launches;                                     \
+    } while (0)
+
+cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int64_t *launches) {
+    const TopkSide s = make_side(p, uplink);
+    dim3 g_tiles(p.TT, s.R);
+    if (uplink && p.gdt == DT_BF16) topk_hist1_kernel<__nv_bfloat16><<<g_tiles, THREADS, 0, st>>>(p, s);
+    else topk_hist1_kernel<float><<<g_tiles, THREADS, 0, st>>>(p, s);
+    CHECK_LAUNCH();
+    return cudaSuccess;
+}
+
+// Everything after the first-digit histogram: the message, the thresholds, and for the
+// downlink the zeroing of the selected error entries.
+cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, int64_t *launches) {
+    const TopkSide s = make_side(p, uplink);
+    dim3 g_tiles(p.TT, s.R), g_probs(p.T, s.R);
+    const bool bf = uplink && p.gdt == DT_BF16;
+    topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 1); CHECK_LAUNCH();
+    if (bf) topk_filter_kernel<__nv_bfloat16><<<g_tiles, THREADS, 0, st>>>(p, s);
+    else topk_filter_kernel<float><<<g_tiles, THREADS, 0, st>>>(p, s);
+    CHECK_LAUNCH();
+    topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();
+    topk_hist3_kernel<<<g_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+    topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 3); CHECK_LAUNCH();
+    topk_count_kernel<<<g_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+    topk_scan_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+    topk_write_kernel<<<g_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+    if (bf) topk_slow_kernel<__nv_bfloat16><<<g_probs, THREADS, 0, st>>>(p, s);
+    else topk_slow_kernel<float><<<g_probs, THREADS, 0, st>>>(p, s);
+    CHECK_LAUNCH();
+    return cudaSuccess;
+}
+
+constexpr size_t SERVER_TOPK_SMEM = sizeof(float) * TILE + sizeof(uint32_t) * DIGIT1_BINS;
+
+cudaError_t configure_topk_kernels() {
+    cudaError_t e = cudaFuncSetAttribute(server_topk_kernel<COMP_TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)SERVER_TOPK_SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(server_topk_kernel<COMP_SIGN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)SERVER_TOPK_SMEM);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(server_topk_kernel<COMP_IDENTITY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)SERVER_TOPK_SMEM);
+}
+
+cudaError_t launch_server_topk(const Params &p, cudaStream_t st, int64_t *launches) {
+    if (p.down == COMP_TOPK) server_topk_kernel<COMP_TOPK><<<p.TT, THREADS, SERVER_TOPK_SMEM, st>>>(p);
+    else if (p.down == COMP_SIGN) server_topk_kernel<COMP_SIGN><<<p.TT, THREADS, SERVER_TOPK_SMEM, st>>>(p);
+    else server_topk_kernel<COMP_IDENTITY><<<p.TT, THREADS, SERVER_TOPK_SMEM, st>>>(p);
+    CHECK_LAUNCH();
+    return cudaSuccess;
+}
+
+}  // namespace liec

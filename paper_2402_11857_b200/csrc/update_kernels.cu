@@ -10,6 +10,7 @@ namespace liec {
 
 template <int UP, int DOWN, typename GT>
 __global__ void __launch_bounds__(THREADS) worker_update_kernel(const __grid_constant__ Params p, const float lr) {
+    __shared__ __align__(16) float p_tile[DOWN == COMP_TOPK ? TILE : 4];  // decoded downlink message (top-k)
     const int worker = blockIdx.y;
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -28,6 +29,22 @@ __global__ void __launch_bounds__(THREADS) worker_update_kernel(const __grid_con
         if (my_widx < nwords) my_word = __ldg(p.down_words + __ldg(p.word_off + ti.t) + ti.rel / 32 + my_widx);
     }
     const uint32_t su_bits = __float_as_uint(su), sd_bits = __float_as_uint(sd);
+    uint32_t up_thresh = 0u, up_cut = 0u;
+    if (UP == COMP_TOPK) {  // the worker's own selection rule: |g| above the threshold, ties up to the cut index
+        const uint32_t *sel = p.up_sel + ((int64_t)worker * p.T + ti.t) * SEL_WORDS;
+        up_thresh = sel[SEL_THRESH];
+        up_cut = sel[SEL_CUT];
+    }
+    if (DOWN == COMP_TOPK) {
+        for (int q = threadIdx.x; q < TILE; q += THREADS) p_tile[q] = 0.0f;
+        __syncthreads();
+        const bool last_tile = (blockIdx.x + 1 == __ldg(p.tile_prefix + ti.t + 1));
+        const uint32_t beg = p.down_outbase[blockIdx.x];
+        const uint32_t end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : p.down_outbase[blockIdx.x + 1];
+        const uint32_t tile_first = (uint32_t)(ti.seg_beg + ti.rel);
+        for (uint32_t q = beg + threadIdx.x; q < end; q += THREADS) p_tile[p.down_idx[q] - tile_first] = p.down_val[q];
+        __syncthreads();
+    }
     const float *v_tile = DOWN == COMP_IDENTITY ? p.vbuf + ti.seg_beg + ti.rel : nullptr;
 
     float g[8][4], x[8][4];
@@ -54,12 +71,23 @@ __global__ void __launch_bounds__(THREADS) worker_update_kernel(const __grid_con
             for (int c = 0; c < 4; ++c) pd[c] = __uint_as_float(sd_bits ^ ((nib << (31 - c)) & 0x80000000u));
         } else if (DOWN == COMP_IDENTITY) {
             load4_guarded(v_tile, pos, ti.len, pd);
+        } else {
+            const float4 q4 = *reinterpret_cast<const float4 *>(&p_tile[pos]);
+            pd[0] = q4.x; pd[1] = q4.y; pd[2] = q4.z; pd[3] = q4.w;
         }
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             float pi;
-            if (UP == COMP_SIGN) pi = __uint_as_float(su_bits ^ (g[j][c] < 0.0f ? 0x80000000u : 0u));
-            else pi = g[j][c];
+            if (UP == COMP_SIGN) {
+                pi = __uint_as_float(su_bits ^ (g[j][c] < 0.0f ? 0x80000000u : 0u));
+            } else if (UP == COMP_TOPK) {
+                const uint32_t key = __float_as_uint(g[j][c]) & 0x7fffffffu;
+                const uint32_t flat = (uint32_t)(ti.seg_beg + ti.rel) + pos + c;
+                const bool kept = key > up_thresh || (key == up_thresh && flat <= up_cut);
+                pi = kept ? g[j][c] : 0.0f;
+            } else {
+                pi = g[j][c];
+            }
             float diff = __fsub_rn(pd[c], pi);
             float u = __fadd_rn(diff, g[j][c]);
             x[j][c] = __fsub_rn(x[j][c], __fmul_rn(lr, u));
@@ -87,6 +115,11 @@ cudaError_t launch_worker_update(const Params &p, float lr, cudaStream_t st) {
     if (p.up == COMP_SIGN && p.down == COMP_IDENTITY) return launch_t<COMP_SIGN, COMP_IDENTITY>(p, lr, st);
     if (p.up == COMP_IDENTITY && p.down == COMP_SIGN) return launch_t<COMP_IDENTITY, COMP_SIGN>(p, lr, st);
     if (p.up == COMP_IDENTITY && p.down == COMP_IDENTITY) return launch_t<COMP_IDENTITY, COMP_IDENTITY>(p, lr, st);
+    if (p.up == COMP_TOPK && p.down == COMP_TOPK) return launch_t<COMP_TOPK, COMP_TOPK>(p, lr, st);
+    if (p.up == COMP_TOPK && p.down == COMP_SIGN) return launch_t<COMP_TOPK, COMP_SIGN>(p, lr, st);
+    if (p.up == COMP_TOPK && p.down == COMP_IDENTITY) return launch_t<COMP_TOPK, COMP_IDENTITY>(p, lr, st);
+    if (p.up == COMP_SIGN && p.down == COMP_TOPK) return launch_t<COMP_SIGN, COMP_TOPK>(p, lr, st);
+    if (p.up == COMP_IDENTITY && p.down == COMP_TOPK) return launch_t<COMP_IDENTITY, COMP_TOPK>(p, lr, st);
     return cudaErrorInvalidValue;
 }
 

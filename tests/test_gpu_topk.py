@@ -1,0 +1,146 @@
+"""Top-k paths of the CUDA library against the CPU oracle (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+from liec_synth import (flat_layout, make_gradients, ragged_layout, resnet50_layout, scaled_layout, topk_counts,
+                        Layout)
+from paper_2402_11857_b200 import liec
+
+pytestmark = pytest.mark.gpu
+
+SIGN, IDENT, TOPK = liec.COMP_SCALED_SIGN, liec.COMP_IDENTITY, liec.COMP_TOPK
+
+
+def _pair(*a, **kw):
+    from gpu_helpers import Pair
+    return Pair(*a, **kw)
+
+
+def test_ragged_topk_one_percent():
+    lay = ragged_layout()
+    k = topk_counts(lay, 1, 100)
+    P = _pair(3, lay.seg_offsets, TOPK, TOPK, k=k)
+    for step in range(4):
+        G = make_gradients("normal", 1.0, 3, lay.dim, step, base_seed=11)
+        P.step(G, 0.1)
+
+
+def test_k_extremes():
+    """k_t = 1 and k_t = n_t (everything kept: e' = 0 everywhere, x <- x - eta*mean-like update)."""
+    lay = ragged_layout()
+    for k in (np.ones(lay.num_segments, np.int64), np.asarray(lay.sizes, np.int64)):
+        P = _pair(2, lay.seg_offsets, TOPK, TOPK, k=k)
+        for step in range(2):
+            G = make_gradients("normal", 1.0, 2, lay.dim, step, base_seed=12)
+            P.step(G, 0.1)
+
+
+def test_heavy_ties_take_lower_index():
+    """Small-integer gradients: a handful of distinct magnitudes, so almost every selection is
+    decided by the index rule, and the groups of equal keys overflow the candidate buffer."""
+    lay = Layout("ties", (100, 5000, 3 * 8192 + 5, 40000))
+    k = np.asarray([7, 50, 245, 333], np.int64)
+    P = _pair(3, lay.seg_offsets, TOPK, TOPK, k=k)
+    g = torch.Generator().manual_seed(13)
+    for step in range(3):
+        G = torch.randint(-3, 4, (3, lay.dim), generator=g).float()
+        P.step(G, 0.25)
+
+
+def test_quantised_values_ties_at_threshold():
+    """Gaussians rounded to multiples of 1/64: ties at the threshold, candidates within the buffer."""
+    lay = Layout("quant", (30000, 8192, 70000))
+    k = topk_counts(lay, 1, 100)
+    P = _pair(4, lay.seg_offsets, TOPK, TOPK, k=k)
+    for step in range(3):
+        G = make_gradients("normal", 1.0, 4, lay.dim, step, base_seed=14)
+        G = torch.round(G * 64) / 64
+        P.step(G, 0.1)
+
+
+def test_all_zero_and_mostly_zero_gradients():
+    lay = Layout("zeros", (5000, 20000))
+    k = np.asarray([50, 200], np.int64)
+    P = _pair(2, lay.seg_offsets, TOPK, TOPK, k=k)
+    G = torch.zeros(2, lay.dim)
+    P.step(G, 0.1)
+    G[0, 17] = -2.0; G[1, 6000] = 1e-30; G[1, 24999] = -0.0
+    P.step(G, 0.1)
+    G = make_gradients("normal", 1.0, 2, lay.dim, 0, base_seed=15)
+    G[:, ::2] = 0.0           # fewer non-zeros than... no: half zero, k small: regular path
+    G[:, 5000:24000] = 0.0    # segment 1 mostly zero: threshold falls on the zeros
+    P.step(G, 0.1)
+
+
+def test_resnet50_scaled_student_t_many_steps():
+    """ResNet-50 tensor list shrunk 32x (161 segments), N=16, heavy-tailed gradients, k = 1 %."""
+    lay = scaled_layout(resnet50_layout(), 32)
+    k = topk_counts(lay, 1, 100)
+    P = _pair(16, lay.seg_offsets, TOPK, TOPK, k=k)
+    for step in range(12):
+        G = make_gradients("student_t3", 1e-3, 16, lay.dim, step, base_seed=16)
+        P.step(G, 0.1, check_messages=(step % 4 == 0))
+
+
+def test_large_single_segment_topk():
+    """One 2.36 M-element tensor (the largest ResNet conv): several hundred tiles per problem."""
+    lay = flat_layout(2359296)
+    for num, den in ((1, 100), (1, 1000)):
+        k = topk_counts(lay, num, den)
+        P = _pair(3, lay.seg_offsets, TOPK, TOPK, k=k)
+        for step in range(2):
+            G = make_gradients("student_t3", 1e-3, 3, lay.dim, step, base_seed=17)
+            P.step(G, 0.1)
+
+
+def test_bf16_topk():
+    lay = ragged_layout()
+    k = topk_counts(lay, 1, 50)
+    P = _pair(3, lay.seg_offsets, TOPK, TOPK, k=k, grad_dtype=liec.BF16)
+    for step in range(3):
+        G = make_gradients("bf16_outliers", 1e-2, 3, lay.dim, step, base_seed=18)   # bf16: many equal magnitudes
+        P.step(G, 0.01)
+
+
+@pytest.mark.parametrize("up,down", [(TOPK, SIGN), (SIGN, TOPK), (TOPK, IDENT), (IDENT, TOPK)])
+def test_mixed_compressors(up, down):
+    lay = ragged_layout()
+    k = topk_counts(lay, 1, 100)
+    P = _pair(3, lay.seg_offsets, up, down, k=k)
+    for step in range(3):
+        G = make_gradients("normal", 1.0, 3, lay.dim, step, base_seed=19)
+        P.step(G, 0.1)
+
+
+def test_unaligned_rows_topk():
+    off = [0, 5, 8192 + 5, 8192 + 5 + 33, 3 * 8192 + 1]
+    k = [1, 80, 3, 160]
+    P = _pair(3, off, TOPK, TOPK, k=k)
+    for step in range(3):
+        G = make_gradients("normal", 1.0, 3, off[-1], step, base_seed=20)
+        P.step(G, 0.1)
+
+
+def test_topk_staged_equals_step_and_deterministic():
+    lay = ragged_layout()
+    k = topk_counts(lay, 1, 100)
+    outs = []
+    for mode in ("step", "staged", "step"):
+        X = torch.zeros(4, lay.dim, device="cuda")
+        e = torch.zeros(lay.dim, device="cuda")
+        ctx = liec.Context(X, e, lay.seg_offsets, TOPK, TOPK, k)
+        for step in range(3):
+            G = make_gradients("normal", 1.0, 4, lay.dim, step, base_seed=21).cuda()
+            if mode == "step":
+                ctx.liec_step(G, 0.1)
+            else:
+                ctx.liec_uplink_compress(G); ctx.liec_server_aggregate(); ctx.liec_downlink_compress(); ctx.liec_worker_update(G, 0.1)
+        torch.cuda.synchronize()
+        assert ctx.liec_device_status() == 0
+        m = ctx.liec_get_messages()
+        outs.append((X.cpu(), e.cpu(), m["down_idx"].cpu(), m["up_idx"].cpu(), m["up_val"].cpu()))
+    for a, b in zip(outs[0], outs[1]):
+        assert torch.equal(a, b)
+    for a, b in zip(outs[0], outs[2]):
+        assert torch.equal(a, b)
