@@ -185,6 +185,23 @@ def time_oracle(w, steps: int, warmup: int):
             "seconds_per_sample_step": mean}
 
 
+# ------------------------------------------------------------------------------------ ranks
+
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of a list of floats over all ranks (identity when not distributed)."""
+    import torch
+    if not (torch.distributed.is_available() and torch.distributed.is_initialized()):
+        return list(values)
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_throughput(units_per_rank: float, world: int, ms_step_max: float) -> float:
+    """Replicas only: every rank processes units_per_rank per step; the job is as slow as its slowest rank."""
+    return units_per_rank * world / (ms_step_max * 1e-3)
+
+
 # ------------------------------------------------------------------------------------ GPU leg
 
 def run_gpu(args, w, rank, world, local_rank):
@@ -267,9 +284,7 @@ def run_gpu(args, w, rank, world, local_rank):
 
     ms_step = total_ms / args.steps
     if world > 1:
-        t = torch.tensor([ms_step, e2e["ms_per_step"] if e2e else 0.0] + stage_ms, device=dev, dtype=torch.float64)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        vals = t.tolist()
+        vals = max_over_ranks([ms_step, e2e["ms_per_step"] if e2e else 0.0] + stage_ms, device=dev)
         ms_step, e2e_max, stage_ms = vals[0], vals[1], vals[2:]
         if e2e:
             e2e["ms_per_step"] = e2e_max
@@ -325,7 +340,7 @@ def main():
         return
 
     units = N * d * world
-    value = units / (r["ms_step"] * 1e-3)
+    value = whole_job_throughput(N * d, world, r["ms_step"])
     bmin = min_bytes_per_step(w)
     step_gbs = bmin / (r["ms_step"] * 1e-3) / 1e9
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
