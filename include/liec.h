@@ -155,6 +155,34 @@ liec_status liec_device_status(liec_ctx *ctx, void *stream, int32_t *out);
 int64_t liec_launch_count(const liec_ctx *ctx);
 
 const char *liec_last_error(const liec_ctx *ctx); /* never NULL; ctx may be NULL */
+
+/*
+ * Scaled-sign compression of ONE vector with no workspace and no allocation.  (The paper has
+ * no counterpart: this is a packaging variant of the uplink compressor, same arithmetic,
+ * same words, same scale as liec_uplink_compress with one worker and one segment.)
+ *
+ * For callers that have no device memory of their own to hand over and must not ask the
+ * driver for any: a gradient hook that runs in the middle of a backward pass, where a
+ * cudaMalloc/cudaFree would stall every stream of the device, or a process whose framework
+ * allocator already owns all of the GPU's memory.  The per-tile partial sums that the
+ * regular path keeps in the caller's workspace live here in a fixed 64 KiB array inside the
+ * library image (present on every GPU that loads the library, until the process exits), which
+ * limits the vector to LIEC_NOALLOC_MAX_ELEMENTS elements; longer vectors are rejected with
+ * LIEC_ERR_UNSUPPORTED and a message.
+ *   x      device, n elements of `dtype` (liec_dtype), 16-byte aligned
+ *   words  device, ceil(n/32) uint32: bit b of word w is 1 iff x[32w+b] < 0, padding bits 0
+ *   scale  device, one float: ||x||_1 / n
+ * Enqueues two kernels on `stream`; calls no allocation routine and does not synchronise.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress);
+ * make that first call outside of any stream capture.  All calls on a GPU share the one
+ * array: calls that may overlap on the GPU (different streams, no ordering between them)
+ * race on it and must be serialised by the caller.  Nothing in it needs clearing: a call
+ * reads only the entries that it wrote itself.
+ */
+#define LIEC_NOALLOC_MAX_ELEMENTS (64ll * 1024 * 1024)
+liec_status liec_sign_compress_noalloc(const void *x, int32_t dtype, int64_t n, uint32_t *words,
+                                       float *scale, void *stream);
+const char *liec_noalloc_last_error(void); /* message of the last failing no-alloc call on this thread */
 void liec_destroy(liec_ctx *ctx);                  /* frees host memory only */
 
 #ifdef __cplusplus

@@ -1,0 +1,165 @@
+// Scaled-sign compression of one vector without any caller-provided or allocated scratch.
+//
+// The regular path keeps its per-tile partial sums in the caller's workspace.  This entry
+// point serves callers that cannot provide one: the partial sums live in a fixed array that
+// is part of the library image on every GPU that loads it (64 KiB, held until the process
+// exits).  The arithmetic is the same as in the regular uplink pass (same tree, same words).
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <mutex>
+
+#include "../../include/liec.h"
+#include "device_common.cuh"
+
+namespace liec {
+
+constexpr int64_t NOALLOC_MAX_ELEMENTS = LIEC_NOALLOC_MAX_ELEMENTS;
+constexpr int NOALLOC_MAX_TILES = (int)(NOALLOC_MAX_ELEMENTS / TILE);
+
+// One binary64 partial per tile.  Shared by every call on this GPU; it keeps the last call's
+// values, which is harmless because a call only reads the partials that it has just written.
+static __device__ __align__(256) double g_noalloc_partials[NOALLOC_MAX_TILES];
+
+template <typename GT>
+__global__ void __launch_bounds__(THREADS) sign_noalloc_kernel(const GT *x, int64_t n, uint32_t *words,
+                                                                double *partials) {
+    __shared__ double warp_sums[8];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t rel = (int64_t)blockIdx.x * TILE;
+    const int64_t left = n - rel;
+    const int len = left < TILE ? (int)left : TILE;
+    const GT *tile_ptr = x + rel;
+    const bool fast = len == TILE;  // x itself is 16-byte aligned (checked on the host)
+    float v[8][4];
+    if (fast) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) load4_stream(tile_ptr + tile_pos(warp, lane, j), v[j]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), len, v[j]);
+    }
+    uint32_t *wtile = words + rel / 32;
+    const int nwords = (len + 31) >> 5;
+    double a[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        a[j] = leaf4(v[j]);
+        uint32_t w = pack_word(sign_nibble(v[j]), lane);
+        int widx = warp * 32 + j * 4 + (lane >> 3);
+        if ((lane & 7) == 0 && widx < nwords) wtile[widx] = w;
+    }
+    double s = cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
+    if (threadIdx.x == 0) partials[blockIdx.x] = s;
+}
+
+// Single CTA: tile partials -> ||x||_1 in tree order (chunks of 2048, then the chunk sums) -> scale.
+constexpr int NA_CHUNK = 2048;
+
+__global__ void __launch_bounds__(THREADS) scale_noalloc_chunked_kernel(const double *partials, int ntiles,
+                                                                         int64_t n, float *scale) {
+    __shared__ double buf[NA_CHUNK];
+    __shared__ double chunk_sums[NOALLOC_MAX_TILES / NA_CHUNK];
+    const int nchunks = (ntiles + NA_CHUNK - 1) / NA_CHUNK;
+    for (int c = 0; c < nchunks; ++c) {
+        for (int q = threadIdx.x; q < NA_CHUNK; q += THREADS) {
+            int idx = c * NA_CHUNK + q;
+            buf[q] = idx < ntiles ? partials[idx] : 0.0;
+        }
+        __syncthreads();
+        for (int width = NA_CHUNK / 2; width >= 1; width >>= 1) {
+            double vals[NA_CHUNK / 2 / THREADS];
+#pragma unroll
+            for (int r = 0; r < NA_CHUNK / 2 / THREADS; ++r) {
+                int q = threadIdx.x + r * THREADS;
+                vals[r] = q < width ? __dadd_rn(buf[2 * q], buf[2 * q + 1]) : 0.0;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int r = 0; r < NA_CHUNK / 2 / THREADS; ++r) {
+                int q = threadIdx.x + r * THREADS;
+                if (q < width) buf[q] = vals[r];
+            }
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) chunk_sums[c] = buf[0];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        int L = 1;
+        while (L < nchunks) L <<= 1;
+        for (int c = nchunks; c < L; ++c) chunk_sums[c] = 0.0;
+        for (int width = L / 2; width >= 1; width >>= 1)
+            for (int q = 0; q < width; ++q) chunk_sums[q] = __dadd_rn(chunk_sums[2 * q], chunk_sums[2 * q + 1]);
+        *scale = __double2float_rn(__ddiv_rn(chunk_sums[0], (double)n));
+    }
+}
+
+// Device address of the scratch array, looked up once per device.  In host code the array's
+// name only stands for the symbol; kernels need the address that the runtime reports.
+static std::mutex g_noalloc_mutex;
+static double *g_noalloc_ptr[64] = {nullptr};
+
+static cudaError_t noalloc_scratch(double **out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_noalloc_partials);
+        if (e != cudaSuccess) return e;
+        g_noalloc_ptr[dev] = static_cast<double *>(ptr);
+    }
+    *out = g_noalloc_ptr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace liec
+
+static thread_local char g_noalloc_error[256] = "";
+
+extern "C" const char *liec_noalloc_last_error(void) { return g_noalloc_error; }
+
+extern "C" liec_status liec_sign_compress_noalloc(const void *x, int32_t dtype, int64_t n, uint32_t *words,
+                                                  float *scale, void *stream) {
+    using namespace liec;
+    auto bail = [](liec_status st, const char *text) {
+        snprintf(g_noalloc_error, sizeof(g_noalloc_error), "%s", text);
+        return st;
+    };
+    if (!x || !words || !scale) return bail(LIEC_ERR_INVALID_ARG, "x, words and scale must be non-NULL");
+    if (reinterpret_cast<uintptr_t>(x) & 15u) return bail(LIEC_ERR_INVALID_ARG, "x must be 16-byte aligned");
+    if (dtype != LIEC_F32 && dtype != LIEC_BF16) return bail(LIEC_ERR_INVALID_ARG, "unknown dtype");
+    if (n < 1) return bail(LIEC_ERR_INVALID_ARG, "n must be >= 1");
+    if (n > NOALLOC_MAX_ELEMENTS) {
+        snprintf(g_noalloc_error, sizeof(g_noalloc_error),
+                 "n = %lld exceeds LIEC_NOALLOC_MAX_ELEMENTS = %lld (fixed built-in scratch); use liec_uplink_compress",
+                 (long long)n, (long long)NOALLOC_MAX_ELEMENTS);
+        return LIEC_ERR_UNSUPPORTED;
+    }
+    double *partials = nullptr;
+    cudaError_t e = noalloc_scratch(&partials);
+    if (e != cudaSuccess) {
+        snprintf(g_noalloc_error, sizeof(g_noalloc_error), "cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+        return LIEC_ERR_CUDA;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int ntiles = (int)((n + TILE - 1) / TILE);
+    if (dtype == LIEC_F32)
+        sign_noalloc_kernel<float><<<ntiles, THREADS, 0, st>>>(static_cast<const float *>(x), n, words, partials);
+    else
+        sign_noalloc_kernel<__nv_bfloat16><<<ntiles, THREADS, 0, st>>>(static_cast<const __nv_bfloat16 *>(x), n, words, partials);
+    e = cudaGetLastError();
+    if (e == cudaSuccess) {
+        scale_noalloc_chunked_kernel<<<1, THREADS, 0, st>>>(partials, ntiles, n, scale);
+        e = cudaGetLastError();
+    }
+    if (e != cudaSuccess) {
+        snprintf(g_noalloc_error, sizeof(g_noalloc_error), "kernel launch failed: %s", cudaGetErrorString(e));
+        return LIEC_ERR_CUDA;
+    }
+    return LIEC_OK;
+}

@@ -78,6 +78,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.liec_last_error.restype = C.c_char_p
     lib.liec_destroy.argtypes = [vp]
     lib.liec_destroy.restype = None
+    lib.liec_sign_compress_noalloc.argtypes = [vp, C.c_int32, C.c_int64, vp, vp, vp]
+    lib.liec_sign_compress_noalloc.restype = C.c_int
+    lib.liec_noalloc_last_error.argtypes = []
+    lib.liec_noalloc_last_error.restype = C.c_char_p
     if path is None:
         _LIB = lib
     return lib
@@ -105,6 +109,22 @@ def workspace_bytes(cfg: liec_config) -> int:
 
 def down_message_bytes(cfg: liec_config) -> int:
     return int(load_library().liec_down_message_bytes(C.byref(cfg)))
+
+
+NOALLOC_MAX_ELEMENTS = 64 * 1024 * 1024
+
+
+def liec_sign_compress_noalloc(x, words, scale, stream=None):
+    """Scaled sign of one CUDA vector into caller-provided `words` (int32, ceil(n/32)) and `scale`
+    (float32, 1 element) without any workspace or allocation; see liec.h for who needs this."""
+    import torch
+    lib = load_library()
+    dtype = BF16 if x.dtype == torch.bfloat16 else F32
+    s = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
+    with torch.cuda.device(x.device):
+        st = lib.liec_sign_compress_noalloc(x.data_ptr(), dtype, x.numel(), words.data_ptr(), scale.data_ptr(), s)
+    if st != 0:
+        raise LiecError(st, lib.liec_noalloc_last_error().decode())
 
 
 class Context:
