@@ -17,18 +17,13 @@ struct TileInfo {
     int tile_in_seg;  // tile index inside the segment
 };
 
-// Segment owning tile `tile`: largest t with tile_prefix[t] <= tile.
+// Segment and extent of tile `tile` (table lookups only).
 __device__ __forceinline__ TileInfo locate_tile(const Params &p, int tile) {
-    int lo = 0, hi = p.T;  // invariant: prefix[lo] <= tile < prefix[hi]
-    while (hi - lo > 1) {
-        int mid = (lo + hi) >> 1;
-        if (__ldg(p.tile_prefix + mid) <= tile) lo = mid; else hi = mid;
-    }
     TileInfo ti;
-    ti.t = lo;
-    ti.seg_beg = __ldg(p.seg_off + lo);
-    ti.n = __ldg(p.seg_off + lo + 1) - ti.seg_beg;
-    ti.tile_in_seg = tile - __ldg(p.tile_prefix + lo);
+    ti.t = __ldg(p.tile_seg + tile);
+    ti.seg_beg = __ldg(p.seg_off + ti.t);
+    ti.n = __ldg(p.seg_off + ti.t + 1) - ti.seg_beg;
+    ti.tile_in_seg = tile - __ldg(p.tile_prefix + ti.t);
     ti.rel = (int64_t)ti.tile_in_seg * TILE;
     int64_t left = ti.n - ti.rel;
     ti.len = left < TILE ? (int)left : TILE;
@@ -80,14 +75,16 @@ __device__ __forceinline__ double shfl_xor_f64(double x, int mask) {
     return __shfl_xor_sync(0xffffffffu, x, mask);
 }
 
-// a[j] = this lane's leaf sum in row j.  Returns, in every lane, the tree sum of the warp's
-// 1024 elements.
-__device__ __forceinline__ double warp_tree_reduce8(double (&a)[8], int lane) {
-    // lane levels 1,2,4 while folding 8 rows -> 1 value per lane
+// a[j] = this lane's leaf sum in row j (ROWS rows per warp, ROWS = 8 or 4).  Returns, in every
+// lane, the tree sum of the warp's 1024 elements.
+template <int ROWS>
+__device__ __forceinline__ double warp_tree_reduce(double (&a)[ROWS], int lane) {
+    constexpr int LOG = ROWS == 8 ? 3 : 2;
+    // lane levels 1,2,(4) while folding ROWS rows -> 1 value per lane
 #pragma unroll
-    for (int step = 0; step < 3; ++step) {
+    for (int step = 0; step < LOG; ++step) {
         const int m = 1 << step;
-        const int half = 4 >> step;
+        const int half = (ROWS / 2) >> step;
         const bool upper = (lane & m) != 0;
 #pragma unroll
         for (int r = 0; r < half; ++r) {
@@ -99,14 +96,15 @@ __device__ __forceinline__ double warp_tree_reduce8(double (&a)[8], int lane) {
     }
     double s = a[0];
     // remaining lane levels of the row this lane now represents
-    s = __dadd_rn(s, shfl_xor_f64(s, 8));
-    s = __dadd_rn(s, shfl_xor_f64(s, 16));
-    // row levels: row bit 0 lives in lane bit 2, row bit 1 in lane bit 1, row bit 2 in lane bit 0
-    s = __dadd_rn(s, shfl_xor_f64(s, 4));
-    s = __dadd_rn(s, shfl_xor_f64(s, 2));
-    s = __dadd_rn(s, shfl_xor_f64(s, 1));
+#pragma unroll
+    for (int m = ROWS; m < 32; m <<= 1) s = __dadd_rn(s, shfl_xor_f64(s, m));
+    // row levels: row bit b lives in lane bit LOG-1-b
+#pragma unroll
+    for (int m = ROWS / 2; m >= 1; m >>= 1) s = __dadd_rn(s, shfl_xor_f64(s, m));
     return s;
 }
+
+__device__ __forceinline__ double warp_tree_reduce8(double (&a)[8], int lane) { return warp_tree_reduce<8>(a, lane); }
 
 // Combine the 8 warp sums of a CTA (tile of 8192 elements) in tree order; result in thread 0.
 __device__ __forceinline__ double cta_tree_reduce(double warp_sum, double *smem8) {

@@ -26,8 +26,8 @@ struct Plan {
     int32_t N = 0, T = 0, TT = 0;
     int64_t d = 0, W = 0, K = 0, CAP = 0;
     std::vector<int64_t> seg_off, word_off, k_off, cap_off, topk_k;
-    std::vector<int32_t> tile_prefix;
-    Region r_seg_off, r_word_off, r_k_off, r_cap_off, r_tile_prefix, r_status;
+    std::vector<int32_t> tile_prefix, tile_seg;
+    Region r_seg_off, r_word_off, r_k_off, r_cap_off, r_tile_prefix, r_tile_seg, r_status;
     Region r_up_words, r_up_scales, r_up_partials, r_down_words, r_down_scales, r_down_partials, r_vbuf;
     Region r_up_idx, r_up_val, r_down_idx, r_down_val;
     Region r_up_hist, r_down_hist, r_up_hist2, r_down_hist2, r_up_sel, r_down_sel;
@@ -112,6 +112,9 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     pl.K = pl.k_off[T];
     pl.CAP = pl.cap_off[T];
     pl.TT = (int32_t)tiles;
+    pl.tile_seg.resize(pl.TT);
+    for (int t = 0; t < T; ++t)
+        for (int q = pl.tile_prefix[t]; q < pl.tile_prefix[t + 1]; ++q) pl.tile_seg[q] = t;
 
     Carver c;
     pl.r_seg_off = c.take(sizeof(int64_t) * (T + 1));
@@ -119,6 +122,7 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     pl.r_k_off = c.take(sizeof(int64_t) * (T + 1));
     pl.r_cap_off = c.take(sizeof(int64_t) * (T + 1));
     pl.r_tile_prefix = c.take(sizeof(int32_t) * (T + 1));
+    pl.r_tile_seg = c.take(sizeof(int32_t) * pl.TT);
     pl.r_status = c.take(256);
     const size_t N = pl.N;
     if (cfg->uplink == LIEC_COMP_SCALED_SIGN) {
@@ -248,6 +252,7 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     p.k_off = at<int64_t>(c, pl.r_k_off);
     p.cap_off = at<int64_t>(c, pl.r_cap_off);
     p.tile_prefix = at<int32_t>(c, pl.r_tile_prefix);
+    p.tile_seg = at<int32_t>(c, pl.r_tile_seg);
     p.status = at<int32_t>(c, pl.r_status);
     p.X = params;
     p.e = error;
@@ -272,6 +277,7 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     const Up ups[] = {
         {&pl.r_seg_off, pl.seg_off.data()}, {&pl.r_word_off, pl.word_off.data()}, {&pl.r_k_off, pl.k_off.data()},
         {&pl.r_cap_off, pl.cap_off.data()}, {&pl.r_tile_prefix, pl.tile_prefix.data()},
+        {&pl.r_tile_seg, pl.tile_seg.data()},
     };
     for (const Up &u : ups) {
         cudaError_t e = cudaMemcpy(c->ws + u.r->off, u.src, u.r->bytes, cudaMemcpyHostToDevice);

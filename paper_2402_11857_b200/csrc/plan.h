@@ -32,6 +32,7 @@ struct Params {
     const int64_t *k_off;        // [T+1] (top-k only)
     const int64_t *cap_off;      // [T+1] candidate capacity prefix (top-k only)
     const int32_t *tile_prefix;  // [T+1] tiles before segment t
+    const int32_t *tile_seg;     // [TT] segment of every tile
 
     // state
     float *X;         // [N][d]

@@ -46,6 +46,65 @@ __global__ void __launch_bounds__(THREADS) sign_uplink_kernel(const __grid_const
     if (threadIdx.x == 0) p.up_partials[(int64_t)worker * p.TT + blockIdx.x] = s;
 }
 
+// bfloat16 gradients: the same tile, read with 128-bit loads.  A warp owns its 1024 elements as
+// 4 rows of 256; lane l owns elements 8l..8l+7 of a row (three tree levels in-thread), four
+// lanes share a 32-bit sign word.  Half the load, shuffle and store instructions per element
+// of the 4-wide version, which matters because this pass is instruction-bound on bf16 input.
+__global__ void __launch_bounds__(THREADS) sign_uplink_bf16_kernel(const __grid_constant__ Params p) {
+    __shared__ double warp_sums[8];
+    const int worker = blockIdx.y;
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t row_beg = (int64_t)worker * p.d + ti.seg_beg;
+    const __nv_bfloat16 *tile_ptr = reinterpret_cast<const __nv_bfloat16 *>(p.G) + row_beg + ti.rel;
+    const bool fast = (ti.len == TILE) && ((row_beg & 7) == 0);
+
+    float v[4][8];
+    if (fast) {
+        uint4 q[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            q[j] = __ldcs(reinterpret_cast<const uint4 *>(tile_ptr + warp * 1024 + j * 256 + lane * 8));
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            v[j][0] = __uint_as_float(q[j].x << 16); v[j][1] = __uint_as_float(q[j].x & 0xffff0000u);
+            v[j][2] = __uint_as_float(q[j].y << 16); v[j][3] = __uint_as_float(q[j].y & 0xffff0000u);
+            v[j][4] = __uint_as_float(q[j].z << 16); v[j][5] = __uint_as_float(q[j].z & 0xffff0000u);
+            v[j][6] = __uint_as_float(q[j].w << 16); v[j][7] = __uint_as_float(q[j].w & 0xffff0000u);
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int pos = warp * 1024 + j * 256 + lane * 8;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) v[j][c] = (pos + c < ti.len) ? load1(tile_ptr + pos + c) : 0.0f;
+        }
+    }
+
+    uint32_t *words = p.up_words + (int64_t)worker * p.W + __ldg(p.word_off + ti.t) + ti.rel / 32;
+    const int nwords = (ti.len + 31) >> 5;
+    double a[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        double d[8];
+        uint32_t byte = 0;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            d[c] = (double)fabsf(v[j][c]);
+            if (v[j][c] < 0.0f) byte |= 1u << c;
+        }
+        a[j] = __dadd_rn(__dadd_rn(__dadd_rn(d[0], d[1]), __dadd_rn(d[2], d[3])),
+                         __dadd_rn(__dadd_rn(d[4], d[5]), __dadd_rn(d[6], d[7])));
+        uint32_t w = byte << (8 * (lane & 3));
+        w |= __shfl_xor_sync(0xffffffffu, w, 1);
+        w |= __shfl_xor_sync(0xffffffffu, w, 2);
+        const int widx = warp * 32 + j * 8 + (lane >> 2);
+        if ((lane & 3) == 0 && widx < nwords) words[widx] = w;
+    }
+    double s = cta_tree_reduce(warp_tree_reduce<4>(a, lane), warp_sums);
+    if (threadIdx.x == 0) p.up_partials[(int64_t)worker * p.TT + blockIdx.x] = s;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Scale: one CTA per (segment, row).  Tile partials are combined pairwise, level by level,
 // over the tile count zero-padded to a power of two (adding +0 is exact), which continues the
@@ -189,6 +248,82 @@ __global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_cons
     }
 }
 
+// Sign uplink, one thread per 32-bit word: thread q of the CTA owns elements 32q..32q+31 of the
+// tile, i.e. exactly one word of every worker's message, so unpacking needs no shuffles
+// (shift + sign-xor + add per element and worker), the word of v is built in-thread and the
+// ||v||_1 leaf covers five tree levels in-thread.
+template <bool DOWN_SIGN>
+__global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_constant__ Params p) {
+    __shared__ double warp_sums[8];
+    extern __shared__ float up_scale_smem[];  // [N] scales of this segment
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const int lane = threadIdx.x & 31;
+    const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
+    const int64_t wbase = __ldg(p.word_off + ti.t) + ti.rel / 32;
+    const int nwords = (ti.len + 31) >> 5;
+    const int my_widx = threadIdx.x;
+    const bool have_word = my_widx < nwords;
+    for (int i = threadIdx.x; i < p.N; i += THREADS) up_scale_smem[i] = p.up_scales[(int64_t)i * p.T + ti.t];
+    __syncthreads();
+
+    float acc[32];
+#pragma unroll
+    for (int c = 0; c < 32; ++c) acc[c] = 0.0f;
+    const uint32_t *wp = p.up_words + wbase + my_widx;
+    uint32_t next = have_word ? __ldg(wp) : 0u;
+    for (int i = 0; i < p.N; ++i) {
+        const uint32_t w = next;
+        if (i + 1 < p.N && have_word) next = __ldg(wp + (int64_t)(i + 1) * p.W);
+        const uint32_t sbits = __float_as_uint(up_scale_smem[i]);
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+            const float pij = __uint_as_float(sbits ^ ((w << (31 - c)) & 0x80000000u));
+            acc[c] = __fadd_rn(acc[c], pij);
+        }
+    }
+
+    const float nf = (float)p.N;
+    const int pos0 = 32 * threadIdx.x;
+    float *e_tile = p.e + ti.seg_beg + ti.rel;
+    uint32_t vword = 0u;
+    double leaf[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int pos = pos0 + 4 * k;
+        float ev[4], v[4];
+        if (fast) {
+            const float4 q = *reinterpret_cast<const float4 *>(e_tile + pos);
+            ev[0] = q.x; ev[1] = q.y; ev[2] = q.z; ev[3] = q.w;
+        } else {
+            load4_guarded(e_tile, pos, ti.len, ev);
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c) v[c] = __fadd_rn(ev[c], __fdiv_rn(acc[4 * k + c], nf));
+        if (fast) {
+            *reinterpret_cast<float4 *>(e_tile + pos) = make_float4(v[0], v[1], v[2], v[3]);
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                if (pos + c < ti.len) e_tile[pos + c] = v[c]; else v[c] = 0.0f;
+            }
+        }
+        if (DOWN_SIGN) {
+            leaf[k] = leaf4(v);
+            vword |= sign_nibble(v) << (4 * k);
+        }
+    }
+    if (DOWN_SIGN) {
+        if (have_word) p.down_words[wbase + my_widx] = vword;
+        double s = __dadd_rn(__dadd_rn(__dadd_rn(leaf[0], leaf[1]), __dadd_rn(leaf[2], leaf[3])),
+                             __dadd_rn(__dadd_rn(leaf[4], leaf[5]), __dadd_rn(leaf[6], leaf[7])));
+#pragma unroll
+        for (int m = 1; m < 32; m <<= 1) s = __dadd_rn(s, shfl_xor_f64(s, m));
+        s = cta_tree_reduce(s, warp_sums);
+        if (threadIdx.x == 0) p.down_partials[blockIdx.x] = s;
+    }
+    (void)lane;
+}
+
 // First half of a sign downlink on a v that is already in the error buffer (used when the
 // aggregation kernel could not fuse it, i.e. after a top-k uplink).
 __global__ void __launch_bounds__(THREADS) sign_downlink_kernel(const __grid_constant__ Params p) {
@@ -266,7 +401,7 @@ __global__ void __launch_bounds__(THREADS) identity_downlink_kernel(const __grid
 cudaError_t launch_sign_uplink(const Params &p, cudaStream_t st) {
     dim3 grid(p.TT, p.N);
     if (p.gdt == DT_F32) sign_uplink_kernel<float><<<grid, THREADS, 0, st>>>(p);
-    else sign_uplink_kernel<__nv_bfloat16><<<grid, THREADS, 0, st>>>(p);
+    else sign_uplink_bf16_kernel<<<grid, THREADS, 0, st>>>(p);
     return cudaGetLastError();
 }
 
@@ -286,7 +421,12 @@ static cudaError_t launch_server_dense_t(const Params &p, cudaStream_t st) {
 }
 
 cudaError_t launch_server_dense(const Params &p, cudaStream_t st) {
-    if (p.up == COMP_SIGN) return launch_server_dense_t<COMP_SIGN, float>(p, st);
+    if (p.up == COMP_SIGN) {
+        const size_t smem = sizeof(float) * (size_t)p.N;
+        if (p.down == COMP_SIGN) server_sign_kernel<true><<<p.TT, THREADS, smem, st>>>(p);
+        else server_sign_kernel<false><<<p.TT, THREADS, smem, st>>>(p);
+        return cudaGetLastError();
+    }
     if (p.gdt == DT_F32) return launch_server_dense_t<COMP_IDENTITY, float>(p, st);
     return launch_server_dense_t<COMP_IDENTITY, __nv_bfloat16>(p, st);
 }
