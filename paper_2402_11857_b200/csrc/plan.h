@@ -64,14 +64,15 @@ struct Params {
 };
 
 // per-problem selection state words
-constexpr int SEL_WORDS = 8;
+constexpr int SEL_WORDS = 12;
 constexpr int SEL_PREFIX = 0;     // key prefix fixed so far (aligned to its bit position)
 constexpr int SEL_REMAIN = 1;     // rank still to find inside the prefix bin (1-based)
 constexpr int SEL_CAND_COUNT = 2; // atomic cursor: candidates appended so far
 constexpr int SEL_THRESH = 3;     // final threshold key T
 constexpr int SEL_TIES = 4;       // number of entries equal to T to accept, lowest index first
 constexpr int SEL_CUT = 5;        // flat index of the last accepted tie
-constexpr int SEL_FLAGS = 6;      // bit0: candidate buffer overflow -> slow path
-constexpr int SEL_NCAND = 7;      // exact number of candidates (elements with digit1 >= bin1)
+constexpr int SEL_FLAGS = 6;      // bit0: slow path (one CTA, dense passes); bit1: refined (24-bit prefix found by a dense second-digit pass)
+constexpr int SEL_NCAND = 7;      // exact number of candidates (entries at or above the prefix)
+constexpr int SEL_ABOVE = 8;      // entries whose first digit is strictly above the threshold's
 
 }  // namespace liec

@@ -149,16 +149,34 @@ __global__ void __launch_bounds__(THREADS) topk_hist1_kernel(const __grid_consta
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constant__ Params p, const TopkSide s,
                                                              const int level) {
-    __shared__ uint32_t bins[DIGIT1_BINS];
+    __shared__ __align__(16) uint32_t bins[DIGIT1_BINS];
     __shared__ uint32_t scratch[THREADS + 4];
     const int t = blockIdx.x, row = blockIdx.y;
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
-    if (level > 1 && (sel[SEL_FLAGS] & 1u)) return;  // handled by the slow path
+    // level 1: first digit.  level 4: second digit of "refined" problems (after their dense
+    // second-digit pass).  level 2: second digit of regular problems.  level 3: last 7 bits.
+    const uint32_t flags_in = level == 1 ? 0u : sel[SEL_FLAGS];
+    if (level == 4 && flags_in != 2u) return;
+    if (level == 2 && flags_in != 0u) return;
+    if (level == 3 && (flags_in & 1u)) return;  // slow path finishes on its own
     const int nbins = level == 3 ? 128 : DIGIT1_BINS;
     uint32_t *gh = (level == 1 ? s.hist : s.hist2) + ((int64_t)row * p.T + t) * DIGIT1_BINS;
-    for (int b = threadIdx.x; b < nbins; b += THREADS) {
-        bins[b] = gh[b];
-        gh[b] = 0u;
+    if (nbins == DIGIT1_BINS) {
+        // 4 independent 128-bit loads per thread, then the clears
+        uint4 tmp[DIGIT1_BINS / 4 / THREADS];
+        uint4 *gh4 = reinterpret_cast<uint4 *>(gh);
+#pragma unroll
+        for (int q = 0; q < DIGIT1_BINS / 4 / THREADS; ++q) tmp[q] = gh4[threadIdx.x + q * THREADS];
+#pragma unroll
+        for (int q = 0; q < DIGIT1_BINS / 4 / THREADS; ++q) {
+            reinterpret_cast<uint4 *>(bins)[threadIdx.x + q * THREADS] = tmp[q];
+            if (tmp[q].x | tmp[q].y | tmp[q].z | tmp[q].w) gh4[threadIdx.x + q * THREADS] = make_uint4(0u, 0u, 0u, 0u);
+        }
+    } else {
+        for (int b = threadIdx.x; b < nbins; b += THREADS) {
+            bins[b] = gh[b];
+            gh[b] = 0u;
+        }
     }
     __syncthreads();
     const uint32_t k = (uint32_t)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
@@ -166,13 +184,21 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
     const PickResult r = block_pick(bins, nbins, rank, scratch);
     if (threadIdx.x == 0) {
         if (!r.ok) { atomicOr(p.status, STATUS_PICK_RANK); return; }
+        const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
         if (level == 1) {
-            const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
             sel[SEL_PREFIX] = r.bin;
             sel[SEL_REMAIN] = r.rank_in_bin;
             sel[SEL_NCAND] = r.count_ge;
+            sel[SEL_ABOVE] = r.count_ge - bins[r.bin];
             sel[SEL_CAND_COUNT] = 0u;
-            sel[SEL_FLAGS] = r.count_ge > cap ? 1u : 0u;
+            // too many entries share the threshold's first digit: look at the second digit first
+            sel[SEL_FLAGS] = r.count_ge > cap ? 2u : 0u;
+        } else if (level == 4) {
+            const uint32_t ncand = sel[SEL_ABOVE] + r.count_ge;
+            sel[SEL_PREFIX] = (sel[SEL_PREFIX] << 12) | r.bin;
+            sel[SEL_REMAIN] = r.rank_in_bin;
+            sel[SEL_NCAND] = ncand;
+            if (ncand > cap) sel[SEL_FLAGS] = 3u;  // still too many (huge groups of equal keys): slow path
         } else if (level == 2) {
             sel[SEL_PREFIX] = (sel[SEL_PREFIX] << 12) | r.bin;
             sel[SEL_REMAIN] = r.rank_in_bin;
@@ -183,18 +209,58 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
     }
 }
 
+// Dense second-digit pass for refined problems only: histogram of key bits 18..7 over the
+// entries whose first digit equals the threshold's.  One CTA per (tile, row).
+template <typename GT>
+__global__ void __launch_bounds__(THREADS) topk_hist2_dense_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    __shared__ uint32_t h[DIGIT1_BINS];
+    const int row = blockIdx.y;
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
+    if (sel[SEL_FLAGS] != 2u) return;
+    const uint32_t b1 = sel[SEL_PREFIX];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) h[b] = 0u;
+    __syncthreads();
+    const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
+    const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
+    const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pos = tile_pos(warp, lane, j);
+        float v[4];
+        if (fast) load4_stream(tile_ptr + pos, v);
+        else load4_guarded(tile_ptr, pos, ti.len, v);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint32_t key = key_of(v[c]);
+            if ((fast || pos + c < ti.len) && (key >> DIGIT1_SHIFT) == b1) atomicAdd(&h[(key >> 7) & 0xfffu], 1u);
+        }
+    }
+    __syncthreads();
+    uint32_t *gh = s.hist2 + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS;
+    for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) {
+        uint32_t c = h[b];
+        if (c) atomicAdd(gh + b, c);
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // filter: one CTA per (tile, row); ordered append of candidates
 // ------------------------------------------------------------------------------------------------
 template <typename GT>
-__global__ void __launch_bounds__(THREADS) topk_filter_kernel(const __grid_constant__ Params p, const TopkSide s) {
+__global__ void __launch_bounds__(THREADS, 3) topk_filter_kernel(const __grid_constant__ Params p, const TopkSide s) {
     __shared__ uint32_t warp_tot[8];
     __shared__ uint32_t tile_base;
     const int row = blockIdx.y;
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
-    if (sel[SEL_FLAGS] & 1u) return;
+    const uint32_t flags = sel[SEL_FLAGS];
+    if (flags & 1u) return;
+    // regular problems compare the first digit; refined ones the 24-bit prefix
+    const bool refined = flags == 2u;
+    const int cmp_shift = refined ? 7 : DIGIT1_SHIFT;
     const uint32_t b1 = sel[SEL_PREFIX];
     const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
     const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
@@ -208,26 +274,41 @@ __global__ void __launch_bounds__(THREADS) topk_filter_kernel(const __grid_const
         for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v[j]);
     }
     uint32_t *gh2 = s.hist2 + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS;
-    const uint32_t lt_mask = (1u << lane) - 1u;
+    // candidate flags: one nibble per row; counts of rows 0-3 and 4-7 packed as bytes of two words
     uint32_t nib[8], rowoff[8];
-    uint32_t running = 0;  // candidates of this warp before the current row
+    uint32_t cnt_lo = 0, cnt_hi = 0;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int pos = tile_pos(warp, lane, j);
-        uint32_t f = 0, before = 0, total = 0;
+        uint32_t f = 0;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             const uint32_t key = key_of(v[j][c]);
-            const uint32_t d1 = key >> DIGIT1_SHIFT;
+            const uint32_t d1 = key >> cmp_shift;
             const bool valid = fast || pos + c < ti.len;
-            const bool cand = valid && d1 >= b1;
-            if (valid && d1 == b1) atomicAdd(gh2 + ((key >> 7) & 0xfffu), 1u);
-            const uint32_t bal = __ballot_sync(0xffffffffu, cand);
-            before += __popc(bal & lt_mask);
-            total += __popc(bal);
-            f |= cand ? (1u << c) : 0u;
+            if (valid && d1 >= b1) {
+                f |= 1u << c;
+                if (!refined && d1 == b1) atomicAdd(gh2 + ((key >> 7) & 0xfffu), 1u);
+            }
         }
         nib[j] = f;
+        if (j < 4) cnt_lo |= (uint32_t)__popc(f) << (8 * j);
+        else cnt_hi |= (uint32_t)__popc(f) << (8 * (j - 4));
+    }
+    // inclusive scan over lanes of the packed per-row counts (a row holds at most 128 < 256)
+    uint32_t inc_lo = cnt_lo, inc_hi = cnt_hi;
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const uint32_t a = __shfl_up_sync(0xffffffffu, inc_lo, m), b = __shfl_up_sync(0xffffffffu, inc_hi, m);
+        if (lane >= m) { inc_lo += a; inc_hi += b; }
+    }
+    const uint32_t tot_lo = __shfl_sync(0xffffffffu, inc_lo, 31), tot_hi = __shfl_sync(0xffffffffu, inc_hi, 31);
+    const uint32_t exc_lo = inc_lo - cnt_lo, exc_hi = inc_hi - cnt_hi;
+    uint32_t running = 0;  // candidates of this warp before the current row
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint32_t before = ((j < 4 ? exc_lo : exc_hi) >> (8 * (j & 3))) & 0xffu;
+        const uint32_t total = ((j < 4 ? tot_lo : tot_hi) >> (8 * (j & 3))) & 0xffu;
         rowoff[j] = running + before;
         running += total;
     }
@@ -283,37 +364,38 @@ __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide 
     return cb;
 }
 
+// The candidate passes give one warp to every tile block (8 tiles per CTA): blocks are small
+// (about 1.4 % of a tile) and warps need no block-wide synchronisation.
 __global__ void __launch_bounds__(THREADS) topk_hist3_kernel(const __grid_constant__ Params p, const TopkSide s) {
-    const int row = blockIdx.y;
-    const CandBlock cb = cand_block(p, s, blockIdx.x, row);
+    const int row = blockIdx.y, lane = threadIdx.x & 31;
+    const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (tile >= p.TT) return;
+    const CandBlock cb = cand_block(p, s, tile, row);
     if (cb.skip) return;
     const uint32_t prefix24 = cb.sel[SEL_PREFIX];
     uint32_t *gh = s.hist2 + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
-    for (uint32_t q = threadIdx.x; q < cb.cnt; q += THREADS) {
+    for (uint32_t q = lane; q < cb.cnt; q += 32) {
         const uint32_t key = key_of(s.cand_val[cb.base + q]);
         if ((key >> 7) == prefix24) atomicAdd(gh + (key & 0x7fu), 1u);
     }
 }
 
 __global__ void __launch_bounds__(THREADS) topk_count_kernel(const __grid_constant__ Params p, const TopkSide s) {
-    __shared__ uint32_t cnt_g, cnt_t;
-    const int row = blockIdx.y;
-    const CandBlock cb = cand_block(p, s, blockIdx.x, row);
+    const int row = blockIdx.y, lane = threadIdx.x & 31;
+    const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (tile >= p.TT) return;
+    const CandBlock cb = cand_block(p, s, tile, row);
     if (cb.skip) return;
-    if (threadIdx.x == 0) { cnt_g = 0u; cnt_t = 0u; }
-    __syncthreads();
     const uint32_t T = cb.sel[SEL_THRESH];
     uint32_t g = 0, e = 0;
-    for (uint32_t q = threadIdx.x; q < cb.cnt; q += THREADS) {
+    for (uint32_t q = lane; q < cb.cnt; q += 32) {
         const uint32_t key = key_of(s.cand_val[cb.base + q]);
         g += key > T ? 1u : 0u;
         e += key == T ? 1u : 0u;
     }
     g = __reduce_add_sync(0xffffffffu, g);
     e = __reduce_add_sync(0xffffffffu, e);
-    if ((threadIdx.x & 31) == 0) { if (g) atomicAdd(&cnt_g, g); if (e) atomicAdd(&cnt_t, e); }
-    __syncthreads();
-    if (threadIdx.x == 0) { cb.meta[2] = cnt_g; cb.meta[3] = cnt_t; }
+    if (lane == 0) { cb.meta[2] = g; cb.meta[3] = e; }
 }
 
 // scan: one CTA per (segment, row); tiles of the segment in order
@@ -365,48 +447,39 @@ __global__ void __launch_bounds__(THREADS) topk_scan_kernel(const __grid_constan
     if (threadIdx.x == 0 && carry_sel != k) atomicOr(p.status, STATUS_COUNT_MISMATCH);
 }
 
-// write: ordered compaction of a tile's candidate block into the message
+// write: ordered compaction of a tile's candidate block into the message (one warp per tile)
 __global__ void __launch_bounds__(THREADS) topk_write_kernel(const __grid_constant__ Params p, const TopkSide s) {
-    __shared__ uint32_t wsel[8], wtie[8];
-    const int row = blockIdx.y;
-    const CandBlock cb = cand_block(p, s, blockIdx.x, row);
+    const int row = blockIdx.y, lane = threadIdx.x & 31;
+    const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (tile >= p.TT) return;
+    const CandBlock cb = cand_block(p, s, tile, row);
     if (cb.skip || cb.cnt == 0) return;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t T = cb.sel[SEL_THRESH];
     const uint32_t allowed = cb.meta[3];
     const bool has_last = cb.meta[2] != 0u;
-    const int64_t obase = (int64_t)row * p.K + s.outbase[(int64_t)row * (p.TT + 1) + blockIdx.x];
+    const int64_t obase = (int64_t)row * p.K + s.outbase[(int64_t)row * (p.TT + 1) + tile];
     const uint32_t lt_mask = (1u << lane) - 1u;
     uint32_t run_sel = 0, run_tie = 0;
-    for (uint32_t c0 = 0; c0 < cb.cnt; c0 += THREADS) {
-        const uint32_t q = c0 + threadIdx.x;
+    for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
+        const uint32_t q = c0 + lane;
         const bool in = q < cb.cnt;
         const float val = in ? s.cand_val[cb.base + q] : 0.0f;
         const uint32_t idx = in ? s.cand_idx[cb.base + q] : 0u;
         const uint32_t key = key_of(val);
         const bool tie = in && key == T;
         const uint32_t tb = __ballot_sync(0xffffffffu, tie);
-        if (lane == 0) wtie[warp] = __popc(tb);
-        __syncthreads();
-        uint32_t tie_rank = run_tie + __popc(tb & lt_mask), tie_tot = 0;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) { if (w < warp) tie_rank += wtie[w]; tie_tot += wtie[w]; }
+        const uint32_t tie_rank = run_tie + __popc(tb & lt_mask);
         const bool take = in && (key > T || (tie && tie_rank < allowed));
         const uint32_t sb = __ballot_sync(0xffffffffu, take);
-        if (lane == 0) wsel[warp] = __popc(sb);
-        __syncthreads();
-        uint32_t out = run_sel + __popc(sb & lt_mask), sel_tot = 0;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) { if (w < warp) out += wsel[w]; sel_tot += wsel[w]; }
         if (take) {
+            const uint32_t out = run_sel + __popc(sb & lt_mask);
             s.idx[obase + out] = idx;
             s.val[obase + out] = val;
             if (s.zero_out) s.zero_out[idx] = 0.0f;
             if (has_last && tie && tie_rank == allowed - 1) cb.sel[SEL_CUT] = idx;
         }
-        run_sel += sel_tot;
-        run_tie += tie_tot;
-        __syncthreads();
+        run_sel += __popc(sb);
+        run_tie += __popc(tb);
     }
 }
 
@@ -425,20 +498,25 @@ __global__ void __launch_bounds__(THREADS) topk_slow_kernel(const __grid_constan
     const int64_t seg_beg = __ldg(p.seg_off + t);
     const int64_t n = __ldg(p.seg_off + t + 1) - seg_beg;
     const GT *src = reinterpret_cast<const GT *>(s.src) + (int64_t)row * s.row_stride + seg_beg;
-    const uint32_t b1 = sel[SEL_PREFIX];
     uint32_t rank = sel[SEL_REMAIN];
-    // second digit
-    for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) bins[b] = 0u;
-    __syncthreads();
-    for (int64_t j = threadIdx.x; j < n; j += THREADS) {
-        const uint32_t key = key_of(load1(src + j));
-        if ((key >> DIGIT1_SHIFT) == b1) atomicAdd(&bins[(key >> 7) & 0xfffu], 1u);
+    uint32_t prefix24;
+    if (sel[SEL_FLAGS] & 2u) {
+        prefix24 = sel[SEL_PREFIX];  // found by the dense second-digit pass
+    } else {
+        const uint32_t b1 = sel[SEL_PREFIX];
+        for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) bins[b] = 0u;
+        __syncthreads();
+        for (int64_t j = threadIdx.x; j < n; j += THREADS) {
+            const uint32_t key = key_of(load1(src + j));
+            if ((key >> DIGIT1_SHIFT) == b1) atomicAdd(&bins[(key >> 7) & 0xfffu], 1u);
+        }
+        __syncthreads();
+        PickResult r2 = block_pick(bins, DIGIT1_BINS, rank, scratch);
+        if (!r2.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
+        prefix24 = (b1 << 12) | r2.bin;
+        rank = r2.rank_in_bin;
     }
-    __syncthreads();
-    PickResult r = block_pick(bins, DIGIT1_BINS, rank, scratch);
-    if (!r.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
-    const uint32_t prefix24 = (b1 << 12) | r.bin;
-    rank = r.rank_in_bin;
+    PickResult r;
     // last 7 bits
     for (int b = threadIdx.x; b < 128; b += THREADS) bins[b] = 0u;
     __syncthreads();
@@ -599,15 +677,20 @@ cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, in
     dim3 g_tiles(p.TT, s.R), g_probs(p.T, s.R);
     const bool bf = uplink && p.gdt == DT_BF16;
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 1); CHECK_LAUNCH();
+    if (bf) topk_hist2_dense_kernel<__nv_bfloat16><<<g_tiles, THREADS, 0, st>>>(p, s);
+    else topk_hist2_dense_kernel<float><<<g_tiles, THREADS, 0, st>>>(p, s);
+    CHECK_LAUNCH();
+    topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 4); CHECK_LAUNCH();
     if (bf) topk_filter_kernel<__nv_bfloat16><<<g_tiles, THREADS, 0, st>>>(p, s);
     else topk_filter_kernel<float><<<g_tiles, THREADS, 0, st>>>(p, s);
     CHECK_LAUNCH();
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();
-    topk_hist3_kernel<<<g_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+    dim3 g_warp_tiles((p.TT + 7) / 8, s.R);
+    topk_hist3_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 3); CHECK_LAUNCH();
-    topk_count_kernel<<<g_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+    topk_count_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     topk_scan_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
-    topk_write_kernel<<<g_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+    topk_write_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     if (bf) topk_slow_kernel<__nv_bfloat16><<<g_probs, THREADS, 0, st>>>(p, s);
     else topk_slow_kernel<float><<<g_probs, THREADS, 0, st>>>(p, s);
     CHECK_LAUNCH();

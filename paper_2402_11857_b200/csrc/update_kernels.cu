@@ -35,16 +35,6 @@ __global__ void __launch_bounds__(THREADS) worker_update_kernel(const __grid_con
         up_thresh = sel[SEL_THRESH];
         up_cut = sel[SEL_CUT];
     }
-    if (DOWN == COMP_TOPK) {
-        for (int q = threadIdx.x; q < TILE; q += THREADS) p_tile[q] = 0.0f;
-        __syncthreads();
-        const bool last_tile = (blockIdx.x + 1 == __ldg(p.tile_prefix + ti.t + 1));
-        const uint32_t beg = p.down_outbase[blockIdx.x];
-        const uint32_t end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : p.down_outbase[blockIdx.x + 1];
-        const uint32_t tile_first = (uint32_t)(ti.seg_beg + ti.rel);
-        for (uint32_t q = beg + threadIdx.x; q < end; q += THREADS) p_tile[p.down_idx[q] - tile_first] = p.down_val[q];
-        __syncthreads();
-    }
     const float *v_tile = DOWN == COMP_IDENTITY ? p.vbuf + ti.seg_beg + ti.rel : nullptr;
 
     float g[8][4], x[8][4];
@@ -59,6 +49,19 @@ __global__ void __launch_bounds__(THREADS) worker_update_kernel(const __grid_con
             load4_guarded(g_tile, tile_pos(warp, lane, j), ti.len, g[j]);
             load4_guarded(x_tile, tile_pos(warp, lane, j), ti.len, x[j]);
         }
+    }
+
+    // decode the downlink top-k message of this tile (after the streaming loads are in flight)
+    if (DOWN == COMP_TOPK) {
+        for (int q = threadIdx.x; q < TILE / 4; q += THREADS)
+            reinterpret_cast<float4 *>(p_tile)[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        __syncthreads();
+        const bool last_tile = (blockIdx.x + 1 == __ldg(p.tile_prefix + ti.t + 1));
+        const uint32_t beg = p.down_outbase[blockIdx.x];
+        const uint32_t end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : p.down_outbase[blockIdx.x + 1];
+        const uint32_t tile_first = (uint32_t)(ti.seg_beg + ti.rel);
+        for (uint32_t q = beg + threadIdx.x; q < end; q += THREADS) p_tile[p.down_idx[q] - tile_first] = p.down_val[q];
+        __syncthreads();
     }
 
 #pragma unroll

@@ -59,6 +59,21 @@ def test_quantised_values_ties_at_threshold():
         P.step(G, 0.1)
 
 
+def test_crowded_threshold_bin_uses_second_digit():
+    """Many entries just around the threshold (what error feedback produces in v): more of them share
+    the threshold's first key digit than the candidate buffer holds, yet their keys are distinct."""
+    lay = Layout("crowded", (50000, 9000, 3 * 8192))
+    k = np.asarray([500, 90, 245], np.int64)
+    P = _pair(3, lay.seg_offsets, TOPK, TOPK, k=k)
+    g = torch.Generator().manual_seed(22)
+    for step in range(3):
+        G = torch.randn(3, lay.dim, generator=g) * 0.01
+        crowd = torch.rand(3, lay.dim, generator=g) < 0.2
+        G = torch.where(crowd, 1.0 + 0.03 * torch.rand(3, lay.dim, generator=g), G)
+        G = G * torch.where(torch.rand(3, lay.dim, generator=g) < 0.5, -1.0, 1.0)
+        P.step(G, 0.1)
+
+
 def test_all_zero_and_mostly_zero_gradients():
     lay = Layout("zeros", (5000, 20000))
     k = np.asarray([50, 200], np.int64)
