@@ -249,22 +249,16 @@ __global__ void __launch_bounds__(THREADS) topk_hist2_dense_kernel(const __grid_
 // filter: one CTA per (tile, row); ordered append of candidates
 // ------------------------------------------------------------------------------------------------
 template <typename GT>
-__global__ void __launch_bounds__(THREADS, 3) topk_filter_kernel(const __grid_constant__ Params p, const TopkSide s) {
+__global__ void __launch_bounds__(THREADS, 5) topk_filter_kernel(const __grid_constant__ Params p, const TopkSide s) {
     __shared__ uint32_t warp_tot[8];
     __shared__ uint32_t tile_base;
     const int row = blockIdx.y;
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
-    const uint32_t flags = sel[SEL_FLAGS];
-    if (flags & 1u) return;
-    // regular problems compare the first digit; refined ones the 24-bit prefix
-    const bool refined = flags == 2u;
-    const int cmp_shift = refined ? 7 : DIGIT1_SHIFT;
-    const uint32_t b1 = sel[SEL_PREFIX];
     const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
     const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
     const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+    // the streaming loads do not depend on the selection state: issue them first
     float v[8][4];
     if (fast) {
 #pragma unroll
@@ -273,29 +267,31 @@ __global__ void __launch_bounds__(THREADS, 3) topk_filter_kernel(const __grid_co
 #pragma unroll
         for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v[j]);
     }
-    uint32_t *gh2 = s.hist2 + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS;
-    // candidate flags: one nibble per row; counts of rows 0-3 and 4-7 packed as bytes of two words
-    uint32_t nib[8], rowoff[8];
-    uint32_t cnt_lo = 0, cnt_hi = 0;
+    uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
+    const uint32_t flags = sel[SEL_FLAGS];
+    if (flags & 1u) return;
+    // regular problems compare the first digit, refined ones the 24-bit prefix: either way a
+    // candidate is an entry whose key is at least the prefix shifted back into place
+    const bool refined = flags == 2u;
+    const uint32_t prefix = sel[SEL_PREFIX];
+    const uint32_t low_key = prefix << (refined ? 7 : DIGIT1_SHIFT);
+    uint32_t mask = 0;  // bit 4j+c: element c of row j is a candidate
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int pos = tile_pos(warp, lane, j);
-        uint32_t f = 0;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            const uint32_t key = key_of(v[j][c]);
-            const uint32_t d1 = key >> cmp_shift;
-            const bool valid = fast || pos + c < ti.len;
-            if (valid && d1 >= b1) {
-                f |= 1u << c;
-                if (!refined && d1 == b1) atomicAdd(gh2 + ((key >> 7) & 0xfffu), 1u);
-            }
+            const bool cand = key_of(v[j][c]) >= low_key && (fast || pos + c < ti.len);
+            if (cand) mask |= 1u << (4 * j + c);
         }
-        nib[j] = f;
-        if (j < 4) cnt_lo |= (uint32_t)__popc(f) << (8 * j);
-        else cnt_hi |= (uint32_t)__popc(f) << (8 * (j - 4));
     }
-    // inclusive scan over lanes of the packed per-row counts (a row holds at most 128 < 256)
+    // per-row counts packed as bytes (rows 0-3, rows 4-7), inclusive scan over lanes
+    uint32_t cnt_lo = 0, cnt_hi = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        cnt_lo |= (uint32_t)__popc((mask >> (4 * j)) & 0xfu) << (8 * j);
+        cnt_hi |= (uint32_t)__popc((mask >> (4 * j + 16)) & 0xfu) << (8 * j);
+    }
     uint32_t inc_lo = cnt_lo, inc_hi = cnt_hi;
 #pragma unroll
     for (int m = 1; m < 32; m <<= 1) {
@@ -304,6 +300,7 @@ __global__ void __launch_bounds__(THREADS, 3) topk_filter_kernel(const __grid_co
     }
     const uint32_t tot_lo = __shfl_sync(0xffffffffu, inc_lo, 31), tot_hi = __shfl_sync(0xffffffffu, inc_hi, 31);
     const uint32_t exc_lo = inc_lo - cnt_lo, exc_hi = inc_hi - cnt_hi;
+    uint32_t rowoff[8];
     uint32_t running = 0;  // candidates of this warp before the current row
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
@@ -320,8 +317,8 @@ __global__ void __launch_bounds__(THREADS, 3) topk_filter_kernel(const __grid_co
         if (w < warp) warp_off += warp_tot[w];
         tile_cnt += warp_tot[w];
     }
-    const uint32_t cap = (uint32_t)(__ldg(p.cap_off + ti.t + 1) - __ldg(p.cap_off + ti.t));
     if (threadIdx.x == 0) {
+        const uint32_t cap = (uint32_t)(__ldg(p.cap_off + ti.t + 1) - __ldg(p.cap_off + ti.t));
         uint32_t pos0 = tile_cnt ? atomicAdd(&sel[SEL_CAND_COUNT], tile_cnt) : 0u;
         if (pos0 + tile_cnt > cap) { atomicOr(p.status, STATUS_CAND_OVERFLOW); pos0 = 0xffffffffu; }
         tile_base = pos0;
@@ -330,19 +327,24 @@ __global__ void __launch_bounds__(THREADS, 3) topk_filter_kernel(const __grid_co
         m[1] = pos0 == 0xffffffffu ? 0u : tile_cnt;
     }
     __syncthreads();
-    if (tile_base == 0xffffffffu) return;
+    if (tile_base == 0xffffffffu || mask == 0u) return;
     const int64_t cbase = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + tile_base + warp_off;
+    uint32_t *gh2 = s.hist2 + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS;
+    const uint32_t flat0 = (uint32_t)(ti.seg_beg + ti.rel);
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
+        uint32_t nib = (mask >> (4 * j)) & 0xfu;
         uint32_t o = rowoff[j];
-        const uint32_t flat = (uint32_t)(ti.seg_beg + ti.rel) + tile_pos(warp, lane, j);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            if (nib[j] & (1u << c)) {
-                s.cand_idx[cbase + o] = flat + c;
-                s.cand_val[cbase + o] = v[j][c];
-                ++o;
-            }
+        while (nib) {  // candidates are rare: usually no iteration at all
+            const int c = __ffs(nib) - 1;
+            nib &= nib - 1;
+            const int pos = tile_pos(warp, lane, j) + c;
+            const float val = load1(tile_ptr + pos);  // read again (cached) rather than kept across the barrier
+            const uint32_t key = key_of(val);
+            s.cand_idx[cbase + o] = flat0 + pos;
+            s.cand_val[cbase + o] = val;
+            if (!refined && (key >> DIGIT1_SHIFT) == prefix) atomicAdd(gh2 + ((key >> 7) & 0xfffu), 1u);
+            ++o;
         }
     }
 }
@@ -596,17 +598,47 @@ __global__ void __launch_bounds__(THREADS) server_topk_kernel(const __grid_const
     __syncthreads();
     const bool last_tile = (blockIdx.x + 1 == __ldg(p.tile_prefix + ti.t + 1));
     const uint32_t tile_first = (uint32_t)(ti.seg_beg + ti.rel);
-    for (int i = 0; i < p.N; ++i) {
-        const uint32_t *ob = p.up_outbase + (int64_t)i * (p.TT + 1) + blockIdx.x;
-        const uint32_t beg = ob[0];
-        const uint32_t end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : ob[1];
-        const uint32_t *idx = p.up_idx + (int64_t)i * p.K;
-        const float *val = p.up_val + (int64_t)i * p.K;
-        for (uint32_t q = beg + threadIdx.x; q < end; q += THREADS) {
-            const uint32_t o = idx[q] - tile_first;
-            acc[o] = __fadd_rn(acc[o], val[q]);
+    // Workers are taken 16 at a time: 16 threads per worker first fetch that worker's entries for
+    // this tile (all fetches in flight together), then the entries are added worker by worker
+    // so that every element sees its contributions in worker order.
+    constexpr int PRE = 8;  // entries prefetched per thread (16 x 8 = 128 per worker and tile)
+    const int ws = threadIdx.x >> 4, sub = threadIdx.x & 15;
+    for (int g0 = 0; g0 < p.N; g0 += 16) {
+        const int i = g0 + ws;
+        uint32_t beg = 0, end = 0;
+        const uint32_t *idx = nullptr;
+        const float *val = nullptr;
+        if (i < p.N) {
+            const uint32_t *ob = p.up_outbase + (int64_t)i * (p.TT + 1) + blockIdx.x;
+            beg = ob[0];
+            end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : ob[1];
+            idx = p.up_idx + (int64_t)i * p.K;
+            val = p.up_val + (int64_t)i * p.K;
         }
-        __syncthreads();
+        uint32_t pidx[PRE];
+        float pval[PRE];
+#pragma unroll
+        for (int m = 0; m < PRE; ++m) {
+            const uint32_t q = beg + sub + 16 * m;
+            pidx[m] = q < end ? idx[q] : 0xffffffffu;
+            pval[m] = q < end ? val[q] : 0.0f;
+        }
+        const int in_group = min(16, p.N - g0);
+        for (int turn = 0; turn < in_group; ++turn) {
+            if (ws == turn) {
+#pragma unroll
+                for (int m = 0; m < PRE; ++m)
+                    if (pidx[m] != 0xffffffffu) {
+                        const uint32_t o = pidx[m] - tile_first;
+                        acc[o] = __fadd_rn(acc[o], pval[m]);
+                    }
+                for (uint32_t q = beg + sub + 16 * PRE; q < end; q += 16) {
+                    const uint32_t o = idx[q] - tile_first;
+                    acc[o] = __fadd_rn(acc[o], val[q]);
+                }
+            }
+            __syncthreads();
+        }
     }
     const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
     const float nf = (float)p.N;

@@ -11,9 +11,13 @@ namespace liec {
 template <int UP, int DOWN, typename GT>
 __global__ void __launch_bounds__(THREADS) worker_update_kernel(const __grid_constant__ Params p, const float lr) {
     __shared__ __align__(16) float p_tile[DOWN == COMP_TOPK ? TILE : 4];  // decoded downlink message (top-k)
-    const int worker = blockIdx.y;
+    // With a top-k downlink a CTA serves WPC workers so that the message is decoded once for them.
+    constexpr int WPC = DOWN == COMP_TOPK ? 4 : 1;
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int wq = 0; wq < WPC; ++wq) {
+    const int worker = blockIdx.y * WPC + wq;
+    if (worker >= p.N) break;
     const int64_t row_beg = (int64_t)worker * p.d + ti.seg_beg;
     const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
     const GT *g_tile = reinterpret_cast<const GT *>(p.G) + row_beg + ti.rel;
@@ -52,7 +56,7 @@ __global__ void __launch_bounds__(THREADS) worker_update_kernel(const __grid_con
     }
 
     // decode the downlink top-k message of this tile (after the streaming loads are in flight)
-    if (DOWN == COMP_TOPK) {
+    if (DOWN == COMP_TOPK && wq == 0) {
         for (int q = threadIdx.x; q < TILE / 4; q += THREADS)
             reinterpret_cast<float4 *>(p_tile)[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         __syncthreads();
@@ -103,11 +107,13 @@ __global__ void __launch_bounds__(THREADS) worker_update_kernel(const __grid_con
                 if (pos + c < ti.len) x_tile[pos + c] = x[j][c];
         }
     }
+    }  // workers of this CTA
 }
 
 template <int UP, int DOWN>
 static cudaError_t launch_t(const Params &p, float lr, cudaStream_t st) {
-    dim3 grid(p.TT, p.N);
+    constexpr int WPC = DOWN == COMP_TOPK ? 4 : 1;
+    dim3 grid(p.TT, (p.N + WPC - 1) / WPC);
     if (p.gdt == DT_F32) worker_update_kernel<UP, DOWN, float><<<grid, THREADS, 0, st>>>(p, lr);
     else worker_update_kernel<UP, DOWN, __nv_bfloat16><<<grid, THREADS, 0, st>>>(p, lr);
     return cudaGetLastError();
