@@ -101,7 +101,12 @@ def scaled_layout(base: Layout, divisor: int, name: str | None = None) -> Layout
     Keeps the size spread and the segment count of the architecture while
     shrinking d so that the CPU oracle runs many steps in seconds.
     """
-    sizes = tuple(max(1, -(-n // divisor)) for n in base.sizes)
+    def shrink(n: int) -> int:
+        m = max(1, -(-n // divisor))
+        if n % 8 == 0:          # keep the 8-element granularity of the original tensor
+            m = -(-m // 8) * 8  # (rows and segments then start 16-byte aligned, as in the full layout)
+        return m
+    sizes = tuple(shrink(n) for n in base.sizes)
     return Layout(name or f"{base.name}/{divisor}", sizes)
 
 

@@ -109,14 +109,23 @@ __device__ PickResult block_pick(const uint32_t *bins, int nbins, uint32_t rank,
 // ------------------------------------------------------------------------------------------------
 // hist1: one CTA per (tile, row)
 // ------------------------------------------------------------------------------------------------
+template <bool FAST>
+__device__ __forceinline__ void hist1_count(uint32_t *h, const float (&v)[8][4], int warp, int lane, int len) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pos = tile_pos(warp, lane, j);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if (FAST || pos + c < len) atomicAdd(&h[key_of(v[j][c]) >> DIGIT1_SHIFT], 1u);
+    }
+}
+
 template <typename GT>
 __global__ void __launch_bounds__(THREADS) topk_hist1_kernel(const __grid_constant__ Params p, const TopkSide s) {
-    __shared__ uint32_t h[DIGIT1_BINS];
+    __shared__ __align__(16) uint32_t h[DIGIT1_BINS];
     const int row = blockIdx.y;
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) h[b] = 0u;
-    __syncthreads();
     const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
     const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
     const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
@@ -128,18 +137,20 @@ __global__ void __launch_bounds__(THREADS) topk_hist1_kernel(const __grid_consta
 #pragma unroll
         for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v[j]);
     }
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int pos = tile_pos(warp, lane, j);
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-            if (fast || pos + c < ti.len) atomicAdd(&h[key_of(v[j][c]) >> DIGIT1_SHIFT], 1u);
-    }
+    for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(h)[b] = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+    if (fast) hist1_count<true>(h, v, warp, lane, ti.len);
+    else hist1_count<false>(h, v, warp, lane, ti.len);
     __syncthreads();
     uint32_t *gh = s.hist + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS;
-    for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) {
-        uint32_t c = h[b];
-        if (c) atomicAdd(gh + b, c);
+    for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) {
+        const uint4 c = reinterpret_cast<const uint4 *>(h)[b];
+        if (c.x | c.y | c.z | c.w) {
+            if (c.x) atomicAdd(gh + 4 * b + 0, c.x);
+            if (c.y) atomicAdd(gh + 4 * b + 1, c.y);
+            if (c.z) atomicAdd(gh + 4 * b + 2, c.z);
+            if (c.w) atomicAdd(gh + 4 * b + 3, c.w);
+        }
     }
 }
 
@@ -248,8 +259,23 @@ __global__ void __launch_bounds__(THREADS) topk_hist2_dense_kernel(const __grid_
 // ------------------------------------------------------------------------------------------------
 // filter: one CTA per (tile, row); ordered append of candidates
 // ------------------------------------------------------------------------------------------------
+// Candidate mask of a thread's 32 elements: bit 4j+c is set when |v[j][c]| is at least `low`
+// (a magnitude bit pattern used as a float: for finite values the order is the same).
+template <bool FAST>
+__device__ __forceinline__ uint32_t filter_mask(const float (&v)[8][4], float low, int warp, int lane, int len) {
+    uint32_t mask = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pos = tile_pos(warp, lane, j);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if (fabsf(v[j][c]) >= low && (FAST || pos + c < len)) mask |= 1u << (4 * j + c);
+    }
+    return mask;
+}
+
 template <typename GT>
-__global__ void __launch_bounds__(THREADS, 5) topk_filter_kernel(const __grid_constant__ Params p, const TopkSide s) {
+__global__ void __launch_bounds__(THREADS, 4) topk_filter_kernel(const __grid_constant__ Params p, const TopkSide s) {
     __shared__ uint32_t warp_tot[8];
     __shared__ uint32_t tile_base;
     const int row = blockIdx.y;
@@ -274,17 +300,9 @@ __global__ void __launch_bounds__(THREADS, 5) topk_filter_kernel(const __grid_co
     // candidate is an entry whose key is at least the prefix shifted back into place
     const bool refined = flags == 2u;
     const uint32_t prefix = sel[SEL_PREFIX];
-    const uint32_t low_key = prefix << (refined ? 7 : DIGIT1_SHIFT);
-    uint32_t mask = 0;  // bit 4j+c: element c of row j is a candidate
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int pos = tile_pos(warp, lane, j);
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const bool cand = key_of(v[j][c]) >= low_key && (fast || pos + c < ti.len);
-            if (cand) mask |= 1u << (4 * j + c);
-        }
-    }
+    const float low = __uint_as_float(prefix << (refined ? 7 : DIGIT1_SHIFT));
+    const uint32_t mask = fast ? filter_mask<true>(v, low, warp, lane, ti.len)
+                               : filter_mask<false>(v, low, warp, lane, ti.len);
     // per-row counts packed as bytes (rows 0-3, rows 4-7), inclusive scan over lanes
     uint32_t cnt_lo = 0, cnt_hi = 0;
 #pragma unroll
@@ -300,13 +318,14 @@ __global__ void __launch_bounds__(THREADS, 5) topk_filter_kernel(const __grid_co
     }
     const uint32_t tot_lo = __shfl_sync(0xffffffffu, inc_lo, 31), tot_hi = __shfl_sync(0xffffffffu, inc_hi, 31);
     const uint32_t exc_lo = inc_lo - cnt_lo, exc_hi = inc_hi - cnt_hi;
-    uint32_t rowoff[8];
-    uint32_t running = 0;  // candidates of this warp before the current row
+    // running row bases of the warp, again packed (a warp holds at most 1024 candidates: 16-bit fields)
+    uint32_t running = 0;
+    uint32_t base01 = 0, base23 = 0, base45 = 0, base67 = 0;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const uint32_t before = ((j < 4 ? exc_lo : exc_hi) >> (8 * (j & 3))) & 0xffu;
         const uint32_t total = ((j < 4 ? tot_lo : tot_hi) >> (8 * (j & 3))) & 0xffu;
-        rowoff[j] = running + before;
+        const uint32_t field = running << (16 * (j & 1));
+        if (j < 2) base01 |= field; else if (j < 4) base23 |= field; else if (j < 6) base45 |= field; else base67 |= field;
         running += total;
     }
     if (lane == 0) warp_tot[warp] = running;
@@ -331,21 +350,23 @@ __global__ void __launch_bounds__(THREADS, 5) topk_filter_kernel(const __grid_co
     const int64_t cbase = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + tile_base + warp_off;
     uint32_t *gh2 = s.hist2 + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS;
     const uint32_t flat0 = (uint32_t)(ti.seg_beg + ti.rel);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        uint32_t nib = (mask >> (4 * j)) & 0xfu;
-        uint32_t o = rowoff[j];
-        while (nib) {  // candidates are rare: usually no iteration at all
-            const int c = __ffs(nib) - 1;
-            nib &= nib - 1;
-            const int pos = tile_pos(warp, lane, j) + c;
-            const float val = load1(tile_ptr + pos);  // read again (cached) rather than kept across the barrier
-            const uint32_t key = key_of(val);
-            s.cand_idx[cbase + o] = flat0 + pos;
-            s.cand_val[cbase + o] = val;
-            if (!refined && (key >> DIGIT1_SHIFT) == prefix) atomicAdd(gh2 + ((key >> 7) & 0xfffu), 1u);
-            ++o;
-        }
+    // walk the set bits (candidates are rare: usually zero or one iteration)
+    uint32_t rest = mask;
+    while (rest) {
+        const int b = __ffs(rest) - 1;
+        rest &= rest - 1;
+        const int j = b >> 2;
+        const uint32_t base_pair = j < 2 ? base01 : j < 4 ? base23 : j < 6 ? base45 : base67;
+        const uint32_t row_base = (base_pair >> (16 * (j & 1))) & 0xffffu;
+        const uint32_t before = ((j < 4 ? exc_lo : exc_hi) >> (8 * (j & 3))) & 0xffu;
+        const uint32_t lower = __popc(mask & ((1u << b) - 1u) & (0xfu << (4 * j)));
+        const uint32_t o = row_base + before + lower;
+        const int pos = tile_pos(warp, lane, j) + (b & 3);
+        const float val = load1(tile_ptr + pos);  // read again (cached) rather than kept across the barrier
+        const uint32_t key = key_of(val);
+        s.cand_idx[cbase + o] = flat0 + pos;
+        s.cand_val[cbase + o] = val;
+        if (!refined && (key >> DIGIT1_SHIFT) == prefix) atomicAdd(gh2 + ((key >> 7) & 0xfffu), 1u);
     }
 }
 
