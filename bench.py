@@ -92,7 +92,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -101,7 +101,13 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.samples.append(line.strip())
+            self.samples.append((time.monotonic(), line.strip()))
+
+    def mark_begin(self):
+        self.t0 = time.monotonic()
+
+    def mark_end(self):
+        self.t1 = time.monotonic()
 
     def stop(self):
         if self.proc is None:
@@ -113,7 +119,9 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for s in self.samples:
+        t0, t1 = getattr(self, "t0", 0.0), getattr(self, "t1", float("inf"))
+        inside = [line for (ts, line) in self.samples if t0 <= ts <= t1 + 0.05]
+        for s in inside:
             parts = [q.strip() for q in s.split(",")]
             if len(parts) < 7:
                 continue
@@ -237,22 +245,23 @@ def run_gpu(args, w, rank, world, local_rank):
         ctx.liec_downlink_compress(); events[3].record()
         ctx.liec_worker_update(G, w["lr"]); events[4].record()
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()          # nvidia-smi needs a moment to start: launch it before the warm-up
     for _ in range(args.warmup):
         one_step()
     torch.cuda.synchronize()
     barrier()
-
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
     launches0 = ctx.liec_launch_count()
     torch.cuda.synchronize()
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.mark_begin()
     start.record()
     for s in range(args.steps):
         one_step(evs[s])
     stop.record()
     torch.cuda.synchronize()
+    sampler.mark_end()
     total_ms = start.elapsed_time(stop)
     launches = ctx.liec_launch_count() - launches0
     barrier()
@@ -294,7 +303,7 @@ def run_gpu(args, w, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4")
