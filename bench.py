@@ -76,6 +76,12 @@ def update_kernel_bytes(w) -> float:
     return N * d * (g + 8) + down
 
 
+# DRAM bytes per element-worker of the worker update, from the committed ncu capture
+# (profiles/sign_kernels_c4_launches_and_c4div8_counters.md: 4.925 GB for 497.8 M element-workers on
+# c4/8; the traffic of this streaming kernel grows in proportion to N*d).  Other variants: not captured.
+UPDATE_TRAFFIC_PER_UNIT = {("sign", "bf16"): 4.924888e9 / 497759232}
+
+
 # ------------------------------------------------------------------------------------ clocks
 
 class ClockSampler:
@@ -367,7 +373,9 @@ def main():
         "pct_of_measured_copy_peak": 100 * step_gbs / peak, "min_bytes_per_step": bmin,
         "stage_ms": r["stage_ms"],
         "roofline": {"bound": "hbm", "kernel": "worker_update_kernel", "achieved": upd_gbs, "peak": peak,
-                     "unit": "GB/s", "frac": upd_gbs / peak, "traffic": None, "peak_source": peak_src,
+                     "unit": "GB/s", "frac": upd_gbs / peak,
+                     "traffic": (UPDATE_TRAFFIC_PER_UNIT[(w["comp"], w["gdt"])] * N * d
+                                 if (w["comp"], w["gdt"]) in UPDATE_TRAFFIC_PER_UNIT else None), "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": update_kernel_bytes(w), "launch_ms": upd_ms},
         "gpu_launches": r["launches"], "clocks": r["clocks"],
     }
