@@ -1,0 +1,107 @@
+"""Parity at the full benchmark sizes (C2, C3, C4), in the launch configuration bench.py times.
+
+The oracle cannot run a whole C3/C4 step in reasonable time, but every stage of the step is
+local to a segment (element-wise work plus per-segment reductions and selections), so the oracle
+is run on a sample of whole segments with all N workers, and the library's outputs restricted
+to those segments must match it bit for bit.  Properties that hold at any size are checked over
+all segments on the device."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_helpers import assert_close, f32, u32, widen
+from liec_synth import WORKLOADS, make_gradients, topk_counts
+from paper_2402_11857_b200 import liec
+
+pytestmark = pytest.mark.gpu
+
+
+def _sample_segments(lay, budget_elems):
+    """A spread of segments by size (largest that fits, median, small ones) within an element budget."""
+    order = sorted(range(lay.num_segments), key=lambda t: -lay.sizes[t])
+    chosen, total = [], 0
+    for t in order[:: max(1, lay.num_segments // 12)] + order[-3:]:
+        if t not in chosen and total + lay.sizes[t] <= budget_elems:
+            chosen.append(t)
+            total += lay.sizes[t]
+    return sorted(chosen)
+
+
+def _run(name, steps, budget_elems):
+    w = WORKLOADS[name]
+    lay = w.layout()
+    N, d, off = w.num_workers, lay.dim, lay.seg_offsets
+    comp = liec.COMP_SCALED_SIGN if w.compressor == "sign" else liec.COMP_TOPK
+    ocomp = oracle.SIGN if w.compressor == "sign" else oracle.TOPK
+    k = topk_counts(lay, *w.topk_frac) if w.compressor == "topk" else None
+    gdt = liec.BF16 if w.grad_dtype == "bf16" else liec.F32
+    X = torch.zeros(N, d, device="cuda")
+    e = torch.zeros(d, device="cuda")
+    ctx = liec.Context(X, e, off, comp, comp, k, gdt)
+    G = torch.empty(N, d, device="cuda", dtype=torch.bfloat16 if gdt == liec.BF16 else torch.float32)
+
+    segs = _sample_segments(lay, budget_elems)
+    sub_sizes = [lay.sizes[t] for t in segs]
+    sub_off = np.concatenate([[0], np.cumsum(sub_sizes)]).astype(np.int64)
+    cols = torch.cat([torch.arange(off[t], off[t + 1], device="cuda") for t in segs])
+    Xh = np.zeros((N, int(sub_off[-1])), np.float32)
+    eh = np.zeros(int(sub_off[-1]), np.float32)
+    ksub = None if k is None else k[segs]
+    woff = np.concatenate([[0], np.cumsum((np.diff(off) + 31) // 32)])
+    koff = None if k is None else np.concatenate([[0], np.cumsum(k)])
+
+    for step in range(steps):
+        make_gradients(w.dist, w.scale, N, d, step, base_seed=77, device="cuda", out=G)
+        ctx.liec_step(G, w.lr)
+        torch.cuda.synchronize()
+        assert ctx.liec_device_status() == 0
+        m = ctx.liec_get_messages()
+        r = oracle.step(Xh, eh, widen(G[:, cols]), w.lr, sub_off, ocomp, ocomp, k=ksub)
+        assert_close(f32(X[:, cols]), Xh, f"{name} step {step}: params on sampled segments")
+        assert_close(f32(e[cols]), eh, f"{name} step {step}: error on sampled segments")
+        if comp == liec.COMP_SCALED_SIGN:
+            sub_woff = np.concatenate([[0], np.cumsum((np.diff(sub_off) + 31) // 32)])
+            for q, t in enumerate(segs):
+                got = u32(m["up_words"][:, woff[t]:woff[t + 1]])
+                assert np.array_equal(got, r.up_words[:, sub_woff[q]:sub_woff[q + 1]]), (name, step, t, "up words")
+                assert np.array_equal(u32(m["down_words"][woff[t]:woff[t + 1]]), r.down_words[sub_woff[q]:sub_woff[q + 1]])
+            assert np.array_equal(f32(m["up_scales"])[:, segs].view(np.uint32), r.up_scales.view(np.uint32))
+            assert np.array_equal(f32(m["down_scales"])[segs].view(np.uint32), r.down_scales.view(np.uint32))
+            # any size: one bit per negative gradient, over all segments and workers
+            neg = (G < 0).sum(dim=1).cpu().numpy()
+            pop = np.array([int(np.unpackbits(u32(m["up_words"][i]).view(np.uint8)).sum()) for i in range(0, N, max(1, N // 4))])
+            assert np.array_equal(pop, neg[:: max(1, N // 4)])
+        else:
+            sub_koff = np.concatenate([[0], np.cumsum(ksub)])
+            for q, t in enumerate(segs):
+                shift = int(off[t]) - int(sub_off[q])
+                got = u32(m["up_idx"][:, koff[t]:koff[t + 1]]).astype(np.int64) - shift
+                assert np.array_equal(got, r.up_idx[:, sub_koff[q]:sub_koff[q + 1]].astype(np.int64)), (name, step, t, "up idx")
+                gotd = u32(m["down_idx"][koff[t]:koff[t + 1]]).astype(np.int64) - shift
+                assert np.array_equal(gotd, r.down_idx[sub_koff[q]:sub_koff[q + 1]].astype(np.int64)), (name, step, t, "down idx")
+            # any size: per segment exactly k_t indices, ascending and inside the segment (worker 0 and N-1)
+            for i in (0, N - 1):
+                idx = u32(m["up_idx"][i]).astype(np.int64)
+                seg_of = np.repeat(np.arange(lay.num_segments), k)
+                assert np.all(idx >= off[seg_of]) and np.all(idx < off[seg_of + 1])
+                inner = np.ones(len(idx), bool); inner[koff[:-1]] = False
+                assert np.all(np.diff(idx)[inner[1:]] > 0)
+                # kept magnitudes dominate the dropped ones in the largest segment
+                t = int(np.argmax(lay.sizes))
+                g = G[i, off[t]:off[t + 1]].float().abs()
+                kept = torch.zeros_like(g, dtype=torch.bool)
+                kept[torch.from_numpy(idx[koff[t]:koff[t + 1]] - off[t]).cuda()] = True
+                assert g[kept].min() >= g[~kept].max()
+
+
+def test_c2_resnet18_sign_full_size():
+    _run("c2", steps=3, budget_elems=4_000_000)
+
+
+def test_c3_resnet50_topk_full_size():
+    _run("c3", steps=2, budget_elems=3_500_000)
+
+
+def test_c4_gpt2_sign_bf16_full_size():
+    _run("c4", steps=2, budget_elems=4_000_000)
