@@ -64,7 +64,7 @@ struct Params {
 };
 
 // per-problem selection state words
-constexpr int SEL_WORDS = 12;
+constexpr int SEL_WORDS = 16;
 constexpr int SEL_PREFIX = 0;     // key prefix fixed so far (aligned to its bit position)
 constexpr int SEL_REMAIN = 1;     // rank still to find inside the prefix bin (1-based)
 constexpr int SEL_CAND_COUNT = 2; // atomic cursor: candidates appended so far
@@ -74,5 +74,13 @@ constexpr int SEL_CUT = 5;        // flat index of the last accepted tie
 constexpr int SEL_FLAGS = 6;      // bit0: slow path (one CTA, dense passes); bit1: refined (24-bit prefix found by a dense second-digit pass)
 constexpr int SEL_NCAND = 7;      // exact number of candidates (entries at or above the prefix)
 constexpr int SEL_ABOVE = 8;      // entries whose first digit is strictly above the threshold's
+constexpr int SEL_LO1 = 9;        // lowest / highest non-empty bin of the first-digit histogram (so that the
+constexpr int SEL_HI1 = 10;       // pick reads and clears only that range); reset to ~0 / 0 after use
+constexpr int SEL_LO2 = 11;       // same for the second-digit histogram
+constexpr int SEL_HI2 = 12;
+
+// words of the status block (int32 each)
+constexpr int STATUS_WORD = 0;        // failed internal checks
+constexpr int STATUS_ANY_REFINE = 8;  // +0 uplink, +1 downlink: some problem needs the dense second-digit pass
 
 }  // namespace liec

@@ -56,6 +56,26 @@ __device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) 
 
 enum { STATUS_PICK_RANK = 1, STATUS_CAND_OVERFLOW = 2, STATUS_COUNT_MISMATCH = 4 };
 
+// Adds a CTA's shared-memory histogram to the problem's global one and widens the problem's
+// record of the non-empty bin range, so that the pick reads and clears only that range.
+__device__ __forceinline__ void flush_hist(const uint32_t *h, uint32_t *gh, uint32_t *sel, int lo_word, int hi_word) {
+    uint32_t lo = 0xffffffffu, hi = 0u;
+    for (uint32_t b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) {
+        const uint32_t c = h[b];
+        if (c) {
+            atomicAdd(gh + b, c);
+            lo = min(lo, b);
+            hi = max(hi, b);
+        }
+    }
+    lo = __reduce_min_sync(0xffffffffu, lo);
+    hi = __reduce_max_sync(0xffffffffu, hi);
+    if ((threadIdx.x & 31) == 0 && lo != 0xffffffffu) {
+        atomicMin(&sel[lo_word], lo);
+        atomicMax(&sel[hi_word], hi);
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Block helper: bins[0..nbins) in shared memory, find the bin that holds the rank-th largest
 // entry counting from the top bin down.  All threads get (bin, rank inside bin, count above+bin).
@@ -142,16 +162,8 @@ __global__ void __launch_bounds__(THREADS) topk_hist1_kernel(const __grid_consta
     if (fast) hist1_count<true>(h, v, warp, lane, ti.len);
     else hist1_count<false>(h, v, warp, lane, ti.len);
     __syncthreads();
-    uint32_t *gh = s.hist + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS;
-    for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) {
-        const uint4 c = reinterpret_cast<const uint4 *>(h)[b];
-        if (c.x | c.y | c.z | c.w) {
-            if (c.x) atomicAdd(gh + 4 * b + 0, c.x);
-            if (c.y) atomicAdd(gh + 4 * b + 1, c.y);
-            if (c.z) atomicAdd(gh + 4 * b + 2, c.z);
-            if (c.w) atomicAdd(gh + 4 * b + 3, c.w);
-        }
-    }
+    flush_hist(h, s.hist + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS,
+               s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS, SEL_LO1, SEL_HI1);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -167,22 +179,26 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
     // level 1: first digit.  level 4: second digit of "refined" problems (after their dense
     // second-digit pass).  level 2: second digit of regular problems.  level 3: last 7 bits.
     const uint32_t flags_in = level == 1 ? 0u : sel[SEL_FLAGS];
+    if (level == 4 && t == 0 && row == 0 && threadIdx.x == 0) p.status[STATUS_ANY_REFINE + (s.zero_out ? 1 : 0)] = 0;
     if (level == 4 && flags_in != 2u) return;
     if (level == 2 && flags_in != 0u) return;
     if (level == 3 && (flags_in & 1u)) return;  // slow path finishes on its own
     const int nbins = level == 3 ? 128 : DIGIT1_BINS;
     uint32_t *gh = (level == 1 ? s.hist : s.hist2) + ((int64_t)row * p.T + t) * DIGIT1_BINS;
     if (nbins == DIGIT1_BINS) {
-        // 4 independent 128-bit loads per thread, then the clears
-        uint4 tmp[DIGIT1_BINS / 4 / THREADS];
-        uint4 *gh4 = reinterpret_cast<uint4 *>(gh);
-#pragma unroll
-        for (int q = 0; q < DIGIT1_BINS / 4 / THREADS; ++q) tmp[q] = gh4[threadIdx.x + q * THREADS];
-#pragma unroll
-        for (int q = 0; q < DIGIT1_BINS / 4 / THREADS; ++q) {
-            reinterpret_cast<uint4 *>(bins)[threadIdx.x + q * THREADS] = tmp[q];
-            if (tmp[q].x | tmp[q].y | tmp[q].z | tmp[q].w) gh4[threadIdx.x + q * THREADS] = make_uint4(0u, 0u, 0u, 0u);
+        // only the recorded non-empty range is read and cleared
+        const int lo_word = level == 1 ? SEL_LO1 : SEL_LO2, hi_word = level == 1 ? SEL_HI1 : SEL_HI2;
+        // (the filter does not record the range of the second-digit histogram: level 2 reads all of it)
+        const uint32_t lo = level == 2 ? 0u : min(sel[lo_word], (uint32_t)DIGIT1_BINS);
+        const uint32_t hi = level == 2 ? (uint32_t)DIGIT1_BINS - 1u : min(sel[hi_word], (uint32_t)DIGIT1_BINS - 1u);
+        for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(bins)[b] = make_uint4(0u, 0u, 0u, 0u);
+        __syncthreads();
+        for (uint32_t b = lo + threadIdx.x; b <= hi; b += THREADS) {
+            const uint32_t c = gh[b];
+            if (c) { bins[b] = c; gh[b] = 0u; }
         }
+        __syncthreads();
+        if (threadIdx.x == 0) { sel[lo_word] = 0xffffffffu; sel[hi_word] = 0u; }
     } else {
         for (int b = threadIdx.x; b < nbins; b += THREADS) {
             bins[b] = gh[b];
@@ -204,6 +220,7 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
             sel[SEL_CAND_COUNT] = 0u;
             // too many entries share the threshold's first digit: look at the second digit first
             sel[SEL_FLAGS] = r.count_ge > cap ? 2u : 0u;
+            if (r.count_ge > cap) p.status[STATUS_ANY_REFINE + (s.zero_out ? 1 : 0)] = 1;
         } else if (level == 4) {
             const uint32_t ncand = sel[SEL_ABOVE] + r.count_ge;
             sel[SEL_PREFIX] = (sel[SEL_PREFIX] << 12) | r.bin;
@@ -225,34 +242,35 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
 template <typename GT>
 __global__ void __launch_bounds__(THREADS) topk_hist2_dense_kernel(const __grid_constant__ Params p, const TopkSide s) {
     __shared__ uint32_t h[DIGIT1_BINS];
+    // usually no problem on this side is refined: a small grid that leaves after one load
+    if (p.status[STATUS_ANY_REFINE + (s.zero_out ? 1 : 0)] == 0) return;
     const int row = blockIdx.y;
-    const TileInfo ti = locate_tile(p, blockIdx.x);
-    const uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
-    if (sel[SEL_FLAGS] != 2u) return;
-    const uint32_t b1 = sel[SEL_PREFIX];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) h[b] = 0u;
-    __syncthreads();
-    const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
-    const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
-    const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+    for (int tile = blockIdx.x; tile < p.TT; tile += gridDim.x) {
+        const TileInfo ti = locate_tile(p, tile);
+        uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
+        if (sel[SEL_FLAGS] != 2u) continue;  // uniform over the CTA
+        const uint32_t b1 = sel[SEL_PREFIX];
+        for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) h[b] = 0u;
+        __syncthreads();
+        const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
+        const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
+        const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int pos = tile_pos(warp, lane, j);
-        float v[4];
-        if (fast) load4_stream(tile_ptr + pos, v);
-        else load4_guarded(tile_ptr, pos, ti.len, v);
+        for (int j = 0; j < 8; ++j) {
+            const int pos = tile_pos(warp, lane, j);
+            float v[4];
+            if (fast) load4_stream(tile_ptr + pos, v);
+            else load4_guarded(tile_ptr, pos, ti.len, v);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const uint32_t key = key_of(v[c]);
-            if ((fast || pos + c < ti.len) && (key >> DIGIT1_SHIFT) == b1) atomicAdd(&h[(key >> 7) & 0xfffu], 1u);
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t key = key_of(v[c]);
+                if ((fast || pos + c < ti.len) && (key >> DIGIT1_SHIFT) == b1) atomicAdd(&h[(key >> 7) & 0xfffu], 1u);
+            }
         }
-    }
-    __syncthreads();
-    uint32_t *gh = s.hist2 + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS;
-    for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) {
-        uint32_t c = h[b];
-        if (c) atomicAdd(gh + b, c);
+        __syncthreads();
+        flush_hist(h, s.hist2 + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS, sel, SEL_LO2, SEL_HI2);
+        __syncthreads();
     }
 }
 
@@ -366,7 +384,10 @@ __global__ void __launch_bounds__(THREADS, 4) topk_filter_kernel(const __grid_co
         const uint32_t key = key_of(val);
         s.cand_idx[cbase + o] = flat0 + pos;
         s.cand_val[cbase + o] = val;
-        if (!refined && (key >> DIGIT1_SHIFT) == prefix) atomicAdd(gh2 + ((key >> 7) & 0xfffu), 1u);
+        if (!refined && (key >> DIGIT1_SHIFT) == prefix) {
+            const uint32_t d2 = (key >> 7) & 0xfffu;
+            atomicAdd(gh2 + d2, 1u);  // (range not tracked here: two more contended atomics cost more than they save)
+        }
     }
 }
 
@@ -696,11 +717,7 @@ __global__ void __launch_bounds__(THREADS) server_topk_kernel(const __grid_const
     }
     if (DOWN == COMP_TOPK) {
         __syncthreads();
-        uint32_t *gh = p.down_hist + (int64_t)ti.t * DIGIT1_BINS;
-        for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) {
-            uint32_t c = h[b];
-            if (c) atomicAdd(gh + b, c);
-        }
+        flush_hist(h, p.down_hist + (int64_t)ti.t * DIGIT1_BINS, p.down_sel + (int64_t)ti.t * SEL_WORDS, SEL_LO1, SEL_HI1);
     }
 }
 
@@ -730,8 +747,9 @@ cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, in
     dim3 g_tiles(p.TT, s.R), g_probs(p.T, s.R);
     const bool bf = uplink && p.gdt == DT_BF16;
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 1); CHECK_LAUNCH();
-    if (bf) topk_hist2_dense_kernel<__nv_bfloat16><<<g_tiles, THREADS, 0, st>>>(p, s);
-    else topk_hist2_dense_kernel<float><<<g_tiles, THREADS, 0, st>>>(p, s);
+    dim3 g_strided(p.TT < 592 ? p.TT : 592, s.R);
+    if (bf) topk_hist2_dense_kernel<__nv_bfloat16><<<g_strided, THREADS, 0, st>>>(p, s);
+    else topk_hist2_dense_kernel<float><<<g_strided, THREADS, 0, st>>>(p, s);
     CHECK_LAUNCH();
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 4); CHECK_LAUNCH();
     if (bf) topk_filter_kernel<__nv_bfloat16><<<g_tiles, THREADS, 0, st>>>(p, s);
