@@ -78,9 +78,12 @@ constexpr int SEL_LO1 = 9;        // lowest / highest non-empty bin of the first
 constexpr int SEL_HI1 = 10;       // pick reads and clears only that range); reset to ~0 / 0 after use
 constexpr int SEL_LO2 = 11;       // same for the second-digit histogram
 constexpr int SEL_HI2 = 12;
+constexpr int SEL_GUESS = 13;      // uplink: lower bound (31-bit key) tried first in the next step; 0 = none
+constexpr int SEL_MODE = 14;       // uplink, this step: 1 = candidates collected with the guess, 0 = regular two-pass path
 
 // words of the status block (int32 each)
 constexpr int STATUS_WORD = 0;        // failed internal checks
+constexpr int STATUS_ANY_REGULAR = 12; // uplink: some problem takes the regular two-pass path this step
 constexpr int STATUS_ANY_REFINE = 8;  // +0 uplink, +1 downlink: some problem needs the dense second-digit pass
 
 }  // namespace liec

@@ -34,6 +34,7 @@ struct TopkSide {
     uint32_t *meta;                        // [R][TT][4]: pos, cnt, n_greater -> unused, ties allowed
     uint32_t *outbase;                     // [R][TT+1]
     float *zero_out;                       // downlink: error buffer, selected entries become +0
+    int spec;                              // uplink: try last step's threshold first (single dense pass)
 };
 
 static TopkSide make_side(const Params &p, bool uplink) {
@@ -43,11 +44,13 @@ static TopkSide make_side(const Params &p, bool uplink) {
         s.idx = p.up_idx; s.val = p.up_val; s.hist = p.up_hist; s.hist2 = p.up_hist2; s.sel = p.up_sel;
         s.cand_idx = p.up_cand_idx; s.cand_val = p.up_cand_val; s.meta = p.up_tile_meta; s.outbase = p.up_outbase;
         s.zero_out = nullptr;
+        s.spec = 1;
     } else {
         s.src = p.e; s.row_stride = 0; s.R = 1;
         s.idx = p.down_idx; s.val = p.down_val; s.hist = p.down_hist; s.hist2 = p.down_hist2; s.sel = p.down_sel;
         s.cand_idx = p.down_cand_idx; s.cand_val = p.down_cand_val; s.meta = p.down_tile_meta; s.outbase = p.down_outbase;
         s.zero_out = p.e;
+        s.spec = 0;
     }
     return s;
 }
@@ -127,6 +130,24 @@ __device__ PickResult block_pick(const uint32_t *bins, int nbins, uint32_t rank,
 }
 
 // ------------------------------------------------------------------------------------------------
+// Uplink, start of a step: a problem that has a guess (a lower bound for its threshold, taken
+// from the previous step) first tries the single-pass route: candidates are collected with the
+// guess and everything else runs on the candidates.  The guess is only a shortcut: it is
+// checked (at least k candidates, buffer not exceeded) and a problem that fails the check, or
+// has no guess, takes the regular two-pass route in the same step.  The result is the same.
+// ------------------------------------------------------------------------------------------------
+__global__ void topk_begin_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x, row = blockIdx.y;
+    if (t >= p.T) return;
+    uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
+    const bool guess = sel[SEL_GUESS] != 0u;
+    sel[SEL_MODE] = guess ? 1u : 0u;
+    sel[SEL_CAND_COUNT] = 0u;
+    sel[SEL_FLAGS] = 0u;
+    if (!guess) p.status[STATUS_ANY_REGULAR] = 1;
+}
+
+// ------------------------------------------------------------------------------------------------
 // hist1: one CTA per (tile, row)
 // ------------------------------------------------------------------------------------------------
 template <bool FAST>
@@ -143,27 +164,32 @@ __device__ __forceinline__ void hist1_count(uint32_t *h, const float (&v)[8][4],
 template <typename GT>
 __global__ void __launch_bounds__(THREADS) topk_hist1_kernel(const __grid_constant__ Params p, const TopkSide s) {
     __shared__ __align__(16) uint32_t h[DIGIT1_BINS];
+    if (s.spec && p.status[STATUS_ANY_REGULAR] == 0) return;  // every problem went the single-pass route
     const int row = blockIdx.y;
-    const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
-    const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
-    const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
-    float v[8][4];
-    if (fast) {
+    for (int tile = blockIdx.x; tile < p.TT; tile += gridDim.x) {
+        const TileInfo ti = locate_tile(p, tile);
+        uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
+        if (s.spec && sel[SEL_MODE] != 0u) continue;  // uniform over the CTA
+        const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
+        const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
+        const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+        float v[8][4];
+        if (fast) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) load4_stream(tile_ptr + tile_pos(warp, lane, j), v[j]);
-    } else {
+            for (int j = 0; j < 8; ++j) load4_stream(tile_ptr + tile_pos(warp, lane, j), v[j]);
+        } else {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v[j]);
+            for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v[j]);
+        }
+        for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(h)[b] = make_uint4(0u, 0u, 0u, 0u);
+        __syncthreads();
+        if (fast) hist1_count<true>(h, v, warp, lane, ti.len);
+        else hist1_count<false>(h, v, warp, lane, ti.len);
+        __syncthreads();
+        flush_hist(h, s.hist + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS, sel, SEL_LO1, SEL_HI1);
+        __syncthreads();
     }
-    for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(h)[b] = make_uint4(0u, 0u, 0u, 0u);
-    __syncthreads();
-    if (fast) hist1_count<true>(h, v, warp, lane, ti.len);
-    else hist1_count<false>(h, v, warp, lane, ti.len);
-    __syncthreads();
-    flush_hist(h, s.hist + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS,
-               s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS, SEL_LO1, SEL_HI1);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -178,19 +204,24 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
     // level 1: first digit.  level 4: second digit of "refined" problems (after their dense
     // second-digit pass).  level 2: second digit of regular problems.  level 3: last 7 bits.
-    const uint32_t flags_in = level == 1 ? 0u : sel[SEL_FLAGS];
+    // level 5 (uplink): first digit from the histogram of the candidates collected with the guess;
+    // checks the guess.
+    if (level == 5 && sel[SEL_MODE] != 1u) return;
+    if (level == 1 && s.spec && sel[SEL_MODE] != 0u) return;
+    const uint32_t flags_in = (level == 1 || level == 5) ? 0u : sel[SEL_FLAGS];
     if (level == 4 && t == 0 && row == 0 && threadIdx.x == 0) p.status[STATUS_ANY_REFINE + (s.zero_out ? 1 : 0)] = 0;
     if (level == 4 && flags_in != 2u) return;
     if (level == 2 && flags_in != 0u) return;
     if (level == 3 && (flags_in & 1u)) return;  // slow path finishes on its own
     const int nbins = level == 3 ? 128 : DIGIT1_BINS;
-    uint32_t *gh = (level == 1 ? s.hist : s.hist2) + ((int64_t)row * p.T + t) * DIGIT1_BINS;
+    uint32_t *gh = ((level == 1 || level == 5) ? s.hist : s.hist2) + ((int64_t)row * p.T + t) * DIGIT1_BINS;
     if (nbins == DIGIT1_BINS) {
         // only the recorded non-empty range is read and cleared
         const int lo_word = level == 1 ? SEL_LO1 : SEL_LO2, hi_word = level == 1 ? SEL_HI1 : SEL_HI2;
         // (the filter does not record the range of the second-digit histogram: level 2 reads all of it)
-        const uint32_t lo = level == 2 ? 0u : min(sel[lo_word], (uint32_t)DIGIT1_BINS);
-        const uint32_t hi = level == 2 ? (uint32_t)DIGIT1_BINS - 1u : min(sel[hi_word], (uint32_t)DIGIT1_BINS - 1u);
+        const bool full = level == 2 || level == 5;  // histograms filled by untracked atomics
+        const uint32_t lo = full ? 0u : min(sel[lo_word], (uint32_t)DIGIT1_BINS);
+        const uint32_t hi = full ? (uint32_t)DIGIT1_BINS - 1u : min(sel[hi_word], (uint32_t)DIGIT1_BINS - 1u);
         for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(bins)[b] = make_uint4(0u, 0u, 0u, 0u);
         __syncthreads();
         for (uint32_t b = lo + threadIdx.x; b <= hi; b += THREADS) {
@@ -198,7 +229,7 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
             if (c) { bins[b] = c; gh[b] = 0u; }
         }
         __syncthreads();
-        if (threadIdx.x == 0) { sel[lo_word] = 0xffffffffu; sel[hi_word] = 0u; }
+        if (threadIdx.x == 0 && !full) { sel[lo_word] = 0xffffffffu; sel[hi_word] = 0u; }
     } else {
         for (int b = threadIdx.x; b < nbins; b += THREADS) {
             bins[b] = gh[b];
@@ -207,9 +238,21 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
     }
     __syncthreads();
     const uint32_t k = (uint32_t)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
-    const uint32_t rank = level == 1 ? k : sel[SEL_REMAIN];
+    const uint32_t rank = (level == 1 || level == 5) ? k : sel[SEL_REMAIN];
     const PickResult r = block_pick(bins, nbins, rank, scratch);
     if (threadIdx.x == 0) {
+        if (level == 5) {
+            if (!r.ok) {  // fewer than k candidates: the guess was too high, take the regular route
+                sel[SEL_MODE] = 0u;
+                p.status[STATUS_ANY_REGULAR] = 1;
+            } else {
+                sel[SEL_PREFIX] = r.bin;
+                sel[SEL_REMAIN] = r.rank_in_bin;
+                sel[SEL_ABOVE] = r.count_ge - bins[r.bin];
+                sel[SEL_NCAND] = sel[SEL_CAND_COUNT];
+            }
+            return;
+        }
         if (!r.ok) { atomicOr(p.status, STATUS_PICK_RANK); return; }
         const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
         if (level == 1) {
@@ -226,13 +269,18 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
             sel[SEL_PREFIX] = (sel[SEL_PREFIX] << 12) | r.bin;
             sel[SEL_REMAIN] = r.rank_in_bin;
             sel[SEL_NCAND] = ncand;
-            if (ncand > cap) sel[SEL_FLAGS] = 3u;  // still too many (huge groups of equal keys): slow path
+            if (ncand > cap) { sel[SEL_FLAGS] = 3u; sel[SEL_GUESS] = 0u; }  // still too many (huge groups of equal keys): slow path
         } else if (level == 2) {
             sel[SEL_PREFIX] = (sel[SEL_PREFIX] << 12) | r.bin;
             sel[SEL_REMAIN] = r.rank_in_bin;
         } else {
-            sel[SEL_THRESH] = (sel[SEL_PREFIX] << 7) | r.bin;
+            const uint32_t thresh = (sel[SEL_PREFIX] << 7) | r.bin;
+            sel[SEL_THRESH] = thresh;
             sel[SEL_TIES] = r.rank_in_bin;
+            if (s.spec) {  // next step's guess: one first-digit bin below this threshold's bin
+                const uint32_t b1 = thresh >> DIGIT1_SHIFT;
+                sel[SEL_GUESS] = (flags_in == 0u && b1 >= 1u) ? (b1 - 1u) << DIGIT1_SHIFT : 0u;
+            }
         }
     }
 }
@@ -292,101 +340,123 @@ __device__ __forceinline__ uint32_t filter_mask(const float (&v)[8][4], float lo
     return mask;
 }
 
-template <typename GT>
+// SPEC = true: the uplink's first pass of a step, for problems that have a guess; candidates are
+// the entries at or above the guess.  SPEC = false: the regular pass (threshold bin known from the
+// histogram); on the uplink it only serves the problems that did not take the single-pass route.
+template <typename GT, bool SPEC>
 __global__ void __launch_bounds__(THREADS, 4) topk_filter_kernel(const __grid_constant__ Params p, const TopkSide s) {
     __shared__ uint32_t warp_tot[8];
     __shared__ uint32_t tile_base;
+    if (!SPEC && s.spec && p.status[STATUS_ANY_REGULAR] == 0) return;
     const int row = blockIdx.y;
-    const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
-    const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
-    const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
-    // the streaming loads do not depend on the selection state: issue them first
-    float v[8][4];
-    if (fast) {
+    for (int tile = blockIdx.x; tile < p.TT; tile += gridDim.x) {
+        const TileInfo ti = locate_tile(p, tile);
+        const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
+        const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
+        const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+        uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
+        if (!SPEC && s.spec && sel[SEL_MODE] != 0u) continue;  // (all `continue`s before the barriers are uniform)
+        // the streaming loads do not depend on the selection state: issue them first
+        float v[8][4];
+        if (fast) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) load4_stream(tile_ptr + tile_pos(warp, lane, j), v[j]);
-    } else {
+            for (int j = 0; j < 8; ++j) load4_stream(tile_ptr + tile_pos(warp, lane, j), v[j]);
+        } else {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v[j]);
-    }
-    uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
-    const uint32_t flags = sel[SEL_FLAGS];
-    if (flags & 1u) return;
-    // regular problems compare the first digit, refined ones the 24-bit prefix: either way a
-    // candidate is an entry whose key is at least the prefix shifted back into place
-    const bool refined = flags == 2u;
-    const uint32_t prefix = sel[SEL_PREFIX];
-    const float low = __uint_as_float(prefix << (refined ? 7 : DIGIT1_SHIFT));
-    const uint32_t mask = fast ? filter_mask<true>(v, low, warp, lane, ti.len)
-                               : filter_mask<false>(v, low, warp, lane, ti.len);
-    // per-row counts packed as bytes (rows 0-3, rows 4-7), inclusive scan over lanes
-    uint32_t cnt_lo = 0, cnt_hi = 0;
+            for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v[j]);
+        }
+        float low;
+        bool refined = false;
+        uint32_t prefix = 0;
+        if (SPEC) {
+            if (sel[SEL_MODE] != 1u) continue;
+            low = __uint_as_float(sel[SEL_GUESS]);
+        } else {
+            const uint32_t flags = sel[SEL_FLAGS];
+            if (flags & 1u) continue;
+            // regular problems compare the first digit, refined ones the 24-bit prefix: either way a
+            // candidate is an entry whose key is at least the prefix shifted back into place
+            refined = flags == 2u;
+            prefix = sel[SEL_PREFIX];
+            low = __uint_as_float(prefix << (refined ? 7 : DIGIT1_SHIFT));
+        }
+        const uint32_t mask = fast ? filter_mask<true>(v, low, warp, lane, ti.len)
+                                   : filter_mask<false>(v, low, warp, lane, ti.len);
+        // per-row counts packed as bytes (rows 0-3, rows 4-7), inclusive scan over lanes
+        uint32_t cnt_lo = 0, cnt_hi = 0;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        cnt_lo |= (uint32_t)__popc((mask >> (4 * j)) & 0xfu) << (8 * j);
-        cnt_hi |= (uint32_t)__popc((mask >> (4 * j + 16)) & 0xfu) << (8 * j);
-    }
-    uint32_t inc_lo = cnt_lo, inc_hi = cnt_hi;
+        for (int j = 0; j < 4; ++j) {
+            cnt_lo |= (uint32_t)__popc((mask >> (4 * j)) & 0xfu) << (8 * j);
+            cnt_hi |= (uint32_t)__popc((mask >> (4 * j + 16)) & 0xfu) << (8 * j);
+        }
+        uint32_t inc_lo = cnt_lo, inc_hi = cnt_hi;
 #pragma unroll
-    for (int m = 1; m < 32; m <<= 1) {
-        const uint32_t a = __shfl_up_sync(0xffffffffu, inc_lo, m), b = __shfl_up_sync(0xffffffffu, inc_hi, m);
-        if (lane >= m) { inc_lo += a; inc_hi += b; }
-    }
-    const uint32_t tot_lo = __shfl_sync(0xffffffffu, inc_lo, 31), tot_hi = __shfl_sync(0xffffffffu, inc_hi, 31);
-    const uint32_t exc_lo = inc_lo - cnt_lo, exc_hi = inc_hi - cnt_hi;
-    // running row bases of the warp, again packed (a warp holds at most 1024 candidates: 16-bit fields)
-    uint32_t running = 0;
-    uint32_t base01 = 0, base23 = 0, base45 = 0, base67 = 0;
+        for (int m = 1; m < 32; m <<= 1) {
+            const uint32_t a = __shfl_up_sync(0xffffffffu, inc_lo, m), b = __shfl_up_sync(0xffffffffu, inc_hi, m);
+            if (lane >= m) { inc_lo += a; inc_hi += b; }
+        }
+        const uint32_t tot_lo = __shfl_sync(0xffffffffu, inc_lo, 31), tot_hi = __shfl_sync(0xffffffffu, inc_hi, 31);
+        const uint32_t exc_lo = inc_lo - cnt_lo, exc_hi = inc_hi - cnt_hi;
+        // running row bases of the warp, again packed (a warp holds at most 1024 candidates: 16-bit fields)
+        uint32_t running = 0;
+        uint32_t base01 = 0, base23 = 0, base45 = 0, base67 = 0;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const uint32_t total = ((j < 4 ? tot_lo : tot_hi) >> (8 * (j & 3))) & 0xffu;
-        const uint32_t field = running << (16 * (j & 1));
-        if (j < 2) base01 |= field; else if (j < 4) base23 |= field; else if (j < 6) base45 |= field; else base67 |= field;
-        running += total;
-    }
-    if (lane == 0) warp_tot[warp] = running;
-    __syncthreads();
-    uint32_t warp_off = 0, tile_cnt = 0;
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t total = ((j < 4 ? tot_lo : tot_hi) >> (8 * (j & 3))) & 0xffu;
+            const uint32_t field = running << (16 * (j & 1));
+            if (j < 2) base01 |= field; else if (j < 4) base23 |= field; else if (j < 6) base45 |= field; else base67 |= field;
+            running += total;
+        }
+        if (lane == 0) warp_tot[warp] = running;
+        __syncthreads();
+        uint32_t warp_off = 0, tile_cnt = 0;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) {
-        if (w < warp) warp_off += warp_tot[w];
-        tile_cnt += warp_tot[w];
-    }
-    if (threadIdx.x == 0) {
-        const uint32_t cap = (uint32_t)(__ldg(p.cap_off + ti.t + 1) - __ldg(p.cap_off + ti.t));
-        uint32_t pos0 = tile_cnt ? atomicAdd(&sel[SEL_CAND_COUNT], tile_cnt) : 0u;
-        if (pos0 + tile_cnt > cap) { atomicOr(p.status, STATUS_CAND_OVERFLOW); pos0 = 0xffffffffu; }
-        tile_base = pos0;
-        uint32_t *m = s.meta + ((int64_t)row * p.TT + blockIdx.x) * 4;
-        m[0] = pos0 == 0xffffffffu ? 0u : pos0;
-        m[1] = pos0 == 0xffffffffu ? 0u : tile_cnt;
-    }
-    __syncthreads();
-    if (tile_base == 0xffffffffu || mask == 0u) return;
-    const int64_t cbase = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + tile_base + warp_off;
-    uint32_t *gh2 = s.hist2 + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS;
-    const uint32_t flat0 = (uint32_t)(ti.seg_beg + ti.rel);
-    // walk the set bits (candidates are rare: usually zero or one iteration)
-    uint32_t rest = mask;
-    while (rest) {
-        const int b = __ffs(rest) - 1;
-        rest &= rest - 1;
-        const int j = b >> 2;
-        const uint32_t base_pair = j < 2 ? base01 : j < 4 ? base23 : j < 6 ? base45 : base67;
-        const uint32_t row_base = (base_pair >> (16 * (j & 1))) & 0xffffu;
-        const uint32_t before = ((j < 4 ? exc_lo : exc_hi) >> (8 * (j & 3))) & 0xffu;
-        const uint32_t lower = __popc(mask & ((1u << b) - 1u) & (0xfu << (4 * j)));
-        const uint32_t o = row_base + before + lower;
-        const int pos = tile_pos(warp, lane, j) + (b & 3);
-        const float val = load1(tile_ptr + pos);  // read again (cached) rather than kept across the barrier
-        const uint32_t key = key_of(val);
-        s.cand_idx[cbase + o] = flat0 + pos;
-        s.cand_val[cbase + o] = val;
-        if (!refined && (key >> DIGIT1_SHIFT) == prefix) {
-            const uint32_t d2 = (key >> 7) & 0xfffu;
-            atomicAdd(gh2 + d2, 1u);  // (range not tracked here: two more contended atomics cost more than they save)
+        for (int w = 0; w < 8; ++w) {
+            if (w < warp) warp_off += warp_tot[w];
+            tile_cnt += warp_tot[w];
+        }
+        if (threadIdx.x == 0) {
+            const uint32_t cap = (uint32_t)(__ldg(p.cap_off + ti.t + 1) - __ldg(p.cap_off + ti.t));
+            uint32_t pos0 = tile_cnt ? atomicAdd(&sel[SEL_CAND_COUNT], tile_cnt) : 0u;
+            if (pos0 + tile_cnt > cap) {
+                if (SPEC) {  // the guess lets too much through: this problem takes the regular route
+                    sel[SEL_MODE] = 0u;
+                    p.status[STATUS_ANY_REGULAR] = 1;
+                } else {
+                    atomicOr(p.status, STATUS_CAND_OVERFLOW);
+                }
+                pos0 = 0xffffffffu;
+            }
+            tile_base = pos0;
+            uint32_t *m = s.meta + ((int64_t)row * p.TT + tile) * 4;
+            m[0] = pos0 == 0xffffffffu ? 0u : pos0;
+            m[1] = pos0 == 0xffffffffu ? 0u : tile_cnt;
+        }
+        __syncthreads();
+        const uint32_t base_now = tile_base;
+        if (base_now == 0xffffffffu || mask == 0u) continue;
+        const int64_t cbase = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + base_now + warp_off;
+        uint32_t *gh2 = s.hist2 + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS;
+        const uint32_t flat0 = (uint32_t)(ti.seg_beg + ti.rel);
+        // walk the set bits (candidates are rare: usually zero or one iteration)
+        uint32_t rest = mask;
+        while (rest) {
+            const int b = __ffs(rest) - 1;
+            rest &= rest - 1;
+            const int j = b >> 2;
+            const uint32_t base_pair = j < 2 ? base01 : j < 4 ? base23 : j < 6 ? base45 : base67;
+            const uint32_t row_base = (base_pair >> (16 * (j & 1))) & 0xffffu;
+            const uint32_t before = ((j < 4 ? exc_lo : exc_hi) >> (8 * (j & 3))) & 0xffu;
+            const uint32_t lower = __popc(mask & ((1u << b) - 1u) & (0xfu << (4 * j)));
+            const uint32_t o = row_base + before + lower;
+            const int pos = tile_pos(warp, lane, j) + (b & 3);
+            const float val = load1(tile_ptr + pos);  // read again (cached) rather than kept across the barrier
+            const uint32_t key = key_of(val);
+            s.cand_idx[cbase + o] = flat0 + pos;
+            s.cand_val[cbase + o] = val;
+            if (!SPEC && !refined && (key >> DIGIT1_SHIFT) == prefix)
+                atomicAdd(gh2 + ((key >> 7) & 0xfffu), 1u);  // (range not tracked: two more contended atomics cost more than they save)
         }
     }
 }
@@ -421,6 +491,31 @@ __global__ void __launch_bounds__(THREADS) topk_hist3_kernel(const __grid_consta
     for (uint32_t q = lane; q < cb.cnt; q += 32) {
         const uint32_t key = key_of(s.cand_val[cb.base + q]);
         if ((key >> 7) == prefix24) atomicAdd(gh + (key & 0x7fu), 1u);
+    }
+}
+
+// Histograms over the candidates of the problems on the single-pass route (one warp per tile
+// block).  level 0: first digit of every candidate; level 1: second digit of the candidates whose
+// first digit is the threshold's.  Lanes holding the same digit add once (match + leader).
+__global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_constant__ Params p, const TopkSide s,
+                                                                  const int level) {
+    const int row = blockIdx.y, lane = threadIdx.x & 31;
+    const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (tile >= p.TT) return;
+    const CandBlock cb = cand_block(p, s, tile, row);
+    if (cb.skip || cb.sel[SEL_MODE] != 1u) return;
+    const uint32_t b1 = cb.sel[SEL_PREFIX];
+    uint32_t *gh = (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
+    for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
+        const uint32_t q = c0 + lane;
+        uint32_t digit = 0xffffffffu;  // lanes with nothing to add
+        if (q < cb.cnt) {
+            const uint32_t key = key_of(s.cand_val[cb.base + q]);
+            if (level == 0) digit = key >> DIGIT1_SHIFT;
+            else if ((key >> DIGIT1_SHIFT) == b1) digit = (key >> 7) & 0xfffu;
+        }
+        const uint32_t same = __match_any_sync(0xffffffffu, digit);
+        if (digit != 0xffffffffu && lane == __ffs(same) - 1) atomicAdd(gh + digit, (uint32_t)__popc(same));
     }
 }
 
@@ -537,6 +632,8 @@ __global__ void __launch_bounds__(THREADS) topk_slow_kernel(const __grid_constan
     __shared__ uint32_t wa[8], wb[8];
     const int t = blockIdx.x, row = blockIdx.y;
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
+    // last kernel of a side: the next step starts with "no problem on the regular route yet"
+    if (s.spec && t == 0 && row == 0 && threadIdx.x == 0) p.status[STATUS_ANY_REGULAR] = 0;
     if (!(sel[SEL_FLAGS] & 1u)) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t seg_beg = __ldg(p.seg_off + t);
@@ -731,11 +828,28 @@ __global__ void __launch_bounds__(THREADS) server_topk_kernel(const __grid_const
         ++*launches;                                     \
     } while (0)
 
+// Grid of the dense passes that usually have nothing to do on the uplink (their CTAs walk the
+// tiles with a stride and leave at once when no problem takes the regular route).
+static dim3 strided_grid(const Params &p, int rows) { return dim3(p.TT < 592 ? p.TT : 592, rows); }
+
+// First dense pass.  Uplink: collect candidates with last step's guess, histogram them and
+// check the guess; then the first-digit histogram for the problems left on the regular route.
+// Downlink without a fused histogram: plain first-digit histogram of v.
 cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int64_t *launches) {
     const TopkSide s = make_side(p, uplink);
-    dim3 g_tiles(p.TT, s.R);
-    if (uplink && p.gdt == DT_BF16) topk_hist1_kernel<__nv_bfloat16><<<g_tiles, THREADS, 0, st>>>(p, s);
-    else topk_hist1_kernel<float><<<g_tiles, THREADS, 0, st>>>(p, s);
+    dim3 g_tiles(p.TT, s.R), g_probs(p.T, s.R), g_warp_tiles((p.TT + 7) / 8, s.R);
+    const bool bf = uplink && p.gdt == DT_BF16;
+    if (s.spec) {
+        topk_begin_kernel<<<dim3((p.T + 127) / 128, s.R), 128, 0, st>>>(p, s); CHECK_LAUNCH();
+        if (bf) topk_filter_kernel<__nv_bfloat16, true><<<g_tiles, THREADS, 0, st>>>(p, s);
+        else topk_filter_kernel<float, true><<<g_tiles, THREADS, 0, st>>>(p, s);
+        CHECK_LAUNCH();
+        topk_cand_hist_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s, 0); CHECK_LAUNCH();
+        topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 5); CHECK_LAUNCH();
+    }
+    const dim3 g_hist = s.spec ? strided_grid(p, s.R) : g_tiles;
+    if (bf) topk_hist1_kernel<__nv_bfloat16><<<g_hist, THREADS, 0, st>>>(p, s);
+    else topk_hist1_kernel<float><<<g_hist, THREADS, 0, st>>>(p, s);
     CHECK_LAUNCH();
     return cudaSuccess;
 }
@@ -744,19 +858,19 @@ cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int
 // downlink the zeroing of the selected error entries.
 cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, int64_t *launches) {
     const TopkSide s = make_side(p, uplink);
-    dim3 g_tiles(p.TT, s.R), g_probs(p.T, s.R);
+    dim3 g_tiles(p.TT, s.R), g_probs(p.T, s.R), g_warp_tiles((p.TT + 7) / 8, s.R);
     const bool bf = uplink && p.gdt == DT_BF16;
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 1); CHECK_LAUNCH();
-    dim3 g_strided(p.TT < 592 ? p.TT : 592, s.R);
-    if (bf) topk_hist2_dense_kernel<__nv_bfloat16><<<g_strided, THREADS, 0, st>>>(p, s);
-    else topk_hist2_dense_kernel<float><<<g_strided, THREADS, 0, st>>>(p, s);
+    if (bf) topk_hist2_dense_kernel<__nv_bfloat16><<<strided_grid(p, s.R), THREADS, 0, st>>>(p, s);
+    else topk_hist2_dense_kernel<float><<<strided_grid(p, s.R), THREADS, 0, st>>>(p, s);
     CHECK_LAUNCH();
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 4); CHECK_LAUNCH();
-    if (bf) topk_filter_kernel<__nv_bfloat16><<<g_tiles, THREADS, 0, st>>>(p, s);
-    else topk_filter_kernel<float><<<g_tiles, THREADS, 0, st>>>(p, s);
+    const dim3 g_filter = s.spec ? strided_grid(p, s.R) : g_tiles;
+    if (bf) topk_filter_kernel<__nv_bfloat16, false><<<g_filter, THREADS, 0, st>>>(p, s);
+    else topk_filter_kernel<float, false><<<g_filter, THREADS, 0, st>>>(p, s);
     CHECK_LAUNCH();
+    if (s.spec) { topk_cand_hist_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s, 1); CHECK_LAUNCH(); }
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();
-    dim3 g_warp_tiles((p.TT + 7) / 8, s.R);
     topk_hist3_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 3); CHECK_LAUNCH();
     topk_count_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();

@@ -74,6 +74,21 @@ def test_crowded_threshold_bin_uses_second_digit():
         P.step(G, 0.1)
 
 
+def test_guess_from_previous_step_can_be_wrong():
+    """The uplink first tries last step's threshold as a lower bound.  Gradients whose scale jumps
+    down (too few candidates) or up (too many) between steps must fall back to the full selection
+    and still give the oracle's result; steady scales take the short route."""
+    lay = Layout("jumps", (40000, 8192, 3 * 8192 + 17, 500))
+    k = topk_counts(lay, 1, 100)
+    P = _pair(3, lay.seg_offsets, TOPK, TOPK, k=k)
+    scales = [1.0, 1.0, 1e-3, 1e-3, 50.0, 50.0, 1.0, 0.0, 1.0, 1.0]
+    for step, sc in enumerate(scales):
+        G = make_gradients("normal", 1.0, 3, lay.dim, step, base_seed=23) * sc
+        if step == 5:
+            G[1] *= 1e-4          # one worker alone changes scale
+        P.step(G, 0.1)
+
+
 def test_all_zero_and_mostly_zero_gradients():
     lay = Layout("zeros", (5000, 20000))
     k = np.asarray([50, 200], np.int64)
