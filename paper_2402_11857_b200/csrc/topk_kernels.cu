@@ -86,25 +86,29 @@ __device__ __forceinline__ void flush_hist(const uint32_t *h, uint32_t *gh, uint
 struct PickResult { uint32_t bin, rank_in_bin, count_ge; bool ok; };
 
 __device__ PickResult block_pick(const uint32_t *bins, int nbins, uint32_t rank, uint32_t *scratch /*[THREADS+4]*/) {
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int per = nbins >= THREADS ? nbins / THREADS : 1;
     const int active = nbins / per;
     uint32_t mine = 0;
     if (tid < active)
         for (int q = 0; q < per; ++q) mine += bins[tid * per + q];
-    // inclusive suffix sum over threads: suf[i] = sum_{i' >= i} mine[i']
-    scratch[tid] = mine;
-    __syncthreads();
-    for (int offs = 1; offs < THREADS; offs <<= 1) {
-        uint32_t add = (tid + offs < THREADS) ? scratch[tid + offs] : 0u;
-        __syncthreads();
-        scratch[tid] += add;
-        __syncthreads();
+    // inclusive suffix sum over threads (higher thread = higher bins): shuffles inside a warp,
+    // then the totals of the warps above
+    uint32_t suf = mine;
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const uint32_t up = __shfl_down_sync(0xffffffffu, suf, m);
+        if (lane + m < 32) suf += up;
     }
-    const uint32_t suf_incl = scratch[tid];
-    const uint32_t suf_excl = suf_incl - mine;
+    if (lane == 0) scratch[warp] = suf;  // warp total
     if (tid == 0) scratch[THREADS + 3] = 0u;  // found flag
     __syncthreads();
+    uint32_t above_warps = 0;
+#pragma unroll
+    for (int w = 0; w < THREADS / 32; ++w)
+        if (w > warp) above_warps += scratch[w];
+    const uint32_t suf_incl = suf + above_warps;
+    const uint32_t suf_excl = suf_incl - mine;
     if (tid < active && suf_excl < rank && rank <= suf_incl) {
         uint32_t above = suf_excl;
         for (int q = per - 1; q >= 0; --q) {
@@ -217,9 +221,11 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
     uint32_t *gh = ((level == 1 || level == 5) ? s.hist : s.hist2) + ((int64_t)row * p.T + t) * DIGIT1_BINS;
     if (nbins == DIGIT1_BINS) {
         // only the recorded non-empty range is read and cleared
-        const int lo_word = level == 1 ? SEL_LO1 : SEL_LO2, hi_word = level == 1 ? SEL_HI1 : SEL_HI2;
+        const bool first = level == 1 || level == 5;
+        const int lo_word = first ? SEL_LO1 : SEL_LO2, hi_word = first ? SEL_HI1 : SEL_HI2;
         // (the filter does not record the range of the second-digit histogram: level 2 reads all of it)
-        const bool full = level == 2 || level == 5;  // histograms filled by untracked atomics
+        // the regular filter fills the second-digit histogram with untracked atomics
+        const bool full = level == 2 && !(s.spec && sel[SEL_MODE] == 1u);
         const uint32_t lo = full ? 0u : min(sel[lo_word], (uint32_t)DIGIT1_BINS);
         const uint32_t hi = full ? (uint32_t)DIGIT1_BINS - 1u : min(sel[hi_word], (uint32_t)DIGIT1_BINS - 1u);
         for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(bins)[b] = make_uint4(0u, 0u, 0u, 0u);
@@ -229,7 +235,7 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
             if (c) { bins[b] = c; gh[b] = 0u; }
         }
         __syncthreads();
-        if (threadIdx.x == 0 && !full) { sel[lo_word] = 0xffffffffu; sel[hi_word] = 0u; }
+        if (threadIdx.x == 0) { sel[lo_word] = 0xffffffffu; sel[hi_word] = 0u; }
     } else {
         for (int b = threadIdx.x; b < nbins; b += THREADS) {
             bins[b] = gh[b];
@@ -506,6 +512,7 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
     if (cb.skip || cb.sel[SEL_MODE] != 1u) return;
     const uint32_t b1 = cb.sel[SEL_PREFIX];
     uint32_t *gh = (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
+    uint32_t lo = 0xffffffffu, hi = 0u;
     for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
         const uint32_t q = c0 + lane;
         uint32_t digit = 0xffffffffu;  // lanes with nothing to add
@@ -515,7 +522,18 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
             else if ((key >> DIGIT1_SHIFT) == b1) digit = (key >> 7) & 0xfffu;
         }
         const uint32_t same = __match_any_sync(0xffffffffu, digit);
-        if (digit != 0xffffffffu && lane == __ffs(same) - 1) atomicAdd(gh + digit, (uint32_t)__popc(same));
+        if (digit != 0xffffffffu) {
+            if (lane == __ffs(same) - 1) atomicAdd(gh + digit, (uint32_t)__popc(same));
+            lo = min(lo, digit);
+            hi = max(hi, digit);
+        }
+    }
+    // the non-empty bin range, so that the pick reads and clears only that
+    lo = __reduce_min_sync(0xffffffffu, lo);
+    hi = __reduce_max_sync(0xffffffffu, hi);
+    if (lane == 0 && lo != 0xffffffffu) {
+        atomicMin(&cb.sel[level == 0 ? SEL_LO1 : SEL_LO2], lo);
+        atomicMax(&cb.sel[level == 0 ? SEL_HI1 : SEL_HI2], hi);
     }
 }
 
