@@ -102,6 +102,18 @@ typedef struct {
  */
 size_t liec_workspace_bytes(const liec_config *cfg);
 
+/*
+ * Bytes that one compressed iteration puts on the wire per worker: its uplink message, the
+ * downlink message it receives, and, for comparison, one full-precision vector (4 d bytes; what
+ * P-SGD sends each way and what a model-averaging iteration of Algorithm 1 is charged per
+ * direction).  This is the accounting behind the paper's "communication cost per iteration"
+ * column (Table of results on CIFAR): total = N * (uplink + downlink).  Pure host arithmetic;
+ * any output pointer may be NULL.  Returns LIEC_ERR_INVALID_ARG / LIEC_ERR_UNSUPPORTED for a bad
+ * configuration.
+ */
+liec_status liec_wire_bytes(const liec_config *cfg, int64_t *uplink_bytes, int64_t *downlink_bytes,
+                            int64_t *full_precision_bytes);
+
 /* Bytes of the downlink message as copied out by liec_step_host (0 for identity/invalid). */
 size_t liec_down_message_bytes(const liec_config *cfg);
 

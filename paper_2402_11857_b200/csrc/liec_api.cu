@@ -212,6 +212,26 @@ size_t liec_workspace_bytes(const liec_config *cfg) {
     return pl.total;
 }
 
+liec_status liec_wire_bytes(const liec_config *cfg, int64_t *uplink_bytes, int64_t *downlink_bytes,
+                            int64_t *full_precision_bytes) {
+    Plan pl;
+    std::string msg;
+    liec_status st = make_plan(cfg, pl, &msg);
+    if (st != LIEC_OK) {
+        snprintf(g_no_ctx_error, sizeof(g_no_ctx_error), "%s", msg.c_str());
+        return st;
+    }
+    auto message = [&](int32_t comp) -> int64_t {
+        if (comp == LIEC_COMP_SCALED_SIGN) return 4 * (pl.W + (int64_t)pl.T);  // packed signs + one scale per segment
+        if (comp == LIEC_COMP_TOPK) return 8 * pl.K;                             // (index, value) pairs
+        return 4 * pl.d;                                                          // identity: the dense vector
+    };
+    if (uplink_bytes) *uplink_bytes = message(cfg->uplink);
+    if (downlink_bytes) *downlink_bytes = message(cfg->downlink);
+    if (full_precision_bytes) *full_precision_bytes = 4 * pl.d;
+    return LIEC_OK;
+}
+
 size_t liec_down_message_bytes(const liec_config *cfg) {
     Plan pl;
     if (make_plan(cfg, pl, nullptr) != LIEC_OK) return 0;

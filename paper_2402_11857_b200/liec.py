@@ -52,6 +52,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     vp, cfgp = C.c_void_p, C.POINTER(liec_config)
     lib.liec_workspace_bytes.argtypes = [cfgp]
     lib.liec_workspace_bytes.restype = C.c_size_t
+    lib.liec_wire_bytes.argtypes = [cfgp, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+    lib.liec_wire_bytes.restype = C.c_int
     lib.liec_down_message_bytes.argtypes = [cfgp]
     lib.liec_down_message_bytes.restype = C.c_size_t
     lib.liec_init.argtypes = [cfgp, vp, vp, vp, C.c_size_t, C.POINTER(vp)]
@@ -105,6 +107,16 @@ def make_config(num_workers: int, seg_offsets: Sequence[int], uplink: int, downl
 
 def workspace_bytes(cfg: liec_config) -> int:
     return int(load_library().liec_workspace_bytes(C.byref(cfg)))
+
+
+def liec_wire_bytes(cfg: liec_config):
+    """(uplink, downlink, full-precision) bytes per worker and iteration."""
+    lib = load_library()
+    up, down, full = C.c_int64(0), C.c_int64(0), C.c_int64(0)
+    st = lib.liec_wire_bytes(C.byref(cfg), C.byref(up), C.byref(down), C.byref(full))
+    if st != 0:
+        raise LiecError(st, lib.liec_last_error(None).decode())
+    return int(up.value), int(down.value), int(full.value)
 
 
 def down_message_bytes(cfg: liec_config) -> int:
