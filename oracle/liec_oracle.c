@@ -40,6 +40,11 @@
  *   - Sign message layout: segment t owns ceil(n_t/32) 32-bit words; bit b of
  *     word w is set iff element off[t]+32w+b is negative; padding bits are 0.
  *
+ * The model-averaging iteration of Algorithm 1 (taken when (t+1) mod floor(1/delta) == 0; the
+ * experiments use a fixed period of 32 or 100) is liec_oracle_average_step below: gradients and
+ * models travel uncompressed, p = v, the global error becomes 0 and every worker restarts from the
+ * averaged model.
+ *
  * Parity pins (tests/test_oracle_*.py): hand-worked iterations, exact rational
  * means, brute-force bit packing and sorting, the contraction identities of
  * Def. 1, p + e' = v, Lemma 3, identity compressor with N=1 reducing to SGD.
@@ -252,4 +257,52 @@ int liec_oracle_step(int32_t N, int64_t d, int32_t T, const int64_t *off,
 done:
     free(P); free(v); free(p); free(tw); free(ts); free(ti); free(tv);
     return rc;
+}
+
+/*
+ * Model-averaging iteration of Algorithm 1 (the branch with (t+1) mod period == 0):
+ *   p^i = g^i,   v = e + (1/N) sum_i g^i,   p = v,   e' = v - p = 0,
+ *   xbar = (1/N) sum_i x^i,   x^i <- xbar - eta (p - p^i + g^i).
+ * Same arithmetic readings as the compressed iteration: sums over workers run in worker order
+ * in binary32 from +0 and are divided by (float)N; the update is ((p - p^i) + g), times eta,
+ * subtracted from xbar.  Optional outputs v_out [d] and xbar_out [d].
+ * Also used for the algorithm's final output, xbar_T = mean_i x_T^i (liec_oracle_mean_params).
+ */
+void liec_oracle_mean_params(int32_t N, int64_t d, const float *X, float *xbar)
+{
+    for (int64_t j = 0; j < d; ++j) {
+        float acc = 0.0f;
+        for (int32_t i = 0; i < N; ++i) acc = acc + X[(size_t)i * d + j];
+        xbar[j] = acc / (float)N;
+    }
+}
+
+int liec_oracle_average_step(int32_t N, int64_t d, const float *G, float lr, float *X, float *e,
+                             float *v_out, float *xbar_out)
+{
+    float *v = (float *)malloc((size_t)d * sizeof(float));
+    float *xbar = (float *)malloc((size_t)d * sizeof(float));
+    if (!v || !xbar) { free(v); free(xbar); return -1; }
+    for (int64_t j = 0; j < d; ++j) {
+        float acc = 0.0f;
+        for (int32_t i = 0; i < N; ++i) acc = acc + G[(size_t)i * d + j];
+        float gmean = acc / (float)N;
+        v[j] = e[j] + gmean;
+    }
+    liec_oracle_mean_params(N, d, X, xbar);
+    for (int32_t i = 0; i < N; ++i) {
+        const float *g = G + (size_t)i * d;
+        float *x = X + (size_t)i * d;
+        for (int64_t j = 0; j < d; ++j) {
+            float delta = v[j] - g[j];    /* p - p^i with p = v, p^i = g^i */
+            float upd = delta + g[j];
+            float scaled = lr * upd;
+            x[j] = xbar[j] - scaled;
+        }
+    }
+    for (int64_t j = 0; j < d; ++j) e[j] = v[j] - v[j];   /* e' = v - p, p = v */
+    if (v_out) memcpy(v_out, v, (size_t)d * sizeof(float));
+    if (xbar_out) memcpy(xbar_out, xbar, (size_t)d * sizeof(float));
+    free(v); free(xbar);
+    return 0;
 }

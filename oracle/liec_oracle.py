@@ -53,6 +53,10 @@ def _bind(lib: C.CDLL) -> C.CDLL:
     lib.liec_oracle_step.argtypes = [C.c_int32, C.c_int64, C.c_int32, p, C.c_int32, C.c_int32, p,
                                      p, C.c_float, p, p] + [p] * 9
     lib.liec_oracle_step.restype = C.c_int
+    lib.liec_oracle_mean_params.argtypes = [C.c_int32, C.c_int64, p, p]
+    lib.liec_oracle_mean_params.restype = None
+    lib.liec_oracle_average_step.argtypes = [C.c_int32, C.c_int64, p, C.c_float, p, p, p, p]
+    lib.liec_oracle_average_step.restype = C.c_int
     return lib
 
 
@@ -178,3 +182,26 @@ def step(X: np.ndarray, e: np.ndarray, G: np.ndarray, lr: float, off, up: int, d
     if rc:
         raise RuntimeError(f"liec_oracle_step failed with code {rc}")
     return r
+
+
+def mean_params(X: np.ndarray, _lib=None) -> np.ndarray:
+    """xbar = (1/N) sum_i x^i, the output of Algorithm 1 and the model sent back by an averaging iteration."""
+    assert X.dtype == np.float32 and X.flags.c_contiguous and X.ndim == 2
+    out = np.empty(X.shape[1], np.float32)
+    (_lib or lib()).liec_oracle_mean_params(X.shape[0], X.shape[1], _ptr(X), _ptr(out))
+    return out
+
+
+def average_step(X: np.ndarray, e: np.ndarray, G: np.ndarray, lr: float, _lib=None):
+    """Model-averaging iteration of Algorithm 1; X and e updated in place; returns (v, xbar)."""
+    assert X.dtype == np.float32 and X.flags.c_contiguous and X.ndim == 2
+    assert e.dtype == np.float32 and e.flags.c_contiguous
+    G = _f32(G)
+    N, d = X.shape
+    assert G.shape == (N, d) and e.shape == (d,)
+    v = np.empty(d, np.float32)
+    xbar = np.empty(d, np.float32)
+    rc = (_lib or lib()).liec_oracle_average_step(N, d, _ptr(G), C.c_float(lr), _ptr(X), _ptr(e), _ptr(v), _ptr(xbar))
+    if rc:
+        raise MemoryError("oracle average step out of memory")
+    return v, xbar

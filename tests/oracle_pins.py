@@ -394,6 +394,49 @@ def pin_lemma3_float(L):
         assert np.max(np.abs(e)) > 0.1
 
 
+def pin_golden_averaging(L):
+    """Hand-worked model-averaging iteration (tests/golden/averaging_step.txt)."""
+    g = read_golden("averaging_step.txt")
+    N = int(g["N"][0])
+    X = np.asarray([g[f"x0.{i}"] for i in range(N)], np.float32)
+    e = np.asarray(g["e0"], np.float32)
+    G = np.asarray([g[f"g.{i}"] for i in range(N)], np.float32)
+    v, xbar = oracle.average_step(X, e, G, g["lr"][0], _lib=L)
+    assert v.tolist() == g["v"] and xbar.tolist() == g["xbar"] and e.tolist() == g["e"]
+    for i in range(N):
+        assert X[i].tolist() == g[f"x.{i}"], (i, X[i])
+
+
+def pin_averaging_properties(L):
+    """Averaging iteration: the error is cleared, all local models coincide afterwards (exactly on
+    dyadic data), the mean model is the plain mean, and Lemma 3 keeps holding across a run that
+    mixes compressed iterations with an averaging one every 3rd step."""
+    rng = np.random.default_rng(41)
+    off = np.asarray([0, 4, 8], np.int64)
+    N, d, lr = 2, 8, 0.5
+    x0 = rng.integers(-4, 5, d).astype(np.float32)
+    X = np.tile(x0, (N, 1)).copy()
+    e = np.zeros(d, np.float32)
+    gsum = np.zeros(d, np.float64)
+    for step in range(6):
+        G = rng.integers(-8, 9, (N, d)).astype(np.float32)
+        if (step + 1) % 3 == 0:
+            xbar_before = X.astype(np.float64).mean(axis=0)
+            v, xbar = oracle.average_step(X, e, G, lr, _lib=L)
+            assert np.array_equal(xbar.astype(np.float64), xbar_before)
+            assert np.all(e == 0.0)
+            assert all(np.array_equal(X[i], X[0]) for i in range(N))
+        else:
+            oracle.step(X, e, G, lr, off, SIGN, SIGN, _lib=L)
+            assert not all(np.array_equal(X[i], X[0]) for i in range(N))
+        gsum += G.astype(np.float64).mean(axis=0)
+        lhs = X.astype(np.float64).mean(axis=0) - (x0.astype(np.float64) - lr * gsum)
+        assert np.array_equal(lhs, lr * e.astype(np.float64)), step
+    # the plain mean on Gaussian rows, against numpy in higher precision
+    Xg = rng.standard_normal((5, 300)).astype(np.float32)
+    assert np.max(np.abs(oracle.mean_params(Xg, _lib=L) - Xg.astype(np.float64).mean(axis=0))) < 1e-6
+
+
 def pin_bf16_widening(L):
     bits = np.asarray([0x3F80, 0xBF80, 0x0000, 0x8000, 0x3DCD, 0x7F7F, 0x0001], np.uint16)
     out = oracle.widen_bf16(bits)
@@ -406,5 +449,5 @@ ALL_PINS = [
     pin_scale_is_exact_mean, pin_tree_shape, pin_sign_bits_bruteforce, pin_sign_contraction,
     pin_blockwise_reduces_to_sign, pin_topk_bruteforce, pin_topk_quantile,
     pin_error_recursion, pin_identity_one_worker_is_sgd, pin_identical_workers,
-    pin_lemma3_exact, pin_lemma3_float, pin_bf16_widening,
+    pin_lemma3_exact, pin_lemma3_float, pin_bf16_widening, pin_golden_averaging, pin_averaging_properties,
 ]

@@ -36,6 +36,10 @@ MUTANTS = {
     "compensation_dropped": ("const float *pi = P + (size_t)i * d;", "const float *pi = g;"),
     "gradient_subtracted": ("float u = diff + g[j];", "float u = diff - g[j];"),
     "learning_rate_dropped": ("float step = lr * u;", "float step = u;"),
+    "averaging_keeps_local_model": ("x[j] = xbar[j] - scaled;", "x[j] = x[j] - scaled;"),
+    "averaging_forgets_error": ("v[j] = e[j] + gmean;", "v[j] = gmean;"),
+    "averaging_keeps_error": ("e[j] = v[j] - v[j];", "e[j] = e[j];"),
+    "mean_model_not_divided": ("xbar[j] = acc / (float)N;", "xbar[j] = acc;"),
     "ascent_instead_of_descent": ("x[j] = x[j] - step;", "x[j] = x[j] + step;"),
 }
 
