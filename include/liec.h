@@ -145,6 +145,22 @@ liec_status liec_worker_update(liec_ctx *ctx, const void *grads, float lr, void 
 liec_status liec_step(liec_ctx *ctx, const void *grads, float lr, void *stream);
 
 /*
+ * The model-averaging iteration of Algorithm 1 (its branch for (t+1) mod floor(1/delta) == 0; the
+ * caller decides when, e.g. every 32nd or 100th call): gradients and models travel uncompressed,
+ *   v = e + (1/N) sum_i g^i,  p = v,  error <- v - p = 0,
+ *   x^i <- (1/N) sum_i x^i - eta (p - g^i + g^i)   for every worker.
+ * Worker sums run in worker order in binary32 from +0 and are divided by (float)N.  Must not be
+ * called between the stages of a compressed iteration (LIEC_ERR_STATE).  One kernel on `stream`.
+ */
+liec_status liec_average_step(liec_ctx *ctx, const void *grads, float lr, void *stream);
+
+/*
+ * The algorithm's output xbar = (1/N) sum_i x^i (last line of Algorithm 1) into `out`
+ * (device, [d] binary32, caller-owned).  One kernel on `stream`.
+ */
+liec_status liec_mean_params(liec_ctx *ctx, float *out, void *stream);
+
+/*
  * One iteration fed from host memory: copies grads_host ([N][d] of cfg.grad_dtype, pinned
  * memory recommended) into grads_dev (device staging buffer of the same size, caller
  * owned), runs liec_step, copies the downlink message (sign: words then scales; top-k:

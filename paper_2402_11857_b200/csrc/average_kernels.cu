@@ -1,0 +1,130 @@
+// Model-averaging iteration of Algorithm 1 (the branch taken every floor(1/delta)-th step; the
+// experiments fix the period at 32 or 100) and the algorithm's output, the mean model.
+//
+//   v = e + (1/N) sum_i g^i,  p = v,  e <- v - p = +0,
+//   xbar = (1/N) sum_i x^i,   x^i <- xbar - eta ((p - g^i) + g^i)
+//
+// One CTA per tile does the whole iteration for its 8192 coordinates: a first sweep over the
+// workers accumulates the gradient and model sums in worker order, a second sweep re-reads each
+// worker's gradients (from L2: a tile's N rows are N x 16-32 KB) and writes the new models.
+#include "device_common.cuh"
+#include "kernels.h"
+
+namespace liec {
+
+template <typename GT>
+__global__ void __launch_bounds__(THREADS) average_step_kernel(const __grid_constant__ Params p, const float lr) {
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float gs[8][4], xs[8][4];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) { gs[j][c] = 0.0f; xs[j][c] = 0.0f; }
+    for (int i = 0; i < p.N; ++i) {
+        const int64_t row_beg = (int64_t)i * p.d + ti.seg_beg;
+        const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+        const GT *g_tile = reinterpret_cast<const GT *>(p.G) + row_beg + ti.rel;
+        const float *x_tile = p.X + row_beg + ti.rel;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int pos = tile_pos(warp, lane, j);
+            float g[4], x[4];
+            if (fast) { load4_cached(g_tile + pos, g); load4_stream(x_tile + pos, x); }
+            else { load4_guarded(g_tile, pos, ti.len, g); load4_guarded(x_tile, pos, ti.len, x); }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                gs[j][c] = __fadd_rn(gs[j][c], g[c]);
+                xs[j][c] = __fadd_rn(xs[j][c], x[c]);
+            }
+        }
+    }
+    const float nf = (float)p.N;
+    const bool efast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
+    float *e_tile = p.e + ti.seg_beg + ti.rel;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pos = tile_pos(warp, lane, j);
+        float ev[4];
+        if (efast) load4_stream(e_tile + pos, ev);
+        else load4_guarded(e_tile, pos, ti.len, ev);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            gs[j][c] = __fadd_rn(ev[c], __fdiv_rn(gs[j][c], nf));  // v
+            xs[j][c] = __fdiv_rn(xs[j][c], nf);                    // xbar
+        }
+        // e' = v - p with p = v
+        if (efast) {
+            *reinterpret_cast<float4 *>(e_tile + pos) = make_float4(__fsub_rn(gs[j][0], gs[j][0]), __fsub_rn(gs[j][1], gs[j][1]),
+                                                                    __fsub_rn(gs[j][2], gs[j][2]), __fsub_rn(gs[j][3], gs[j][3]));
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                if (pos + c < ti.len) e_tile[pos + c] = __fsub_rn(gs[j][c], gs[j][c]);
+        }
+    }
+    for (int i = 0; i < p.N; ++i) {
+        const int64_t row_beg = (int64_t)i * p.d + ti.seg_beg;
+        const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+        const GT *g_tile = reinterpret_cast<const GT *>(p.G) + row_beg + ti.rel;
+        float *x_tile = p.X + row_beg + ti.rel;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int pos = tile_pos(warp, lane, j);
+            float g[4], x[4];
+            if (fast) load4_cached(g_tile + pos, g);
+            else load4_guarded(g_tile, pos, ti.len, g);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const float diff = __fsub_rn(gs[j][c], g[c]);   // p - p^i, p = v, p^i = g^i
+                const float u = __fadd_rn(diff, g[c]);
+                x[c] = __fsub_rn(xs[j][c], __fmul_rn(lr, u));
+            }
+            if (fast) {
+                __stcs(reinterpret_cast<float4 *>(x_tile + pos), make_float4(x[0], x[1], x[2], x[3]));
+            } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if (pos + c < ti.len) x_tile[pos + c] = x[c];
+            }
+        }
+    }
+}
+
+// xbar = (1/N) sum_i x^i (the ENSURE line of Algorithm 1), one CTA per tile.
+__global__ void __launch_bounds__(THREADS) mean_params_kernel(const __grid_constant__ Params p, float *out) {
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const float nf = (float)p.N;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pos = tile_pos(warp, lane, j);
+        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        for (int i = 0; i < p.N; ++i) {
+            const int64_t row_beg = (int64_t)i * p.d + ti.seg_beg;
+            const float *x_tile = p.X + row_beg + ti.rel;
+            float x[4];
+            if ((ti.len == TILE) && ((row_beg & 3) == 0)) load4_stream(x_tile + pos, x);
+            else load4_guarded(x_tile, pos, ti.len, x);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[c] = __fadd_rn(acc[c], x[c]);
+        }
+        float *o = out + ti.seg_beg + ti.rel;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            if (pos + c < ti.len) o[pos + c] = __fdiv_rn(acc[c], nf);
+    }
+}
+
+cudaError_t launch_average_step(const Params &p, float lr, cudaStream_t st) {
+    if (p.gdt == DT_F32) average_step_kernel<float><<<p.TT, THREADS, 0, st>>>(p, lr);
+    else average_step_kernel<__nv_bfloat16><<<p.TT, THREADS, 0, st>>>(p, lr);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mean_params(const Params &p, float *out, cudaStream_t st) {
+    mean_params_kernel<<<p.TT, THREADS, 0, st>>>(p, out);
+    return cudaGetLastError();
+}
+
+}  // namespace liec

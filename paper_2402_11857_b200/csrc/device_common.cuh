@@ -43,6 +43,18 @@ __device__ __forceinline__ void load4_stream(const __nv_bfloat16 *ptr, float (&v
     v[2] = __uint_as_float(q.y << 16);
     v[3] = __uint_as_float(q.y & 0xffff0000u);
 }
+// Same, through the normal caching path (for data that is read again soon).
+__device__ __forceinline__ void load4_cached(const float *ptr, float (&v)[4]) {
+    float4 q = __ldg(reinterpret_cast<const float4 *>(ptr));
+    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+}
+__device__ __forceinline__ void load4_cached(const __nv_bfloat16 *ptr, float (&v)[4]) {
+    uint2 q = __ldg(reinterpret_cast<const uint2 *>(ptr));
+    v[0] = __uint_as_float(q.x << 16);
+    v[1] = __uint_as_float(q.x & 0xffff0000u);
+    v[2] = __uint_as_float(q.y << 16);
+    v[3] = __uint_as_float(q.y & 0xffff0000u);
+}
 __device__ __forceinline__ float load1(const float *ptr) { return *ptr; }
 __device__ __forceinline__ float load1(const __nv_bfloat16 *ptr) {
     return __uint_as_float((uint32_t)(*reinterpret_cast<const unsigned short *>(ptr)) << 16);

@@ -406,6 +406,22 @@ liec_status liec_step(liec_ctx *c, const void *grads, float lr, void *stream) {
     return liec_worker_update(c, grads, lr, stream);
 }
 
+liec_status liec_average_step(liec_ctx *c, const void *grads, float lr, void *stream) {
+    liec_status st = check_stage(c, 0, "liec_average_step");
+    if (st != LIEC_OK) return st;
+    if (!grads || !aligned16(grads)) { c->err = "grads must be non-NULL and 16-byte aligned"; return LIEC_ERR_INVALID_ARG; }
+    c->p.G = grads;
+    LIEC_LAUNCH(c, launch_average_step(c->p, lr, static_cast<cudaStream_t>(stream)));
+    return LIEC_OK;
+}
+
+liec_status liec_mean_params(liec_ctx *c, float *out, void *stream) {
+    if (!c) return LIEC_ERR_INVALID_ARG;
+    if (!out) { c->err = "out must be non-NULL"; return LIEC_ERR_INVALID_ARG; }
+    LIEC_LAUNCH(c, launch_mean_params(c->p, out, static_cast<cudaStream_t>(stream)));
+    return LIEC_OK;
+}
+
 liec_status liec_step_host(liec_ctx *c, const void *grads_host, void *grads_dev, float lr, void *down_msg_host,
                            void *stream) {
     if (!c) return LIEC_ERR_INVALID_ARG;

@@ -68,6 +68,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.liec_worker_update.restype = C.c_int
     lib.liec_step.argtypes = [vp, vp, C.c_float, vp]
     lib.liec_step.restype = C.c_int
+    lib.liec_average_step.argtypes = [vp, vp, C.c_float, vp]
+    lib.liec_average_step.restype = C.c_int
+    lib.liec_mean_params.argtypes = [vp, vp, vp]
+    lib.liec_mean_params.restype = C.c_int
     lib.liec_step_host.argtypes = [vp, vp, vp, C.c_float, vp, vp]
     lib.liec_step_host.restype = C.c_int
     lib.liec_get_messages.argtypes = [vp, C.POINTER(liec_messages)]
@@ -202,6 +206,14 @@ class Context:
     def liec_step(self, grads, lr: float, stream=None):
         self._check_grads(grads)
         self._check(self.lib.liec_step(self._ctx, grads.data_ptr(), float(lr), self._stream(stream)))
+
+    def liec_average_step(self, grads, lr: float, stream=None):
+        self._check_grads(grads)
+        self._check(self.lib.liec_average_step(self._ctx, grads.data_ptr(), float(lr), self._stream(stream)))
+
+    def liec_mean_params(self, out, stream=None):
+        assert out.is_cuda and out.dtype == self._torch.float32 and out.numel() == self.d and out.is_contiguous()
+        self._check(self.lib.liec_mean_params(self._ctx, out.data_ptr(), self._stream(stream)))
 
     def liec_step_host(self, grads_host, grads_dev, lr: float, down_msg_host=None, stream=None):
         self._check_grads(grads_dev)
