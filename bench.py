@@ -76,9 +76,9 @@ def update_kernel_bytes(w) -> float:
     return N * d * (g + 8) + down
 
 
-# DRAM bytes per element-worker of the worker update, from the committed ncu capture
-# (profiles/sign_kernels_c4_launches_and_c4div8_counters.md: 4.925 GB for 497.8 M element-workers on
-# c4/8; the traffic of this streaming kernel grows in proportion to N*d).  Other variants: not captured.
+# DRAM bytes per element-worker of the worker update, from an ncu capture of that kernel on the
+# c4/8 workload (dram__bytes_read + dram__bytes_write = 4.925 GB for 497.8 M element-workers; the
+# traffic of this streaming kernel grows in proportion to N*d).  Other variants: not captured.
 UPDATE_TRAFFIC_PER_UNIT = {("sign", "bf16"): 4.924888e9 / 497759232}
 
 

@@ -167,17 +167,11 @@ __global__ void __launch_bounds__(THREADS) scale_finalize_kernel(const __grid_co
 template <int UP, bool DOWN_SIGN, typename GT>
 __global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_constant__ Params p) {
     __shared__ double warp_sums[8];
-    extern __shared__ float up_scale_smem[];  // [N] scales of this segment (sign uplink)
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
     const int64_t wbase = __ldg(p.word_off + ti.t) + ti.rel / 32;
     const int nwords = (ti.len + 31) >> 5;
-
-    if (UP == COMP_SIGN) {
-        for (int i = threadIdx.x; i < p.N; i += THREADS) up_scale_smem[i] = p.up_scales[(int64_t)i * p.T + ti.t];
-        __syncthreads();
-    }
 
     float acc[8][4];
 #pragma unroll
@@ -185,22 +179,7 @@ __global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_cons
 #pragma unroll
         for (int c = 0; c < 4; ++c) acc[j][c] = 0.0f;
 
-    if (UP == COMP_SIGN) {
-        const int my_widx = warp * 32 + lane;
-        for (int i = 0; i < p.N; ++i) {
-            const uint32_t sbits = __float_as_uint(up_scale_smem[i]);
-            uint32_t my_word = my_widx < nwords ? __ldg(p.up_words + (int64_t)i * p.W + wbase + my_widx) : 0u;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                uint32_t nib = nibble_from_words(my_word, lane, j);
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    float pij = __uint_as_float(sbits ^ ((nib << (31 - c)) & 0x80000000u));
-                    acc[j][c] = __fadd_rn(acc[j][c], pij);
-                }
-            }
-        }
-    } else {  // identity uplink: the message is the gradient itself
+    {  // identity uplink: the message is the gradient itself
         for (int i = 0; i < p.N; ++i) {
             const int64_t row_beg = (int64_t)i * p.d + ti.seg_beg;
             const GT *tile_ptr = reinterpret_cast<const GT *>(p.G) + row_beg + ti.rel;
@@ -269,16 +248,31 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
     float acc[32];
 #pragma unroll
     for (int c = 0; c < 32; ++c) acc[c] = 0.0f;
+    // workers four at a time: their four words are fetched together, one group ahead of use
+    constexpr int WG = 4;
     const uint32_t *wp = p.up_words + wbase + my_widx;
-    uint32_t next = have_word ? __ldg(wp) : 0u;
-    for (int i = 0; i < p.N; ++i) {
-        const uint32_t w = next;
-        if (i + 1 < p.N && have_word) next = __ldg(wp + (int64_t)(i + 1) * p.W);
-        const uint32_t sbits = __float_as_uint(up_scale_smem[i]);
+    uint32_t nextw[WG];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-            const float pij = __uint_as_float(sbits ^ ((w << (31 - c)) & 0x80000000u));
-            acc[c] = __fadd_rn(acc[c], pij);
+    for (int u = 0; u < WG; ++u) nextw[u] = (have_word && u < p.N) ? __ldg(wp + (int64_t)u * p.W) : 0u;
+    for (int i0 = 0; i0 < p.N; i0 += WG) {
+        uint32_t w[WG];
+#pragma unroll
+        for (int u = 0; u < WG; ++u) w[u] = nextw[u];
+#pragma unroll
+        for (int u = 0; u < WG; ++u) {
+            const int i = i0 + WG + u;
+            nextw[u] = (have_word && i < p.N) ? __ldg(wp + (int64_t)i * p.W) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < WG; ++u) {
+            if (i0 + u < p.N) {  // uniform over the CTA
+                const uint32_t sbits = __float_as_uint(up_scale_smem[i0 + u]);
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    const float pij = __uint_as_float(sbits ^ ((w[u] << (31 - c)) & 0x80000000u));
+                    acc[c] = __fadd_rn(acc[c], pij);
+                }
+            }
         }
     }
 
@@ -414,9 +408,8 @@ cudaError_t launch_scale_finalize(const Params &p, bool uplink, cudaStream_t st)
 
 template <int UP, typename GT>
 static cudaError_t launch_server_dense_t(const Params &p, cudaStream_t st) {
-    size_t smem = UP == COMP_SIGN ? sizeof(float) * (size_t)p.N : 0;
-    if (p.down == COMP_SIGN) server_dense_kernel<UP, true, GT><<<p.TT, THREADS, smem, st>>>(p);
-    else server_dense_kernel<UP, false, GT><<<p.TT, THREADS, smem, st>>>(p);
+    if (p.down == COMP_SIGN) server_dense_kernel<UP, true, GT><<<p.TT, THREADS, 0, st>>>(p);
+    else server_dense_kernel<UP, false, GT><<<p.TT, THREADS, 0, st>>>(p);
     return cudaGetLastError();
 }
 
