@@ -13,22 +13,27 @@
 namespace liec {
 
 template <typename GT>
-__global__ void __launch_bounds__(THREADS) average_step_kernel(const __grid_constant__ Params p, const float lr) {
+__global__ void __launch_bounds__(THREADS, 3) average_step_kernel(const __grid_constant__ Params p, const float lr) {
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float gs[8][4], xs[8][4];
+    // two CTAs share a tile (rows 0-3 and rows 4-7 of every warp's slice): half the accumulators
+    // per thread, twice the CTAs in flight
+    constexpr int HR = 4;
+    const int j0 = HR * blockIdx.y;
+    float gs[HR][4], xs[HR][4];
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
+    for (int j = 0; j < HR; ++j)
 #pragma unroll
         for (int c = 0; c < 4; ++c) { gs[j][c] = 0.0f; xs[j][c] = 0.0f; }
+#pragma unroll 2
     for (int i = 0; i < p.N; ++i) {
         const int64_t row_beg = (int64_t)i * p.d + ti.seg_beg;
         const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
         const GT *g_tile = reinterpret_cast<const GT *>(p.G) + row_beg + ti.rel;
         const float *x_tile = p.X + row_beg + ti.rel;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int pos = tile_pos(warp, lane, j);
+        for (int j = 0; j < HR; ++j) {
+            const int pos = tile_pos(warp, lane, j0 + j);
             float g[4], x[4];
             if (fast) { load4_cached(g_tile + pos, g); load4_stream(x_tile + pos, x); }
             else { load4_guarded(g_tile, pos, ti.len, g); load4_guarded(x_tile, pos, ti.len, x); }
@@ -43,8 +48,8 @@ __global__ void __launch_bounds__(THREADS) average_step_kernel(const __grid_cons
     const bool efast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
     float *e_tile = p.e + ti.seg_beg + ti.rel;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int pos = tile_pos(warp, lane, j);
+    for (int j = 0; j < HR; ++j) {
+        const int pos = tile_pos(warp, lane, j0 + j);
         float ev[4];
         if (efast) load4_stream(e_tile + pos, ev);
         else load4_guarded(e_tile, pos, ti.len, ev);
@@ -63,14 +68,15 @@ __global__ void __launch_bounds__(THREADS) average_step_kernel(const __grid_cons
                 if (pos + c < ti.len) e_tile[pos + c] = __fsub_rn(gs[j][c], gs[j][c]);
         }
     }
+#pragma unroll 2
     for (int i = 0; i < p.N; ++i) {
         const int64_t row_beg = (int64_t)i * p.d + ti.seg_beg;
         const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
         const GT *g_tile = reinterpret_cast<const GT *>(p.G) + row_beg + ti.rel;
         float *x_tile = p.X + row_beg + ti.rel;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int pos = tile_pos(warp, lane, j);
+        for (int j = 0; j < HR; ++j) {
+            const int pos = tile_pos(warp, lane, j0 + j);
             float g[4], x[4];
             if (fast) load4_cached(g_tile + pos, g);
             else load4_guarded(g_tile, pos, ti.len, g);
@@ -117,8 +123,9 @@ __global__ void __launch_bounds__(THREADS) mean_params_kernel(const __grid_const
 }
 
 cudaError_t launch_average_step(const Params &p, float lr, cudaStream_t st) {
-    if (p.gdt == DT_F32) average_step_kernel<float><<<p.TT, THREADS, 0, st>>>(p, lr);
-    else average_step_kernel<__nv_bfloat16><<<p.TT, THREADS, 0, st>>>(p, lr);
+    const dim3 grid(p.TT, 2);
+    if (p.gdt == DT_F32) average_step_kernel<float><<<grid, THREADS, 0, st>>>(p, lr);
+    else average_step_kernel<__nv_bfloat16><<<grid, THREADS, 0, st>>>(p, lr);
     return cudaGetLastError();
 }
 
