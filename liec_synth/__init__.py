@@ -5,11 +5,11 @@ method's arithmetic (compressors, aggregation, updates) lives here, so that the
 oracle and the CUDA library can both be fed the same bytes without sharing code.
 """
 from .layouts import (Layout, flat_layout, resnet18_layout, resnet50_layout,
-                      gpt2_small_layout, scaled_layout, ragged_layout, topk_counts)
+                      gpt2_small_layout, scaled_layout, ragged_layout, topk_counts, equal_blocks_layout)
 from .grads import (WORKLOADS, Workload, make_gradients, gradient_seed)
 
 __all__ = [
     "Layout", "flat_layout", "resnet18_layout", "resnet50_layout", "gpt2_small_layout",
-    "scaled_layout", "ragged_layout", "topk_counts",
+    "scaled_layout", "ragged_layout", "topk_counts", "equal_blocks_layout",
     "WORKLOADS", "Workload", "make_gradients", "gradient_seed",
 ]

@@ -115,6 +115,15 @@ def ragged_layout() -> Layout:
     return Layout("ragged", (1, 7, 33, 64, 1000, 8191, 8193, 3 * 8192 + 5, 31, 32, 2 * 8192, 4099))
 
 
+def equal_blocks_layout(d: int, num_blocks: int, name: str | None = None) -> Layout:
+    """d elements cut into num_blocks contiguous blocks of (almost) equal size, the first d % num_blocks
+    one element longer: the paper's Blockwise-SignSGD runs split the gradient into 10, 18 or 14 blocks
+    without saying how; this is the plain reading."""
+    base, extra = divmod(int(d), int(num_blocks))
+    assert base >= 1
+    return Layout(name or f"blocks{num_blocks}x{d}", tuple(base + (1 if b < extra else 0) for b in range(num_blocks)))
+
+
 def topk_counts(layout: Layout, num: int, den: int) -> np.ndarray:
     """k_t = max(1, floor(n_t * num / den)) in integer arithmetic."""
     return np.asarray([max(1, (n * num) // den) for n in layout.sizes], dtype=np.int64)

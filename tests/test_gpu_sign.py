@@ -57,6 +57,44 @@ def test_resnet18_scaled_layout_sign_many_steps():
         P.step(G, 0.05, check_messages=(step % 10 == 0))
 
 
+@pytest.mark.parametrize("blocks", [10, 18, 14])
+def test_blockwise_equal_blocks(blocks):
+    """Blockwise-SignSGD with the block counts of the paper's runs (10, 18, 14 equal blocks); the
+    block boundaries fall at arbitrary offsets, not at multiples of 32 or of the tile."""
+    from liec_synth import equal_blocks_layout
+    lay = equal_blocks_layout(200_003, blocks)
+    P = _pair(4, lay.seg_offsets, SIGN, SIGN)
+    for step in range(3):
+        G = make_gradients("normal", 0.01, 4, lay.dim, step, base_seed=40 + blocks)
+        P.step(G, 0.1)
+
+
+def test_step_from_host_memory_matches_device_step():
+    """liec_step_host (gradients copied from pinned host memory, downlink message copied back)
+    leaves the same state as liec_step and returns the message bytes that sit in the workspace."""
+    lay = ragged_layout()
+    N = 3
+    outs = []
+    for mode in ("device", "host"):
+        X = torch.zeros(N, lay.dim, device="cuda"); e = torch.zeros(lay.dim, device="cuda")
+        ctx = liec.Context(X, e, lay.seg_offsets, SIGN, SIGN)
+        msg = torch.zeros(liec.down_message_bytes(ctx.cfg), dtype=torch.uint8).pin_memory()
+        for step in range(3):
+            G = make_gradients("normal", 1.0, N, lay.dim, step, base_seed=41)
+            if mode == "device":
+                ctx.liec_step(G.cuda(), 0.1)
+            else:
+                ctx.liec_step_host(G.pin_memory(), torch.empty_like(G, device="cuda"), 0.1, msg)
+        torch.cuda.synchronize()
+        m = ctx.liec_get_messages()
+        outs.append((X.cpu(), e.cpu(), m["down_words"].cpu(), m["down_scales"].cpu(), msg.clone()))
+    for a, b in zip(outs[0][:4], outs[1][:4]):
+        assert torch.equal(a, b)
+    words, scales, msg = outs[1][2], outs[1][3], outs[1][4]
+    assert torch.equal(msg[: 4 * words.numel()].view(torch.int32), words)
+    assert torch.equal(msg[4 * words.numel():].view(torch.float32), scales)
+
+
 def test_bf16_gradients_sign():
     """bf16 gradients with sparse +-0.1 outliers, GPT-2 tensor list shrunk 64x, N=5 (not a power of two)."""
     lay = scaled_layout(gpt2_small_layout(), 64)
