@@ -98,6 +98,30 @@ float liec_oracle_scale(const float *x, int64_t n)
     return (float)mean;
 }
 
+/* ---- telemetry: squared norms ------------------------------------------------------- */
+
+static double tree_sq_node(const float *x, int64_t n, int64_t lo, int64_t len)
+{
+    if (len == 1) {
+        if (lo >= n) return 0.0;
+        double a = (double)x[lo];
+        return a * a;                  /* exact: 24-bit significands */
+    }
+    double left = tree_sq_node(x, n, lo, len / 2);
+    double right = tree_sq_node(x, n, lo + len / 2, len / 2);
+    return left + right;
+}
+
+/* ||x||_2^2 in binary64 over the same balanced tree as the L1 norm.  With it the quantities the
+ * paper reports follow: the error norm ||e_t|| (its figure of error norms) and the measured
+ * contraction delta = 1 - ||x - C(x)||^2 / ||x||^2 of Def. 1 (its table of measured delta). */
+double liec_oracle_tree_sumsq(const float *x, int64_t n)
+{
+    int64_t L = 1;
+    while (L < n) L *= 2;
+    return tree_sq_node(x, n, 0, L);
+}
+
 static int64_t words_of(int64_t n) { return (n + 31) / 32; }
 
 /* Segment-wise scaled sign of x[0..off[T]).  words: sum_t ceil(n_t/32) entries,

@@ -44,6 +44,8 @@ def _bind(lib: C.CDLL) -> C.CDLL:
     lib.liec_oracle_widen_bf16.restype = None
     lib.liec_oracle_tree_abs_sum.argtypes = [p, C.c_int64]
     lib.liec_oracle_tree_abs_sum.restype = C.c_double
+    lib.liec_oracle_tree_sumsq.argtypes = [p, C.c_int64]
+    lib.liec_oracle_tree_sumsq.restype = C.c_double
     lib.liec_oracle_scale.argtypes = [p, C.c_int64]
     lib.liec_oracle_scale.restype = C.c_float
     lib.liec_oracle_sign.argtypes = [p, C.c_int32, p, p, p, p]
@@ -98,6 +100,12 @@ def widen_bf16(bits_u16: np.ndarray) -> np.ndarray:
 def tree_abs_sum(x, _lib=None) -> float:
     x = _f32(x)
     return float((_lib or lib()).liec_oracle_tree_abs_sum(_ptr(x), x.size))
+
+
+def tree_sumsq(x, _lib=None) -> float:
+    """||x||_2^2 in binary64 (balanced tree)."""
+    x = _f32(x)
+    return float((_lib or lib()).liec_oracle_tree_sumsq(_ptr(x), x.size))
 
 
 def scale(x, _lib=None) -> np.float32:

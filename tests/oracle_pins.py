@@ -437,6 +437,29 @@ def pin_averaging_properties(L):
     assert np.max(np.abs(oracle.mean_params(Xg, _lib=L) - Xg.astype(np.float64).mean(axis=0))) < 1e-6
 
 
+def pin_sumsq_and_delta(L):
+    """Squared norms against exact rational arithmetic, and the measured contraction of Def. 1
+    computed from them: for the scaled sign delta = d s^2 / ||x||^2 (-> 2/pi on Gaussians), for
+    top-k delta = ||C(x)||^2 / ||x||^2 >= k/d."""
+    rng = np.random.default_rng(43)
+    for n in (1, 3, 64, 1000):
+        x = (rng.standard_normal(n) * np.exp(rng.uniform(-5, 5, n))).astype(np.float32)
+        exact = sum((Fraction(float(v)) ** 2 for v in x), Fraction(0))
+        got = oracle.tree_sumsq(x, _lib=L)
+        assert abs(Fraction(got) - exact) <= exact * Fraction(1, 10 ** 14), n
+    assert oracle.tree_sumsq(np.asarray([3, -4], np.float32), _lib=L) == 25.0
+    x = rng.standard_normal(100_000).astype(np.float32)
+    _, s, dec = oracle.sign_compress(x, [0, x.size], _lib=L)
+    xx = oracle.tree_sumsq(x, _lib=L)
+    delta = x.size * float(s[0]) ** 2 / xx
+    resid = oracle.tree_sumsq(x - dec, _lib=L)
+    assert abs((1 - resid / xx) - delta) < 1e-6 and abs(delta - 2 / math.pi) < 0.01
+    k = 1000
+    _, val, dec = oracle.topk_compress(x, [0, x.size], [k], _lib=L)
+    delta_k = oracle.tree_sumsq(val, _lib=L) / xx
+    assert abs((1 - oracle.tree_sumsq(x - dec, _lib=L) / xx) - delta_k) < 1e-9 and delta_k >= k / x.size
+
+
 def pin_bf16_widening(L):
     bits = np.asarray([0x3F80, 0xBF80, 0x0000, 0x8000, 0x3DCD, 0x7F7F, 0x0001], np.uint16)
     out = oracle.widen_bf16(bits)
@@ -449,5 +472,5 @@ ALL_PINS = [
     pin_scale_is_exact_mean, pin_tree_shape, pin_sign_bits_bruteforce, pin_sign_contraction,
     pin_blockwise_reduces_to_sign, pin_topk_bruteforce, pin_topk_quantile,
     pin_error_recursion, pin_identity_one_worker_is_sgd, pin_identical_workers,
-    pin_lemma3_exact, pin_lemma3_float, pin_bf16_widening, pin_golden_averaging, pin_averaging_properties,
+    pin_lemma3_exact, pin_lemma3_float, pin_bf16_widening, pin_golden_averaging, pin_averaging_properties, pin_sumsq_and_delta,
 ]

@@ -40,6 +40,7 @@ MUTANTS = {
     "averaging_forgets_error": ("v[j] = e[j] + gmean;", "v[j] = gmean;"),
     "averaging_keeps_error": ("e[j] = v[j] - v[j];", "e[j] = e[j];"),
     "mean_model_not_divided": ("xbar[j] = acc / (float)N;", "xbar[j] = acc;"),
+    "sumsq_not_squared": ("return a * a;                  /* exact: 24-bit significands */", "return a < 0 ? -a : a;"),
     "ascent_instead_of_descent": ("x[j] = x[j] - step;", "x[j] = x[j] + step;"),
 }
 
