@@ -161,6 +161,24 @@ liec_status liec_average_step(liec_ctx *ctx, const void *grads, float lr, void *
 liec_status liec_mean_params(liec_ctx *ctx, float *out, void *stream);
 
 /*
+ * Squared Euclidean norms per segment, for monitoring: out[r][t] = sum of x_j^2 over segment t of
+ * row r, accumulated in binary64 over the same balanced tree as the L1 norms (deterministic).
+ *   which = LIEC_SUMSQ_ERROR : the global error e (1 row)  -> ||e_t||, the quantity of the paper's
+ *                              figure of error norms;
+ *           LIEC_SUMSQ_GRADS : `grads` ([N][d] of cfg.grad_dtype, N rows);
+ *           LIEC_SUMSQ_PARAMS: the local models (N rows).
+ * With these the measured contraction of Def. 1, delta = 1 - ||x - C(x)||^2 / ||x||^2 (the paper's
+ * table of measured delta), follows without touching the hot path: scaled sign
+ * delta = n s^2 / ||x||^2 per segment (worker side: x = g^i; server side: ||v||^2 = ||e'||^2 + n s^2);
+ * top-k delta = ||kept values||^2 / ||x||^2.  One extra read of the chosen array when called.
+ *   out  device, [rows][T] binary64, caller-owned.  Two kernels on `stream`.
+ */
+#define LIEC_SUMSQ_ERROR 0
+#define LIEC_SUMSQ_GRADS 1
+#define LIEC_SUMSQ_PARAMS 2
+liec_status liec_sumsq(liec_ctx *ctx, int32_t which, const void *grads, double *out, void *stream);
+
+/*
  * One iteration fed from host memory: copies grads_host ([N][d] of cfg.grad_dtype, pinned
  * memory recommended) into grads_dev (device staging buffer of the same size, caller
  * owned), runs liec_step, copies the downlink message (sign: words then scales; top-k:

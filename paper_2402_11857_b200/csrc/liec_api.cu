@@ -28,6 +28,7 @@ struct Plan {
     std::vector<int64_t> seg_off, word_off, k_off, cap_off, topk_k;
     std::vector<int32_t> tile_prefix, tile_seg;
     Region r_seg_off, r_word_off, r_k_off, r_cap_off, r_tile_prefix, r_tile_seg, r_status;
+    Region r_tel_partials;
     Region r_up_words, r_up_scales, r_up_partials, r_down_words, r_down_scales, r_down_partials, r_vbuf;
     Region r_up_idx, r_up_val, r_down_idx, r_down_val;
     Region r_up_hist, r_down_hist, r_up_hist2, r_down_hist2, r_up_sel, r_down_sel;
@@ -124,6 +125,7 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     pl.r_tile_prefix = c.take(sizeof(int32_t) * (T + 1));
     pl.r_tile_seg = c.take(sizeof(int32_t) * pl.TT);
     pl.r_status = c.take(256);
+    pl.r_tel_partials = c.take(sizeof(double) * (size_t)pl.N * pl.TT);
     const size_t N = pl.N;
     if (cfg->uplink == LIEC_COMP_SCALED_SIGN) {
         pl.r_up_words = c.take(sizeof(uint32_t) * N * pl.W);
@@ -283,6 +285,7 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     p.down_scales = at<float>(c, pl.r_down_scales);
     p.down_partials = at<double>(c, pl.r_down_partials);
     p.vbuf = at<float>(c, pl.r_vbuf);
+    p.tel_partials = at<double>(c, pl.r_tel_partials);
     p.up_idx = at<uint32_t>(c, pl.r_up_idx);       p.up_val = at<float>(c, pl.r_up_val);
     p.down_idx = at<uint32_t>(c, pl.r_down_idx);   p.down_val = at<float>(c, pl.r_down_val);
     p.up_hist = at<uint32_t>(c, pl.r_up_hist);     p.down_hist = at<uint32_t>(c, pl.r_down_hist);
@@ -419,6 +422,20 @@ liec_status liec_mean_params(liec_ctx *c, float *out, void *stream) {
     if (!c) return LIEC_ERR_INVALID_ARG;
     if (!out) { c->err = "out must be non-NULL"; return LIEC_ERR_INVALID_ARG; }
     LIEC_LAUNCH(c, launch_mean_params(c->p, out, static_cast<cudaStream_t>(stream)));
+    return LIEC_OK;
+}
+
+liec_status liec_sumsq(liec_ctx *c, int32_t which, const void *grads, double *out, void *stream) {
+    if (!c) return LIEC_ERR_INVALID_ARG;
+    if (!out) { c->err = "out must be non-NULL"; return LIEC_ERR_INVALID_ARG; }
+    if (which < 0 || which > 2) { c->err = "which must be LIEC_SUMSQ_ERROR, _GRADS or _PARAMS"; return LIEC_ERR_INVALID_ARG; }
+    if (which == 1 && (!grads || !aligned16(grads))) { c->err = "grads must be non-NULL and 16-byte aligned"; return LIEC_ERR_INVALID_ARG; }
+    const void *src = which == 0 ? (const void *)c->p.e : which == 1 ? grads : (const void *)c->p.X;
+    const int rows = which == 0 ? 1 : c->p.N;
+    const bool bf16 = which == 1 && c->p.gdt == DT_BF16;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    LIEC_LAUNCH(c, launch_sumsq(c->p, src, which == 0 ? 0 : c->p.d, rows, bf16, s));
+    LIEC_LAUNCH(c, launch_sum_finalize(c->p, rows, out, s));
     return LIEC_OK;
 }
 

@@ -46,6 +46,7 @@ struct Params {
     uint32_t *down_words;  // [W]
     float *down_scales;    // [T]
     double *down_partials; // [TT]
+    double *tel_partials;  // [N][TT] telemetry (squared norms)
 
     // top-k messages and scratch (row count R = N for uplink, 1 for downlink)
     uint32_t *up_idx;  float *up_val;    // [N][K]

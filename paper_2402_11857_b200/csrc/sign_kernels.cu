@@ -113,7 +113,8 @@ __global__ void __launch_bounds__(THREADS) sign_uplink_bf16_kernel(const __grid_
 constexpr int FIN_CHUNK = 2048;
 
 __global__ void __launch_bounds__(THREADS) scale_finalize_kernel(const __grid_constant__ Params p,
-                                                                  const double *partials, float *scales) {
+                                                                  const double *partials, float *scales,
+                                                                  double *sums /* when set: the plain sums instead */) {
     __shared__ double buf[FIN_CHUNK];
     __shared__ double chunk_sums[512];  // 2^32 / TILE / FIN_CHUNK = 256 chunks at most
     const int t = blockIdx.x, row = blockIdx.y;
@@ -154,8 +155,12 @@ __global__ void __launch_bounds__(THREADS) scale_finalize_kernel(const __grid_co
         for (int width = L / 2; width >= 1; width >>= 1)
             for (int q = 0; q < width; ++q) chunk_sums[q] = __dadd_rn(chunk_sums[2 * q], chunk_sums[2 * q + 1]);
         const int64_t n = __ldg(p.seg_off + t + 1) - __ldg(p.seg_off + t);
-        double mean = __ddiv_rn(chunk_sums[0], (double)n);
-        scales[(int64_t)row * p.T + t] = __double2float_rn(mean);
+        if (sums) {
+            sums[(int64_t)row * p.T + t] = chunk_sums[0];
+        } else {
+            double mean = __ddiv_rn(chunk_sums[0], (double)n);
+            scales[(int64_t)row * p.T + t] = __double2float_rn(mean);
+        }
     }
 }
 
@@ -390,8 +395,47 @@ __global__ void __launch_bounds__(THREADS) identity_downlink_kernel(const __grid
 }
 
 // ------------------------------------------------------------------------------------------------
+// Squared norms per tile (monitoring): leaves x^2 in binary64 (exact), same tree as the L1 norm.
+// ------------------------------------------------------------------------------------------------
+template <typename GT>
+__global__ void __launch_bounds__(THREADS) sumsq_kernel(const __grid_constant__ Params p, const GT *src,
+                                                         const int64_t row_stride) {
+    __shared__ double warp_sums[8];
+    const int row = blockIdx.y;
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t row_beg = (int64_t)row * row_stride + ti.seg_beg;
+    const GT *tile_ptr = src + row_beg + ti.rel;
+    const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+    double a[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        float v[4];
+        if (fast) load4_stream(tile_ptr + tile_pos(warp, lane, j), v);
+        else load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v);
+        const double d0 = (double)v[0], d1 = (double)v[1], d2 = (double)v[2], d3 = (double)v[3];
+        a[j] = __dadd_rn(__dadd_rn(__dmul_rn(d0, d0), __dmul_rn(d1, d1)), __dadd_rn(__dmul_rn(d2, d2), __dmul_rn(d3, d3)));
+    }
+    double s = cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
+    if (threadIdx.x == 0) p.tel_partials[(int64_t)row * p.TT + blockIdx.x] = s;
+}
+
+// ------------------------------------------------------------------------------------------------
 // launchers
 // ------------------------------------------------------------------------------------------------
+cudaError_t launch_sumsq(const Params &p, const void *src, int64_t row_stride, int rows, bool bf16, cudaStream_t st) {
+    dim3 grid(p.TT, rows);
+    if (bf16) sumsq_kernel<__nv_bfloat16><<<grid, THREADS, 0, st>>>(p, static_cast<const __nv_bfloat16 *>(src), row_stride);
+    else sumsq_kernel<float><<<grid, THREADS, 0, st>>>(p, static_cast<const float *>(src), row_stride);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sum_finalize(const Params &p, int rows, double *out, cudaStream_t st) {
+    dim3 grid(p.T, rows);
+    scale_finalize_kernel<<<grid, THREADS, 0, st>>>(p, p.tel_partials, nullptr, out);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_sign_uplink(const Params &p, cudaStream_t st) {
     dim3 grid(p.TT, p.N);
     if (p.gdt == DT_F32) sign_uplink_kernel<float><<<grid, THREADS, 0, st>>>(p);
@@ -402,7 +446,7 @@ cudaError_t launch_sign_uplink(const Params &p, cudaStream_t st) {
 cudaError_t launch_scale_finalize(const Params &p, bool uplink, cudaStream_t st) {
     dim3 grid(p.T, uplink ? p.N : 1);
     scale_finalize_kernel<<<grid, THREADS, 0, st>>>(p, uplink ? p.up_partials : p.down_partials,
-                                                    uplink ? p.up_scales : p.down_scales);
+                                                    uplink ? p.up_scales : p.down_scales, nullptr);
     return cudaGetLastError();
 }
 

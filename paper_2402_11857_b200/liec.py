@@ -12,6 +12,7 @@ from typing import Optional, Sequence
 import numpy as np
 
 COMP_IDENTITY, COMP_SCALED_SIGN, COMP_TOPK = 0, 1, 2
+SUMSQ_ERROR, SUMSQ_GRADS, SUMSQ_PARAMS = 0, 1, 2
 F32, BF16 = 0, 1
 
 STATUS_NAMES = {0: "LIEC_OK", 1: "LIEC_ERR_INVALID_ARG", 2: "LIEC_ERR_UNSUPPORTED", 3: "LIEC_ERR_WORKSPACE",
@@ -72,6 +73,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.liec_average_step.restype = C.c_int
     lib.liec_mean_params.argtypes = [vp, vp, vp]
     lib.liec_mean_params.restype = C.c_int
+    lib.liec_sumsq.argtypes = [vp, C.c_int32, vp, vp, vp]
+    lib.liec_sumsq.restype = C.c_int
     lib.liec_step_host.argtypes = [vp, vp, vp, C.c_float, vp, vp]
     lib.liec_step_host.restype = C.c_int
     lib.liec_get_messages.argtypes = [vp, C.POINTER(liec_messages)]
@@ -214,6 +217,16 @@ class Context:
     def liec_mean_params(self, out, stream=None):
         assert out.is_cuda and out.dtype == self._torch.float32 and out.numel() == self.d and out.is_contiguous()
         self._check(self.lib.liec_mean_params(self._ctx, out.data_ptr(), self._stream(stream)))
+
+    def liec_sumsq(self, which: int, out, grads=None, stream=None):
+        """Per-segment squared norms (SUMSQ_ERROR / SUMSQ_GRADS / SUMSQ_PARAMS) into `out` [rows, T] float64."""
+        rows = 1 if which == SUMSQ_ERROR else self.N
+        assert out.is_cuda and out.dtype == self._torch.float64 and out.numel() == rows * self.T and out.is_contiguous()
+        gptr = None
+        if which == SUMSQ_GRADS:
+            self._check_grads(grads)
+            gptr = grads.data_ptr()
+        self._check(self.lib.liec_sumsq(self._ctx, int(which), gptr, out.data_ptr(), self._stream(stream)))
 
     def liec_step_host(self, grads_host, grads_dev, lr: float, down_msg_host=None, stream=None):
         self._check_grads(grads_dev)
