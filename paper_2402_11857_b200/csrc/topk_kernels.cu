@@ -2,21 +2,25 @@
 // ties broken toward the lower index, output (index, value) compacted in ascending index.
 //
 // One selection "problem" is a (row, segment) pair; the uplink has N rows (the workers'
-// gradients), the downlink one row (v, held in the error buffer).  Pipeline per side:
+// gradients), the downlink one row (v, held in the error buffer).  Regular route per side:
 //
 //   hist1   dense pass 1: histogram of the first key digit (bits 30..19) per problem
-//   pick1   bin b1 holding the k-th largest key, rank left inside it, exact candidate count
-//   filter  dense pass 2: entries with digit >= b1 appended (in index order inside each tile)
-//           to the problem's candidate buffer; histogram of the second digit (bits 18..7)
-//           over the entries whose first digit equals b1
-//   pick2   second digit
-//   hist3   candidates only: histogram of the last 7 key bits under the 24-bit prefix
-//   pick3   threshold key and number of ties to accept
-//   count   candidates only: per tile, entries above the threshold and entries equal to it
+//           (for the downlink after a top-k uplink it is fused into the server pass)
+//   pick 1  bin b1 holding the k-th largest key, rank left inside it, exact candidate count
+//   hist2_dense + pick 4   only for problems whose bin b1 is too crowded for the candidate
+//           buffer: dense second-digit histogram, 24-bit prefix
+//   filter  dense pass 2: entries at or above the prefix appended, in index order inside each
+//           tile, to the problem's region of the candidate buffer
+//   finish  per problem, on its candidates: second digit and last 7 bits -> exact threshold key
+//           and the number of ties to accept
+//   count   per tile block: entries above the threshold and entries equal to it
 //   scan    per problem: first output slot and accepted ties of every tile
-//   write   candidates only: ordered compaction into (idx, val); records the last accepted tie
-//   slow    one CTA per problem, only for problems whose candidates exceed the buffer
+//   write   ordered compaction into (idx, val); records the last accepted tie
+//   slow    one CTA per problem, only when even the 24-bit prefix leaves too many candidates
 //           (huge groups of equal magnitudes, e.g. mostly-zero rows): same result, dense passes
+//
+// The uplink first tries a single-pass route (begin, filter with a guess, cand_hist, pick 5),
+// described at topk_begin_kernel.
 //
 // Nothing waits on another CTA; cross-CTA order comes from kernel boundaries.
 #include "device_common.cuh"
@@ -206,88 +210,61 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
     __shared__ uint32_t scratch[THREADS + 4];
     const int t = blockIdx.x, row = blockIdx.y;
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
-    // level 1: first digit.  level 4: second digit of "refined" problems (after their dense
-    // second-digit pass).  level 2: second digit of regular problems.  level 3: last 7 bits.
-    // level 5 (uplink): first digit from the histogram of the candidates collected with the guess;
-    // checks the guess.
+    // level 1: first digit from the dense histogram (regular route).
+    // level 5: first digit from the histogram of the candidates collected with the guess
+    //          (uplink single-pass route); checks the guess.
+    // level 4: second digit of "refined" problems, after their dense second-digit pass.
     if (level == 5 && sel[SEL_MODE] != 1u) return;
     if (level == 1 && s.spec && sel[SEL_MODE] != 0u) return;
-    const uint32_t flags_in = (level == 1 || level == 5) ? 0u : sel[SEL_FLAGS];
     if (level == 4 && t == 0 && row == 0 && threadIdx.x == 0) p.status[STATUS_ANY_REFINE + (s.zero_out ? 1 : 0)] = 0;
-    if (level == 4 && flags_in != 2u) return;
-    if (level == 2 && flags_in != 0u) return;
-    if (level == 3 && (flags_in & 1u)) return;  // slow path finishes on its own
-    const int nbins = level == 3 ? 128 : DIGIT1_BINS;
-    uint32_t *gh = ((level == 1 || level == 5) ? s.hist : s.hist2) + ((int64_t)row * p.T + t) * DIGIT1_BINS;
-    if (nbins == DIGIT1_BINS) {
-        // only the recorded non-empty range is read and cleared
-        const bool first = level == 1 || level == 5;
-        const int lo_word = first ? SEL_LO1 : SEL_LO2, hi_word = first ? SEL_HI1 : SEL_HI2;
-        // (the filter does not record the range of the second-digit histogram: level 2 reads all of it)
-        // the regular filter fills the second-digit histogram with untracked atomics
-        const bool full = level == 2 && !(s.spec && sel[SEL_MODE] == 1u);
-        const uint32_t lo = full ? 0u : min(sel[lo_word], (uint32_t)DIGIT1_BINS);
-        const uint32_t hi = full ? (uint32_t)DIGIT1_BINS - 1u : min(sel[hi_word], (uint32_t)DIGIT1_BINS - 1u);
-        for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(bins)[b] = make_uint4(0u, 0u, 0u, 0u);
-        __syncthreads();
-        for (uint32_t b = lo + threadIdx.x; b <= hi; b += THREADS) {
-            const uint32_t c = gh[b];
-            if (c) { bins[b] = c; gh[b] = 0u; }
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) { sel[lo_word] = 0xffffffffu; sel[hi_word] = 0u; }
-    } else {
-        for (int b = threadIdx.x; b < nbins; b += THREADS) {
-            bins[b] = gh[b];
-            gh[b] = 0u;
-        }
+    if (level == 4 && sel[SEL_FLAGS] != 2u) return;
+    const bool first = level != 4;
+    uint32_t *gh = (first ? s.hist : s.hist2) + ((int64_t)row * p.T + t) * DIGIT1_BINS;
+    // only the recorded non-empty range of the histogram is read and cleared
+    const int lo_word = first ? SEL_LO1 : SEL_LO2, hi_word = first ? SEL_HI1 : SEL_HI2;
+    const uint32_t lo = min(sel[lo_word], (uint32_t)DIGIT1_BINS);
+    const uint32_t hi = min(sel[hi_word], (uint32_t)DIGIT1_BINS - 1u);
+    for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(bins)[b] = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+    for (uint32_t b = lo + threadIdx.x; b <= hi; b += THREADS) {
+        const uint32_t c = gh[b];
+        if (c) { bins[b] = c; gh[b] = 0u; }
     }
     __syncthreads();
+    if (threadIdx.x == 0) { sel[lo_word] = 0xffffffffu; sel[hi_word] = 0u; }
     const uint32_t k = (uint32_t)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
-    const uint32_t rank = (level == 1 || level == 5) ? k : sel[SEL_REMAIN];
-    const PickResult r = block_pick(bins, nbins, rank, scratch);
-    if (threadIdx.x == 0) {
-        if (level == 5) {
-            if (!r.ok) {  // fewer than k candidates: the guess was too high, take the regular route
-                sel[SEL_MODE] = 0u;
-                p.status[STATUS_ANY_REGULAR] = 1;
-            } else {
-                sel[SEL_PREFIX] = r.bin;
-                sel[SEL_REMAIN] = r.rank_in_bin;
-                sel[SEL_ABOVE] = r.count_ge - bins[r.bin];
-                sel[SEL_NCAND] = sel[SEL_CAND_COUNT];
-            }
-            return;
-        }
-        if (!r.ok) { atomicOr(p.status, STATUS_PICK_RANK); return; }
-        const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
-        if (level == 1) {
+    const uint32_t rank = first ? k : sel[SEL_REMAIN];
+    const PickResult r = block_pick(bins, DIGIT1_BINS, rank, scratch);
+    if (threadIdx.x != 0) return;
+    if (level == 5) {
+        if (!r.ok) {  // fewer than k candidates: the guess was too high, take the regular route
+            sel[SEL_MODE] = 0u;
+            p.status[STATUS_ANY_REGULAR] = 1;
+        } else {
             sel[SEL_PREFIX] = r.bin;
             sel[SEL_REMAIN] = r.rank_in_bin;
-            sel[SEL_NCAND] = r.count_ge;
             sel[SEL_ABOVE] = r.count_ge - bins[r.bin];
-            sel[SEL_CAND_COUNT] = 0u;
-            // too many entries share the threshold's first digit: look at the second digit first
-            sel[SEL_FLAGS] = r.count_ge > cap ? 2u : 0u;
-            if (r.count_ge > cap) p.status[STATUS_ANY_REFINE + (s.zero_out ? 1 : 0)] = 1;
-        } else if (level == 4) {
-            const uint32_t ncand = sel[SEL_ABOVE] + r.count_ge;
-            sel[SEL_PREFIX] = (sel[SEL_PREFIX] << 12) | r.bin;
-            sel[SEL_REMAIN] = r.rank_in_bin;
-            sel[SEL_NCAND] = ncand;
-            if (ncand > cap) { sel[SEL_FLAGS] = 3u; sel[SEL_GUESS] = 0u; }  // still too many (huge groups of equal keys): slow path
-        } else if (level == 2) {
-            sel[SEL_PREFIX] = (sel[SEL_PREFIX] << 12) | r.bin;
-            sel[SEL_REMAIN] = r.rank_in_bin;
-        } else {
-            const uint32_t thresh = (sel[SEL_PREFIX] << 7) | r.bin;
-            sel[SEL_THRESH] = thresh;
-            sel[SEL_TIES] = r.rank_in_bin;
-            if (s.spec) {  // next step's guess: one first-digit bin below this threshold's bin
-                const uint32_t b1 = thresh >> DIGIT1_SHIFT;
-                sel[SEL_GUESS] = (flags_in == 0u && b1 >= 1u) ? (b1 - 1u) << DIGIT1_SHIFT : 0u;
-            }
+            sel[SEL_NCAND] = sel[SEL_CAND_COUNT];
         }
+        return;
+    }
+    if (!r.ok) { atomicOr(p.status, STATUS_PICK_RANK); return; }
+    const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
+    if (level == 1) {
+        sel[SEL_PREFIX] = r.bin;
+        sel[SEL_REMAIN] = r.rank_in_bin;
+        sel[SEL_NCAND] = r.count_ge;
+        sel[SEL_ABOVE] = r.count_ge - bins[r.bin];
+        sel[SEL_CAND_COUNT] = 0u;
+        // too many entries share the threshold's first digit: look at the second digit first
+        sel[SEL_FLAGS] = r.count_ge > cap ? 2u : 0u;
+        if (r.count_ge > cap) p.status[STATUS_ANY_REFINE + (s.zero_out ? 1 : 0)] = 1;
+    } else {
+        const uint32_t ncand = sel[SEL_ABOVE] + r.count_ge;
+        sel[SEL_PREFIX] = (sel[SEL_PREFIX] << 12) | r.bin;
+        sel[SEL_REMAIN] = r.rank_in_bin;
+        sel[SEL_NCAND] = ncand;
+        if (ncand > cap) { sel[SEL_FLAGS] = 3u; sel[SEL_GUESS] = 0u; }  // still too many (huge groups of equal keys): slow path
     }
 }
 
@@ -443,7 +420,6 @@ __global__ void __launch_bounds__(THREADS, 4) topk_filter_kernel(const __grid_co
         const uint32_t base_now = tile_base;
         if (base_now == 0xffffffffu || mask == 0u) continue;
         const int64_t cbase = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + base_now + warp_off;
-        uint32_t *gh2 = s.hist2 + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS;
         const uint32_t flat0 = (uint32_t)(ti.seg_beg + ti.rel);
         // walk the set bits (candidates are rare: usually zero or one iteration)
         uint32_t rest = mask;
@@ -458,11 +434,8 @@ __global__ void __launch_bounds__(THREADS, 4) topk_filter_kernel(const __grid_co
             const uint32_t o = row_base + before + lower;
             const int pos = tile_pos(warp, lane, j) + (b & 3);
             const float val = load1(tile_ptr + pos);  // read again (cached) rather than kept across the barrier
-            const uint32_t key = key_of(val);
             s.cand_idx[cbase + o] = flat0 + pos;
             s.cand_val[cbase + o] = val;
-            if (!SPEC && !refined && (key >> DIGIT1_SHIFT) == prefix)
-                atomicAdd(gh2 + ((key >> 7) & 0xfffu), 1u);  // (range not tracked: two more contended atomics cost more than they save)
         }
     }
 }
@@ -486,41 +459,20 @@ __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide 
 
 // The candidate passes give one warp to every tile block (8 tiles per CTA): blocks are small
 // (about 1.4 % of a tile) and warps need no block-wide synchronisation.
-__global__ void __launch_bounds__(THREADS) topk_hist3_kernel(const __grid_constant__ Params p, const TopkSide s) {
-    const int row = blockIdx.y, lane = threadIdx.x & 31;
-    const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (tile >= p.TT) return;
-    const CandBlock cb = cand_block(p, s, tile, row);
-    if (cb.skip) return;
-    const uint32_t prefix24 = cb.sel[SEL_PREFIX];
-    uint32_t *gh = s.hist2 + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
-    for (uint32_t q = lane; q < cb.cnt; q += 32) {
-        const uint32_t key = key_of(s.cand_val[cb.base + q]);
-        if ((key >> 7) == prefix24) atomicAdd(gh + (key & 0x7fu), 1u);
-    }
-}
-
-// Histograms over the candidates of the problems on the single-pass route (one warp per tile
-// block).  level 0: first digit of every candidate; level 1: second digit of the candidates whose
-// first digit is the threshold's.  Lanes holding the same digit add once (match + leader).
-__global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_constant__ Params p, const TopkSide s,
-                                                                  const int level) {
+// First-digit histogram over the candidates of the problems on the single-pass route (one warp
+// per tile block).  Lanes holding the same digit add once (match + leader).
+__global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_constant__ Params p, const TopkSide s) {
     const int row = blockIdx.y, lane = threadIdx.x & 31;
     const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (tile >= p.TT) return;
     const CandBlock cb = cand_block(p, s, tile, row);
     if (cb.skip || cb.sel[SEL_MODE] != 1u) return;
-    const uint32_t b1 = cb.sel[SEL_PREFIX];
-    uint32_t *gh = (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
+    uint32_t *gh = s.hist + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
     uint32_t lo = 0xffffffffu, hi = 0u;
     for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
         const uint32_t q = c0 + lane;
         uint32_t digit = 0xffffffffu;  // lanes with nothing to add
-        if (q < cb.cnt) {
-            const uint32_t key = key_of(s.cand_val[cb.base + q]);
-            if (level == 0) digit = key >> DIGIT1_SHIFT;
-            else if ((key >> DIGIT1_SHIFT) == b1) digit = (key >> 7) & 0xfffu;
-        }
+        if (q < cb.cnt) digit = key_of(s.cand_val[cb.base + q]) >> DIGIT1_SHIFT;
         const uint32_t same = __match_any_sync(0xffffffffu, digit);
         if (digit != 0xffffffffu) {
             if (lane == __ffs(same) - 1) atomicAdd(gh + digit, (uint32_t)__popc(same));
@@ -532,8 +484,8 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
     lo = __reduce_min_sync(0xffffffffu, lo);
     hi = __reduce_max_sync(0xffffffffu, hi);
     if (lane == 0 && lo != 0xffffffffu) {
-        atomicMin(&cb.sel[level == 0 ? SEL_LO1 : SEL_LO2], lo);
-        atomicMax(&cb.sel[level == 0 ? SEL_HI1 : SEL_HI2], hi);
+        atomicMin(&cb.sel[SEL_LO1], lo);
+        atomicMax(&cb.sel[SEL_HI1], hi);
     }
 }
 
@@ -553,6 +505,57 @@ __global__ void __launch_bounds__(THREADS) topk_count_kernel(const __grid_consta
     g = __reduce_add_sync(0xffffffffu, g);
     e = __reduce_add_sync(0xffffffffu, e);
     if (lane == 0) { cb.meta[2] = g; cb.meta[3] = e; }
+}
+
+// finish: one CTA per (segment, row).  The first digit (or, for refined problems, the 24-bit
+// prefix) of the threshold is known and the problem's candidates sit in one contiguous region of
+// the candidate buffer (a few per cent of the segment, cache resident): two sweeps over that
+// region with shared-memory histograms (second digit, then the last 7 bits) give the exact
+// threshold key and the number of ties to accept.
+__global__ void __launch_bounds__(THREADS) topk_finish_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    __shared__ __align__(16) uint32_t bins[DIGIT1_BINS];
+    __shared__ uint32_t scratch[THREADS + 4];
+    const int t = blockIdx.x, row = blockIdx.y;
+    uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
+    const uint32_t flags = sel[SEL_FLAGS];
+    if (flags & 1u) return;  // slow path finishes on its own
+    const float *cand = s.cand_val + (int64_t)row * p.CAP + __ldg(p.cap_off + t);
+    const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
+    const uint32_t ncand = min(sel[SEL_CAND_COUNT], cap);  // (the cursor can run past the buffer when a tile was refused)
+    uint32_t prefix24 = sel[SEL_PREFIX];
+    uint32_t rank = sel[SEL_REMAIN];
+    if (!(flags & 2u)) {
+        const uint32_t b1 = prefix24;
+        for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(bins)[b] = make_uint4(0u, 0u, 0u, 0u);
+        __syncthreads();
+        for (uint32_t q = threadIdx.x; q < ncand; q += THREADS) {
+            const uint32_t key = key_of(cand[q]);
+            if ((key >> DIGIT1_SHIFT) == b1) atomicAdd(&bins[(key >> 7) & 0xfffu], 1u);
+        }
+        __syncthreads();
+        const PickResult r2 = block_pick(bins, DIGIT1_BINS, rank, scratch);
+        if (!r2.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
+        prefix24 = (b1 << 12) | r2.bin;
+        rank = r2.rank_in_bin;
+    }
+    if (threadIdx.x < 128) bins[threadIdx.x] = 0u;
+    __syncthreads();
+    for (uint32_t q = threadIdx.x; q < ncand; q += THREADS) {
+        const uint32_t key = key_of(cand[q]);
+        if ((key >> 7) == prefix24) atomicAdd(&bins[key & 0x7fu], 1u);
+    }
+    __syncthreads();
+    const PickResult r3 = block_pick(bins, 128, rank, scratch);
+    if (!r3.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
+    if (threadIdx.x == 0) {
+        const uint32_t thresh = (prefix24 << 7) | r3.bin;
+        sel[SEL_THRESH] = thresh;
+        sel[SEL_TIES] = r3.rank_in_bin;
+        if (s.spec) {  // next step's guess: one first-digit bin below this threshold's bin
+            const uint32_t b1 = thresh >> DIGIT1_SHIFT;
+            sel[SEL_GUESS] = (flags == 0u && b1 >= 1u) ? (b1 - 1u) << DIGIT1_SHIFT : 0u;
+        }
+    }
 }
 
 // scan: one CTA per (segment, row); tiles of the segment in order
@@ -615,6 +618,7 @@ __global__ void __launch_bounds__(THREADS) topk_write_kernel(const __grid_consta
     const uint32_t allowed = cb.meta[3];
     const bool has_last = cb.meta[2] != 0u;
     const int64_t obase = (int64_t)row * p.K + s.outbase[(int64_t)row * (p.TT + 1) + tile];
+    const int64_t oend = (int64_t)row * p.K + __ldg(p.k_off + cb.t + 1);  // never write past the segment's slots
     const uint32_t lt_mask = (1u << lane) - 1u;
     uint32_t run_sel = 0, run_tie = 0;
     for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
@@ -628,7 +632,9 @@ __global__ void __launch_bounds__(THREADS) topk_write_kernel(const __grid_consta
         const uint32_t tie_rank = run_tie + __popc(tb & lt_mask);
         const bool take = in && (key > T || (tie && tie_rank < allowed));
         const uint32_t sb = __ballot_sync(0xffffffffu, take);
-        if (take) {
+        if (take && obase + run_sel + __popc(sb & lt_mask) >= oend) {
+            atomicOr(p.status, STATUS_COUNT_MISMATCH);  // inconsistent selection state: drop the write
+        } else if (take) {
             const uint32_t out = run_sel + __popc(sb & lt_mask);
             s.idx[obase + out] = idx;
             s.val[obase + out] = val;
@@ -716,7 +722,9 @@ __global__ void __launch_bounds__(THREADS) topk_slow_kernel(const __grid_constan
         uint32_t out = run_sel + __popc(sb & lt_mask), sel_tot = 0;
 #pragma unroll
         for (int w = 0; w < 8; ++w) { if (w < warp) out += wb[w]; sel_tot += wb[w]; }
-        if (take) {
+        if (take && out >= k) {
+            atomicOr(p.status, STATUS_COUNT_MISMATCH);
+        } else if (take) {
             const uint32_t flat = (uint32_t)(seg_beg + j);
             s.idx[obase + out] = flat;
             s.val[obase + out] = val;
@@ -862,7 +870,7 @@ cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int
         if (bf) topk_filter_kernel<__nv_bfloat16, true><<<g_tiles, THREADS, 0, st>>>(p, s);
         else topk_filter_kernel<float, true><<<g_tiles, THREADS, 0, st>>>(p, s);
         CHECK_LAUNCH();
-        topk_cand_hist_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s, 0); CHECK_LAUNCH();
+        topk_cand_hist_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
         topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 5); CHECK_LAUNCH();
     }
     const dim3 g_hist = s.spec ? strided_grid(p, s.R) : g_tiles;
@@ -887,10 +895,7 @@ cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, in
     if (bf) topk_filter_kernel<__nv_bfloat16, false><<<g_filter, THREADS, 0, st>>>(p, s);
     else topk_filter_kernel<float, false><<<g_filter, THREADS, 0, st>>>(p, s);
     CHECK_LAUNCH();
-    if (s.spec) { topk_cand_hist_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s, 1); CHECK_LAUNCH(); }
-    topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();
-    topk_hist3_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
-    topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 3); CHECK_LAUNCH();
+    topk_finish_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     topk_count_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     topk_scan_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     topk_write_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
