@@ -24,7 +24,7 @@ struct Region {
 
 struct Plan {
     int32_t N = 0, T = 0, TT = 0;
-    int64_t d = 0, W = 0, K = 0, CAP = 0;
+    int64_t d = 0, W = 0, K = 0, CAP = 0, cap_max = 0;
     std::vector<int64_t> seg_off, word_off, k_off, cap_off, topk_k;
     std::vector<int32_t> tile_prefix, tile_seg;
     Region r_seg_off, r_word_off, r_k_off, r_cap_off, r_tile_prefix, r_tile_seg, r_status;
@@ -107,6 +107,7 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
             int64_t cap = 2 * k + 2048;  // room for the entries sharing the threshold's first digit
             if (cap > n) cap = n;
             pl.cap_off[t + 1] = pl.cap_off[t] + cap;
+            if (cap > pl.cap_max) pl.cap_max = cap;
         }
     }
     pl.W = pl.word_off[T];
@@ -267,7 +268,7 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     c->ws = static_cast<char *>(workspace);
     Params &p = c->p;
     memset(&p, 0, sizeof(p));
-    p.N = pl.N; p.T = pl.T; p.TT = pl.TT; p.d = pl.d; p.W = pl.W; p.K = pl.K; p.CAP = pl.CAP;
+    p.N = pl.N; p.T = pl.T; p.TT = pl.TT; p.d = pl.d; p.W = pl.W; p.K = pl.K; p.CAP = pl.CAP; p.cap_max = pl.cap_max;
     p.up = cfg->uplink; p.down = cfg->downlink; p.gdt = cfg->grad_dtype;
     p.seg_off = at<int64_t>(c, pl.r_seg_off);
     p.word_off = at<int64_t>(c, pl.r_word_off);

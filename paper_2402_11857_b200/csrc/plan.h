@@ -59,6 +59,7 @@ struct Params {
     uint32_t *up_tile_meta, *down_tile_meta; // [R][TT][4] pos, cnt, n_greater, n_ties
     uint32_t *up_outbase, *down_outbase;     // [R][TT+1] first output slot of each tile
     int64_t CAP;                              // candidate capacity per row
+    int64_t cap_max;                          // largest candidate capacity of one segment
 
     float *vbuf;      // [d] identity downlink copy of v
     int32_t *status;  // device status word

@@ -214,11 +214,14 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
     // level 5: first digit from the histogram of the candidates collected with the guess
     //          (uplink single-pass route); checks the guess.
     // level 4: second digit of "refined" problems, after their dense second-digit pass.
+    // levels 2, 3: wide form of the finish step (second digit, last 7 bits) from candidate histograms.
     if (level == 5 && sel[SEL_MODE] != 1u) return;
+    if (level == 2 && sel[SEL_FLAGS] != 0u) return;
+    if (level == 3 && (sel[SEL_FLAGS] & 1u)) return;
     if (level == 1 && s.spec && sel[SEL_MODE] != 0u) return;
     if (level == 4 && t == 0 && row == 0 && threadIdx.x == 0) p.status[STATUS_ANY_REFINE + (s.zero_out ? 1 : 0)] = 0;
     if (level == 4 && sel[SEL_FLAGS] != 2u) return;
-    const bool first = level != 4;
+    const bool first = level == 1 || level == 5;
     uint32_t *gh = (first ? s.hist : s.hist2) + ((int64_t)row * p.T + t) * DIGIT1_BINS;
     // only the recorded non-empty range of the histogram is read and cleared
     const int lo_word = first ? SEL_LO1 : SEL_LO2, hi_word = first ? SEL_HI1 : SEL_HI2;
@@ -250,7 +253,18 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
     }
     if (!r.ok) { atomicOr(p.status, STATUS_PICK_RANK); return; }
     const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
-    if (level == 1) {
+    if (level == 2) {
+        sel[SEL_PREFIX] = (sel[SEL_PREFIX] << 12) | r.bin;
+        sel[SEL_REMAIN] = r.rank_in_bin;
+    } else if (level == 3) {
+        const uint32_t thresh = (sel[SEL_PREFIX] << 7) | r.bin;
+        sel[SEL_THRESH] = thresh;
+        sel[SEL_TIES] = r.rank_in_bin;
+        if (s.spec) {  // next step's guess: one first-digit bin below this threshold's bin
+            const uint32_t b1 = thresh >> DIGIT1_SHIFT;
+            sel[SEL_GUESS] = (sel[SEL_FLAGS] == 0u && b1 >= 1u) ? (b1 - 1u) << DIGIT1_SHIFT : 0u;
+        }
+    } else if (level == 1) {
         sel[SEL_PREFIX] = r.bin;
         sel[SEL_REMAIN] = r.rank_in_bin;
         sel[SEL_NCAND] = r.count_ge;
@@ -459,20 +473,33 @@ __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide 
 
 // The candidate passes give one warp to every tile block (8 tiles per CTA): blocks are small
 // (about 1.4 % of a tile) and warps need no block-wide synchronisation.
-// First-digit histogram over the candidates of the problems on the single-pass route (one warp
-// per tile block).  Lanes holding the same digit add once (match + leader).
-__global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_constant__ Params p, const TopkSide s) {
+// Histograms over candidates, one warp per tile block; lanes holding the same digit add once
+// (match + leader).  level 0: first digit, problems on the single-pass route.  level 1 and 2 are
+// the wide form of the finish step, for segments whose candidates are too many for one CTA:
+// level 1 = second digit of the candidates whose first digit is the threshold's, level 2 = last
+// 7 bits of the candidates under the 24-bit prefix.
+__global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_constant__ Params p, const TopkSide s,
+                                                                  const int level) {
     const int row = blockIdx.y, lane = threadIdx.x & 31;
     const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (tile >= p.TT) return;
     const CandBlock cb = cand_block(p, s, tile, row);
-    if (cb.skip || cb.sel[SEL_MODE] != 1u) return;
-    uint32_t *gh = s.hist + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
+    if (cb.skip) return;
+    const uint32_t flags = cb.sel[SEL_FLAGS];
+    if (level == 0 && cb.sel[SEL_MODE] != 1u) return;
+    if (level == 1 && flags != 0u) return;  // refined problems already have their 24-bit prefix
+    const uint32_t prefix = cb.sel[SEL_PREFIX];
+    uint32_t *gh = (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
     uint32_t lo = 0xffffffffu, hi = 0u;
     for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
         const uint32_t q = c0 + lane;
         uint32_t digit = 0xffffffffu;  // lanes with nothing to add
-        if (q < cb.cnt) digit = key_of(s.cand_val[cb.base + q]) >> DIGIT1_SHIFT;
+        if (q < cb.cnt) {
+            const uint32_t key = key_of(s.cand_val[cb.base + q]);
+            if (level == 0) digit = key >> DIGIT1_SHIFT;
+            else if (level == 1) { if ((key >> DIGIT1_SHIFT) == prefix) digit = (key >> 7) & 0xfffu; }
+            else if ((key >> 7) == prefix) digit = key & 0x7fu;
+        }
         const uint32_t same = __match_any_sync(0xffffffffu, digit);
         if (digit != 0xffffffffu) {
             if (lane == __ffs(same) - 1) atomicAdd(gh + digit, (uint32_t)__popc(same));
@@ -484,8 +511,8 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
     lo = __reduce_min_sync(0xffffffffu, lo);
     hi = __reduce_max_sync(0xffffffffu, hi);
     if (lane == 0 && lo != 0xffffffffu) {
-        atomicMin(&cb.sel[SEL_LO1], lo);
-        atomicMax(&cb.sel[SEL_HI1], hi);
+        atomicMin(&cb.sel[level == 0 ? SEL_LO1 : SEL_LO2], lo);
+        atomicMax(&cb.sel[level == 0 ? SEL_HI1 : SEL_HI2], hi);
     }
 }
 
@@ -854,6 +881,10 @@ __global__ void __launch_bounds__(THREADS) server_topk_kernel(const __grid_const
         ++*launches;                                     \
     } while (0)
 
+// Largest per-segment candidate capacity that the one-CTA finish kernel handles (two sweeps over
+// that many cached values by 256 threads); beyond it the finish step runs as four wide launches.
+constexpr int64_t FINISH_ONE_CTA_MAX = 1 << 17;
+
 // Grid of the dense passes that usually have nothing to do on the uplink (their CTAs walk the
 // tiles with a stride and leave at once when no problem takes the regular route).
 static dim3 strided_grid(const Params &p, int rows) { return dim3(p.TT < 592 ? p.TT : 592, rows); }
@@ -870,7 +901,7 @@ cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int
         if (bf) topk_filter_kernel<__nv_bfloat16, true><<<g_tiles, THREADS, 0, st>>>(p, s);
         else topk_filter_kernel<float, true><<<g_tiles, THREADS, 0, st>>>(p, s);
         CHECK_LAUNCH();
-        topk_cand_hist_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+        topk_cand_hist_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s, 0); CHECK_LAUNCH();
         topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 5); CHECK_LAUNCH();
     }
     const dim3 g_hist = s.spec ? strided_grid(p, s.R) : g_tiles;
@@ -895,7 +926,14 @@ cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, in
     if (bf) topk_filter_kernel<__nv_bfloat16, false><<<g_filter, THREADS, 0, st>>>(p, s);
     else topk_filter_kernel<float, false><<<g_filter, THREADS, 0, st>>>(p, s);
     CHECK_LAUNCH();
-    topk_finish_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+    if (p.cap_max <= FINISH_ONE_CTA_MAX) {
+        topk_finish_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+    } else {  // some segment has too many candidates for one CTA: the same two steps, spread over the tile blocks
+        topk_cand_hist_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s, 1); CHECK_LAUNCH();
+        topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();
+        topk_cand_hist_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();
+        topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 3); CHECK_LAUNCH();
+    }
     topk_count_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     topk_scan_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     topk_write_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();

@@ -124,6 +124,17 @@ def test_large_single_segment_topk():
             P.step(G, 0.1)
 
 
+def test_many_candidates_take_the_wide_finish():
+    """k = 10 % of a 700 k-element tensor: more candidates than one CTA is given to finish, so the
+    threshold is found by the wide (multi-CTA) form of the finish step; a small tensor rides along."""
+    lay = Layout("wide", (700_000, 5000))
+    k = np.asarray([70_000, 50], np.int64)
+    P = _pair(2, lay.seg_offsets, TOPK, TOPK, k=k)
+    for step in range(3):
+        G = make_gradients("normal", 1.0, 2, lay.dim, step, base_seed=24)
+        P.step(G, 0.1)
+
+
 def test_bf16_topk():
     lay = ragged_layout()
     k = topk_counts(lay, 1, 50)
