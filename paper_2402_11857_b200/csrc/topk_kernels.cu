@@ -480,39 +480,68 @@ __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide 
 // 7 bits of the candidates under the 24-bit prefix.
 __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_constant__ Params p, const TopkSide s,
                                                                   const int level) {
+    __shared__ uint32_t h[DIGIT1_BINS];
     const int row = blockIdx.y, lane = threadIdx.x & 31;
-    const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (tile >= p.TT) return;
-    const CandBlock cb = cand_block(p, s, tile, row);
-    if (cb.skip) return;
-    const uint32_t flags = cb.sel[SEL_FLAGS];
-    if (level == 0 && cb.sel[SEL_MODE] != 1u) return;
-    if (level == 1 && flags != 0u) return;  // refined problems already have their 24-bit prefix
-    const uint32_t prefix = cb.sel[SEL_PREFIX];
-    uint32_t *gh = (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
+    const int tile0 = blockIdx.x * 8;
+    const int tile = tile0 + (threadIdx.x >> 5);
+    // When the CTA's 8 tiles lie in one very large segment the counts are
+    // first gathered in shared memory, so that the segment's global histogram sees a few atomics
+    // per CTA instead of a few per warp and iteration.
+    const int tlast = min(tile0 + 7, p.TT - 1);
+    const int seg0 = __ldg(p.tile_seg + tile0);
+    // (worth its fixed cost only where many CTAs hammer one histogram: segments of 1024+ tiles)
+    const bool gather = seg0 == __ldg(p.tile_seg + tlast) &&
+                        __ldg(p.tile_prefix + seg0 + 1) - __ldg(p.tile_prefix + seg0) >= 1024;
+    if (gather) {
+        for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) h[b] = 0u;
+        __syncthreads();
+    }
+    bool active = tile < p.TT;
+    CandBlock cb;
+    uint32_t prefix = 0;
+    if (active) {
+        cb = cand_block(p, s, tile, row);
+        const uint32_t flags = cb.sel[SEL_FLAGS];
+        active = !cb.skip && !(level == 0 && cb.sel[SEL_MODE] != 1u) && !(level == 1 && flags != 0u);
+        prefix = cb.sel[SEL_PREFIX];
+    }
     uint32_t lo = 0xffffffffu, hi = 0u;
-    for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
-        const uint32_t q = c0 + lane;
-        uint32_t digit = 0xffffffffu;  // lanes with nothing to add
-        if (q < cb.cnt) {
-            const uint32_t key = key_of(s.cand_val[cb.base + q]);
-            if (level == 0) digit = key >> DIGIT1_SHIFT;
-            else if (level == 1) { if ((key >> DIGIT1_SHIFT) == prefix) digit = (key >> 7) & 0xfffu; }
-            else if ((key >> 7) == prefix) digit = key & 0x7fu;
-        }
-        const uint32_t same = __match_any_sync(0xffffffffu, digit);
-        if (digit != 0xffffffffu) {
-            if (lane == __ffs(same) - 1) atomicAdd(gh + digit, (uint32_t)__popc(same));
-            lo = min(lo, digit);
-            hi = max(hi, digit);
+    if (active) {
+        uint32_t *gh = (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
+        for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
+            const uint32_t q = c0 + lane;
+            uint32_t digit = 0xffffffffu;  // lanes with nothing to add
+            if (q < cb.cnt) {
+                const uint32_t key = key_of(s.cand_val[cb.base + q]);
+                if (level == 0) digit = key >> DIGIT1_SHIFT;
+                else if (level == 1) { if ((key >> DIGIT1_SHIFT) == prefix) digit = (key >> 7) & 0xfffu; }
+                else if ((key >> 7) == prefix) digit = key & 0x7fu;
+            }
+            const uint32_t same = __match_any_sync(0xffffffffu, digit);
+            if (digit != 0xffffffffu) {
+                if (lane == __ffs(same) - 1) {
+                    if (gather) atomicAdd(&h[digit], (uint32_t)__popc(same));
+                    else atomicAdd(gh + digit, (uint32_t)__popc(same));
+                }
+                lo = min(lo, digit);
+                hi = max(hi, digit);
+            }
         }
     }
-    // the non-empty bin range, so that the pick reads and clears only that
-    lo = __reduce_min_sync(0xffffffffu, lo);
-    hi = __reduce_max_sync(0xffffffffu, hi);
-    if (lane == 0 && lo != 0xffffffffu) {
-        atomicMin(&cb.sel[level == 0 ? SEL_LO1 : SEL_LO2], lo);
-        atomicMax(&cb.sel[level == 0 ? SEL_HI1 : SEL_HI2], hi);
+    const int lo_word = level == 0 ? SEL_LO1 : SEL_LO2, hi_word = level == 0 ? SEL_HI1 : SEL_HI2;
+    if (gather) {
+        __syncthreads();
+        // (all tiles of the CTA share the segment, hence the selection state and the histogram)
+        const int t = __ldg(p.tile_seg + tile0);
+        flush_hist(h, (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + t) * DIGIT1_BINS,
+                   s.sel + ((int64_t)row * p.T + t) * SEL_WORDS, lo_word, hi_word);
+    } else if (active) {
+        lo = __reduce_min_sync(0xffffffffu, lo);
+        hi = __reduce_max_sync(0xffffffffu, hi);
+        if (lane == 0 && lo != 0xffffffffu) {
+            atomicMin(&cb.sel[lo_word], lo);
+            atomicMax(&cb.sel[hi_word], hi);
+        }
     }
 }
 
@@ -586,50 +615,74 @@ __global__ void __launch_bounds__(THREADS) topk_finish_kernel(const __grid_const
 }
 
 // scan: one CTA per (segment, row); tiles of the segment in order
+// Exclusive prefix sum of one value per thread over the CTA (shuffles inside warps, warp totals in
+// shared memory); `total` receives the CTA's sum.  Two barriers.
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t x, uint32_t *warp_tot /*[8]*/, uint32_t &total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = x;
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xffffffffu, inc, m);
+        if (lane >= m) inc += up;
+    }
+    __syncthreads();  // warp_tot may still be read from the previous call
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    uint32_t before = 0;
+    total = 0;
+#pragma unroll
+    for (int w = 0; w < THREADS / 32; ++w) {
+        if (w < warp) before += warp_tot[w];
+        total += warp_tot[w];
+    }
+    return before + inc - x;
+}
+
 __global__ void __launch_bounds__(THREADS) topk_scan_kernel(const __grid_constant__ Params p, const TopkSide s) {
-    __shared__ uint32_t sg[THREADS], st[THREADS];
-    __shared__ uint32_t carry_sel, carry_ties;
+    __shared__ uint32_t warp_tot[8];
+    constexpr int PER = 4;  // consecutive tiles per thread and round
     const int t = blockIdx.x, row = blockIdx.y;
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
     if (sel[SEL_FLAGS] & 1u) return;
     const int first = __ldg(p.tile_prefix + t), ntiles = __ldg(p.tile_prefix + t + 1) - first;
     const uint32_t ties_wanted = sel[SEL_TIES];
     const uint32_t kbeg = (uint32_t)__ldg(p.k_off + t), k = (uint32_t)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
-    if (threadIdx.x == 0) { carry_sel = 0u; carry_ties = 0u; }
-    __syncthreads();
-    for (int c0 = 0; c0 < ntiles; c0 += THREADS) {
-        const int q = c0 + threadIdx.x;
-        uint32_t *m = s.meta + ((int64_t)row * p.TT + first + (q < ntiles ? q : 0)) * 4;
-        const uint32_t g = q < ntiles ? m[2] : 0u, e = q < ntiles ? m[3] : 0u;
-        // exclusive prefix of the tie counts inside the chunk
-        st[threadIdx.x] = e;
-        __syncthreads();
-        for (int offs = 1; offs < THREADS; offs <<= 1) {
-            uint32_t add = threadIdx.x >= offs ? st[threadIdx.x - offs] : 0u;
-            __syncthreads();
-            st[threadIdx.x] += add;
-            __syncthreads();
+    uint32_t carry_sel = 0, carry_ties = 0;  // uniform over the CTA
+    for (int c0 = 0; c0 < ntiles; c0 += THREADS * PER) {
+        const int q0 = c0 + threadIdx.x * PER;
+        uint32_t g[PER], e[PER], esum = 0;
+#pragma unroll
+        for (int u = 0; u < PER; ++u) {
+            const bool in = q0 + u < ntiles;
+            const uint32_t *m = s.meta + ((int64_t)row * p.TT + first + (in ? q0 + u : 0)) * 4;
+            g[u] = in ? m[2] : 0u;
+            e[u] = in ? m[3] : 0u;
+            esum += e[u];
         }
-        const uint32_t ties_before = carry_ties + st[threadIdx.x] - e;
-        uint32_t allowed = 0;
-        if (ties_before < ties_wanted) allowed = min(e, ties_wanted - ties_before);
-        const uint32_t mine = g + allowed;
-        sg[threadIdx.x] = mine;
-        __syncthreads();
-        for (int offs = 1; offs < THREADS; offs <<= 1) {
-            uint32_t add = threadIdx.x >= offs ? sg[threadIdx.x - offs] : 0u;
-            __syncthreads();
-            sg[threadIdx.x] += add;
-            __syncthreads();
+        uint32_t ties_total, sel_total;
+        uint32_t ties_before = carry_ties + block_exclusive_scan(esum, warp_tot, ties_total);
+        uint32_t allowed[PER], mine = 0;
+#pragma unroll
+        for (int u = 0; u < PER; ++u) {
+            allowed[u] = ties_before < ties_wanted ? min(e[u], ties_wanted - ties_before) : 0u;
+            ties_before += e[u];
+            mine += g[u] + allowed[u];
         }
-        if (q < ntiles) {
-            s.outbase[(int64_t)row * (p.TT + 1) + first + q] = kbeg + carry_sel + sg[threadIdx.x] - mine;
-            m[3] = allowed;
-            m[2] = (ties_before + allowed == ties_wanted && allowed > 0) ? 1u : 0u;  // holds the last accepted tie
+        uint32_t out = kbeg + carry_sel + block_exclusive_scan(mine, warp_tot, sel_total);
+        uint32_t tb = ties_before - esum;  // ties before this thread's first tile
+#pragma unroll
+        for (int u = 0; u < PER; ++u) {
+            if (q0 + u < ntiles) {
+                uint32_t *m = s.meta + ((int64_t)row * p.TT + first + q0 + u) * 4;
+                s.outbase[(int64_t)row * (p.TT + 1) + first + q0 + u] = out;
+                m[3] = allowed[u];
+                m[2] = (tb + allowed[u] == ties_wanted && allowed[u] > 0) ? 1u : 0u;  // holds the last accepted tie
+            }
+            out += g[u] + allowed[u];
+            tb += e[u];
         }
-        __syncthreads();
-        if (threadIdx.x == THREADS - 1) { carry_sel += sg[THREADS - 1]; carry_ties += st[THREADS - 1]; }
-        __syncthreads();
+        carry_sel += sel_total;
+        carry_ties += ties_total;
     }
     if (threadIdx.x == 0 && carry_sel != k) atomicOr(p.status, STATUS_COUNT_MISMATCH);
 }
@@ -887,7 +940,10 @@ constexpr int64_t FINISH_ONE_CTA_MAX = 1 << 17;
 
 // Grid of the dense passes that usually have nothing to do on the uplink (their CTAs walk the
 // tiles with a stride and leave at once when no problem takes the regular route).
-static dim3 strided_grid(const Params &p, int rows) { return dim3(p.TT < 592 ? p.TT : 592, rows); }
+static dim3 strided_grid(const Params &p, int rows) {
+    const int per_row = (2368 + rows - 1) / rows;  // about 16 CTAs per SM over all rows
+    return dim3(p.TT < per_row ? p.TT : per_row, rows);
+}
 
 // First dense pass.  Uplink: collect candidates with last step's guess, histogram them and
 // check the guess; then the first-digit histogram for the problems left on the regular route.
