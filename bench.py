@@ -276,6 +276,31 @@ def run_gpu(args, w, rank, world, local_rank):
 
     stage_ms = [statistics.mean(evs[s][q].elapsed_time(evs[s][q + 1]) for s in range(args.steps)) for q in range(4)]
 
+    # the same step replayed from a CUDA graph (one capture of liec_step, K replays): shows what the
+    # launch gaps cost on small workloads; reported beside the headline, not instead of it
+    graph_ms = None
+    if args.cuda_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            ctx.liec_step(G, w["lr"], stream=side)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            ctx.liec_step(G, w["lr"])
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record()
+        for _ in range(args.steps):
+            graph.replay()
+        g1.record()
+        torch.cuda.synchronize()
+        graph_ms = g0.elapsed_time(g1) / args.steps
+        assert ctx.liec_device_status() == 0
+
     # the model-averaging iteration (every 32nd / 100th step in the paper's runs): timed on its own,
     # not part of the headline step
     a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -316,7 +341,7 @@ def run_gpu(args, w, rank, world, local_rank):
         if e2e:
             e2e["ms_per_step"] = e2e_max
     return dict(ms_step=ms_step, stage_ms=dict(zip(stage_names, stage_ms)), launches=launches, clocks=clocks, e2e=e2e,
-                average_ms=average_ms)
+                average_ms=average_ms, graph_ms=graph_ms)
 
 
 def main():
@@ -329,6 +354,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cuda-graph", action="store_true", help="also time the step replayed from a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -395,6 +421,8 @@ def main():
                          "gbs": (N * d * ((2 if w["gdt"] == "bf16" else 4) + 8) + 8 * d) / (r["average_ms"] * 1e-3) / 1e9,
                          "note": "model-averaging iteration of Algorithm 1, timed separately (5 runs)"},
     }
+    if r["graph_ms"] is not None:
+        line["cuda_graph"] = {"ms_per_step": r["graph_ms"], "value": units / (r["graph_ms"] * 1e-3), "unit": UNIT}
     if r["e2e"]:
         line["e2e"] = {"value": units / (r["e2e"]["ms_per_step"] * 1e-3), "unit": UNIT,
                        "h2d_bytes_per_step": r["e2e"]["h2d"], "d2h_bytes_per_step": r["e2e"]["d2h"],
