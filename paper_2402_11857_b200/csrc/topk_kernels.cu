@@ -322,6 +322,29 @@ __global__ void __launch_bounds__(THREADS) topk_hist2_dense_kernel(const __grid_
 // ------------------------------------------------------------------------------------------------
 // filter: one CTA per (tile, row); ordered append of candidates
 // ------------------------------------------------------------------------------------------------
+// Exclusive prefix sum of one value per thread over the CTA (shuffles inside warps, warp totals in
+// shared memory); `total` receives the CTA's sum.  Two barriers.
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t x, uint32_t *warp_tot /*[8]*/, uint32_t &total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = x;
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xffffffffu, inc, m);
+        if (lane >= m) inc += up;
+    }
+    __syncthreads();  // warp_tot may still be read from the previous call
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    uint32_t before = 0;
+    total = 0;
+#pragma unroll
+    for (int w = 0; w < THREADS / 32; ++w) {
+        if (w < warp) before += warp_tot[w];
+        total += warp_tot[w];
+    }
+    return before + inc - x;
+}
+
 // Candidate mask of a thread's 32 elements: bit 4j+c is set when |v[j][c]| is at least `low`
 // (a magnitude bit pattern used as a float: for finite values the order is the same).
 template <bool FAST>
@@ -451,6 +474,122 @@ __global__ void __launch_bounds__(THREADS, 4) topk_filter_kernel(const __grid_co
             s.cand_idx[cbase + o] = flat0 + pos;
             s.cand_val[cbase + o] = val;
         }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// filter for binary32 sources, staged through shared memory by one TMA bulk copy per tile.
+//
+// With the tile in shared memory a thread can own 32 CONSECUTIVE elements (eight 16-byte chunks,
+// read in a lane-rotated order that keeps the banks conflict-free), so its 32-bit candidate mask is
+// already in index order and the position of every candidate follows from one exclusive scan of
+// the per-thread counts: about a third of the instructions of the register version above, which
+// is what this pass is bound by.  Ragged or misaligned tiles are copied with guarded loads instead
+// of the bulk copy and then take the same path.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void *ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
+
+enum { STATUS_COPY_TIMEOUT = 8 };
+
+template <bool SPEC>
+__global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    __shared__ __align__(128) float tile_s[TILE];
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ uint32_t warp_tot[8];
+    __shared__ uint32_t tile_base;
+    if (!SPEC && s.spec && p.status[STATUS_ANY_REGULAR] == 0) return;
+    const int row = blockIdx.y, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bar)));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    uint32_t phase = 0;
+    for (int tile = blockIdx.x; tile < p.TT; tile += gridDim.x) {
+        const TileInfo ti = locate_tile(p, tile);
+        uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
+        float low;
+        if (SPEC) {
+            if (sel[SEL_MODE] != 1u) continue;  // (uniform over the CTA, like every `continue` before the barriers)
+            low = __uint_as_float(sel[SEL_GUESS]);
+        } else {
+            if (s.spec && sel[SEL_MODE] != 0u) continue;
+            const uint32_t flags = sel[SEL_FLAGS];
+            if (flags & 1u) continue;
+            low = __uint_as_float(sel[SEL_PREFIX] << (flags == 2u ? 7 : DIGIT1_SHIFT));
+        }
+        const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
+        const float *tile_ptr = reinterpret_cast<const float *>(s.src) + row_beg + ti.rel;
+        const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+        if (fast) {
+            if (threadIdx.x == 0) {
+                const uint32_t bytes = TILE * sizeof(float);
+                // earlier ordinary reads/writes of the buffer (ordered by the barrier above) before the async copy
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(&bar)), "r"(bytes) : "memory");
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(smem_addr(tile_s)), "l"(tile_ptr), "r"(bytes), "r"(smem_addr(&bar)) : "memory");
+            }
+            // bounded wait for the copy (a wait that never ends must not hang the GPU: flag it and leave)
+            uint32_t done = 0;
+            for (int spin = 0; spin < (1 << 20) && !done; ++spin)
+                asm volatile("{ .reg .pred q; mbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2; selp.u32 %0, 1, 0, q; }"
+                             : "=r"(done) : "r"(smem_addr(&bar)), "r"(phase) : "memory");
+            if (!done) { atomicOr(p.status, STATUS_COPY_TIMEOUT); return; }
+            phase ^= 1u;
+        } else {
+            for (int q = threadIdx.x; q < TILE; q += THREADS) tile_s[q] = q < ti.len ? tile_ptr[q] : 0.0f;
+            __syncthreads();
+        }
+        // 32 consecutive elements per thread, chunk order rotated by the lane
+        const int pos0 = 32 * threadIdx.x;
+        uint32_t mask = 0;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+            const int c = (kk + lane) & 7;
+            const float4 q4 = *reinterpret_cast<const float4 *>(&tile_s[pos0 + 4 * c]);
+            uint32_t nib = (fabsf(q4.x) >= low ? 1u : 0u) | (fabsf(q4.y) >= low ? 2u : 0u) |
+                           (fabsf(q4.z) >= low ? 4u : 0u) | (fabsf(q4.w) >= low ? 8u : 0u);
+            mask |= nib << (4 * c);
+        }
+        if (!fast) {  // drop the padding of a ragged tile
+            const int valid = ti.len - pos0;
+            mask = valid >= 32 ? mask : (valid <= 0 ? 0u : (mask & ((1u << valid) - 1u)));
+        }
+        uint32_t tile_cnt;
+        const uint32_t before = block_exclusive_scan((uint32_t)__popc(mask), warp_tot, tile_cnt);
+        if (threadIdx.x == 0) {
+            const uint32_t cap = (uint32_t)(__ldg(p.cap_off + ti.t + 1) - __ldg(p.cap_off + ti.t));
+            uint32_t at = tile_cnt ? atomicAdd(&sel[SEL_CAND_COUNT], tile_cnt) : 0u;
+            if (at + tile_cnt > cap) {
+                if (SPEC) {  // the guess lets too much through: this problem takes the regular route
+                    sel[SEL_MODE] = 0u;
+                    p.status[STATUS_ANY_REGULAR] = 1;
+                } else {
+                    atomicOr(p.status, STATUS_CAND_OVERFLOW);
+                }
+                at = 0xffffffffu;
+            }
+            tile_base = at;
+            uint32_t *m = s.meta + ((int64_t)row * p.TT + tile) * 4;
+            m[0] = at == 0xffffffffu ? 0u : at;
+            m[1] = at == 0xffffffffu ? 0u : tile_cnt;
+        }
+        __syncthreads();
+        const uint32_t base_now = tile_base;
+        if (base_now != 0xffffffffu && mask != 0u) {
+            const int64_t cbase = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + base_now + before;
+            const uint32_t flat0 = (uint32_t)(ti.seg_beg + ti.rel) + pos0;
+            uint32_t rest = mask, o = 0;
+            while (rest) {  // candidates are rare: usually zero or one iteration
+                const int b = __ffs(rest) - 1;
+                rest &= rest - 1;
+                s.cand_idx[cbase + o] = flat0 + b;
+                s.cand_val[cbase + o] = tile_s[pos0 + b];
+                ++o;
+            }
+        }
+        __syncthreads();  // the tile buffer, warp_tot and tile_base are rewritten by the next tile
     }
 }
 
@@ -615,29 +754,6 @@ __global__ void __launch_bounds__(THREADS) topk_finish_kernel(const __grid_const
 }
 
 // scan: one CTA per (segment, row); tiles of the segment in order
-// Exclusive prefix sum of one value per thread over the CTA (shuffles inside warps, warp totals in
-// shared memory); `total` receives the CTA's sum.  Two barriers.
-__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t x, uint32_t *warp_tot /*[8]*/, uint32_t &total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t inc = x;
-#pragma unroll
-    for (int m = 1; m < 32; m <<= 1) {
-        const uint32_t up = __shfl_up_sync(0xffffffffu, inc, m);
-        if (lane >= m) inc += up;
-    }
-    __syncthreads();  // warp_tot may still be read from the previous call
-    if (lane == 31) warp_tot[warp] = inc;
-    __syncthreads();
-    uint32_t before = 0;
-    total = 0;
-#pragma unroll
-    for (int w = 0; w < THREADS / 32; ++w) {
-        if (w < warp) before += warp_tot[w];
-        total += warp_tot[w];
-    }
-    return before + inc - x;
-}
-
 __global__ void __launch_bounds__(THREADS) topk_scan_kernel(const __grid_constant__ Params p, const TopkSide s) {
     __shared__ uint32_t warp_tot[8];
     constexpr int PER = 4;  // consecutive tiles per thread and round
@@ -955,7 +1071,7 @@ cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int
     if (s.spec) {
         topk_begin_kernel<<<dim3((p.T + 127) / 128, s.R), 128, 0, st>>>(p, s); CHECK_LAUNCH();
         if (bf) topk_filter_kernel<__nv_bfloat16, true><<<g_tiles, THREADS, 0, st>>>(p, s);
-        else topk_filter_kernel<float, true><<<g_tiles, THREADS, 0, st>>>(p, s);
+        else topk_filter_tma_kernel<true><<<g_tiles, THREADS, 0, st>>>(p, s);
         CHECK_LAUNCH();
         topk_cand_hist_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s, 0); CHECK_LAUNCH();
         topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 5); CHECK_LAUNCH();
@@ -980,7 +1096,7 @@ cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, in
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 4); CHECK_LAUNCH();
     const dim3 g_filter = s.spec ? strided_grid(p, s.R) : g_tiles;
     if (bf) topk_filter_kernel<__nv_bfloat16, false><<<g_filter, THREADS, 0, st>>>(p, s);
-    else topk_filter_kernel<float, false><<<g_filter, THREADS, 0, st>>>(p, s);
+    else topk_filter_tma_kernel<false><<<g_filter, THREADS, 0, st>>>(p, s);
     CHECK_LAUNCH();
     if (p.cap_max <= FINISH_ONE_CTA_MAX) {
         topk_finish_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
