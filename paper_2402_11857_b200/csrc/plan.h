@@ -85,6 +85,7 @@ constexpr int SEL_MODE = 14;       // uplink, this step: 1 = candidates collecte
 
 // words of the status block (int32 each)
 constexpr int STATUS_WORD = 0;        // failed internal checks
+constexpr unsigned STATUS_COPY_TIMEOUT = 8;  // bit of the status word: a TMA bulk copy did not land within the wait limit
 constexpr int STATUS_ANY_REGULAR = 12; // uplink: some problem takes the regular two-pass path this step
 constexpr int STATUS_ANY_REFINE = 8;  // +0 uplink, +1 downlink: some problem needs the dense second-digit pass
 

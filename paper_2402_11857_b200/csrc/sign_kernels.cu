@@ -46,62 +46,80 @@ __global__ void __launch_bounds__(THREADS) sign_uplink_kernel(const __grid_const
     if (threadIdx.x == 0) p.up_partials[(int64_t)worker * p.TT + blockIdx.x] = s;
 }
 
-// bfloat16 gradients: the same tile, read with 128-bit loads.  A warp owns its 1024 elements as
-// 4 rows of 256; lane l owns elements 8l..8l+7 of a row (three tree levels in-thread), four
-// lanes share a 32-bit sign word.  Half the load, shuffle and store instructions per element
-// of the 4-wide version, which matters because this pass is instruction-bound on bf16 input.
+// bfloat16 gradients: the tile (16 KB) is staged in shared memory by one TMA bulk copy, then
+// thread q owns elements 32q..32q+31: its sign word needs no shuffles, five tree levels are summed
+// in-thread and one coalesced store writes the warp's 32 words.  This pass is bound by instruction
+// issue (float->double conversions, sign tests), so the saved shuffles, selects and predicated
+// stores matter.  The four 16-byte chunks of a thread are read in a lane-rotated order (bank
+// conflicts), which permutes the chunk sums; only two pairings occur and both are handled below.
+__device__ __forceinline__ uint32_t smem_addr_of(const void *ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
+
 __global__ void __launch_bounds__(THREADS) sign_uplink_bf16_kernel(const __grid_constant__ Params p) {
+    __shared__ __align__(128) unsigned short tile_s[TILE];
+    __shared__ __align__(8) unsigned long long bar;
     __shared__ double warp_sums[8];
     const int worker = blockIdx.y;
     const TileInfo ti = locate_tile(p, blockIdx.x);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int lane = threadIdx.x & 31;
     const int64_t row_beg = (int64_t)worker * p.d + ti.seg_beg;
-    const __nv_bfloat16 *tile_ptr = reinterpret_cast<const __nv_bfloat16 *>(p.G) + row_beg + ti.rel;
+    const unsigned short *tile_ptr = reinterpret_cast<const unsigned short *>(p.G) + row_beg + ti.rel;
     const bool fast = (ti.len == TILE) && ((row_beg & 7) == 0);
-
-    float v[4][8];
     if (fast) {
-        uint4 q[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            q[j] = __ldcs(reinterpret_cast<const uint4 *>(tile_ptr + warp * 1024 + j * 256 + lane * 8));
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            v[j][0] = __uint_as_float(q[j].x << 16); v[j][1] = __uint_as_float(q[j].x & 0xffff0000u);
-            v[j][2] = __uint_as_float(q[j].y << 16); v[j][3] = __uint_as_float(q[j].y & 0xffff0000u);
-            v[j][4] = __uint_as_float(q[j].z << 16); v[j][5] = __uint_as_float(q[j].z & 0xffff0000u);
-            v[j][6] = __uint_as_float(q[j].w << 16); v[j][7] = __uint_as_float(q[j].w & 0xffff0000u);
+        if (threadIdx.x == 0) {
+            const uint32_t bytes = TILE * sizeof(unsigned short);
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr_of(&bar)));
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr_of(&bar)), "r"(bytes) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_addr_of(tile_s)), "l"(tile_ptr), "r"(bytes), "r"(smem_addr_of(&bar)) : "memory");
         }
+        __syncthreads();  // the barrier is initialised before anyone waits on it
+        uint32_t done = 0;  // bounded wait: a copy that never lands is flagged, not waited for
+        for (int spin = 0; spin < (1 << 20) && !done; ++spin)
+            asm volatile("{ .reg .pred q; mbarrier.try_wait.parity.shared::cta.b64 q, [%1], 0; selp.u32 %0, 1, 0, q; }"
+                         : "=r"(done) : "r"(smem_addr_of(&bar)) : "memory");
+        if (!done) { atomicOr(p.status, STATUS_COPY_TIMEOUT); return; }
     } else {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int pos = warp * 1024 + j * 256 + lane * 8;
-#pragma unroll
-            for (int c = 0; c < 8; ++c) v[j][c] = (pos + c < ti.len) ? load1(tile_ptr + pos + c) : 0.0f;
-        }
+        for (int q = threadIdx.x; q < TILE; q += THREADS) tile_s[q] = q < ti.len ? tile_ptr[q] : (unsigned short)0;
+        __syncthreads();
     }
 
-    uint32_t *words = p.up_words + (int64_t)worker * p.W + __ldg(p.word_off + ti.t) + ti.rel / 32;
-    const int nwords = (ti.len + 31) >> 5;
-    double a[4];
+    const int pos0 = 32 * threadIdx.x;
+    const int rot = (lane >> 1) & 3;
+    double cs[4];
+    uint32_t word = 0;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int kk = 0; kk < 4; ++kk) {
+        const int c = (kk + rot) & 3;
+        const uint4 q = *reinterpret_cast<const uint4 *>(&tile_s[pos0 + 8 * c]);
+        float v[8];
+        v[0] = __uint_as_float(q.x << 16); v[1] = __uint_as_float(q.x & 0xffff0000u);
+        v[2] = __uint_as_float(q.y << 16); v[3] = __uint_as_float(q.y & 0xffff0000u);
+        v[4] = __uint_as_float(q.z << 16); v[5] = __uint_as_float(q.z & 0xffff0000u);
+        v[6] = __uint_as_float(q.w << 16); v[7] = __uint_as_float(q.w & 0xffff0000u);
         double d[8];
         uint32_t byte = 0;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            d[c] = (double)fabsf(v[j][c]);
-            if (v[j][c] < 0.0f) byte |= 1u << c;
+        for (int e = 0; e < 8; ++e) {
+            d[e] = (double)fabsf(v[e]);
+            if (v[e] < 0.0f) byte |= 1u << e;
         }
-        a[j] = __dadd_rn(__dadd_rn(__dadd_rn(d[0], d[1]), __dadd_rn(d[2], d[3])),
-                         __dadd_rn(__dadd_rn(d[4], d[5]), __dadd_rn(d[6], d[7])));
-        uint32_t w = byte << (8 * (lane & 3));
-        w |= __shfl_xor_sync(0xffffffffu, w, 1);
-        w |= __shfl_xor_sync(0xffffffffu, w, 2);
-        const int widx = warp * 32 + j * 8 + (lane >> 2);
-        if ((lane & 3) == 0 && widx < nwords) words[widx] = w;
+        cs[kk] = __dadd_rn(__dadd_rn(__dadd_rn(d[0], d[1]), __dadd_rn(d[2], d[3])),
+                           __dadd_rn(__dadd_rn(d[4], d[5]), __dadd_rn(d[6], d[7])));
+        word |= byte << (8 * c);
     }
-    double s = cta_tree_reduce(warp_tree_reduce<4>(a, lane), warp_sums);
+    // chunk c = (kk + rot) mod 4 holds cs[kk]; the tree wants (chunk0 + chunk1) + (chunk2 + chunk3):
+    // rot even -> (cs0 + cs1) + (cs2 + cs3), rot odd -> (cs3 + cs0) + (cs1 + cs2), up to commutation
+    const bool odd = (rot & 1) != 0;
+    const double x = odd ? cs[3] : cs[1], y = odd ? cs[1] : cs[3];
+    double sum = __dadd_rn(__dadd_rn(cs[0], x), __dadd_rn(cs[2], y));
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) sum = __dadd_rn(sum, shfl_xor_f64(sum, m));
+
+    uint32_t *words = p.up_words + (int64_t)worker * p.W + __ldg(p.word_off + ti.t) + ti.rel / 32;
+    const int nwords = (ti.len + 31) >> 5;
+    if ((int)threadIdx.x < nwords) words[threadIdx.x] = word;
+    double s = cta_tree_reduce(sum, warp_sums);
     if (threadIdx.x == 0) p.up_partials[(int64_t)worker * p.TT + blockIdx.x] = s;
 }
 

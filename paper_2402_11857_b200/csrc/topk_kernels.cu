@@ -489,7 +489,6 @@ __global__ void __launch_bounds__(THREADS, 4) topk_filter_kernel(const __grid_co
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_addr(const void *ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
 
-enum { STATUS_COPY_TIMEOUT = 8 };
 
 template <bool SPEC>
 __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_constant__ Params p, const TopkSide s) {
