@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(THREADS, 3) average_step_kernel(const __grid_c
             }
         }
     }
-    const float nf = (float)p.N;
+    const WorkerDivisor by_n(p.N);
     const bool efast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
     float *e_tile = p.e + ti.seg_beg + ti.rel;
 #pragma unroll
@@ -55,8 +55,8 @@ __global__ void __launch_bounds__(THREADS, 3) average_step_kernel(const __grid_c
         else load4_guarded(e_tile, pos, ti.len, ev);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            gs[j][c] = __fadd_rn(ev[c], __fdiv_rn(gs[j][c], nf));  // v
-            xs[j][c] = __fdiv_rn(xs[j][c], nf);                    // xbar
+            gs[j][c] = __fadd_rn(ev[c], by_n(gs[j][c]));  // v
+            xs[j][c] = by_n(xs[j][c]);                    // xbar
         }
         // e' = v - p with p = v
         if (efast) {
@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(THREADS, 3) average_step_kernel(const __grid_c
 __global__ void __launch_bounds__(THREADS) mean_params_kernel(const __grid_constant__ Params p, float *out) {
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const float nf = (float)p.N;
+    const WorkerDivisor by_n(p.N);
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int pos = tile_pos(warp, lane, j);
@@ -118,7 +118,7 @@ __global__ void __launch_bounds__(THREADS) mean_params_kernel(const __grid_const
         float *o = out + ti.seg_beg + ti.rel;
 #pragma unroll
         for (int c = 0; c < 4; ++c)
-            if (pos + c < ti.len) o[pos + c] = __fdiv_rn(acc[c], nf);
+            if (pos + c < ti.len) o[pos + c] = by_n(acc[c]);
     }
 }
 

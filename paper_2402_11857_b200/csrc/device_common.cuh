@@ -67,6 +67,25 @@ __device__ __forceinline__ void load4_guarded(const GT *tile_ptr, int pos, int l
 }
 
 // Position (relative to the tile) of the 4 elements a thread owns in row j of its warp.
+// a / N in binary32, round to nearest even.  When N is a power of two, a / N and a * (1/N) are the
+// same real number (1/N is exact), so one multiplication rounds to the same float as the IEEE
+// division, subnormal results included; every other N takes the division.
+struct WorkerDivisor {
+    float n, inv;
+    bool pow2;
+    __device__ __forceinline__ explicit WorkerDivisor(int N) : n((float)N), inv(1.0f / (float)N), pow2((N & (N - 1)) == 0) {}
+    __device__ __forceinline__ float operator()(float a) const { return pow2 ? __fmul_rn(a, inv) : __fdiv_rn(a, n); }
+    __device__ __forceinline__ void div4(const float (&a)[4], float (&q)[4]) const {
+        if (pow2) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) q[c] = __fmul_rn(a[c], inv);
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) q[c] = __fdiv_rn(a[c], n);
+        }
+    }
+};
+
 __device__ __forceinline__ int tile_pos(int warp, int lane, int j) { return warp * 1024 + j * 128 + lane * 4; }
 
 // ---- balanced binary64 tree -----------------------------------------------------------------

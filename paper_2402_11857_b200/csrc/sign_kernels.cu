@@ -218,7 +218,7 @@ __global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_cons
         }
     }
 
-    const float nf = (float)p.N;
+    const WorkerDivisor by_n(p.N);
     float *e_tile = p.e + ti.seg_beg + ti.rel;
     double a[8];
 #pragma unroll
@@ -227,8 +227,9 @@ __global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_cons
         float ev[4], v[4];
         if (fast) load4_stream(e_tile + pos, ev);
         else load4_guarded(e_tile, pos, ti.len, ev);
+        by_n.div4(acc[j], v);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) v[c] = __fadd_rn(ev[c], __fdiv_rn(acc[j][c], nf));
+        for (int c = 0; c < 4; ++c) v[c] = __fadd_rn(ev[c], v[c]);
         if (fast) {
             *reinterpret_cast<float4 *>(e_tile + pos) = make_float4(v[0], v[1], v[2], v[3]);
         } else {
@@ -299,7 +300,7 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
         }
     }
 
-    const float nf = (float)p.N;
+    const WorkerDivisor by_n(p.N);
     const int pos0 = 32 * threadIdx.x;
     float *e_tile = p.e + ti.seg_beg + ti.rel;
     uint32_t vword = 0u;
@@ -314,8 +315,12 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
         } else {
             load4_guarded(e_tile, pos, ti.len, ev);
         }
+        {
+            const float a4[4] = {acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]};
+            by_n.div4(a4, v);
+        }
 #pragma unroll
-        for (int c = 0; c < 4; ++c) v[c] = __fadd_rn(ev[c], __fdiv_rn(acc[4 * k + c], nf));
+        for (int c = 0; c < 4; ++c) v[c] = __fadd_rn(ev[c], v[c]);
         if (fast) {
             *reinterpret_cast<float4 *>(e_tile + pos) = make_float4(v[0], v[1], v[2], v[3]);
         } else {

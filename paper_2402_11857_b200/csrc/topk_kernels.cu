@@ -945,16 +945,26 @@ __global__ void __launch_bounds__(THREADS) topk_slow_kernel(const __grid_constan
 // ||v||_1 partial (scaled sign).
 // ------------------------------------------------------------------------------------------------
 template <int DOWN>
-__global__ void __launch_bounds__(THREADS) server_topk_kernel(const __grid_constant__ Params p) {
+__global__ void __launch_bounds__(THREADS, 4) server_topk_kernel(const __grid_constant__ Params p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *acc = reinterpret_cast<float *>(smem_raw);                       // [TILE]
     uint32_t *h = reinterpret_cast<uint32_t *>(smem_raw + sizeof(float) * TILE);  // [DIGIT1_BINS] (top-k downlink)
     __shared__ double warp_sums[8];
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int q = threadIdx.x; q < TILE; q += THREADS) acc[q] = 0.0f;
+    for (int q = threadIdx.x; q < TILE / 4; q += THREADS) reinterpret_cast<float4 *>(acc)[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
     if (DOWN == COMP_TOPK)
-        for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) h[b] = 0u;
+        for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(h)[b] = make_uint4(0u, 0u, 0u, 0u);
+    // the tile of e is fetched now, so that its latency overlaps the message entries'
+    const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
+    float *e_tile = p.e + ti.seg_beg + ti.rel;
+    float ev[8][4];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pos = tile_pos(warp, lane, j);
+        if (fast) load4_stream(e_tile + pos, ev[j]);
+        else load4_guarded(e_tile, pos, ti.len, ev[j]);
+    }
     __syncthreads();
     const bool last_tile = (blockIdx.x + 1 == __ldg(p.tile_prefix + ti.t + 1));
     const uint32_t tile_first = (uint32_t)(ti.seg_beg + ti.rel);
@@ -1000,26 +1010,23 @@ __global__ void __launch_bounds__(THREADS) server_topk_kernel(const __grid_const
             __syncthreads();
         }
     }
-    const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
-    const float nf = (float)p.N;
-    float *e_tile = p.e + ti.seg_beg + ti.rel;
+    const WorkerDivisor by_n(p.N);
     const int64_t wbase = __ldg(p.word_off + ti.t) + ti.rel / 32;
     const int nwords = (ti.len + 31) >> 5;
     double a[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int pos = tile_pos(warp, lane, j);
-        float ev[4], v[4];
-        if (fast) load4_stream(e_tile + pos, ev);
-        else load4_guarded(e_tile, pos, ti.len, ev);
+        float v[4];
         const float4 a4 = *reinterpret_cast<const float4 *>(&acc[pos]);
         const float av[4] = {a4.x, a4.y, a4.z, a4.w};
+        by_n.div4(av, v);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             const bool valid = fast || pos + c < ti.len;
-            v[c] = __fadd_rn(ev[c], __fdiv_rn(av[c], nf));
+            v[c] = __fadd_rn(ev[j][c], v[c]);
             if (!valid) v[c] = 0.0f;
-            if (valid && __float_as_uint(v[c]) != __float_as_uint(ev[c])) e_tile[pos + c] = v[c];
+            if (valid && __float_as_uint(v[c]) != __float_as_uint(ev[j][c])) e_tile[pos + c] = v[c];
             if (DOWN == COMP_TOPK && valid) atomicAdd(&h[key_of(v[c]) >> DIGIT1_SHIFT], 1u);
         }
         if (DOWN == COMP_SIGN) {
