@@ -57,6 +57,7 @@ __device__ __forceinline__ uint32_t smem_addr_of(const void *ptr) { return (uint
 __global__ void __launch_bounds__(THREADS) sign_uplink_bf16_kernel(const __grid_constant__ Params p) {
     __shared__ __align__(128) unsigned short tile_s[TILE];
     __shared__ __align__(8) unsigned long long bar;
+    __shared__ int copy_ok;
     __shared__ double warp_sums[8];
     const int worker = blockIdx.y;
     const TileInfo ti = locate_tile(p, blockIdx.x);
@@ -65,6 +66,8 @@ __global__ void __launch_bounds__(THREADS) sign_uplink_bf16_kernel(const __grid_
     const unsigned short *tile_ptr = reinterpret_cast<const unsigned short *>(p.G) + row_beg + ti.rel;
     const bool fast = (ti.len == TILE) && ((row_beg & 7) == 0);
     if (fast) {
+        // one thread issues the copy and waits for it (bounded); the others sleep at the CTA barrier
+        // instead of spending issue slots on polling
         if (threadIdx.x == 0) {
             const uint32_t bytes = TILE * sizeof(unsigned short);
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr_of(&bar)));
@@ -72,13 +75,15 @@ __global__ void __launch_bounds__(THREADS) sign_uplink_bf16_kernel(const __grid_
             asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr_of(&bar)), "r"(bytes) : "memory");
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                          ::"r"(smem_addr_of(tile_s)), "l"(tile_ptr), "r"(bytes), "r"(smem_addr_of(&bar)) : "memory");
+            uint32_t done = 0;
+            for (int spin = 0; spin < (1 << 20) && !done; ++spin)
+                asm volatile("{ .reg .pred q; mbarrier.try_wait.parity.shared::cta.b64 q, [%1], 0; selp.u32 %0, 1, 0, q; }"
+                             : "=r"(done) : "r"(smem_addr_of(&bar)) : "memory");
+            if (!done) atomicOr(p.status, STATUS_COPY_TIMEOUT);  // a copy that never lands is flagged, not waited for
+            copy_ok = (int)done;
         }
-        __syncthreads();  // the barrier is initialised before anyone waits on it
-        uint32_t done = 0;  // bounded wait: a copy that never lands is flagged, not waited for
-        for (int spin = 0; spin < (1 << 20) && !done; ++spin)
-            asm volatile("{ .reg .pred q; mbarrier.try_wait.parity.shared::cta.b64 q, [%1], 0; selp.u32 %0, 1, 0, q; }"
-                         : "=r"(done) : "r"(smem_addr_of(&bar)) : "memory");
-        if (!done) { atomicOr(p.status, STATUS_COPY_TIMEOUT); return; }
+        __syncthreads();
+        if (!copy_ok) return;
     } else {
         for (int q = threadIdx.x; q < TILE; q += THREADS) tile_s[q] = q < ti.len ? tile_ptr[q] : (unsigned short)0;
         __syncthreads();
@@ -88,22 +93,23 @@ __global__ void __launch_bounds__(THREADS) sign_uplink_bf16_kernel(const __grid_
     const int rot = (lane >> 1) & 3;
     double cs[4];
     uint32_t word = 0;
+    const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.0f, 0.0f);
 #pragma unroll
     for (int kk = 0; kk < 4; ++kk) {
         const int c = (kk + rot) & 3;
         const uint4 q = *reinterpret_cast<const uint4 *>(&tile_s[pos0 + 8 * c]);
-        float v[8];
-        v[0] = __uint_as_float(q.x << 16); v[1] = __uint_as_float(q.x & 0xffff0000u);
-        v[2] = __uint_as_float(q.y << 16); v[3] = __uint_as_float(q.y & 0xffff0000u);
-        v[4] = __uint_as_float(q.z << 16); v[5] = __uint_as_float(q.z & 0xffff0000u);
-        v[6] = __uint_as_float(q.w << 16); v[7] = __uint_as_float(q.w & 0xffff0000u);
+        const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
         double d[8];
-        uint32_t byte = 0;
+        uint32_t bits = 0;  // element 2m of the chunk at bit 2m, element 2m+1 at bit 16+2m
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            d[e] = (double)fabsf(v[e]);
-            if (v[e] < 0.0f) byte |= 1u << e;
+        for (int m = 0; m < 4; ++m) {
+            // x < 0 for both halves in one packed bf16 comparison (false for -0, true for negative subnormals)
+            const uint32_t neg = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&w4[m]), zero2);
+            bits |= neg & (0x00010001u << (2 * m));
+            d[2 * m] = (double)__uint_as_float((w4[m] << 16) & 0x7fffffffu);
+            d[2 * m + 1] = (double)__uint_as_float(w4[m] & 0x7fff0000u);
         }
+        const uint32_t byte = (bits | (bits >> 15)) & 0xffu;
         cs[kk] = __dadd_rn(__dadd_rn(__dadd_rn(d[0], d[1]), __dadd_rn(d[2], d[3])),
                            __dadd_rn(__dadd_rn(d[4], d[5]), __dadd_rn(d[6], d[7])));
         word |= byte << (8 * c);

@@ -104,6 +104,26 @@ def test_bf16_gradients_sign():
         P.step(G, 1e-3)
 
 
+def test_bf16_special_values_sign():
+    """Signed zeros, subnormals of both signs, the largest finite values: the sign bit is x < 0, so -0 packs as 0
+    and a negative subnormal as 1; magnitudes enter the L1 sum exactly."""
+    off = [0, 8192 * 3 + 8, 8192 * 3 + 8 + 777]
+    P = _pair(4, off, SIGN, SIGN, grad_dtype=liec.BF16)
+    special = torch.tensor([0x0000, 0x8000, 0x0001, 0x8001, 0x007F, 0x807F, 0x0080, 0x8080, 0x7F7F, 0xFF7F, 0x3F80, 0xBF80],
+                           dtype=torch.int32).to(torch.int16)
+    gen = torch.Generator().manual_seed(77)
+    for step in range(3):
+        G = make_gradients("bf16_outliers", 1e-2, 4, off[-1], step, base_seed=77)
+        bits = G.view(torch.int16)
+        where = torch.randint(0, off[-1], (4, 4000), generator=gen)
+        what = special[torch.randint(0, special.numel(), (4, 4000), generator=gen)]
+        bits.scatter_(1, where, what)
+        if step == 2:  # one whole tile of negative zeros and one of negative subnormals
+            bits[0, :8192] = special[1]
+            bits[1, 8192:16384] = special[3]
+        P.step(G, 1e-3)
+
+
 @pytest.mark.parametrize("up,down", [(IDENT, IDENT), (SIGN, IDENT), (IDENT, SIGN)])
 def test_identity_combinations(up, down):
     lay = ragged_layout()
