@@ -193,7 +193,9 @@ liec_status liec_get_messages(const liec_ctx *ctx, liec_messages *out);
 
 /*
  * Synchronises `stream` and reads the device status word: 0 = clean; non-zero bits name an
- * internal check that failed.  Returns LIEC_ERR_DEVICE_CHECK when non-zero.
+ * internal check that failed (1 selection rank, 2 candidate buffer, 4 output count, 8 a bulk
+ * copy into shared memory that did not complete within its bounded wait; the kernel that saw it
+ * returned without touching its outputs).  Returns LIEC_ERR_DEVICE_CHECK when non-zero.
  */
 liec_status liec_device_status(liec_ctx *ctx, void *stream, int32_t *out);
 
