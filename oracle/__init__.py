@@ -3,8 +3,8 @@
 TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
 benchmark's CPU-baseline leg.  The product library never imports this package.
 """
-from .liec_oracle import (IDENTITY, SIGN, TOPK, build, lib, scale, sign_compress, step,
+from .liec_oracle import (IDENTITY, SIGN, TOPK, RANDK, randk_compress, build, lib, scale, sign_compress, step,
                           topk_compress, tree_abs_sum, widen_bf16, StepResult, average_step, mean_params, tree_sumsq)
 
-__all__ = ["IDENTITY", "SIGN", "TOPK", "build", "lib", "scale", "sign_compress", "step",
+__all__ = ["IDENTITY", "SIGN", "TOPK", "RANDK", "randk_compress", "build", "lib", "scale", "sign_compress", "step",
            "topk_compress", "tree_abs_sum", "widen_bf16", "StepResult", "average_step", "mean_params", "tree_sumsq"]

@@ -19,6 +19,7 @@
  * with C one of
  *   scaled sign, per segment:  C(x)_j = (||x_t||_1 / n_t) sign(x_j)   Def. 4 / Def. 5
  *   top-k, per segment:        keep the k_t entries of largest |x_j|   Def. 2
+ *   random-k, per segment:     keep the entries of a given k_t-subset  Def. 3
  *   identity:                  C(x) = x
  *
  * Readings fixed where the paper is silent (every one is arithmetic that the
@@ -33,6 +34,9 @@
  *   - top-k compares magnitudes through the binary32 bit pattern with the sign
  *     bit cleared; among equal magnitudes the lower index wins, so the selected
  *     set is unique.  The message lists (index, value) ascending by index.
+ *   - random-k draws nothing here: the k_t-subset of every segment (one per worker for the
+ *     uplink, one for the downlink) is an input, listed as flat indices ascending inside the
+ *     segment; the caller samples it uniformly (Def. 3).  The message has the top-k layout.
  *   - The server sums messages in worker order in binary32 starting from +0,
  *     divides by (float)N, then adds e.
  *   - The update is evaluated left to right as printed: ((p - p^i) + g), times
@@ -53,7 +57,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { ORACLE_IDENTITY = 0, ORACLE_SIGN = 1, ORACLE_TOPK = 2 };
+enum { ORACLE_IDENTITY = 0, ORACLE_SIGN = 1, ORACLE_TOPK = 2, ORACLE_RANDK = 3 };
 
 static uint32_t f32_bits(float x) { uint32_t u; memcpy(&u, &x, 4); return u; }
 
@@ -192,14 +196,36 @@ int liec_oracle_topk(const float *x, int32_t T, const int64_t *off, const int64_
     return 0;
 }
 
+/* Segment-wise random-k (Def. 3) with the subset given: set lists, segment after segment, the
+ * k_t flat indices kept in segment t, ascending.  idx/val/dec as for top-k.  Returns 0, or -3
+ * when the set leaves its segment or is not strictly ascending. */
+int liec_oracle_randk(const float *x, int32_t T, const int64_t *off, const int64_t *k,
+                      const uint32_t *set, uint32_t *idx, float *val, float *dec)
+{
+    int64_t q = 0;
+    for (int32_t t = 0; t < T; ++t) {
+        if (dec) for (int64_t j = off[t]; j < off[t + 1]; ++j) dec[j] = 0.0f;
+        for (int64_t r = 0; r < k[t]; ++r, ++q) {
+            int64_t j = (int64_t)set[q];
+            if (j < off[t] || j >= off[t + 1]) return -3;
+            if (r > 0 && set[q - 1] >= set[q]) return -3;
+            idx[q] = set[q];
+            val[q] = x[j];
+            if (dec) dec[j] = x[j];
+        }
+    }
+    return 0;
+}
+
 /* ---- one iteration ----------------------------------------------------------------- */
 
 static int compress(int32_t kind, const float *x, int64_t d, int32_t T, const int64_t *off,
-                    const int64_t *k, uint32_t *words, float *scales, uint32_t *idx, float *val,
-                    float *dec)
+                    const int64_t *k, const uint32_t *set, uint32_t *words, float *scales,
+                    uint32_t *idx, float *val, float *dec)
 {
     if (kind == ORACLE_SIGN) { liec_oracle_sign(x, T, off, words, scales, dec); return 0; }
     if (kind == ORACLE_TOPK) return liec_oracle_topk(x, T, off, k, idx, val, dec);
+    if (kind == ORACLE_RANDK) return set ? liec_oracle_randk(x, T, off, k, set, idx, val, dec) : -3;
     if (kind == ORACLE_IDENTITY) { memcpy(dec, x, (size_t)d * sizeof(float)); return 0; }
     return -2;
 }
@@ -212,10 +238,12 @@ static int compress(int32_t kind, const float *x, int64_t d, int32_t T, const in
  * (up_words [N][W], up_scales [N][T], up_idx/up_val [N][K]), the downlink message
  * (down_words [W], down_scales [T], down_idx/down_val [K]) and v [d].
  * W = sum_t ceil(n_t/32), K = sum_t k_t.
- * Returns 0 on success, -1 out of memory, -2 unknown compressor.
+ * Random-k sides take their subsets from up_sets [N][K] and down_set [K] (NULL otherwise).
+ * Returns 0 on success, -1 out of memory, -2 unknown compressor, -3 bad or missing subset.
  */
-int liec_oracle_step(int32_t N, int64_t d, int32_t T, const int64_t *off,
+int liec_oracle_step_sets(int32_t N, int64_t d, int32_t T, const int64_t *off,
                      int32_t up, int32_t down, const int64_t *k,
+                     const uint32_t *up_sets, const uint32_t *down_set,
                      const float *G, float lr, float *X, float *e,
                      uint32_t *up_words, float *up_scales, uint32_t *up_idx, float *up_val,
                      uint32_t *down_words, float *down_scales, uint32_t *down_idx, float *down_val,
@@ -239,6 +267,7 @@ int liec_oracle_step(int32_t N, int64_t d, int32_t T, const int64_t *off,
     /* Uplink: every worker compresses its own gradient. */
     for (int32_t i = 0; i < N && rc == 0; ++i) {
         rc = compress(up, G + (size_t)i * d, d, T, off, k,
+                      up_sets ? up_sets + (size_t)i * K : NULL,
                       up_words ? up_words + (size_t)i * W : tw,
                       up_scales ? up_scales + (size_t)i * T : ts,
                       up_idx ? up_idx + (size_t)i * K : ti,
@@ -257,7 +286,7 @@ int liec_oracle_step(int32_t N, int64_t d, int32_t T, const int64_t *off,
     if (v_out) memcpy(v_out, v, (size_t)d * sizeof(float));
 
     /* Downlink: the same operator applied to v. */
-    rc = compress(down, v, d, T, off, k,
+    rc = compress(down, v, d, T, off, k, down_set,
                   down_words ? down_words : tw, down_scales ? down_scales : ts,
                   down_idx ? down_idx : ti, down_val ? down_val : tv, p);
     if (rc) goto done;
@@ -281,6 +310,19 @@ int liec_oracle_step(int32_t N, int64_t d, int32_t T, const int64_t *off,
 done:
     free(P); free(v); free(p); free(tw); free(ts); free(ti); free(tv);
     return rc;
+}
+
+/* The same iteration for the compressors that need no subset. */
+int liec_oracle_step(int32_t N, int64_t d, int32_t T, const int64_t *off,
+                     int32_t up, int32_t down, const int64_t *k,
+                     const float *G, float lr, float *X, float *e,
+                     uint32_t *up_words, float *up_scales, uint32_t *up_idx, float *up_val,
+                     uint32_t *down_words, float *down_scales, uint32_t *down_idx, float *down_val,
+                     float *v_out)
+{
+    return liec_oracle_step_sets(N, d, T, off, up, down, k, NULL, NULL, G, lr, X, e,
+                                 up_words, up_scales, up_idx, up_val,
+                                 down_words, down_scales, down_idx, down_val, v_out);
 }
 
 /*

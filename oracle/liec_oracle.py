@@ -14,7 +14,7 @@ from typing import Optional
 
 import numpy as np
 
-IDENTITY, SIGN, TOPK = 0, 1, 2
+IDENTITY, SIGN, TOPK, RANDK = 0, 1, 2, 3
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "liec_oracle.c")
@@ -52,6 +52,11 @@ def _bind(lib: C.CDLL) -> C.CDLL:
     lib.liec_oracle_sign.restype = None
     lib.liec_oracle_topk.argtypes = [p, C.c_int32, p, p, p, p, p]
     lib.liec_oracle_topk.restype = C.c_int
+    lib.liec_oracle_randk.argtypes = [p, C.c_int32, p, p, p, p, p, p]
+    lib.liec_oracle_randk.restype = C.c_int
+    lib.liec_oracle_step_sets.argtypes = [C.c_int32, C.c_int64, C.c_int32, p, C.c_int32, C.c_int32, p, p, p,
+                                          p, C.c_float, p, p] + [p] * 9
+    lib.liec_oracle_step_sets.restype = C.c_int
     lib.liec_oracle_step.argtypes = [C.c_int32, C.c_int64, C.c_int32, p, C.c_int32, C.c_int32, p,
                                      p, C.c_float, p, p] + [p] * 9
     lib.liec_oracle_step.restype = C.c_int
@@ -139,6 +144,24 @@ def topk_compress(x, off, k, _lib=None):
     return idx, val, dec
 
 
+def randk_compress(x, off, k, subset, _lib=None):
+    """(idx, val, decoded) of the segment-wise random-k of x (Def. 3) for the given subset:
+    flat indices, k_t per segment, ascending inside each segment."""
+    x, off = _f32(x), _off(off)
+    k = np.ascontiguousarray(k, dtype=np.int64)
+    subset = np.ascontiguousarray(subset, dtype=np.uint32)
+    T = off.size - 1
+    K = int(k.sum())
+    assert subset.shape == (K,)
+    idx = np.empty(K, dtype=np.uint32)
+    val = np.empty(K, dtype=np.float32)
+    dec = np.empty_like(x)
+    rc = (_lib or lib()).liec_oracle_randk(_ptr(x), T, _ptr(off), _ptr(k), _ptr(subset), _ptr(idx), _ptr(val), _ptr(dec))
+    if rc:
+        raise ValueError(f"oracle random-k rejected the subset (code {rc})")
+    return idx, val, dec
+
+
 @dataclass
 class StepResult:
     up_words: Optional[np.ndarray]
@@ -153,10 +176,12 @@ class StepResult:
 
 
 def step(X: np.ndarray, e: np.ndarray, G: np.ndarray, lr: float, off, up: int, down: int,
-         k=None, _lib=None) -> StepResult:
+         k=None, _lib=None, up_sets=None, down_set=None) -> StepResult:
     """One compressed iteration; X [N,d] and e [d] (float32, contiguous) are updated in place.
 
-    G is [N,d] float32 (widen bf16 with ``widen_bf16`` first).  Returns the messages and v.
+    G is [N,d] float32 (widen bf16 with ``widen_bf16`` first).  A random-k side takes its
+    subsets from ``up_sets`` [N,K] / ``down_set`` [K] (uint32 flat indices, ascending inside each
+    segment).  Returns the messages and v.
     """
     assert X.dtype == np.float32 and X.flags.c_contiguous and X.ndim == 2
     assert e.dtype == np.float32 and e.flags.c_contiguous
@@ -168,23 +193,34 @@ def step(X: np.ndarray, e: np.ndarray, G: np.ndarray, lr: float, off, up: int, d
     W = num_words(off)
     karr = None
     K = 0
-    if TOPK in (up, down):
+    sparse = (TOPK, RANDK)
+    if up in sparse or down in sparse:
         karr = np.ascontiguousarray(k, dtype=np.int64)
         assert karr.shape == (T,)
         K = int(karr.sum())
     r = StepResult(
         up_words=np.zeros((N, W), np.uint32) if up == SIGN else None,
         up_scales=np.zeros((N, T), np.float32) if up == SIGN else None,
-        up_idx=np.zeros((N, K), np.uint32) if up == TOPK else None,
-        up_val=np.zeros((N, K), np.float32) if up == TOPK else None,
+        up_idx=np.zeros((N, K), np.uint32) if up in sparse else None,
+        up_val=np.zeros((N, K), np.float32) if up in sparse else None,
         down_words=np.zeros(W, np.uint32) if down == SIGN else None,
         down_scales=np.zeros(T, np.float32) if down == SIGN else None,
-        down_idx=np.zeros(K, np.uint32) if down == TOPK else None,
-        down_val=np.zeros(K, np.float32) if down == TOPK else None,
+        down_idx=np.zeros(K, np.uint32) if down in sparse else None,
+        down_val=np.zeros(K, np.float32) if down in sparse else None,
         v=np.zeros(d, np.float32),
     )
-    rc = (_lib or lib()).liec_oracle_step(
-        N, d, T, _ptr(off), up, down, _ptr(karr), _ptr(G), C.c_float(lr), _ptr(X), _ptr(e),
+    if up == RANDK:
+        up_sets = np.ascontiguousarray(up_sets, dtype=np.uint32)
+        assert up_sets.shape == (N, K)
+    else:
+        up_sets = None
+    if down == RANDK:
+        down_set = np.ascontiguousarray(down_set, dtype=np.uint32)
+        assert down_set.shape == (K,)
+    else:
+        down_set = None
+    rc = (_lib or lib()).liec_oracle_step_sets(
+        N, d, T, _ptr(off), up, down, _ptr(karr), _ptr(up_sets), _ptr(down_set), _ptr(G), C.c_float(lr), _ptr(X), _ptr(e),
         _ptr(r.up_words), _ptr(r.up_scales), _ptr(r.up_idx), _ptr(r.up_val),
         _ptr(r.down_words), _ptr(r.down_scales), _ptr(r.down_idx), _ptr(r.down_val), _ptr(r.v))
     if rc:

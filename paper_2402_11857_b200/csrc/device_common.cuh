@@ -66,7 +66,6 @@ __device__ __forceinline__ void load4_guarded(const GT *tile_ptr, int pos, int l
     for (int c = 0; c < 4; ++c) v[c] = (pos + c < len) ? load1(tile_ptr + pos + c) : 0.0f;
 }
 
-// Position (relative to the tile) of the 4 elements a thread owns in row j of its warp.
 // a / N in binary32, round to nearest even.  When N is a power of two, a / N and a * (1/N) are the
 // same real number (1/N is exact), so one multiplication rounds to the same float as the IEEE
 // division, subnormal results included; every other N takes the division.
@@ -86,6 +85,7 @@ struct WorkerDivisor {
     }
 };
 
+// Position (relative to the tile) of the 4 elements a thread owns in row j of its warp.
 __device__ __forceinline__ int tile_pos(int warp, int lane, int j) { return warp * 1024 + j * 128 + lane * 4; }
 
 // ---- balanced binary64 tree -----------------------------------------------------------------

@@ -9,7 +9,8 @@ and raises AssertionError when the oracle disagrees with
   * brute-force Python loops for bit packing and for sorting by magnitude (Def. 2),
   * the contraction property of Def. 1 and the identities that follow from Def. 4,
   * the error recursion e_{t+1} = v_t - p_t and Lemma 3,
-  * plain SGD for the identity operator with one worker.
+  * plain SGD for the identity operator with one worker,
+  * Def. 3 / Assumption 4 averaged exactly over every k-subset of a small vector.
 """
 from __future__ import annotations
 
@@ -20,7 +21,7 @@ from fractions import Fraction
 import numpy as np
 
 import oracle
-from oracle import IDENTITY, SIGN, TOPK
+from oracle import IDENTITY, SIGN, TOPK, RANDK
 
 GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
 
@@ -269,6 +270,100 @@ def pin_topk_quantile(L):
     assert np.max(np.abs(x[mask])) <= np.min(np.abs(val))
 
 
+# ----------------------------------------------------------------------------- random-k
+
+def pin_randk_all_subsets(L):
+    """Def. 3 over every k-subset of a small vector, in exact rational arithmetic:
+    the mean of C(x) is (k/d) x (Assumption 4) and the mean of ||x - C(x)||^2 is (1 - k/d) ||x||^2
+    (Def. 1 holds with equality and delta = k/d)."""
+    from itertools import combinations
+    x = np.asarray([1.5, -2.25, 0.0, 3.0, -0.125, 7.0, -1.0], np.float32)
+    d = len(x)
+    xq = [Fraction(float(v)) for v in x]
+    for k in (1, 3, 6, 7):
+        subsets = list(combinations(range(d), k))
+        mean = [Fraction(0)] * d
+        err = Fraction(0)
+        for S in subsets:
+            idx, val, dec = oracle.randk_compress(x, [0, d], [k], np.asarray(S, np.uint32), _lib=L)
+            assert idx.tolist() == list(S) and np.array_equal(val, x[list(S)])
+            assert all((dec[j] == x[j]) if j in S else (dec[j] == 0.0) for j in range(d))
+            for j in range(d):
+                mean[j] += Fraction(float(dec[j]))
+                err += (xq[j] - Fraction(float(dec[j]))) ** 2
+        assert all(mean[j] / len(subsets) == Fraction(k, d) * xq[j] for j in range(d))
+        assert err / len(subsets) == (1 - Fraction(k, d)) * sum(v * v for v in xq)
+
+
+def pin_randk_segments_and_rejects(L):
+    """Flat indices, one subset per segment; a subset that leaves its segment, repeats an index or
+    is not ascending is refused."""
+    x = (np.arange(30, dtype=np.float32) - 11.5)
+    off, k = [0, 4, 5, 30], [2, 1, 6]
+    S = np.asarray([1, 3, 4, 5, 9, 10, 20, 28, 29], np.uint32)
+    idx, val, dec = oracle.randk_compress(x, off, k, S, _lib=L)
+    assert idx.tolist() == S.tolist() and np.array_equal(val, x[S.astype(np.int64)])
+    want = np.zeros_like(x)
+    want[S.astype(np.int64)] = x[S.astype(np.int64)]
+    assert np.array_equal(dec, want)
+    for bad in ([1, 4, 4, 5, 9, 10, 20, 28, 29],      # first segment reaches into the second
+                [1, 3, 4, 5, 9, 9, 20, 28, 29],       # repeated index
+                [3, 1, 4, 5, 9, 10, 20, 28, 29],      # descending
+                [1, 3, 3, 5, 9, 10, 20, 28, 29]):     # second segment's index outside it
+        try:
+            oracle.randk_compress(x, off, k, np.asarray(bad, np.uint32), _lib=L)
+        except ValueError:
+            continue
+        raise AssertionError(f"subset {bad} was accepted")
+
+
+def pin_randk_step_special_cases(L):
+    """Whole iterations with random-k: with every index kept it is the identity operator's step, and
+    with the subsets that top-k would pick it is the top-k step, bit for bit; in general p + e' = v
+    with e' = +0 on the downlink subset, and each worker's update uses its own subset."""
+    rng = np.random.default_rng(91)
+    off = np.asarray([0, 7, 40, 101], np.int64)
+    d, N = 101, 3
+    n = np.diff(off)
+    G = rng.standard_normal((N, d)).astype(np.float32)
+    X0 = rng.standard_normal((N, d)).astype(np.float32)
+    e0 = (rng.standard_normal(d) * 0.1).astype(np.float32)
+    # (a) k_t = n_t
+    full = np.arange(d, dtype=np.uint32)
+    Xa, ea, Xb, eb = X0.copy(), e0.copy(), X0.copy(), e0.copy()
+    ra = oracle.step(Xa, ea, G, 0.1, off, RANDK, RANDK, k=n, up_sets=np.tile(full, (N, 1)), down_set=full, _lib=L)
+    rb = oracle.step(Xb, eb, G, 0.1, off, IDENTITY, IDENTITY, _lib=L)
+    assert np.array_equal(Xa, Xb) and np.array_equal(ea, eb) and np.array_equal(ra.v, rb.v)
+    # (b) the subsets of top-k
+    k = np.asarray([2, 5, 9], np.int64)
+    Xa, ea, Xb, eb = X0.copy(), e0.copy(), X0.copy(), e0.copy()
+    rb = oracle.step(Xb, eb, G, 0.1, off, TOPK, TOPK, k=k, _lib=L)
+    try:
+        ra = oracle.step(Xa, ea, G, 0.1, off, RANDK, RANDK, k=k, up_sets=rb.up_idx, down_set=rb.down_idx, _lib=L)
+    except RuntimeError as err:  # top-k's own index lists must be valid subsets
+        raise AssertionError(str(err))
+    assert np.array_equal(Xa, Xb) and np.array_equal(ea, eb)
+    assert np.array_equal(ra.up_val, rb.up_val) and np.array_equal(ra.down_val, rb.down_val)
+    # (c) arbitrary subsets, the iteration written out with numpy float32
+    sets = np.stack([np.concatenate([np.sort(rng.choice(int(n[t]), int(k[t]), replace=False)) + off[t] for t in range(3)])
+                     for _ in range(N + 1)]).astype(np.uint32)
+    Xa, ea = X0.copy(), e0.copy()
+    ra = oracle.step(Xa, ea, G, 0.1, off, RANDK, RANDK, k=k, up_sets=sets[:N], down_set=sets[N], _lib=L)
+    P = np.zeros((N, d), np.float32)
+    for i in range(N):
+        P[i, sets[i].astype(np.int64)] = G[i, sets[i].astype(np.int64)]
+    acc = np.zeros(d, np.float32)
+    for i in range(N):
+        acc = acc + P[i]
+    v = e0 + acc / np.float32(N)
+    p = np.zeros(d, np.float32)
+    p[sets[N].astype(np.int64)] = v[sets[N].astype(np.int64)]
+    assert np.array_equal(ra.v, v) and np.array_equal(ea, v - p) and np.all(ea[sets[N].astype(np.int64)] == 0.0)
+    assert np.array_equal(ra.down_idx, sets[N]) and np.array_equal(ra.down_val, v[sets[N].astype(np.int64)])
+    for i in range(N):
+        assert np.array_equal(Xa[i], X0[i] - np.float32(0.1) * ((p - P[i]) + G[i]))
+
+
 # ----------------------------------------------------------------------------- whole step
 
 def _random_problem(rng, N, off, integer=False):
@@ -473,4 +568,5 @@ ALL_PINS = [
     pin_blockwise_reduces_to_sign, pin_topk_bruteforce, pin_topk_quantile,
     pin_error_recursion, pin_identity_one_worker_is_sgd, pin_identical_workers,
     pin_lemma3_exact, pin_lemma3_float, pin_bf16_widening, pin_golden_averaging, pin_averaging_properties, pin_sumsq_and_delta,
+    pin_randk_all_subsets, pin_randk_segments_and_rejects, pin_randk_step_special_cases,
 ]

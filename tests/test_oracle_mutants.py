@@ -30,7 +30,7 @@ MUTANTS = {
     "global_error_not_added": ("v[j] = e[j] + mean;", "v[j] = mean;"),
     "global_error_subtracted": ("v[j] = e[j] + mean;", "v[j] = e[j] - mean;"),
     "workers_summed_backwards": ("acc = acc + P[(size_t)i * d + j];", "acc = acc + P[(size_t)(N - 1 - i) * d + j];"),
-    "downlink_compresses_error": ("rc = compress(down, v, d, T, off, k,", "rc = compress(down, e, d, T, off, k,"),
+    "downlink_compresses_error": ("rc = compress(down, v, d, T, off, k, down_set,", "rc = compress(down, e, d, T, off, k, down_set,"),
     "error_update_sign": ("e[j] = v[j] - p[j];", "e[j] = p[j] - v[j];"),
     "compensation_sign": ("float diff = p[j] - pi[j];", "float diff = pi[j] - p[j];"),
     "compensation_dropped": ("const float *pi = P + (size_t)i * d;", "const float *pi = g;"),
@@ -41,6 +41,11 @@ MUTANTS = {
     "averaging_keeps_error": ("e[j] = v[j] - v[j];", "e[j] = e[j];"),
     "mean_model_not_divided": ("xbar[j] = acc / (float)N;", "xbar[j] = acc;"),
     "sumsq_not_squared": ("return a * a;                  /* exact: 24-bit significands */", "return a < 0 ? -a : a;"),
+    "randk_value_from_slot_not_index": ("val[q] = x[j];", "val[q] = x[q];"),
+    "randk_segment_check_dropped": ("if (j < off[t] || j >= off[t + 1]) return -3;", ""),
+    "randk_order_check_dropped": ("if (r > 0 && set[q - 1] >= set[q]) return -3;", ""),
+    "randk_every_worker_uses_first_subset": ("up_sets ? up_sets + (size_t)i * K : NULL", "up_sets"),
+    "randk_downlink_uses_uplink_subset": ("rc = compress(down, v, d, T, off, k, down_set,", "rc = compress(down, v, d, T, off, k, up_sets,"),
     "ascent_instead_of_descent": ("x[j] = x[j] - step;", "x[j] = x[j] + step;"),
 }
 
