@@ -37,22 +37,28 @@ def resolve_workload(name: str):
     """Returns dict(name, N, layout, dist, scale, comp, k, lr, gdt)."""
     from liec_synth import WORKLOADS, flat_layout, scaled_layout, topk_counts
     base, _, div = name.partition("/")
-    if base in WORKLOADS:
+    base, _, variant = base.partition("-")
+    if base in WORKLOADS and variant in ("", "randk"):
         w = WORKLOADS[base]
         lay = w.layout()
         if div:   # "c4/8": same tensor list with every size divided by 8 (profiling-sized case)
             lay = scaled_layout(lay, int(div))
-        k = topk_counts(lay, *w.topk_frac) if w.compressor == "topk" else None
-        return dict(name=name, N=w.num_workers, layout=lay, dist=w.dist, scale=w.scale, comp=w.compressor,
+        comp = w.compressor
+        if variant == "randk":   # "c3-randk": the same tensor list and k, random-k (Def. 3) both ways
+            comp = "randk"
+        k = topk_counts(lay, *w.topk_frac) if comp in ("topk", "randk") else None
+        return dict(name=name, N=w.num_workers, layout=lay, dist=w.dist, scale=w.scale, comp=comp,
                     k=k, lr=w.lr, gdt=w.grad_dtype)
     if name.startswith("sweep-"):
-        # sweep-sign-26, sweep-topk1000-28 (k = n/1000), sweep-topk100-24 (k = n/100): N=8, flat, N(0,1)
+        # sweep-sign-26, sweep-topk1000-28 (k = n/1000), sweep-topk100-24 (k = n/100),
+        # sweep-randk100-26 (random-k, k = n/100): N=8, flat, N(0,1)
         _, comp, logd = name.split("-")
         lay = flat_layout(1 << int(logd))
         if comp == "sign":
             return dict(name=name, N=8, layout=lay, dist="normal", scale=1.0, comp="sign", k=None, lr=0.1, gdt="f32")
-        den = int(comp[len("topk"):])
-        return dict(name=name, N=8, layout=lay, dist="normal", scale=1.0, comp="topk",
+        kind = "randk" if comp.startswith("randk") else "topk"
+        den = int(comp[len(kind):])
+        return dict(name=name, N=8, layout=lay, dist="normal", scale=1.0, comp=kind,
                     k=topk_counts(lay, 1, den), lr=0.1, gdt="f32")
     raise SystemExit(f"unknown workload {name!r}")
 
@@ -64,6 +70,8 @@ def min_bytes_per_step(w) -> float:
     if w["comp"] == "sign":
         return N * d * (2 * g + 8 + 1 / 8) + d * (8 + N / 8 + 1 / 4) + 4 * T * (N + 1)
     K = int(w["k"].sum())
+    if w["comp"] == "randk":   # no dense pass over g on the uplink: the subsets are read, the kept entries gathered
+        return N * d * (g + 8) + 8 * d + 8 * K * (2 * N + 2) + 4 * K * (N + 1)
     return N * d * (2 * g + 8) + 8 * d + 8 * K * (2 * N + 2)
 
 
@@ -73,7 +81,8 @@ def update_kernel_bytes(w) -> float:
     N, d = w["N"], w["layout"].dim
     g = 2 if w["gdt"] == "bf16" else 4
     down = d / 8 if w["comp"] == "sign" else 8 * int(w["k"].sum())
-    return N * d * (g + 8) + down
+    own = 4 * N * int(w["k"].sum()) if w["comp"] == "randk" else 0   # each worker's own index list
+    return N * d * (g + 8) + down + own
 
 
 # DRAM bytes per element-worker of the worker update, from an ncu capture of that kernel on the
@@ -179,18 +188,21 @@ def time_oracle(w, steps: int, warmup: int):
     from liec_synth import make_gradients, topk_counts
     sub, chosen, desc = oracle_sample(w)
     N, d = w["N"], sub.dim
-    comp = oracle.SIGN if w["comp"] == "sign" else oracle.TOPK
+    from liec_synth import random_subsets
+    comp = {"sign": oracle.SIGN, "topk": oracle.TOPK, "randk": oracle.RANDK}[w["comp"]]
     k = None
-    if w["comp"] == "topk":
+    if w["comp"] in ("topk", "randk"):
         k = w["k"][chosen] if chosen is not None else np.asarray([max(1, int(w["k"][0] * d // w["layout"].dim))], np.int64)
     X = np.zeros((N, d), np.float32)
     e = np.zeros(d, np.float32)
+    sets = random_subsets(sub.seg_offsets, k, N + 1, 0, 99) if w["comp"] == "randk" else None
     times = []
     for s in range(warmup + steps):
         G = make_gradients(w["dist"], w["scale"], N, d, s, base_seed=99)
         Gf = oracle.widen_bf16(G.view(torch.int16).numpy().view(np.uint16)) if G.dtype == torch.bfloat16 else G.numpy()
         t0 = time.perf_counter()
-        oracle.step(X, e, Gf, w["lr"], sub.seg_offsets, comp, comp, k=k)
+        oracle.step(X, e, Gf, w["lr"], sub.seg_offsets, comp, comp, k=k,
+                    up_sets=None if sets is None else sets[:N], down_set=None if sets is None else sets[N])
         dt = time.perf_counter() - t0
         if s >= warmup:
             times.append(dt)
@@ -227,12 +239,19 @@ def run_gpu(args, w, rank, world, local_rank):
     torch.cuda.set_device(dev)
     lay = w["layout"]
     N, d = w["N"], lay.dim
-    comp = liec.COMP_SCALED_SIGN if w["comp"] == "sign" else liec.COMP_TOPK
+    comp = {"sign": liec.COMP_SCALED_SIGN, "topk": liec.COMP_TOPK, "randk": liec.COMP_RANDK}[w["comp"]]
     gdt = liec.BF16 if w["gdt"] == "bf16" else liec.F32
     X = torch.zeros(N, d, device=dev)
     e = torch.zeros(d, device=dev)
     ctx = liec.Context(X, e, lay.seg_offsets, comp, comp, w["k"], gdt)
     G = make_gradients(w["dist"], w["scale"], N, d, step=0, base_seed=1000 + rank, device=dev)
+    if w["comp"] == "randk":   # the subsets are inputs: drawn once on the host, resident like the gradients
+        import numpy as np
+        from liec_synth import random_subsets
+        sets = random_subsets(lay.seg_offsets, w["k"], N + 1, 0, 1000 + rank)
+        up_sets = torch.from_numpy(np.ascontiguousarray(sets[:N]).view(np.int32)).to(dev)
+        down_set = torch.from_numpy(np.ascontiguousarray(sets[N]).view(np.int32)).to(dev)
+        ctx.liec_set_subsets(up_sets, down_set)
     torch.cuda.synchronize()
 
     def barrier():

@@ -65,7 +65,7 @@ typedef enum {
     LIEC_ERR_DEVICE_CHECK = 6  /* a kernel recorded an internal inconsistency in the status word */
 } liec_status;
 
-typedef enum { LIEC_COMP_IDENTITY = 0, LIEC_COMP_SCALED_SIGN = 1, LIEC_COMP_TOPK = 2 } liec_comp;
+typedef enum { LIEC_COMP_IDENTITY = 0, LIEC_COMP_SCALED_SIGN = 1, LIEC_COMP_TOPK = 2, LIEC_COMP_RANDK = 3 } liec_comp;
 typedef enum { LIEC_F32 = 0, LIEC_BF16 = 1 } liec_dtype;
 
 typedef struct {
@@ -75,7 +75,7 @@ typedef struct {
     const int64_t *seg_offsets; /* host, T+1 entries, [0] = 0, [T] = d, strictly increasing; copied */
     int32_t uplink;             /* liec_comp used by the workers  (C in the worker compress step) */
     int32_t downlink;           /* liec_comp used by the server   (C in the server compress step) */
-    const int64_t *topk_k;      /* host, T entries, 1 <= k_t <= n_t; needed iff a side is TOPK; copied */
+    const int64_t *topk_k;      /* host, T entries, 1 <= k_t <= n_t; needed iff a side is TOPK or RANDK; copied */
     int32_t grad_dtype;         /* liec_dtype of the gradient rows; params, error, messages are binary32 */
 } liec_config;
 
@@ -83,16 +83,16 @@ typedef struct {
 typedef struct {
     const uint32_t *up_words;    /* [N][W]   sign uplink */
     const float *up_scales;      /* [N][T] */
-    const uint32_t *up_idx;      /* [N][K]   top-k uplink */
+    const uint32_t *up_idx;      /* [N][K]   top-k / random-k uplink */
     const float *up_val;         /* [N][K] */
     const uint32_t *down_words;  /* [W]      sign downlink */
     const float *down_scales;    /* [T] */
-    const uint32_t *down_idx;    /* [K]      top-k downlink */
+    const uint32_t *down_idx;    /* [K]      top-k / random-k downlink */
     const float *down_val;       /* [K] */
     const float *v;              /* [d] v_t; valid between liec_server_aggregate and
                                     liec_downlink_compress (it aliases the error buffer) */
     int64_t num_words;           /* W */
-    int64_t num_topk;            /* K (0 when no side is top-k) */
+    int64_t num_topk;            /* K (0 when no side is top-k or random-k) */
 } liec_messages;
 
 /*
@@ -140,6 +140,26 @@ liec_status liec_uplink_compress(liec_ctx *ctx, const void *grads, void *stream)
 liec_status liec_server_aggregate(liec_ctx *ctx, void *stream);                      /* v = e + mean_i p^i (into error) */
 liec_status liec_downlink_compress(liec_ctx *ctx, void *stream);                     /* p = C(v); error <- v - p */
 liec_status liec_worker_update(liec_ctx *ctx, const void *grads, float lr, void *stream); /* x^i -= lr (p - p^i + g^i) */
+
+/*
+ * Random-k (Def. 3: keep the entries of a k_t-subset of every segment, the subset drawn uniformly
+ * from all k_t-subsets).  The library draws nothing: the caller samples the subsets and hands them
+ * over before the iteration that uses them.
+ *   up_sets   device, [N][K] uint32, K = sum_t k_t: for worker i and segment t the k_t kept flat
+ *             indices (positions in [0, d)), listed segment after segment, strictly ascending
+ *             inside a segment.  Needed iff the uplink is RANDK, else may be NULL.
+ *   down_set  device, [K] uint32, the server's subset in the same layout.  Needed iff the
+ *             downlink is RANDK.
+ * The pointers are kept, not copied: the arrays are the caller's and must stay unchanged until
+ * the iteration's liec_worker_update has run on the stream.  They may be replaced before every
+ * iteration or kept for several.  The message of a RANDK side has the top-k layout (index,
+ * value).  An index outside its segment or out of order is not read: the entry is dropped, bit 16
+ * of the device status word is set and the iteration's results are unspecified (but no access
+ * leaves the buffers).  LIEC_ERR_STATE when called between the stages of an iteration;
+ * liec_uplink_compress / liec_downlink_compress return LIEC_ERR_STATE when a RANDK side has no
+ * subset.
+ */
+liec_status liec_set_subsets(liec_ctx *ctx, const uint32_t *up_sets, const uint32_t *down_set);
 
 /* The four stages in sequence; produces the same bytes as calling them one by one. */
 liec_status liec_step(liec_ctx *ctx, const void *grads, float lr, void *stream);
@@ -195,7 +215,8 @@ liec_status liec_get_messages(const liec_ctx *ctx, liec_messages *out);
  * Synchronises `stream` and reads the device status word: 0 = clean; non-zero bits name an
  * internal check that failed (1 selection rank, 2 candidate buffer, 4 output count, 8 a bulk
  * copy into shared memory that did not complete within its bounded wait; the kernel that saw it
- * returned without touching its outputs).  Returns LIEC_ERR_DEVICE_CHECK when non-zero.
+ * returned without touching its outputs; 16 a random-k subset entry outside its segment or out of
+ * order).  Returns LIEC_ERR_DEVICE_CHECK when non-zero.
  */
 liec_status liec_device_status(liec_ctx *ctx, void *stream, int32_t *out);
 

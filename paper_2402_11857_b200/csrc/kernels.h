@@ -20,6 +20,9 @@ cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, in
 cudaError_t launch_server_topk(const Params &p, cudaStream_t st, int64_t *launches);
 cudaError_t configure_topk_kernels();  // opt-in shared memory sizes; call once per device
 
+// random-k: messages gathered at the caller's subsets, per-tile offsets into them
+cudaError_t launch_randk_compress(const Params &p, bool uplink, cudaStream_t st, int64_t *launches);
+
 // model-averaging iteration and mean model
 cudaError_t launch_average_step(const Params &p, float lr, cudaStream_t st);
 cudaError_t launch_mean_params(const Params &p, float *out, cudaStream_t st);

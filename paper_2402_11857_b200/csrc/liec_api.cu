@@ -65,7 +65,7 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     if (cfg->num_segments < 1) return fail(msg, LIEC_ERR_INVALID_ARG, "num_segments must be >= 1");
     if (cfg->num_segments > 65535) return fail(msg, LIEC_ERR_UNSUPPORTED, "num_segments above 65535 (grid limit)");
     if (!cfg->seg_offsets) return fail(msg, LIEC_ERR_INVALID_ARG, "seg_offsets is NULL");
-    auto comp_ok = [](int32_t c) { return c == LIEC_COMP_IDENTITY || c == LIEC_COMP_SCALED_SIGN || c == LIEC_COMP_TOPK; };
+    auto comp_ok = [](int32_t c) { return c == LIEC_COMP_IDENTITY || c == LIEC_COMP_SCALED_SIGN || c == LIEC_COMP_TOPK || c == LIEC_COMP_RANDK; };
     if (!comp_ok(cfg->uplink) || !comp_ok(cfg->downlink)) return fail(msg, LIEC_ERR_INVALID_ARG, "unknown compressor");
     if (cfg->grad_dtype != LIEC_F32 && cfg->grad_dtype != LIEC_BF16) return fail(msg, LIEC_ERR_INVALID_ARG, "unknown grad_dtype");
     const int T = cfg->num_segments;
@@ -74,9 +74,9 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     for (int t = 0; t < T; ++t)
         if (cfg->seg_offsets[t + 1] <= cfg->seg_offsets[t])
             return fail(msg, LIEC_ERR_INVALID_ARG, "seg_offsets must be strictly increasing");
-    const bool any_topk = cfg->uplink == LIEC_COMP_TOPK || cfg->downlink == LIEC_COMP_TOPK;
+    const bool any_topk = comp_is_sparse(cfg->uplink) || comp_is_sparse(cfg->downlink);  // sides with k entries per segment
     if (any_topk) {
-        if (!cfg->topk_k) return fail(msg, LIEC_ERR_INVALID_ARG, "topk_k is NULL but a side uses top-k");
+        if (!cfg->topk_k) return fail(msg, LIEC_ERR_INVALID_ARG, "topk_k is NULL but a side uses top-k or random-k");
         for (int t = 0; t < T; ++t) {
             int64_t n = cfg->seg_offsets[t + 1] - cfg->seg_offsets[t];
             if (cfg->topk_k[t] < 1 || cfg->topk_k[t] > n)
@@ -156,6 +156,16 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
         meta = c.take(sizeof(uint32_t) * rows * pl.TT * 4);
         outbase = c.take(sizeof(uint32_t) * rows * (pl.TT + 1));
     };
+    // random-k needs the message and the per-tile offsets only
+    auto randk_regions = [&](size_t rows, Region &idx, Region &val, Region &outbase) {
+        idx = c.take(sizeof(uint32_t) * rows * pl.K * 2);
+        idx.bytes = sizeof(uint32_t) * rows * pl.K;
+        val.off = idx.off + idx.bytes;
+        val.bytes = sizeof(float) * rows * pl.K;
+        outbase = c.take(sizeof(uint32_t) * rows * (pl.TT + 1));
+    };
+    if (cfg->uplink == LIEC_COMP_RANDK) randk_regions(N, pl.r_up_idx, pl.r_up_val, pl.r_up_outbase);
+    if (cfg->downlink == LIEC_COMP_RANDK) randk_regions(1, pl.r_down_idx, pl.r_down_val, pl.r_down_outbase);
     if (cfg->uplink == LIEC_COMP_TOPK)
         topk_regions(N, pl.r_up_idx, pl.r_up_val, pl.r_up_hist, pl.r_up_hist2, pl.r_up_sel, pl.r_up_cand_idx,
                      pl.r_up_cand_val, pl.r_up_tile_meta, pl.r_up_outbase);
@@ -226,7 +236,7 @@ liec_status liec_wire_bytes(const liec_config *cfg, int64_t *uplink_bytes, int64
     }
     auto message = [&](int32_t comp) -> int64_t {
         if (comp == LIEC_COMP_SCALED_SIGN) return 4 * (pl.W + (int64_t)pl.T);  // packed signs + one scale per segment
-        if (comp == LIEC_COMP_TOPK) return 8 * pl.K;                             // (index, value) pairs
+        if (comp_is_sparse(comp)) return 8 * pl.K;                               // (index, value) pairs
         return 4 * pl.d;                                                          // identity: the dense vector
     };
     if (uplink_bytes) *uplink_bytes = message(cfg->uplink);
@@ -239,7 +249,7 @@ size_t liec_down_message_bytes(const liec_config *cfg) {
     Plan pl;
     if (make_plan(cfg, pl, nullptr) != LIEC_OK) return 0;
     if (cfg->downlink == LIEC_COMP_SCALED_SIGN) return sizeof(uint32_t) * pl.W + sizeof(float) * pl.T;
-    if (cfg->downlink == LIEC_COMP_TOPK) return (sizeof(uint32_t) + sizeof(float)) * pl.K;
+    if (comp_is_sparse(cfg->downlink)) return (sizeof(uint32_t) + sizeof(float)) * pl.K;
     return 0;
 }
 
@@ -356,6 +366,9 @@ liec_status liec_uplink_compress(liec_ctx *c, const void *grads, void *stream) {
     } else if (c->p.up == COMP_TOPK) {
         LIEC_CALL(c, launch_topk_hist1(c->p, true, s, &c->launches));
         LIEC_CALL(c, launch_topk_select(c->p, true, s, &c->launches));
+    } else if (c->p.up == COMP_RANDK) {
+        if (!c->p.up_sets) { c->err = "random-k uplink: no subsets given (liec_set_subsets)"; return LIEC_ERR_STATE; }
+        LIEC_CALL(c, launch_randk_compress(c->p, true, s, &c->launches));
     }
     c->stage = 1;
     return LIEC_OK;
@@ -365,7 +378,7 @@ liec_status liec_server_aggregate(liec_ctx *c, void *stream) {
     liec_status st = check_stage(c, 1, "liec_server_aggregate");
     if (st != LIEC_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (c->p.up == COMP_TOPK) {
+    if (comp_is_sparse(c->p.up)) {
         LIEC_CALL(c, launch_server_topk(c->p, s, &c->launches));
     } else {
         LIEC_LAUNCH(c, launch_server_dense(c->p, s));
@@ -383,9 +396,12 @@ liec_status liec_downlink_compress(liec_ctx *c, void *stream) {
         LIEC_LAUNCH(c, launch_sign_error(c->p, s));
     } else if (c->p.down == COMP_IDENTITY) {
         LIEC_LAUNCH(c, launch_identity_downlink(c->p, s));
+    } else if (c->p.down == COMP_RANDK) {
+        if (!c->p.down_set) { c->err = "random-k downlink: no subset given (liec_set_subsets)"; return LIEC_ERR_STATE; }
+        LIEC_CALL(c, launch_randk_compress(c->p, false, s, &c->launches));
     } else {
-        // the first-digit histogram of v is fused into the server pass after a top-k uplink
-        if (c->p.up != COMP_TOPK) LIEC_CALL(c, launch_topk_hist1(c->p, false, s, &c->launches));
+        // the first-digit histogram of v is fused into the server pass after a sparse uplink
+        if (!comp_is_sparse(c->p.up)) LIEC_CALL(c, launch_topk_hist1(c->p, false, s, &c->launches));
         LIEC_CALL(c, launch_topk_select(c->p, false, s, &c->launches));
     }
     c->stage = 3;
@@ -399,6 +415,18 @@ liec_status liec_worker_update(liec_ctx *c, const void *grads, float lr, void *s
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     LIEC_LAUNCH(c, launch_worker_update(c->p, lr, s));
     c->stage = 0;
+    return LIEC_OK;
+}
+
+liec_status liec_set_subsets(liec_ctx *c, const uint32_t *up_sets, const uint32_t *down_set) {
+    liec_status st = check_stage(c, 0, "liec_set_subsets");
+    if (st != LIEC_OK) return st;
+    if ((reinterpret_cast<uintptr_t>(up_sets) | reinterpret_cast<uintptr_t>(down_set)) & 3u) {
+        c->err = "subsets must be 4-byte aligned";
+        return LIEC_ERR_INVALID_ARG;
+    }
+    c->p.up_sets = up_sets;
+    c->p.down_set = down_set;
     return LIEC_OK;
 }
 
@@ -459,7 +487,7 @@ liec_status liec_step_host(liec_ctx *c, const void *grads_host, void *grads_dev,
         const void *src = nullptr;
         size_t bytes = 0;
         if (c->p.down == COMP_SIGN) { src = c->p.down_words; bytes = sizeof(uint32_t) * c->p.W + sizeof(float) * c->p.T; }
-        else if (c->p.down == COMP_TOPK) { src = c->p.down_idx; bytes = 2 * sizeof(uint32_t) * c->p.K; }
+        else if (comp_is_sparse(c->p.down)) { src = c->p.down_idx; bytes = 2 * sizeof(uint32_t) * c->p.K; }
         if (bytes) {
             cudaError_t e = cudaMemcpyAsync(down_msg_host, src, bytes, cudaMemcpyDeviceToHost, s);
             if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpyAsync(down message)");

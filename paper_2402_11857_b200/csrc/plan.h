@@ -13,7 +13,9 @@ constexpr int TILE = 8192;             // elements per tile
 constexpr int TILE_WORDS = TILE / 32;  // sign words per tile
 constexpr int THREADS = 256;           // threads per CTA in the tile kernels (8 warps x 1024 elements)
 
-constexpr int COMP_IDENTITY = 0, COMP_SIGN = 1, COMP_TOPK = 2;
+constexpr int COMP_IDENTITY = 0, COMP_SIGN = 1, COMP_TOPK = 2, COMP_RANDK = 3;
+// top-k and random-k share the (index, value) message layout and everything that consumes it
+constexpr bool comp_is_sparse(int c) { return c == COMP_TOPK || c == COMP_RANDK; }
 constexpr int DT_F32 = 0, DT_BF16 = 1;
 
 // top-k selection constants
@@ -49,6 +51,7 @@ struct Params {
     double *tel_partials;  // [N][TT] telemetry (squared norms)
 
     // top-k messages and scratch (row count R = N for uplink, 1 for downlink)
+    const uint32_t *up_sets, *down_set;  // random-k: the caller's subsets [N][K] / [K]
     uint32_t *up_idx;  float *up_val;    // [N][K]
     uint32_t *down_idx; float *down_val; // [K]
     uint32_t *up_hist, *down_hist;       // [R][T][DIGIT1_BINS]
@@ -85,6 +88,7 @@ constexpr int SEL_MODE = 14;       // uplink, this step: 1 = candidates collecte
 
 // words of the status block (int32 each)
 constexpr int STATUS_WORD = 0;        // failed internal checks
+constexpr unsigned STATUS_BAD_SUBSET = 16;   // bit of the status word: a random-k subset entry outside its segment or out of order
 constexpr unsigned STATUS_COPY_TIMEOUT = 8;  // bit of the status word: a TMA bulk copy did not land within the wait limit
 constexpr int STATUS_ANY_REGULAR = 12; // uplink: some problem takes the regular two-pass path this step
 constexpr int STATUS_ANY_REFINE = 8;  // +0 uplink, +1 downlink: some problem needs the dense second-digit pass

@@ -1000,11 +1000,11 @@ __global__ void __launch_bounds__(THREADS, 4) server_topk_kernel(const __grid_co
                 for (int m = 0; m < PRE; ++m)
                     if (pidx[m] != 0xffffffffu) {
                         const uint32_t o = pidx[m] - tile_first;
-                        acc[o] = __fadd_rn(acc[o], pval[m]);
+                        if (o < (uint32_t)TILE) acc[o] = __fadd_rn(acc[o], pval[m]);  // (an entry of a refused subset may lie elsewhere)
                     }
                 for (uint32_t q = beg + sub + 16 * PRE; q < end; q += 16) {
                     const uint32_t o = idx[q] - tile_first;
-                    acc[o] = __fadd_rn(acc[o], val[q]);
+                    if (o < (uint32_t)TILE) acc[o] = __fadd_rn(acc[o], val[q]);
                 }
             }
             __syncthreads();

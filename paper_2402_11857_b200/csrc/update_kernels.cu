@@ -1,8 +1,9 @@
 // Local immediate error compensation and model update (last worker step of Algorithm 1):
 //   x^i_j <- x^i_j - eta * ((p_j - p^i_j) + g^i_j)
 // p^i is not stored: it is recomputed from g^i and the worker's own scale (sign), its
-// selection threshold (top-k) or taken as g^i itself (identity).  p is decoded from the
-// downlink message.
+// selection threshold (top-k), its subset (random-k, decoded from the index list into a bit mask
+// of the tile) or taken as g^i itself (identity).  p is decoded from the downlink message; a
+// random-k downlink has the top-k layout and takes the top-k path (DOWN == COMP_TOPK).
 #include "device_common.cuh"
 #include "kernels.h"
 
@@ -11,6 +12,7 @@ namespace liec {
 template <int UP, int DOWN, typename GT>
 __global__ void __launch_bounds__(THREADS) worker_update_kernel(const __grid_constant__ Params p, const float lr) {
     __shared__ __align__(16) float p_tile[DOWN == COMP_TOPK ? TILE : 4];  // decoded downlink message (top-k)
+    __shared__ uint32_t own_mask[UP == COMP_RANDK ? TILE_WORDS : 1];       // the worker's own subset inside this tile
     // With a top-k downlink a CTA serves WPC workers so that the message is decoded once for them.
     constexpr int WPC = DOWN == COMP_TOPK ? 4 : 1;
     const TileInfo ti = locate_tile(p, blockIdx.x);
@@ -64,7 +66,26 @@ __global__ void __launch_bounds__(THREADS) worker_update_kernel(const __grid_con
         const uint32_t beg = p.down_outbase[blockIdx.x];
         const uint32_t end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : p.down_outbase[blockIdx.x + 1];
         const uint32_t tile_first = (uint32_t)(ti.seg_beg + ti.rel);
-        for (uint32_t q = beg + threadIdx.x; q < end; q += THREADS) p_tile[p.down_idx[q] - tile_first] = p.down_val[q];
+        for (uint32_t q = beg + threadIdx.x; q < end; q += THREADS) {
+            const uint32_t o = p.down_idx[q] - tile_first;
+            if (o < (uint32_t)TILE) p_tile[o] = p.down_val[q];
+        }
+        __syncthreads();
+    }
+    if (UP == COMP_RANDK) {
+        if (wq > 0) __syncthreads();  // the previous worker's mask has been read by everyone
+        own_mask[threadIdx.x] = 0u;   // THREADS == TILE_WORDS
+        __syncthreads();
+        const bool last_tile = (blockIdx.x + 1 == __ldg(p.tile_prefix + ti.t + 1));
+        const uint32_t *ob = p.up_outbase + (int64_t)worker * (p.TT + 1) + blockIdx.x;
+        const uint32_t beg = ob[0];
+        const uint32_t end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : ob[1];
+        const uint32_t tile_first = (uint32_t)(ti.seg_beg + ti.rel);
+        const uint32_t *own_idx = p.up_idx + (int64_t)worker * p.K;
+        for (uint32_t q = beg + threadIdx.x; q < end; q += THREADS) {
+            const uint32_t o = own_idx[q] - tile_first;
+            if (o < (uint32_t)TILE) atomicOr(&own_mask[o >> 5], 1u << (o & 31));
+        }
         __syncthreads();
     }
 
@@ -82,10 +103,14 @@ __global__ void __launch_bounds__(THREADS) worker_update_kernel(const __grid_con
             const float4 q4 = *reinterpret_cast<const float4 *>(&p_tile[pos]);
             pd[0] = q4.x; pd[1] = q4.y; pd[2] = q4.z; pd[3] = q4.w;
         }
+        uint32_t own_nib = 0u;
+        if (UP == COMP_RANDK) own_nib = own_mask[pos >> 5] >> (pos & 31);  // pos is a multiple of 4: the four bits share a word
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             float pi;
-            if (UP == COMP_SIGN) {
+            if (UP == COMP_RANDK) {
+                pi = ((own_nib >> c) & 1u) ? g[j][c] : 0.0f;
+            } else if (UP == COMP_SIGN) {
                 pi = __uint_as_float(su_bits ^ (g[j][c] < 0.0f ? 0x80000000u : 0u));
             } else if (UP == COMP_TOPK) {
                 const uint32_t key = __float_as_uint(g[j][c]) & 0x7fffffffu;
@@ -119,7 +144,12 @@ static cudaError_t launch_t(const Params &p, float lr, cudaStream_t st) {
     return cudaGetLastError();
 }
 
-cudaError_t launch_worker_update(const Params &p, float lr, cudaStream_t st) {
+cudaError_t launch_worker_update(const Params &p_in, float lr, cudaStream_t st) {
+    Params p = p_in;
+    if (p.down == COMP_RANDK) p.down = COMP_TOPK;  // same message layout, same decode
+    if (p.up == COMP_RANDK && p.down == COMP_TOPK) return launch_t<COMP_RANDK, COMP_TOPK>(p, lr, st);
+    if (p.up == COMP_RANDK && p.down == COMP_SIGN) return launch_t<COMP_RANDK, COMP_SIGN>(p, lr, st);
+    if (p.up == COMP_RANDK && p.down == COMP_IDENTITY) return launch_t<COMP_RANDK, COMP_IDENTITY>(p, lr, st);
     if (p.up == COMP_SIGN && p.down == COMP_SIGN) return launch_t<COMP_SIGN, COMP_SIGN>(p, lr, st);
     if (p.up == COMP_SIGN && p.down == COMP_IDENTITY) return launch_t<COMP_SIGN, COMP_IDENTITY>(p, lr, st);
     if (p.up == COMP_IDENTITY && p.down == COMP_SIGN) return launch_t<COMP_IDENTITY, COMP_SIGN>(p, lr, st);

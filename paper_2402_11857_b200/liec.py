@@ -11,7 +11,7 @@ from typing import Optional, Sequence
 
 import numpy as np
 
-COMP_IDENTITY, COMP_SCALED_SIGN, COMP_TOPK = 0, 1, 2
+COMP_IDENTITY, COMP_SCALED_SIGN, COMP_TOPK, COMP_RANDK = 0, 1, 2, 3
 SUMSQ_ERROR, SUMSQ_GRADS, SUMSQ_PARAMS = 0, 1, 2
 F32, BF16 = 0, 1
 
@@ -67,6 +67,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.liec_downlink_compress.restype = C.c_int
     lib.liec_worker_update.argtypes = [vp, vp, C.c_float, vp]
     lib.liec_worker_update.restype = C.c_int
+    lib.liec_set_subsets.argtypes = [vp, vp, vp]
+    lib.liec_set_subsets.restype = C.c_int
     lib.liec_step.argtypes = [vp, vp, C.c_float, vp]
     lib.liec_step.restype = C.c_int
     lib.liec_average_step.argtypes = [vp, vp, C.c_float, vp]
@@ -205,6 +207,19 @@ class Context:
     def liec_worker_update(self, grads, lr: float, stream=None):
         self._check_grads(grads)
         self._check(self.lib.liec_worker_update(self._ctx, grads.data_ptr(), float(lr), self._stream(stream)))
+
+    def liec_set_subsets(self, up_sets=None, down_set=None):
+        """Random-k: int32/uint32 CUDA tensors [N, K] / [K] of kept flat indices (ascending inside each
+        segment).  The tensors are referenced, not copied; this object keeps them alive."""
+        t = self._torch
+        for name, s, shape in (("up_sets", up_sets, (self.N, -1)), ("down_set", down_set, (-1,))):
+            if s is None:
+                continue
+            if not s.is_cuda or s.dtype not in (t.int32, t.uint32) or not s.is_contiguous() or s.dim() != len(shape):
+                raise ValueError(f"{name} must be a contiguous CUDA tensor of 32-bit indices")
+        self._subsets = (up_sets, down_set)
+        self._check(self.lib.liec_set_subsets(self._ctx, None if up_sets is None else up_sets.data_ptr(),
+                                              None if down_set is None else down_set.data_ptr()))
 
     def liec_step(self, grads, lr: float, stream=None):
         self._check_grads(grads)

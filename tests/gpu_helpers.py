@@ -40,10 +40,16 @@ class Pair:
         self.ed = torch.from_numpy(self.eh.copy()).to(DEV)
         self.ctx = liec.Context(self.Xd, self.ed, self.off, up, down, self.k, grad_dtype)
 
-    def step(self, G: torch.Tensor, lr: float, staged: bool = False, check_messages: bool = True):
-        """Runs one iteration on both sides and asserts parity of messages and state."""
+    def step(self, G: torch.Tensor, lr: float, staged: bool = False, check_messages: bool = True,
+             up_sets=None, down_set=None):
+        """Runs one iteration on both sides and asserts parity of messages and state.
+        up_sets [N,K] / down_set [K] (numpy uint32): the subsets of a random-k side."""
         Gd = G.to(DEV).contiguous()
-        r = oracle.step(self.Xh, self.eh, widen(G), lr, self.off, self.up, self.down, k=self.k)
+        r = oracle.step(self.Xh, self.eh, widen(G), lr, self.off, self.up, self.down, k=self.k,
+                        up_sets=up_sets, down_set=down_set)
+        if up_sets is not None or down_set is not None:
+            as_dev = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a).view(np.int32)).to(DEV)
+            self.ctx.liec_set_subsets(as_dev(up_sets), as_dev(down_set))
         if staged or check_messages:
             self.ctx.liec_uplink_compress(Gd)
             self.ctx.liec_server_aggregate()
@@ -61,13 +67,13 @@ class Pair:
             if self.up == oracle.SIGN:
                 assert np.array_equal(u32(m["up_words"]), r.up_words), "uplink sign words"
                 assert np.array_equal(f32(m["up_scales"]).view(np.uint32), r.up_scales.view(np.uint32)), "uplink scales"
-            if self.up == oracle.TOPK:
+            if self.up in (oracle.TOPK, oracle.RANDK):
                 assert np.array_equal(u32(m["up_idx"]), r.up_idx), "uplink top-k indices"
                 assert np.array_equal(f32(m["up_val"]).view(np.uint32), r.up_val.view(np.uint32)), "uplink top-k values"
             if self.down == oracle.SIGN:
                 assert np.array_equal(u32(m["down_words"]), r.down_words), "downlink sign words"
                 assert np.array_equal(f32(m["down_scales"]).view(np.uint32), r.down_scales.view(np.uint32)), "downlink scales"
-            if self.down == oracle.TOPK:
+            if self.down in (oracle.TOPK, oracle.RANDK):
                 assert np.array_equal(u32(m["down_idx"]), r.down_idx), "downlink top-k indices"
                 assert np.array_equal(f32(m["down_val"]).view(np.uint32), r.down_val.view(np.uint32)), "downlink top-k values"
         if v is not None:

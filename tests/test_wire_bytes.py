@@ -44,6 +44,12 @@ def test_wire_bytes_of_the_other_messages():
     cfg, keep = liec.make_config(4, off, liec.COMP_SCALED_SIGN, liec.COMP_TOPK, [1, 5, 80])
     up, down, full = liec.liec_wire_bytes(cfg)
     assert up == 4 * ((4 + 2 + 27) + 3) and down == 8 * 86
+    cfg, keep = liec.make_config(4, off, liec.COMP_RANDK, liec.COMP_RANDK, [1, 5, 80])   # (index, value) like top-k
+    up, down, full = liec.liec_wire_bytes(cfg)
+    assert up == down == 8 * 86 and liec.down_message_bytes(cfg) == 8 * 86
+    cfg, keep = liec.make_config(4, off, liec.COMP_RANDK, liec.COMP_RANDK)                # k is required
+    with pytest.raises(liec.LiecError):
+        liec.liec_wire_bytes(cfg)
     cfg, keep = liec.make_config(0, off, 1, 1)
     with pytest.raises(liec.LiecError):
         liec.liec_wire_bytes(cfg)
