@@ -11,7 +11,7 @@ import torch
 
 import oracle
 from gpu_helpers import assert_close, f32, u32, widen
-from liec_synth import WORKLOADS, make_gradients, topk_counts
+from liec_synth import WORKLOADS, make_gradients, random_subsets, topk_counts
 from paper_2402_11857_b200 import liec
 
 pytestmark = pytest.mark.gpu
@@ -28,12 +28,14 @@ def _sample_segments(lay, budget_elems):
     return sorted(chosen)
 
 
-def _run(name, steps, budget_elems):
+def _run(name, steps, budget_elems, randk=False):
     w = WORKLOADS[name]
     lay = w.layout()
     N, d, off = w.num_workers, lay.dim, lay.seg_offsets
     comp = liec.COMP_SCALED_SIGN if w.compressor == "sign" else liec.COMP_TOPK
     ocomp = oracle.SIGN if w.compressor == "sign" else oracle.TOPK
+    if randk:   # the same tensor list and k_t with random-k (Def. 3) both ways
+        comp, ocomp = liec.COMP_RANDK, oracle.RANDK
     k = topk_counts(lay, *w.topk_frac) if w.compressor == "topk" else None
     gdt = liec.BF16 if w.grad_dtype == "bf16" else liec.F32
     X = torch.zeros(N, d, device="cuda")
@@ -53,11 +55,20 @@ def _run(name, steps, budget_elems):
 
     for step in range(steps):
         make_gradients(w.dist, w.scale, N, d, step, base_seed=77, device="cuda", out=G)
+        sub_sets = {}
+        if randk:
+            sets = random_subsets(off, k, N + 1, step, 78)
+            sets_dev = torch.from_numpy(sets.view(np.int32)).cuda()
+            ctx.liec_set_subsets(sets_dev[:N].contiguous(), sets_dev[N].contiguous())
+            # the sampled segments' part of every subset, re-based to the sample's own offsets
+            part = np.concatenate([sets[:, koff[t]:koff[t + 1]].astype(np.int64) - (int(off[t]) - int(sub_off[q]))
+                                   for q, t in enumerate(segs)], axis=1).astype(np.uint32)
+            sub_sets = dict(up_sets=part[:N], down_set=part[N])
         ctx.liec_step(G, w.lr)
         torch.cuda.synchronize()
         assert ctx.liec_device_status() == 0
         m = ctx.liec_get_messages()
-        r = oracle.step(Xh, eh, widen(G[:, cols]), w.lr, sub_off, ocomp, ocomp, k=ksub)
+        r = oracle.step(Xh, eh, widen(G[:, cols]), w.lr, sub_off, ocomp, ocomp, k=ksub, **sub_sets)
         assert_close(f32(X[:, cols]), Xh, f"{name} step {step}: params on sampled segments")
         assert_close(f32(e[cols]), eh, f"{name} step {step}: error on sampled segments")
         if comp == liec.COMP_SCALED_SIGN:
@@ -80,6 +91,12 @@ def _run(name, steps, budget_elems):
                 assert np.array_equal(got, r.up_idx[:, sub_koff[q]:sub_koff[q + 1]].astype(np.int64)), (name, step, t, "up idx")
                 gotd = u32(m["down_idx"][koff[t]:koff[t + 1]]).astype(np.int64) - shift
                 assert np.array_equal(gotd, r.down_idx[sub_koff[q]:sub_koff[q + 1]].astype(np.int64)), (name, step, t, "down idx")
+            if randk:
+                # any size: the message is the subset itself and the values found there, for every worker
+                assert torch.equal(m["up_idx"].view(torch.int32), sets_dev[:N]) and torch.equal(m["down_idx"].view(torch.int32), sets_dev[N])
+                assert torch.equal(m["up_val"], torch.gather(G.float(), 1, sets_dev[:N].long()))
+                assert bool((e[sets_dev[N].long()] == 0).all())
+                continue
             # any size: per segment exactly k_t indices, ascending and inside the segment (worker 0 and N-1)
             for i in (0, N - 1):
                 idx = u32(m["up_idx"][i]).astype(np.int64)
@@ -105,3 +122,7 @@ def test_c3_resnet50_topk_full_size():
 
 def test_c4_gpt2_sign_bf16_full_size():
     _run("c4", steps=2, budget_elems=4_000_000)
+
+
+def test_c3_resnet50_randk_full_size():
+    _run("c3", steps=2, budget_elems=3_500_000, randk=True)
