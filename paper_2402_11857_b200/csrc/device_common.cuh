@@ -66,6 +66,32 @@ __device__ __forceinline__ void load4_guarded(const GT *tile_ptr, int pos, int l
     for (int c = 0; c < 4; ++c) v[c] = (pos + c < len) ? load1(tile_ptr + pos + c) : 0.0f;
 }
 
+// Copies a ragged or misaligned tile into shared memory with ordinary loads; positions at or beyond
+// `len` become +0.  With a 16-byte aligned source whole 16-byte chunks move at once (the chunk
+// that straddles `len` is assembled element by element by the thread that owns it); several loads
+// per thread are in flight either way.  The caller synchronises afterwards.
+template <typename T>
+__device__ __forceinline__ void stage_tile_guarded(T *dst, const T *src, int len, bool aligned16) {
+    constexpr int PER = 16 / (int)sizeof(T);
+    if (aligned16) {
+        const int full = len / PER;
+#pragma unroll 4
+        for (int c = threadIdx.x; c < TILE / PER; c += THREADS) {
+            if (c < full) {
+                reinterpret_cast<uint4 *>(dst)[c] = __ldcs(reinterpret_cast<const uint4 *>(src) + c);
+            } else if (c > full) {
+                reinterpret_cast<uint4 *>(dst)[c] = make_uint4(0u, 0u, 0u, 0u);
+            } else {
+#pragma unroll
+                for (int e = 0; e < PER; ++e) dst[c * PER + e] = (c * PER + e < len) ? src[c * PER + e] : T(0);
+            }
+        }
+    } else {
+#pragma unroll 8
+        for (int q = threadIdx.x; q < TILE; q += THREADS) dst[q] = q < len ? src[q] : T(0);
+    }
+}
+
 // a / N in binary32, round to nearest even.  When N is a power of two, a / N and a * (1/N) are the
 // same real number (1/N is exact), so one multiplication rounds to the same float as the IEEE
 // division, subnormal results included; every other N takes the division.

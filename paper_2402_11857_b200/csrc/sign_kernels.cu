@@ -46,87 +46,132 @@ __global__ void __launch_bounds__(THREADS) sign_uplink_kernel(const __grid_const
     if (threadIdx.x == 0) p.up_partials[(int64_t)worker * p.TT + blockIdx.x] = s;
 }
 
-// bfloat16 gradients: the tile (16 KB) is staged in shared memory by one TMA bulk copy, then
-// thread q owns elements 32q..32q+31: its sign word needs no shuffles, five tree levels are summed
-// in-thread and one coalesced store writes the warp's 32 words.  This pass is bound by instruction
-// issue (float->double conversions, sign tests), so the saved shuffles, selects and predicated
-// stores matter.  The four 16-byte chunks of a thread are read in a lane-rotated order (bank
-// conflicts), which permutes the chunk sums; only two pairings occur and both are handled below.
+// bfloat16 gradients.  A CTA walks UPLINK_TPC consecutive tiles of one worker through a two-stage
+// pipeline: each 16 KB tile is staged in shared memory by one TMA bulk copy (cp.async.bulk + an
+// mbarrier per buffer), and the copy of tile i+2 is issued as soon as tile i has been consumed, so
+// the table lookups and the copy latency of the next tiles hide behind the arithmetic of this one.
+// Thread q owns elements 32q..32q+31 of the tile: its sign word needs no shuffles, five tree
+// levels are summed in-thread and one coalesced store writes the warp's 32 words.  The four
+// 16-byte chunks of a thread are read in an order XOR-rotated by the lane (bank conflicts); an XOR
+// permutes the leaves of the chunk-level tree only inside its own pairs, so the sum is unchanged.
+// One thread polls the mbarrier with a bounded wait; the others sleep at the CTA barrier.
+constexpr int UPLINK_TPC = 4;
+
 __device__ __forceinline__ uint32_t smem_addr_of(const void *ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
 
 __global__ void __launch_bounds__(THREADS) sign_uplink_bf16_kernel(const __grid_constant__ Params p) {
-    __shared__ __align__(128) unsigned short tile_s[TILE];
-    __shared__ __align__(8) unsigned long long bar;
+    __shared__ __align__(128) unsigned short tile_s[2][TILE];
+    __shared__ __align__(8) unsigned long long bar[2];
+    __shared__ int64_t t_src[UPLINK_TPC], t_words[UPLINK_TPC];  // per tile: first element in the row, first word in the row's message
+    __shared__ int t_len[UPLINK_TPC], t_fast[UPLINK_TPC];
     __shared__ int copy_ok;
     __shared__ double warp_sums[8];
     const int worker = blockIdx.y;
-    const TileInfo ti = locate_tile(p, blockIdx.x);
-    const int lane = threadIdx.x & 31;
-    const int64_t row_beg = (int64_t)worker * p.d + ti.seg_beg;
-    const unsigned short *tile_ptr = reinterpret_cast<const unsigned short *>(p.G) + row_beg + ti.rel;
-    const bool fast = (ti.len == TILE) && ((row_beg & 7) == 0);
-    if (fast) {
-        // one thread issues the copy and waits for it (bounded); the others sleep at the CTA barrier
-        // instead of spending issue slots on polling
-        if (threadIdx.x == 0) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int tile0 = blockIdx.x * UPLINK_TPC;
+    const int ntiles = min(UPLINK_TPC, p.TT - tile0);
+    const unsigned short *row = reinterpret_cast<const unsigned short *>(p.G) + (int64_t)worker * p.d;
+    const bool row_aligned = (((int64_t)worker * p.d) & 7) == 0;
+
+    // all table lookups of this CTA's tiles at once, off the per-tile critical path
+    if ((int)threadIdx.x < ntiles) {
+        const TileInfo tn = locate_tile(p, tile0 + threadIdx.x);
+        t_src[threadIdx.x] = tn.seg_beg + tn.rel;
+        t_words[threadIdx.x] = __ldg(p.word_off + tn.t) + tn.rel / 32;
+        t_len[threadIdx.x] = tn.len;
+        t_fast[threadIdx.x] = (tn.len == TILE && row_aligned && (tn.seg_beg & 7) == 0) ? 1 : 0;  // a 16-byte aligned full tile
+    }
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr_of(&bar[0])));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr_of(&bar[1])));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        copy_ok = 1;
+    }
+    __syncthreads();
+
+    uint32_t phase = 0u, pending = 0u;  // thread 0: bit b = parity of the next wait on / a copy in flight into buffer b
+    // thread 0: start the copy of tile tile0 + i into buffer i & 1, if that tile takes the bulk path
+    auto issue = [&](int i) {
+        if (t_fast[i]) {
+            pending |= 1u << (i & 1);
             const uint32_t bytes = TILE * sizeof(unsigned short);
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr_of(&bar)));
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr_of(&bar)), "r"(bytes) : "memory");
+            const uint32_t b = smem_addr_of(&bar[i & 1]);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // earlier generic accesses of the buffer come first
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(bytes) : "memory");
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         ::"r"(smem_addr_of(tile_s)), "l"(tile_ptr), "r"(bytes), "r"(smem_addr_of(&bar)) : "memory");
-            uint32_t done = 0;
-            for (int spin = 0; spin < (1 << 20) && !done; ++spin)
-                asm volatile("{ .reg .pred q; mbarrier.try_wait.parity.shared::cta.b64 q, [%1], 0; selp.u32 %0, 1, 0, q; }"
-                             : "=r"(done) : "r"(smem_addr_of(&bar)) : "memory");
-            if (!done) atomicOr(p.status, STATUS_COPY_TIMEOUT);  // a copy that never lands is flagged, not waited for
-            copy_ok = (int)done;
+                         ::"r"(smem_addr_of(tile_s[i & 1])), "l"(row + t_src[i]), "r"(bytes), "r"(b) : "memory");
+        }
+    };
+    auto wait_for = [&](int buf) -> uint32_t {  // thread 0: bounded wait for the copy in flight into buffer buf
+        uint32_t done = 0;
+        for (int spin = 0; spin < (1 << 20) && !done; ++spin)
+            asm volatile("{ .reg .pred q; mbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2; selp.u32 %0, 1, 0, q; }"
+                         : "=r"(done) : "r"(smem_addr_of(&bar[buf])), "r"((phase >> buf) & 1u) : "memory");
+        if (done) { phase ^= 1u << buf; pending &= ~(1u << buf); }
+        return done;
+    };
+    if (threadIdx.x == 0) {
+        issue(0);
+        if (ntiles > 1) issue(1);
+    }
+
+    for (int i = 0; i < ntiles; ++i) {
+        const int buf = i & 1;
+        const int len = t_len[i];
+        if (t_fast[i]) {
+            if (threadIdx.x == 0 && !wait_for(buf)) {
+                // a copy that does not land is flagged; the other buffer's copy gets one more bounded
+                // wait so that nothing is in flight into this CTA's shared memory when it leaves
+                atomicOr(p.status, STATUS_COPY_TIMEOUT);
+                if (pending & (1u << (buf ^ 1))) wait_for(buf ^ 1);
+                wait_for(buf);
+                copy_ok = 0;
+            }
+        } else {
+            const int64_t src = t_src[i];
+            stage_tile_guarded(tile_s[buf], row + src, len, row_aligned && (src & 7) == 0);
         }
         __syncthreads();
         if (!copy_ok) return;
-    } else {
-        for (int q = threadIdx.x; q < TILE; q += THREADS) tile_s[q] = q < ti.len ? tile_ptr[q] : (unsigned short)0;
-        __syncthreads();
-    }
 
-    const int pos0 = 32 * threadIdx.x;
-    const int rot = (lane >> 1) & 3;
-    double cs[4];
-    uint32_t word = 0;
-    const __nv_bfloat162 zero2 = __floats2bfloat162_rn(0.0f, 0.0f);
+        const int pos0 = 32 * threadIdx.x;
+        const int rot = (lane >> 1) & 3;
+        double cs[4];
+        uint32_t word = 0;
 #pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-        const int c = (kk + rot) & 3;
-        const uint4 q = *reinterpret_cast<const uint4 *>(&tile_s[pos0 + 8 * c]);
-        const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
-        double d[8];
-        uint32_t bits = 0;  // element 2m of the chunk at bit 2m, element 2m+1 at bit 16+2m
+        for (int kk = 0; kk < 4; ++kk) {
+            const int c = kk ^ rot;
+            const uint4 q = *reinterpret_cast<const uint4 *>(&tile_s[buf][pos0 + 8 * c]);
+            const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
+            double d[8];
+            uint32_t byte = 0;
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            // x < 0 for both halves in one packed bf16 comparison (false for -0, true for negative subnormals)
-            const uint32_t neg = __hlt2_mask(*reinterpret_cast<const __nv_bfloat162 *>(&w4[m]), zero2);
-            bits |= neg & (0x00010001u << (2 * m));
-            d[2 * m] = (double)__uint_as_float((w4[m] << 16) & 0x7fffffffu);
-            d[2 * m + 1] = (double)__uint_as_float(w4[m] & 0x7fff0000u);
+            for (int m = 0; m < 4; ++m) {
+                const float lo = __uint_as_float(w4[m] << 16), hi = __uint_as_float(w4[m] & 0xffff0000u);
+                if (lo < 0.0f) byte |= 1u << (2 * m);
+                if (hi < 0.0f) byte |= 2u << (2 * m);
+                d[2 * m] = (double)fabsf(lo);
+                d[2 * m + 1] = (double)fabsf(hi);
+            }
+            cs[kk] = __dadd_rn(__dadd_rn(__dadd_rn(d[0], d[1]), __dadd_rn(d[2], d[3])),
+                               __dadd_rn(__dadd_rn(d[4], d[5]), __dadd_rn(d[6], d[7])));
+            word |= byte << (8 * c);
         }
-        const uint32_t byte = (bits | (bits >> 15)) & 0xffu;
-        cs[kk] = __dadd_rn(__dadd_rn(__dadd_rn(d[0], d[1]), __dadd_rn(d[2], d[3])),
-                           __dadd_rn(__dadd_rn(d[4], d[5]), __dadd_rn(d[6], d[7])));
-        word |= byte << (8 * c);
-    }
-    // chunk c = (kk + rot) mod 4 holds cs[kk]; the tree wants (chunk0 + chunk1) + (chunk2 + chunk3):
-    // rot even -> (cs0 + cs1) + (cs2 + cs3), rot odd -> (cs3 + cs0) + (cs1 + cs2), up to commutation
-    const bool odd = (rot & 1) != 0;
-    const double x = odd ? cs[3] : cs[1], y = odd ? cs[1] : cs[3];
-    double sum = __dadd_rn(__dadd_rn(cs[0], x), __dadd_rn(cs[2], y));
+        // cs[kk] is chunk kk ^ rot: pairs (0,1), (2,3) stay pairs, only their order may swap
+        double sum = __dadd_rn(__dadd_rn(cs[0], cs[1]), __dadd_rn(cs[2], cs[3]));
 #pragma unroll
-    for (int m = 1; m < 32; m <<= 1) sum = __dadd_rn(sum, shfl_xor_f64(sum, m));
+        for (int m = 1; m < 32; m <<= 1) sum = __dadd_rn(sum, shfl_xor_f64(sum, m));
 
-    uint32_t *words = p.up_words + (int64_t)worker * p.W + __ldg(p.word_off + ti.t) + ti.rel / 32;
-    const int nwords = (ti.len + 31) >> 5;
-    if ((int)threadIdx.x < nwords) words[threadIdx.x] = word;
-    double s = cta_tree_reduce(sum, warp_sums);
-    if (threadIdx.x == 0) p.up_partials[(int64_t)worker * p.TT + blockIdx.x] = s;
+        if ((int)threadIdx.x < ((len + 31) >> 5)) p.up_words[(int64_t)worker * p.W + t_words[i] + threadIdx.x] = word;
+        if (lane == 0) warp_sums[warp] = sum;
+        __syncthreads();  // the buffer has been read by everyone; the warp sums are in place
+        if (threadIdx.x == 0 && i + 2 < ntiles) issue(i + 2);
+        if (threadIdx.x == 32) {  // (not thread 0: it is busy with the copies)
+            const double s01 = __dadd_rn(warp_sums[0], warp_sums[1]), s23 = __dadd_rn(warp_sums[2], warp_sums[3]);
+            const double s45 = __dadd_rn(warp_sums[4], warp_sums[5]), s67 = __dadd_rn(warp_sums[6], warp_sums[7]);
+            p.up_partials[(int64_t)worker * p.TT + tile0 + i] = __dadd_rn(__dadd_rn(s01, s23), __dadd_rn(s45, s67));
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -468,7 +513,7 @@ cudaError_t launch_sum_finalize(const Params &p, int rows, double *out, cudaStre
 cudaError_t launch_sign_uplink(const Params &p, cudaStream_t st) {
     dim3 grid(p.TT, p.N);
     if (p.gdt == DT_F32) sign_uplink_kernel<float><<<grid, THREADS, 0, st>>>(p);
-    else sign_uplink_bf16_kernel<<<grid, THREADS, 0, st>>>(p);
+    else sign_uplink_bf16_kernel<<<dim3((p.TT + UPLINK_TPC - 1) / UPLINK_TPC, p.N), THREADS, 0, st>>>(p);
     return cudaGetLastError();
 }
 

@@ -537,7 +537,7 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
             if (!done) { atomicOr(p.status, STATUS_COPY_TIMEOUT); return; }
             phase ^= 1u;
         } else {
-            for (int q = threadIdx.x; q < TILE; q += THREADS) tile_s[q] = q < ti.len ? tile_ptr[q] : 0.0f;
+            stage_tile_guarded(tile_s, tile_ptr, ti.len, (row_beg & 3) == 0);
             __syncthreads();
         }
         // 32 consecutive elements per thread, chunk order rotated by the lane
