@@ -950,6 +950,7 @@ __global__ void __launch_bounds__(THREADS, 4) server_topk_kernel(const __grid_co
     float *acc = reinterpret_cast<float *>(smem_raw);                       // [TILE]
     uint32_t *h = reinterpret_cast<uint32_t *>(smem_raw + sizeof(float) * TILE);  // [DIGIT1_BINS] (top-k downlink)
     __shared__ double warp_sums[8];
+    __shared__ uint32_t s_beg[16], s_end[16];  // this tile's range in each message of the current group of workers
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int q = threadIdx.x; q < TILE / 4; q += THREADS) reinterpret_cast<float4 *>(acc)[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
@@ -968,46 +969,47 @@ __global__ void __launch_bounds__(THREADS, 4) server_topk_kernel(const __grid_co
     __syncthreads();
     const bool last_tile = (blockIdx.x + 1 == __ldg(p.tile_prefix + ti.t + 1));
     const uint32_t tile_first = (uint32_t)(ti.seg_beg + ti.rel);
-    // Workers are taken 16 at a time: 16 threads per worker first fetch that worker's entries for
-    // this tile (all fetches in flight together), then the entries are added worker by worker
-    // so that every element sees its contributions in worker order.
-    constexpr int PRE = 8;  // entries prefetched per thread (16 x 8 = 128 per worker and tile)
-    const int ws = threadIdx.x >> 4, sub = threadIdx.x & 15;
-    for (int g0 = 0; g0 < p.N; g0 += 16) {
-        const int i = g0 + ws;
-        uint32_t beg = 0, end = 0;
-        const uint32_t *idx = nullptr;
-        const float *val = nullptr;
-        if (i < p.N) {
-            const uint32_t *ob = p.up_outbase + (int64_t)i * (p.TT + 1) + blockIdx.x;
-            beg = ob[0];
-            end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : ob[1];
-            idx = p.up_idx + (int64_t)i * p.K;
-            val = p.up_val + (int64_t)i * p.K;
-        }
-        uint32_t pidx[PRE];
-        float pval[PRE];
-#pragma unroll
-        for (int m = 0; m < PRE; ++m) {
-            const uint32_t q = beg + sub + 16 * m;
-            pidx[m] = q < end ? idx[q] : 0xffffffffu;
-            pval[m] = q < end ? val[q] : 0.0f;
-        }
-        const int in_group = min(16, p.N - g0);
-        for (int turn = 0; turn < in_group; ++turn) {
-            if (ws == turn) {
-#pragma unroll
-                for (int m = 0; m < PRE; ++m)
-                    if (pidx[m] != 0xffffffffu) {
-                        const uint32_t o = pidx[m] - tile_first;
-                        if (o < (uint32_t)TILE) acc[o] = __fadd_rn(acc[o], pval[m]);  // (an entry of a refused subset may lie elsewhere)
-                    }
-                for (uint32_t q = beg + sub + 16 * PRE; q < end; q += 16) {
-                    const uint32_t o = idx[q] - tile_first;
-                    if (o < (uint32_t)TILE) acc[o] = __fadd_rn(acc[o], val[q]);
-                }
+    // Workers are taken 8 at a time.  Thread q first fetches entry q of this tile from each of the
+    // 8 messages (all fetches in flight together); then the entries are added worker by worker, one
+    // barrier apart, so that every element sees its contributions in worker order.  Inside one
+    // worker's turn the indices are distinct, so its additions do not depend on one another.
+    constexpr int WG = 8;
+    for (int g0 = 0; g0 < p.N; g0 += WG) {
+        if (threadIdx.x < WG) {
+            const int i = g0 + threadIdx.x;
+            uint32_t beg = 0, end = 0;
+            if (i < p.N) {
+                const uint32_t *ob = p.up_outbase + (int64_t)i * (p.TT + 1) + blockIdx.x;
+                beg = ob[0];
+                end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : ob[1];
             }
-            __syncthreads();
+            s_beg[threadIdx.x] = beg;
+            s_end[threadIdx.x] = end;
+        }
+        __syncthreads();
+        uint32_t pidx[WG];
+        float pval[WG];
+#pragma unroll
+        for (int u = 0; u < WG; ++u) {
+            const uint32_t q = s_beg[u] + threadIdx.x;
+            const bool have = q < s_end[u];   // (beg = end = 0 for workers beyond N)
+            const int64_t at = (int64_t)(g0 + u) * p.K + q;
+            pidx[u] = have ? p.up_idx[at] : 0xffffffffu;
+            pval[u] = have ? p.up_val[at] : 0.0f;
+        }
+#pragma unroll
+        for (int u = 0; u < WG; ++u) {
+            if (g0 + u < p.N) {  // uniform over the CTA
+                const uint32_t o = pidx[u] - tile_first;
+                if (o < (uint32_t)TILE) acc[o] = __fadd_rn(acc[o], pval[u]);  // (absent entries and those of a refused subset fall outside)
+                const uint32_t *idx = p.up_idx + (int64_t)(g0 + u) * p.K;
+                const float *val = p.up_val + (int64_t)(g0 + u) * p.K;
+                for (uint32_t q = s_beg[u] + threadIdx.x + THREADS; q < s_end[u]; q += THREADS) {  // more than 256 entries in this tile
+                    const uint32_t o2 = idx[q] - tile_first;
+                    if (o2 < (uint32_t)TILE) acc[o2] = __fadd_rn(acc[o2], val[q]);
+                }
+                __syncthreads();
+            }
         }
     }
     const WorkerDivisor by_n(p.N);
