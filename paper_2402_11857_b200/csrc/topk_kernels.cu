@@ -617,69 +617,72 @@ __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide 
 // level 1 = second digit of the candidates whose first digit is the threshold's, level 2 = last
 // 7 bits of the candidates under the 24-bit prefix.
 __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_constant__ Params p, const TopkSide s,
-                                                                  const int level) {
+                                                                  const int level, const int reps) {
     __shared__ uint32_t h[DIGIT1_BINS];
     const int row = blockIdx.y, lane = threadIdx.x & 31;
-    const int tile0 = blockIdx.x * 8;
-    const int tile = tile0 + (threadIdx.x >> 5);
-    // When the CTA's 8 tiles lie in one very large segment the counts are
+    // a CTA owns 8 * reps consecutive tiles; warp w takes tiles tile0 + w, tile0 + 8 + w, ...
+    const int tile0 = blockIdx.x * 8 * reps;
+    // When all of the CTA's tiles lie in one very large segment the counts are
     // first gathered in shared memory, so that the segment's global histogram sees a few atomics
     // per CTA instead of a few per warp and iteration.
-    const int tlast = min(tile0 + 7, p.TT - 1);
+    const int tlast = min(tile0 + 8 * reps - 1, p.TT - 1);
     const int seg0 = __ldg(p.tile_seg + tile0);
     // (worth its fixed cost only where many CTAs hammer one histogram: segments of 1024+ tiles)
     const bool gather = seg0 == __ldg(p.tile_seg + tlast) &&
                         __ldg(p.tile_prefix + seg0 + 1) - __ldg(p.tile_prefix + seg0) >= 1024;
     if (gather) {
-        for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) h[b] = 0u;
+        for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(h)[b] = make_uint4(0u, 0u, 0u, 0u);
         __syncthreads();
     }
-    bool active = tile < p.TT;
-    CandBlock cb;
-    uint32_t prefix = 0;
-    if (active) {
-        cb = cand_block(p, s, tile, row);
-        const uint32_t flags = cb.sel[SEL_FLAGS];
-        active = !cb.skip && !(level == 0 && cb.sel[SEL_MODE] != 1u) && !(level == 1 && flags != 0u);
-        prefix = cb.sel[SEL_PREFIX];
-    }
-    uint32_t lo = 0xffffffffu, hi = 0u;
-    if (active) {
-        uint32_t *gh = (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
-        for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
-            const uint32_t q = c0 + lane;
-            uint32_t digit = 0xffffffffu;  // lanes with nothing to add
-            if (q < cb.cnt) {
-                const uint32_t key = key_of(s.cand_val[cb.base + q]);
-                if (level == 0) digit = key >> DIGIT1_SHIFT;
-                else if (level == 1) { if ((key >> DIGIT1_SHIFT) == prefix) digit = (key >> 7) & 0xfffu; }
-                else if ((key >> 7) == prefix) digit = key & 0x7fu;
-            }
-            const uint32_t same = __match_any_sync(0xffffffffu, digit);
-            if (digit != 0xffffffffu) {
-                if (lane == __ffs(same) - 1) {
-                    if (gather) atomicAdd(&h[digit], (uint32_t)__popc(same));
-                    else atomicAdd(gh + digit, (uint32_t)__popc(same));
+    const int lo_word = level == 0 ? SEL_LO1 : SEL_LO2, hi_word = level == 0 ? SEL_HI1 : SEL_HI2;
+    for (int rep = 0; rep < reps; ++rep) {
+        const int tile = tile0 + rep * 8 + (threadIdx.x >> 5);
+        bool active = tile < p.TT;
+        CandBlock cb;
+        uint32_t prefix = 0;
+        if (active) {
+            cb = cand_block(p, s, tile, row);
+            const uint32_t flags = cb.sel[SEL_FLAGS];
+            active = !cb.skip && !(level == 0 && cb.sel[SEL_MODE] != 1u) && !(level == 1 && flags != 0u);
+            prefix = cb.sel[SEL_PREFIX];
+        }
+        uint32_t lo = 0xffffffffu, hi = 0u;
+        if (active) {
+            uint32_t *gh = (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
+            for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
+                const uint32_t q = c0 + lane;
+                uint32_t digit = 0xffffffffu;  // lanes with nothing to add
+                if (q < cb.cnt) {
+                    const uint32_t key = key_of(s.cand_val[cb.base + q]);
+                    if (level == 0) digit = key >> DIGIT1_SHIFT;
+                    else if (level == 1) { if ((key >> DIGIT1_SHIFT) == prefix) digit = (key >> 7) & 0xfffu; }
+                    else if ((key >> 7) == prefix) digit = key & 0x7fu;
                 }
-                lo = min(lo, digit);
-                hi = max(hi, digit);
+                const uint32_t same = __match_any_sync(0xffffffffu, digit);
+                if (digit != 0xffffffffu) {
+                    if (lane == __ffs(same) - 1) {
+                        if (gather) atomicAdd(&h[digit], (uint32_t)__popc(same));
+                        else atomicAdd(gh + digit, (uint32_t)__popc(same));
+                    }
+                    lo = min(lo, digit);
+                    hi = max(hi, digit);
+                }
+            }
+        }
+        if (!gather && active) {  // (uniform over the warp)
+            lo = __reduce_min_sync(0xffffffffu, lo);
+            hi = __reduce_max_sync(0xffffffffu, hi);
+            if (lane == 0 && lo != 0xffffffffu) {
+                atomicMin(&cb.sel[lo_word], lo);
+                atomicMax(&cb.sel[hi_word], hi);
             }
         }
     }
-    const int lo_word = level == 0 ? SEL_LO1 : SEL_LO2, hi_word = level == 0 ? SEL_HI1 : SEL_HI2;
     if (gather) {
         __syncthreads();
         // (all tiles of the CTA share the segment, hence the selection state and the histogram)
-        const int t = __ldg(p.tile_seg + tile0);
-        flush_hist(h, (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + t) * DIGIT1_BINS,
-                   s.sel + ((int64_t)row * p.T + t) * SEL_WORDS, lo_word, hi_word);
-    } else if (active) {
-        lo = __reduce_min_sync(0xffffffffu, lo);
-        hi = __reduce_max_sync(0xffffffffu, hi);
-        if (lane == 0 && lo != 0xffffffffu) {
-            atomicMin(&cb.sel[lo_word], lo);
-            atomicMax(&cb.sel[hi_word], hi);
-        }
+        flush_hist(h, (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + seg0) * DIGIT1_BINS,
+                   s.sel + ((int64_t)row * p.T + seg0) * SEL_WORDS, lo_word, hi_word);
     }
 }
 
@@ -1069,6 +1072,14 @@ static dim3 strided_grid(const Params &p, int rows) {
     return dim3(p.TT < per_row ? p.TT : per_row, rows);
 }
 
+// Candidate histograms: 8 tiles per CTA, or 64 where some segment is large enough for the wide
+// finish step (its CTAs then gather in shared memory and flush once per 64 tiles).
+static int cand_hist_reps(const Params &p) { return p.cap_max > FINISH_ONE_CTA_MAX ? 8 : 1; }
+static dim3 cand_hist_grid(const Params &p, int rows) {
+    const int per = 8 * cand_hist_reps(p);
+    return dim3((p.TT + per - 1) / per, rows);
+}
+
 // First dense pass.  Uplink: collect candidates with last step's guess, histogram them and
 // check the guess; then the first-digit histogram for the problems left on the regular route.
 // Downlink without a fused histogram: plain first-digit histogram of v.
@@ -1081,7 +1092,7 @@ cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int
         if (bf) topk_filter_kernel<__nv_bfloat16, true><<<g_tiles, THREADS, 0, st>>>(p, s);
         else topk_filter_tma_kernel<true><<<g_tiles, THREADS, 0, st>>>(p, s);
         CHECK_LAUNCH();
-        topk_cand_hist_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s, 0); CHECK_LAUNCH();
+        topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 0, cand_hist_reps(p)); CHECK_LAUNCH();
         topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 5); CHECK_LAUNCH();
     }
     const dim3 g_hist = s.spec ? strided_grid(p, s.R) : g_tiles;
@@ -1109,9 +1120,9 @@ cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, in
     if (p.cap_max <= FINISH_ONE_CTA_MAX) {
         topk_finish_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     } else {  // some segment has too many candidates for one CTA: the same two steps, spread over the tile blocks
-        topk_cand_hist_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s, 1); CHECK_LAUNCH();
+        topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 1, cand_hist_reps(p)); CHECK_LAUNCH();
         topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();
-        topk_cand_hist_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();
+        topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 2, cand_hist_reps(p)); CHECK_LAUNCH();
         topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 3); CHECK_LAUNCH();
     }
     topk_count_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
