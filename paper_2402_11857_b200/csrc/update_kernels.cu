@@ -10,7 +10,7 @@
 namespace liec {
 
 template <int UP, int DOWN, typename GT>
-__global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK ? 3 : 1)) worker_update_kernel(const __grid_constant__ Params p, const float lr) {
+__global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK ? 3 : 0)) worker_update_kernel(const __grid_constant__ Params p, const float lr) {
     __shared__ __align__(16) float p_tile[DOWN == COMP_TOPK ? TILE : 4];  // decoded downlink message (top-k)
     __shared__ uint32_t own_mask[UP == COMP_RANDK ? TILE_WORDS : 1];       // the worker's own subset inside this tile
     // With a top-k downlink a CTA serves WPC workers so that the message is decoded once for them.
