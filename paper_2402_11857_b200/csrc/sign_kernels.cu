@@ -193,12 +193,17 @@ __global__ void __launch_bounds__(THREADS) scale_finalize_kernel(const __grid_co
     const int nchunks = (ntiles + FIN_CHUNK - 1) / FIN_CHUNK;
 
     for (int c = 0; c < nchunks; ++c) {
-        for (int q = threadIdx.x; q < FIN_CHUNK; q += THREADS) {
+        // the chunk's tree over the next power of two of its tile count: the levels above it would
+        // only add +0, which changes nothing
+        const int here = min(FIN_CHUNK, ntiles - c * FIN_CHUNK);
+        int span = 1;
+        while (span < here) span <<= 1;
+        for (int q = threadIdx.x; q < span; q += THREADS) {
             int idx = c * FIN_CHUNK + q;
             buf[q] = idx < ntiles ? src[idx] : 0.0;
         }
         __syncthreads();
-        for (int width = FIN_CHUNK / 2; width >= 1; width >>= 1) {
+        for (int width = span / 2; width >= 1; width >>= 1) {
             // pairwise: new[q] = old[2q] + old[2q+1]; done in two phases to avoid overwrite hazards
             double vals[FIN_CHUNK / 2 / THREADS];
 #pragma unroll
