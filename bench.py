@@ -373,7 +373,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cuda-graph", action="store_true", help="also time the step replayed from a CUDA graph")
+    ap.add_argument("--cuda-graph", dest="cuda_graph", action="store_true", default=True,
+                    help="also time the step replayed from a CUDA graph (default; reported beside the headline)")
+    ap.add_argument("--no-cuda-graph", dest="cuda_graph", action="store_false")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
