@@ -220,6 +220,13 @@ liec_status liec_get_messages(const liec_ctx *ctx, liec_messages *out);
  */
 liec_status liec_device_status(liec_ctx *ctx, void *stream, int32_t *out);
 
+/*
+ * Clears the device status word (one 4-byte memset on `stream`).  The word is sticky: once a check
+ * has failed it stays non-zero until this call, so that a failure anywhere in a run is not lost.
+ * The state (params, error) after a flagged iteration is unspecified; restore it before going on.
+ */
+liec_status liec_clear_status(liec_ctx *ctx, void *stream);
+
 /* Number of kernel launches enqueued by this context so far (host-side counter). */
 int64_t liec_launch_count(const liec_ctx *ctx);
 

@@ -523,6 +523,13 @@ liec_status liec_device_status(liec_ctx *c, void *stream, int32_t *out) {
     return LIEC_OK;
 }
 
+liec_status liec_clear_status(liec_ctx *c, void *stream) {
+    if (!c) return LIEC_ERR_INVALID_ARG;
+    cudaError_t e = cudaMemsetAsync(c->p.status, 0, sizeof(int32_t), static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemsetAsync(status)");
+    return LIEC_OK;
+}
+
 int64_t liec_launch_count(const liec_ctx *c) { return c ? c->launches : 0; }
 
 const char *liec_last_error(const liec_ctx *c) { return c ? c->err.c_str() : g_no_ctx_error; }

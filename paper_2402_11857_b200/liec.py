@@ -83,6 +83,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.liec_get_messages.restype = C.c_int
     lib.liec_device_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
     lib.liec_device_status.restype = C.c_int
+    lib.liec_clear_status.argtypes = [vp, vp]
+    lib.liec_clear_status.restype = C.c_int
     lib.liec_launch_count.argtypes = [vp]
     lib.liec_launch_count.restype = C.c_int64
     lib.liec_last_error.argtypes = [vp]
@@ -256,6 +258,9 @@ class Context:
         if st not in (0, 6):
             self._check(st)
         return int(out.value)
+
+    def liec_clear_status(self, stream=None):
+        self._check(self.lib.liec_clear_status(self._ctx, self._stream(stream)))
 
     def liec_launch_count(self) -> int:
         return int(self.lib.liec_launch_count(self._ctx))

@@ -90,6 +90,9 @@ def test_randk_refused_subsets_are_flagged_and_stay_in_bounds():
         ctx.liec_set_subsets(dev(bad), dev(good[0]))
         ctx.liec_step(G, 0.1)
         assert ctx.liec_device_status() & 16
+        assert ctx.liec_device_status() & 16       # sticky until cleared
+        ctx.liec_clear_status()
+        assert ctx.liec_device_status() == 0
         # the same subsets on the downlink
         ctx = liec.Context(torch.zeros(N, d, device=DEV), torch.zeros(d, device=DEV), off, RANDK, RANDK, k)
         ctx.liec_set_subsets(dev(good), dev(bad[1]))
