@@ -23,6 +23,8 @@
 // described at topk_begin_kernel.
 //
 // Nothing waits on another CTA; cross-CTA order comes from kernel boundaries.
+#include <type_traits>
+
 #include "device_common.cuh"
 #include "kernels.h"
 
@@ -345,154 +347,31 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t x, uint32_t *w
     return before + inc - x;
 }
 
-// Candidate mask of a thread's 32 elements: bit 4j+c is set when |v[j][c]| is at least `low`
-// (a magnitude bit pattern used as a float: for finite values the order is the same).
-template <bool FAST>
-__device__ __forceinline__ uint32_t filter_mask(const float (&v)[8][4], float low, int warp, int lane, int len) {
-    uint32_t mask = 0;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int pos = tile_pos(warp, lane, j);
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-            if (fabsf(v[j][c]) >= low && (FAST || pos + c < len)) mask |= 1u << (4 * j + c);
-    }
-    return mask;
-}
-
+// ------------------------------------------------------------------------------------------------
+// filter: the tile is staged through shared memory by one TMA bulk copy.
+//
 // SPEC = true: the uplink's first pass of a step, for problems that have a guess; candidates are
 // the entries at or above the guess.  SPEC = false: the regular pass (threshold bin known from the
 // histogram); on the uplink it only serves the problems that did not take the single-pass route.
-template <typename GT, bool SPEC>
-__global__ void __launch_bounds__(THREADS, 4) topk_filter_kernel(const __grid_constant__ Params p, const TopkSide s) {
-    __shared__ uint32_t warp_tot[8];
-    __shared__ uint32_t tile_base;
-    if (!SPEC && s.spec && p.status[STATUS_ANY_REGULAR] == 0) return;
-    const int row = blockIdx.y;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int tile = blockIdx.x; tile < p.TT; tile += gridDim.x) {
-        const TileInfo ti = locate_tile(p, tile);
-        const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
-        const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
-        const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
-        uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
-        if (!SPEC && s.spec && sel[SEL_MODE] != 0u) continue;  // (all `continue`s before the barriers are uniform)
-        // the streaming loads do not depend on the selection state: issue them first
-        float v[8][4];
-        if (fast) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) load4_stream(tile_ptr + tile_pos(warp, lane, j), v[j]);
-        } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v[j]);
-        }
-        float low;
-        bool refined = false;
-        uint32_t prefix = 0;
-        if (SPEC) {
-            if (sel[SEL_MODE] != 1u) continue;
-            low = __uint_as_float(sel[SEL_GUESS]);
-        } else {
-            const uint32_t flags = sel[SEL_FLAGS];
-            if (flags & 1u) continue;
-            // regular problems compare the first digit, refined ones the 24-bit prefix: either way a
-            // candidate is an entry whose key is at least the prefix shifted back into place
-            refined = flags == 2u;
-            prefix = sel[SEL_PREFIX];
-            low = __uint_as_float(prefix << (refined ? 7 : DIGIT1_SHIFT));
-        }
-        const uint32_t mask = fast ? filter_mask<true>(v, low, warp, lane, ti.len)
-                                   : filter_mask<false>(v, low, warp, lane, ti.len);
-        // per-row counts packed as bytes (rows 0-3, rows 4-7), inclusive scan over lanes
-        uint32_t cnt_lo = 0, cnt_hi = 0;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            cnt_lo |= (uint32_t)__popc((mask >> (4 * j)) & 0xfu) << (8 * j);
-            cnt_hi |= (uint32_t)__popc((mask >> (4 * j + 16)) & 0xfu) << (8 * j);
-        }
-        uint32_t inc_lo = cnt_lo, inc_hi = cnt_hi;
-#pragma unroll
-        for (int m = 1; m < 32; m <<= 1) {
-            const uint32_t a = __shfl_up_sync(0xffffffffu, inc_lo, m), b = __shfl_up_sync(0xffffffffu, inc_hi, m);
-            if (lane >= m) { inc_lo += a; inc_hi += b; }
-        }
-        const uint32_t tot_lo = __shfl_sync(0xffffffffu, inc_lo, 31), tot_hi = __shfl_sync(0xffffffffu, inc_hi, 31);
-        const uint32_t exc_lo = inc_lo - cnt_lo, exc_hi = inc_hi - cnt_hi;
-        // running row bases of the warp, again packed (a warp holds at most 1024 candidates: 16-bit fields)
-        uint32_t running = 0;
-        uint32_t base01 = 0, base23 = 0, base45 = 0, base67 = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const uint32_t total = ((j < 4 ? tot_lo : tot_hi) >> (8 * (j & 3))) & 0xffu;
-            const uint32_t field = running << (16 * (j & 1));
-            if (j < 2) base01 |= field; else if (j < 4) base23 |= field; else if (j < 6) base45 |= field; else base67 |= field;
-            running += total;
-        }
-        if (lane == 0) warp_tot[warp] = running;
-        __syncthreads();
-        uint32_t warp_off = 0, tile_cnt = 0;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) {
-            if (w < warp) warp_off += warp_tot[w];
-            tile_cnt += warp_tot[w];
-        }
-        if (threadIdx.x == 0) {
-            const uint32_t cap = (uint32_t)(__ldg(p.cap_off + ti.t + 1) - __ldg(p.cap_off + ti.t));
-            uint32_t pos0 = tile_cnt ? atomicAdd(&sel[SEL_CAND_COUNT], tile_cnt) : 0u;
-            if (pos0 + tile_cnt > cap) {
-                if (SPEC) {  // the guess lets too much through: this problem takes the regular route
-                    sel[SEL_MODE] = 0u;
-                    p.status[STATUS_ANY_REGULAR] = 1;
-                } else {
-                    atomicOr(p.status, STATUS_CAND_OVERFLOW);
-                }
-                pos0 = 0xffffffffu;
-            }
-            tile_base = pos0;
-            uint32_t *m = s.meta + ((int64_t)row * p.TT + tile) * 4;
-            m[0] = pos0 == 0xffffffffu ? 0u : pos0;
-            m[1] = pos0 == 0xffffffffu ? 0u : tile_cnt;
-        }
-        __syncthreads();
-        const uint32_t base_now = tile_base;
-        if (base_now == 0xffffffffu || mask == 0u) continue;
-        const int64_t cbase = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + base_now + warp_off;
-        const uint32_t flat0 = (uint32_t)(ti.seg_beg + ti.rel);
-        // walk the set bits (candidates are rare: usually zero or one iteration)
-        uint32_t rest = mask;
-        while (rest) {
-            const int b = __ffs(rest) - 1;
-            rest &= rest - 1;
-            const int j = b >> 2;
-            const uint32_t base_pair = j < 2 ? base01 : j < 4 ? base23 : j < 6 ? base45 : base67;
-            const uint32_t row_base = (base_pair >> (16 * (j & 1))) & 0xffffu;
-            const uint32_t before = ((j < 4 ? exc_lo : exc_hi) >> (8 * (j & 3))) & 0xffu;
-            const uint32_t lower = __popc(mask & ((1u << b) - 1u) & (0xfu << (4 * j)));
-            const uint32_t o = row_base + before + lower;
-            const int pos = tile_pos(warp, lane, j) + (b & 3);
-            const float val = load1(tile_ptr + pos);  // read again (cached) rather than kept across the barrier
-            s.cand_idx[cbase + o] = flat0 + pos;
-            s.cand_val[cbase + o] = val;
-        }
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// filter for binary32 sources, staged through shared memory by one TMA bulk copy per tile.
 //
-// With the tile in shared memory a thread can own 32 CONSECUTIVE elements (eight 16-byte chunks,
-// read in a lane-rotated order that keeps the banks conflict-free), so its 32-bit candidate mask is
+// With the tile in shared memory a thread can own 32 CONSECUTIVE elements (16-byte chunks read in
+// a lane-rotated order that keeps the banks conflict-free), so its 32-bit candidate mask is
 // already in index order and the position of every candidate follows from one exclusive scan of
-// the per-thread counts: about a third of the instructions of the register version above, which
-// is what this pass is bound by.  Ragged or misaligned tiles are copied with guarded loads instead
-// of the bulk copy and then take the same path.
+// the per-thread counts.  A candidate is an entry whose magnitude is at least `low` (a magnitude
+// bit pattern used as a float: for finite values the order is the same).  Ragged or misaligned
+// tiles are copied with guarded loads instead of the bulk copy and then take the same path.
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_addr(const void *ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
 
 
-template <bool SPEC>
+// GT = float or __nv_bfloat16: the element type of the source (bf16 tiles are half the bytes; a
+// thread's 32 elements are then four 16-byte chunks instead of eight).
+template <typename GT, bool SPEC>
 __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_constant__ Params p, const TopkSide s) {
-    __shared__ __align__(128) float tile_s[TILE];
+    constexpr bool F32 = sizeof(GT) == 4;
+    using ST = typename std::conditional<F32, float, unsigned short>::type;  // storage type of one element
+    constexpr int ALIGN_MASK = F32 ? 3 : 7;                                  // elements per 16 bytes, minus one
+    __shared__ __align__(128) ST tile_s[TILE];
     __shared__ __align__(8) unsigned long long bar;
     __shared__ uint32_t warp_tot[8];
     __shared__ uint32_t tile_base;
@@ -518,11 +397,11 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
             low = __uint_as_float(sel[SEL_PREFIX] << (flags == 2u ? 7 : DIGIT1_SHIFT));
         }
         const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
-        const float *tile_ptr = reinterpret_cast<const float *>(s.src) + row_beg + ti.rel;
-        const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+        const ST *tile_ptr = reinterpret_cast<const ST *>(s.src) + row_beg + ti.rel;
+        const bool fast = (ti.len == TILE) && ((row_beg & ALIGN_MASK) == 0);
         if (fast) {
             if (threadIdx.x == 0) {
-                const uint32_t bytes = TILE * sizeof(float);
+                const uint32_t bytes = TILE * sizeof(ST);
                 // earlier ordinary reads/writes of the buffer (ordered by the barrier above) before the async copy
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(&bar)), "r"(bytes) : "memory");
@@ -537,19 +416,35 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
             if (!done) { atomicOr(p.status, STATUS_COPY_TIMEOUT); return; }
             phase ^= 1u;
         } else {
-            stage_tile_guarded(tile_s, tile_ptr, ti.len, (row_beg & 3) == 0);
+            stage_tile_guarded(tile_s, tile_ptr, ti.len, (row_beg & ALIGN_MASK) == 0);
             __syncthreads();
         }
         // 32 consecutive elements per thread, chunk order rotated by the lane
         const int pos0 = 32 * threadIdx.x;
         uint32_t mask = 0;
+        if constexpr (F32) {
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-            const int c = (kk + lane) & 7;
-            const float4 q4 = *reinterpret_cast<const float4 *>(&tile_s[pos0 + 4 * c]);
-            uint32_t nib = (fabsf(q4.x) >= low ? 1u : 0u) | (fabsf(q4.y) >= low ? 2u : 0u) |
-                           (fabsf(q4.z) >= low ? 4u : 0u) | (fabsf(q4.w) >= low ? 8u : 0u);
-            mask |= nib << (4 * c);
+            for (int kk = 0; kk < 8; ++kk) {
+                const int c = (kk + lane) & 7;
+                const float4 q4 = *reinterpret_cast<const float4 *>(&tile_s[pos0 + 4 * c]);
+                uint32_t nib = (fabsf(q4.x) >= low ? 1u : 0u) | (fabsf(q4.y) >= low ? 2u : 0u) |
+                               (fabsf(q4.z) >= low ? 4u : 0u) | (fabsf(q4.w) >= low ? 8u : 0u);
+                mask |= nib << (4 * c);
+            }
+        } else {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const int c = (kk + (lane >> 1)) & 3;
+                const uint4 q4 = *reinterpret_cast<const uint4 *>(&tile_s[pos0 + 8 * c]);
+                const uint32_t w4[4] = {q4.x, q4.y, q4.z, q4.w};
+                uint32_t byte = 0;
+#pragma unroll
+                for (int m = 0; m < 4; ++m) {
+                    if (fabsf(__uint_as_float(w4[m] << 16)) >= low) byte |= 1u << (2 * m);
+                    if (fabsf(__uint_as_float(w4[m] & 0xffff0000u)) >= low) byte |= 2u << (2 * m);
+                }
+                mask |= byte << (8 * c);
+            }
         }
         if (!fast) {  // drop the padding of a ragged tile
             const int valid = ti.len - pos0;
@@ -584,7 +479,8 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
                 const int b = __ffs(rest) - 1;
                 rest &= rest - 1;
                 s.cand_idx[cbase + o] = flat0 + b;
-                s.cand_val[cbase + o] = tile_s[pos0 + b];
+                if constexpr (F32) s.cand_val[cbase + o] = tile_s[pos0 + b];
+                else s.cand_val[cbase + o] = __uint_as_float((uint32_t)tile_s[pos0 + b] << 16);
                 ++o;
             }
         }
@@ -1089,8 +985,8 @@ cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int
     const bool bf = uplink && p.gdt == DT_BF16;
     if (s.spec) {
         topk_begin_kernel<<<dim3((p.T + 127) / 128, s.R), 128, 0, st>>>(p, s); CHECK_LAUNCH();
-        if (bf) topk_filter_kernel<__nv_bfloat16, true><<<g_tiles, THREADS, 0, st>>>(p, s);
-        else topk_filter_tma_kernel<true><<<g_tiles, THREADS, 0, st>>>(p, s);
+        if (bf) topk_filter_tma_kernel<__nv_bfloat16, true><<<g_tiles, THREADS, 0, st>>>(p, s);
+        else topk_filter_tma_kernel<float, true><<<g_tiles, THREADS, 0, st>>>(p, s);
         CHECK_LAUNCH();
         topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 0, cand_hist_reps(p)); CHECK_LAUNCH();
         topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 5); CHECK_LAUNCH();
@@ -1114,8 +1010,8 @@ cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, in
     CHECK_LAUNCH();
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 4); CHECK_LAUNCH();
     const dim3 g_filter = s.spec ? strided_grid(p, s.R) : g_tiles;
-    if (bf) topk_filter_kernel<__nv_bfloat16, false><<<g_filter, THREADS, 0, st>>>(p, s);
-    else topk_filter_tma_kernel<false><<<g_filter, THREADS, 0, st>>>(p, s);
+    if (bf) topk_filter_tma_kernel<__nv_bfloat16, false><<<g_filter, THREADS, 0, st>>>(p, s);
+    else topk_filter_tma_kernel<float, false><<<g_filter, THREADS, 0, st>>>(p, s);
     CHECK_LAUNCH();
     if (p.cap_max <= FINISH_ONE_CTA_MAX) {
         topk_finish_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
