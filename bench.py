@@ -38,15 +38,16 @@ def resolve_workload(name: str):
     from liec_synth import WORKLOADS, flat_layout, scaled_layout, topk_counts
     base, _, div = name.partition("/")
     base, _, variant = base.partition("-")
-    if base in WORKLOADS and variant in ("", "randk"):
+    if base in WORKLOADS and variant in ("", "randk", "topk", "sign"):
         w = WORKLOADS[base]
         lay = w.layout()
         if div:   # "c4/8": same tensor list with every size divided by 8 (profiling-sized case)
             lay = scaled_layout(lay, int(div))
-        comp = w.compressor
-        if variant == "randk":   # "c3-randk": the same tensor list and k, random-k (Def. 3) both ways
-            comp = "randk"
-        k = topk_counts(lay, *w.topk_frac) if comp in ("topk", "randk") else None
+        # "c3-randk", "c4-topk", "c3-sign": the same tensor list, workers and gradients with another
+        # operator both ways (k = 1 % per tensor where the workload names no fraction)
+        comp = variant or w.compressor
+        frac = w.topk_frac if w.topk_frac[0] else (1, 100)
+        k = topk_counts(lay, *frac) if comp in ("topk", "randk") else None
         return dict(name=name, N=w.num_workers, layout=lay, dist=w.dist, scale=w.scale, comp=comp,
                     k=k, lr=w.lr, gdt=w.grad_dtype)
     if name.startswith("sweep-"):
