@@ -12,9 +12,9 @@ namespace liec {
 template <int UP, int DOWN, typename GT>
 __global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK ? 3 : 0)) worker_update_kernel(const __grid_constant__ Params p, const float lr) {
     __shared__ __align__(16) float p_tile[DOWN == COMP_TOPK ? TILE : 4];  // decoded downlink message (top-k)
-    __shared__ uint32_t own_mask[UP == COMP_RANDK ? TILE_WORDS : 1];       // the worker's own subset inside this tile
     // With a top-k downlink a CTA serves WPC workers so that the message is decoded once for them.
     constexpr int WPC = DOWN == COMP_TOPK ? 4 : 1;
+    __shared__ uint32_t own_mask[UP == COMP_RANDK ? WPC : 1][UP == COMP_RANDK ? TILE_WORDS : 1];  // each worker's own subset inside this tile
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int wq = 0; wq < WPC; ++wq) {
@@ -72,19 +72,25 @@ __global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK ? 3 : 0)) worker_u
         }
         __syncthreads();
     }
-    if (UP == COMP_RANDK) {
-        if (wq > 0) __syncthreads();  // the previous worker's mask has been read by everyone
-        own_mask[threadIdx.x] = 0u;   // THREADS == TILE_WORDS
+    if (UP == COMP_RANDK && wq == 0) {  // the subsets of all of this CTA's workers, decoded together
+#pragma unroll
+        for (int u = 0; u < WPC; ++u) own_mask[u][threadIdx.x] = 0u;   // THREADS == TILE_WORDS
         __syncthreads();
         const bool last_tile = (blockIdx.x + 1 == __ldg(p.tile_prefix + ti.t + 1));
-        const uint32_t *ob = p.up_outbase + (int64_t)worker * (p.TT + 1) + blockIdx.x;
-        const uint32_t beg = ob[0];
-        const uint32_t end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : ob[1];
         const uint32_t tile_first = (uint32_t)(ti.seg_beg + ti.rel);
-        const uint32_t *own_idx = p.up_idx + (int64_t)worker * p.K;
-        for (uint32_t q = beg + threadIdx.x; q < end; q += THREADS) {
-            const uint32_t o = own_idx[q] - tile_first;
-            if (o < (uint32_t)TILE) atomicOr(&own_mask[o >> 5], 1u << (o & 31));
+#pragma unroll
+        for (int u = 0; u < WPC; ++u) {
+            const int wu = blockIdx.y * WPC + u;
+            if (wu < p.N) {
+                const uint32_t *ob = p.up_outbase + (int64_t)wu * (p.TT + 1) + blockIdx.x;
+                const uint32_t beg = ob[0];
+                const uint32_t end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : ob[1];
+                const uint32_t *own_idx = p.up_idx + (int64_t)wu * p.K;
+                for (uint32_t q = beg + threadIdx.x; q < end; q += THREADS) {
+                    const uint32_t o = own_idx[q] - tile_first;
+                    if (o < (uint32_t)TILE) atomicOr(&own_mask[u][o >> 5], 1u << (o & 31));
+                }
+            }
         }
         __syncthreads();
     }
@@ -104,7 +110,7 @@ __global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK ? 3 : 0)) worker_u
             pd[0] = q4.x; pd[1] = q4.y; pd[2] = q4.z; pd[3] = q4.w;
         }
         uint32_t own_nib = 0u;
-        if (UP == COMP_RANDK) own_nib = own_mask[pos >> 5] >> (pos & 31);  // pos is a multiple of 4: the four bits share a word
+        if (UP == COMP_RANDK) own_nib = own_mask[wq][pos >> 5] >> (pos & 31);  // pos is a multiple of 4: the four bits share a word
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             float pi;
