@@ -135,6 +135,10 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error,
  * cudaStream_t passed as void* (NULL = legacy default stream).
  *   grads  device, [N][d] of cfg.grad_dtype, row stride d, 16-byte aligned; read-only; the
  *          same pointer and contents must be given to liec_worker_update of the same step.
+ * Inputs are expected to be finite.  NaN or infinite gradients, parameters or errors do not
+ * fault, but what they produce is unspecified: a NaN in a segment makes its scale NaN, top-k
+ * orders bit patterns (so NaNs rank above every finite magnitude), and the error entry of a kept
+ * top-k / random-k element is stored as +0 rather than computed as v - v.
  */
 liec_status liec_uplink_compress(liec_ctx *ctx, const void *grads, void *stream);   /* p^i = C(g^i) */
 liec_status liec_server_aggregate(liec_ctx *ctx, void *stream);                      /* v = e + mean_i p^i (into error) */
