@@ -12,30 +12,28 @@
 
 namespace liec {
 
-template <typename GT>
-__global__ void __launch_bounds__(THREADS, 3) average_step_kernel(const __grid_constant__ Params p, const float lr) {
-    const TileInfo ti = locate_tile(p, blockIdx.x);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // two CTAs share a tile (rows 0-3 and rows 4-7 of every warp's slice): half the accumulators
-    // per thread, twice the CTAs in flight
+// FAST: every worker's row of this tile is full and 16-byte aligned (the same for all workers, so
+// the sweeps over the workers carry no branch and their loads can be issued several workers ahead).
+template <typename GT, bool FAST>
+__device__ __forceinline__ void average_tile(const Params &p, const TileInfo &ti, const float lr, const int j0) {
     constexpr int HR = 4;
-    const int j0 = HR * blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float gs[HR][4], xs[HR][4];
 #pragma unroll
     for (int j = 0; j < HR; ++j)
 #pragma unroll
         for (int c = 0; c < 4; ++c) { gs[j][c] = 0.0f; xs[j][c] = 0.0f; }
+    const GT *g_tile0 = reinterpret_cast<const GT *>(p.G) + ti.seg_beg + ti.rel;
+    float *x_tile0 = p.X + ti.seg_beg + ti.rel;
 #pragma unroll 2
     for (int i = 0; i < p.N; ++i) {
-        const int64_t row_beg = (int64_t)i * p.d + ti.seg_beg;
-        const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
-        const GT *g_tile = reinterpret_cast<const GT *>(p.G) + row_beg + ti.rel;
-        const float *x_tile = p.X + row_beg + ti.rel;
+        const GT *g_tile = g_tile0 + (int64_t)i * p.d;
+        const float *x_tile = x_tile0 + (int64_t)i * p.d;
 #pragma unroll
         for (int j = 0; j < HR; ++j) {
             const int pos = tile_pos(warp, lane, j0 + j);
             float g[4], x[4];
-            if (fast) { load4_cached(g_tile + pos, g); load4_stream(x_tile + pos, x); }
+            if (FAST) { load4_cached(g_tile + pos, g); load4_stream(x_tile + pos, x); }
             else { load4_guarded(g_tile, pos, ti.len, g); load4_guarded(x_tile, pos, ti.len, x); }
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -45,13 +43,12 @@ __global__ void __launch_bounds__(THREADS, 3) average_step_kernel(const __grid_c
         }
     }
     const WorkerDivisor by_n(p.N);
-    const bool efast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
     float *e_tile = p.e + ti.seg_beg + ti.rel;
 #pragma unroll
     for (int j = 0; j < HR; ++j) {
         const int pos = tile_pos(warp, lane, j0 + j);
         float ev[4];
-        if (efast) load4_stream(e_tile + pos, ev);
+        if (FAST) load4_stream(e_tile + pos, ev);
         else load4_guarded(e_tile, pos, ti.len, ev);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -59,7 +56,7 @@ __global__ void __launch_bounds__(THREADS, 3) average_step_kernel(const __grid_c
             xs[j][c] = by_n(xs[j][c]);                    // xbar
         }
         // e' = v - p with p = v
-        if (efast) {
+        if (FAST) {
             *reinterpret_cast<float4 *>(e_tile + pos) = make_float4(__fsub_rn(gs[j][0], gs[j][0]), __fsub_rn(gs[j][1], gs[j][1]),
                                                                     __fsub_rn(gs[j][2], gs[j][2]), __fsub_rn(gs[j][3], gs[j][3]));
         } else {
@@ -68,17 +65,15 @@ __global__ void __launch_bounds__(THREADS, 3) average_step_kernel(const __grid_c
                 if (pos + c < ti.len) e_tile[pos + c] = __fsub_rn(gs[j][c], gs[j][c]);
         }
     }
-#pragma unroll 2
+#pragma unroll 4
     for (int i = 0; i < p.N; ++i) {
-        const int64_t row_beg = (int64_t)i * p.d + ti.seg_beg;
-        const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
-        const GT *g_tile = reinterpret_cast<const GT *>(p.G) + row_beg + ti.rel;
-        float *x_tile = p.X + row_beg + ti.rel;
+        const GT *g_tile = g_tile0 + (int64_t)i * p.d;
+        float *x_tile = x_tile0 + (int64_t)i * p.d;
 #pragma unroll
         for (int j = 0; j < HR; ++j) {
             const int pos = tile_pos(warp, lane, j0 + j);
             float g[4], x[4];
-            if (fast) load4_cached(g_tile + pos, g);
+            if (FAST) load4_cached(g_tile + pos, g);
             else load4_guarded(g_tile, pos, ti.len, g);
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -86,7 +81,7 @@ __global__ void __launch_bounds__(THREADS, 3) average_step_kernel(const __grid_c
                 const float u = __fadd_rn(diff, g[c]);
                 x[c] = __fsub_rn(xs[j][c], __fmul_rn(lr, u));
             }
-            if (fast) {
+            if (FAST) {
                 __stcs(reinterpret_cast<float4 *>(x_tile + pos), make_float4(x[0], x[1], x[2], x[3]));
             } else {
 #pragma unroll
@@ -95,6 +90,17 @@ __global__ void __launch_bounds__(THREADS, 3) average_step_kernel(const __grid_c
             }
         }
     }
+}
+
+template <typename GT>
+__global__ void __launch_bounds__(THREADS, 3) average_step_kernel(const __grid_constant__ Params p, const float lr) {
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    // two CTAs share a tile (rows 0-3 and rows 4-7 of every warp's slice): half the accumulators
+    // per thread, twice the CTAs in flight
+    const int j0 = 4 * blockIdx.y;
+    const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0) && ((p.d & 3) == 0);
+    if (fast) average_tile<GT, true>(p, ti, lr, j0);
+    else average_tile<GT, false>(p, ti, lr, j0);
 }
 
 // xbar = (1/N) sum_i x^i (the ENSURE line of Algorithm 1), one CTA per tile.
