@@ -93,7 +93,7 @@ __device__ __forceinline__ void average_tile(const Params &p, const TileInfo &ti
 }
 
 template <typename GT>
-__global__ void __launch_bounds__(THREADS, 3) average_step_kernel(const __grid_constant__ Params p, const float lr) {
+__global__ void __launch_bounds__(THREADS, (sizeof(GT) == 4 ? 2 : 3)) average_step_kernel(const __grid_constant__ Params p, const float lr) {
     const TileInfo ti = locate_tile(p, blockIdx.x);
     // two CTAs share a tile (rows 0-3 and rows 4-7 of every warp's slice): half the accumulators
     // per thread, twice the CTAs in flight
@@ -104,28 +104,44 @@ __global__ void __launch_bounds__(THREADS, 3) average_step_kernel(const __grid_c
 }
 
 // xbar = (1/N) sum_i x^i (the ENSURE line of Algorithm 1), one CTA per tile.
-__global__ void __launch_bounds__(THREADS) mean_params_kernel(const __grid_constant__ Params p, float *out) {
-    const TileInfo ti = locate_tile(p, blockIdx.x);
+template <bool FAST>
+__device__ __forceinline__ void mean_tile(const Params &p, const TileInfo &ti, float *out) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const WorkerDivisor by_n(p.N);
+    const float *x_tile0 = p.X + ti.seg_beg + ti.rel;
+    float acc[8][4];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) acc[j][c] = 0.0f;
+#pragma unroll 2
+    for (int i = 0; i < p.N; ++i) {   // worker order; the 8 rows of a worker are fetched together
+        const float *x_tile = x_tile0 + (int64_t)i * p.d;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int pos = tile_pos(warp, lane, j);
+            float x[4];
+            if (FAST) load4_stream(x_tile + pos, x);
+            else load4_guarded(x_tile, pos, ti.len, x);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[j][c] = __fadd_rn(acc[j][c], x[c]);
+        }
+    }
+    float *o = out + ti.seg_beg + ti.rel;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int pos = tile_pos(warp, lane, j);
-        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        for (int i = 0; i < p.N; ++i) {
-            const int64_t row_beg = (int64_t)i * p.d + ti.seg_beg;
-            const float *x_tile = p.X + row_beg + ti.rel;
-            float x[4];
-            if ((ti.len == TILE) && ((row_beg & 3) == 0)) load4_stream(x_tile + pos, x);
-            else load4_guarded(x_tile, pos, ti.len, x);
-#pragma unroll
-            for (int c = 0; c < 4; ++c) acc[c] = __fadd_rn(acc[c], x[c]);
-        }
-        float *o = out + ti.seg_beg + ti.rel;
 #pragma unroll
         for (int c = 0; c < 4; ++c)
-            if (pos + c < ti.len) o[pos + c] = by_n(acc[c]);
+            if (pos + c < ti.len) o[pos + c] = by_n(acc[j][c]);
     }
+}
+
+__global__ void __launch_bounds__(THREADS) mean_params_kernel(const __grid_constant__ Params p, float *out) {
+    const TileInfo ti = locate_tile(p, blockIdx.x);
+    // full tile and every worker's row 16-byte aligned: the sweep over the workers carries no branch
+    if ((ti.len == TILE) && ((ti.seg_beg & 3) == 0) && ((p.d & 3) == 0)) mean_tile<true>(p, ti, out);
+    else mean_tile<false>(p, ti, out);
 }
 
 cudaError_t launch_average_step(const Params &p, float lr, cudaStream_t st) {
