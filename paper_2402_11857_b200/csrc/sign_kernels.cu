@@ -259,10 +259,12 @@ __global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_cons
         for (int c = 0; c < 4; ++c) acc[j][c] = 0.0f;
 
     {  // identity uplink: the message is the gradient itself
+        // (one answer for all workers, so that the loop carries no branch and its loads pipeline)
+        const bool gfast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0) && ((p.d & 3) == 0);
+#pragma unroll 2
         for (int i = 0; i < p.N; ++i) {
             const int64_t row_beg = (int64_t)i * p.d + ti.seg_beg;
             const GT *tile_ptr = reinterpret_cast<const GT *>(p.G) + row_beg + ti.rel;
-            const bool gfast = (ti.len == TILE) && ((row_beg & 3) == 0);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 float g[4];
