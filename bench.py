@@ -86,10 +86,13 @@ def update_kernel_bytes(w) -> float:
     return N * d * (g + 8) + down + own
 
 
-# DRAM bytes per element-worker of the worker update, from an ncu capture of that kernel on the
-# c4/8 workload (dram__bytes_read + dram__bytes_write = 4.925 GB for 497.8 M element-workers; the
-# traffic of this streaming kernel grows in proportion to N*d).  Other variants: not captured.
-UPDATE_TRAFFIC_PER_UNIT = {("sign", "bf16"): 4.924888e9 / 497759232}
+# DRAM bytes (dram__bytes_read + dram__bytes_write, ncu) of one worker-update launch, per named
+# workload.  c4: captured on c4/8 (4.925 GB for 497.8 M element-workers) and scaled by N*d, because
+# this streaming kernel's traffic grows in proportion; c3 and c2: captured at full size (the tail
+# of the parameter writes is still in the L2 when the kernel ends, hence slightly fewer bytes than
+# the algorithmic count).  Any other workload or variant: not captured.
+UPDATE_TRAFFIC_BYTES = {"c4": 4.924888e9 / 497759232 * 32 * 124439808, "c3": 3274704384 + 1587624448,
+                        "c2": 749634816 + 323100160}
 
 
 # ------------------------------------------------------------------------------------ clocks
@@ -435,8 +438,7 @@ def main():
         "stage_ms": r["stage_ms"],
         "roofline": {"bound": "hbm", "kernel": "worker_update_kernel", "achieved": upd_gbs, "peak": peak,
                      "unit": "GB/s", "frac": upd_gbs / peak,
-                     "traffic": (UPDATE_TRAFFIC_PER_UNIT[(w["comp"], w["gdt"])] * N * d
-                                 if (w["comp"], w["gdt"]) in UPDATE_TRAFFIC_PER_UNIT else None), "peak_source": peak_src,
+                     "traffic": UPDATE_TRAFFIC_BYTES.get(w["name"]), "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": update_kernel_bytes(w), "launch_ms": upd_ms},
         "gpu_launches": r["launches"], "clocks": r["clocks"],
         "average_step": {"ms": r["average_ms"],
