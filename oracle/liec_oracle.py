@@ -94,11 +94,11 @@ def num_words(off) -> int:
     return int(((np.diff(off) + 31) // 32).sum())
 
 
-def widen_bf16(bits_u16: np.ndarray) -> np.ndarray:
+def widen_bf16(bits_u16: np.ndarray, _lib=None) -> np.ndarray:
     """bf16 bit patterns (uint16) -> float32, exactly."""
     a = np.ascontiguousarray(bits_u16, dtype=np.uint16)
     out = np.empty(a.shape, dtype=np.float32)
-    lib().liec_oracle_widen_bf16(_ptr(a), _ptr(out), a.size)
+    (_lib or lib()).liec_oracle_widen_bf16(_ptr(a), _ptr(out), a.size)
     return out
 
 

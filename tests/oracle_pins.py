@@ -556,10 +556,30 @@ def pin_sumsq_and_delta(L):
 
 
 def pin_bf16_widening(L):
-    bits = np.asarray([0x3F80, 0xBF80, 0x0000, 0x8000, 0x3DCD, 0x7F7F, 0x0001], np.uint16)
-    out = oracle.widen_bf16(bits)
-    assert out.view(np.uint32).tolist() == [int(b) << 16 for b in bits]
-    assert out[0] == 1.0 and out[1] == -1.0
+    """bfloat16 -> binary32 against values worked out by hand from the format (1 sign bit, 8 exponent
+    bits with bias 127, 7 fraction bits): 0x3DCD = 2^-4 (1 + 77/128), 0x4049 = 2 (1 + 73/128),
+    0xC2F7 = -64 (1 + 119/128), 0x7F7F = 2^127 (2 - 2^-7), 0x0001 = 2^-126 2^-7 (subnormal)."""
+    bits = np.asarray([0x3F80, 0xBF80, 0x0000, 0x8000, 0x3DCD, 0x4049, 0xC2F7, 0x7F7F, 0x0001], np.uint16)
+    out = oracle.widen_bf16(bits, _lib=L)
+    want = [1.0, -1.0, 0.0, -0.0, 0.10009765625, 3.140625, -123.5, (2.0 - 2.0 ** -7) * 2.0 ** 127, 2.0 ** -133]
+    assert [float(v) for v in out] == want
+    assert math.copysign(1.0, float(out[3])) == -1.0 and math.copysign(1.0, float(out[2])) == 1.0
+
+
+def pin_sumsq_tree_shape(L):
+    """The squared norm follows the same balanced tree as the L1 norm (the order is part of what the
+    CUDA path has to reproduce bit for bit).  Expected values by hand from round-to-nearest-even:
+    (2^27)^2 = 2^54 has a unit in the last place of 4, so 2^54 + 1 rounds back, 2^54 + 2 is a tie
+    that goes to the even neighbour (2^54; but 2^54 + 6 goes up to 2^54 + 8), sums of small squares are exact."""
+    b = float(2 ** 27)
+    big = float(2 ** 54)
+    t = lambda v: oracle.tree_sumsq(np.asarray(v, np.float32), _lib=L)
+    assert t([b, 1, 1, 1, 1, 1, 1, 1]) == big + 4     # ((big+1)+(1+1)) + ((1+1)+(1+1)) = big + 4; a running sum stays at big
+    assert t([b, 2, 1, 1]) == big + 8                 # (big+4) + (1+1) = big + 6 -> tie to even; a running sum gives big + 4
+    assert t([1, 1, b, 2]) == big + 8                 # (1+1) + (big+4)
+    assert t([b, 1, 1]) == big                        # padded to 4: (big+1) + (1+0) = big + 1 -> big
+    assert t([1, 1, 1, 1, b, 1, 1, 1, 1]) == big + 4  # padded to 16: (4 + ((big+1)+(1+1))) + (1+0+...) = (big+4) + 1 -> big + 4
+    assert t([-3, 4]) == 25.0
 
 
 ALL_PINS = [
@@ -567,6 +587,6 @@ ALL_PINS = [
     pin_scale_is_exact_mean, pin_tree_shape, pin_sign_bits_bruteforce, pin_sign_contraction,
     pin_blockwise_reduces_to_sign, pin_topk_bruteforce, pin_topk_quantile,
     pin_error_recursion, pin_identity_one_worker_is_sgd, pin_identical_workers,
-    pin_lemma3_exact, pin_lemma3_float, pin_bf16_widening, pin_golden_averaging, pin_averaging_properties, pin_sumsq_and_delta,
+    pin_lemma3_exact, pin_lemma3_float, pin_bf16_widening, pin_sumsq_tree_shape, pin_golden_averaging, pin_averaging_properties, pin_sumsq_and_delta,
     pin_randk_all_subsets, pin_randk_segments_and_rejects, pin_randk_step_special_cases,
 ]

@@ -40,6 +40,10 @@ MUTANTS = {
     "averaging_forgets_error": ("v[j] = e[j] + gmean;", "v[j] = gmean;"),
     "averaging_keeps_error": ("e[j] = v[j] - v[j];", "e[j] = e[j];"),
     "mean_model_not_divided": ("xbar[j] = acc / (float)N;", "xbar[j] = acc;"),
+    "sumsq_running_sum": ("double left = tree_sq_node(x, n, lo, len / 2);\n    double right = tree_sq_node(x, n, lo + len / 2, len / 2);\n    return left + right;",
+                          "double s = 0.0; for (int64_t q = lo; q < lo + len && q < n; ++q) s += (double)x[q] * (double)x[q];\n    return s;"),
+    "sumsq_summed_in_binary32": ("double left = tree_sq_node", "float left = tree_sq_node"),
+    "bf16_widened_into_low_half": ("uint32_t u = (uint32_t)in[j] << 16;", "uint32_t u = (uint32_t)in[j];"),
     "sumsq_not_squared": ("return a * a;                  /* exact: 24-bit significands */", "return a < 0 ? -a : a;"),
     "randk_value_from_slot_not_index": ("val[q] = x[j];", "val[q] = x[q];"),
     "randk_segment_check_dropped": ("if (j < off[t] || j >= off[t + 1]) return -3;", ""),
