@@ -58,7 +58,7 @@ typedef struct liec_ctx liec_ctx; /* opaque, lives in host memory */
 typedef enum {
     LIEC_OK = 0,
     LIEC_ERR_INVALID_ARG = 1,  /* NULL / misaligned pointer, bad sizes, bad segment table, bad k */
-    LIEC_ERR_UNSUPPORTED = 2,  /* d >= 2^32, too many workers or segments for the launch grid */
+    LIEC_ERR_UNSUPPORTED = 2,  /* d >= 2^32, more than 65535 workers or segments (launch grid) */
     LIEC_ERR_WORKSPACE = 3,    /* workspace smaller than liec_workspace_bytes() */
     LIEC_ERR_STATE = 4,        /* staged calls made out of order */
     LIEC_ERR_CUDA = 5,         /* a CUDA runtime call failed; see liec_last_error() */
@@ -165,8 +165,22 @@ liec_status liec_worker_update(liec_ctx *ctx, const void *grads, float lr, void 
  */
 liec_status liec_set_subsets(liec_ctx *ctx, const uint32_t *up_sets, const uint32_t *down_set);
 
-/* The four stages in sequence; produces the same bytes as calling them one by one. */
+/*
+ * The four stages in sequence (one iteration of Algorithm 1's compressed branch); produces the same
+ * bytes as calling them one by one.  If a stage fails after an earlier one was enqueued, the context
+ * returns to idle (the next iteration may start) and params / error are unspecified, as after
+ * liec_abort_step.
+ */
 liec_status liec_step(liec_ctx *ctx, const void *grads, float lr, void *stream);
+
+/*
+ * Gives up the iteration in progress (Algorithm 1 has no such step: this is error recovery for the
+ * staged calls).  After a stage has failed, or when the caller decides not to finish an iteration,
+ * this returns the context to idle so that liec_uplink_compress / liec_step are accepted again.
+ * Enqueues nothing.  The stages already enqueued still run; params and error are then somewhere
+ * between two iterations (error may hold v_t): restore them from a copy before going on.
+ */
+liec_status liec_abort_step(liec_ctx *ctx);
 
 /*
  * The model-averaging iteration of Algorithm 1 (its branch for (t+1) mod floor(1/delta) == 0; the
@@ -205,9 +219,10 @@ liec_status liec_sumsq(liec_ctx *ctx, int32_t which, const void *grads, double *
 /*
  * One iteration fed from host memory: copies grads_host ([N][d] of cfg.grad_dtype, pinned
  * memory recommended) into grads_dev (device staging buffer of the same size, caller
- * owned), runs liec_step, copies the downlink message (sign: words then scales; top-k:
- * idx then val; liec_down_message_bytes() bytes) to down_msg_host, all on `stream`.
- * down_msg_host may be NULL to skip the read-back.  Does not synchronise.
+ * owned, 16-byte aligned), runs liec_step, copies the downlink message (sign: words then scales;
+ * top-k: idx then val; liec_down_message_bytes() bytes) to down_msg_host, all on `stream`.
+ * down_msg_host may be NULL to skip the read-back.  Does not synchronise.  LIEC_ERR_STATE, with
+ * nothing enqueued, when called between the stages of an iteration.
  */
 liec_status liec_step_host(liec_ctx *ctx, const void *grads_host, void *grads_dev, float lr,
                            void *down_msg_host, void *stream);
@@ -230,6 +245,31 @@ liec_status liec_device_status(liec_ctx *ctx, void *stream, int32_t *out);
  * The state (params, error) after a flagged iteration is unspecified; restore it before going on.
  */
 liec_status liec_clear_status(liec_ctx *ctx, void *stream);
+
+/*
+ * Diagnostics for the bounded waits (no counterpart in the paper).  Kernels that stage a tile in
+ * shared memory with a bulk copy poll the copy's barrier at most `poll_limit` times (0 = the default,
+ * 2^20) before they set bit 8 of the status word and return without touching their outputs.
+ * `expect_extra_bytes` (a multiple of 16, at most 1024; 0 in operation) is added to the byte count
+ * that each copy's barrier is told to expect: the copy still lands, but its barrier never completes,
+ * so every such wait runs out.  That is how a test drives the timeout path without any fault; a
+ * flagged kernel waits a further millisecond before it returns, so that nothing is in flight into
+ * its shared memory.  Takes effect from the next stage call.
+ */
+liec_status liec_set_copy_wait(liec_ctx *ctx, uint32_t poll_limit, uint32_t expect_extra_bytes);
+
+/*
+ * Diagnostics: which route the top-k selections (Def. 2) of the last iteration took on one side
+ * (uplink != 0: the N*T worker problems; 0: the T server problems).  Synchronises `stream`, copies
+ * the selection state to the host and counts:
+ *   out[0] problems, out[1] uplink problems that finished on the single dense pass seeded by the
+ *   previous threshold, out[2] problems that needed the dense second-digit pass (more entries
+ *   share the threshold's leading key bits than the candidate buffer holds), out[3] problems that
+ *   fell back to the one-CTA dense path (huge groups of equal magnitudes).
+ * The result of the selection never depends on the route.  LIEC_ERR_INVALID_ARG when the side does
+ * not use top-k.
+ */
+liec_status liec_topk_route_counts(liec_ctx *ctx, void *stream, int32_t uplink, int64_t *out /* [4] */);
 
 /* Number of kernel launches enqueued by this context so far (host-side counter). */
 int64_t liec_launch_count(const liec_ctx *ctx);

@@ -177,6 +177,59 @@ __device__ __forceinline__ double cta_tree_reduce(double warp_sum, double *smem8
     return s;
 }
 
+// Combines per-tile partial sums (binary64) of one segment in tree order: pairwise, level by level,
+// over the tile count zero-padded to a power of two (adding +0 is exact), which continues the
+// segment's balanced tree above the tile level.  Segments of more than FIN_CHUNK tiles are reduced
+// chunk by chunk (a chunk of FIN_CHUNK tiles is an aligned subtree) and the chunk sums are combined
+// by the same rule.  Whole CTA (THREADS threads); the result is valid in thread 0.
+constexpr int FIN_CHUNK = 2048;
+constexpr int FIN_MAX_CHUNKS = 256;  // 2^32 elements / TILE / FIN_CHUNK
+
+__device__ __forceinline__ double tree_reduce_partials(const double *src, int ntiles, double *buf /*[FIN_CHUNK]*/,
+                                                       double *chunk_sums /*[FIN_MAX_CHUNKS]*/) {
+    const int nchunks = (ntiles + FIN_CHUNK - 1) / FIN_CHUNK;
+    for (int c = 0; c < nchunks; ++c) {
+        // the chunk's tree over the next power of two of its tile count: the levels above it would
+        // only add +0, which changes nothing
+        const int here = min(FIN_CHUNK, ntiles - c * FIN_CHUNK);
+        int span = 1;
+        while (span < here) span <<= 1;
+        for (int q = threadIdx.x; q < span; q += THREADS) {
+            const int idx = c * FIN_CHUNK + q;
+            buf[q] = idx < ntiles ? src[idx] : 0.0;
+        }
+        __syncthreads();
+        for (int width = span / 2; width >= 1; width >>= 1) {
+            // pairwise: new[q] = old[2q] + old[2q+1]; done in two phases to avoid overwrite hazards
+            double vals[FIN_CHUNK / 2 / THREADS];
+#pragma unroll
+            for (int r = 0; r < FIN_CHUNK / 2 / THREADS; ++r) {
+                const int q = threadIdx.x + r * THREADS;
+                vals[r] = q < width ? __dadd_rn(buf[2 * q], buf[2 * q + 1]) : 0.0;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int r = 0; r < FIN_CHUNK / 2 / THREADS; ++r) {
+                const int q = threadIdx.x + r * THREADS;
+                if (q < width) buf[q] = vals[r];
+            }
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) chunk_sums[c] = buf[0];
+        __syncthreads();
+    }
+    double total = 0.0;
+    if (threadIdx.x == 0) {
+        int L = 1;
+        while (L < nchunks) L <<= 1;
+        for (int c = nchunks; c < L; ++c) chunk_sums[c] = 0.0;
+        for (int width = L / 2; width >= 1; width >>= 1)
+            for (int q = 0; q < width; ++q) chunk_sums[q] = __dadd_rn(chunk_sums[2 * q], chunk_sums[2 * q + 1]);
+        total = chunk_sums[0];
+    }
+    return total;
+}
+
 // ---- sign words -------------------------------------------------------------------------------
 
 __device__ __forceinline__ uint32_t sign_nibble(const float (&v)[4]) {
@@ -193,10 +246,76 @@ __device__ __forceinline__ uint32_t pack_word(uint32_t nibble, int lane) {
     return w;
 }
 
+// Scaled sign of one tile held in global memory (4-wide layout): writes the tile's sign words and
+// returns, in thread 0, the binary64 tree sum of its magnitudes.  `fast`: the tile is full and its
+// first element 16-byte aligned.  Whole CTA.
+template <typename GT>
+__device__ __forceinline__ double sign_tile(const GT *tile_ptr, int len, bool fast, uint32_t *tile_words,
+                                            double *warp_sums /*[8]*/) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float v[8][4];
+    if (fast) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) load4_stream(tile_ptr + tile_pos(warp, lane, j), v[j]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), len, v[j]);
+    }
+    const int nwords = (len + 31) >> 5;
+    double a[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        a[j] = leaf4(v[j]);
+        const uint32_t w = pack_word(sign_nibble(v[j]), lane);
+        const int widx = warp * 32 + j * 4 + (lane >> 3);
+        if ((lane & 7) == 0 && widx < nwords) tile_words[widx] = w;
+    }
+    return cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
+}
+
 // Nibble of this lane's 4 elements in row j, taken from the warp's 32 words (lane l holds word l).
 __device__ __forceinline__ uint32_t nibble_from_words(uint32_t my_word, int lane, int j) {
     uint32_t w = __shfl_sync(0xffffffffu, my_word, 4 * j + (lane >> 3));
     return (w >> (4 * (lane & 7))) & 0xfu;
+}
+
+// ---- bulk copies into shared memory (TMA, untiled) and their bounded waits -----------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void *ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
+
+// One thread: announce `expect` bytes on the mbarrier and start a bulk copy of `bytes` bytes
+// (both addresses 16-byte aligned, bytes a multiple of 16).  expect == bytes in normal operation.
+__device__ __forceinline__ void bulk_copy_g2s(void *dst_smem, const void *src, uint32_t bytes, uint32_t expect,
+                                              unsigned long long *bar) {
+    const uint32_t b = smem_u32(bar);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // earlier generic accesses of the buffer come first
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(expect) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst_smem)), "l"(src), "r"(bytes), "r"(b) : "memory");
+}
+
+// Polls the mbarrier's phase `parity` at most `limit` times; true when the phase completed.
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long *bar, uint32_t parity, uint32_t limit) {
+    uint32_t done = 0;
+    const uint32_t b = smem_u32(bar);
+    for (uint32_t spin = 0; spin < limit && !done; ++spin)
+        asm volatile("{ .reg .pred q; mbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2; selp.u32 %0, 1, 0, q; }"
+                     : "=r"(done) : "r"(b), "r"(parity) : "memory");
+    return done != 0;
+}
+
+// After a wait that ran out: before the CTA gives its shared memory back, give a copy that may
+// still be in flight time to land.  Polls until the phase completes, but for at least a
+// millisecond (a healthy copy of a tile takes microseconds) and at most 2^22 polls.
+__device__ __forceinline__ bool mbar_drain(unsigned long long *bar, uint32_t parity) {
+    unsigned long long t0, t1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    for (uint32_t round = 0; round < (1u << 12); ++round) {
+        if (mbar_wait_bounded(bar, parity, 1u << 10)) return true;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+        if (t1 - t0 > 1000000ull) break;
+    }
+    return false;
 }
 
 }  // namespace liec

@@ -10,7 +10,6 @@ namespace liec {
 cudaError_t launch_sign_uplink(const Params &p, cudaStream_t st);
 cudaError_t launch_scale_finalize(const Params &p, bool uplink, cudaStream_t st);
 cudaError_t launch_server_dense(const Params &p, cudaStream_t st);
-cudaError_t launch_sign_downlink(const Params &p, cudaStream_t st);
 cudaError_t launch_sign_error(const Params &p, cudaStream_t st);
 cudaError_t launch_identity_downlink(const Params &p, cudaStream_t st);
 

@@ -280,6 +280,8 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     memset(&p, 0, sizeof(p));
     p.N = pl.N; p.T = pl.T; p.TT = pl.TT; p.d = pl.d; p.W = pl.W; p.K = pl.K; p.CAP = pl.CAP; p.cap_max = pl.cap_max;
     p.up = cfg->uplink; p.down = cfg->downlink; p.gdt = cfg->grad_dtype;
+    p.copy_wait_limit = COPY_WAIT_LIMIT_DEFAULT;
+    p.copy_expect_extra = 0u;
     p.seg_off = at<int64_t>(c, pl.r_seg_off);
     p.word_off = at<int64_t>(c, pl.r_word_off);
     p.k_off = at<int64_t>(c, pl.r_k_off);
@@ -432,10 +434,26 @@ liec_status liec_set_subsets(liec_ctx *c, const uint32_t *up_sets, const uint32_
 
 liec_status liec_step(liec_ctx *c, const void *grads, float lr, void *stream) {
     liec_status st = liec_uplink_compress(c, grads, stream);
-    if (st != LIEC_OK) return st;
-    if ((st = liec_server_aggregate(c, stream)) != LIEC_OK) return st;
-    if ((st = liec_downlink_compress(c, stream)) != LIEC_OK) return st;
-    return liec_worker_update(c, grads, lr, stream);
+    if (st != LIEC_OK) return st;  // nothing was enqueued: the context is where it was
+    if ((st = liec_server_aggregate(c, stream)) == LIEC_OK && (st = liec_downlink_compress(c, stream)) == LIEC_OK)
+        st = liec_worker_update(c, grads, lr, stream);
+    if (st != LIEC_OK) c->stage = 0;  // a half-done iteration: back to idle, state unspecified (see liec_abort_step)
+    return st;
+}
+
+liec_status liec_abort_step(liec_ctx *c) {
+    if (!c) return LIEC_ERR_INVALID_ARG;
+    c->stage = 0;
+    return LIEC_OK;
+}
+
+liec_status liec_set_copy_wait(liec_ctx *c, uint32_t poll_limit, uint32_t expect_extra_bytes) {
+    if (!c) return LIEC_ERR_INVALID_ARG;
+    if (expect_extra_bytes & 15u) { c->err = "expect_extra_bytes must be a multiple of 16"; return LIEC_ERR_INVALID_ARG; }
+    if (expect_extra_bytes > 1024u) { c->err = "expect_extra_bytes must be at most 1024"; return LIEC_ERR_INVALID_ARG; }
+    c->p.copy_wait_limit = poll_limit ? poll_limit : COPY_WAIT_LIMIT_DEFAULT;
+    c->p.copy_expect_extra = expect_extra_bytes;
+    return LIEC_OK;
 }
 
 liec_status liec_average_step(liec_ctx *c, const void *grads, float lr, void *stream) {
@@ -472,6 +490,11 @@ liec_status liec_step_host(liec_ctx *c, const void *grads_host, void *grads_dev,
                            void *stream) {
     if (!c) return LIEC_ERR_INVALID_ARG;
     if (!grads_host || !grads_dev) { c->err = "grads_host and grads_dev must be non-NULL"; return LIEC_ERR_INVALID_ARG; }
+    // before anything is enqueued: a copy into grads_dev in the middle of an iteration would overwrite
+    // the gradients that the pending worker update still has to read
+    liec_status st0 = check_stage(c, 0, "liec_step_host");
+    if (st0 != LIEC_OK) return st0;
+    if (!aligned16(grads_dev)) { c->err = "grads_dev must be 16-byte aligned"; return LIEC_ERR_INVALID_ARG; }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t esz = c->p.gdt == DT_BF16 ? 2 : 4;
     const size_t row_bytes = esz * (size_t)c->p.d;
@@ -520,6 +543,28 @@ liec_status liec_device_status(liec_ctx *c, void *stream, int32_t *out) {
     e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(c, e, "cudaStreamSynchronize");
     if (*out != 0) { c->err = "a kernel recorded a failed internal check"; return LIEC_ERR_DEVICE_CHECK; }
+    return LIEC_OK;
+}
+
+liec_status liec_topk_route_counts(liec_ctx *c, void *stream, int32_t uplink, int64_t *out) {
+    if (!c || !out) return LIEC_ERR_INVALID_ARG;
+    const uint32_t *sel = uplink ? c->p.up_sel : c->p.down_sel;
+    const int64_t problems = (int64_t)(uplink ? c->p.N : 1) * c->p.T;
+    out[0] = out[1] = out[2] = out[3] = 0;
+    if (!sel) { c->err = "this side does not use top-k"; return LIEC_ERR_INVALID_ARG; }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::vector<uint32_t> host((size_t)problems * SEL_WORDS);
+    cudaError_t e = cudaMemcpyAsync(host.data(), sel, host.size() * sizeof(uint32_t), cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpyAsync(selection state)");
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaStreamSynchronize");
+    out[0] = problems;
+    for (int64_t q = 0; q < problems; ++q) {
+        const uint32_t *w = host.data() + q * SEL_WORDS;
+        if (uplink && w[SEL_MODE] == 1u) ++out[1];
+        if (w[SEL_FLAGS] & 2u) ++out[2];
+        if (w[SEL_FLAGS] & 1u) ++out[3];
+    }
     return LIEC_OK;
 }
 

@@ -66,7 +66,13 @@ struct Params {
 
     float *vbuf;      // [d] identity downlink copy of v
     int32_t *status;  // device status word
+
+    // bounded waits on bulk copies into shared memory: polls before a copy is declared lost, and
+    // bytes added to what its barrier is told to expect (0 in operation; a diagnostic setting
+    // makes the barrier never complete although the copy lands, which exercises the timeout path)
+    uint32_t copy_wait_limit, copy_expect_extra;
 };
+constexpr uint32_t COPY_WAIT_LIMIT_DEFAULT = 1u << 20;
 
 // per-problem selection state words
 constexpr int SEL_WORDS = 16;
@@ -85,6 +91,8 @@ constexpr int SEL_LO2 = 11;       // same for the second-digit histogram
 constexpr int SEL_HI2 = 12;
 constexpr int SEL_GUESS = 13;      // uplink: lower bound (31-bit key) tried first in the next step; 0 = none
 constexpr int SEL_MODE = 14;       // uplink, this step: 1 = candidates collected with the guess, 0 = regular two-pass path
+constexpr int SEL_SPEC_FAIL = 15;  // uplink, this step: the guess let too many candidates through (written by the
+                                   // filter, read only by later kernels, which then send the problem down the regular path)
 
 // words of the status block (int32 each)
 constexpr int STATUS_WORD = 0;        // failed internal checks

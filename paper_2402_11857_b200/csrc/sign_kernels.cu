@@ -18,31 +18,11 @@ __global__ void __launch_bounds__(THREADS) sign_uplink_kernel(const __grid_const
     __shared__ double warp_sums[8];
     const int worker = blockIdx.y;
     const TileInfo ti = locate_tile(p, blockIdx.x);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t row_beg = (int64_t)worker * p.d + ti.seg_beg;  // segment start in the [N][d] array
     const GT *tile_ptr = reinterpret_cast<const GT *>(p.G) + row_beg + ti.rel;
     const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
-
-    float v[8][4];
-    if (fast) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) load4_stream(tile_ptr + tile_pos(warp, lane, j), v[j]);
-    } else {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v[j]);
-    }
-
     uint32_t *words = p.up_words + (int64_t)worker * p.W + __ldg(p.word_off + ti.t) + ti.rel / 32;
-    const int nwords = (ti.len + 31) >> 5;
-    double a[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        a[j] = leaf4(v[j]);
-        uint32_t w = pack_word(sign_nibble(v[j]), lane);
-        int widx = warp * 32 + j * 4 + (lane >> 3);
-        if ((lane & 7) == 0 && widx < nwords) words[widx] = w;
-    }
-    double s = cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
+    const double s = sign_tile(tile_ptr, ti.len, fast, words, warp_sums);
     if (threadIdx.x == 0) p.up_partials[(int64_t)worker * p.TT + blockIdx.x] = s;
 }
 
@@ -56,8 +36,6 @@ __global__ void __launch_bounds__(THREADS) sign_uplink_kernel(const __grid_const
 // permutes the leaves of the chunk-level tree only inside its own pairs, so the sum is unchanged.
 // One thread polls the mbarrier with a bounded wait; the others sleep at the CTA barrier.
 constexpr int UPLINK_TPC = 4;
-
-__device__ __forceinline__ uint32_t smem_addr_of(const void *ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
 
 __global__ void __launch_bounds__(THREADS) sign_uplink_bf16_kernel(const __grid_constant__ Params p) {
     __shared__ __align__(128) unsigned short tile_s[2][TILE];
@@ -82,8 +60,8 @@ __global__ void __launch_bounds__(THREADS) sign_uplink_bf16_kernel(const __grid_
         t_fast[threadIdx.x] = (tn.len == TILE && row_aligned && (tn.seg_beg & 7) == 0) ? 1 : 0;  // a 16-byte aligned full tile
     }
     if (threadIdx.x == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr_of(&bar[0])));
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr_of(&bar[1])));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bar[0])));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bar[1])));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         copy_ok = 1;
     }
@@ -95,18 +73,11 @@ __global__ void __launch_bounds__(THREADS) sign_uplink_bf16_kernel(const __grid_
         if (t_fast[i]) {
             pending |= 1u << (i & 1);
             const uint32_t bytes = TILE * sizeof(unsigned short);
-            const uint32_t b = smem_addr_of(&bar[i & 1]);
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // earlier generic accesses of the buffer come first
-            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(bytes) : "memory");
-            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         ::"r"(smem_addr_of(tile_s[i & 1])), "l"(row + t_src[i]), "r"(bytes), "r"(b) : "memory");
+            bulk_copy_g2s(tile_s[i & 1], row + t_src[i], bytes, bytes + p.copy_expect_extra, &bar[i & 1]);
         }
     };
-    auto wait_for = [&](int buf) -> uint32_t {  // thread 0: bounded wait for the copy in flight into buffer buf
-        uint32_t done = 0;
-        for (int spin = 0; spin < (1 << 20) && !done; ++spin)
-            asm volatile("{ .reg .pred q; mbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2; selp.u32 %0, 1, 0, q; }"
-                         : "=r"(done) : "r"(smem_addr_of(&bar[buf])), "r"((phase >> buf) & 1u) : "memory");
+    auto wait_for = [&](int buf) -> bool {  // thread 0: bounded wait for the copy in flight into buffer buf
+        const bool done = mbar_wait_bounded(&bar[buf], (phase >> buf) & 1u, p.copy_wait_limit);
         if (done) { phase ^= 1u << buf; pending &= ~(1u << buf); }
         return done;
     };
@@ -120,11 +91,11 @@ __global__ void __launch_bounds__(THREADS) sign_uplink_bf16_kernel(const __grid_
         const int len = t_len[i];
         if (t_fast[i]) {
             if (threadIdx.x == 0 && !wait_for(buf)) {
-                // a copy that does not land is flagged; the other buffer's copy gets one more bounded
+                // a copy that does not land is flagged; both buffers' copies get one more bounded
                 // wait so that nothing is in flight into this CTA's shared memory when it leaves
                 atomicOr(p.status, STATUS_COPY_TIMEOUT);
-                if (pending & (1u << (buf ^ 1))) wait_for(buf ^ 1);
-                wait_for(buf);
+                if (pending & (1u << (buf ^ 1))) mbar_drain(&bar[buf ^ 1], (phase >> (buf ^ 1)) & 1u);
+                mbar_drain(&bar[buf], (phase >> buf) & 1u);
                 copy_ok = 0;
             }
         } else {
@@ -175,75 +146,34 @@ __global__ void __launch_bounds__(THREADS) sign_uplink_bf16_kernel(const __grid_
 }
 
 // ------------------------------------------------------------------------------------------------
-// Scale: one CTA per (segment, row).  Tile partials are combined pairwise, level by level,
-// over the tile count zero-padded to a power of two (adding +0 is exact), which continues the
-// segment's balanced tree above the tile level.
+// Scale: one CTA per (segment, row).  Tile partials are combined in tree order
+// (tree_reduce_partials), then scale = S / n.
 // ------------------------------------------------------------------------------------------------
-constexpr int FIN_CHUNK = 2048;
-
 __global__ void __launch_bounds__(THREADS) scale_finalize_kernel(const __grid_constant__ Params p,
                                                                   const double *partials, float *scales,
                                                                   double *sums /* when set: the plain sums instead */) {
     __shared__ double buf[FIN_CHUNK];
-    __shared__ double chunk_sums[512];  // 2^32 / TILE / FIN_CHUNK = 256 chunks at most
+    __shared__ double chunk_sums[FIN_MAX_CHUNKS];
     const int t = blockIdx.x, row = blockIdx.y;
     const int first = __ldg(p.tile_prefix + t);
     const int ntiles = __ldg(p.tile_prefix + t + 1) - first;
-    const double *src = partials + (int64_t)row * p.TT + first;
-    const int nchunks = (ntiles + FIN_CHUNK - 1) / FIN_CHUNK;
-
-    for (int c = 0; c < nchunks; ++c) {
-        // the chunk's tree over the next power of two of its tile count: the levels above it would
-        // only add +0, which changes nothing
-        const int here = min(FIN_CHUNK, ntiles - c * FIN_CHUNK);
-        int span = 1;
-        while (span < here) span <<= 1;
-        for (int q = threadIdx.x; q < span; q += THREADS) {
-            int idx = c * FIN_CHUNK + q;
-            buf[q] = idx < ntiles ? src[idx] : 0.0;
-        }
-        __syncthreads();
-        for (int width = span / 2; width >= 1; width >>= 1) {
-            // pairwise: new[q] = old[2q] + old[2q+1]; done in two phases to avoid overwrite hazards
-            double vals[FIN_CHUNK / 2 / THREADS];
-#pragma unroll
-            for (int r = 0; r < FIN_CHUNK / 2 / THREADS; ++r) {
-                int q = threadIdx.x + r * THREADS;
-                vals[r] = q < width ? __dadd_rn(buf[2 * q], buf[2 * q + 1]) : 0.0;
-            }
-            __syncthreads();
-#pragma unroll
-            for (int r = 0; r < FIN_CHUNK / 2 / THREADS; ++r) {
-                int q = threadIdx.x + r * THREADS;
-                if (q < width) buf[q] = vals[r];
-            }
-            __syncthreads();
-        }
-        if (threadIdx.x == 0) chunk_sums[c] = buf[0];
-        __syncthreads();
-    }
+    const double total = tree_reduce_partials(partials + (int64_t)row * p.TT + first, ntiles, buf, chunk_sums);
     if (threadIdx.x == 0) {
-        int L = 1;
-        while (L < nchunks) L <<= 1;
-        for (int c = nchunks; c < L; ++c) chunk_sums[c] = 0.0;
-        for (int width = L / 2; width >= 1; width >>= 1)
-            for (int q = 0; q < width; ++q) chunk_sums[q] = __dadd_rn(chunk_sums[2 * q], chunk_sums[2 * q + 1]);
         const int64_t n = __ldg(p.seg_off + t + 1) - __ldg(p.seg_off + t);
         if (sums) {
-            sums[(int64_t)row * p.T + t] = chunk_sums[0];
+            sums[(int64_t)row * p.T + t] = total;
         } else {
-            double mean = __ddiv_rn(chunk_sums[0], (double)n);
-            scales[(int64_t)row * p.T + t] = __double2float_rn(mean);
+            scales[(int64_t)row * p.T + t] = __double2float_rn(__ddiv_rn(total, (double)n));
         }
     }
 }
 
 // ------------------------------------------------------------------------------------------------
-// Server pass for dense uplink messages (sign words or raw gradients): one CTA per tile.
+// Server pass for an identity uplink (the messages are the raw gradients): one CTA per tile.
 //   acc = +0; for i = 0..N-1: acc = acc + p^i_j;   v_j = e_j + acc / N        (written over e)
 // and, when the downlink is scaled sign, the words of v and the tile partial of ||v||_1.
 // ------------------------------------------------------------------------------------------------
-template <int UP, bool DOWN_SIGN, typename GT>
+template <bool DOWN_SIGN, typename GT>
 __global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_constant__ Params p) {
     __shared__ double warp_sums[8];
     const TileInfo ti = locate_tile(p, blockIdx.x);
@@ -316,7 +246,8 @@ __global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_cons
 template <bool DOWN_SIGN>
 __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_constant__ Params p) {
     __shared__ double warp_sums[8];
-    extern __shared__ float up_scale_smem[];  // [N] scales of this segment
+    constexpr int SCALE_CHUNK = 1024;              // workers whose scales are staged at once (a multiple of WG)
+    __shared__ float up_scale_smem[SCALE_CHUNK];   // this segment's scales of workers c0 .. c0 + SCALE_CHUNK - 1
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int lane = threadIdx.x & 31;
     const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
@@ -324,8 +255,6 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
     const int nwords = (ti.len + 31) >> 5;
     const int my_widx = threadIdx.x;
     const bool have_word = my_widx < nwords;
-    for (int i = threadIdx.x; i < p.N; i += THREADS) up_scale_smem[i] = p.up_scales[(int64_t)i * p.T + ti.t];
-    __syncthreads();
 
     float acc[32];
 #pragma unroll
@@ -337,6 +266,12 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
 #pragma unroll
     for (int u = 0; u < WG; ++u) nextw[u] = (have_word && u < p.N) ? __ldg(wp + (int64_t)u * p.W) : 0u;
     for (int i0 = 0; i0 < p.N; i0 += WG) {
+        if ((i0 & (SCALE_CHUNK - 1)) == 0) {  // (uniform over the CTA) next chunk of scales
+            if (i0) __syncthreads();
+            for (int i = threadIdx.x; i < SCALE_CHUNK && i0 + i < p.N; i += THREADS)
+                up_scale_smem[i] = p.up_scales[(int64_t)(i0 + i) * p.T + ti.t];
+            __syncthreads();
+        }
         uint32_t w[WG];
 #pragma unroll
         for (int u = 0; u < WG; ++u) w[u] = nextw[u];
@@ -348,7 +283,7 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
 #pragma unroll
         for (int u = 0; u < WG; ++u) {
             if (i0 + u < p.N) {  // uniform over the CTA
-                const uint32_t sbits = __float_as_uint(up_scale_smem[i0 + u]);
+                const uint32_t sbits = __float_as_uint(up_scale_smem[(i0 + u) & (SCALE_CHUNK - 1)]);
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
                     const float pij = __uint_as_float(sbits ^ ((w[u] << (31 - c)) & 0x80000000u));
@@ -402,32 +337,6 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
         if (threadIdx.x == 0) p.down_partials[blockIdx.x] = s;
     }
     (void)lane;
-}
-
-// First half of a sign downlink on a v that is already in the error buffer (used when the
-// aggregation kernel could not fuse it, i.e. after a top-k uplink).
-__global__ void __launch_bounds__(THREADS) sign_downlink_kernel(const __grid_constant__ Params p) {
-    __shared__ double warp_sums[8];
-    const TileInfo ti = locate_tile(p, blockIdx.x);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
-    const int64_t wbase = __ldg(p.word_off + ti.t) + ti.rel / 32;
-    const int nwords = (ti.len + 31) >> 5;
-    const float *v_tile = p.e + ti.seg_beg + ti.rel;
-    double a[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const int pos = tile_pos(warp, lane, j);
-        float v[4];
-        if (fast) load4_stream(v_tile + pos, v);
-        else load4_guarded(v_tile, pos, ti.len, v);
-        a[j] = leaf4(v);
-        uint32_t w = pack_word(sign_nibble(v), lane);
-        int widx = warp * 32 + j * 4 + (lane >> 3);
-        if ((lane & 7) == 0 && widx < nwords) p.down_words[wbase + widx] = w;
-    }
-    double s = cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
-    if (threadIdx.x == 0) p.down_partials[blockIdx.x] = s;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -531,27 +440,21 @@ cudaError_t launch_scale_finalize(const Params &p, bool uplink, cudaStream_t st)
     return cudaGetLastError();
 }
 
-template <int UP, typename GT>
+template <typename GT>
 static cudaError_t launch_server_dense_t(const Params &p, cudaStream_t st) {
-    if (p.down == COMP_SIGN) server_dense_kernel<UP, true, GT><<<p.TT, THREADS, 0, st>>>(p);
-    else server_dense_kernel<UP, false, GT><<<p.TT, THREADS, 0, st>>>(p);
+    if (p.down == COMP_SIGN) server_dense_kernel<true, GT><<<p.TT, THREADS, 0, st>>>(p);
+    else server_dense_kernel<false, GT><<<p.TT, THREADS, 0, st>>>(p);
     return cudaGetLastError();
 }
 
 cudaError_t launch_server_dense(const Params &p, cudaStream_t st) {
     if (p.up == COMP_SIGN) {
-        const size_t smem = sizeof(float) * (size_t)p.N;
-        if (p.down == COMP_SIGN) server_sign_kernel<true><<<p.TT, THREADS, smem, st>>>(p);
-        else server_sign_kernel<false><<<p.TT, THREADS, smem, st>>>(p);
+        if (p.down == COMP_SIGN) server_sign_kernel<true><<<p.TT, THREADS, 0, st>>>(p);
+        else server_sign_kernel<false><<<p.TT, THREADS, 0, st>>>(p);
         return cudaGetLastError();
     }
-    if (p.gdt == DT_F32) return launch_server_dense_t<COMP_IDENTITY, float>(p, st);
-    return launch_server_dense_t<COMP_IDENTITY, __nv_bfloat16>(p, st);
-}
-
-cudaError_t launch_sign_downlink(const Params &p, cudaStream_t st) {
-    sign_downlink_kernel<<<p.TT, THREADS, 0, st>>>(p);
-    return cudaGetLastError();
+    if (p.gdt == DT_F32) return launch_server_dense_t<float>(p, st);
+    return launch_server_dense_t<__nv_bfloat16>(p, st);
 }
 
 cudaError_t launch_sign_error(const Params &p, cudaStream_t st) {

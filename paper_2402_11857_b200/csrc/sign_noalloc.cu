@@ -22,78 +22,26 @@ constexpr int NOALLOC_MAX_TILES = (int)(NOALLOC_MAX_ELEMENTS / TILE);
 // values, which is harmless because a call only reads the partials that it has just written.
 static __device__ __align__(256) double g_noalloc_partials[NOALLOC_MAX_TILES];
 
+// One CTA per tile: the same tile routine as the regular uplink pass, partials into the fixed array.
 template <typename GT>
 __global__ void __launch_bounds__(THREADS) sign_noalloc_kernel(const GT *x, int64_t n, uint32_t *words,
                                                                 double *partials) {
     __shared__ double warp_sums[8];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t rel = (int64_t)blockIdx.x * TILE;
     const int64_t left = n - rel;
     const int len = left < TILE ? (int)left : TILE;
-    const GT *tile_ptr = x + rel;
-    const bool fast = len == TILE;  // x itself is 16-byte aligned (checked on the host)
-    float v[8][4];
-    if (fast) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) load4_stream(tile_ptr + tile_pos(warp, lane, j), v[j]);
-    } else {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), len, v[j]);
-    }
-    uint32_t *wtile = words + rel / 32;
-    const int nwords = (len + 31) >> 5;
-    double a[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        a[j] = leaf4(v[j]);
-        uint32_t w = pack_word(sign_nibble(v[j]), lane);
-        int widx = warp * 32 + j * 4 + (lane >> 3);
-        if ((lane & 7) == 0 && widx < nwords) wtile[widx] = w;
-    }
-    double s = cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
+    // x itself is 16-byte aligned (checked on the host), hence every full tile is
+    const double s = sign_tile(x + rel, len, len == TILE, words + rel / 32, warp_sums);
     if (threadIdx.x == 0) partials[blockIdx.x] = s;
 }
 
-// Single CTA: tile partials -> ||x||_1 in tree order (chunks of 2048, then the chunk sums) -> scale.
-constexpr int NA_CHUNK = 2048;
-
-__global__ void __launch_bounds__(THREADS) scale_noalloc_chunked_kernel(const double *partials, int ntiles,
-                                                                         int64_t n, float *scale) {
-    __shared__ double buf[NA_CHUNK];
-    __shared__ double chunk_sums[NOALLOC_MAX_TILES / NA_CHUNK];
-    const int nchunks = (ntiles + NA_CHUNK - 1) / NA_CHUNK;
-    for (int c = 0; c < nchunks; ++c) {
-        for (int q = threadIdx.x; q < NA_CHUNK; q += THREADS) {
-            int idx = c * NA_CHUNK + q;
-            buf[q] = idx < ntiles ? partials[idx] : 0.0;
-        }
-        __syncthreads();
-        for (int width = NA_CHUNK / 2; width >= 1; width >>= 1) {
-            double vals[NA_CHUNK / 2 / THREADS];
-#pragma unroll
-            for (int r = 0; r < NA_CHUNK / 2 / THREADS; ++r) {
-                int q = threadIdx.x + r * THREADS;
-                vals[r] = q < width ? __dadd_rn(buf[2 * q], buf[2 * q + 1]) : 0.0;
-            }
-            __syncthreads();
-#pragma unroll
-            for (int r = 0; r < NA_CHUNK / 2 / THREADS; ++r) {
-                int q = threadIdx.x + r * THREADS;
-                if (q < width) buf[q] = vals[r];
-            }
-            __syncthreads();
-        }
-        if (threadIdx.x == 0) chunk_sums[c] = buf[0];
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-        int L = 1;
-        while (L < nchunks) L <<= 1;
-        for (int c = nchunks; c < L; ++c) chunk_sums[c] = 0.0;
-        for (int width = L / 2; width >= 1; width >>= 1)
-            for (int q = 0; q < width; ++q) chunk_sums[q] = __dadd_rn(chunk_sums[2 * q], chunk_sums[2 * q + 1]);
-        *scale = __double2float_rn(__ddiv_rn(chunk_sums[0], (double)n));
-    }
+// Single CTA: tile partials -> ||x||_1 in tree order (the regular path's reducer) -> scale.
+__global__ void __launch_bounds__(THREADS) scale_noalloc_kernel(const double *partials, int ntiles, int64_t n,
+                                                                 float *scale) {
+    __shared__ double buf[FIN_CHUNK];
+    __shared__ double chunk_sums[FIN_MAX_CHUNKS];
+    const double total = tree_reduce_partials(partials, ntiles, buf, chunk_sums);
+    if (threadIdx.x == 0) *scale = __double2float_rn(__ddiv_rn(total, (double)n));
 }
 
 // Device address of the scratch array, looked up once per device.  In host code the array's
@@ -154,7 +102,7 @@ extern "C" liec_status liec_sign_compress_noalloc(const void *x, int32_t dtype, 
         sign_noalloc_kernel<__nv_bfloat16><<<ntiles, THREADS, 0, st>>>(static_cast<const __nv_bfloat16 *>(x), n, words, partials);
     e = cudaGetLastError();
     if (e == cudaSuccess) {
-        scale_noalloc_chunked_kernel<<<1, THREADS, 0, st>>>(partials, ntiles, n, scale);
+        scale_noalloc_kernel<<<1, THREADS, 0, st>>>(partials, ntiles, n, scale);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) {

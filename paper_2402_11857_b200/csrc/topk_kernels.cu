@@ -152,6 +152,7 @@ __global__ void topk_begin_kernel(const __grid_constant__ Params p, const TopkSi
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
     const bool guess = sel[SEL_GUESS] != 0u;
     sel[SEL_MODE] = guess ? 1u : 0u;
+    sel[SEL_SPEC_FAIL] = 0u;
     sel[SEL_CAND_COUNT] = 0u;
     sel[SEL_FLAGS] = 0u;
     if (!guess) p.status[STATUS_ANY_REGULAR] = 1;
@@ -217,7 +218,14 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
     //          (uplink single-pass route); checks the guess.
     // level 4: second digit of "refined" problems, after their dense second-digit pass.
     // levels 2, 3: wide form of the finish step (second digit, last 7 bits) from candidate histograms.
-    if (level == 5 && sel[SEL_MODE] != 1u) return;
+    if (level == 5) {
+        if (sel[SEL_MODE] != 1u) return;
+        if (sel[SEL_SPEC_FAIL] != 0u) {  // the guess let too much through: regular route (nothing was added to the histogram)
+            __syncthreads();             // every thread has read the mode before it changes
+            if (threadIdx.x == 0) { sel[SEL_MODE] = 0u; p.status[STATUS_ANY_REGULAR] = 1; }
+            return;
+        }
+    }
     if (level == 2 && sel[SEL_FLAGS] != 0u) return;
     if (level == 3 && (sel[SEL_FLAGS] & 1u)) return;
     if (level == 1 && s.spec && sel[SEL_MODE] != 0u) return;
@@ -361,9 +369,6 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t x, uint32_t *w
 // bit pattern used as a float: for finite values the order is the same).  Ragged or misaligned
 // tiles are copied with guarded loads instead of the bulk copy and then take the same path.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_addr(const void *ptr) { return (uint32_t)__cvta_generic_to_shared(ptr); }
-
-
 // GT = float or __nv_bfloat16: the element type of the source (bf16 tiles are half the bytes; a
 // thread's 32 elements are then four 16-byte chunks instead of eight).
 template <typename GT, bool SPEC>
@@ -378,7 +383,7 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
     if (!SPEC && s.spec && p.status[STATUS_ANY_REGULAR] == 0) return;
     const int row = blockIdx.y, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bar)));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bar)));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -388,7 +393,10 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
         uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
         float low;
         if (SPEC) {
-            if (sel[SEL_MODE] != 1u) continue;  // (uniform over the CTA, like every `continue` before the barriers)
+            // (uniform over the CTA, like every `continue` before the barriers: no kernel writes, in the
+            // launch in which it runs, a word that it branches on; a guess that fails is recorded in
+            // SEL_SPEC_FAIL, which only later launches read)
+            if (sel[SEL_MODE] != 1u) continue;
             low = __uint_as_float(sel[SEL_GUESS]);
         } else {
             if (s.spec && sel[SEL_MODE] != 0u) continue;
@@ -402,18 +410,16 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
         if (fast) {
             if (threadIdx.x == 0) {
                 const uint32_t bytes = TILE * sizeof(ST);
-                // earlier ordinary reads/writes of the buffer (ordered by the barrier above) before the async copy
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(&bar)), "r"(bytes) : "memory");
-                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                             ::"r"(smem_addr(tile_s)), "l"(tile_ptr), "r"(bytes), "r"(smem_addr(&bar)) : "memory");
+                // (earlier ordinary reads of the buffer are ordered before the copy by the barrier above)
+                bulk_copy_g2s(tile_s, tile_ptr, bytes, bytes + p.copy_expect_extra, &bar);
             }
-            // bounded wait for the copy (a wait that never ends must not hang the GPU: flag it and leave)
-            uint32_t done = 0;
-            for (int spin = 0; spin < (1 << 20) && !done; ++spin)
-                asm volatile("{ .reg .pred q; mbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2; selp.u32 %0, 1, 0, q; }"
-                             : "=r"(done) : "r"(smem_addr(&bar)), "r"(phase) : "memory");
-            if (!done) { atomicOr(p.status, STATUS_COPY_TIMEOUT); return; }
+            // bounded wait for the copy (a wait that never ends must not hang the GPU): flag it, give a
+            // copy that may still be in flight time to land, and leave without touching any output
+            if (!mbar_wait_bounded(&bar, phase, p.copy_wait_limit)) {
+                atomicOr(p.status, STATUS_COPY_TIMEOUT);
+                mbar_drain(&bar, phase);
+                return;
+            }
             phase ^= 1u;
         } else {
             stage_tile_guarded(tile_s, tile_ptr, ti.len, (row_beg & ALIGN_MASK) == 0);
@@ -457,7 +463,7 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
             uint32_t at = tile_cnt ? atomicAdd(&sel[SEL_CAND_COUNT], tile_cnt) : 0u;
             if (at + tile_cnt > cap) {
                 if (SPEC) {  // the guess lets too much through: this problem takes the regular route
-                    sel[SEL_MODE] = 0u;
+                    sel[SEL_SPEC_FAIL] = 1u;
                     p.status[STATUS_ANY_REGULAR] = 1;
                 } else {
                     atomicOr(p.status, STATUS_CAND_OVERFLOW);
@@ -539,7 +545,8 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
         if (active) {
             cb = cand_block(p, s, tile, row);
             const uint32_t flags = cb.sel[SEL_FLAGS];
-            active = !cb.skip && !(level == 0 && cb.sel[SEL_MODE] != 1u) && !(level == 1 && flags != 0u);
+            active = !cb.skip && !(level == 0 && (cb.sel[SEL_MODE] != 1u || cb.sel[SEL_SPEC_FAIL] != 0u)) &&
+                     !(level == 1 && flags != 0u);
             prefix = cb.sel[SEL_PREFIX];
         }
         uint32_t lo = 0xffffffffu, hi = 0u;

@@ -71,6 +71,12 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.liec_set_subsets.restype = C.c_int
     lib.liec_step.argtypes = [vp, vp, C.c_float, vp]
     lib.liec_step.restype = C.c_int
+    lib.liec_topk_route_counts.argtypes = [vp, vp, C.c_int32, C.POINTER(C.c_int64)]
+    lib.liec_topk_route_counts.restype = C.c_int
+    lib.liec_abort_step.argtypes = [vp]
+    lib.liec_abort_step.restype = C.c_int
+    lib.liec_set_copy_wait.argtypes = [vp, C.c_uint32, C.c_uint32]
+    lib.liec_set_copy_wait.restype = C.c_int
     lib.liec_average_step.argtypes = [vp, vp, C.c_float, vp]
     lib.liec_average_step.restype = C.c_int
     lib.liec_mean_params.argtypes = [vp, vp, vp]
@@ -142,6 +148,14 @@ def liec_sign_compress_noalloc(x, words, scale, stream=None):
     (float32, 1 element) without any workspace or allocation; see liec.h for who needs this."""
     import torch
     lib = load_library()
+    n = x.numel()
+    if not (x.is_cuda and x.is_contiguous() and x.dtype in (torch.float32, torch.bfloat16)):
+        raise ValueError("x must be a contiguous CUDA tensor of float32 or bfloat16")
+    if not (words.is_cuda and words.is_contiguous() and words.dtype in (torch.int32, torch.uint32)
+            and words.numel() == (n + 31) // 32 and words.device == x.device):
+        raise ValueError("words must be a contiguous CUDA tensor of ceil(n/32) 32-bit integers on x's device")
+    if not (scale.is_cuda and scale.dtype == torch.float32 and scale.numel() == 1 and scale.device == x.device):
+        raise ValueError("scale must be a one-element float32 CUDA tensor on x's device")
     dtype = BF16 if x.dtype == torch.bfloat16 else F32
     s = (stream if stream is not None else torch.cuda.current_stream(x.device)).cuda_stream
     with torch.cuda.device(x.device):
@@ -226,6 +240,17 @@ class Context:
     def liec_step(self, grads, lr: float, stream=None):
         self._check_grads(grads)
         self._check(self.lib.liec_step(self._ctx, grads.data_ptr(), float(lr), self._stream(stream)))
+
+    def liec_topk_route_counts(self, uplink: bool, stream=None) -> dict:
+        out = (C.c_int64 * 4)()
+        self._check(self.lib.liec_topk_route_counts(self._ctx, self._stream(stream), 1 if uplink else 0, out))
+        return {"problems": int(out[0]), "single_pass": int(out[1]), "refined": int(out[2]), "slow": int(out[3])}
+
+    def liec_abort_step(self):
+        self._check(self.lib.liec_abort_step(self._ctx))
+
+    def liec_set_copy_wait(self, poll_limit: int = 0, expect_extra_bytes: int = 0):
+        self._check(self.lib.liec_set_copy_wait(self._ctx, int(poll_limit), int(expect_extra_bytes)))
 
     def liec_average_step(self, grads, lr: float, stream=None):
         self._check_grads(grads)

@@ -28,7 +28,34 @@ def _sample_segments(lay, budget_elems):
     return sorted(chosen)
 
 
-def _run(name, steps, budget_elems, randk=False):
+def _pack_negative(x):
+    """Sign words by the definition, on the device: bit b of word w is set iff x[32w+b] < 0 (int64 tensor)."""
+    n = x.numel()
+    neg = torch.zeros(((n + 31) // 32) * 32, dtype=torch.bool, device=x.device)
+    neg[:n] = x < 0
+    return (neg.view(-1, 32).to(torch.int64) << torch.arange(32, device=x.device)).sum(dim=1)
+
+
+def _check_whole_segment_sign(ctx, m, G, v_seg, lay, t, woff):
+    """One segment too large for an oracle step with all workers (the 38.6 M-element embedding):
+    every worker's scale and the server's against the oracle's scale of the same bytes, the words
+    against the definition."""
+    off = lay.seg_offsets
+    lo, hi = int(off[t]), int(off[t + 1])
+    for i in range(G.shape[0]):
+        want = oracle.scale(widen(G[i, lo:hi]))
+        got = f32(m["up_scales"][i, t:t + 1])[0]
+        assert np.float32(got).view(np.uint32) == np.float32(want).view(np.uint32), ("up scale", i, got, want)
+        words = m["up_words"][i, woff[t]:woff[t + 1]].to(torch.int64) & 0xFFFFFFFF
+        assert torch.equal(words, _pack_negative(G[i, lo:hi].float())), ("up words", i)
+    want = oracle.scale(f32(v_seg))
+    got = f32(m["down_scales"][t:t + 1])[0]
+    assert np.float32(got).view(np.uint32) == np.float32(want).view(np.uint32), ("down scale", got, want)
+    words = m["down_words"][woff[t]:woff[t + 1]].to(torch.int64) & 0xFFFFFFFF
+    assert torch.equal(words, _pack_negative(v_seg)), "down words"
+
+
+def _run(name, steps, budget_elems, randk=False, whole_segment=None, routes=None):
     w = WORKLOADS[name]
     lay = w.layout()
     N, d, off = w.num_workers, lay.dim, lay.seg_offsets
@@ -64,10 +91,24 @@ def _run(name, steps, budget_elems, randk=False):
             part = np.concatenate([sets[:, koff[t]:koff[t + 1]].astype(np.int64) - (int(off[t]) - int(sub_off[q]))
                                    for q, t in enumerate(segs)], axis=1).astype(np.uint32)
             sub_sets = dict(up_sets=part[:N], down_set=part[N])
-        ctx.liec_step(G, w.lr)
+        v_seg = None
+        if whole_segment is not None and step == steps - 1:
+            # staged, so that v of the large segment can be read before the downlink overwrites it
+            ctx.liec_uplink_compress(G)
+            ctx.liec_server_aggregate()
+            torch.cuda.synchronize()
+            v_seg = e[int(off[whole_segment]):int(off[whole_segment + 1])].clone()
+            ctx.liec_downlink_compress()
+            ctx.liec_worker_update(G, w.lr)
+        else:
+            ctx.liec_step(G, w.lr)
         torch.cuda.synchronize()
         assert ctx.liec_device_status() == 0
         m = ctx.liec_get_messages()
+        if v_seg is not None:
+            _check_whole_segment_sign(ctx, m, G, v_seg, lay, whole_segment, woff)
+        if routes is not None:
+            routes.append((ctx.liec_topk_route_counts(True), ctx.liec_topk_route_counts(False)))
         r = oracle.step(Xh, eh, widen(G[:, cols]), w.lr, sub_off, ocomp, ocomp, k=ksub, **sub_sets)
         assert_close(f32(X[:, cols]), Xh, f"{name} step {step}: params on sampled segments")
         assert_close(f32(e[cols]), eh, f"{name} step {step}: error on sampled segments")
@@ -113,15 +154,26 @@ def _run(name, steps, budget_elems, randk=False):
 
 
 def test_c2_resnet18_sign_full_size():
-    _run("c2", steps=3, budget_elems=4_000_000)
+    _run("c2", steps=10, budget_elems=4_000_000)
 
 
 def test_c3_resnet50_topk_full_size():
-    _run("c3", steps=2, budget_elems=3_500_000)
+    """20 iterations on fresh gradients: error feedback has piled v up under the thresholds and the
+    uplink runs on the thresholds of the step before."""
+    routes = []
+    _run("c3", steps=20, budget_elems=3_500_000, routes=routes)
+    up, down = routes[-1]
+    assert up["problems"] == 16 * 161 and down["problems"] == 161
+    # after the first step the uplink takes the single-pass route for most problems (the rest are
+    # mainly the k = 1 problems of the small tensors, whose threshold is a maximum and moves a lot)
+    assert all(u["single_pass"] > 0.5 * u["problems"] for u, _ in routes[1:]), [u for u, _ in routes]
+    assert all(u["slow"] == 0 and dn["slow"] == 0 for u, dn in routes)
+    print("c3 routes per step (uplink single-pass, uplink refined, downlink refined):",
+          [(u["single_pass"], u["refined"], dn["refined"]) for u, dn in routes])
 
 
 def test_c4_gpt2_sign_bf16_full_size():
-    _run("c4", steps=2, budget_elems=4_000_000)
+    _run("c4", steps=5, budget_elems=4_000_000, whole_segment=0)
 
 
 def test_c3_resnet50_randk_full_size():

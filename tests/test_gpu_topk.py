@@ -196,3 +196,25 @@ def test_topk_staged_equals_step_and_deterministic():
         assert torch.equal(a, b)
     for a, b in zip(outs[0], outs[2]):
         assert torch.equal(a, b)
+
+
+def test_guess_overflow_on_a_segment_of_hundreds_of_tiles():
+    """The gradient scale rises 50-fold step after step (what a learning-rate warm-up does), so each
+    step's guess, last step's threshold, lets far more through than the candidate buffer holds.  With
+    288 tiles per problem many CTAs are in flight when the first one finds the buffer full; the problem
+    must fall back to the regular route as a whole, with a clean status word."""
+    lay = flat_layout(2359296)
+    k = topk_counts(lay, 1, 100)
+    P = _pair(3, lay.seg_offsets, TOPK, TOPK, k=k)
+    scale = 1e-6
+    for step in range(7):
+        G = make_gradients("normal", 1.0, 3, lay.dim, step, base_seed=26) * scale
+        P.step(G, 0.1, check_messages=(step in (0, 3, 6)))
+        routes = P.ctx.liec_topk_route_counts(True)
+        assert routes["single_pass"] == 0, (step, routes)   # first step: no guess; later: every guess overflows
+        scale *= 50.0
+    # steady scale again: the guess holds
+    for step in range(7, 9):
+        G = make_gradients("normal", 1.0, 3, lay.dim, step, base_seed=26) * scale
+        P.step(G, 0.1)
+    assert P.ctx.liec_topk_route_counts(True)["single_pass"] == 3
