@@ -546,7 +546,7 @@ liec_status liec_device_status(liec_ctx *c, void *stream, int32_t *out) {
     return LIEC_OK;
 }
 
-liec_status liec_topk_route_counts(liec_ctx *c, void *stream, int32_t uplink, int64_t *out) {
+liec_status liec_topk_route_counts(liec_ctx *c, void *stream, int32_t uplink, int64_t *out, uint8_t *per_problem) {
     if (!c || !out) return LIEC_ERR_INVALID_ARG;
     const uint32_t *sel = uplink ? c->p.up_sel : c->p.down_sel;
     const int64_t problems = (int64_t)(uplink ? c->p.N : 1) * c->p.T;
@@ -561,9 +561,9 @@ liec_status liec_topk_route_counts(liec_ctx *c, void *stream, int32_t uplink, in
     out[0] = problems;
     for (int64_t q = 0; q < problems; ++q) {
         const uint32_t *w = host.data() + q * SEL_WORDS;
-        if (uplink && w[SEL_MODE] == 1u) ++out[1];
-        if (w[SEL_FLAGS] & 2u) ++out[2];
-        if (w[SEL_FLAGS] & 1u) ++out[3];
+        const bool single = uplink && w[SEL_MODE] == 1u, refined = (w[SEL_FLAGS] & 2u) != 0u, slow = (w[SEL_FLAGS] & 1u) != 0u;
+        out[1] += single; out[2] += refined; out[3] += slow;
+        if (per_problem) per_problem[q] = (uint8_t)((single ? 1 : 0) | (refined ? 2 : 0) | (slow ? 4 : 0));
     }
     return LIEC_OK;
 }

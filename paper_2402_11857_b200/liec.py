@@ -71,7 +71,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.liec_set_subsets.restype = C.c_int
     lib.liec_step.argtypes = [vp, vp, C.c_float, vp]
     lib.liec_step.restype = C.c_int
-    lib.liec_topk_route_counts.argtypes = [vp, vp, C.c_int32, C.POINTER(C.c_int64)]
+    lib.liec_topk_route_counts.argtypes = [vp, vp, C.c_int32, C.POINTER(C.c_int64), vp]
     lib.liec_topk_route_counts.restype = C.c_int
     lib.liec_abort_step.argtypes = [vp]
     lib.liec_abort_step.restype = C.c_int
@@ -241,10 +241,17 @@ class Context:
         self._check_grads(grads)
         self._check(self.lib.liec_step(self._ctx, grads.data_ptr(), float(lr), self._stream(stream)))
 
-    def liec_topk_route_counts(self, uplink: bool, stream=None) -> dict:
+    def liec_topk_route_counts(self, uplink: bool, stream=None, per_problem: bool = False) -> dict:
+        """Counts of the routes taken by the last iteration's selections; with per_problem also a uint8
+        array [rows, T] of flags (1 single pass, 2 second-digit pass, 4 one-CTA path)."""
         out = (C.c_int64 * 4)()
-        self._check(self.lib.liec_topk_route_counts(self._ctx, self._stream(stream), 1 if uplink else 0, out))
-        return {"problems": int(out[0]), "single_pass": int(out[1]), "refined": int(out[2]), "slow": int(out[3])}
+        flags = np.zeros(((self.N if uplink else 1), self.T), np.uint8) if per_problem else None
+        self._check(self.lib.liec_topk_route_counts(self._ctx, self._stream(stream), 1 if uplink else 0, out,
+                                                    None if flags is None else flags.ctypes.data_as(C.c_void_p)))
+        r = {"problems": int(out[0]), "single_pass": int(out[1]), "refined": int(out[2]), "slow": int(out[3])}
+        if flags is not None:
+            r["flags"] = flags
+        return r
 
     def liec_abort_step(self):
         self._check(self.lib.liec_abort_step(self._ctx))
