@@ -342,7 +342,7 @@ def run_gpu(args, w, rank, world, local_rank, steps=None, extras=True):
     X = torch.zeros(N, d, device=dev)
     e = torch.zeros(d, device=dev)
     ctx = liec.Context(X, e, lay.seg_offsets, comp, comp, w["k"], gdt)
-    NUM_BATCHES = num_batches(w)
+    NUM_BATCHES = args.batches or num_batches(w)
     # the gradient of worker i at step t is drawn from seed (i, t): NUM_BATCHES consecutive steps'
     # draws are resident and the steps cycle through them (every step sees other values than the one
     # before, which matters for top-k: its uplink starts from the previous step's thresholds)
@@ -407,15 +407,20 @@ def run_gpu(args, w, rank, world, local_rank, steps=None, extras=True):
     # count needs a synchronisation and a copy of the selection state)
     routes = None
     if w["comp"] == "topk":
-        acc = {"uplink_single_pass": 0, "uplink_refined": 0, "downlink_refined": 0, "slow": 0}
-        extra = 2 * NUM_BATCHES
+        acc = {"uplink_single_pass": 0, "uplink_direct": 0, "uplink_refined": 0, "downlink_refined": 0, "slow": 0}
+        extra = min(2 * NUM_BATCHES, 16)
         for _ in range(extra):
             one_step()
             up, down = ctx.liec_topk_route_counts(True), ctx.liec_topk_route_counts(False)
             acc["uplink_single_pass"] += up["single_pass"]; acc["uplink_refined"] += up["refined"]
+            acc["uplink_direct"] += up["direct"]
             acc["downlink_refined"] += down["refined"]; acc["slow"] += up["slow"] + down["slow"]
         routes = {"uplink_problems": up["problems"], "downlink_problems": down["problems"], "steps_counted": extra,
+                  "uplink_single_tile_fraction": acc["uplink_direct"] / (extra * up["problems"]),
                   "uplink_single_pass_fraction": acc["uplink_single_pass"] / (extra * up["problems"]),
+                  "note": "single tile: segments of at most 8192 elements, selected by one CTA; single pass: "
+                          "finished on the one dense pass seeded by the previous step's threshold; the rest "
+                          "took the two-pass route",
                   "uplink_refined_per_step": acc["uplink_refined"] / extra,
                   "downlink_refined_per_step": acc["downlink_refined"] / extra, "slow_per_step": acc["slow"] / extra}
     if not extras:
@@ -552,6 +557,8 @@ def main():
     ap.add_argument("--workload", default=None,
                     help="one workload only (c1..c4, c4/8, c3-randk, sweep-sign-28, ...); default: c4 as the headline "
                          "plus c3 and two sweep points under their own keys")
+    ap.add_argument("--batches", type=int, default=0,
+                    help="resident gradient batches the steps cycle through (default: as many as fit in 40 GB, 4 to 16)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -265,13 +265,14 @@ liec_status liec_set_copy_wait(liec_ctx *ctx, uint32_t poll_limit, uint32_t expe
  *   out[0] problems, out[1] uplink problems that finished on the single dense pass seeded by the
  *   previous threshold, out[2] problems that needed the dense second-digit pass (more entries
  *   share the threshold's leading key bits than the candidate buffer holds), out[3] problems that
- *   fell back to the one-CTA dense path (huge groups of equal magnitudes).
+ *   fell back to the dense path of one CTA (huge groups of equal magnitudes), out[4] problems of a
+ *   single-tile segment (at most 8192 elements), which one CTA selects directly in shared memory.
  * per_problem (host, one byte per problem in [row][segment] order, or NULL) receives the same per
- * problem: bit 0 single pass, bit 1 second-digit pass, bit 2 one-CTA path.
+ * problem: bit 0 single pass, bit 1 second-digit pass, bit 2 dense one-CTA path, bit 3 single tile.
  * The result of the selection never depends on the route.  LIEC_ERR_INVALID_ARG when the side does
  * not use top-k.
  */
-liec_status liec_topk_route_counts(liec_ctx *ctx, void *stream, int32_t uplink, int64_t *out /* [4] */,
+liec_status liec_topk_route_counts(liec_ctx *ctx, void *stream, int32_t uplink, int64_t *out /* [5] */,
                                    uint8_t *per_problem);
 
 /* Number of kernel launches enqueued by this context so far (host-side counter). */

@@ -15,6 +15,7 @@ struct TileInfo {
     int64_t rel;      // first element of the tile, relative to the segment
     int len;          // valid elements in the tile (1..TILE)
     int tile_in_seg;  // tile index inside the segment
+    int seg_tiles;    // tiles of the segment
 };
 
 // Segment and extent of tile `tile` (table lookups only).
@@ -23,7 +24,9 @@ __device__ __forceinline__ TileInfo locate_tile(const Params &p, int tile) {
     ti.t = __ldg(p.tile_seg + tile);
     ti.seg_beg = __ldg(p.seg_off + ti.t);
     ti.n = __ldg(p.seg_off + ti.t + 1) - ti.seg_beg;
-    ti.tile_in_seg = tile - __ldg(p.tile_prefix + ti.t);
+    const int first_tile = __ldg(p.tile_prefix + ti.t);
+    ti.tile_in_seg = tile - first_tile;
+    ti.seg_tiles = __ldg(p.tile_prefix + ti.t + 1) - first_tile;
     ti.rel = (int64_t)ti.tile_in_seg * TILE;
     int64_t left = ti.n - ti.rel;
     ti.len = left < TILE ? (int)left : TILE;

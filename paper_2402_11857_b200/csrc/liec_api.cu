@@ -2,6 +2,7 @@
 // Every numeric step runs in the kernels launched from here.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -26,8 +27,8 @@ struct Plan {
     int32_t N = 0, T = 0, TT = 0;
     int64_t d = 0, W = 0, K = 0, CAP = 0, cap_max = 0;
     std::vector<int64_t> seg_off, word_off, k_off, cap_off, topk_k;
-    std::vector<int32_t> tile_prefix, tile_seg;
-    Region r_seg_off, r_word_off, r_k_off, r_cap_off, r_tile_prefix, r_tile_seg, r_status;
+    std::vector<int32_t> tile_prefix, tile_seg, small_seg, large_seg;
+    Region r_seg_off, r_word_off, r_k_off, r_cap_off, r_tile_prefix, r_tile_seg, r_small_seg, r_large_seg, r_status;
     Region r_tel_partials;
     Region r_up_words, r_up_scales, r_up_partials, r_down_words, r_down_scales, r_down_partials, r_vbuf;
     Region r_up_idx, r_up_val, r_down_idx, r_down_val;
@@ -110,13 +111,19 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
             if (cap > pl.cap_max) pl.cap_max = cap;
         }
     }
+    // the per-problem kernels take the largest segments first
+    std::stable_sort(pl.large_seg.begin(), pl.large_seg.end(), [&](int32_t a, int32_t b) {
+        return pl.seg_off[a + 1] - pl.seg_off[a] > pl.seg_off[b + 1] - pl.seg_off[b];
+    });
     pl.W = pl.word_off[T];
     pl.K = pl.k_off[T];
     pl.CAP = pl.cap_off[T];
     pl.TT = (int32_t)tiles;
     pl.tile_seg.resize(pl.TT);
-    for (int t = 0; t < T; ++t)
+    for (int t = 0; t < T; ++t) {
         for (int q = pl.tile_prefix[t]; q < pl.tile_prefix[t + 1]; ++q) pl.tile_seg[q] = t;
+        (pl.tile_prefix[t + 1] - pl.tile_prefix[t] == 1 ? pl.small_seg : pl.large_seg).push_back(t);
+    }
 
     Carver c;
     pl.r_seg_off = c.take(sizeof(int64_t) * (T + 1));
@@ -125,6 +132,8 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     pl.r_cap_off = c.take(sizeof(int64_t) * (T + 1));
     pl.r_tile_prefix = c.take(sizeof(int32_t) * (T + 1));
     pl.r_tile_seg = c.take(sizeof(int32_t) * pl.TT);
+    pl.r_small_seg = c.take(sizeof(int32_t) * pl.small_seg.size());
+    pl.r_large_seg = c.take(sizeof(int32_t) * pl.large_seg.size());
     pl.r_status = c.take(256);
     pl.r_tel_partials = c.take(sizeof(double) * (size_t)pl.N * pl.TT);
     const size_t N = pl.N;
@@ -288,6 +297,12 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     p.cap_off = at<int64_t>(c, pl.r_cap_off);
     p.tile_prefix = at<int32_t>(c, pl.r_tile_prefix);
     p.tile_seg = at<int32_t>(c, pl.r_tile_seg);
+    p.small_seg = at<int32_t>(c, pl.r_small_seg);
+    p.large_seg = at<int32_t>(c, pl.r_large_seg);
+    p.n_small = (int32_t)pl.small_seg.size();
+    p.n_large = (int32_t)pl.large_seg.size();
+    p.max_seg_tiles = 0;
+    for (int t = 0; t < pl.T; ++t) p.max_seg_tiles = std::max(p.max_seg_tiles, pl.tile_prefix[t + 1] - pl.tile_prefix[t]);
     p.status = at<int32_t>(c, pl.r_status);
     p.X = params;
     p.e = error;
@@ -313,9 +328,10 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     const Up ups[] = {
         {&pl.r_seg_off, pl.seg_off.data()}, {&pl.r_word_off, pl.word_off.data()}, {&pl.r_k_off, pl.k_off.data()},
         {&pl.r_cap_off, pl.cap_off.data()}, {&pl.r_tile_prefix, pl.tile_prefix.data()},
-        {&pl.r_tile_seg, pl.tile_seg.data()},
+        {&pl.r_tile_seg, pl.tile_seg.data()}, {&pl.r_small_seg, pl.small_seg.data()}, {&pl.r_large_seg, pl.large_seg.data()},
     };
     for (const Up &u : ups) {
+        if (!u.r->bytes) continue;
         cudaError_t e = cudaMemcpy(c->ws + u.r->off, u.src, u.r->bytes, cudaMemcpyHostToDevice);
         if (e != cudaSuccess) {
             snprintf(g_no_ctx_error, sizeof(g_no_ctx_error), "cudaMemcpy of tables failed: %s", cudaGetErrorString(e));
@@ -367,7 +383,7 @@ liec_status liec_uplink_compress(liec_ctx *c, const void *grads, void *stream) {
         LIEC_LAUNCH(c, launch_scale_finalize(c->p, true, s));
     } else if (c->p.up == COMP_TOPK) {
         LIEC_CALL(c, launch_topk_hist1(c->p, true, s, &c->launches));
-        LIEC_CALL(c, launch_topk_select(c->p, true, s, &c->launches));
+        LIEC_CALL(c, launch_topk_select(c->p, true, true, s, &c->launches));
     } else if (c->p.up == COMP_RANDK) {
         if (!c->p.up_sets) { c->err = "random-k uplink: no subsets given (liec_set_subsets)"; return LIEC_ERR_STATE; }
         LIEC_CALL(c, launch_randk_compress(c->p, true, s, &c->launches));
@@ -403,8 +419,9 @@ liec_status liec_downlink_compress(liec_ctx *c, void *stream) {
         LIEC_CALL(c, launch_randk_compress(c->p, false, s, &c->launches));
     } else {
         // the first-digit histogram of v is fused into the server pass after a sparse uplink
-        if (!comp_is_sparse(c->p.up)) LIEC_CALL(c, launch_topk_hist1(c->p, false, s, &c->launches));
-        LIEC_CALL(c, launch_topk_select(c->p, false, s, &c->launches));
+        const bool fused_hist = comp_is_sparse(c->p.up);
+        if (!fused_hist) LIEC_CALL(c, launch_topk_hist1(c->p, false, s, &c->launches));
+        LIEC_CALL(c, launch_topk_select(c->p, false, !fused_hist, s, &c->launches));
     }
     c->stage = 3;
     return LIEC_OK;
@@ -550,7 +567,7 @@ liec_status liec_topk_route_counts(liec_ctx *c, void *stream, int32_t uplink, in
     if (!c || !out) return LIEC_ERR_INVALID_ARG;
     const uint32_t *sel = uplink ? c->p.up_sel : c->p.down_sel;
     const int64_t problems = (int64_t)(uplink ? c->p.N : 1) * c->p.T;
-    out[0] = out[1] = out[2] = out[3] = 0;
+    out[0] = out[1] = out[2] = out[3] = out[4] = 0;
     if (!sel) { c->err = "this side does not use top-k"; return LIEC_ERR_INVALID_ARG; }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     std::vector<uint32_t> host((size_t)problems * SEL_WORDS);
@@ -561,9 +578,10 @@ liec_status liec_topk_route_counts(liec_ctx *c, void *stream, int32_t uplink, in
     out[0] = problems;
     for (int64_t q = 0; q < problems; ++q) {
         const uint32_t *w = host.data() + q * SEL_WORDS;
-        const bool single = uplink && w[SEL_MODE] == 1u, refined = (w[SEL_FLAGS] & 2u) != 0u, slow = (w[SEL_FLAGS] & 1u) != 0u;
-        out[1] += single; out[2] += refined; out[3] += slow;
-        if (per_problem) per_problem[q] = (uint8_t)((single ? 1 : 0) | (refined ? 2 : 0) | (slow ? 4 : 0));
+        const uint32_t route = w[SEL_ROUTE];
+        out[1] += (route & ROUTE_SINGLE) != 0; out[2] += (route & ROUTE_REFINED) != 0;
+        out[3] += (route & ROUTE_SLOW) != 0;   out[4] += (route & ROUTE_DIRECT) != 0;
+        if (per_problem) per_problem[q] = (uint8_t)route;
     }
     return LIEC_OK;
 }

@@ -35,6 +35,10 @@ struct Params {
     const int64_t *cap_off;      // [T+1] candidate capacity prefix (top-k only)
     const int32_t *tile_prefix;  // [T+1] tiles before segment t
     const int32_t *tile_seg;     // [TT] segment of every tile
+    const int32_t *small_seg;    // [n_small] segments of one tile (top-k: selected directly by one CTA)
+    const int32_t *large_seg;    // [n_large] segments of several tiles
+    int32_t n_small, n_large;
+    int32_t max_seg_tiles;       // tiles of the longest segment
 
     // state
     float *X;         // [N][d]
@@ -75,7 +79,7 @@ struct Params {
 constexpr uint32_t COPY_WAIT_LIMIT_DEFAULT = 1u << 20;
 
 // per-problem selection state words
-constexpr int SEL_WORDS = 16;
+constexpr int SEL_WORDS = 20;
 constexpr int SEL_PREFIX = 0;     // key prefix fixed so far (aligned to its bit position)
 constexpr int SEL_REMAIN = 1;     // rank still to find inside the prefix bin (1-based)
 constexpr int SEL_CAND_COUNT = 2; // atomic cursor: candidates appended so far
@@ -83,6 +87,7 @@ constexpr int SEL_THRESH = 3;     // final threshold key T
 constexpr int SEL_TIES = 4;       // number of entries equal to T to accept, lowest index first
 constexpr int SEL_CUT = 5;        // flat index of the last accepted tie
 constexpr int SEL_FLAGS = 6;      // bit0: slow path (one CTA, dense passes); bit1: refined (24-bit prefix found by a dense second-digit pass)
+                                  // (segments of a single tile never enter this machinery: one CTA selects them directly)
 constexpr int SEL_NCAND = 7;      // exact number of candidates (entries at or above the prefix)
 constexpr int SEL_ABOVE = 8;      // entries whose first digit is strictly above the threshold's
 constexpr int SEL_LO1 = 9;        // lowest / highest non-empty bin of the first-digit histogram (so that the
@@ -91,6 +96,9 @@ constexpr int SEL_LO2 = 11;       // same for the second-digit histogram
 constexpr int SEL_HI2 = 12;
 constexpr int SEL_GUESS = 13;      // uplink: lower bound (31-bit key) tried first in the next step; 0 = none
 constexpr int SEL_MODE = 14;       // uplink, this step: 1 = candidates collected with the guess, 0 = regular two-pass path
+constexpr int SEL_ROUTE = 16;      // how the last iteration's selection was done (ROUTE_* bits; diagnostics)
+constexpr int SEL_MARGIN = 17;     // uplink: first-digit bins between the next guess and the threshold's bin (0 = not yet chosen)
+constexpr int ROUTE_SINGLE = 1, ROUTE_REFINED = 2, ROUTE_SLOW = 4, ROUTE_DIRECT = 8;
 constexpr int SEL_SPEC_FAIL = 15;  // uplink, this step: the guess let too many candidates through (written by the
                                    // filter, read only by later kernels, which then send the problem down the regular path)
 

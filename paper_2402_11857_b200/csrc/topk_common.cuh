@@ -1,0 +1,245 @@
+// Shared by the top-k kernels (Def. 2): the description of one side of the iteration, the status
+// bits, and the block-wide helpers (histogram flush, rank pick, prefix sum).
+#pragma once
+#include "device_common.cuh"
+
+namespace liec {
+
+struct TopkSide {
+    const void *src;      // rows of the vector being compressed
+    int64_t row_stride;   // elements between rows (d for the uplink, 0 for the single downlink row)
+    int R;                // rows
+    uint32_t *idx; float *val;            // [R][K] output message
+    uint32_t *hist, *hist2, *sel;         // [R][T][...]
+    uint32_t *cand_idx; float *cand_val;  // [R][CAP]
+    uint32_t *meta;                        // [R][TT][4]: pos, cnt, n_greater -> unused, ties allowed
+    uint32_t *outbase;                     // [R][TT+1]
+    float *zero_out;                       // downlink: error buffer, selected entries become +0
+    int spec;                              // uplink: try last step's threshold first (single dense pass)
+};
+
+inline TopkSide make_side(const Params &p, bool uplink) {
+    TopkSide s;
+    if (uplink) {
+        s.src = p.G; s.row_stride = p.d; s.R = p.N;
+        s.idx = p.up_idx; s.val = p.up_val; s.hist = p.up_hist; s.hist2 = p.up_hist2; s.sel = p.up_sel;
+        s.cand_idx = p.up_cand_idx; s.cand_val = p.up_cand_val; s.meta = p.up_tile_meta; s.outbase = p.up_outbase;
+        s.zero_out = nullptr;
+        s.spec = 1;
+    } else {
+        s.src = p.e; s.row_stride = 0; s.R = 1;
+        s.idx = p.down_idx; s.val = p.down_val; s.hist = p.down_hist; s.hist2 = p.down_hist2; s.sel = p.down_sel;
+        s.cand_idx = p.down_cand_idx; s.cand_val = p.down_cand_val; s.meta = p.down_tile_meta; s.outbase = p.down_outbase;
+        s.zero_out = p.e;
+        s.spec = 0;
+    }
+    return s;
+}
+
+__device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) & 0x7fffffffu; }
+
+enum { STATUS_PICK_RANK = 1, STATUS_CAND_OVERFLOW = 2, STATUS_COUNT_MISMATCH = 4 };
+
+// Adds a CTA's shared-memory histogram to the problem's global one and widens the problem's
+// record of the non-empty bin range, so that the pick reads and clears only that range.
+__device__ __forceinline__ void flush_hist(const uint32_t *h, uint32_t *gh, uint32_t *sel, int lo_word, int hi_word) {
+    uint32_t lo = 0xffffffffu, hi = 0u;
+    for (uint32_t b = threadIdx.x; b < DIGIT1_BINS; b += blockDim.x) {
+        const uint32_t c = h[b];
+        if (c) {
+            atomicAdd(gh + b, c);
+            lo = min(lo, b);
+            hi = max(hi, b);
+        }
+    }
+    lo = __reduce_min_sync(0xffffffffu, lo);
+    hi = __reduce_max_sync(0xffffffffu, hi);
+    if ((threadIdx.x & 31) == 0 && lo != 0xffffffffu) {
+        atomicMin(&sel[lo_word], lo);
+        atomicMax(&sel[hi_word], hi);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Block helper: bins[0..nbins) in shared memory, find the bin that holds the rank-th largest
+// entry counting from the top bin down.  All threads get (bin, rank inside bin, count above+bin).
+// ------------------------------------------------------------------------------------------------
+struct PickResult { uint32_t bin, rank_in_bin, count_ge; bool ok; };
+
+template <int NT = THREADS>
+__device__ PickResult block_pick(const uint32_t *bins, int nbins, uint32_t rank, uint32_t *scratch /*[NT+4]*/) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per = nbins >= NT ? nbins / NT : 1;
+    const int active = nbins / per;
+    uint32_t mine = 0;
+    if (tid < active)
+        for (int q = 0; q < per; ++q) mine += bins[tid * per + q];
+    // inclusive suffix sum over threads (higher thread = higher bins): shuffles inside a warp,
+    // then the totals of the warps above
+    uint32_t suf = mine;
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const uint32_t up = __shfl_down_sync(0xffffffffu, suf, m);
+        if (lane + m < 32) suf += up;
+    }
+    if (lane == 0) scratch[warp] = suf;  // warp total
+    if (tid == 0) scratch[NT + 3] = 0u;  // found flag
+    __syncthreads();
+    uint32_t above_warps = 0;
+#pragma unroll
+    for (int w = 0; w < NT / 32; ++w)
+        if (w > warp) above_warps += scratch[w];
+    const uint32_t suf_incl = suf + above_warps;
+    const uint32_t suf_excl = suf_incl - mine;
+    if (tid < active && suf_excl < rank && rank <= suf_incl) {
+        uint32_t above = suf_excl;
+        for (int q = per - 1; q >= 0; --q) {
+            uint32_t c = bins[tid * per + q];
+            if (above + c >= rank) {
+                scratch[NT + 0] = (uint32_t)(tid * per + q);
+                scratch[NT + 1] = rank - above;
+                scratch[NT + 2] = above + c;
+                scratch[NT + 3] = 1u;
+                break;
+            }
+            above += c;
+        }
+    }
+    __syncthreads();
+    PickResult r;
+    r.bin = scratch[NT + 0];
+    r.rank_in_bin = scratch[NT + 1];
+    r.count_ge = scratch[NT + 2];
+    r.ok = scratch[NT + 3] != 0u;
+    __syncthreads();
+    return r;
+}
+
+// Exclusive prefix sum of one value per thread over the CTA (shuffles inside warps, warp totals in
+// shared memory); `total` receives the CTA's sum.  Two barriers.
+template <int NT = THREADS>
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t x, uint32_t *warp_tot /*[NT/32]*/, uint32_t &total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = x;
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xffffffffu, inc, m);
+        if (lane >= m) inc += up;
+    }
+    __syncthreads();  // warp_tot may still be read from the previous call
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    uint32_t before = 0;
+    total = 0;
+#pragma unroll
+    for (int w = 0; w < NT / 32; ++w) {
+        if (w < warp) before += warp_tot[w];
+        total += warp_tot[w];
+    }
+    return before + inc - x;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Dense path of one problem whose candidates did not fit the buffer even under a 24-bit prefix (huge
+// groups of equal magnitudes, e.g. mostly-zero rows): the CTA walks the segment itself.
+// ------------------------------------------------------------------------------------------------
+template <typename GT, int NT>
+__device__ void slow_select(const Params &p, const TopkSide &s, int t, int row, uint32_t *sel, uint32_t *bins,
+                            uint32_t *scratch, uint32_t *wa, uint32_t *wb) {
+    constexpr int NW = NT / 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t seg_beg = __ldg(p.seg_off + t);
+    const int64_t n = __ldg(p.seg_off + t + 1) - seg_beg;
+    const GT *src = reinterpret_cast<const GT *>(s.src) + (int64_t)row * s.row_stride + seg_beg;
+    uint32_t rank = sel[SEL_REMAIN];
+    uint32_t prefix24;
+    const uint32_t flags = sel[SEL_FLAGS];
+    if (flags & 2u) {
+        prefix24 = sel[SEL_PREFIX];  // found by the dense second-digit pass
+    } else {
+        const uint32_t b1 = sel[SEL_PREFIX];
+        for (int b = threadIdx.x; b < DIGIT1_BINS; b += NT) bins[b] = 0u;
+        __syncthreads();
+        for (int64_t j = threadIdx.x; j < n; j += NT) {
+            const uint32_t key = key_of(load1(src + j));
+            if ((key >> DIGIT1_SHIFT) == b1) atomicAdd(&bins[(key >> 7) & 0xfffu], 1u);
+        }
+        __syncthreads();
+        const PickResult r2 = block_pick<NT>(bins, DIGIT1_BINS, rank, scratch);
+        if (!r2.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
+        prefix24 = (b1 << 12) | r2.bin;
+        rank = r2.rank_in_bin;
+    }
+    // last 7 bits
+    for (int b = threadIdx.x; b < NT; b += NT) bins[b] = 0u;
+    __syncthreads();
+    for (int64_t j = threadIdx.x; j < n; j += NT) {
+        const uint32_t key = key_of(load1(src + j));
+        if ((key >> 7) == prefix24) atomicAdd(&bins[key & 0x7fu], 1u);
+    }
+    __syncthreads();
+    const PickResult r = block_pick<NT>(bins, NT, rank, scratch);
+    if (!r.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
+    const uint32_t T = (prefix24 << 7) | r.bin;
+    const uint32_t ties_wanted = r.rank_in_bin;
+    __syncthreads();
+    if (threadIdx.x == 0) { sel[SEL_THRESH] = T; sel[SEL_TIES] = ties_wanted; }
+    // ordered compaction over the dense segment
+    const int first_tile = __ldg(p.tile_prefix + t);
+    const uint32_t kbeg = (uint32_t)__ldg(p.k_off + t), k = (uint32_t)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
+    const int64_t obase = (int64_t)row * p.K + kbeg;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    uint32_t run_sel = 0, run_tie = 0;
+    for (int64_t j0 = 0; j0 < n; j0 += NT) {
+        if ((j0 % TILE) == 0 && threadIdx.x == 0)
+            s.outbase[(int64_t)row * (p.TT + 1) + first_tile + (int)(j0 / TILE)] = kbeg + run_sel;
+        const int64_t j = j0 + threadIdx.x;
+        const bool in = j < n;
+        const float val = in ? load1(src + j) : 0.0f;
+        const uint32_t key = key_of(val);
+        const bool tie = in && key == T;
+        const uint32_t tb = __ballot_sync(0xffffffffu, tie);
+        if (lane == 0) wa[warp] = __popc(tb);
+        __syncthreads();
+        uint32_t tie_rank = run_tie + __popc(tb & lt_mask), tie_tot = 0;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) { if (w < warp) tie_rank += wa[w]; tie_tot += wa[w]; }
+        const bool take = in && (key > T || (tie && tie_rank < ties_wanted));
+        const uint32_t sb = __ballot_sync(0xffffffffu, take);
+        if (lane == 0) wb[warp] = __popc(sb);
+        __syncthreads();
+        uint32_t out = run_sel + __popc(sb & lt_mask), sel_tot = 0;
+#pragma unroll
+        for (int w = 0; w < NW; ++w) { if (w < warp) out += wb[w]; sel_tot += wb[w]; }
+        if (take && out >= k) {
+            atomicOr(p.status, STATUS_COUNT_MISMATCH);
+        } else if (take) {
+            const uint32_t flat = (uint32_t)(seg_beg + j);
+            s.idx[obase + out] = flat;
+            s.val[obase + out] = val;
+            if (tie && tie_rank == ties_wanted - 1) sel[SEL_CUT] = flat;
+        }
+        run_sel += sel_tot;
+        run_tie += tie_tot;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0 && run_sel != k) atomicOr(p.status, STATUS_COUNT_MISMATCH);
+    // downlink: selected entries of the error become +0 (after every read of the segment is done)
+    if (s.zero_out) {
+        __syncthreads();
+        for (uint32_t q = threadIdx.x; q < k; q += NT) s.zero_out[s.idx[obase + q]] = 0.0f;
+    }
+}
+
+// one launch each (defined in topk_tail.cu)
+cudaError_t launch_topk_small(const Params &p, const TopkSide &s, bool bf16, cudaStream_t st);
+cudaError_t launch_topk_check(const Params &p, const TopkSide &s, cudaStream_t st);
+cudaError_t launch_topk_tail(const Params &p, const TopkSide &s, bool bf16, cudaStream_t st);
+
+// Limits of the one-CTA-per-problem tail: candidates of one segment that it sweeps, tiles of one
+// segment that its shared-memory tables hold.  Beyond either, the same steps run as wide launches.
+constexpr int64_t TAIL_MAX_CAND = 1 << 17;
+constexpr int TAIL_MAX_TILES = 1024;
+inline bool use_fused_tail(const Params &p) { return p.cap_max <= TAIL_MAX_CAND && p.max_seg_tiles <= TAIL_MAX_TILES; }
+
+}  // namespace liec

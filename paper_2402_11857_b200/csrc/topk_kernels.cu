@@ -2,7 +2,9 @@
 // ties broken toward the lower index, output (index, value) compacted in ascending index.
 //
 // One selection "problem" is a (row, segment) pair; the uplink has N rows (the workers'
-// gradients), the downlink one row (v, held in the error buffer).  Regular route per side:
+// gradients), the downlink one row (v, held in the error buffer).  A segment of a single tile is
+// selected directly by one CTA (topk_small_kernel) and takes no part in what follows.  Regular
+// route per side, for the other segments:
 //
 //   hist1   dense pass 1: histogram of the first key digit (bits 30..19) per problem
 //           (for the downlink after a top-k uplink it is fused into the server pass)
@@ -11,152 +13,25 @@
 //           buffer: dense second-digit histogram, 24-bit prefix
 //   filter  dense pass 2: entries at or above the prefix appended, in index order inside each
 //           tile, to the problem's region of the candidate buffer
-//   finish  per problem, on its candidates: second digit and last 7 bits -> exact threshold key
-//           and the number of ties to accept
-//   count   per tile block: entries above the threshold and entries equal to it
-//   scan    per problem: first output slot and accepted ties of every tile
-//   write   ordered compaction into (idx, val); records the last accepted tie
-//   slow    one CTA per problem, only when even the 24-bit prefix leaves too many candidates
-//           (huge groups of equal magnitudes, e.g. mostly-zero rows): same result, dense passes
+//   tail    one CTA per problem, on its candidates: remaining digits -> exact threshold key and
+//           the number of ties to accept -> per-tile counts -> output offsets -> ordered
+//           compaction into (idx, val) (topk_tail_kernel).  When a segment has more candidates or
+//           tiles than one CTA is given, the same steps run as wide launches instead:
+//           cand_hist + pick (levels 2, 3), count, scan, write, slow.
 //
-// The uplink first tries a single-pass route (begin, filter with a guess, cand_hist, pick 5),
-// described at topk_begin_kernel.
+// The uplink first tries a single-pass route: filter with a guess (a lower bound taken from the
+// previous step's threshold), check (did the guess hold?), and straight to the tail; a problem whose
+// guess fails, or that has none, takes the regular route in the same step.  The result never
+// depends on the guess.
 //
 // Nothing waits on another CTA; cross-CTA order comes from kernel boundaries.
 #include <type_traits>
 
 #include "device_common.cuh"
 #include "kernels.h"
+#include "topk_common.cuh"
 
 namespace liec {
-
-struct TopkSide {
-    const void *src;      // rows of the vector being compressed
-    int64_t row_stride;   // elements between rows (d for the uplink, 0 for the single downlink row)
-    int R;                // rows
-    uint32_t *idx; float *val;            // [R][K] output message
-    uint32_t *hist, *hist2, *sel;         // [R][T][...]
-    uint32_t *cand_idx; float *cand_val;  // [R][CAP]
-    uint32_t *meta;                        // [R][TT][4]: pos, cnt, n_greater -> unused, ties allowed
-    uint32_t *outbase;                     // [R][TT+1]
-    float *zero_out;                       // downlink: error buffer, selected entries become +0
-    int spec;                              // uplink: try last step's threshold first (single dense pass)
-};
-
-static TopkSide make_side(const Params &p, bool uplink) {
-    TopkSide s;
-    if (uplink) {
-        s.src = p.G; s.row_stride = p.d; s.R = p.N;
-        s.idx = p.up_idx; s.val = p.up_val; s.hist = p.up_hist; s.hist2 = p.up_hist2; s.sel = p.up_sel;
-        s.cand_idx = p.up_cand_idx; s.cand_val = p.up_cand_val; s.meta = p.up_tile_meta; s.outbase = p.up_outbase;
-        s.zero_out = nullptr;
-        s.spec = 1;
-    } else {
-        s.src = p.e; s.row_stride = 0; s.R = 1;
-        s.idx = p.down_idx; s.val = p.down_val; s.hist = p.down_hist; s.hist2 = p.down_hist2; s.sel = p.down_sel;
-        s.cand_idx = p.down_cand_idx; s.cand_val = p.down_cand_val; s.meta = p.down_tile_meta; s.outbase = p.down_outbase;
-        s.zero_out = p.e;
-        s.spec = 0;
-    }
-    return s;
-}
-
-__device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) & 0x7fffffffu; }
-
-enum { STATUS_PICK_RANK = 1, STATUS_CAND_OVERFLOW = 2, STATUS_COUNT_MISMATCH = 4 };
-
-// Adds a CTA's shared-memory histogram to the problem's global one and widens the problem's
-// record of the non-empty bin range, so that the pick reads and clears only that range.
-__device__ __forceinline__ void flush_hist(const uint32_t *h, uint32_t *gh, uint32_t *sel, int lo_word, int hi_word) {
-    uint32_t lo = 0xffffffffu, hi = 0u;
-    for (uint32_t b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) {
-        const uint32_t c = h[b];
-        if (c) {
-            atomicAdd(gh + b, c);
-            lo = min(lo, b);
-            hi = max(hi, b);
-        }
-    }
-    lo = __reduce_min_sync(0xffffffffu, lo);
-    hi = __reduce_max_sync(0xffffffffu, hi);
-    if ((threadIdx.x & 31) == 0 && lo != 0xffffffffu) {
-        atomicMin(&sel[lo_word], lo);
-        atomicMax(&sel[hi_word], hi);
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// Block helper: bins[0..nbins) in shared memory, find the bin that holds the rank-th largest
-// entry counting from the top bin down.  All threads get (bin, rank inside bin, count above+bin).
-// ------------------------------------------------------------------------------------------------
-struct PickResult { uint32_t bin, rank_in_bin, count_ge; bool ok; };
-
-__device__ PickResult block_pick(const uint32_t *bins, int nbins, uint32_t rank, uint32_t *scratch /*[THREADS+4]*/) {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int per = nbins >= THREADS ? nbins / THREADS : 1;
-    const int active = nbins / per;
-    uint32_t mine = 0;
-    if (tid < active)
-        for (int q = 0; q < per; ++q) mine += bins[tid * per + q];
-    // inclusive suffix sum over threads (higher thread = higher bins): shuffles inside a warp,
-    // then the totals of the warps above
-    uint32_t suf = mine;
-#pragma unroll
-    for (int m = 1; m < 32; m <<= 1) {
-        const uint32_t up = __shfl_down_sync(0xffffffffu, suf, m);
-        if (lane + m < 32) suf += up;
-    }
-    if (lane == 0) scratch[warp] = suf;  // warp total
-    if (tid == 0) scratch[THREADS + 3] = 0u;  // found flag
-    __syncthreads();
-    uint32_t above_warps = 0;
-#pragma unroll
-    for (int w = 0; w < THREADS / 32; ++w)
-        if (w > warp) above_warps += scratch[w];
-    const uint32_t suf_incl = suf + above_warps;
-    const uint32_t suf_excl = suf_incl - mine;
-    if (tid < active && suf_excl < rank && rank <= suf_incl) {
-        uint32_t above = suf_excl;
-        for (int q = per - 1; q >= 0; --q) {
-            uint32_t c = bins[tid * per + q];
-            if (above + c >= rank) {
-                scratch[THREADS + 0] = (uint32_t)(tid * per + q);
-                scratch[THREADS + 1] = rank - above;
-                scratch[THREADS + 2] = above + c;
-                scratch[THREADS + 3] = 1u;
-                break;
-            }
-            above += c;
-        }
-    }
-    __syncthreads();
-    PickResult r;
-    r.bin = scratch[THREADS + 0];
-    r.rank_in_bin = scratch[THREADS + 1];
-    r.count_ge = scratch[THREADS + 2];
-    r.ok = scratch[THREADS + 3] != 0u;
-    __syncthreads();
-    return r;
-}
-
-// ------------------------------------------------------------------------------------------------
-// Uplink, start of a step: a problem that has a guess (a lower bound for its threshold, taken
-// from the previous step) first tries the single-pass route: candidates are collected with the
-// guess and everything else runs on the candidates.  The guess is only a shortcut: it is
-// checked (at least k candidates, buffer not exceeded) and a problem that fails the check, or
-// has no guess, takes the regular two-pass route in the same step.  The result is the same.
-// ------------------------------------------------------------------------------------------------
-__global__ void topk_begin_kernel(const __grid_constant__ Params p, const TopkSide s) {
-    const int t = blockIdx.x * blockDim.x + threadIdx.x, row = blockIdx.y;
-    if (t >= p.T) return;
-    uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
-    const bool guess = sel[SEL_GUESS] != 0u;
-    sel[SEL_MODE] = guess ? 1u : 0u;
-    sel[SEL_SPEC_FAIL] = 0u;
-    sel[SEL_CAND_COUNT] = 0u;
-    sel[SEL_FLAGS] = 0u;
-    if (!guess) p.status[STATUS_ANY_REGULAR] = 1;
-}
 
 // ------------------------------------------------------------------------------------------------
 // hist1: one CTA per (tile, row)
@@ -180,6 +55,7 @@ __global__ void __launch_bounds__(THREADS) topk_hist1_kernel(const __grid_consta
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int tile = blockIdx.x; tile < p.TT; tile += gridDim.x) {
         const TileInfo ti = locate_tile(p, tile);
+        if (ti.seg_tiles == 1) continue;              // selected directly by one CTA
         uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
         if (s.spec && sel[SEL_MODE] != 0u) continue;  // uniform over the CTA
         const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
@@ -213,23 +89,17 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
     __shared__ uint32_t scratch[THREADS + 4];
     const int t = blockIdx.x, row = blockIdx.y;
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
+    if (level == 4 && t == 0 && row == 0 && threadIdx.x == 0) p.status[STATUS_ANY_REFINE + (s.zero_out ? 1 : 0)] = 0;
+    if (__ldg(p.tile_prefix + t + 1) - __ldg(p.tile_prefix + t) == 1) return;   // selected directly by one CTA
     // level 1: first digit from the dense histogram (regular route).
     // level 5: first digit from the histogram of the candidates collected with the guess
     //          (uplink single-pass route); checks the guess.
     // level 4: second digit of "refined" problems, after their dense second-digit pass.
     // levels 2, 3: wide form of the finish step (second digit, last 7 bits) from candidate histograms.
-    if (level == 5) {
-        if (sel[SEL_MODE] != 1u) return;
-        if (sel[SEL_SPEC_FAIL] != 0u) {  // the guess let too much through: regular route (nothing was added to the histogram)
-            __syncthreads();             // every thread has read the mode before it changes
-            if (threadIdx.x == 0) { sel[SEL_MODE] = 0u; p.status[STATUS_ANY_REGULAR] = 1; }
-            return;
-        }
-    }
+    if (level == 5 && sel[SEL_MODE] != 1u) return;
     if (level == 2 && sel[SEL_FLAGS] != 0u) return;
     if (level == 3 && (sel[SEL_FLAGS] & 1u)) return;
     if (level == 1 && s.spec && sel[SEL_MODE] != 0u) return;
-    if (level == 4 && t == 0 && row == 0 && threadIdx.x == 0) p.status[STATUS_ANY_REFINE + (s.zero_out ? 1 : 0)] = 0;
     if (level == 4 && sel[SEL_FLAGS] != 2u) return;
     const bool first = level == 1 || level == 5;
     uint32_t *gh = (first ? s.hist : s.hist2) + ((int64_t)row * p.T + t) * DIGIT1_BINS;
@@ -249,19 +119,14 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
     const uint32_t rank = first ? k : sel[SEL_REMAIN];
     const PickResult r = block_pick(bins, DIGIT1_BINS, rank, scratch);
     if (threadIdx.x != 0) return;
-    if (level == 5) {
-        if (!r.ok) {  // fewer than k candidates: the guess was too high, take the regular route
-            sel[SEL_MODE] = 0u;
-            p.status[STATUS_ANY_REGULAR] = 1;
-        } else {
-            sel[SEL_PREFIX] = r.bin;
-            sel[SEL_REMAIN] = r.rank_in_bin;
-            sel[SEL_ABOVE] = r.count_ge - bins[r.bin];
-            sel[SEL_NCAND] = sel[SEL_CAND_COUNT];
-        }
+    if (!r.ok) { atomicOr(p.status, STATUS_PICK_RANK); return; }
+    if (level == 5) {   // (the check kernel has made sure that there are at least k candidates)
+        sel[SEL_PREFIX] = r.bin;
+        sel[SEL_REMAIN] = r.rank_in_bin;
+        sel[SEL_ABOVE] = r.count_ge - bins[r.bin];
+        sel[SEL_NCAND] = sel[SEL_CAND_COUNT];
         return;
     }
-    if (!r.ok) { atomicOr(p.status, STATUS_PICK_RANK); return; }
     const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
     if (level == 2) {
         sel[SEL_PREFIX] = (sel[SEL_PREFIX] << 12) | r.bin;
@@ -332,29 +197,6 @@ __global__ void __launch_bounds__(THREADS) topk_hist2_dense_kernel(const __grid_
 // ------------------------------------------------------------------------------------------------
 // filter: one CTA per (tile, row); ordered append of candidates
 // ------------------------------------------------------------------------------------------------
-// Exclusive prefix sum of one value per thread over the CTA (shuffles inside warps, warp totals in
-// shared memory); `total` receives the CTA's sum.  Two barriers.
-__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t x, uint32_t *warp_tot /*[8]*/, uint32_t &total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t inc = x;
-#pragma unroll
-    for (int m = 1; m < 32; m <<= 1) {
-        const uint32_t up = __shfl_up_sync(0xffffffffu, inc, m);
-        if (lane >= m) inc += up;
-    }
-    __syncthreads();  // warp_tot may still be read from the previous call
-    if (lane == 31) warp_tot[warp] = inc;
-    __syncthreads();
-    uint32_t before = 0;
-    total = 0;
-#pragma unroll
-    for (int w = 0; w < THREADS / 32; ++w) {
-        if (w < warp) before += warp_tot[w];
-        total += warp_tot[w];
-    }
-    return before + inc - x;
-}
-
 // ------------------------------------------------------------------------------------------------
 // filter: the tile is staged through shared memory by one TMA bulk copy.
 //
@@ -390,14 +232,16 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
     uint32_t phase = 0;
     for (int tile = blockIdx.x; tile < p.TT; tile += gridDim.x) {
         const TileInfo ti = locate_tile(p, tile);
+        if (ti.seg_tiles == 1) continue;   // selected directly by one CTA
         uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
         float low;
         if (SPEC) {
             // (uniform over the CTA, like every `continue` before the barriers: no kernel writes, in the
             // launch in which it runs, a word that it branches on; a guess that fails is recorded in
             // SEL_SPEC_FAIL, which only later launches read)
-            if (sel[SEL_MODE] != 1u) continue;
-            low = __uint_as_float(sel[SEL_GUESS]);
+            const uint32_t guess = sel[SEL_GUESS];
+            if (guess == 0u) continue;
+            low = __uint_as_float(guess);
         } else {
             if (s.spec && sel[SEL_MODE] != 0u) continue;
             const uint32_t flags = sel[SEL_FLAGS];
@@ -505,7 +349,7 @@ __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide 
     cb.t = ti.t;
     cb.sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
     cb.meta = s.meta + ((int64_t)row * p.TT + tile) * 4;
-    cb.skip = (cb.sel[SEL_FLAGS] & 1u) != 0u;
+    cb.skip = (cb.sel[SEL_FLAGS] & 1u) != 0u || ti.seg_tiles == 1;
     cb.cnt = cb.skip ? 0u : cb.meta[1];
     cb.base = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + cb.meta[0];
     return cb;
@@ -545,8 +389,7 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
         if (active) {
             cb = cand_block(p, s, tile, row);
             const uint32_t flags = cb.sel[SEL_FLAGS];
-            active = !cb.skip && !(level == 0 && (cb.sel[SEL_MODE] != 1u || cb.sel[SEL_SPEC_FAIL] != 0u)) &&
-                     !(level == 1 && flags != 0u);
+            active = !cb.skip && !(level == 0 && cb.sel[SEL_MODE] != 1u) && !(level == 1 && flags != 0u);
             prefix = cb.sel[SEL_PREFIX];
         }
         uint32_t lo = 0xffffffffu, hi = 0u;
@@ -607,57 +450,6 @@ __global__ void __launch_bounds__(THREADS) topk_count_kernel(const __grid_consta
     if (lane == 0) { cb.meta[2] = g; cb.meta[3] = e; }
 }
 
-// finish: one CTA per (segment, row).  The first digit (or, for refined problems, the 24-bit
-// prefix) of the threshold is known and the problem's candidates sit in one contiguous region of
-// the candidate buffer (a few per cent of the segment, cache resident): two sweeps over that
-// region with shared-memory histograms (second digit, then the last 7 bits) give the exact
-// threshold key and the number of ties to accept.
-__global__ void __launch_bounds__(THREADS) topk_finish_kernel(const __grid_constant__ Params p, const TopkSide s) {
-    __shared__ __align__(16) uint32_t bins[DIGIT1_BINS];
-    __shared__ uint32_t scratch[THREADS + 4];
-    const int t = blockIdx.x, row = blockIdx.y;
-    uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
-    const uint32_t flags = sel[SEL_FLAGS];
-    if (flags & 1u) return;  // slow path finishes on its own
-    const float *cand = s.cand_val + (int64_t)row * p.CAP + __ldg(p.cap_off + t);
-    const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
-    const uint32_t ncand = min(sel[SEL_CAND_COUNT], cap);  // (the cursor can run past the buffer when a tile was refused)
-    uint32_t prefix24 = sel[SEL_PREFIX];
-    uint32_t rank = sel[SEL_REMAIN];
-    if (!(flags & 2u)) {
-        const uint32_t b1 = prefix24;
-        for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(bins)[b] = make_uint4(0u, 0u, 0u, 0u);
-        __syncthreads();
-        for (uint32_t q = threadIdx.x; q < ncand; q += THREADS) {
-            const uint32_t key = key_of(cand[q]);
-            if ((key >> DIGIT1_SHIFT) == b1) atomicAdd(&bins[(key >> 7) & 0xfffu], 1u);
-        }
-        __syncthreads();
-        const PickResult r2 = block_pick(bins, DIGIT1_BINS, rank, scratch);
-        if (!r2.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
-        prefix24 = (b1 << 12) | r2.bin;
-        rank = r2.rank_in_bin;
-    }
-    if (threadIdx.x < 128) bins[threadIdx.x] = 0u;
-    __syncthreads();
-    for (uint32_t q = threadIdx.x; q < ncand; q += THREADS) {
-        const uint32_t key = key_of(cand[q]);
-        if ((key >> 7) == prefix24) atomicAdd(&bins[key & 0x7fu], 1u);
-    }
-    __syncthreads();
-    const PickResult r3 = block_pick(bins, 128, rank, scratch);
-    if (!r3.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
-    if (threadIdx.x == 0) {
-        const uint32_t thresh = (prefix24 << 7) | r3.bin;
-        sel[SEL_THRESH] = thresh;
-        sel[SEL_TIES] = r3.rank_in_bin;
-        if (s.spec) {  // next step's guess: one first-digit bin below this threshold's bin
-            const uint32_t b1 = thresh >> DIGIT1_SHIFT;
-            sel[SEL_GUESS] = (flags == 0u && b1 >= 1u) ? (b1 - 1u) << DIGIT1_SHIFT : 0u;
-        }
-    }
-}
-
 // scan: one CTA per (segment, row); tiles of the segment in order
 __global__ void __launch_bounds__(THREADS) topk_scan_kernel(const __grid_constant__ Params p, const TopkSide s) {
     __shared__ uint32_t warp_tot[8];
@@ -666,6 +458,7 @@ __global__ void __launch_bounds__(THREADS) topk_scan_kernel(const __grid_constan
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
     if (sel[SEL_FLAGS] & 1u) return;
     const int first = __ldg(p.tile_prefix + t), ntiles = __ldg(p.tile_prefix + t + 1) - first;
+    if (ntiles == 1) return;   // selected directly by one CTA
     const uint32_t ties_wanted = sel[SEL_TIES];
     const uint32_t kbeg = (uint32_t)__ldg(p.k_off + t), k = (uint32_t)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
     uint32_t carry_sel = 0, carry_ties = 0;  // uniform over the CTA
@@ -748,7 +541,8 @@ __global__ void __launch_bounds__(THREADS) topk_write_kernel(const __grid_consta
 }
 
 // ------------------------------------------------------------------------------------------------
-// slow path: one CTA per problem whose candidates did not fit.  Dense passes over the segment.
+// Wide form, last kernel of a side: one CTA per problem.  Runs the dense path for problems whose
+// candidates did not fit (slow_select) and closes the step's bookkeeping for every problem.
 // ------------------------------------------------------------------------------------------------
 template <typename GT>
 __global__ void __launch_bounds__(THREADS) topk_slow_kernel(const __grid_constant__ Params p, const TopkSide s) {
@@ -757,90 +551,19 @@ __global__ void __launch_bounds__(THREADS) topk_slow_kernel(const __grid_constan
     __shared__ uint32_t wa[8], wb[8];
     const int t = blockIdx.x, row = blockIdx.y;
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
-    // last kernel of a side: the next step starts with "no problem on the regular route yet"
+    // the next step starts with "no problem on the regular route yet"
     if (s.spec && t == 0 && row == 0 && threadIdx.x == 0) p.status[STATUS_ANY_REGULAR] = 0;
-    if (!(sel[SEL_FLAGS] & 1u)) return;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t seg_beg = __ldg(p.seg_off + t);
-    const int64_t n = __ldg(p.seg_off + t + 1) - seg_beg;
-    const GT *src = reinterpret_cast<const GT *>(s.src) + (int64_t)row * s.row_stride + seg_beg;
-    uint32_t rank = sel[SEL_REMAIN];
-    uint32_t prefix24;
-    if (sel[SEL_FLAGS] & 2u) {
-        prefix24 = sel[SEL_PREFIX];  // found by the dense second-digit pass
-    } else {
-        const uint32_t b1 = sel[SEL_PREFIX];
-        for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) bins[b] = 0u;
-        __syncthreads();
-        for (int64_t j = threadIdx.x; j < n; j += THREADS) {
-            const uint32_t key = key_of(load1(src + j));
-            if ((key >> DIGIT1_SHIFT) == b1) atomicAdd(&bins[(key >> 7) & 0xfffu], 1u);
-        }
-        __syncthreads();
-        PickResult r2 = block_pick(bins, DIGIT1_BINS, rank, scratch);
-        if (!r2.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
-        prefix24 = (b1 << 12) | r2.bin;
-        rank = r2.rank_in_bin;
-    }
-    PickResult r;
-    // last 7 bits
-    for (int b = threadIdx.x; b < 128; b += THREADS) bins[b] = 0u;
+    if (__ldg(p.tile_prefix + t + 1) - __ldg(p.tile_prefix + t) == 1) return;   // selected directly by one CTA
+    const uint32_t flags = sel[SEL_FLAGS];
+    const bool single = s.spec && sel[SEL_MODE] == 1u;
     __syncthreads();
-    for (int64_t j = threadIdx.x; j < n; j += THREADS) {
-        const uint32_t key = key_of(load1(src + j));
-        if ((key >> 7) == prefix24) atomicAdd(&bins[key & 0x7fu], 1u);
+    if (threadIdx.x == 0) {
+        sel[SEL_CAND_COUNT] = 0u;
+        sel[SEL_SPEC_FAIL] = 0u;
+        sel[SEL_ROUTE] = (single ? ROUTE_SINGLE : 0) | ((flags & 2u) ? ROUTE_REFINED : 0) | ((flags & 1u) ? ROUTE_SLOW : 0);
     }
-    __syncthreads();
-    r = block_pick(bins, 128, rank, scratch);
-    if (!r.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
-    const uint32_t T = (prefix24 << 7) | r.bin;
-    const uint32_t ties_wanted = r.rank_in_bin;
-    if (threadIdx.x == 0) { sel[SEL_THRESH] = T; sel[SEL_TIES] = ties_wanted; }
-    // ordered compaction over the dense segment
-    const int first_tile = __ldg(p.tile_prefix + t);
-    const uint32_t kbeg = (uint32_t)__ldg(p.k_off + t), k = (uint32_t)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
-    const int64_t obase = (int64_t)row * p.K + kbeg;
-    const uint32_t lt_mask = (1u << lane) - 1u;
-    uint32_t run_sel = 0, run_tie = 0;
-    for (int64_t j0 = 0; j0 < n; j0 += THREADS) {
-        if ((j0 % TILE) == 0 && threadIdx.x == 0)
-            s.outbase[(int64_t)row * (p.TT + 1) + first_tile + (int)(j0 / TILE)] = kbeg + run_sel;
-        const int64_t j = j0 + threadIdx.x;
-        const bool in = j < n;
-        const float val = in ? load1(src + j) : 0.0f;
-        const uint32_t key = key_of(val);
-        const bool tie = in && key == T;
-        const uint32_t tb = __ballot_sync(0xffffffffu, tie);
-        if (lane == 0) wa[warp] = __popc(tb);
-        __syncthreads();
-        uint32_t tie_rank = run_tie + __popc(tb & lt_mask), tie_tot = 0;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) { if (w < warp) tie_rank += wa[w]; tie_tot += wa[w]; }
-        const bool take = in && (key > T || (tie && tie_rank < ties_wanted));
-        const uint32_t sb = __ballot_sync(0xffffffffu, take);
-        if (lane == 0) wb[warp] = __popc(sb);
-        __syncthreads();
-        uint32_t out = run_sel + __popc(sb & lt_mask), sel_tot = 0;
-#pragma unroll
-        for (int w = 0; w < 8; ++w) { if (w < warp) out += wb[w]; sel_tot += wb[w]; }
-        if (take && out >= k) {
-            atomicOr(p.status, STATUS_COUNT_MISMATCH);
-        } else if (take) {
-            const uint32_t flat = (uint32_t)(seg_beg + j);
-            s.idx[obase + out] = flat;
-            s.val[obase + out] = val;
-            if (tie && tie_rank == ties_wanted - 1) sel[SEL_CUT] = flat;
-        }
-        run_sel += sel_tot;
-        run_tie += tie_tot;
-        __syncthreads();
-    }
-    if (threadIdx.x == 0 && run_sel != k) atomicOr(p.status, STATUS_COUNT_MISMATCH);
-    // downlink: selected entries of the error become +0 (after every read of the segment is done)
-    if (s.zero_out) {
-        __syncthreads();
-        for (uint32_t q = threadIdx.x; q < k; q += THREADS) s.zero_out[s.idx[obase + q]] = 0.0f;
-    }
+    if (!(flags & 1u)) return;
+    slow_select<GT, THREADS>(p, s, t, row, sel, bins, scratch, wa, wb);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -935,7 +658,7 @@ __global__ void __launch_bounds__(THREADS, 4) server_topk_kernel(const __grid_co
             v[c] = __fadd_rn(ev[j][c], v[c]);
             if (!valid) v[c] = 0.0f;
             if (valid && __float_as_uint(v[c]) != __float_as_uint(ev[j][c])) e_tile[pos + c] = v[c];
-            if (DOWN == COMP_TOPK && valid) atomicAdd(&h[key_of(v[c]) >> DIGIT1_SHIFT], 1u);
+            if (DOWN == COMP_TOPK && valid && ti.seg_tiles > 1) atomicAdd(&h[key_of(v[c]) >> DIGIT1_SHIFT], 1u);
         }
         if (DOWN == COMP_SIGN) {
             a[j] = leaf4(v);
@@ -948,7 +671,7 @@ __global__ void __launch_bounds__(THREADS, 4) server_topk_kernel(const __grid_co
         double sum = cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
         if (threadIdx.x == 0) p.down_partials[blockIdx.x] = sum;
     }
-    if (DOWN == COMP_TOPK) {
+    if (DOWN == COMP_TOPK && ti.seg_tiles > 1) {   // (single-tile segments are selected directly from v)
         __syncthreads();
         flush_hist(h, p.down_hist + (int64_t)ti.t * DIGIT1_BINS, p.down_sel + (int64_t)ti.t * SEL_WORDS, SEL_LO1, SEL_HI1);
     }
@@ -964,10 +687,6 @@ __global__ void __launch_bounds__(THREADS, 4) server_topk_kernel(const __grid_co
         ++*launches;                                     \
     } while (0)
 
-// Largest per-segment candidate capacity that the one-CTA finish kernel handles (two sweeps over
-// that many cached values by 256 threads); beyond it the finish step runs as four wide launches.
-constexpr int64_t FINISH_ONE_CTA_MAX = 1 << 17;
-
 // Grid of the dense passes that usually have nothing to do on the uplink (their CTAs walk the
 // tiles with a stride and leave at once when no problem takes the regular route).
 static dim3 strided_grid(const Params &p, int rows) {
@@ -975,28 +694,39 @@ static dim3 strided_grid(const Params &p, int rows) {
     return dim3(p.TT < per_row ? p.TT : per_row, rows);
 }
 
-// Candidate histograms: 8 tiles per CTA, or 64 where some segment is large enough for the wide
-// finish step (its CTAs then gather in shared memory and flush once per 64 tiles).
-static int cand_hist_reps(const Params &p) { return p.cap_max > FINISH_ONE_CTA_MAX ? 8 : 1; }
+// Candidate histograms of the wide form: 64 tiles per CTA (its CTAs gather in shared memory and
+// flush once per 64 tiles).
+static int cand_hist_reps(const Params &) { return 8; }
 static dim3 cand_hist_grid(const Params &p, int rows) {
     const int per = 8 * cand_hist_reps(p);
     return dim3((p.TT + per - 1) / per, rows);
 }
 
-// First dense pass.  Uplink: collect candidates with last step's guess, histogram them and
-// check the guess; then the first-digit histogram for the problems left on the regular route.
-// Downlink without a fused histogram: plain first-digit histogram of v.
+// First part of a side.  Single-tile segments are selected directly.  Uplink: candidates are
+// collected with last step's guess and the guess is checked; then, for the problems left on the
+// regular route, the first-digit histogram.  Downlink without a fused histogram: plain first-digit
+// histogram of v.
 cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int64_t *launches) {
     const TopkSide s = make_side(p, uplink);
-    dim3 g_tiles(p.TT, s.R), g_probs(p.T, s.R), g_warp_tiles((p.TT + 7) / 8, s.R);
+    dim3 g_tiles(p.TT, s.R), g_probs(p.T, s.R);
     const bool bf = uplink && p.gdt == DT_BF16;
+    if (p.n_small) {
+        cudaError_t e = launch_topk_small(p, s, bf, st);
+        if (e != cudaSuccess) return e;
+        ++*launches;
+    }
+    if (!p.n_large) return cudaSuccess;
     if (s.spec) {
-        topk_begin_kernel<<<dim3((p.T + 127) / 128, s.R), 128, 0, st>>>(p, s); CHECK_LAUNCH();
         if (bf) topk_filter_tma_kernel<__nv_bfloat16, true><<<g_tiles, THREADS, 0, st>>>(p, s);
         else topk_filter_tma_kernel<float, true><<<g_tiles, THREADS, 0, st>>>(p, s);
         CHECK_LAUNCH();
-        topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 0, cand_hist_reps(p)); CHECK_LAUNCH();
-        topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 5); CHECK_LAUNCH();
+        cudaError_t e = launch_topk_check(p, s, st);
+        if (e != cudaSuccess) return e;
+        ++*launches;
+        if (!use_fused_tail(p)) {   // wide form: first digit of the single-pass problems from a global histogram
+            topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 0, cand_hist_reps(p)); CHECK_LAUNCH();
+            topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 5); CHECK_LAUNCH();
+        }
     }
     const dim3 g_hist = s.spec ? strided_grid(p, s.R) : g_tiles;
     if (bf) topk_hist1_kernel<__nv_bfloat16><<<g_hist, THREADS, 0, st>>>(p, s);
@@ -1006,11 +736,18 @@ cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int
 }
 
 // Everything after the first-digit histogram: the message, the thresholds, and for the
-// downlink the zeroing of the selected error entries.
-cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, int64_t *launches) {
+// downlink the zeroing of the selected error entries.  (When the downlink's histogram is fused
+// into the server pass this is the whole downlink, so the single-tile segments are selected here.)
+cudaError_t launch_topk_select(const Params &p, bool uplink, bool small_done, cudaStream_t st, int64_t *launches) {
     const TopkSide s = make_side(p, uplink);
     dim3 g_tiles(p.TT, s.R), g_probs(p.T, s.R), g_warp_tiles((p.TT + 7) / 8, s.R);
     const bool bf = uplink && p.gdt == DT_BF16;
+    if (p.n_small && !small_done) {
+        cudaError_t e = launch_topk_small(p, s, bf, st);
+        if (e != cudaSuccess) return e;
+        ++*launches;
+    }
+    if (!p.n_large) return cudaSuccess;
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 1); CHECK_LAUNCH();
     if (bf) topk_hist2_dense_kernel<__nv_bfloat16><<<strided_grid(p, s.R), THREADS, 0, st>>>(p, s);
     else topk_hist2_dense_kernel<float><<<strided_grid(p, s.R), THREADS, 0, st>>>(p, s);
@@ -1020,14 +757,17 @@ cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, in
     if (bf) topk_filter_tma_kernel<__nv_bfloat16, false><<<g_filter, THREADS, 0, st>>>(p, s);
     else topk_filter_tma_kernel<float, false><<<g_filter, THREADS, 0, st>>>(p, s);
     CHECK_LAUNCH();
-    if (p.cap_max <= FINISH_ONE_CTA_MAX) {
-        topk_finish_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
-    } else {  // some segment has too many candidates for one CTA: the same two steps, spread over the tile blocks
-        topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 1, cand_hist_reps(p)); CHECK_LAUNCH();
-        topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();
-        topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 2, cand_hist_reps(p)); CHECK_LAUNCH();
-        topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 3); CHECK_LAUNCH();
+    if (use_fused_tail(p)) {
+        cudaError_t e = launch_topk_tail(p, s, bf, st);
+        if (e != cudaSuccess) return e;
+        ++*launches;
+        return cudaSuccess;
     }
+    // some segment has too many candidates or tiles for one CTA: the same steps, spread over the tile blocks
+    topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 1, cand_hist_reps(p)); CHECK_LAUNCH();
+    topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();
+    topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 2, cand_hist_reps(p)); CHECK_LAUNCH();
+    topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 3); CHECK_LAUNCH();
     topk_count_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     topk_scan_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     topk_write_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();

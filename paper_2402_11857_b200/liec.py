@@ -243,12 +243,13 @@ class Context:
 
     def liec_topk_route_counts(self, uplink: bool, stream=None, per_problem: bool = False) -> dict:
         """Counts of the routes taken by the last iteration's selections; with per_problem also a uint8
-        array [rows, T] of flags (1 single pass, 2 second-digit pass, 4 one-CTA path)."""
-        out = (C.c_int64 * 4)()
+        array [rows, T] of flags (1 single pass, 2 second-digit pass, 4 dense one-CTA path, 8 single tile)."""
+        out = (C.c_int64 * 5)()
         flags = np.zeros(((self.N if uplink else 1), self.T), np.uint8) if per_problem else None
         self._check(self.lib.liec_topk_route_counts(self._ctx, self._stream(stream), 1 if uplink else 0, out,
                                                     None if flags is None else flags.ctypes.data_as(C.c_void_p)))
-        r = {"problems": int(out[0]), "single_pass": int(out[1]), "refined": int(out[2]), "slow": int(out[3])}
+        r = {"problems": int(out[0]), "single_pass": int(out[1]), "refined": int(out[2]), "slow": int(out[3]),
+             "direct": int(out[4])}
         if flags is not None:
             r["flags"] = flags
         return r

@@ -97,5 +97,6 @@ def test_bulk_copy_wait_runs_out_sign_bf16():
 
 
 def test_bulk_copy_wait_runs_out_topk_filter():
-    G = make_gradients("normal", 1.0, 1, 8192, 0, base_seed=75)
-    _flagged_then_recovers(lambda: Pair(1, [0, 8192], TOPK, TOPK, k=[81]), G, 0.1)
+    """Two full tiles of one segment (a single-tile segment would be selected without any bulk copy)."""
+    G = make_gradients("normal", 1.0, 1, 16384, 0, base_seed=75)
+    _flagged_then_recovers(lambda: Pair(1, [0, 16384], TOPK, TOPK, k=[163]), G, 0.1)
