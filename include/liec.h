@@ -37,8 +37,12 @@
  *   identity: no message buffer; the dense vector itself.
  *
  * Ownership: the caller owns every device buffer (params, error, gradients, workspace).
- * The library owns only the host-side context.  The hot calls allocate nothing, never
- * synchronise the device and only enqueue work on the given stream.
+ * The library owns only the host-side context (for top-k configurations with segments of at
+ * most 8192 elements also one helper stream and two events, created by liec_init and released
+ * by liec_destroy).  The hot calls allocate nothing, never synchronise the device and only
+ * enqueue work that is ordered on the given stream: a top-k stage may run part of its kernels
+ * on the helper stream, forked from and joined back to the given stream by events inside the
+ * same call (this also works while the given stream is being captured into a CUDA graph).
  *
  * Errors: every call returns a liec_status; nothing throws, aborts or traps the GPU.
  * liec_last_error() gives a message for the last failing call on that context.
@@ -307,7 +311,7 @@ const char *liec_last_error(const liec_ctx *ctx); /* never NULL; ctx may be NULL
 liec_status liec_sign_compress_noalloc(const void *x, int32_t dtype, int64_t n, uint32_t *words,
                                        float *scale, void *stream);
 const char *liec_noalloc_last_error(void); /* message of the last failing no-alloc call on this thread */
-void liec_destroy(liec_ctx *ctx);                  /* frees host memory only */
+void liec_destroy(liec_ctx *ctx);                  /* frees the host-side context (and its helper stream and events) */
 
 #ifdef __cplusplus
 }

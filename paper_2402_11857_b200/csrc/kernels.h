@@ -15,7 +15,8 @@ cudaError_t launch_identity_downlink(const Params &p, cudaStream_t st);
 
 // top-k (launch counters are bumped per kernel)
 cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int64_t *launches);
-cudaError_t launch_topk_select(const Params &p, bool uplink, bool small_done, cudaStream_t st, int64_t *launches);
+cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, int64_t *launches);
+cudaError_t launch_topk_small_segments(const Params &p, bool uplink, cudaStream_t st, int64_t *launches);
 cudaError_t launch_server_topk(const Params &p, cudaStream_t st, int64_t *launches);
 cudaError_t configure_topk_kernels();  // opt-in shared memory sizes; call once per device
 

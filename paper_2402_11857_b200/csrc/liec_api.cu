@@ -195,6 +195,10 @@ struct liec_ctx {
     int stage = 0;  // 0 idle, 1 after uplink, 2 after aggregate, 3 after downlink
     int64_t launches = 0;
     std::string err;
+    // top-k: the single-tile segments are selected on a stream of the context's own, forked from
+    // and joined to the caller's stream by events, so that they overlap the dense passes
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 
 namespace {
@@ -223,6 +227,31 @@ liec_status cuda_fail(liec_ctx *c, cudaError_t e, const char *what) {
     } while (0)
 
 bool aligned16(const void *ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
+
+void release_side(liec_ctx *c) {
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
+    if (c->side) cudaStreamDestroy(c->side);
+    c->ev_fork = c->ev_join = nullptr;
+    c->side = nullptr;
+}
+
+// Top-k side: the single-tile segments on the context's own stream (between a fork after what `s`
+// holds so far and a join that the caller issues with join_side), the rest on `s`.
+liec_status fork_small_segments(liec_ctx *c, bool uplink, cudaStream_t s) {
+    if (!c->side || c->p.n_small == 0) return LIEC_OK;
+    LIEC_CALL(c, cudaEventRecord(c->ev_fork, s));
+    LIEC_CALL(c, cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+    LIEC_CALL(c, launch_topk_small_segments(c->p, uplink, c->side, &c->launches));
+    LIEC_CALL(c, cudaEventRecord(c->ev_join, c->side));
+    return LIEC_OK;
+}
+
+liec_status join_side(liec_ctx *c, cudaStream_t s) {
+    if (!c->side || c->p.n_small == 0) return LIEC_OK;
+    LIEC_CALL(c, cudaStreamWaitEvent(s, c->ev_join, 0));
+    return LIEC_OK;
+}
 
 }  // namespace
 
@@ -353,6 +382,12 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
         }
     }
     cudaError_t e = configure_topk_kernels();
+    if (e == cudaSuccess && c->plan.K > 0 && !c->plan.small_seg.empty()) {
+        e = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
+        if (e != cudaSuccess) release_side(c);
+    }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         snprintf(g_no_ctx_error, sizeof(g_no_ctx_error), "kernel configuration / synchronize failed: %s", cudaGetErrorString(e));
@@ -382,8 +417,10 @@ liec_status liec_uplink_compress(liec_ctx *c, const void *grads, void *stream) {
         LIEC_LAUNCH(c, launch_sign_uplink(c->p, s));
         LIEC_LAUNCH(c, launch_scale_finalize(c->p, true, s));
     } else if (c->p.up == COMP_TOPK) {
+        if ((st = fork_small_segments(c, true, s)) != LIEC_OK) return st;
         LIEC_CALL(c, launch_topk_hist1(c->p, true, s, &c->launches));
-        LIEC_CALL(c, launch_topk_select(c->p, true, true, s, &c->launches));
+        LIEC_CALL(c, launch_topk_select(c->p, true, s, &c->launches));
+        if ((st = join_side(c, s)) != LIEC_OK) return st;
     } else if (c->p.up == COMP_RANDK) {
         if (!c->p.up_sets) { c->err = "random-k uplink: no subsets given (liec_set_subsets)"; return LIEC_ERR_STATE; }
         LIEC_CALL(c, launch_randk_compress(c->p, true, s, &c->launches));
@@ -419,9 +456,10 @@ liec_status liec_downlink_compress(liec_ctx *c, void *stream) {
         LIEC_CALL(c, launch_randk_compress(c->p, false, s, &c->launches));
     } else {
         // the first-digit histogram of v is fused into the server pass after a sparse uplink
-        const bool fused_hist = comp_is_sparse(c->p.up);
-        if (!fused_hist) LIEC_CALL(c, launch_topk_hist1(c->p, false, s, &c->launches));
-        LIEC_CALL(c, launch_topk_select(c->p, false, !fused_hist, s, &c->launches));
+        if ((st = fork_small_segments(c, false, s)) != LIEC_OK) return st;
+        if (!comp_is_sparse(c->p.up)) LIEC_CALL(c, launch_topk_hist1(c->p, false, s, &c->launches));
+        LIEC_CALL(c, launch_topk_select(c->p, false, s, &c->launches));
+        if ((st = join_side(c, s)) != LIEC_OK) return st;
     }
     c->stage = 3;
     return LIEC_OK;
@@ -597,6 +635,10 @@ int64_t liec_launch_count(const liec_ctx *c) { return c ? c->launches : 0; }
 
 const char *liec_last_error(const liec_ctx *c) { return c ? c->err.c_str() : g_no_ctx_error; }
 
-void liec_destroy(liec_ctx *c) { delete c; }
+void liec_destroy(liec_ctx *c) {
+    if (!c) return;
+    release_side(c);
+    delete c;
+}
 
 }  // extern "C"

@@ -235,6 +235,7 @@ __device__ void slow_select(const Params &p, const TopkSide &s, int t, int row, 
 cudaError_t launch_topk_small(const Params &p, const TopkSide &s, bool bf16, cudaStream_t st);
 cudaError_t launch_topk_check(const Params &p, const TopkSide &s, cudaStream_t st);
 cudaError_t launch_topk_tail(const Params &p, const TopkSide &s, bool bf16, cudaStream_t st);
+cudaError_t configure_topk_tail_kernels();
 
 // Limits of the one-CTA-per-problem tail: candidates of one segment that it sweeps, tiles of one
 // segment that its shared-memory tables hold.  Beyond either, the same steps run as wide launches.

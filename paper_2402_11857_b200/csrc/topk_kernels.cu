@@ -702,7 +702,7 @@ static dim3 cand_hist_grid(const Params &p, int rows) {
     return dim3((p.TT + per - 1) / per, rows);
 }
 
-// First part of a side.  Single-tile segments are selected directly.  Uplink: candidates are
+// First part of a side (multi-tile segments).  Uplink: candidates are
 // collected with last step's guess and the guess is checked; then, for the problems left on the
 // regular route, the first-digit histogram.  Downlink without a fused histogram: plain first-digit
 // histogram of v.
@@ -710,11 +710,6 @@ cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int
     const TopkSide s = make_side(p, uplink);
     dim3 g_tiles(p.TT, s.R), g_probs(p.T, s.R);
     const bool bf = uplink && p.gdt == DT_BF16;
-    if (p.n_small) {
-        cudaError_t e = launch_topk_small(p, s, bf, st);
-        if (e != cudaSuccess) return e;
-        ++*launches;
-    }
     if (!p.n_large) return cudaSuccess;
     if (s.spec) {
         if (bf) topk_filter_tma_kernel<__nv_bfloat16, true><<<g_tiles, THREADS, 0, st>>>(p, s);
@@ -736,17 +731,11 @@ cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int
 }
 
 // Everything after the first-digit histogram: the message, the thresholds, and for the
-// downlink the zeroing of the selected error entries.  (When the downlink's histogram is fused
-// into the server pass this is the whole downlink, so the single-tile segments are selected here.)
-cudaError_t launch_topk_select(const Params &p, bool uplink, bool small_done, cudaStream_t st, int64_t *launches) {
+// downlink the zeroing of the selected error entries.
+cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, int64_t *launches) {
     const TopkSide s = make_side(p, uplink);
     dim3 g_tiles(p.TT, s.R), g_probs(p.T, s.R), g_warp_tiles((p.TT + 7) / 8, s.R);
     const bool bf = uplink && p.gdt == DT_BF16;
-    if (p.n_small && !small_done) {
-        cudaError_t e = launch_topk_small(p, s, bf, st);
-        if (e != cudaSuccess) return e;
-        ++*launches;
-    }
     if (!p.n_large) return cudaSuccess;
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 1); CHECK_LAUNCH();
     if (bf) topk_hist2_dense_kernel<__nv_bfloat16><<<strided_grid(p, s.R), THREADS, 0, st>>>(p, s);
@@ -780,7 +769,9 @@ cudaError_t launch_topk_select(const Params &p, bool uplink, bool small_done, cu
 constexpr size_t SERVER_TOPK_SMEM = sizeof(float) * TILE + sizeof(uint32_t) * DIGIT1_BINS;
 
 cudaError_t configure_topk_kernels() {
-    cudaError_t e = cudaFuncSetAttribute(server_topk_kernel<COMP_TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = configure_topk_tail_kernels();
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(server_topk_kernel<COMP_TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)SERVER_TOPK_SMEM);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(server_topk_kernel<COMP_SIGN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -788,6 +779,16 @@ cudaError_t configure_topk_kernels() {
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(server_topk_kernel<COMP_IDENTITY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)SERVER_TOPK_SMEM);
+}
+
+// Single-tile segments of one side, selected directly (independent of everything else on that side:
+// the caller may run it on a stream of its own).
+cudaError_t launch_topk_small_segments(const Params &p, bool uplink, cudaStream_t st, int64_t *launches) {
+    if (!p.n_small) return cudaSuccess;
+    const TopkSide s = make_side(p, uplink);
+    cudaError_t e = launch_topk_small(p, s, uplink && p.gdt == DT_BF16, st);
+    if (e == cudaSuccess) ++*launches;
+    return e;
 }
 
 cudaError_t launch_server_topk(const Params &p, cudaStream_t st, int64_t *launches) {

@@ -27,8 +27,9 @@ template <typename GT>
 __global__ void __launch_bounds__(THREADS) topk_small_kernel(const __grid_constant__ Params p, const TopkSide s) {
     constexpr bool F32 = sizeof(GT) == 4;
     using ST = typename std::conditional<F32, float, unsigned short>::type;
-    __shared__ __align__(16) ST tile_s[TILE];
-    __shared__ uint32_t hist[256];
+    extern __shared__ __align__(16) unsigned char small_smem[];
+    uint32_t *hist = reinterpret_cast<uint32_t *>(small_smem);                               // [DIGIT1_BINS]
+    ST *tile_s = reinterpret_cast<ST *>(small_smem + sizeof(uint32_t) * DIGIT1_BINS);        // [TILE]
     __shared__ uint32_t scratch[THREADS + 4];
     __shared__ uint32_t warp_tot[THREADS / 32];
     const int t = __ldg(p.small_seg + blockIdx.x), row = blockIdx.y;
@@ -39,7 +40,6 @@ __global__ void __launch_bounds__(THREADS) topk_small_kernel(const __grid_consta
     const int64_t row_beg = (int64_t)row * s.row_stride + seg_beg;
     const ST *src = reinterpret_cast<const ST *>(s.src) + row_beg;
     stage_tile_guarded(tile_s, src, n, (row_beg & (F32 ? 3 : 7)) == 0);
-    __syncthreads();
 
     // thread q owns elements 32q .. 32q+31; it visits them in an order rotated by the lane so that
     // the lanes of a warp hit different banks
@@ -51,26 +51,31 @@ __global__ void __launch_bounds__(THREADS) topk_small_kernel(const __grid_consta
         else return ((uint32_t)tile_s[pos0 + j] & 0x7fffu) << 16;
     };
 
-    // radix select, most significant digit first (binary32: 8+8+8+7 bits; bfloat16 keys have only 15 bits: 8+7)
-    constexpr int LEVELS = F32 ? 4 : 2;
+    // radix select, most significant digit first: 12 + 12 + 7 key bits (bfloat16 keys have 15 bits: 12 + 3).
+    // The wide first digit spreads the entries over many bins (the exponent alone would put nearly
+    // all of them into a handful), which keeps the shared-memory atomics from serialising.
+    constexpr int LEVELS = F32 ? 3 : 2;
     constexpr int LOW = F32 ? 0 : 16;   // key bits below the last digit (all zero for bfloat16)
     uint32_t prefix = 0u, rank = k;
     bool ok = true;
 #pragma unroll
     for (int level = 0; level < LEVELS; ++level) {
-        const int bits = (level == LEVELS - 1) ? 7 : 8;
-        const int shift = F32 ? (level == 3 ? 0 : 23 - 8 * level) : (level == 0 ? 23 : 16);
-        hist[threadIdx.x] = 0u;   // THREADS == 256 bins
-        __syncthreads();
-        for (int i = 0; i < 32; ++i) {
-            const int j = (i + rot) & 31;
-            if (j < valid) {
-                const uint32_t key = key_at(j);
-                if ((key >> (shift + bits)) == prefix) atomicAdd(&hist[(key >> shift) & ((1u << bits) - 1u)], 1u);
+        const int bits = level == 0 ? 12 : (F32 ? (level == 1 ? 12 : 7) : 3);
+        const int shift = level == 0 ? DIGIT1_SHIFT : (F32 ? (level == 1 ? 7 : 0) : 16);
+        const int nbins = bits == 12 ? DIGIT1_BINS : THREADS;   // (block_pick wants at least one bin per thread)
+        for (int b = threadIdx.x; b < nbins / 4; b += THREADS) reinterpret_cast<uint4 *>(hist)[b] = make_uint4(0u, 0u, 0u, 0u);
+        __syncthreads();   // (also: the staged tile is complete)
+        if (valid > 0) {   // (short segments leave most threads without elements)
+            for (int i = 0; i < 32; ++i) {
+                const int j = (i + rot) & 31;
+                if (j < valid) {
+                    const uint32_t key = key_at(j);
+                    if ((key >> (shift + bits)) == prefix) atomicAdd(&hist[(key >> shift) & ((1u << bits) - 1u)], 1u);
+                }
             }
         }
         __syncthreads();
-        const PickResult r = block_pick<THREADS>(hist, 256, rank, scratch);
+        const PickResult r = block_pick<THREADS>(hist, nbins, rank, scratch);
         ok = ok && r.ok;
         prefix = (prefix << bits) | r.bin;
         rank = r.rank_in_bin;
@@ -169,17 +174,29 @@ __global__ void topk_check_kernel(const __grid_constant__ Params p, const TopkSi
 // ------------------------------------------------------------------------------------------------
 constexpr int TAIL_THREADS = 512;
 
+// Words of one bitmap over a problem's candidates, rounded up to whole rounds of the CTA.
+static inline int tail_bitmap_words(const Params &p) {
+    const int words = (int)((p.cap_max + 31) / 32);
+    return (words + TAIL_THREADS - 1) / TAIL_THREADS * TAIL_THREADS;
+}
+
 template <typename GT>
-__global__ void __launch_bounds__(TAIL_THREADS) topk_tail_kernel(const __grid_constant__ Params p, const TopkSide s) {
+__global__ void __launch_bounds__(TAIL_THREADS) topk_tail_kernel(const __grid_constant__ Params p, const TopkSide s,
+                                                                  const int bitmap_words) {
     constexpr int NT = TAIL_THREADS, NW = NT / 32;
     __shared__ __align__(16) uint32_t bins[DIGIT1_BINS];
     __shared__ uint32_t scratch[NT + 4];
     __shared__ uint32_t warp_tot[NW], warp_tot2[NW];
-    __shared__ uint32_t t_gt[TAIL_MAX_TILES], t_eq[TAIL_MAX_TILES];   // per tile: entries above the threshold / equal to it;
-                                                                      // after the scan: first output slot / ties to accept
-    __shared__ uint32_t t_tb[TAIL_MAX_TILES];                         // ties in the tiles before
+    // per tile: entries above the threshold / equal to it; after the scan over the tiles: first
+    // output slot / ties to accept; ties in the tiles before; start of the tile's candidate block
+    __shared__ uint32_t t_gt[TAIL_MAX_TILES], t_eq[TAIL_MAX_TILES], t_tb[TAIL_MAX_TILES], t_pos[TAIL_MAX_TILES];
+    // one bit per candidate (above the threshold / equal to it) and, per 32-bit word of those
+    // bitmaps, the number of set bits in the words before
+    extern __shared__ uint32_t tail_smem[];
+    uint32_t *gt_bits = tail_smem, *eq_bits = tail_smem + bitmap_words;
+    uint32_t *gt_before = tail_smem + 2 * bitmap_words, *eq_before = tail_smem + 3 * bitmap_words;
     const int t = __ldg(p.large_seg + blockIdx.x), row = blockIdx.y;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int lane = threadIdx.x & 31;
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
     // last kernel of a side: the next step starts with "no problem on the regular route yet"
     if (s.spec && blockIdx.x == 0 && row == 0 && threadIdx.x == 0) p.status[STATUS_ANY_REGULAR] = 0;
@@ -191,6 +208,13 @@ __global__ void __launch_bounds__(TAIL_THREADS) topk_tail_kernel(const __grid_co
     const uint32_t ncand = min(sel[SEL_CAND_COUNT], cap);  // (the cursor can run past the buffer when a tile was refused)
     uint32_t prefix = sel[SEL_PREFIX], rank = sel[SEL_REMAIN];
     uint32_t margin = sel[SEL_MARGIN];
+    const int first = __ldg(p.tile_prefix + t), ntiles = __ldg(p.tile_prefix + t + 1) - first;
+    const uint32_t seg_first = (uint32_t)__ldg(p.seg_off + t);
+    for (int q = threadIdx.x; q < ntiles; q += NT) {
+        t_pos[q] = s.meta[((int64_t)row * p.TT + first + q) * 4];
+        t_gt[q] = 0u;
+        t_eq[q] = 0u;
+    }
     __syncthreads();   // every thread holds the state before thread 0 starts rewriting it
     if (threadIdx.x == 0) {   // the next step starts from a clean slate
         sel[SEL_CAND_COUNT] = 0u;
@@ -206,65 +230,133 @@ __global__ void __launch_bounds__(TAIL_THREADS) topk_tail_kernel(const __grid_co
     }
     const int64_t cbase = (int64_t)row * p.CAP + __ldg(p.cap_off + t);
     const float *cand = s.cand_val + cbase;
-    auto fail = [&]() { if (threadIdx.x == 0) { atomicOr(p.status, STATUS_PICK_RANK); if (s.spec) sel[SEL_GUESS] = 0u; } };
+    const uint32_t *cidx = s.cand_idx + cbase;
+    auto fail = [&](int bit) { if (threadIdx.x == 0) { atomicOr(p.status, bit); if (s.spec) sel[SEL_GUESS] = 0u; } };
     auto clear_bins = [&](int nb) {
         for (int b = threadIdx.x; b < nb / 4; b += NT) reinterpret_cast<uint4 *>(bins)[b] = make_uint4(0u, 0u, 0u, 0u);
         __syncthreads();
     };
 
+    // Sweeps over the candidates' values: a thread fetches B values (B stripes of NT consecutive
+    // candidates) before it uses any, so that the loads are in flight together.
+    constexpr int B = 8;
+    auto sweep_keys = [&](auto &&use) {   // use(key) for every candidate of this thread
+        for (uint32_t q0 = threadIdx.x; q0 < ncand; q0 += NT * B) {
+            uint32_t key[B];
+#pragma unroll
+            for (int u = 0; u < B; ++u) key[u] = q0 + u * NT < ncand ? key_of(cand[q0 + u * NT]) : 0xffffffffu;
+#pragma unroll
+            for (int u = 0; u < B; ++u)
+                if (key[u] != 0xffffffffu) use(key[u]);
+        }
+    };
+
     bool refined = (flags & 2u) != 0u;
-    if (single) {   // first digit from the candidates themselves (all entries at or above the guess)
-        clear_bins(DIGIT1_BINS);
-        for (uint32_t q = threadIdx.x; q < ncand; q += NT) atomicAdd(&bins[key_of(cand[q]) >> DIGIT1_SHIFT], 1u);
+    if (single) {
+        // First digit from the candidates themselves (all entries at or above the guess).  They crowd
+        // into the bins just above the guess, where histogram atomics on one address would serialise:
+        // count in registers how many reach each of the WIN lowest bins; the bin of the k-th largest
+        // is almost always among them.
+        constexpr int WIN = 8;
+        const uint32_t gbin = sel[SEL_GUESS] >> DIGIT1_SHIFT;
+        uint32_t reach[WIN];
+#pragma unroll
+        for (int r = 0; r < WIN; ++r) reach[r] = 0u;
+        sweep_keys([&](uint32_t key) {
+            const uint32_t d1 = key >> DIGIT1_SHIFT;
+#pragma unroll
+            for (int r = 0; r < WIN; ++r) reach[r] += d1 >= gbin + r + 1u ? 1u : 0u;   // entries above bin gbin + r
+        });
+        if (threadIdx.x < WIN) bins[threadIdx.x] = 0u;
         __syncthreads();
-        const PickResult r1 = block_pick<NT>(bins, DIGIT1_BINS, k, scratch);
-        if (!r1.ok) { fail(); return; }
-        prefix = r1.bin;
-        rank = r1.rank_in_bin;
+#pragma unroll
+        for (int r = 0; r < WIN; ++r) {
+            const uint32_t c = __reduce_add_sync(0xffffffffu, reach[r]);
+            if (lane == 0 && c) atomicAdd(&bins[r], c);
+        }
+        __syncthreads();
+        // above[r] = entries above bin gbin + r; all ncand entries are at or above bin gbin
+        int found = -1;
+        uint32_t above_found = 0u;
+#pragma unroll
+        for (int r = WIN - 1; r >= 0; --r) {
+            const uint32_t above = bins[r];
+            if (above < k) { found = r; above_found = above; }   // keeps the lowest r with fewer than k entries above it
+        }
+        __syncthreads();   // bins are reused below
+        if (found >= 0) {
+            prefix = gbin + (uint32_t)found;
+            rank = k - above_found;
+        } else {   // the threshold moved up by more than WIN bins: plain histogram
+            clear_bins(DIGIT1_BINS);
+            sweep_keys([&](uint32_t key) { atomicAdd(&bins[key >> DIGIT1_SHIFT], 1u); });
+            __syncthreads();
+            const PickResult r1 = block_pick<NT>(bins, DIGIT1_BINS, k, scratch);
+            if (!r1.ok) { fail(STATUS_PICK_RANK); return; }
+            prefix = r1.bin;
+            rank = r1.rank_in_bin;
+        }
         refined = false;
     }
     if (!refined) {   // second digit among the entries that share the threshold's first digit
         const uint32_t b1 = prefix;
         clear_bins(DIGIT1_BINS);
-        for (uint32_t q = threadIdx.x; q < ncand; q += NT) {
-            const uint32_t key = key_of(cand[q]);
-            if ((key >> DIGIT1_SHIFT) == b1) atomicAdd(&bins[(key >> 7) & 0xfffu], 1u);
-        }
+        sweep_keys([&](uint32_t key) { if ((key >> DIGIT1_SHIFT) == b1) atomicAdd(&bins[(key >> 7) & 0xfffu], 1u); });
         __syncthreads();
         const PickResult r2 = block_pick<NT>(bins, DIGIT1_BINS, rank, scratch);
-        if (!r2.ok) { fail(); return; }
+        if (!r2.ok) { fail(STATUS_PICK_RANK); return; }
         prefix = (b1 << 12) | r2.bin;
         rank = r2.rank_in_bin;
     }
-    clear_bins(512);   // last 7 bits (block_pick wants at least NT bins; those above 127 stay empty)
-    for (uint32_t q = threadIdx.x; q < ncand; q += NT) {
-        const uint32_t key = key_of(cand[q]);
-        if ((key >> 7) == prefix) atomicAdd(&bins[key & 0x7fu], 1u);
-    }
+    clear_bins(NT);   // last 7 bits (block_pick wants at least NT bins; those above 127 stay empty)
+    sweep_keys([&](uint32_t key) { if ((key >> 7) == prefix) atomicAdd(&bins[key & 0x7fu], 1u); });
     __syncthreads();
     const PickResult r3 = block_pick<NT>(bins, NT, rank, scratch);
-    if (!r3.ok) { fail(); return; }
+    if (!r3.ok) { fail(STATUS_PICK_RANK); return; }
     const uint32_t T = (prefix << 7) | r3.bin;
     const uint32_t ties_wanted = r3.rank_in_bin;
 
-    // per tile (one warp each, no barrier between a warp's tiles): entries above T, entries equal to T
-    const int first = __ldg(p.tile_prefix + t), ntiles = __ldg(p.tile_prefix + t + 1) - first;
-    const uint32_t *meta0 = s.meta + ((int64_t)row * p.TT + first) * 4;
-    for (int q = warp; q < ntiles; q += NW) {
-        const uint32_t pos = meta0[4 * q], cnt = meta0[4 * q + 1];
-        uint32_t g = 0, e = 0;
-        for (uint32_t c = lane; c < cnt; c += 32) {
-            const uint32_t key = key_of(cand[pos + c]);
-            g += key > T ? 1u : 0u;
-            e += key == T ? 1u : 0u;
+    // Sweep over the candidates in buffer order (a warp takes 32 consecutive ones = one bitmap word):
+    // the two bitmaps, and per tile the number of entries above the threshold and equal to it.
+    // The tile of a candidate follows from its index.
+    const uint32_t nwords = (ncand + 31) >> 5;
+    constexpr int BX = 4;
+    for (uint32_t q0 = threadIdx.x & ~31u; q0 < ncand; q0 += NT * BX) {   // (bounds uniform over the warp)
+        uint32_t key[BX], tile[BX];
+#pragma unroll
+        for (int u = 0; u < BX; ++u) {
+            const uint32_t q = q0 + u * NT + lane;
+            const bool in = q < ncand;
+            key[u] = in ? key_of(cand[q]) : 0u;
+            tile[u] = in ? (cidx[q] - seg_first) >> 13 : 0xffffffffu;   // TILE = 2^13
         }
-        g = __reduce_add_sync(0xffffffffu, g);
-        e = __reduce_add_sync(0xffffffffu, e);
-        if (lane == 0) { t_gt[q] = g; t_eq[q] = e; }
+#pragma unroll
+        for (int u = 0; u < BX; ++u) {
+            const uint32_t qw = q0 + u * NT;
+            if (qw >= ncand) break;   // (uniform over the warp)
+            const bool in = tile[u] != 0xffffffffu;
+            const bool gt = in && key[u] > T, eq = in && key[u] == T;
+            const uint32_t gb = __ballot_sync(0xffffffffu, gt), eb = __ballot_sync(0xffffffffu, eq);
+            if (lane == 0) { gt_bits[qw >> 5] = gb; eq_bits[qw >> 5] = eb; }
+            // lanes of the first lane's tile add once; the others (a block boundary inside the word) one by one
+            const uint32_t tile0 = __shfl_sync(0xffffffffu, tile[u], 0);
+            const uint32_t same = __ballot_sync(0xffffffffu, tile[u] == tile0);
+            if (lane == 0 && tile0 < (uint32_t)ntiles) {
+                const uint32_t g = __popc(gb & same), e = __popc(eb & same);
+                if (g) atomicAdd(&t_gt[tile0], g);
+                if (e) atomicAdd(&t_eq[tile0], e);
+            }
+            if (in && tile[u] != tile0 && tile[u] < (uint32_t)ntiles) {
+                if (gt) atomicAdd(&t_gt[tile[u]], 1u);
+                if (eq) atomicAdd(&t_eq[tile[u]], 1u);
+            }
+        }
     }
+    for (uint32_t w = nwords + threadIdx.x; w < (uint32_t)bitmap_words; w += NT) { gt_bits[w] = 0u; eq_bits[w] = 0u; }
     __syncthreads();
     // tiles in order: ties accepted per tile (lowest index first) and first output slot
     constexpr int PER = TAIL_MAX_TILES / NT;
+    bool all_ties;   // every entry equal to the threshold is kept (the usual case: distinct magnitudes)
     {
         const int q0 = threadIdx.x * PER;
         uint32_t g[PER], e[PER], esum = 0;
@@ -298,39 +390,101 @@ __global__ void __launch_bounds__(TAIL_THREADS) topk_tail_kernel(const __grid_co
             tb += e[u];
         }
         if (sel_total != k) {   // (uniform over the CTA) inconsistent selection state: write nothing
-            if (threadIdx.x == 0) { atomicOr(p.status, STATUS_COUNT_MISMATCH); if (s.spec) sel[SEL_GUESS] = 0u; }
+            fail(STATUS_COUNT_MISMATCH);
             return;
+        }
+        all_ties = ties_total == ties_wanted;
+    }
+    // set bits in the bitmap words before each word (when every tie is kept, the first bitmap
+    // becomes "kept": above the threshold or equal to it)
+    {
+        const int perw = bitmap_words / NT;
+        const int w0 = threadIdx.x * perw;
+        uint32_t gsum = 0, esum = 0;
+        if (all_ties)
+            for (int u = 0; u < perw; ++u) gt_bits[w0 + u] |= eq_bits[w0 + u];
+        for (int u = 0; u < perw; ++u) { gsum += __popc(gt_bits[w0 + u]); esum += __popc(eq_bits[w0 + u]); }
+        uint32_t tot;
+        uint32_t gpre = block_exclusive_scan<NT>(gsum, warp_tot, tot);
+        uint32_t epre = block_exclusive_scan<NT>(esum, warp_tot2, tot);
+        for (int u = 0; u < perw; ++u) {
+            gt_before[w0 + u] = gpre; gpre += __popc(gt_bits[w0 + u]);
+            eq_before[w0 + u] = epre; epre += __popc(eq_bits[w0 + u]);
         }
     }
     __syncthreads();
-    // ordered compaction, one warp per tile
-    const uint32_t lt_mask = (1u << lane) - 1u;
+    // Ordered compaction, candidate-parallel: the slot of a kept candidate is its tile's first slot
+    // plus the kept candidates before it in its tile's block (blocks are contiguous and in index
+    // order; ties are accepted lowest index first, so the accepted ones before it number
+    // min(ties before it in the block, ties accepted in the tile)).
     const int64_t obase = (int64_t)row * p.K + kbeg;
-    const uint32_t *cidx = s.cand_idx + cbase;
-    for (int q = warp; q < ntiles; q += NW) {
-        const uint32_t pos = meta0[4 * q], cnt = meta0[4 * q + 1];
-        const uint32_t out0 = t_gt[q], allowed = t_eq[q], tb0 = t_tb[q];
-        uint32_t run_sel = 0, run_tie = 0;
-        for (uint32_t c0 = 0; c0 < cnt; c0 += 32) {
-            const uint32_t c = c0 + lane;
-            const bool in = c < cnt;
-            const float val = in ? cand[pos + c] : 0.0f;
-            const uint32_t idx = in ? cidx[pos + c] : 0u;
-            const uint32_t key = key_of(val);
-            const bool tie = in && key == T;
-            const uint32_t tbal = __ballot_sync(0xffffffffu, tie);
-            const uint32_t tie_rank = run_tie + __popc(tbal & lt_mask);
-            const bool take = in && (key > T || (tie && tie_rank < allowed));
-            const uint32_t sbal = __ballot_sync(0xffffffffu, take);
-            if (take) {
-                const uint32_t out = out0 + run_sel + __popc(sbal & lt_mask);   // < k by the scan above
-                s.idx[obase + out] = idx;
-                s.val[obase + out] = val;
-                if (s.zero_out) s.zero_out[idx] = 0.0f;
-                if (tie && tb0 + tie_rank + 1u == ties_wanted) sel[SEL_CUT] = idx;
+    if (all_ties) {
+        // the slot of a kept candidate = (its tile's first slot - kept candidates before the tile's block)
+        // + kept candidates before it in the buffer
+        for (int q = threadIdx.x; q < ntiles; q += NT) {
+            const uint32_t pb = t_pos[q], pw = pb >> 5;
+            t_gt[q] -= gt_before[pw] + __popc(gt_bits[pw] & ((1u << (pb & 31u)) - 1u));
+        }
+        __syncthreads();
+        for (uint32_t q0 = threadIdx.x; q0 < ncand; q0 += NT * BX) {
+            uint32_t idx[BX];
+            float val[BX];
+#pragma unroll
+            for (int u = 0; u < BX; ++u) {
+                const uint32_t q = q0 + u * NT;
+                idx[u] = q < ncand ? cidx[q] : 0xffffffffu;
+                val[u] = q < ncand ? cand[q] : 0.0f;
             }
-            run_sel += __popc(sbal);
-            run_tie += __popc(tbal);
+#pragma unroll
+            for (int u = 0; u < BX; ++u) {
+                const uint32_t q = q0 + u * NT;
+                if (q >= ncand) break;
+                const uint32_t w = q >> 5, bit = q & 31u, kw = gt_bits[w];
+                if (!((kw >> bit) & 1u)) continue;
+                const uint32_t tile = (idx[u] - seg_first) >> 13;
+                if (tile >= (uint32_t)ntiles) continue;
+                const uint32_t out = t_gt[tile] + gt_before[w] + __popc(kw & ((1u << bit) - 1u));   // < k by the scan above
+                s.idx[obase + out] = idx[u];
+                s.val[obase + out] = val[u];
+                if (s.zero_out) s.zero_out[idx[u]] = 0.0f;
+                if ((eq_bits[w] >> bit) & 1u) {   // the last tie (all are kept): the one with ties_wanted - 1 ties before it
+                    const uint32_t pb = t_pos[tile], pw = pb >> 5;
+                    const uint32_t e_in_block = eq_before[w] + __popc(eq_bits[w] & ((1u << bit) - 1u)) -
+                                                (eq_before[pw] + __popc(eq_bits[pw] & ((1u << (pb & 31u)) - 1u)));
+                    if (t_tb[tile] + e_in_block + 1u == ties_wanted) sel[SEL_CUT] = idx[u];
+                }
+            }
+        }
+    } else
+    for (uint32_t q0 = threadIdx.x; q0 < ncand; q0 += NT * BX) {
+        uint32_t idx[BX];
+        float val[BX];
+#pragma unroll
+        for (int u = 0; u < BX; ++u) {   // (all of them: most candidates are kept)
+            const uint32_t q = q0 + u * NT;
+            idx[u] = q < ncand ? cidx[q] : 0xffffffffu;
+            val[u] = q < ncand ? cand[q] : 0.0f;
+        }
+#pragma unroll
+        for (int u = 0; u < BX; ++u) {
+            const uint32_t q = q0 + u * NT;
+            if (q >= ncand) break;
+            const uint32_t w = q >> 5, below = (1u << (q & 31u)) - 1u;
+            const uint32_t gw = gt_bits[w], ew = eq_bits[w];
+            const bool gt = (gw >> (q & 31u)) & 1u, eq = (ew >> (q & 31u)) & 1u;
+            if (!gt && !eq) continue;
+            const uint32_t tile = (idx[u] - seg_first) >> 13;
+            if (tile >= (uint32_t)ntiles) continue;   // (an index outside the segment cannot come out of the filter)
+            const uint32_t pb = t_pos[tile], pw = pb >> 5, pbelow = (1u << (pb & 31u)) - 1u;
+            const uint32_t g_in_block = gt_before[w] + __popc(gw & below) - (gt_before[pw] + __popc(gt_bits[pw] & pbelow));
+            const uint32_t e_in_block = eq_before[w] + __popc(ew & below) - (eq_before[pw] + __popc(eq_bits[pw] & pbelow));
+            const uint32_t allowed = t_eq[tile];
+            if (eq && e_in_block >= allowed) continue;   // a tie beyond the accepted ones
+            const uint32_t out = t_gt[tile] + g_in_block + min(e_in_block, allowed);   // < k by the scan above
+            s.idx[obase + out] = idx[u];
+            s.val[obase + out] = val[u];
+            if (s.zero_out) s.zero_out[idx[u]] = 0.0f;
+            if (eq && t_tb[tile] + e_in_block + 1u == ties_wanted) sel[SEL_CUT] = idx[u];
         }
     }
     if (threadIdx.x == 0) {
@@ -348,10 +502,13 @@ __global__ void __launch_bounds__(TAIL_THREADS) topk_tail_kernel(const __grid_co
 // ------------------------------------------------------------------------------------------------
 // launchers
 // ------------------------------------------------------------------------------------------------
+constexpr size_t SMALL_SMEM_F32 = sizeof(uint32_t) * DIGIT1_BINS + sizeof(float) * TILE;
+constexpr size_t SMALL_SMEM_BF16 = sizeof(uint32_t) * DIGIT1_BINS + sizeof(unsigned short) * TILE;
+
 cudaError_t launch_topk_small(const Params &p, const TopkSide &s, bool bf16, cudaStream_t st) {
     const dim3 grid(p.n_small, s.R);
-    if (bf16) topk_small_kernel<__nv_bfloat16><<<grid, THREADS, 0, st>>>(p, s);
-    else topk_small_kernel<float><<<grid, THREADS, 0, st>>>(p, s);
+    if (bf16) topk_small_kernel<__nv_bfloat16><<<grid, THREADS, SMALL_SMEM_BF16, st>>>(p, s);
+    else topk_small_kernel<float><<<grid, THREADS, SMALL_SMEM_F32, st>>>(p, s);
     return cudaGetLastError();
 }
 
@@ -362,9 +519,21 @@ cudaError_t launch_topk_check(const Params &p, const TopkSide &s, cudaStream_t s
 
 cudaError_t launch_topk_tail(const Params &p, const TopkSide &s, bool bf16, cudaStream_t st) {
     const dim3 grid(p.n_large, s.R);
-    if (bf16) topk_tail_kernel<__nv_bfloat16><<<grid, TAIL_THREADS, 0, st>>>(p, s);
-    else topk_tail_kernel<float><<<grid, TAIL_THREADS, 0, st>>>(p, s);
+    const int words = tail_bitmap_words(p);
+    const size_t smem = sizeof(uint32_t) * 4 * (size_t)words;
+    if (bf16) topk_tail_kernel<__nv_bfloat16><<<grid, TAIL_THREADS, smem, st>>>(p, s, words);
+    else topk_tail_kernel<float><<<grid, TAIL_THREADS, smem, st>>>(p, s, words);
     return cudaGetLastError();
+}
+
+// Opt-in shared memory sizes of the kernels in this file (once per device).
+cudaError_t configure_topk_tail_kernels() {
+    const int tail_max = (int)(sizeof(uint32_t) * 4 * ((TAIL_MAX_CAND + 31) / 32 + TAIL_THREADS));
+    cudaError_t e = cudaFuncSetAttribute(topk_tail_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, tail_max);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_tail_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, tail_max);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_small_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMALL_SMEM_F32);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_small_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMALL_SMEM_BF16);
+    return e;
 }
 
 }  // namespace liec
