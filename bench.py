@@ -423,13 +423,44 @@ def run_gpu(args, w, rank, world, local_rank, steps=None, extras=True):
                           "took the two-pass route",
                   "uplink_refined_per_step": acc["uplink_refined"] / extra,
                   "downlink_refined_per_step": acc["downlink_refined"] / extra, "slow_per_step": acc["slow"] / extra}
+    # the same iteration with the fused telemetry switched on (squared norms of e, v and g left by the
+    # server pass and the worker update), the accessor that reduces them, and, for comparison, the
+    # separate passes that give the same numbers on demand (liec_sumsq over e and over the gradients)
+    telemetry = None
+    if args.telemetry:
+        tsteps = max(3, min(steps, 10))
+        ctx.liec_set_telemetry(True)
+        for _ in range(2):
+            one_step()
+        t0, t1, t2, t3 = (torch.cuda.Event(enable_timing=True) for _ in range(4))
+        torch.cuda.synchronize()
+        t0.record()
+        for _ in range(tsteps):
+            one_step()
+        t1.record()
+        tel = ctx.liec_get_telemetry()
+        t2.record()
+        out_e = torch.empty(1, lay.num_segments, dtype=torch.float64, device=dev)
+        out_g = torch.empty(N, lay.num_segments, dtype=torch.float64, device=dev)
+        ctx.liec_sumsq(liec.SUMSQ_ERROR, out_e)
+        ctx.liec_sumsq(liec.SUMSQ_GRADS, out_g, grads=batches[(counter[0] - 1) % NUM_BATCHES])
+        t3.record()
+        torch.cuda.synchronize()
+        assert torch.equal(out_g, tel["g_sumsq"]), "fused and separate squared norms of g differ"
+        ctx.liec_set_telemetry(False)
+        on_ms = t0.elapsed_time(t1) / tsteps
+        telemetry = {"ms_per_step_on": on_ms, "ms_per_step_off": total_ms / steps, "steps": tsteps,
+                     "overhead_pct": 100 * (on_ms / (total_ms / steps) - 1), "accessor_ms": t1.elapsed_time(t2),
+                     "separate_passes_ms": t2.elapsed_time(t3),
+                     "note": "on: the server pass also leaves ||e_t||^2 and ||v_t||^2, the worker update ||g^i_t||^2 per "
+                             "tile; accessor: liec_get_telemetry; separate passes: liec_sumsq over e and over the gradients"}
     if not extras:
         ms_step = total_ms / steps
         if world > 1:
             vals = max_over_ranks([ms_step] + stage_ms, device=dev)
             ms_step, stage_ms = vals[0], vals[1:]
         return dict(ms_step=ms_step, stage_ms=dict(zip(stage_names, stage_ms)), launches=launches, clocks=clocks,
-                    e2e=None, average_ms=None, graph_ms=None, routes=routes, steps=steps)
+                    e2e=None, average_ms=None, graph_ms=None, routes=routes, steps=steps, telemetry=telemetry)
 
     # the same step replayed from a CUDA graph (one capture of liec_step, K replays): shows what the
     # launch gaps cost on small workloads; reported beside the headline, not instead of it
@@ -498,7 +529,7 @@ def run_gpu(args, w, rank, world, local_rank, steps=None, extras=True):
         if e2e:
             e2e["ms_per_step"] = e2e_max
     return dict(ms_step=ms_step, stage_ms=dict(zip(stage_names, stage_ms)), launches=launches, clocks=clocks, e2e=e2e,
-                average_ms=average_ms, graph_ms=graph_ms, routes=routes, steps=steps)
+                average_ms=average_ms, graph_ms=graph_ms, routes=routes, steps=steps, telemetry=telemetry)
 
 
 def describe(w, gpus):
@@ -540,6 +571,8 @@ def throughput_fields(w, r, world):
     }
     if r["routes"] is not None:
         out["topk_routes"] = r["routes"]
+    if r.get("telemetry") is not None:
+        out["telemetry"] = r["telemetry"]
     return out
 
 
@@ -560,6 +593,8 @@ def main():
     ap.add_argument("--batches", type=int, default=0,
                     help="resident gradient batches the steps cycle through (default: as many as fit in 40 GB, 4 to 16)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-telemetry", dest="telemetry", action="store_false", default=True,
+                    help="skip the extra steps that time the iteration with the fused telemetry switched on")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cuda-graph", dest="cuda_graph", action="store_true", default=True,

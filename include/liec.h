@@ -221,6 +221,40 @@ liec_status liec_mean_params(liec_ctx *ctx, float *out, void *stream);
 liec_status liec_sumsq(liec_ctx *ctx, int32_t which, const void *grads, double *out, void *stream);
 
 /*
+ * Telemetry fused into the iteration's own passes: the quantities behind the paper's figure of
+ * error norms (||e_t||) and its table of measured delta (Def. 1: delta = 1 - ||x - C(x)||^2 / ||x||^2,
+ * worker side x = g^i, server side x = v) at no extra pass over the model-sized arrays.
+ *
+ * liec_set_telemetry(ctx, 1) makes the following iterations use kernel variants that also leave
+ * per-tile partial sums of squares, taken where the values are in registers anyway: e_t^2 and v_t^2
+ * in the server pass (which reads e_t and writes v_t), (g^i_t)^2 in the worker update.  With 0 (the
+ * state after liec_init) the kernels without any of it run.  Parameters, error and messages are bit
+ * for bit the same either way.  LIEC_ERR_STATE between the stages of an iteration.
+ *
+ * liec_get_telemetry reduces the partial sums of the last completed iteration to per-segment sums,
+ * in binary64 over the same balanced tree as liec_sumsq (deterministic, bit-exact with a plain
+ * recursive evaluation).  Every output pointer is device memory owned by the caller and may be NULL:
+ *   e_sumsq          [T]     ||e_t||^2 per segment: the global error as it ENTERED the iteration
+ *                            (Algorithm 1's e_t; the error it left behind, e_{t+1}, is what the next
+ *                            iteration reports, or liec_sumsq(LIEC_SUMSQ_ERROR) at any time)
+ *   v_sumsq          [T]     ||v_t||^2 per segment
+ *   g_sumsq          [N][T]  ||g^i_t||^2 per worker and segment
+ *   up_kept_sumsq    [N][T]  top-k / random-k uplink only: sum of squares of the k_t values of the
+ *                            worker's message for the segment, over the tree on those k_t values in
+ *                            message order (one read of the message values, K floats per row, when called)
+ *   down_kept_sumsq  [T]     the same for a top-k / random-k downlink message
+ * From these: ||e_t|| = sqrt(sum_t e_sumsq[t]);  scaled sign: ||x - C(x)||^2 = ||x||^2 - 2 s ||x||_1 + n s^2
+ * with s the message's scale (delta = n s^2 / ||x||^2 up to the rounding of s);  top-k / random-k:
+ * delta = kept / ||x||^2 (the kept entries are copied exactly).
+ * A few small kernels on `stream`.  LIEC_ERR_STATE when no iteration has completed since the telemetry
+ * was switched on, or between the stages of an iteration; LIEC_ERR_INVALID_ARG when a kept-value norm
+ * is asked of a side that sends no (index, value) message.
+ */
+liec_status liec_set_telemetry(liec_ctx *ctx, int32_t on);
+liec_status liec_get_telemetry(liec_ctx *ctx, double *e_sumsq, double *v_sumsq, double *g_sumsq,
+                               double *up_kept_sumsq, double *down_kept_sumsq, void *stream);
+
+/*
  * One iteration fed from host memory: copies grads_host ([N][d] of cfg.grad_dtype, pinned
  * memory recommended) into grads_dev (device staging buffer of the same size, caller
  * owned, 16-byte aligned), runs liec_step, copies the downlink message (sign: words then scales;

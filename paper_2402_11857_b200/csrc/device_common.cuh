@@ -131,6 +131,13 @@ __device__ __forceinline__ double leaf4(const float (&v)[4]) {
     return __dadd_rn(__dadd_rn(a0, a1), __dadd_rn(a2, a3));
 }
 
+// Same two levels over the squares (telemetry: squared norms over the same tree).  A binary32
+// value squared is exact in binary64 (24-bit significands).
+__device__ __forceinline__ double leaf4_sq(const float (&v)[4]) {
+    const double d0 = (double)v[0], d1 = (double)v[1], d2 = (double)v[2], d3 = (double)v[3];
+    return __dadd_rn(__dadd_rn(__dmul_rn(d0, d0), __dmul_rn(d1, d1)), __dadd_rn(__dmul_rn(d2, d2), __dmul_rn(d3, d3)));
+}
+
 __device__ __forceinline__ double shfl_xor_f64(double x, int mask) {
     return __shfl_xor_sync(0xffffffffu, x, mask);
 }
@@ -178,6 +185,19 @@ __device__ __forceinline__ double cta_tree_reduce(double warp_sum, double *smem8
         s = __dadd_rn(__dadd_rn(s01, s23), __dadd_rn(s45, s67));
     }
     return s;
+}
+
+// Two tile sums at once (one barrier): results in thread 0.
+__device__ __forceinline__ void cta_tree_reduce_pair(double wa, double wb, double *smem16, double &ra, double &rb) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) { smem16[warp] = wa; smem16[8 + warp] = wb; }
+    __syncthreads();
+    ra = rb = 0.0;
+    if (threadIdx.x == 0) {
+        const double *a = smem16, *b = smem16 + 8;
+        ra = __dadd_rn(__dadd_rn(__dadd_rn(a[0], a[1]), __dadd_rn(a[2], a[3])), __dadd_rn(__dadd_rn(a[4], a[5]), __dadd_rn(a[6], a[7])));
+        rb = __dadd_rn(__dadd_rn(__dadd_rn(b[0], b[1]), __dadd_rn(b[2], b[3])), __dadd_rn(__dadd_rn(b[4], b[5]), __dadd_rn(b[6], b[7])));
+    }
 }
 
 // Combines per-tile partial sums (binary64) of one segment in tree order: pairwise, level by level,

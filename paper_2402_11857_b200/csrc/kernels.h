@@ -29,7 +29,7 @@ cudaError_t launch_mean_params(const Params &p, float *out, cudaStream_t st);
 
 // squared norms (monitoring)
 cudaError_t launch_sumsq(const Params &p, const void *src, int64_t row_stride, int rows, bool bf16, cudaStream_t st);
-cudaError_t launch_sum_finalize(const Params &p, int rows, double *out, cudaStream_t st);
+cudaError_t launch_sum_finalize(const Params &p, const double *partials, int rows, double *out, cudaStream_t st);
 
 // worker update
 cudaError_t launch_worker_update(const Params &p, float lr, cudaStream_t st);

@@ -24,12 +24,12 @@ struct Region {
 };
 
 struct Plan {
-    int32_t N = 0, T = 0, TT = 0;
+    int32_t N = 0, T = 0, TT = 0, KTT = 0;
     int64_t d = 0, W = 0, K = 0, CAP = 0, cap_max = 0;
     std::vector<int64_t> seg_off, word_off, k_off, cap_off, topk_k;
-    std::vector<int32_t> tile_prefix, tile_seg, small_seg, large_seg;
+    std::vector<int32_t> tile_prefix, tile_seg, small_seg, large_seg, ktile_prefix, ktile_seg;
     Region r_seg_off, r_word_off, r_k_off, r_cap_off, r_tile_prefix, r_tile_seg, r_small_seg, r_large_seg, r_status;
-    Region r_tel_partials;
+    Region r_tel_partials, r_tel_e, r_tel_v, r_tel_g, r_tel_kept, r_ktile_prefix, r_ktile_seg;
     Region r_up_words, r_up_scales, r_up_partials, r_down_words, r_down_scales, r_down_partials, r_vbuf;
     Region r_up_idx, r_up_val, r_down_idx, r_down_val;
     Region r_up_hist, r_down_hist, r_up_hist2, r_down_hist2, r_up_sel, r_down_sel;
@@ -115,6 +115,19 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     std::stable_sort(pl.large_seg.begin(), pl.large_seg.end(), [&](int32_t a, int32_t b) {
         return pl.seg_off[a + 1] - pl.seg_off[a] > pl.seg_off[b + 1] - pl.seg_off[b];
     });
+    // a sparse message's values, tiled like the model (for their squared norms): segment t owns k_t entries
+    pl.ktile_prefix.assign(T + 1, 0);
+    if (any_topk) {
+        int64_t ktiles = 0;
+        for (int t = 0; t < T; ++t) {
+            ktiles += (pl.topk_k[t] + TILE - 1) / TILE;
+            pl.ktile_prefix[t + 1] = (int32_t)ktiles;   // (at most the model's own tile count)
+        }
+        pl.KTT = (int32_t)ktiles;
+        pl.ktile_seg.resize(pl.KTT);
+        for (int t = 0; t < T; ++t)
+            for (int q = pl.ktile_prefix[t]; q < pl.ktile_prefix[t + 1]; ++q) pl.ktile_seg[q] = t;
+    }
     pl.W = pl.word_off[T];
     pl.K = pl.k_off[T];
     pl.CAP = pl.cap_off[T];
@@ -136,6 +149,12 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     pl.r_large_seg = c.take(sizeof(int32_t) * pl.large_seg.size());
     pl.r_status = c.take(256);
     pl.r_tel_partials = c.take(sizeof(double) * (size_t)pl.N * pl.TT);
+    pl.r_tel_e = c.take(sizeof(double) * (size_t)pl.TT);
+    pl.r_tel_v = c.take(sizeof(double) * (size_t)pl.TT);
+    pl.r_tel_g = c.take(sizeof(double) * (size_t)pl.N * pl.TT);
+    pl.r_ktile_prefix = c.take(sizeof(int32_t) * (T + 1));
+    pl.r_ktile_seg = c.take(sizeof(int32_t) * pl.KTT);
+    pl.r_tel_kept = c.take(sizeof(double) * (size_t)pl.N * pl.KTT);
     const size_t N = pl.N;
     if (cfg->uplink == LIEC_COMP_SCALED_SIGN) {
         pl.r_up_words = c.take(sizeof(uint32_t) * N * pl.W);
@@ -194,6 +213,7 @@ struct liec_ctx {
     char *ws = nullptr;
     int stage = 0;  // 0 idle, 1 after uplink, 2 after aggregate, 3 after downlink
     int64_t launches = 0;
+    bool telemetry_valid = false;  // an iteration has completed with the telemetry switched on
     std::string err;
     // top-k: the single-tile segments are selected on a stream of the context's own, forked from
     // and joined to the caller's stream by events, so that they overlap the dense passes
@@ -343,6 +363,14 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     p.down_partials = at<double>(c, pl.r_down_partials);
     p.vbuf = at<float>(c, pl.r_vbuf);
     p.tel_partials = at<double>(c, pl.r_tel_partials);
+    p.telemetry = 0;
+    p.tel_e = at<double>(c, pl.r_tel_e);
+    p.tel_v = at<double>(c, pl.r_tel_v);
+    p.tel_g = at<double>(c, pl.r_tel_g);
+    p.tel_kept = at<double>(c, pl.r_tel_kept);
+    p.KTT = pl.KTT;
+    p.ktile_prefix = at<int32_t>(c, pl.r_ktile_prefix);
+    p.ktile_seg = at<int32_t>(c, pl.r_ktile_seg);
     p.up_idx = at<uint32_t>(c, pl.r_up_idx);       p.up_val = at<float>(c, pl.r_up_val);
     p.down_idx = at<uint32_t>(c, pl.r_down_idx);   p.down_val = at<float>(c, pl.r_down_val);
     p.up_hist = at<uint32_t>(c, pl.r_up_hist);     p.down_hist = at<uint32_t>(c, pl.r_down_hist);
@@ -358,6 +386,7 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
         {&pl.r_seg_off, pl.seg_off.data()}, {&pl.r_word_off, pl.word_off.data()}, {&pl.r_k_off, pl.k_off.data()},
         {&pl.r_cap_off, pl.cap_off.data()}, {&pl.r_tile_prefix, pl.tile_prefix.data()},
         {&pl.r_tile_seg, pl.tile_seg.data()}, {&pl.r_small_seg, pl.small_seg.data()}, {&pl.r_large_seg, pl.large_seg.data()},
+        {&pl.r_ktile_prefix, pl.ktile_prefix.data()}, {&pl.r_ktile_seg, pl.ktile_seg.data()},
     };
     for (const Up &u : ups) {
         if (!u.r->bytes) continue;
@@ -472,6 +501,7 @@ liec_status liec_worker_update(liec_ctx *c, const void *grads, float lr, void *s
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     LIEC_LAUNCH(c, launch_worker_update(c->p, lr, s));
     c->stage = 0;
+    c->telemetry_valid = c->p.telemetry != 0;
     return LIEC_OK;
 }
 
@@ -537,7 +567,53 @@ liec_status liec_sumsq(liec_ctx *c, int32_t which, const void *grads, double *ou
     const bool bf16 = which == 1 && c->p.gdt == DT_BF16;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     LIEC_LAUNCH(c, launch_sumsq(c->p, src, which == 0 ? 0 : c->p.d, rows, bf16, s));
-    LIEC_LAUNCH(c, launch_sum_finalize(c->p, rows, out, s));
+    LIEC_LAUNCH(c, launch_sum_finalize(c->p, c->p.tel_partials, rows, out, s));
+    return LIEC_OK;
+}
+
+liec_status liec_set_telemetry(liec_ctx *c, int32_t on) {
+    liec_status st = check_stage(c, 0, "liec_set_telemetry");
+    if (st != LIEC_OK) return st;
+    c->p.telemetry = on ? 1 : 0;
+    c->telemetry_valid = false;
+    return LIEC_OK;
+}
+
+liec_status liec_get_telemetry(liec_ctx *c, double *e_sumsq, double *v_sumsq, double *g_sumsq,
+                               double *up_kept_sumsq, double *down_kept_sumsq, void *stream) {
+    liec_status st = check_stage(c, 0, "liec_get_telemetry");
+    if (st != LIEC_OK) return st;
+    if (!c->telemetry_valid) {
+        c->err = "liec_get_telemetry: no iteration has run since liec_set_telemetry switched the telemetry on";
+        return LIEC_ERR_STATE;
+    }
+    if ((up_kept_sumsq && !comp_is_sparse(c->p.up)) || (down_kept_sumsq && !comp_is_sparse(c->p.down))) {
+        c->err = "liec_get_telemetry: kept-value norms exist only for a top-k or random-k side";
+        return LIEC_ERR_INVALID_ARG;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const Params &p = c->p;
+    if (e_sumsq) LIEC_LAUNCH(c, launch_sum_finalize(p, p.tel_e, 1, e_sumsq, s));
+    if (v_sumsq) LIEC_LAUNCH(c, launch_sum_finalize(p, p.tel_v, 1, v_sumsq, s));
+    if (g_sumsq) LIEC_LAUNCH(c, launch_sum_finalize(p, p.tel_g, p.N, g_sumsq, s));
+    if (up_kept_sumsq || down_kept_sumsq) {
+        // the message values laid out like a model of K entries with segments of k_t: the same two
+        // kernels as liec_sumsq, driven by the tables of that layout
+        Params pk = p;
+        pk.seg_off = p.k_off;
+        pk.tile_prefix = p.ktile_prefix;
+        pk.tile_seg = p.ktile_seg;
+        pk.TT = p.KTT;
+        pk.tel_partials = p.tel_kept;
+        if (up_kept_sumsq) {
+            LIEC_LAUNCH(c, launch_sumsq(pk, p.up_val, p.K, p.N, false, s));
+            LIEC_LAUNCH(c, launch_sum_finalize(pk, pk.tel_partials, p.N, up_kept_sumsq, s));
+        }
+        if (down_kept_sumsq) {
+            LIEC_LAUNCH(c, launch_sumsq(pk, p.down_val, 0, 1, false, s));
+            LIEC_LAUNCH(c, launch_sum_finalize(pk, pk.tel_partials, 1, down_kept_sumsq, s));
+        }
+    }
     return LIEC_OK;
 }
 

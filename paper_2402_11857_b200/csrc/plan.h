@@ -52,7 +52,19 @@ struct Params {
     uint32_t *down_words;  // [W]
     float *down_scales;    // [T]
     double *down_partials; // [TT]
-    double *tel_partials;  // [N][TT] telemetry (squared norms)
+    double *tel_partials;  // [N][TT] squared norms on demand (liec_sumsq)
+
+    // telemetry fused into the iteration's own passes (switched by liec_set_telemetry): per-tile
+    // binary64 partial sums of squares, written by the kernels that hold the values anyway
+    int32_t telemetry;     // 0 = off: the kernels without any of it
+    double *tel_e;         // [TT]    ||e_t||^2, the error as the server pass reads it
+    double *tel_v;         // [TT]    ||v_t||^2, as the server pass writes it
+    double *tel_g;         // [N][TT] ||g^i_t||^2, from the worker update
+    // the values of a sparse message are tiled like the model: segment t owns k_t entries
+    int32_t KTT;                  // tiles of one row of a sparse message
+    const int32_t *ktile_prefix;  // [T+1]
+    const int32_t *ktile_seg;     // [KTT]
+    double *tel_kept;             // [N][KTT] scratch for the squared norms of message values
 
     // top-k messages and scratch (row count R = N for uplink, 1 for downlink)
     const uint32_t *up_sets, *down_set;  // random-k: the caller's subsets [N][K] / [K]

@@ -173,9 +173,11 @@ __global__ void __launch_bounds__(THREADS) scale_finalize_kernel(const __grid_co
 //   acc = +0; for i = 0..N-1: acc = acc + p^i_j;   v_j = e_j + acc / N        (written over e)
 // and, when the downlink is scaled sign, the words of v and the tile partial of ||v||_1.
 // ------------------------------------------------------------------------------------------------
-template <bool DOWN_SIGN, typename GT>
+// TEL: also the tile's partial sums of e^2 (as read) and v^2 (as written), same tree as the L1 norm.
+template <bool DOWN_SIGN, typename GT, bool TEL>
 __global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_constant__ Params p) {
     __shared__ double warp_sums[8];
+    __shared__ double tel_sums[TEL ? 16 : 1];
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
@@ -209,12 +211,14 @@ __global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_cons
     const WorkerDivisor by_n(p.N);
     float *e_tile = p.e + ti.seg_beg + ti.rel;
     double a[8];
+    double te[TEL ? 8 : 1], tv[TEL ? 8 : 1];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int pos = tile_pos(warp, lane, j);
         float ev[4], v[4];
         if (fast) load4_stream(e_tile + pos, ev);
         else load4_guarded(e_tile, pos, ti.len, ev);
+        if constexpr (TEL) te[j] = leaf4_sq(ev);
         by_n.div4(acc[j], v);
 #pragma unroll
         for (int c = 0; c < 4; ++c) v[c] = __fadd_rn(ev[c], v[c]);
@@ -226,6 +230,7 @@ __global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_cons
                 if (pos + c < ti.len) e_tile[pos + c] = v[c]; else v[c] = 0.0f;  // padding: +0, bit 0
             }
         }
+        if constexpr (TEL) tv[j] = leaf4_sq(v);
         if (DOWN_SIGN) {
             a[j] = leaf4(v);
             uint32_t w = pack_word(sign_nibble(v), lane);
@@ -237,15 +242,21 @@ __global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_cons
         double s = cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
         if (threadIdx.x == 0) p.down_partials[blockIdx.x] = s;
     }
+    if constexpr (TEL) {
+        double re, rv;
+        cta_tree_reduce_pair(warp_tree_reduce8(te, lane), warp_tree_reduce8(tv, lane), tel_sums, re, rv);
+        if (threadIdx.x == 0) { p.tel_e[blockIdx.x] = re; p.tel_v[blockIdx.x] = rv; }
+    }
 }
 
 // Sign uplink, one thread per 32-bit word: thread q of the CTA owns elements 32q..32q+31 of the
 // tile, i.e. exactly one word of every worker's message, so unpacking needs no shuffles
 // (shift + sign-xor + add per element and worker), the word of v is built in-thread and the
 // ||v||_1 leaf covers five tree levels in-thread.
-template <bool DOWN_SIGN>
+template <bool DOWN_SIGN, bool TEL>
 __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_constant__ Params p) {
     __shared__ double warp_sums[8];
+    __shared__ double tel_sums[TEL ? 16 : 1];
     constexpr int SCALE_CHUNK = 1024;              // workers whose scales are staged at once (a multiple of WG)
     __shared__ float up_scale_smem[SCALE_CHUNK];   // this segment's scales of workers c0 .. c0 + SCALE_CHUNK - 1
     const TileInfo ti = locate_tile(p, blockIdx.x);
@@ -298,6 +309,7 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
     float *e_tile = p.e + ti.seg_beg + ti.rel;
     uint32_t vword = 0u;
     double leaf[8];
+    double te[TEL ? 8 : 1], tv[TEL ? 8 : 1];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
         const int pos = pos0 + 4 * k;
@@ -308,6 +320,7 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
         } else {
             load4_guarded(e_tile, pos, ti.len, ev);
         }
+        if constexpr (TEL) te[k] = leaf4_sq(ev);
         {
             const float a4[4] = {acc[4 * k], acc[4 * k + 1], acc[4 * k + 2], acc[4 * k + 3]};
             by_n.div4(a4, v);
@@ -322,19 +335,29 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
                 if (pos + c < ti.len) e_tile[pos + c] = v[c]; else v[c] = 0.0f;
             }
         }
+        if constexpr (TEL) tv[k] = leaf4_sq(v);
         if (DOWN_SIGN) {
             leaf[k] = leaf4(v);
             vword |= sign_nibble(v) << (4 * k);
         }
     }
-    if (DOWN_SIGN) {
-        if (have_word) p.down_words[wbase + my_widx] = vword;
-        double s = __dadd_rn(__dadd_rn(__dadd_rn(leaf[0], leaf[1]), __dadd_rn(leaf[2], leaf[3])),
-                             __dadd_rn(__dadd_rn(leaf[4], leaf[5]), __dadd_rn(leaf[6], leaf[7])));
+    // a thread's 32 consecutive elements: three more tree levels in-thread, five across the lanes
+    auto thread_then_warp = [](const double (&l)[8]) {
+        double s = __dadd_rn(__dadd_rn(__dadd_rn(l[0], l[1]), __dadd_rn(l[2], l[3])),
+                             __dadd_rn(__dadd_rn(l[4], l[5]), __dadd_rn(l[6], l[7])));
 #pragma unroll
         for (int m = 1; m < 32; m <<= 1) s = __dadd_rn(s, shfl_xor_f64(s, m));
-        s = cta_tree_reduce(s, warp_sums);
+        return s;
+    };
+    if (DOWN_SIGN) {
+        if (have_word) p.down_words[wbase + my_widx] = vword;
+        const double s = cta_tree_reduce(thread_then_warp(leaf), warp_sums);
         if (threadIdx.x == 0) p.down_partials[blockIdx.x] = s;
+    }
+    if constexpr (TEL) {
+        double re, rv;
+        cta_tree_reduce_pair(thread_then_warp(te), thread_then_warp(tv), tel_sums, re, rv);
+        if (threadIdx.x == 0) { p.tel_e[blockIdx.x] = re; p.tel_v[blockIdx.x] = rv; }
     }
     (void)lane;
 }
@@ -396,15 +419,15 @@ __global__ void __launch_bounds__(THREADS) sumsq_kernel(const __grid_constant__ 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t row_beg = (int64_t)row * row_stride + ti.seg_beg;
     const GT *tile_ptr = src + row_beg + ti.rel;
-    const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
+    // (the source may be a message buffer, whose rows start on 4-byte boundaries only: look at the address)
+    const bool fast = (ti.len == TILE) && ((reinterpret_cast<uintptr_t>(tile_ptr) & (4 * sizeof(GT) - 1)) == 0);
     double a[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         float v[4];
         if (fast) load4_stream(tile_ptr + tile_pos(warp, lane, j), v);
         else load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v);
-        const double d0 = (double)v[0], d1 = (double)v[1], d2 = (double)v[2], d3 = (double)v[3];
-        a[j] = __dadd_rn(__dadd_rn(__dmul_rn(d0, d0), __dmul_rn(d1, d1)), __dadd_rn(__dmul_rn(d2, d2), __dmul_rn(d3, d3)));
+        a[j] = leaf4_sq(v);
     }
     double s = cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
     if (threadIdx.x == 0) p.tel_partials[(int64_t)row * p.TT + blockIdx.x] = s;
@@ -420,9 +443,9 @@ cudaError_t launch_sumsq(const Params &p, const void *src, int64_t row_stride, i
     return cudaGetLastError();
 }
 
-cudaError_t launch_sum_finalize(const Params &p, int rows, double *out, cudaStream_t st) {
+cudaError_t launch_sum_finalize(const Params &p, const double *partials, int rows, double *out, cudaStream_t st) {
     dim3 grid(p.T, rows);
-    scale_finalize_kernel<<<grid, THREADS, 0, st>>>(p, p.tel_partials, nullptr, out);
+    scale_finalize_kernel<<<grid, THREADS, 0, st>>>(p, partials, nullptr, out);
     return cudaGetLastError();
 }
 
@@ -440,21 +463,26 @@ cudaError_t launch_scale_finalize(const Params &p, bool uplink, cudaStream_t st)
     return cudaGetLastError();
 }
 
-template <typename GT>
+template <typename GT, bool TEL>
 static cudaError_t launch_server_dense_t(const Params &p, cudaStream_t st) {
-    if (p.down == COMP_SIGN) server_dense_kernel<true, GT><<<p.TT, THREADS, 0, st>>>(p);
-    else server_dense_kernel<false, GT><<<p.TT, THREADS, 0, st>>>(p);
+    if (p.down == COMP_SIGN) server_dense_kernel<true, GT, TEL><<<p.TT, THREADS, 0, st>>>(p);
+    else server_dense_kernel<false, GT, TEL><<<p.TT, THREADS, 0, st>>>(p);
     return cudaGetLastError();
 }
 
-cudaError_t launch_server_dense(const Params &p, cudaStream_t st) {
+template <bool TEL>
+static cudaError_t launch_server_dense_tel(const Params &p, cudaStream_t st) {
     if (p.up == COMP_SIGN) {
-        if (p.down == COMP_SIGN) server_sign_kernel<true><<<p.TT, THREADS, 0, st>>>(p);
-        else server_sign_kernel<false><<<p.TT, THREADS, 0, st>>>(p);
+        if (p.down == COMP_SIGN) server_sign_kernel<true, TEL><<<p.TT, THREADS, 0, st>>>(p);
+        else server_sign_kernel<false, TEL><<<p.TT, THREADS, 0, st>>>(p);
         return cudaGetLastError();
     }
-    if (p.gdt == DT_F32) return launch_server_dense_t<float>(p, st);
-    return launch_server_dense_t<__nv_bfloat16>(p, st);
+    if (p.gdt == DT_F32) return launch_server_dense_t<float, TEL>(p, st);
+    return launch_server_dense_t<__nv_bfloat16, TEL>(p, st);
+}
+
+cudaError_t launch_server_dense(const Params &p, cudaStream_t st) {
+    return p.telemetry ? launch_server_dense_tel<true>(p, st) : launch_server_dense_tel<false>(p, st);
 }
 
 cudaError_t launch_sign_error(const Params &p, cudaStream_t st) {

@@ -573,12 +573,14 @@ __global__ void __launch_bounds__(THREADS) topk_slow_kernel(const __grid_constan
 // fused with the first step of the downlink: first-digit histogram (top-k) or sign words and
 // ||v||_1 partial (scaled sign).
 // ------------------------------------------------------------------------------------------------
-template <int DOWN>
-__global__ void __launch_bounds__(THREADS, 4) server_topk_kernel(const __grid_constant__ Params p) {
+// TEL: also the tile's partial sums of e^2 (as read) and v^2 (as written), in tree order.
+template <int DOWN, bool TEL>
+__global__ void __launch_bounds__(THREADS, TEL ? 3 : 4) server_topk_kernel(const __grid_constant__ Params p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *acc = reinterpret_cast<float *>(smem_raw);                       // [TILE]
     uint32_t *h = reinterpret_cast<uint32_t *>(smem_raw + sizeof(float) * TILE);  // [DIGIT1_BINS] (top-k downlink)
     __shared__ double warp_sums[8];
+    __shared__ double tel_sums[TEL ? 16 : 1];
     __shared__ uint32_t s_beg[16], s_end[16];  // this tile's range in each message of the current group of workers
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -594,6 +596,13 @@ __global__ void __launch_bounds__(THREADS, 4) server_topk_kernel(const __grid_co
         const int pos = tile_pos(warp, lane, j);
         if (fast) load4_stream(e_tile + pos, ev[j]);
         else load4_guarded(e_tile, pos, ti.len, ev[j]);
+    }
+    double warp_e2 = 0.0;   // TEL: this warp's sum of e^2, kept while the messages are applied
+    if constexpr (TEL) {
+        double te[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) te[j] = leaf4_sq(ev[j]);
+        warp_e2 = warp_tree_reduce8(te, lane);
     }
     __syncthreads();
     const bool last_tile = (blockIdx.x + 1 == __ldg(p.tile_prefix + ti.t + 1));
@@ -645,6 +654,7 @@ __global__ void __launch_bounds__(THREADS, 4) server_topk_kernel(const __grid_co
     const int64_t wbase = __ldg(p.word_off + ti.t) + ti.rel / 32;
     const int nwords = (ti.len + 31) >> 5;
     double a[8];
+    double tv[TEL ? 8 : 1];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int pos = tile_pos(warp, lane, j);
@@ -660,6 +670,7 @@ __global__ void __launch_bounds__(THREADS, 4) server_topk_kernel(const __grid_co
             if (valid && __float_as_uint(v[c]) != __float_as_uint(ev[j][c])) e_tile[pos + c] = v[c];
             if (DOWN == COMP_TOPK && valid && ti.seg_tiles > 1) atomicAdd(&h[key_of(v[c]) >> DIGIT1_SHIFT], 1u);
         }
+        if constexpr (TEL) tv[j] = leaf4_sq(v);
         if (DOWN == COMP_SIGN) {
             a[j] = leaf4(v);
             uint32_t w = pack_word(sign_nibble(v), lane);
@@ -670,6 +681,11 @@ __global__ void __launch_bounds__(THREADS, 4) server_topk_kernel(const __grid_co
     if (DOWN == COMP_SIGN) {
         double sum = cta_tree_reduce(warp_tree_reduce8(a, lane), warp_sums);
         if (threadIdx.x == 0) p.down_partials[blockIdx.x] = sum;
+    }
+    if constexpr (TEL) {
+        double re, rv;
+        cta_tree_reduce_pair(warp_e2, warp_tree_reduce8(tv, lane), tel_sums, re, rv);
+        if (threadIdx.x == 0) { p.tel_e[blockIdx.x] = re; p.tel_v[blockIdx.x] = rv; }
     }
     if (DOWN == COMP_TOPK && ti.seg_tiles > 1) {   // (single-tile segments are selected directly from v)
         __syncthreads();
@@ -770,15 +786,12 @@ constexpr size_t SERVER_TOPK_SMEM = sizeof(float) * TILE + sizeof(uint32_t) * DI
 
 cudaError_t configure_topk_kernels() {
     cudaError_t e = configure_topk_tail_kernels();
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(server_topk_kernel<COMP_TOPK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)SERVER_TOPK_SMEM);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(server_topk_kernel<COMP_SIGN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)SERVER_TOPK_SMEM);
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(server_topk_kernel<COMP_IDENTITY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)SERVER_TOPK_SMEM);
+    const void *kernels[] = {(const void *)server_topk_kernel<COMP_TOPK, false>, (const void *)server_topk_kernel<COMP_SIGN, false>,
+                             (const void *)server_topk_kernel<COMP_IDENTITY, false>, (const void *)server_topk_kernel<COMP_TOPK, true>,
+                             (const void *)server_topk_kernel<COMP_SIGN, true>, (const void *)server_topk_kernel<COMP_IDENTITY, true>};
+    for (const void *k : kernels)
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SERVER_TOPK_SMEM);
+    return e;
 }
 
 // Single-tile segments of one side, selected directly (independent of everything else on that side:
@@ -791,10 +804,16 @@ cudaError_t launch_topk_small_segments(const Params &p, bool uplink, cudaStream_
     return e;
 }
 
+template <bool TEL>
+static void launch_server_topk_t(const Params &p, cudaStream_t st) {
+    if (p.down == COMP_TOPK) server_topk_kernel<COMP_TOPK, TEL><<<p.TT, THREADS, SERVER_TOPK_SMEM, st>>>(p);
+    else if (p.down == COMP_SIGN) server_topk_kernel<COMP_SIGN, TEL><<<p.TT, THREADS, SERVER_TOPK_SMEM, st>>>(p);
+    else server_topk_kernel<COMP_IDENTITY, TEL><<<p.TT, THREADS, SERVER_TOPK_SMEM, st>>>(p);
+}
+
 cudaError_t launch_server_topk(const Params &p, cudaStream_t st, int64_t *launches) {
-    if (p.down == COMP_TOPK) server_topk_kernel<COMP_TOPK><<<p.TT, THREADS, SERVER_TOPK_SMEM, st>>>(p);
-    else if (p.down == COMP_SIGN) server_topk_kernel<COMP_SIGN><<<p.TT, THREADS, SERVER_TOPK_SMEM, st>>>(p);
-    else server_topk_kernel<COMP_IDENTITY><<<p.TT, THREADS, SERVER_TOPK_SMEM, st>>>(p);
+    if (p.telemetry) launch_server_topk_t<true>(p, st);
+    else launch_server_topk_t<false>(p, st);
     CHECK_LAUNCH();
     return cudaSuccess;
 }

@@ -9,11 +9,14 @@
 
 namespace liec {
 
-template <int UP, int DOWN, typename GT>
-__global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK ? 3 : 0)) worker_update_kernel(const __grid_constant__ Params p, const float lr) {
+// TEL: the kernel also leaves, per (worker, tile), the binary64 partial sum of g^2 over the tile's
+// part of the summation tree (the gradient is in registers here anyway).
+template <int UP, int DOWN, typename GT, bool TEL>
+__global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK || TEL ? 3 : 0)) worker_update_kernel(const __grid_constant__ Params p, const float lr) {
     __shared__ __align__(16) float p_tile[DOWN == COMP_TOPK ? TILE : 4];  // decoded downlink message (top-k)
     // With a top-k downlink a CTA serves WPC workers so that the message is decoded once for them.
     constexpr int WPC = DOWN == COMP_TOPK ? 4 : 1;
+    __shared__ double tel_sums[TEL ? WPC : 1][TEL ? 8 : 1];
     __shared__ uint32_t own_mask[UP == COMP_RANDK ? WPC : 1][UP == COMP_RANDK ? TILE_WORDS : 1];  // each worker's own subset inside this tile
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -95,9 +98,11 @@ __global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK ? 3 : 0)) worker_u
         __syncthreads();
     }
 
+    double tg[TEL ? 8 : 1];   // TEL: this lane's sums of g^2, row by row, as the rows are consumed
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int pos = tile_pos(warp, lane, j);
+        if constexpr (TEL) tg[j] = leaf4_sq(g[j]);
         float pd[4];
         if (DOWN == COMP_SIGN) {
             uint32_t nib = nibble_from_words(my_word, lane, j);
@@ -138,6 +143,10 @@ __global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK ? 3 : 0)) worker_u
                 if (pos + c < ti.len) x_tile[pos + c] = x[j][c];
         }
     }
+    if constexpr (TEL) {
+        const double s = cta_tree_reduce(warp_tree_reduce8(tg, lane), tel_sums[wq]);
+        if (threadIdx.x == 0) p.tel_g[(int64_t)worker * p.TT + blockIdx.x] = s;
+    }
     }  // workers of this CTA
 }
 
@@ -145,8 +154,13 @@ template <int UP, int DOWN>
 static cudaError_t launch_t(const Params &p, float lr, cudaStream_t st) {
     constexpr int WPC = DOWN == COMP_TOPK ? 4 : 1;
     dim3 grid(p.TT, (p.N + WPC - 1) / WPC);
-    if (p.gdt == DT_F32) worker_update_kernel<UP, DOWN, float><<<grid, THREADS, 0, st>>>(p, lr);
-    else worker_update_kernel<UP, DOWN, __nv_bfloat16><<<grid, THREADS, 0, st>>>(p, lr);
+    if (p.telemetry) {
+        if (p.gdt == DT_F32) worker_update_kernel<UP, DOWN, float, true><<<grid, THREADS, 0, st>>>(p, lr);
+        else worker_update_kernel<UP, DOWN, __nv_bfloat16, true><<<grid, THREADS, 0, st>>>(p, lr);
+    } else {
+        if (p.gdt == DT_F32) worker_update_kernel<UP, DOWN, float, false><<<grid, THREADS, 0, st>>>(p, lr);
+        else worker_update_kernel<UP, DOWN, __nv_bfloat16, false><<<grid, THREADS, 0, st>>>(p, lr);
+    }
     return cudaGetLastError();
 }
 

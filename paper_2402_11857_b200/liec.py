@@ -83,6 +83,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.liec_mean_params.restype = C.c_int
     lib.liec_sumsq.argtypes = [vp, C.c_int32, vp, vp, vp]
     lib.liec_sumsq.restype = C.c_int
+    lib.liec_set_telemetry.argtypes = [vp, C.c_int32]
+    lib.liec_set_telemetry.restype = C.c_int
+    lib.liec_get_telemetry.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.liec_get_telemetry.restype = C.c_int
     lib.liec_step_host.argtypes = [vp, vp, vp, C.c_float, vp, vp]
     lib.liec_step_host.restype = C.c_int
     lib.liec_get_messages.argtypes = [vp, C.POINTER(liec_messages)]
@@ -277,6 +281,25 @@ class Context:
             self._check_grads(grads)
             gptr = grads.data_ptr()
         self._check(self.lib.liec_sumsq(self._ctx, int(which), gptr, out.data_ptr(), self._stream(stream)))
+
+    def liec_set_telemetry(self, on: bool):
+        self._check(self.lib.liec_set_telemetry(self._ctx, 1 if on else 0))
+
+    def liec_get_telemetry(self, stream=None, kept: bool = True) -> dict:
+        """Per-segment squared norms of the last iteration (float64 CUDA tensors, allocated here):
+        e_sumsq [T], v_sumsq [T], g_sumsq [N, T] and, for sides with (index, value) messages and
+        kept=True, up_kept_sumsq [N, T] / down_kept_sumsq [T]."""
+        t = self._torch
+        dev, f64 = self.params.device, t.float64
+        sparse = (COMP_TOPK, COMP_RANDK)
+        out = {"e_sumsq": t.empty(self.T, dtype=f64, device=dev), "v_sumsq": t.empty(self.T, dtype=f64, device=dev),
+               "g_sumsq": t.empty(self.N, self.T, dtype=f64, device=dev),
+               "up_kept_sumsq": t.empty(self.N, self.T, dtype=f64, device=dev) if kept and self.cfg.uplink in sparse else None,
+               "down_kept_sumsq": t.empty(self.T, dtype=f64, device=dev) if kept and self.cfg.downlink in sparse else None}
+        ptr = lambda name: None if out[name] is None else out[name].data_ptr()
+        self._check(self.lib.liec_get_telemetry(self._ctx, ptr("e_sumsq"), ptr("v_sumsq"), ptr("g_sumsq"),
+                                                ptr("up_kept_sumsq"), ptr("down_kept_sumsq"), self._stream(stream)))
+        return out
 
     def liec_step_host(self, grads_host, grads_dev, lr: float, down_msg_host=None, stream=None):
         self._check_grads(grads_dev)
