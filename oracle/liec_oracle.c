@@ -34,9 +34,12 @@
  *   - top-k compares magnitudes through the binary32 bit pattern with the sign
  *     bit cleared; among equal magnitudes the lower index wins, so the selected
  *     set is unique.  The message lists (index, value) ascending by index.
- *   - random-k draws nothing here: the k_t-subset of every segment (one per worker for the
- *     uplink, one for the downlink) is an input, listed as flat indices ascending inside the
- *     segment; the caller samples it uniformly (Def. 3).  The message has the top-k layout.
+ *   - random-k: the k_t-subset of every segment (one per worker for the uplink, one for the
+ *     downlink) is an input of the iteration, listed as flat indices ascending inside the
+ *     segment (Def. 3 wants it uniform over the k_t-subsets).  The message has the top-k layout.
+ *     liec_oracle_draw_subsets below is the seeded draw of such subsets: every element gets a
+ *     pseudo-random score from a counter-based generator and the k_t highest scores of a segment
+ *     are its subset (equal scores: lower index first).
  *   - The server sums messages in worker order in binary32 starting from +0,
  *     divides by (float)N, then adds e.
  *   - The update is evaluated left to right as printed: ((p - p^i) + g), times
@@ -371,4 +374,115 @@ int liec_oracle_average_step(int32_t N, int64_t d, const float *G, float lr, flo
     if (xbar_out) memcpy(xbar_out, xbar, (size_t)d * sizeof(float));
     free(v); free(xbar);
     return 0;
+}
+
+/* ---- seeded draw of the random-k subsets (Def. 3) ----------------------------------------
+ *
+ * Def. 3 asks for S uniform over the k-element subsets of a segment.  Ranking the elements by
+ * independent, identically distributed scores and keeping the k highest gives exactly that (the
+ * ranking is a uniformly random permutation), up to equal scores, which go to the lower index.
+ * The scores come from the counter-based generator Philox4x32-10 (Salmon, Moraes, Dror, Shaw:
+ * "Parallel random numbers: as easy as 1, 2, 3", SC 2011), so that a sender and a receiver who
+ * share (seed, epoch) compute the same subsets without exchanging indices:
+ *
+ *   key     = (seed mod 2^32, seed div 2^32)
+ *   counter = (q, t, row, epoch)   q = block of four consecutive elements of segment t,
+ *                                  row = worker index for an uplink subset, N for the server's
+ *   the four output words go to elements 4q, 4q+1, 4q+2, 4q+3 of the segment (in that order)
+ *   score   = word >> 2            (30 bits)
+ */
+
+static void philox_round(uint32_t c[4], const uint32_t k[2])
+{
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c[0];
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c[2];
+    const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+    const uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+    const uint32_t n0 = hi1 ^ c[1] ^ k[0];
+    const uint32_t n2 = hi0 ^ c[3] ^ k[1];
+    c[0] = n0; c[1] = lo1; c[2] = n2; c[3] = lo0;
+}
+
+/* Philox4x32 with 10 rounds: out = the block for this counter and key. */
+void liec_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c[4] = { ctr[0], ctr[1], ctr[2], ctr[3] };
+    uint32_t k[2] = { key[0], key[1] };
+    for (int r = 0; r < 10; ++r) {
+        if (r > 0) { k[0] += 0x9E3779B9u; k[1] += 0xBB67AE85u; }   /* key schedule: Weyl sequence */
+        philox_round(c, k);
+    }
+    out[0] = c[0]; out[1] = c[1]; out[2] = c[2]; out[3] = c[3];
+}
+
+/* Scores of the n elements of segment t for the subset of `row` in draw `epoch`. */
+void liec_oracle_subset_scores(uint64_t seed, uint32_t epoch, uint32_t row, uint32_t t,
+                               int64_t n, uint32_t *scores)
+{
+    const uint32_t key[2] = { (uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32) };
+    for (int64_t j = 0; j < n; ++j) {
+        const uint32_t ctr[4] = { (uint32_t)(j / 4), t, row, epoch };
+        uint32_t out[4];
+        liec_oracle_philox4x32_10(ctr, key, out);
+        scores[j] = out[j % 4] >> 2;
+    }
+}
+
+typedef struct { uint32_t score; uint32_t pos; } scorepos;
+
+static int by_score_then_index(const void *a, const void *b)
+{
+    const scorepos *p = (const scorepos *)a, *q = (const scorepos *)b;
+    if (p->score != q->score) return p->score > q->score ? -1 : 1;   /* higher score first */
+    if (p->pos != q->pos) return p->pos > q->pos ? 1 : -1;           /* lower index first */
+    return 0;
+}
+
+static int by_value(const void *a, const void *b)
+{
+    const uint32_t x = *(const uint32_t *)a, y = *(const uint32_t *)b;
+    return x < y ? -1 : (x > y ? 1 : 0);
+}
+
+/* The k positions (0-based inside the segment) with the highest scores, ascending.  Returns 0,
+ * or -1 when memory runs out. */
+int liec_oracle_subset_from_scores(const uint32_t *scores, int64_t n, int64_t k, uint32_t *subset)
+{
+    scorepos *order = (scorepos *)malloc((size_t)n * sizeof(scorepos));
+    if (!order) return -1;
+    for (int64_t j = 0; j < n; ++j) { order[j].score = scores[j]; order[j].pos = (uint32_t)j; }
+    qsort(order, (size_t)n, sizeof(scorepos), by_score_then_index);
+    for (int64_t r = 0; r < k; ++r) subset[r] = order[r].pos;
+    qsort(subset, (size_t)k, sizeof(uint32_t), by_value);
+    free(order);
+    return 0;
+}
+
+/* The subsets of `rows` rows (workers 0..N-1, then the server as row N when rows = N+1) for
+ * every segment: sets [rows][K] flat indices, segment after segment, ascending inside a
+ * segment; the layout liec_oracle_step_sets takes.  Returns 0, or -1 when memory runs out. */
+int liec_oracle_draw_subsets(uint64_t seed, uint32_t epoch, int32_t rows, int32_t T,
+                             const int64_t *off, const int64_t *k, uint32_t *sets)
+{
+    int64_t K = 0, nmax = 0;
+    for (int32_t t = 0; t < T; ++t) {
+        K += k[t];
+        if (off[t + 1] - off[t] > nmax) nmax = off[t + 1] - off[t];
+    }
+    uint32_t *scores = (uint32_t *)malloc((size_t)nmax * sizeof(uint32_t));
+    if (!scores) return -1;
+    int rc = 0;
+    for (int32_t row = 0; row < rows && rc == 0; ++row) {
+        int64_t koff = 0;
+        for (int32_t t = 0; t < T && rc == 0; ++t) {
+            const int64_t n = off[t + 1] - off[t];
+            uint32_t *dst = sets + (size_t)row * K + koff;
+            liec_oracle_subset_scores(seed, epoch, (uint32_t)row, (uint32_t)t, n, scores);
+            rc = liec_oracle_subset_from_scores(scores, n, k[t], dst);
+            for (int64_t r = 0; r < k[t]; ++r) dst[r] += (uint32_t)off[t];   /* flat index */
+            koff += k[t];
+        }
+    }
+    free(scores);
+    return rc;
 }

@@ -60,6 +60,14 @@ def _bind(lib: C.CDLL) -> C.CDLL:
     lib.liec_oracle_step.argtypes = [C.c_int32, C.c_int64, C.c_int32, p, C.c_int32, C.c_int32, p,
                                      p, C.c_float, p, p] + [p] * 9
     lib.liec_oracle_step.restype = C.c_int
+    lib.liec_oracle_philox4x32_10.argtypes = [p, p, p]
+    lib.liec_oracle_philox4x32_10.restype = None
+    lib.liec_oracle_subset_scores.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_int64, p]
+    lib.liec_oracle_subset_scores.restype = None
+    lib.liec_oracle_subset_from_scores.argtypes = [p, C.c_int64, C.c_int64, p]
+    lib.liec_oracle_subset_from_scores.restype = C.c_int
+    lib.liec_oracle_draw_subsets.argtypes = [C.c_uint64, C.c_uint32, C.c_int32, C.c_int32, p, p, p]
+    lib.liec_oracle_draw_subsets.restype = C.c_int
     lib.liec_oracle_mean_params.argtypes = [C.c_int32, C.c_int64, p, p]
     lib.liec_oracle_mean_params.restype = None
     lib.liec_oracle_average_step.argtypes = [C.c_int32, C.c_int64, p, C.c_float, p, p, p, p]
@@ -249,3 +257,42 @@ def average_step(X: np.ndarray, e: np.ndarray, G: np.ndarray, lr: float, _lib=No
     if rc:
         raise MemoryError("oracle average step out of memory")
     return v, xbar
+
+
+def philox4x32_10(ctr, key, _lib=None) -> np.ndarray:
+    """One block of the counter-based generator behind the seeded subset draw."""
+    c = np.ascontiguousarray(ctr, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    assert c.shape == (4,) and k.shape == (2,)
+    out = np.empty(4, np.uint32)
+    (_lib or lib()).liec_oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def subset_scores(seed: int, epoch: int, row: int, t: int, n: int, _lib=None) -> np.ndarray:
+    out = np.empty(n, np.uint32)
+    (_lib or lib()).liec_oracle_subset_scores(int(seed), int(epoch), int(row), int(t), int(n), _ptr(out))
+    return out
+
+
+def subset_from_scores(scores, k: int, _lib=None) -> np.ndarray:
+    """Positions of the k highest scores (equal scores: lower index first), ascending."""
+    sc = np.ascontiguousarray(scores, dtype=np.uint32)
+    out = np.empty(int(k), np.uint32)
+    rc = (_lib or lib()).liec_oracle_subset_from_scores(_ptr(sc), sc.size, int(k), _ptr(out))
+    if rc:
+        raise MemoryError("oracle subset selection out of memory")
+    return out
+
+
+def draw_subsets(seed: int, epoch: int, rows: int, off, k, _lib=None) -> np.ndarray:
+    """Seeded random-k subsets (Def. 3) of `rows` rows: [rows, K] flat indices, ascending inside
+    each segment.  Row i < N is worker i's subset, row N the server's."""
+    off = _off(off)
+    k = np.ascontiguousarray(k, dtype=np.int64)
+    T = off.size - 1
+    out = np.empty((int(rows), int(k.sum())), np.uint32)
+    rc = (_lib or lib()).liec_oracle_draw_subsets(int(seed), int(epoch), int(rows), T, _ptr(off), _ptr(k), _ptr(out))
+    if rc:
+        raise MemoryError("oracle subset draw out of memory")
+    return out

@@ -582,6 +582,145 @@ def pin_sumsq_tree_shape(L):
     assert t([-3, 4]) == 25.0
 
 
+# ----------------------------------------------------------------------------- seeded subsets (Def. 3)
+
+def _philox_kat():
+    rows = []
+    with open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")) as fh:
+        for line in fh:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            ctr, key, out = (tuple(int(w, 16) for w in part.split()) for part in line.split("|"))
+            rows.append((ctr, key, out))
+    assert len(rows) == 3
+    return rows
+
+
+def pin_philox_known_answers(L):
+    """The generator against its published known-answer vectors."""
+    for ctr, key, out in _philox_kat():
+        got = oracle.philox4x32_10(ctr, key, _lib=L)
+        assert tuple(int(w) for w in got) == out, (ctr, key, [hex(int(w)) for w in got])
+
+
+def pin_subset_scores_layout(L):
+    """Which counter word, key word and output word go where, from the published vectors alone:
+    seed 0, epoch 0, row 0, segment 0 is counter (0,0,0,0) under key (0,0), whose block the first
+    vector gives; elements 0..3 take its words in order, shifted right by two."""
+    (_, _, out0) = _philox_kat()[0]
+    sc = oracle.subset_scores(0, 0, 0, 0, 4, _lib=L)
+    assert [int(v) for v in sc] == [w >> 2 for w in out0]
+    # the two highest of (6627e8d5, e169c58d, bc57ac4c, 9b00dbd8) are elements 1 and 2; the highest is 1
+    assert list(oracle.subset_from_scores(sc, 2, _lib=L)) == [1, 2]
+    assert list(oracle.subset_from_scores(sc, 1, _lib=L)) == [1]
+    assert list(oracle.subset_from_scores(sc, 3, _lib=L)) == [1, 2, 3]
+    # the third vector, read as (block, segment, row, epoch) under seed = k1:k0
+    (c, k, out) = _philox_kat()[2]
+    seed = (k[1] << 32) | k[0]
+    blk = oracle.philox4x32_10(c, k, _lib=L)
+    assert tuple(int(w) for w in blk) == out
+    # element 4q+m of (segment c1, row c2, epoch c3) has block q = c0: too far out to list a segment
+    # of that length, so take q = 1 and check it against the block function itself, word by word,
+    # and that every one of the six inputs matters
+    base = dict(seed=seed, epoch=c[3], row=c[2], t=c[1])
+    sc = oracle.subset_scores(base["seed"], base["epoch"], base["row"], base["t"], 8, _lib=L)
+    want = oracle.philox4x32_10((1, c[1], c[2], c[3]), k, _lib=L)
+    assert [int(v) for v in sc[4:8]] == [int(w) >> 2 for w in want]
+    for name, other in (("seed", seed ^ 1), ("seed", seed ^ (1 << 32)), ("epoch", c[3] ^ 1), ("row", c[2] ^ 1), ("t", c[1] ^ 1)):
+        changed = dict(base, **{name: other})
+        sc2 = oracle.subset_scores(changed["seed"], changed["epoch"], changed["row"], changed["t"], 8, _lib=L)
+        assert not np.array_equal(sc, sc2), name
+    # swapping two of the inputs is not the same draw either
+    assert not np.array_equal(oracle.subset_scores(5, 1, 2, 3, 8, _lib=L), oracle.subset_scores(5, 2, 1, 3, 8, _lib=L))
+    assert not np.array_equal(oracle.subset_scores(5, 1, 2, 3, 8, _lib=L), oracle.subset_scores(5, 1, 3, 2, 8, _lib=L))
+    assert not np.array_equal(oracle.subset_scores(5, 1, 2, 3, 8, _lib=L), oracle.subset_scores(5, 3, 2, 1, 8, _lib=L))
+
+
+def pin_subset_from_scores_is_uniform(L):
+    """Ranking by scores: over all orderings of distinct scores every k-subset comes out equally
+    often (Def. 3 asks for the uniform distribution over k-subsets), listed ascending; equal
+    scores go to the lower index (checked against a plain Python sort over every score vector
+    from a three-letter alphabet)."""
+    import itertools
+    n = 5
+    for k in (1, 2, 3, 5):
+        counts = {}
+        for perm in itertools.permutations(range(10, 10 + n)):
+            sub = tuple(int(v) for v in oracle.subset_from_scores(np.asarray(perm, np.uint32) * 1000003, k, _lib=L))
+            assert list(sub) == sorted(set(sub)) and len(sub) == k and all(0 <= j < n for j in sub)
+            top = tuple(sorted(sorted(range(n), key=lambda j: -perm[j])[:k]))
+            assert sub == top
+            counts[sub] = counts.get(sub, 0) + 1
+        assert len(counts) == math.comb(n, k) and len(set(counts.values())) == 1, (k, counts)
+    for scores in itertools.product((0, 7, 9), repeat=4):
+        for k in (1, 2, 3, 4):
+            want = sorted(sorted(range(4), key=lambda j: (-scores[j], j))[:k])
+            got = [int(v) for v in oracle.subset_from_scores(np.asarray(scores, np.uint32), k, _lib=L)]
+            assert got == want, (scores, k, got, want)
+
+
+def pin_subset_draw_layout(L):
+    """draw_subsets: row r, segment t holds flat indices of segment t, k_t of them, ascending, equal to
+    the ranking of that (row, segment)'s own scores; rows differ; the iteration accepts them."""
+    off = np.asarray([0, 5, 6, 40, 173], np.int64)
+    k = np.asarray([2, 1, 34, 17], np.int64)
+    rows, seed, epoch = 4, 0x1234567890abcdef, 7
+    sets = oracle.draw_subsets(seed, epoch, rows, off, k, _lib=L)
+    koff = np.concatenate([[0], np.cumsum(k)])
+    assert sets.shape == (rows, int(k.sum()))
+    for r in range(rows):
+        for t in range(4):
+            n = int(off[t + 1] - off[t])
+            sc = oracle.subset_scores(seed, epoch, r, t, n, _lib=L)
+            want = sorted(sorted(range(n), key=lambda j: (-int(sc[j]), j))[:int(k[t])])
+            got = [int(v) for v in sets[r, koff[t]:koff[t + 1]]]
+            assert got == [int(off[t]) + j for j in want], (r, t)
+    assert list(sets[0, koff[2]:koff[3]]) == list(range(6, 40))        # k_t = n_t keeps the whole segment
+    assert not np.array_equal(sets[0], sets[1])
+    assert not np.array_equal(sets, oracle.draw_subsets(seed, epoch + 1, rows, off, k, _lib=L))
+    assert np.array_equal(sets, oracle.draw_subsets(seed, epoch, rows, off, k, _lib=L))
+    rng = np.random.default_rng(5)
+    N = rows - 1
+    G = rng.standard_normal((N, 173)).astype(np.float32)
+    X = np.zeros((N, 173), np.float32)
+    e = np.zeros(173, np.float32)
+    r = oracle.step(X, e, G, 0.1, off, RANDK, RANDK, k=k, up_sets=sets[:N], down_set=sets[N], _lib=L)
+    assert np.array_equal(r.up_idx, sets[:N]) and np.array_equal(r.down_idx, sets[N])
+
+
+def pin_subset_statistics(L):
+    """Over many draws: every element is kept with frequency k/n, every pair with k(k-1)/(n(n-1)), and
+    E ||C(x) - x||^2 = (1 - k/n) ||x||^2 (Assumption 4 with delta = k/d, the value the paper states for
+    random-k), all within five standard deviations of the uniform law."""
+    n, k, draws = 24, 6, 6000
+    off, karr = np.asarray([0, n], np.int64), np.asarray([k], np.int64)
+    single = np.zeros(n)
+    pair = np.zeros((n, n))
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal(n)
+    resid = 0.0
+    for epoch in range(draws):
+        sub = oracle.draw_subsets(99, epoch, 1, off, karr, _lib=L)[0].astype(np.int64)
+        single[sub] += 1
+        pair[np.ix_(sub, sub)] += 1
+        keep = np.zeros(n, bool)
+        keep[sub] = True
+        resid += float(np.sum(x[~keep] ** 2))
+    p1 = k / n
+    assert np.all(np.abs(single / draws - p1) < 5 * math.sqrt(p1 * (1 - p1) / draws)), single / draws
+    p2 = k * (k - 1) / (n * (n - 1))
+    offdiag = pair[~np.eye(n, dtype=bool)] / draws
+    assert np.all(np.abs(offdiag - p2) < 5 * math.sqrt(p2 * (1 - p2) / draws)), (offdiag.min(), offdiag.max(), p2)
+    want = (1 - k / n) * float(np.sum(x ** 2))
+    assert abs(resid / draws - want) < 0.03 * want, (resid / draws, want)
+    # different rows and different seeds are different streams with the same law
+    a = oracle.draw_subsets(1, 0, 64, np.asarray([0, 4096], np.int64), np.asarray([41], np.int64), _lib=L)
+    assert len({tuple(r) for r in a}) == 64
+    flat = np.bincount(a.ravel(), minlength=4096)
+    assert flat.max() <= 6      # 64 * 41 draws over 4096 positions: no position favoured
+
+
 ALL_PINS = [
     pin_golden_sign, pin_golden_blockwise, pin_golden_topk,
     pin_scale_is_exact_mean, pin_tree_shape, pin_sign_bits_bruteforce, pin_sign_contraction,
@@ -589,4 +728,6 @@ ALL_PINS = [
     pin_error_recursion, pin_identity_one_worker_is_sgd, pin_identical_workers,
     pin_lemma3_exact, pin_lemma3_float, pin_bf16_widening, pin_sumsq_tree_shape, pin_golden_averaging, pin_averaging_properties, pin_sumsq_and_delta,
     pin_randk_all_subsets, pin_randk_segments_and_rejects, pin_randk_step_special_cases,
+    pin_philox_known_answers, pin_subset_scores_layout, pin_subset_from_scores_is_uniform, pin_subset_draw_layout,
+    pin_subset_statistics,
 ]

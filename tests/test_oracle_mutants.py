@@ -50,6 +50,22 @@ MUTANTS = {
     "randk_order_check_dropped": ("if (r > 0 && set[q - 1] >= set[q]) return -3;", ""),
     "randk_every_worker_uses_first_subset": ("up_sets ? up_sets + (size_t)i * K : NULL", "up_sets"),
     "randk_downlink_uses_uplink_subset": ("rc = compress(down, v, d, T, off, k, down_set,", "rc = compress(down, v, d, T, off, k, up_sets,"),
+    "philox_nine_rounds": ("for (int r = 0; r < 10; ++r) {", "for (int r = 0; r < 9; ++r) {"),
+    "philox_multipliers_swapped": ("const uint64_t p0 = (uint64_t)0xD2511F53u * c[0];\n    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c[2];",
+                                   "const uint64_t p0 = (uint64_t)0xCD9E8D57u * c[0];\n    const uint64_t p1 = (uint64_t)0xD2511F53u * c[2];"),
+    "philox_key_bumped_before_first_round": ("if (r > 0) { k[0] += 0x9E3779B9u; k[1] += 0xBB67AE85u; }", "{ k[0] += 0x9E3779B9u; k[1] += 0xBB67AE85u; }"),
+    "philox_halves_not_crossed": ("const uint32_t n0 = hi1 ^ c[1] ^ k[0];\n    const uint32_t n2 = hi0 ^ c[3] ^ k[1];",
+                                  "const uint32_t n0 = hi0 ^ c[1] ^ k[0];\n    const uint32_t n2 = hi1 ^ c[3] ^ k[1];"),
+    "subset_words_in_reverse_order": ("scores[j] = out[j % 4] >> 2;", "scores[j] = out[3 - j % 4] >> 2;"),
+    "subset_score_keeps_31_bits": ("scores[j] = out[j % 4] >> 2;", "scores[j] = out[j % 4] >> 1;"),
+    "subset_row_and_epoch_swapped": ("const uint32_t ctr[4] = { (uint32_t)(j / 4), t, row, epoch };", "const uint32_t ctr[4] = { (uint32_t)(j / 4), t, epoch, row };"),
+    "subset_one_block_per_element": ("const uint32_t ctr[4] = { (uint32_t)(j / 4), t, row, epoch };", "const uint32_t ctr[4] = { (uint32_t)j, t, row, epoch };"),
+    "subset_seed_high_half_ignored": ("(uint32_t)(seed >> 32) };", "0u };"),
+    "subset_lowest_scores": ("return p->score > q->score ? -1 : 1;", "return p->score > q->score ? 1 : -1;"),
+    "subset_tie_higher_index": ("return p->pos > q->pos ? 1 : -1;", "return p->pos > q->pos ? -1 : 1;"),
+    "subset_not_sorted": ("qsort(subset, (size_t)k, sizeof(uint32_t), by_value);", ""),
+    "subset_indices_segment_relative": ("for (int64_t r = 0; r < k[t]; ++r) dst[r] += (uint32_t)off[t];   /* flat index */", ""),
+    "subset_same_for_every_row": ("liec_oracle_subset_scores(seed, epoch, (uint32_t)row, (uint32_t)t, n, scores);", "liec_oracle_subset_scores(seed, epoch, 0u, (uint32_t)t, n, scores);"),
     "ascent_instead_of_descent": ("x[j] = x[j] - step;", "x[j] = x[j] + step;"),
 }
 
