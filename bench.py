@@ -38,6 +38,9 @@ def resolve_workload(name: str):
     from liec_synth import WORKLOADS, flat_layout, scaled_layout, topk_counts
     base, _, div = name.partition("/")
     base, _, variant = base.partition("-")
+    seeded = variant == "randkseed"   # random-k with the subsets drawn on the GPU from (seed, step) every iteration
+    if seeded:
+        variant = "randk"
     if base in WORKLOADS and variant in ("", "randk", "topk", "sign"):
         w = WORKLOADS[base]
         lay = w.layout()
@@ -49,7 +52,7 @@ def resolve_workload(name: str):
         frac = w.topk_frac if w.topk_frac[0] else (1, 100)
         k = topk_counts(lay, *frac) if comp in ("topk", "randk") else None
         return dict(name=name, N=w.num_workers, layout=lay, dist=w.dist, scale=w.scale, comp=comp,
-                    k=k, lr=w.lr, gdt=w.grad_dtype)
+                    k=k, lr=w.lr, gdt=w.grad_dtype, seeded=seeded)
     if name.startswith("sweep-"):
         # sweep-sign-26, sweep-topk1000-28 (k = n/1000), sweep-topk100-24 (k = n/100),
         # sweep-randk100-26 (random-k, k = n/100): N=8, flat, N(0,1)
@@ -349,7 +352,8 @@ def run_gpu(args, w, rank, world, local_rank, steps=None, extras=True):
     batches = [make_gradients(w["dist"], w["scale"], N, d, step=b, base_seed=1000 + rank, device=dev)
                for b in range(NUM_BATCHES)]
     G = batches[0]
-    if w["comp"] == "randk":   # the subsets are inputs: drawn once on the host, resident like the gradients
+    seeded = bool(w.get("seeded"))
+    if w["comp"] == "randk" and not seeded:   # the subsets are inputs: drawn once on the host, resident like the gradients
         import numpy as np
         from liec_synth import random_subsets
         sets = random_subsets(lay.seg_offsets, w["k"], N + 1, 0, 1000 + rank)
@@ -370,9 +374,13 @@ def run_gpu(args, w, rank, world, local_rank, steps=None, extras=True):
         g = batches[counter[0] % NUM_BATCHES]
         counter[0] += 1
         if events is None:
+            if seeded:
+                ctx.liec_draw_subsets(1000 + rank, counter[0])
             ctx.liec_step(g, w["lr"])
             return
         events[0].record()
+        if seeded:   # (the draw is timed as part of the uplink stage)
+            ctx.liec_draw_subsets(1000 + rank, counter[0])
         ctx.liec_uplink_compress(g); events[1].record()
         ctx.liec_server_aggregate(); events[2].record()
         ctx.liec_downlink_compress(); events[3].record()

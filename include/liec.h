@@ -151,8 +151,9 @@ liec_status liec_worker_update(liec_ctx *ctx, const void *grads, float lr, void 
 
 /*
  * Random-k (Def. 3: keep the entries of a k_t-subset of every segment, the subset drawn uniformly
- * from all k_t-subsets).  The library draws nothing: the caller samples the subsets and hands them
- * over before the iteration that uses them.
+ * from all k_t-subsets) with subsets brought by the caller: the caller samples them and hands them
+ * over before the iteration that uses them (liec_draw_subsets is the alternative that draws them
+ * on the GPU from a seed).
  *   up_sets   device, [N][K] uint32, K = sum_t k_t: for worker i and segment t the k_t kept flat
  *             indices (positions in [0, d)), listed segment after segment, strictly ascending
  *             inside a segment.  Needed iff the uplink is RANDK, else may be NULL.
@@ -168,6 +169,37 @@ liec_status liec_worker_update(liec_ctx *ctx, const void *grads, float lr, void 
  * subset.
  */
 liec_status liec_set_subsets(liec_ctx *ctx, const uint32_t *up_sets, const uint32_t *down_set);
+
+/*
+ * Random-k with a seed instead of index lists (Def. 3: S uniform over the k_t-subsets of a segment;
+ * Assumption 4).  Draws the subsets of all N workers and of the server on the GPU and installs them
+ * as liec_set_subsets would, without any list crossing the PCIe bus.  Two parties that share
+ * (seed, epoch) compute the same subsets, so a message needs to carry the values only
+ * (liec_wire_bytes_seeded).  Specification (bit-exact with a plain CPU restatement):
+ *   - every element gets a score from the counter-based generator Philox4x32-10 (Salmon, Moraes,
+ *     Dror, Shaw, SC 2011): key = (seed mod 2^32, seed div 2^32); counter = (q, t, row, epoch) with
+ *     q the block of four consecutive elements of segment t (element j of the segment lies in block
+ *     j div 4 and takes output word j mod 4), row = i for worker i and N for the server;
+ *     score = word >> 2 (30 bits);
+ *   - the subset of (row, t) is the k_t elements of the segment with the highest scores, equal scores
+ *     going to the lower index; listed ascending.
+ * Ranking by independent uniform scores gives every k_t-subset the same probability; equal scores at
+ * the cut (probability about n_t / 2^30 per draw) are the only departure from it.
+ * The draw is a top-k selection on a computed vector and runs through the top-k kernels; its cost is
+ * about one dense pass of integer arithmetic over N+1 rows.  The lists live in the workspace and stay
+ * in use until the next liec_draw_subsets or liec_set_subsets; call it before every iteration with a
+ * new epoch (e.g. the iteration number) to redraw, or less often to keep the subsets.
+ * LIEC_ERR_STATE between the stages of an iteration; LIEC_ERR_INVALID_ARG when no side is RANDK.
+ */
+liec_status liec_draw_subsets(liec_ctx *ctx, uint64_t seed, uint32_t epoch, void *stream);
+
+/*
+ * As liec_wire_bytes, for parties that share the seed of liec_draw_subsets: a RANDK message then
+ * carries its k_t values per segment and no indices (4 K bytes instead of 8 K).  Other operators
+ * are charged as in liec_wire_bytes.
+ */
+liec_status liec_wire_bytes_seeded(const liec_config *cfg, int64_t *uplink_bytes, int64_t *downlink_bytes,
+                                   int64_t *full_precision_bytes);
 
 /*
  * The four stages in sequence (one iteration of Algorithm 1's compressed branch); produces the same

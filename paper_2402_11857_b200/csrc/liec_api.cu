@@ -12,6 +12,7 @@
 #include "../../include/liec.h"
 #include "kernels.h"
 #include "plan.h"
+#include "topk_common.cuh"
 
 using namespace liec;
 
@@ -35,6 +36,7 @@ struct Plan {
     Region r_up_hist, r_down_hist, r_up_hist2, r_down_hist2, r_up_sel, r_down_sel;
     Region r_up_cand_idx, r_up_cand_val, r_down_cand_idx, r_down_cand_val;
     Region r_up_tile_meta, r_down_tile_meta, r_up_outbase, r_down_outbase;
+    Region r_gen_sets, r_gen_val, r_gen_hist, r_gen_hist2, r_gen_sel, r_gen_cand_idx, r_gen_cand_val, r_gen_meta, r_gen_outbase;
     size_t total = 0;
 };
 
@@ -194,6 +196,9 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     };
     if (cfg->uplink == LIEC_COMP_RANDK) randk_regions(N, pl.r_up_idx, pl.r_up_val, pl.r_up_outbase);
     if (cfg->downlink == LIEC_COMP_RANDK) randk_regions(1, pl.r_down_idx, pl.r_down_val, pl.r_down_outbase);
+    if (cfg->uplink == LIEC_COMP_RANDK || cfg->downlink == LIEC_COMP_RANDK)   // scratch of the seeded draw (liec_draw_subsets)
+        topk_regions(N + 1, pl.r_gen_sets, pl.r_gen_val, pl.r_gen_hist, pl.r_gen_hist2, pl.r_gen_sel, pl.r_gen_cand_idx,
+                     pl.r_gen_cand_val, pl.r_gen_meta, pl.r_gen_outbase);
     if (cfg->uplink == LIEC_COMP_TOPK)
         topk_regions(N, pl.r_up_idx, pl.r_up_val, pl.r_up_hist, pl.r_up_hist2, pl.r_up_sel, pl.r_up_cand_idx,
                      pl.r_up_cand_val, pl.r_up_tile_meta, pl.r_up_outbase);
@@ -283,8 +288,8 @@ size_t liec_workspace_bytes(const liec_config *cfg) {
     return pl.total;
 }
 
-liec_status liec_wire_bytes(const liec_config *cfg, int64_t *uplink_bytes, int64_t *downlink_bytes,
-                            int64_t *full_precision_bytes) {
+static liec_status wire_bytes(const liec_config *cfg, bool shared_seed, int64_t *uplink_bytes, int64_t *downlink_bytes,
+                              int64_t *full_precision_bytes) {
     Plan pl;
     std::string msg;
     liec_status st = make_plan(cfg, pl, &msg);
@@ -294,6 +299,7 @@ liec_status liec_wire_bytes(const liec_config *cfg, int64_t *uplink_bytes, int64
     }
     auto message = [&](int32_t comp) -> int64_t {
         if (comp == LIEC_COMP_SCALED_SIGN) return 4 * (pl.W + (int64_t)pl.T);  // packed signs + one scale per segment
+        if (comp == LIEC_COMP_RANDK && shared_seed) return 4 * pl.K;             // values only: the receiver redraws the subset
         if (comp_is_sparse(comp)) return 8 * pl.K;                               // (index, value) pairs
         return 4 * pl.d;                                                          // identity: the dense vector
     };
@@ -301,6 +307,16 @@ liec_status liec_wire_bytes(const liec_config *cfg, int64_t *uplink_bytes, int64
     if (downlink_bytes) *downlink_bytes = message(cfg->downlink);
     if (full_precision_bytes) *full_precision_bytes = 4 * pl.d;
     return LIEC_OK;
+}
+
+liec_status liec_wire_bytes(const liec_config *cfg, int64_t *uplink_bytes, int64_t *downlink_bytes,
+                            int64_t *full_precision_bytes) {
+    return wire_bytes(cfg, false, uplink_bytes, downlink_bytes, full_precision_bytes);
+}
+
+liec_status liec_wire_bytes_seeded(const liec_config *cfg, int64_t *uplink_bytes, int64_t *downlink_bytes,
+                                   int64_t *full_precision_bytes) {
+    return wire_bytes(cfg, true, uplink_bytes, downlink_bytes, full_precision_bytes);
 }
 
 size_t liec_down_message_bytes(const liec_config *cfg) {
@@ -380,6 +396,11 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     p.up_cand_val = at<float>(c, pl.r_up_cand_val);      p.down_cand_val = at<float>(c, pl.r_down_cand_val);
     p.up_tile_meta = at<uint32_t>(c, pl.r_up_tile_meta); p.down_tile_meta = at<uint32_t>(c, pl.r_down_tile_meta);
     p.up_outbase = at<uint32_t>(c, pl.r_up_outbase);     p.down_outbase = at<uint32_t>(c, pl.r_down_outbase);
+    p.gen_sets = at<uint32_t>(c, pl.r_gen_sets);         p.gen_val = at<float>(c, pl.r_gen_val);
+    p.gen_hist = at<uint32_t>(c, pl.r_gen_hist);         p.gen_hist2 = at<uint32_t>(c, pl.r_gen_hist2);
+    p.gen_sel = at<uint32_t>(c, pl.r_gen_sel);           p.gen_meta = at<uint32_t>(c, pl.r_gen_meta);
+    p.gen_cand_idx = at<uint32_t>(c, pl.r_gen_cand_idx); p.gen_cand_val = at<float>(c, pl.r_gen_cand_val);
+    p.gen_outbase = at<uint32_t>(c, pl.r_gen_outbase);
 
     struct Up { const Region *r; const void *src; };
     const Up ups[] = {
@@ -401,7 +422,8 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     auto zero = [&](const Region &r) { return r.bytes ? cudaMemset(c->ws + r.off, 0, r.bytes) : cudaSuccess; };
     const Region *zs[] = {&pl.r_status, &pl.r_up_hist, &pl.r_down_hist, &pl.r_up_hist2, &pl.r_down_hist2,
                           &pl.r_up_sel, &pl.r_down_sel, &pl.r_up_tile_meta, &pl.r_down_tile_meta,
-                          &pl.r_up_outbase, &pl.r_down_outbase};
+                          &pl.r_up_outbase, &pl.r_down_outbase,
+                          &pl.r_gen_hist, &pl.r_gen_hist2, &pl.r_gen_sel, &pl.r_gen_meta, &pl.r_gen_outbase};
     for (const Region *r : zs) {
         cudaError_t e = zero(*r);
         if (e != cudaSuccess) {
@@ -514,6 +536,27 @@ liec_status liec_set_subsets(liec_ctx *c, const uint32_t *up_sets, const uint32_
     }
     c->p.up_sets = up_sets;
     c->p.down_set = down_set;
+    return LIEC_OK;
+}
+
+liec_status liec_draw_subsets(liec_ctx *c, uint64_t seed, uint32_t epoch, void *stream) {
+    liec_status st = check_stage(c, 0, "liec_draw_subsets");
+    if (st != LIEC_OK) return st;
+    if (c->p.up != COMP_RANDK && c->p.down != COMP_RANDK) {
+        c->err = "liec_draw_subsets: no side uses random-k";
+        return LIEC_ERR_INVALID_ARG;
+    }
+    const Params &p = c->p;
+    TopkSide s;
+    s.src = nullptr; s.row_stride = 0; s.R = p.N + 1;
+    s.gen = ScoreStream{(uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), epoch};
+    s.idx = p.gen_sets; s.val = p.gen_val; s.hist = p.gen_hist; s.hist2 = p.gen_hist2; s.sel = p.gen_sel;
+    s.cand_idx = p.gen_cand_idx; s.cand_val = p.gen_cand_val; s.meta = p.gen_meta; s.outbase = p.gen_outbase;
+    s.zero_out = nullptr;
+    s.spec = 1;
+    LIEC_CALL(c, launch_randk_draw(p, s, static_cast<cudaStream_t>(stream), &c->launches));
+    c->p.up_sets = p.up == COMP_RANDK ? p.gen_sets : nullptr;
+    c->p.down_set = p.down == COMP_RANDK ? p.gen_sets + (int64_t)p.N * p.K : nullptr;
     return LIEC_OK;
 }
 

@@ -80,6 +80,14 @@ struct Params {
     int64_t CAP;                              // candidate capacity per row
     int64_t cap_max;                          // largest candidate capacity of one segment
 
+    // seeded random-k draw (rows 0..N-1: the workers' subsets, row N: the server's): the subset lists
+    // it produces and the scratch of the selection that produces them
+    uint32_t *gen_sets;                       // [N+1][K]
+    float *gen_val;                           // [N+1][K] scores of the kept elements (scratch)
+    uint32_t *gen_hist, *gen_hist2, *gen_sel; // [N+1][T][...]
+    uint32_t *gen_cand_idx; float *gen_cand_val;  // [N+1][CAP]
+    uint32_t *gen_meta, *gen_outbase;         // [N+1][TT][4], [N+1][TT+1]
+
     float *vbuf;      // [d] identity downlink copy of v
     int32_t *status;  // device status word
 

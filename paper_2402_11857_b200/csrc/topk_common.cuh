@@ -1,12 +1,20 @@
 // Shared by the top-k kernels (Def. 2): the description of one side of the iteration, the status
 // bits, and the block-wide helpers (histogram flush, rank pick, prefix sum).
 #pragma once
+#include <type_traits>
+
 #include "device_common.cuh"
+#include "philox.cuh"
 
 namespace liec {
 
+// Element type tag of a selection whose values are not in memory: the pseudo-random scores of the
+// seeded random-k draw, computed where they are needed (as binary32 bit patterns, see philox.cuh).
+struct ScoreGen { float unused; };
+
 struct TopkSide {
-    const void *src;      // rows of the vector being compressed
+    const void *src;      // rows of the vector being compressed (unused for generated scores)
+    ScoreStream gen;      // generated scores: key and draw number
     int64_t row_stride;   // elements between rows (d for the uplink, 0 for the single downlink row)
     int R;                // rows
     uint32_t *idx; float *val;            // [R][K] output message
@@ -20,6 +28,7 @@ struct TopkSide {
 
 inline TopkSide make_side(const Params &p, bool uplink) {
     TopkSide s;
+    s.gen = ScoreStream{0u, 0u, 0u};
     if (uplink) {
         s.src = p.G; s.row_stride = p.d; s.R = p.N;
         s.idx = p.up_idx; s.val = p.up_val; s.hist = p.up_hist; s.hist2 = p.up_hist2; s.sel = p.up_sel;
@@ -37,6 +46,54 @@ inline TopkSide make_side(const Params &p, bool uplink) {
 }
 
 __device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) & 0x7fffffffu; }
+
+// ---- where a selection's values come from -----------------------------------------------------
+// Four consecutive values of a tile at position `pos` (a multiple of 4) in the 4-wide layout;
+// positions at or beyond the tile's length read as +0.
+template <typename GT>
+__device__ __forceinline__ void fetch4(const TopkSide &s, int row, const TileInfo &ti, int pos, float (&v)[4]) {
+    if constexpr (std::is_same<GT, ScoreGen>::value) {
+        const uint4 w = s.gen.block((uint32_t)((ti.rel + pos) >> 2), (uint32_t)ti.t, (uint32_t)row);
+        const uint32_t w4[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) v[c] = pos + c < ti.len ? __uint_as_float(w4[c]) : 0.0f;
+    } else {
+        const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
+        const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
+        if ((ti.len == TILE) && ((row_beg & 3) == 0)) load4_stream(tile_ptr + pos, v);
+        else load4_guarded(tile_ptr, pos, ti.len, v);
+    }
+}
+
+// One value of segment t (position j relative to the segment); the dense one-CTA path only.
+template <typename GT>
+__device__ __forceinline__ float fetch1(const TopkSide &s, int row, int t, int64_t seg_beg, int64_t j) {
+    if constexpr (std::is_same<GT, ScoreGen>::value) {
+        const uint4 w = s.gen.block((uint32_t)(j >> 2), (uint32_t)t, (uint32_t)row);
+        const uint32_t w4[4] = {w.x, w.y, w.z, w.w};
+        return __uint_as_float(w4[j & 3]);
+    } else {
+        return load1(reinterpret_cast<const GT *>(s.src) + (int64_t)row * s.row_stride + seg_beg + j);
+    }
+}
+
+// Generated scores of a whole tile into shared memory (binary32 patterns, +0 beyond `len`): thread
+// q writes elements 32q .. 32q+31, the ones it reads back in the 32-per-thread layout.
+__device__ __forceinline__ void stage_tile_scores(float *dst, const TopkSide &s, int row, int t, int64_t rel, int len) {
+    const int pos0 = 32 * threadIdx.x;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+        const int pos = pos0 + 4 * b;
+        uint4 w = make_uint4(0u, 0u, 0u, 0u);
+        if (pos < len) {
+            w = s.gen.block((uint32_t)((rel + pos) >> 2), (uint32_t)t, (uint32_t)row);
+            if (pos + 1 >= len) w.y = 0u;
+            if (pos + 2 >= len) w.z = 0u;
+            if (pos + 3 >= len) w.w = 0u;
+        }
+        *reinterpret_cast<uint4 *>(dst + pos) = w;
+    }
+}
 
 enum { STATUS_PICK_RANK = 1, STATUS_CAND_OVERFLOW = 2, STATUS_COUNT_MISMATCH = 4 };
 
@@ -150,7 +207,7 @@ __device__ void slow_select(const Params &p, const TopkSide &s, int t, int row, 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t seg_beg = __ldg(p.seg_off + t);
     const int64_t n = __ldg(p.seg_off + t + 1) - seg_beg;
-    const GT *src = reinterpret_cast<const GT *>(s.src) + (int64_t)row * s.row_stride + seg_beg;
+    auto value_at = [&](int64_t j) { return fetch1<GT>(s, row, t, seg_beg, j); };
     uint32_t rank = sel[SEL_REMAIN];
     uint32_t prefix24;
     const uint32_t flags = sel[SEL_FLAGS];
@@ -161,7 +218,7 @@ __device__ void slow_select(const Params &p, const TopkSide &s, int t, int row, 
         for (int b = threadIdx.x; b < DIGIT1_BINS; b += NT) bins[b] = 0u;
         __syncthreads();
         for (int64_t j = threadIdx.x; j < n; j += NT) {
-            const uint32_t key = key_of(load1(src + j));
+            const uint32_t key = key_of(value_at(j));
             if ((key >> DIGIT1_SHIFT) == b1) atomicAdd(&bins[(key >> 7) & 0xfffu], 1u);
         }
         __syncthreads();
@@ -174,7 +231,7 @@ __device__ void slow_select(const Params &p, const TopkSide &s, int t, int row, 
     for (int b = threadIdx.x; b < NT; b += NT) bins[b] = 0u;
     __syncthreads();
     for (int64_t j = threadIdx.x; j < n; j += NT) {
-        const uint32_t key = key_of(load1(src + j));
+        const uint32_t key = key_of(value_at(j));
         if ((key >> 7) == prefix24) atomicAdd(&bins[key & 0x7fu], 1u);
     }
     __syncthreads();
@@ -195,7 +252,7 @@ __device__ void slow_select(const Params &p, const TopkSide &s, int t, int row, 
             s.outbase[(int64_t)row * (p.TT + 1) + first_tile + (int)(j0 / TILE)] = kbeg + run_sel;
         const int64_t j = j0 + threadIdx.x;
         const bool in = j < n;
-        const float val = in ? load1(src + j) : 0.0f;
+        const float val = in ? value_at(j) : 0.0f;
         const uint32_t key = key_of(val);
         const bool tie = in && key == T;
         const uint32_t tb = __ballot_sync(0xffffffffu, tie);
@@ -232,10 +289,14 @@ __device__ void slow_select(const Params &p, const TopkSide &s, int t, int row, 
 }
 
 // one launch each (defined in topk_tail.cu)
-cudaError_t launch_topk_small(const Params &p, const TopkSide &s, bool bf16, cudaStream_t st);
+// src_kind: element type of the selection's source
+constexpr int SRC_F32 = 0, SRC_BF16 = 1, SRC_SCORES = 2;
+cudaError_t launch_topk_small(const Params &p, const TopkSide &s, int src_kind, cudaStream_t st);
 cudaError_t launch_topk_check(const Params &p, const TopkSide &s, cudaStream_t st);
-cudaError_t launch_topk_tail(const Params &p, const TopkSide &s, bool bf16, cudaStream_t st);
+cudaError_t launch_topk_tail(const Params &p, const TopkSide &s, int src_kind, cudaStream_t st);
 cudaError_t configure_topk_tail_kernels();
+// seeded random-k draw: the selection on generated scores (defined in topk_kernels.cu)
+cudaError_t launch_randk_draw(const Params &p, const TopkSide &s, cudaStream_t st, int64_t *launches);
 
 // Limits of the one-CTA-per-problem tail: candidates of one segment that it sweeps, tiles of one
 // segment that its shared-memory tables hold.  Beyond either, the same steps run as wide launches.

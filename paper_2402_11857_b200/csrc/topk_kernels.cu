@@ -58,20 +58,12 @@ __global__ void __launch_bounds__(THREADS) topk_hist1_kernel(const __grid_consta
         if (ti.seg_tiles == 1) continue;              // selected directly by one CTA
         uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
         if (s.spec && sel[SEL_MODE] != 0u) continue;  // uniform over the CTA
-        const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
-        const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
-        const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
         float v[8][4];
-        if (fast) {
 #pragma unroll
-            for (int j = 0; j < 8; ++j) load4_stream(tile_ptr + tile_pos(warp, lane, j), v[j]);
-        } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) load4_guarded(tile_ptr, tile_pos(warp, lane, j), ti.len, v[j]);
-        }
+        for (int j = 0; j < 8; ++j) fetch4<GT>(s, row, ti, tile_pos(warp, lane, j), v[j]);
         for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(h)[b] = make_uint4(0u, 0u, 0u, 0u);
         __syncthreads();
-        if (fast) hist1_count<true>(h, v, warp, lane, ti.len);
+        if (ti.len == TILE) hist1_count<true>(h, v, warp, lane, ti.len);
         else hist1_count<false>(h, v, warp, lane, ti.len);
         __syncthreads();
         flush_hist(h, s.hist + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS, sel, SEL_LO1, SEL_HI1);
@@ -173,19 +165,15 @@ __global__ void __launch_bounds__(THREADS) topk_hist2_dense_kernel(const __grid_
         const uint32_t b1 = sel[SEL_PREFIX];
         for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) h[b] = 0u;
         __syncthreads();
-        const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
-        const GT *tile_ptr = reinterpret_cast<const GT *>(s.src) + row_beg + ti.rel;
-        const bool fast = (ti.len == TILE) && ((row_beg & 3) == 0);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int pos = tile_pos(warp, lane, j);
             float v[4];
-            if (fast) load4_stream(tile_ptr + pos, v);
-            else load4_guarded(tile_ptr, pos, ti.len, v);
+            fetch4<GT>(s, row, ti, pos, v);
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 const uint32_t key = key_of(v[c]);
-                if ((fast || pos + c < ti.len) && (key >> DIGIT1_SHIFT) == b1) atomicAdd(&h[(key >> 7) & 0xfffu], 1u);
+                if (pos + c < ti.len && (key >> DIGIT1_SHIFT) == b1) atomicAdd(&h[(key >> 7) & 0xfffu], 1u);
             }
         }
         __syncthreads();
@@ -216,6 +204,7 @@ __global__ void __launch_bounds__(THREADS) topk_hist2_dense_kernel(const __grid_
 template <typename GT, bool SPEC>
 __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_constant__ Params p, const TopkSide s) {
     constexpr bool F32 = sizeof(GT) == 4;
+    constexpr bool GEN = std::is_same<GT, ScoreGen>::value;                  // generated scores: nothing to copy
     using ST = typename std::conditional<F32, float, unsigned short>::type;  // storage type of one element
     constexpr int ALIGN_MASK = F32 ? 3 : 7;                                  // elements per 16 bytes, minus one
     __shared__ __align__(128) ST tile_s[TILE];
@@ -249,9 +238,12 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
             low = __uint_as_float(sel[SEL_PREFIX] << (flags == 2u ? 7 : DIGIT1_SHIFT));
         }
         const int64_t row_beg = (int64_t)row * s.row_stride + ti.seg_beg;
-        const ST *tile_ptr = reinterpret_cast<const ST *>(s.src) + row_beg + ti.rel;
-        const bool fast = (ti.len == TILE) && ((row_beg & ALIGN_MASK) == 0);
-        if (fast) {
+        const ST *tile_ptr = GEN ? nullptr : reinterpret_cast<const ST *>(s.src) + row_beg + ti.rel;
+        const bool fast = (ti.len == TILE) && (GEN || (row_beg & ALIGN_MASK) == 0);
+        if constexpr (GEN) {
+            stage_tile_scores(reinterpret_cast<float *>(tile_s), s, row, ti.t, ti.rel, ti.len);
+            __syncthreads();
+        } else if (fast) {
             if (threadIdx.x == 0) {
                 const uint32_t bytes = TILE * sizeof(ST);
                 // (earlier ordinary reads of the buffer are ordered before the copy by the barrier above)
@@ -722,15 +714,21 @@ static dim3 cand_hist_grid(const Params &p, int rows) {
 // collected with last step's guess and the guess is checked; then, for the problems left on the
 // regular route, the first-digit histogram.  Downlink without a fused histogram: plain first-digit
 // histogram of v.
-cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int64_t *launches) {
-    const TopkSide s = make_side(p, uplink);
+// One launch of a kernel template over the element type of the side's source.
+#define LAUNCH_BY_SOURCE(kernel, grid, ...)                                                      \
+    do {                                                                                         \
+        if (src_kind == SRC_BF16) kernel<__nv_bfloat16 __VA_ARGS__><<<grid, THREADS, 0, st>>>(p, s); \
+        else if (src_kind == SRC_SCORES) kernel<ScoreGen __VA_ARGS__><<<grid, THREADS, 0, st>>>(p, s);  \
+        else kernel<float __VA_ARGS__><<<grid, THREADS, 0, st>>>(p, s);                           \
+        CHECK_LAUNCH();                                                                          \
+    } while (0)
+#define COMMA ,
+
+cudaError_t topk_first_part(const Params &p, const TopkSide &s, int src_kind, cudaStream_t st, int64_t *launches) {
     dim3 g_tiles(p.TT, s.R), g_probs(p.T, s.R);
-    const bool bf = uplink && p.gdt == DT_BF16;
     if (!p.n_large) return cudaSuccess;
     if (s.spec) {
-        if (bf) topk_filter_tma_kernel<__nv_bfloat16, true><<<g_tiles, THREADS, 0, st>>>(p, s);
-        else topk_filter_tma_kernel<float, true><<<g_tiles, THREADS, 0, st>>>(p, s);
-        CHECK_LAUNCH();
+        LAUNCH_BY_SOURCE(topk_filter_tma_kernel, g_tiles, COMMA true);
         cudaError_t e = launch_topk_check(p, s, st);
         if (e != cudaSuccess) return e;
         ++*launches;
@@ -740,30 +738,27 @@ cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int
         }
     }
     const dim3 g_hist = s.spec ? strided_grid(p, s.R) : g_tiles;
-    if (bf) topk_hist1_kernel<__nv_bfloat16><<<g_hist, THREADS, 0, st>>>(p, s);
-    else topk_hist1_kernel<float><<<g_hist, THREADS, 0, st>>>(p, s);
-    CHECK_LAUNCH();
+    LAUNCH_BY_SOURCE(topk_hist1_kernel, g_hist);
     return cudaSuccess;
+}
+
+cudaError_t launch_topk_hist1(const Params &p, bool uplink, cudaStream_t st, int64_t *launches) {
+    return topk_first_part(p, make_side(p, uplink), uplink && p.gdt == DT_BF16 ? SRC_BF16 : SRC_F32, st, launches);
 }
 
 // Everything after the first-digit histogram: the message, the thresholds, and for the
 // downlink the zeroing of the selected error entries.
-cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, int64_t *launches) {
-    const TopkSide s = make_side(p, uplink);
+cudaError_t topk_second_part(const Params &p, const TopkSide &s, int src_kind, cudaStream_t st, int64_t *launches) {
     dim3 g_tiles(p.TT, s.R), g_probs(p.T, s.R), g_warp_tiles((p.TT + 7) / 8, s.R);
-    const bool bf = uplink && p.gdt == DT_BF16;
     if (!p.n_large) return cudaSuccess;
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 1); CHECK_LAUNCH();
-    if (bf) topk_hist2_dense_kernel<__nv_bfloat16><<<strided_grid(p, s.R), THREADS, 0, st>>>(p, s);
-    else topk_hist2_dense_kernel<float><<<strided_grid(p, s.R), THREADS, 0, st>>>(p, s);
-    CHECK_LAUNCH();
+    const dim3 g_strided = strided_grid(p, s.R);
+    LAUNCH_BY_SOURCE(topk_hist2_dense_kernel, g_strided);
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 4); CHECK_LAUNCH();
     const dim3 g_filter = s.spec ? strided_grid(p, s.R) : g_tiles;
-    if (bf) topk_filter_tma_kernel<__nv_bfloat16, false><<<g_filter, THREADS, 0, st>>>(p, s);
-    else topk_filter_tma_kernel<float, false><<<g_filter, THREADS, 0, st>>>(p, s);
-    CHECK_LAUNCH();
+    LAUNCH_BY_SOURCE(topk_filter_tma_kernel, g_filter, COMMA false);
     if (use_fused_tail(p)) {
-        cudaError_t e = launch_topk_tail(p, s, bf, st);
+        cudaError_t e = launch_topk_tail(p, s, src_kind, st);
         if (e != cudaSuccess) return e;
         ++*launches;
         return cudaSuccess;
@@ -776,10 +771,12 @@ cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, in
     topk_count_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     topk_scan_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     topk_write_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
-    if (bf) topk_slow_kernel<__nv_bfloat16><<<g_probs, THREADS, 0, st>>>(p, s);
-    else topk_slow_kernel<float><<<g_probs, THREADS, 0, st>>>(p, s);
-    CHECK_LAUNCH();
+    LAUNCH_BY_SOURCE(topk_slow_kernel, g_probs);
     return cudaSuccess;
+}
+
+cudaError_t launch_topk_select(const Params &p, bool uplink, cudaStream_t st, int64_t *launches) {
+    return topk_second_part(p, make_side(p, uplink), uplink && p.gdt == DT_BF16 ? SRC_BF16 : SRC_F32, st, launches);
 }
 
 constexpr size_t SERVER_TOPK_SMEM = sizeof(float) * TILE + sizeof(uint32_t) * DIGIT1_BINS;
@@ -799,9 +796,48 @@ cudaError_t configure_topk_kernels() {
 cudaError_t launch_topk_small_segments(const Params &p, bool uplink, cudaStream_t st, int64_t *launches) {
     if (!p.n_small) return cudaSuccess;
     const TopkSide s = make_side(p, uplink);
-    cudaError_t e = launch_topk_small(p, s, uplink && p.gdt == DT_BF16, st);
+    cudaError_t e = launch_topk_small(p, s, uplink && p.gdt == DT_BF16 ? SRC_BF16 : SRC_F32, st);
     if (e == cudaSuccess) ++*launches;
     return e;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Seeded draw of the random-k subsets (Def. 3): every element of a segment gets a pseudo-random
+// 30-bit score (philox.cuh) and the k_t highest scores are the segment's subset, equal scores to the
+// lower index.  That is a top-k selection on a vector that is computed instead of read, so the
+// kernels above run it unchanged, with ScoreGen as their source type: rows 0..N-1 are the workers'
+// subsets, row N the server's; the output "message" is the subset list itself (ascending indices).
+// Scores are uniform, so the threshold is known in advance up to sampling noise: the single-pass
+// route starts from that bound instead of last step's threshold (and, like every guess, is checked).
+// ------------------------------------------------------------------------------------------------
+__global__ void randk_draw_begin_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x, row = blockIdx.y;
+    if (t >= p.T) return;
+    if (__ldg(p.tile_prefix + t + 1) - __ldg(p.tile_prefix + t) == 1) return;   // selected directly
+    uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
+    const double n = (double)(__ldg(p.seg_off + t + 1) - __ldg(p.seg_off + t));
+    const double k = (double)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
+    // candidates wanted: k plus six standard deviations of their count and some more
+    const double want = k + 6.0 * sqrt(k) + 64.0;
+    uint32_t bound = 1u;   // (0 would mean "no guess")
+    if (want < n) bound = max(1u, (uint32_t)(1073741824.0 * (1.0 - want / n)));
+    sel[SEL_GUESS] = bound;
+}
+
+cudaError_t launch_randk_draw(const Params &p, const TopkSide &s, cudaStream_t st, int64_t *launches) {
+    const int src_kind = SRC_SCORES;
+    (void)src_kind;
+    if (p.n_small) {
+        cudaError_t e = launch_topk_small(p, s, SRC_SCORES, st);
+        if (e != cudaSuccess) return e;
+        ++*launches;
+    }
+    if (!p.n_large) return cudaSuccess;
+    randk_draw_begin_kernel<<<dim3((p.T + 127) / 128, s.R), 128, 0, st>>>(p, s);
+    CHECK_LAUNCH();
+    cudaError_t e = topk_first_part(p, s, SRC_SCORES, st, launches);
+    if (e != cudaSuccess) return e;
+    return topk_second_part(p, s, SRC_SCORES, st, launches);
 }
 
 template <bool TEL>

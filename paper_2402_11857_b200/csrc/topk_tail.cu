@@ -37,9 +37,13 @@ __global__ void __launch_bounds__(THREADS) topk_small_kernel(const __grid_consta
     const int64_t seg_beg = __ldg(p.seg_off + t);
     const int n = (int)(__ldg(p.seg_off + t + 1) - seg_beg);
     const uint32_t kbeg = (uint32_t)__ldg(p.k_off + t), k = (uint32_t)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
-    const int64_t row_beg = (int64_t)row * s.row_stride + seg_beg;
-    const ST *src = reinterpret_cast<const ST *>(s.src) + row_beg;
-    stage_tile_guarded(tile_s, src, n, (row_beg & (F32 ? 3 : 7)) == 0);
+    if constexpr (std::is_same<GT, ScoreGen>::value) {
+        stage_tile_scores(reinterpret_cast<float *>(tile_s), s, row, t, 0, n);
+    } else {
+        const int64_t row_beg = (int64_t)row * s.row_stride + seg_beg;
+        const ST *src = reinterpret_cast<const ST *>(s.src) + row_beg;
+        stage_tile_guarded(tile_s, src, n, (row_beg & (F32 ? 3 : 7)) == 0);
+    }
 
     // thread q owns elements 32q .. 32q+31; it visits them in an order rotated by the lane so that
     // the lanes of a warp hit different banks
@@ -505,9 +509,10 @@ __global__ void __launch_bounds__(TAIL_THREADS) topk_tail_kernel(const __grid_co
 constexpr size_t SMALL_SMEM_F32 = sizeof(uint32_t) * DIGIT1_BINS + sizeof(float) * TILE;
 constexpr size_t SMALL_SMEM_BF16 = sizeof(uint32_t) * DIGIT1_BINS + sizeof(unsigned short) * TILE;
 
-cudaError_t launch_topk_small(const Params &p, const TopkSide &s, bool bf16, cudaStream_t st) {
+cudaError_t launch_topk_small(const Params &p, const TopkSide &s, int src_kind, cudaStream_t st) {
     const dim3 grid(p.n_small, s.R);
-    if (bf16) topk_small_kernel<__nv_bfloat16><<<grid, THREADS, SMALL_SMEM_BF16, st>>>(p, s);
+    if (src_kind == SRC_BF16) topk_small_kernel<__nv_bfloat16><<<grid, THREADS, SMALL_SMEM_BF16, st>>>(p, s);
+    else if (src_kind == SRC_SCORES) topk_small_kernel<ScoreGen><<<grid, THREADS, SMALL_SMEM_F32, st>>>(p, s);
     else topk_small_kernel<float><<<grid, THREADS, SMALL_SMEM_F32, st>>>(p, s);
     return cudaGetLastError();
 }
@@ -517,11 +522,12 @@ cudaError_t launch_topk_check(const Params &p, const TopkSide &s, cudaStream_t s
     return cudaGetLastError();
 }
 
-cudaError_t launch_topk_tail(const Params &p, const TopkSide &s, bool bf16, cudaStream_t st) {
+cudaError_t launch_topk_tail(const Params &p, const TopkSide &s, int src_kind, cudaStream_t st) {
     const dim3 grid(p.n_large, s.R);
     const int words = tail_bitmap_words(p);
     const size_t smem = sizeof(uint32_t) * 4 * (size_t)words;
-    if (bf16) topk_tail_kernel<__nv_bfloat16><<<grid, TAIL_THREADS, smem, st>>>(p, s, words);
+    if (src_kind == SRC_BF16) topk_tail_kernel<__nv_bfloat16><<<grid, TAIL_THREADS, smem, st>>>(p, s, words);
+    else if (src_kind == SRC_SCORES) topk_tail_kernel<ScoreGen><<<grid, TAIL_THREADS, smem, st>>>(p, s, words);
     else topk_tail_kernel<float><<<grid, TAIL_THREADS, smem, st>>>(p, s, words);
     return cudaGetLastError();
 }
@@ -531,6 +537,8 @@ cudaError_t configure_topk_tail_kernels() {
     const int tail_max = (int)(sizeof(uint32_t) * 4 * ((TAIL_MAX_CAND + 31) / 32 + TAIL_THREADS));
     cudaError_t e = cudaFuncSetAttribute(topk_tail_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, tail_max);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_tail_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, tail_max);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_tail_kernel<ScoreGen>, cudaFuncAttributeMaxDynamicSharedMemorySize, tail_max);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_small_kernel<ScoreGen>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMALL_SMEM_F32);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_small_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMALL_SMEM_F32);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_small_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMALL_SMEM_BF16);
     return e;

@@ -69,6 +69,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.liec_worker_update.restype = C.c_int
     lib.liec_set_subsets.argtypes = [vp, vp, vp]
     lib.liec_set_subsets.restype = C.c_int
+    lib.liec_draw_subsets.argtypes = [vp, C.c_uint64, C.c_uint32, vp]
+    lib.liec_draw_subsets.restype = C.c_int
+    lib.liec_wire_bytes_seeded.argtypes = [cfgp, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+    lib.liec_wire_bytes_seeded.restype = C.c_int
     lib.liec_step.argtypes = [vp, vp, C.c_float, vp]
     lib.liec_step.restype = C.c_int
     lib.liec_topk_route_counts.argtypes = [vp, vp, C.c_int32, C.POINTER(C.c_int64), vp]
@@ -130,11 +134,17 @@ def workspace_bytes(cfg: liec_config) -> int:
     return int(load_library().liec_workspace_bytes(C.byref(cfg)))
 
 
-def liec_wire_bytes(cfg: liec_config):
+def liec_wire_bytes_seeded(cfg: liec_config):
+    """As liec_wire_bytes when sender and receiver draw the random-k subsets from a shared seed."""
+    return liec_wire_bytes(cfg, _seeded=True)
+
+
+def liec_wire_bytes(cfg: liec_config, _seeded: bool = False):
     """(uplink, downlink, full-precision) bytes per worker and iteration."""
     lib = load_library()
     up, down, full = C.c_int64(0), C.c_int64(0), C.c_int64(0)
-    st = lib.liec_wire_bytes(C.byref(cfg), C.byref(up), C.byref(down), C.byref(full))
+    fn = lib.liec_wire_bytes_seeded if _seeded else lib.liec_wire_bytes
+    st = fn(C.byref(cfg), C.byref(up), C.byref(down), C.byref(full))
     if st != 0:
         raise LiecError(st, lib.liec_last_error(None).decode())
     return int(up.value), int(down.value), int(full.value)
@@ -240,6 +250,11 @@ class Context:
         self._subsets = (up_sets, down_set)
         self._check(self.lib.liec_set_subsets(self._ctx, None if up_sets is None else up_sets.data_ptr(),
                                               None if down_set is None else down_set.data_ptr()))
+
+    def liec_draw_subsets(self, seed: int, epoch: int, stream=None):
+        """Random-k: draws and installs the subsets of all workers and the server from (seed, epoch)."""
+        self._subsets = None
+        self._check(self.lib.liec_draw_subsets(self._ctx, int(seed), int(epoch), self._stream(stream)))
 
     def liec_step(self, grads, lr: float, stream=None):
         self._check_grads(grads)

@@ -41,15 +41,25 @@ class Pair:
         self.ctx = liec.Context(self.Xd, self.ed, self.off, up, down, self.k, grad_dtype)
 
     def step(self, G: torch.Tensor, lr: float, staged: bool = False, check_messages: bool = True,
-             up_sets=None, down_set=None):
+             up_sets=None, down_set=None, draw=None):
         """Runs one iteration on both sides and asserts parity of messages and state.
-        up_sets [N,K] / down_set [K] (numpy uint32): the subsets of a random-k side."""
+        up_sets [N,K] / down_set [K] (numpy uint32): the subsets of a random-k side; or
+        draw = (seed, epoch): both sides draw them from the seed, each with its own code."""
         Gd = G.to(DEV).contiguous()
+        if draw is not None:
+            sets = oracle.draw_subsets(draw[0], draw[1], self.N + 1, self.off, self.k)
+            r = oracle.step(self.Xh, self.eh, widen(G), lr, self.off, self.up, self.down, k=self.k,
+                            up_sets=sets[:self.N], down_set=sets[self.N])
+            self.ctx.liec_draw_subsets(draw[0], draw[1])
+            return self._gpu_step_and_compare(Gd, lr, r, staged, check_messages)
         r = oracle.step(self.Xh, self.eh, widen(G), lr, self.off, self.up, self.down, k=self.k,
                         up_sets=up_sets, down_set=down_set)
         if up_sets is not None or down_set is not None:
             as_dev = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a).view(np.int32)).to(DEV)
             self.ctx.liec_set_subsets(as_dev(up_sets), as_dev(down_set))
+        return self._gpu_step_and_compare(Gd, lr, r, staged, check_messages)
+
+    def _gpu_step_and_compare(self, Gd, lr, r, staged, check_messages):
         if staged or check_messages:
             self.ctx.liec_uplink_compress(Gd)
             self.ctx.liec_server_aggregate()

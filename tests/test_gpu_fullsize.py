@@ -181,3 +181,43 @@ def test_c4_gpt2_sign_bf16_full_size():
 
 def test_c3_resnet50_randk_full_size():
     _run("c3", steps=2, budget_elems=3_500_000, randk=True)
+
+
+def test_c3_resnet50_seeded_randk_full_size():
+    """The seeded draw at full size (N = 16 workers + the server, 161 tensors): the subsets of sampled
+    (row, segment) pairs against the oracle's own draw; for all rows and segments, what holds at any
+    size (k_t ascending indices inside the segment); then a whole iteration on them."""
+    w = WORKLOADS["c3"]
+    lay = w.layout()
+    N, d, off = w.num_workers, lay.dim, lay.seg_offsets
+    k = topk_counts(lay, *w.topk_frac)
+    koff = np.concatenate([[0], np.cumsum(k)])
+    X = torch.zeros(N, d, device="cuda")
+    e = torch.zeros(d, device="cuda")
+    ctx = liec.Context(X, e, off, liec.COMP_RANDK, liec.COMP_RANDK, k)
+    G = make_gradients(w.dist, w.scale, N, d, 0, base_seed=79, device="cuda")
+    seed = 0xC0FFEE1234567
+    for epoch in (0, 1):
+        ctx.liec_draw_subsets(seed, epoch)
+        ctx.liec_step(G, w.lr)
+        torch.cuda.synchronize()
+        assert ctx.liec_device_status() == 0
+        m = ctx.liec_get_messages()
+        lists = np.concatenate([u32(m["up_idx"]), u32(m["down_idx"])[None, :]], axis=0)   # rows 0..N-1, then the server
+        seg_of = np.repeat(np.arange(lay.num_segments), k)
+        inner = np.ones(lists.shape[1], bool)
+        inner[koff[:-1]] = False
+        for row in range(N + 1):
+            idx = lists[row].astype(np.int64)
+            assert np.all(idx >= off[seg_of]) and np.all(idx < off[seg_of + 1]), row
+            assert np.all(np.diff(idx)[inner[1:]] > 0), row
+        assert len({lists[row].tobytes() for row in range(N + 1)}) == N + 1          # every row has its own subsets
+        # sampled (row, segment) pairs: the largest tensor once, a spread of the others over the rows
+        segs = _sample_segments(lay, 5_000_000)
+        for q, t in enumerate(segs):
+            for row in {q % (N + 1), N}:
+                n = int(off[t + 1] - off[t])
+                want = oracle.subset_from_scores(oracle.subset_scores(seed, epoch, row, t, n), int(k[t])).astype(np.int64) + int(off[t])
+                assert np.array_equal(lists[row, koff[t]:koff[t + 1]].astype(np.int64), want), (epoch, row, t)
+        # the messages carry the values found at the subsets
+        assert torch.equal(m["up_val"], torch.gather(G, 1, m["up_idx"].long()))

@@ -53,3 +53,14 @@ def test_wire_bytes_of_the_other_messages():
     cfg, keep = liec.make_config(0, off, 1, 1)
     with pytest.raises(liec.LiecError):
         liec.liec_wire_bytes(cfg)
+
+
+def test_wire_bytes_with_a_shared_seed():
+    """Sender and receiver draw the same random-k subsets from a seed: values only on the wire."""
+    off = [0, 100, 164, 1000]
+    cfg, keep = liec.make_config(4, off, liec.COMP_RANDK, liec.COMP_RANDK, [1, 5, 80])
+    assert liec.liec_wire_bytes_seeded(cfg) == (4 * 86, 4 * 86, 4000)
+    cfg, keep = liec.make_config(4, off, liec.COMP_RANDK, liec.COMP_TOPK, [1, 5, 80])     # top-k still sends its indices
+    assert liec.liec_wire_bytes_seeded(cfg) == (4 * 86, 8 * 86, 4000)
+    cfg, keep = liec.make_config(4, off, liec.COMP_SCALED_SIGN, liec.COMP_SCALED_SIGN)
+    assert liec.liec_wire_bytes_seeded(cfg) == liec.liec_wire_bytes(cfg)
