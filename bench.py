@@ -90,12 +90,12 @@ def update_kernel_bytes(w) -> float:
 
 
 # DRAM bytes (dram__bytes_read + dram__bytes_write, ncu) of one worker-update launch, per named
-# workload.  c4: captured on c4/8 (4.925 GB for 497.8 M element-workers) and scaled by N*d, because
+# workload.  c4: captured on c4/8 (4.924 GB for 497.8 M element-workers) and scaled by N*d, because
 # this streaming kernel's traffic grows in proportion; c3 and c2: captured at full size (the tail
 # of the parameter writes is still in the L2 when the kernel ends, hence slightly fewer bytes than
 # the algorithmic count).  Any other workload or variant: not captured.
-UPDATE_TRAFFIC_BYTES = {"c4": 4.924888e9 / 497759232 * 32 * 124439808, "c3": 3274704384 + 1587624448,
-                        "c2": 749634816 + 323100160}
+UPDATE_TRAFFIC_BYTES = {"c4": (2.989412e9 + 1.934865e9) / 497759232 * 32 * 124439808, "c3": 3274834432 + 1588320000,
+                        "c2": 749630720 + 322008320}
 
 
 # ------------------------------------------------------------------------------------ clocks

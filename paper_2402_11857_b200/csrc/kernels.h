@@ -26,6 +26,7 @@ cudaError_t launch_randk_compress(const Params &p, bool uplink, cudaStream_t st,
 // model-averaging iteration and mean model
 cudaError_t launch_average_step(const Params &p, float lr, cudaStream_t st);
 cudaError_t launch_mean_params(const Params &p, float *out, cudaStream_t st);
+cudaError_t configure_average_kernels();  // opt-in shared memory sizes; call once per device
 
 // squared norms (monitoring)
 cudaError_t launch_sumsq(const Params &p, const void *src, int64_t row_stride, int rows, bool bf16, cudaStream_t st);

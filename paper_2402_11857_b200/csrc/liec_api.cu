@@ -433,6 +433,7 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
         }
     }
     cudaError_t e = configure_topk_kernels();
+    if (e == cudaSuccess) e = configure_average_kernels();
     if (e == cudaSuccess && c->plan.K > 0 && !c->plan.small_seg.empty()) {
         e = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);

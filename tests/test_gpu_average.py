@@ -61,3 +61,48 @@ def test_averaging_unaligned_rows_and_stage_order():
     with pytest.raises(liec.LiecError) as ei:
         P.ctx.liec_average_step(Gd, 0.1)       # in the middle of a compressed iteration
     assert ei.value.status == 4
+
+
+@pytest.mark.parametrize("N,gdt", [(8, liec.F32), (16, liec.F32), (32, liec.BF16), (40, liec.F32), (300, liec.F32)])
+def test_averaging_staged_in_shared_memory(N, gdt):
+    """Full aligned tiles take the variant that keeps the workers' gradients of a slice in shared memory
+    between the two sweeps (2048-element slices for N = 8 float rows, 1024-element slices for 16 float
+    or 32 bfloat16 rows); 40 and 300 float rows of a slice exceed the shared-memory budget and take the
+    re-reading variant; the ragged tail and the 8-element segment take the guarded path inside the
+    same launch."""
+    off = [0, 3 * 8192, 3 * 8192 + 8, 5 * 8192 + 8 + 77]
+    dist = ("bf16_outliers", 1e-2) if gdt == liec.BF16 else ("normal", 1.0)
+    rng = np.random.default_rng(4)
+    P = Pair(N, off, liec.COMP_SCALED_SIGN, liec.COMP_SCALED_SIGN, grad_dtype=gdt,
+             x0=rng.standard_normal(off[-1]), e0=rng.standard_normal(off[-1]) * 0.1)
+    for step in range(2):
+        G = make_gradients(dist[0], dist[1], N, off[-1], step, base_seed=34)
+        P.step(G, 0.05, check_messages=False)      # rows drift apart
+        _average(P, G, 0.05)
+
+
+def test_averaging_bulk_copy_wait_runs_out():
+    """The staged variant waits for its bulk copies with a bound: told to expect 16 bytes more than they
+    deliver, the wait runs out, bit 8 of the status word is set and the CTA writes nothing."""
+    off = [0, 8192]
+    N = 2
+    X0 = torch.randn(N, 8192, device="cuda")
+    X = X0.clone()
+    e = torch.randn(8192, device="cuda")
+    e0 = e.clone()
+    ctx = liec.Context(X, e, off, liec.COMP_SCALED_SIGN, liec.COMP_SCALED_SIGN)
+    G = make_gradients("normal", 1.0, N, 8192, 0, base_seed=35).cuda()
+    ctx.liec_set_copy_wait(poll_limit=1000, expect_extra_bytes=16)
+    ctx.liec_average_step(G, 0.1)
+    torch.cuda.synchronize()
+    assert ctx.liec_device_status() & 8
+    assert torch.equal(X, X0) and torch.equal(e, e0)
+    ctx.liec_set_copy_wait()
+    ctx.liec_clear_status()
+    ctx.liec_average_step(G, 0.1)
+    torch.cuda.synchronize()
+    assert ctx.liec_device_status() == 0
+    Xh, eh = X0.cpu().numpy().copy(), e0.cpu().numpy().copy()
+    oracle.average_step(Xh, eh, G.cpu().numpy(), 0.1)
+    assert_close(f32(X), Xh, "params after averaging")
+    assert np.all(f32(e) == 0.0)
