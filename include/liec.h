@@ -37,9 +37,9 @@
  *   identity: no message buffer; the dense vector itself.
  *
  * Ownership: the caller owns every device buffer (params, error, gradients, workspace).
- * The library owns only the host-side context (for top-k configurations with segments of at
- * most 8192 elements also one helper stream and two events, created by liec_init and released
- * by liec_destroy).  The hot calls allocate nothing, never synchronise the device and only
+ * The library owns only the host-side context (for top-k / random-k configurations that have
+ * segments of at most 8192 elements, or segments with 16384 or more selection candidates, also one
+ * helper stream and four events, created by liec_init and released by liec_destroy).  The hot calls allocate nothing, never synchronise the device and only
  * enqueue work that is ordered on the given stream: a top-k stage may run part of its kernels
  * on the helper stream, forked from and joined back to the given stream by events inside the
  * same call (this also works while the given stream is being captured into a CUDA graph).

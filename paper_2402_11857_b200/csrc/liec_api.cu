@@ -113,10 +113,6 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
             if (cap > pl.cap_max) pl.cap_max = cap;
         }
     }
-    // the per-problem kernels take the largest segments first
-    std::stable_sort(pl.large_seg.begin(), pl.large_seg.end(), [&](int32_t a, int32_t b) {
-        return pl.seg_off[a + 1] - pl.seg_off[a] > pl.seg_off[b + 1] - pl.seg_off[b];
-    });
     // a sparse message's values, tiled like the model (for their squared norms): segment t owns k_t entries
     pl.ktile_prefix.assign(T + 1, 0);
     if (any_topk) {
@@ -139,6 +135,10 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
         for (int q = pl.tile_prefix[t]; q < pl.tile_prefix[t + 1]; ++q) pl.tile_seg[q] = t;
         (pl.tile_prefix[t + 1] - pl.tile_prefix[t] == 1 ? pl.small_seg : pl.large_seg).push_back(t);
     }
+    // the per-problem kernels take the largest segments first (their CTAs run longest)
+    std::stable_sort(pl.large_seg.begin(), pl.large_seg.end(), [&](int32_t a, int32_t b) {
+        return pl.seg_off[a + 1] - pl.seg_off[a] > pl.seg_off[b + 1] - pl.seg_off[b];
+    });
 
     Carver c;
     pl.r_seg_off = c.take(sizeof(int64_t) * (T + 1));
@@ -224,6 +224,7 @@ struct liec_ctx {
     // and joined to the caller's stream by events, so that they overlap the dense passes
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    cudaEvent_t ev_tail_fork = nullptr, ev_tail_join = nullptr;   // the tail launch of the big problems
 };
 
 namespace {
@@ -254,11 +255,12 @@ liec_status cuda_fail(liec_ctx *c, cudaError_t e, const char *what) {
 bool aligned16(const void *ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
 
 void release_side(liec_ctx *c) {
-    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
-    if (c->ev_join) cudaEventDestroy(c->ev_join);
+    for (cudaEvent_t ev : {c->ev_fork, c->ev_join, c->ev_tail_fork, c->ev_tail_join})
+        if (ev) cudaEventDestroy(ev);
     if (c->side) cudaStreamDestroy(c->side);
-    c->ev_fork = c->ev_join = nullptr;
+    c->ev_fork = c->ev_join = c->ev_tail_fork = c->ev_tail_join = nullptr;
     c->side = nullptr;
+    c->p.tail_stream = c->p.tail_fork = c->p.tail_join = nullptr;
 }
 
 // Top-k side: the single-tile segments on the context's own stream (between a fork after what `s`
@@ -366,6 +368,19 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     p.large_seg = at<int32_t>(c, pl.r_large_seg);
     p.n_small = (int32_t)pl.small_seg.size();
     p.n_large = (int32_t)pl.large_seg.size();
+    // the leading (largest) multi-tile segments whose candidate buffers are big: their tails get a launch of their own
+    p.n_big = 0;
+    p.cap_rest_max = 0;
+    if (pl.K > 0) {
+        auto cap_of = [&](int q) { return pl.cap_off[pl.large_seg[q] + 1] - pl.cap_off[pl.large_seg[q]]; };
+        while (p.n_big < p.n_large && cap_of(p.n_big) >= TAIL_BIG_CAP) ++p.n_big;
+        for (int q = p.n_big; q < p.n_large; ++q) p.cap_rest_max = std::max<int64_t>(p.cap_rest_max, cap_of(q));
+    }
+    {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms = 0;
+        p.num_sms = sms;
+    }
     p.max_seg_tiles = 0;
     for (int t = 0; t < pl.T; ++t) p.max_seg_tiles = std::max(p.max_seg_tiles, pl.tile_prefix[t + 1] - pl.tile_prefix[t]);
     p.status = at<int32_t>(c, pl.r_status);
@@ -434,11 +449,14 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     }
     cudaError_t e = configure_topk_kernels();
     if (e == cudaSuccess) e = configure_average_kernels();
-    if (e == cudaSuccess && c->plan.K > 0 && !c->plan.small_seg.empty()) {
-        e = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking);
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming);
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming);
+    if (e == cudaSuccess && c->plan.K > 0 && (!c->plan.small_seg.empty() || p.n_big > 0)) {
+        int prio_low = 0, prio_high = 0;   // the helper stream carries the longest-running CTAs of a stage: they go first
+        e = cudaDeviceGetStreamPriorityRange(&prio_low, &prio_high);
+        if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&c->side, cudaStreamNonBlocking, prio_high);
+        for (cudaEvent_t *ev : {&c->ev_fork, &c->ev_join, &c->ev_tail_fork, &c->ev_tail_join})
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
         if (e != cudaSuccess) release_side(c);
+        else { p.tail_stream = c->side; p.tail_fork = c->ev_tail_fork; p.tail_join = c->ev_tail_join; }
     }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {

@@ -38,6 +38,12 @@ struct Params {
     const int32_t *small_seg;    // [n_small] segments of one tile (top-k: selected directly by one CTA)
     const int32_t *large_seg;    // [n_large] segments of several tiles
     int32_t n_small, n_large;
+    int32_t n_big;               // leading entries of large_seg whose candidate capacity is TAIL_BIG_CAP or more
+    int64_t cap_rest_max;        // largest candidate capacity among the other entries of large_seg
+    // host side only: the context's helper stream and the events that fork / join the tail launch of
+    // the big problems (cudaStream_t / cudaEvent_t; NULL = everything on the caller's stream)
+    void *tail_stream, *tail_fork, *tail_join;
+    int32_t num_sms;             // SMs of the device the context was created on
     int32_t max_seg_tiles;       // tiles of the longest segment
 
     // state

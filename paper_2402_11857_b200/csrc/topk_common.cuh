@@ -293,7 +293,8 @@ __device__ void slow_select(const Params &p, const TopkSide &s, int t, int row, 
 constexpr int SRC_F32 = 0, SRC_BF16 = 1, SRC_SCORES = 2;
 cudaError_t launch_topk_small(const Params &p, const TopkSide &s, int src_kind, cudaStream_t st);
 cudaError_t launch_topk_check(const Params &p, const TopkSide &s, cudaStream_t st);
-cudaError_t launch_topk_tail(const Params &p, const TopkSide &s, int src_kind, cudaStream_t st);
+cudaError_t launch_topk_tail(const Params &p, const TopkSide &s, int src_kind, cudaStream_t st, int64_t *launches);
+constexpr int64_t TAIL_BIG_CAP = 16384;   // candidate capacity from which a problem's tail gets the larger CTA
 cudaError_t configure_topk_tail_kernels();
 // seeded random-k draw: the selection on generated scores (defined in topk_kernels.cu)
 cudaError_t launch_randk_draw(const Params &p, const TopkSide &s, cudaStream_t st, int64_t *launches);

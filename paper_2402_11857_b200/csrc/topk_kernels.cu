@@ -757,12 +757,7 @@ cudaError_t topk_second_part(const Params &p, const TopkSide &s, int src_kind, c
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 4); CHECK_LAUNCH();
     const dim3 g_filter = s.spec ? strided_grid(p, s.R) : g_tiles;
     LAUNCH_BY_SOURCE(topk_filter_tma_kernel, g_filter, COMMA false);
-    if (use_fused_tail(p)) {
-        cudaError_t e = launch_topk_tail(p, s, src_kind, st);
-        if (e != cudaSuccess) return e;
-        ++*launches;
-        return cudaSuccess;
-    }
+    if (use_fused_tail(p)) return launch_topk_tail(p, s, src_kind, st, launches);
     // some segment has too many candidates or tiles for one CTA: the same steps, spread over the tile blocks
     topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 1, cand_hist_reps(p)); CHECK_LAUNCH();
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();

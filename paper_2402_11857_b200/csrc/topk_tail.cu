@@ -12,6 +12,7 @@
 //                      remaining key digits -> exact threshold and number of ties to accept ->
 //                      per-tile counts -> output offsets -> ordered compaction into (index, value).
 //                      Replaces a chain of seven small launches; nothing waits on another CTA.
+#include <algorithm>
 #include <type_traits>
 
 #include "device_common.cuh"
@@ -176,18 +177,25 @@ __global__ void topk_check_kernel(const __grid_constant__ Params p, const TopkSi
 // ------------------------------------------------------------------------------------------------
 // Tail: grid (n_large, rows), NT threads.  Largest segments first (the host orders large_seg so).
 // ------------------------------------------------------------------------------------------------
-constexpr int TAIL_THREADS = 512;
+// CTAs of this kernel are latency-bound chains (sweeps over the candidates with a block-wide pick or
+// scan between them), so the launch as a whole is bound by how many of them are resident.  The few
+// largest problems (candidate capacity of TAIL_BIG_CAP or more: their CTAs run longest) get 512
+// threads in a launch of their own on the context's helper stream (higher priority, so that they
+// start first); the many others get 256 threads and bitmaps sized for their own, smaller candidate
+// buffers, so that one big CTA and two small ones, or four to five small ones, share an SM.
+constexpr int TAIL_THREADS = 256, TAIL_THREADS_BIG = 512;
 
-// Words of one bitmap over a problem's candidates, rounded up to whole rounds of the CTA.
-static inline int tail_bitmap_words(const Params &p) {
-    const int words = (int)((p.cap_max + 31) / 32);
-    return (words + TAIL_THREADS - 1) / TAIL_THREADS * TAIL_THREADS;
+// Words of one bitmap over `cap` candidates, rounded up to whole rounds of the largest CTA.
+static inline int tail_bitmap_words(int64_t cap) {
+    const int words = (int)((cap + 31) / 32);
+    return (words + TAIL_THREADS_BIG - 1) / TAIL_THREADS_BIG * TAIL_THREADS_BIG;
 }
 
-template <typename GT>
-__global__ void __launch_bounds__(TAIL_THREADS) topk_tail_kernel(const __grid_constant__ Params p, const TopkSide s,
-                                                                  const int bitmap_words) {
-    constexpr int NT = TAIL_THREADS, NW = NT / 32;
+// Problems large_seg[first_problem + blockIdx.x] of every row.
+template <typename GT, int NT>
+__global__ void __launch_bounds__(NT) topk_tail_kernel(const __grid_constant__ Params p, const TopkSide s,
+                                                        const int bitmap_words, const int first_problem) {
+    constexpr int NW = NT / 32;
     __shared__ __align__(16) uint32_t bins[DIGIT1_BINS];
     __shared__ uint32_t scratch[NT + 4];
     __shared__ uint32_t warp_tot[NW], warp_tot2[NW];
@@ -199,10 +207,10 @@ __global__ void __launch_bounds__(TAIL_THREADS) topk_tail_kernel(const __grid_co
     extern __shared__ uint32_t tail_smem[];
     uint32_t *gt_bits = tail_smem, *eq_bits = tail_smem + bitmap_words;
     uint32_t *gt_before = tail_smem + 2 * bitmap_words, *eq_before = tail_smem + 3 * bitmap_words;
-    const int t = __ldg(p.large_seg + blockIdx.x), row = blockIdx.y;
+    const int t = __ldg(p.large_seg + first_problem + blockIdx.x), row = blockIdx.y;
     const int lane = threadIdx.x & 31;
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
-    // last kernel of a side: the next step starts with "no problem on the regular route yet"
+    // last kernel(s) of a side: the next step starts with "no problem on the regular route yet"
     if (s.spec && blockIdx.x == 0 && row == 0 && threadIdx.x == 0) p.status[STATUS_ANY_REGULAR] = 0;
     const uint32_t flags = sel[SEL_FLAGS];
     const bool single = s.spec && sel[SEL_MODE] == 1u;
@@ -359,7 +367,7 @@ __global__ void __launch_bounds__(TAIL_THREADS) topk_tail_kernel(const __grid_co
     for (uint32_t w = nwords + threadIdx.x; w < (uint32_t)bitmap_words; w += NT) { gt_bits[w] = 0u; eq_bits[w] = 0u; }
     __syncthreads();
     // tiles in order: ties accepted per tile (lowest index first) and first output slot
-    constexpr int PER = TAIL_MAX_TILES / NT;
+    constexpr int PER = (TAIL_MAX_TILES + NT - 1) / NT;
     bool all_ties;   // every entry equal to the threshold is kept (the usual case: distinct magnitudes)
     {
         const int q0 = threadIdx.x * PER;
@@ -522,22 +530,53 @@ cudaError_t launch_topk_check(const Params &p, const TopkSide &s, cudaStream_t s
     return cudaGetLastError();
 }
 
-cudaError_t launch_topk_tail(const Params &p, const TopkSide &s, int src_kind, cudaStream_t st) {
-    const dim3 grid(p.n_large, s.R);
-    const int words = tail_bitmap_words(p);
+template <int NT>
+static cudaError_t launch_tail_part(const Params &p, const TopkSide &s, int src_kind, int first, int count, int64_t cap,
+                                    cudaStream_t st) {
+    const dim3 grid(count, s.R);
+    const int words = tail_bitmap_words(cap);
     const size_t smem = sizeof(uint32_t) * 4 * (size_t)words;
-    if (src_kind == SRC_BF16) topk_tail_kernel<__nv_bfloat16><<<grid, TAIL_THREADS, smem, st>>>(p, s, words);
-    else if (src_kind == SRC_SCORES) topk_tail_kernel<ScoreGen><<<grid, TAIL_THREADS, smem, st>>>(p, s, words);
-    else topk_tail_kernel<float><<<grid, TAIL_THREADS, smem, st>>>(p, s, words);
+    if (src_kind == SRC_BF16) topk_tail_kernel<__nv_bfloat16, NT><<<grid, NT, smem, st>>>(p, s, words, first);
+    else if (src_kind == SRC_SCORES) topk_tail_kernel<ScoreGen, NT><<<grid, NT, smem, st>>>(p, s, words, first);
+    else topk_tail_kernel<float, NT><<<grid, NT, smem, st>>>(p, s, words, first);
     return cudaGetLastError();
+}
+
+// Two concurrent launches when the context has a helper stream and some problems are big: those
+// (first in large_seg) on the helper stream, forked from and joined to `st` by events, the others
+// on `st`; otherwise one launch on `st`.
+cudaError_t launch_topk_tail(const Params &p, const TopkSide &s, int src_kind, cudaStream_t st, int64_t *launches) {
+    // at most one big problem per SM: a second one would wait behind the first
+    const int n_big = p.tail_stream ? std::min(p.n_big, p.num_sms / s.R) : 0;
+    cudaError_t e = cudaSuccess;
+    if (n_big > 0) {
+        cudaStream_t side = static_cast<cudaStream_t>(p.tail_stream);
+        cudaEvent_t fork = static_cast<cudaEvent_t>(p.tail_fork), join = static_cast<cudaEvent_t>(p.tail_join);
+        if ((e = cudaEventRecord(fork, st)) != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(side, fork, 0)) != cudaSuccess) return e;
+        if ((e = launch_tail_part<TAIL_THREADS_BIG>(p, s, src_kind, 0, n_big, p.cap_max, side)) != cudaSuccess) return e;
+        ++*launches;
+        if ((e = cudaEventRecord(join, side)) != cudaSuccess) return e;
+    }
+    if (p.n_large > n_big) {
+        // (big problems that found no SM of their own stay in this launch, which then sizes its bitmaps for them)
+        const int64_t cap = n_big == p.n_big ? p.cap_rest_max : p.cap_max;
+        if ((e = launch_tail_part<TAIL_THREADS>(p, s, src_kind, n_big, p.n_large - n_big, cap, st)) != cudaSuccess) return e;
+        ++*launches;
+    }
+    if (n_big > 0) e = cudaStreamWaitEvent(st, static_cast<cudaEvent_t>(p.tail_join), 0);
+    return e;
 }
 
 // Opt-in shared memory sizes of the kernels in this file (once per device).
 cudaError_t configure_topk_tail_kernels() {
-    const int tail_max = (int)(sizeof(uint32_t) * 4 * ((TAIL_MAX_CAND + 31) / 32 + TAIL_THREADS));
-    cudaError_t e = cudaFuncSetAttribute(topk_tail_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, tail_max);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_tail_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, tail_max);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_tail_kernel<ScoreGen>, cudaFuncAttributeMaxDynamicSharedMemorySize, tail_max);
+    const int tail_max = (int)(sizeof(uint32_t) * 4 * ((TAIL_MAX_CAND + 31) / 32 + TAIL_THREADS_BIG));
+    const void *tails[] = {(const void *)topk_tail_kernel<float, TAIL_THREADS>, (const void *)topk_tail_kernel<__nv_bfloat16, TAIL_THREADS>,
+                           (const void *)topk_tail_kernel<ScoreGen, TAIL_THREADS>, (const void *)topk_tail_kernel<float, TAIL_THREADS_BIG>,
+                           (const void *)topk_tail_kernel<__nv_bfloat16, TAIL_THREADS_BIG>, (const void *)topk_tail_kernel<ScoreGen, TAIL_THREADS_BIG>};
+    cudaError_t e = cudaSuccess;
+    for (const void *k : tails)
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, tail_max);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_small_kernel<ScoreGen>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMALL_SMEM_F32);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_small_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMALL_SMEM_F32);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(topk_small_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMALL_SMEM_BF16);
