@@ -208,6 +208,20 @@ __device__ void slow_select(const Params &p, const TopkSide &s, int t, int row, 
     const int64_t seg_beg = __ldg(p.seg_off + t);
     const int64_t n = __ldg(p.seg_off + t + 1) - seg_beg;
     auto value_at = [&](int64_t j) { return fetch1<GT>(s, row, t, seg_beg, j); };
+    // U stripes of NT consecutive elements per round: a thread's U loads are in flight together
+    constexpr int U = 8;
+    static_assert(TILE % (NT * U) == 0, "a round of the dense path must not straddle a tile boundary");
+    __shared__ uint32_t cnt_tie[U][NW], cnt_sel[U][NW];
+    auto dense_sweep = [&](auto &&use) {   // use(key) for every element of the segment
+        for (int64_t j0 = threadIdx.x; j0 < n; j0 += (int64_t)NT * U) {
+            uint32_t key[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) key[u] = j0 + (int64_t)u * NT < n ? key_of(value_at(j0 + (int64_t)u * NT)) : 0xffffffffu;
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (key[u] != 0xffffffffu) use(key[u]);
+        }
+    };
     uint32_t rank = sel[SEL_REMAIN];
     uint32_t prefix24;
     const uint32_t flags = sel[SEL_FLAGS];
@@ -217,10 +231,7 @@ __device__ void slow_select(const Params &p, const TopkSide &s, int t, int row, 
         const uint32_t b1 = sel[SEL_PREFIX];
         for (int b = threadIdx.x; b < DIGIT1_BINS; b += NT) bins[b] = 0u;
         __syncthreads();
-        for (int64_t j = threadIdx.x; j < n; j += NT) {
-            const uint32_t key = key_of(value_at(j));
-            if ((key >> DIGIT1_SHIFT) == b1) atomicAdd(&bins[(key >> 7) & 0xfffu], 1u);
-        }
+        dense_sweep([&](uint32_t key) { if ((key >> DIGIT1_SHIFT) == b1) atomicAdd(&bins[(key >> 7) & 0xfffu], 1u); });
         __syncthreads();
         const PickResult r2 = block_pick<NT>(bins, DIGIT1_BINS, rank, scratch);
         if (!r2.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
@@ -230,10 +241,7 @@ __device__ void slow_select(const Params &p, const TopkSide &s, int t, int row, 
     // last 7 bits
     for (int b = threadIdx.x; b < NT; b += NT) bins[b] = 0u;
     __syncthreads();
-    for (int64_t j = threadIdx.x; j < n; j += NT) {
-        const uint32_t key = key_of(value_at(j));
-        if ((key >> 7) == prefix24) atomicAdd(&bins[key & 0x7fu], 1u);
-    }
+    dense_sweep([&](uint32_t key) { if ((key >> 7) == prefix24) atomicAdd(&bins[key & 0x7fu], 1u); });
     __syncthreads();
     const PickResult r = block_pick<NT>(bins, NT, rank, scratch);
     if (!r.ok) { if (threadIdx.x == 0) atomicOr(p.status, STATUS_PICK_RANK); return; }
@@ -247,38 +255,60 @@ __device__ void slow_select(const Params &p, const TopkSide &s, int t, int row, 
     const int64_t obase = (int64_t)row * p.K + kbeg;
     const uint32_t lt_mask = (1u << lane) - 1u;
     uint32_t run_sel = 0, run_tie = 0;
-    for (int64_t j0 = 0; j0 < n; j0 += NT) {
-        if ((j0 % TILE) == 0 && threadIdx.x == 0)
+    for (int64_t j0 = 0; j0 < n; j0 += (int64_t)NT * U) {
+        if ((j0 % TILE) == 0 && threadIdx.x == 0)   // (a round never straddles a tile boundary)
             s.outbase[(int64_t)row * (p.TT + 1) + first_tile + (int)(j0 / TILE)] = kbeg + run_sel;
-        const int64_t j = j0 + threadIdx.x;
-        const bool in = j < n;
-        const float val = in ? value_at(j) : 0.0f;
-        const uint32_t key = key_of(val);
-        const bool tie = in && key == T;
-        const uint32_t tb = __ballot_sync(0xffffffffu, tie);
-        if (lane == 0) wa[warp] = __popc(tb);
-        __syncthreads();
-        uint32_t tie_rank = run_tie + __popc(tb & lt_mask), tie_tot = 0;
+        // stripe u holds elements j0 + u*NT .. +NT-1: stripes, and the threads inside one, are in index order
+        float val[U];
+        uint32_t tb[U], sb[U], tie_rank[U];
 #pragma unroll
-        for (int w = 0; w < NW; ++w) { if (w < warp) tie_rank += wa[w]; tie_tot += wa[w]; }
-        const bool take = in && (key > T || (tie && tie_rank < ties_wanted));
-        const uint32_t sb = __ballot_sync(0xffffffffu, take);
-        if (lane == 0) wb[warp] = __popc(sb);
-        __syncthreads();
-        uint32_t out = run_sel + __popc(sb & lt_mask), sel_tot = 0;
-#pragma unroll
-        for (int w = 0; w < NW; ++w) { if (w < warp) out += wb[w]; sel_tot += wb[w]; }
-        if (take && out >= k) {
-            atomicOr(p.status, STATUS_COUNT_MISMATCH);
-        } else if (take) {
-            const uint32_t flat = (uint32_t)(seg_beg + j);
-            s.idx[obase + out] = flat;
-            s.val[obase + out] = val;
-            if (tie && tie_rank == ties_wanted - 1) sel[SEL_CUT] = flat;
+        for (int u = 0; u < U; ++u) {
+            const int64_t j = j0 + (int64_t)u * NT + threadIdx.x;
+            val[u] = j < n ? value_at(j) : __uint_as_float(0xffffffffu);   // (a pattern no key equals: keys have 31 bits)
         }
-        run_sel += sel_tot;
-        run_tie += tie_tot;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const bool in = j0 + (int64_t)u * NT + threadIdx.x < n;
+            tb[u] = __ballot_sync(0xffffffffu, in && key_of(val[u]) == T);
+            if (lane == 0) cnt_tie[u][warp] = __popc(tb[u]);
+        }
         __syncthreads();
+        uint32_t ties_so_far = run_tie;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const bool in = j0 + (int64_t)u * NT + threadIdx.x < n;
+            const uint32_t key = key_of(val[u]);
+            uint32_t before = ties_so_far + __popc(tb[u] & lt_mask), tot = 0;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) { if (w < warp) before += cnt_tie[u][w]; tot += cnt_tie[u][w]; }
+            tie_rank[u] = before;
+            const bool tie = (tb[u] >> lane) & 1u;
+            const bool take = in && (key > T || (tie && before < ties_wanted));
+            sb[u] = __ballot_sync(0xffffffffu, take);
+            if (lane == 0) cnt_sel[u][warp] = __popc(sb[u]);
+            ties_so_far += tot;
+        }
+        __syncthreads();
+        uint32_t sel_so_far = run_sel;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            uint32_t out = sel_so_far + __popc(sb[u] & lt_mask), tot = 0;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) { if (w < warp) out += cnt_sel[u][w]; tot += cnt_sel[u][w]; }
+            const bool take = (sb[u] >> lane) & 1u;
+            if (take && out >= k) {
+                atomicOr(p.status, STATUS_COUNT_MISMATCH);
+            } else if (take) {
+                const uint32_t flat = (uint32_t)(seg_beg + j0 + (int64_t)u * NT + threadIdx.x);
+                s.idx[obase + out] = flat;
+                s.val[obase + out] = val[u];
+                if (((tb[u] >> lane) & 1u) && tie_rank[u] == ties_wanted - 1) sel[SEL_CUT] = flat;
+            }
+            sel_so_far += tot;
+        }
+        run_sel = sel_so_far;
+        run_tie = ties_so_far;
+        __syncthreads();   // the counters are rewritten by the next round
     }
     if (threadIdx.x == 0 && run_sel != k) atomicOr(p.status, STATUS_COUNT_MISMATCH);
     // downlink: selected entries of the error become +0 (after every read of the segment is done)

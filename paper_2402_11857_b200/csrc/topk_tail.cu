@@ -193,7 +193,7 @@ static inline int tail_bitmap_words(int64_t cap) {
 
 // Problems large_seg[first_problem + blockIdx.x] of every row.
 template <typename GT, int NT>
-__global__ void __launch_bounds__(NT) topk_tail_kernel(const __grid_constant__ Params p, const TopkSide s,
+__global__ void __launch_bounds__(NT, 1024 / NT) topk_tail_kernel(const __grid_constant__ Params p, const TopkSide s,
                                                         const int bitmap_words, const int first_problem) {
     constexpr int NW = NT / 32;
     __shared__ __align__(16) uint32_t bins[DIGIT1_BINS];

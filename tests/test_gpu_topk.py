@@ -48,6 +48,24 @@ def test_heavy_ties_take_lower_index():
         P.step(G, 0.25)
 
 
+def test_mostly_zero_segments_with_k_above_the_nonzero_count():
+    """Rows of which one entry in a hundred is non-zero (an embedding gradient that saw a few tokens)
+    with k_t = 5 %: the threshold is the key of zero and millions of entries tie at it, so the dense
+    one-CTA path does the selection (both the one-launch-per-problem form and, for the segment of
+    more than 1024 tiles, the wide form); its rounds span several tiles and a ragged tail."""
+    lay = Layout("sparse", (37 * 8192 + 11, 1030 * 8192 + 3, 9000))
+    k = topk_counts(lay, 5, 100)
+    N = 2
+    P = _pair(N, lay.seg_offsets, TOPK, TOPK, k=k)
+    g = torch.Generator().manual_seed(15)
+    for step in range(2):
+        G = make_gradients("normal", 1.0, N, lay.dim, step, base_seed=15)
+        G = torch.where(torch.rand(G.shape, generator=g) < 0.01, G, torch.zeros_like(G))
+        P.step(G, 0.1)
+    up = P.ctx.liec_topk_route_counts(True)
+    assert up["slow"] >= N            # (the 9000-element segment may or may not need it)
+
+
 def test_quantised_values_ties_at_threshold():
     """Gaussians rounded to multiples of 1/64: ties at the threshold, candidates within the buffer."""
     lay = Layout("quant", (30000, 8192, 70000))
