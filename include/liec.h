@@ -335,10 +335,11 @@ liec_status liec_set_copy_wait(liec_ctx *ctx, uint32_t poll_limit, uint32_t expe
  *   out[0] problems, out[1] uplink problems that finished on the single dense pass seeded by the
  *   previous threshold, out[2] problems that needed the dense second-digit pass (more entries
  *   share the threshold's leading key bits than the candidate buffer holds), out[3] problems that
- *   fell back to the dense path of one CTA (huge groups of equal magnitudes), out[4] problems of a
+ *   were finished in the dense source because even then their candidates did not fit (huge groups of
+ *   equal magnitudes, e.g. a mostly-zero row whose k exceeds its non-zero count), out[4] problems of a
  *   single-tile segment (at most 8192 elements), which one CTA selects directly in shared memory.
  * per_problem (host, one byte per problem in [row][segment] order, or NULL) receives the same per
- * problem: bit 0 single pass, bit 1 second-digit pass, bit 2 dense one-CTA path, bit 3 single tile.
+ * problem: bit 0 single pass, bit 1 second-digit pass, bit 2 finished in the dense source, bit 3 single tile.
  * The result of the selection never depends on the route.  LIEC_ERR_INVALID_ARG when the side does
  * not use top-k.
  */

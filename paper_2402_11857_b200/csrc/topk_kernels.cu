@@ -17,7 +17,9 @@
 //           the number of ties to accept -> per-tile counts -> output offsets -> ordered
 //           compaction into (idx, val) (topk_tail_kernel).  When a segment has more candidates or
 //           tiles than one CTA is given, the same steps run as wide launches instead:
-//           cand_hist + pick (levels 2, 3), count, scan, write, slow.
+//           cand_hist + pick (levels 2, 3), count, scan, write, close.  A problem whose candidates do
+//           not fit the buffer even under a 24-bit prefix (huge groups of equal keys) is walked in the
+//           dense source: by its one CTA in the tail, tile-parallel by the wide launches.
 //
 // The uplink first tries a single-pass route: filter with a guess (a lower bound taken from the
 // previous step's threshold), check (did the guess hold?), and straight to the tail; a problem whose
@@ -90,7 +92,6 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
     // levels 2, 3: wide form of the finish step (second digit, last 7 bits) from candidate histograms.
     if (level == 5 && sel[SEL_MODE] != 1u) return;
     if (level == 2 && sel[SEL_FLAGS] != 0u) return;
-    if (level == 3 && (sel[SEL_FLAGS] & 1u)) return;
     if (level == 1 && s.spec && sel[SEL_MODE] != 0u) return;
     if (level == 4 && sel[SEL_FLAGS] != 2u) return;
     const bool first = level == 1 || level == 5;
@@ -333,7 +334,13 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
 // ------------------------------------------------------------------------------------------------
 // candidate passes: one CTA per (tile, row) walks that tile's block of the candidate buffer
 // ------------------------------------------------------------------------------------------------
-struct CandBlock { int64_t base; uint32_t cnt; int t; uint32_t *sel; uint32_t *meta; bool skip; };
+// A problem whose candidates did not fit the buffer even under a 24-bit prefix (huge groups of equal
+// magnitudes, e.g. a mostly-zero row whose k exceeds its non-zero count) has no candidate blocks: its
+// tiles are walked in the dense source instead (`dense`), element by element, in the same kernels.
+struct CandBlock {
+    int64_t base; uint32_t cnt; int t; uint32_t *sel; uint32_t *meta; bool skip;
+    bool dense; int64_t seg_beg, rel;   // dense: cnt = the tile's length, entry q = element rel + q of the segment
+};
 
 __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide &s, int tile, int row) {
     CandBlock cb;
@@ -341,12 +348,18 @@ __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide 
     cb.t = ti.t;
     cb.sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
     cb.meta = s.meta + ((int64_t)row * p.TT + tile) * 4;
-    cb.skip = (cb.sel[SEL_FLAGS] & 1u) != 0u || ti.seg_tiles == 1;
-    cb.cnt = cb.skip ? 0u : cb.meta[1];
+    cb.skip = ti.seg_tiles == 1;
+    cb.dense = !cb.skip && (cb.sel[SEL_FLAGS] & 1u) != 0u;
+    cb.cnt = cb.skip ? 0u : (cb.dense ? (uint32_t)ti.len : cb.meta[1]);
     cb.base = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + cb.meta[0];
+    cb.seg_beg = ti.seg_beg;
+    cb.rel = ti.rel;
     return cb;
 }
 
+// The kernels below run their loop over a tile's entries once for each kind of working set (candidate
+// block / dense tile), with the way an entry is fetched as a functor, so that the common candidate
+// path compiles to exactly the loop over the candidate arrays.
 // The candidate passes give one warp to every tile block (8 tiles per CTA): blocks are small
 // (about 1.4 % of a tile) and warps need no block-wide synchronisation.
 // Histograms over candidates, one warp per tile block; lanes holding the same digit add once
@@ -354,6 +367,7 @@ __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide 
 // the wide form of the finish step, for segments whose candidates are too many for one CTA:
 // level 1 = second digit of the candidates whose first digit is the threshold's, level 2 = last
 // 7 bits of the candidates under the 24-bit prefix.
+template <typename GT>
 __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_constant__ Params p, const TopkSide s,
                                                                   const int level, const int reps) {
     __shared__ uint32_t h[DIGIT1_BINS];
@@ -381,31 +395,36 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
         if (active) {
             cb = cand_block(p, s, tile, row);
             const uint32_t flags = cb.sel[SEL_FLAGS];
-            active = !cb.skip && !(level == 0 && cb.sel[SEL_MODE] != 1u) && !(level == 1 && flags != 0u);
+            // (a dense problem knows its 24-bit prefix from the dense second-digit pass: level 2 only)
+            active = !cb.skip && !(cb.dense && level != 2) && !(level == 0 && cb.sel[SEL_MODE] != 1u) && !(level == 1 && flags != 0u);
             prefix = cb.sel[SEL_PREFIX];
         }
         uint32_t lo = 0xffffffffu, hi = 0u;
         if (active) {
             uint32_t *gh = (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
-            for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
-                const uint32_t q = c0 + lane;
-                uint32_t digit = 0xffffffffu;  // lanes with nothing to add
-                if (q < cb.cnt) {
-                    const uint32_t key = key_of(s.cand_val[cb.base + q]);
-                    if (level == 0) digit = key >> DIGIT1_SHIFT;
-                    else if (level == 1) { if ((key >> DIGIT1_SHIFT) == prefix) digit = (key >> 7) & 0xfffu; }
-                    else if ((key >> 7) == prefix) digit = key & 0x7fu;
-                }
-                const uint32_t same = __match_any_sync(0xffffffffu, digit);
-                if (digit != 0xffffffffu) {
-                    if (lane == __ffs(same) - 1) {
-                        if (gather) atomicAdd(&h[digit], (uint32_t)__popc(same));
-                        else atomicAdd(gh + digit, (uint32_t)__popc(same));
+            auto walk = [&](auto &&value_at) {
+                for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
+                    const uint32_t q = c0 + lane;
+                    uint32_t digit = 0xffffffffu;  // lanes with nothing to add
+                    if (q < cb.cnt) {
+                        const uint32_t key = key_of(value_at(q));
+                        if (level == 0) digit = key >> DIGIT1_SHIFT;
+                        else if (level == 1) { if ((key >> DIGIT1_SHIFT) == prefix) digit = (key >> 7) & 0xfffu; }
+                        else if ((key >> 7) == prefix) digit = key & 0x7fu;
                     }
-                    lo = min(lo, digit);
-                    hi = max(hi, digit);
+                    const uint32_t same = __match_any_sync(0xffffffffu, digit);
+                    if (digit != 0xffffffffu) {
+                        if (lane == __ffs(same) - 1) {
+                            if (gather) atomicAdd(&h[digit], (uint32_t)__popc(same));
+                            else atomicAdd(gh + digit, (uint32_t)__popc(same));
+                        }
+                        lo = min(lo, digit);
+                        hi = max(hi, digit);
+                    }
                 }
-            }
+            };
+            if (cb.dense) walk([&](uint32_t q) { return fetch1<GT>(s, row, cb.t, cb.seg_beg, cb.rel + q); });
+            else walk([&](uint32_t q) { return s.cand_val[cb.base + q]; });
         }
         if (!gather && active) {  // (uniform over the warp)
             lo = __reduce_min_sync(0xffffffffu, lo);
@@ -424,6 +443,7 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
     }
 }
 
+template <typename GT>
 __global__ void __launch_bounds__(THREADS) topk_count_kernel(const __grid_constant__ Params p, const TopkSide s) {
     const int row = blockIdx.y, lane = threadIdx.x & 31;
     const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -432,10 +452,26 @@ __global__ void __launch_bounds__(THREADS) topk_count_kernel(const __grid_consta
     if (cb.skip) return;
     const uint32_t T = cb.sel[SEL_THRESH];
     uint32_t g = 0, e = 0;
-    for (uint32_t q = lane; q < cb.cnt; q += 32) {
-        const uint32_t key = key_of(s.cand_val[cb.base + q]);
-        g += key > T ? 1u : 0u;
-        e += key == T ? 1u : 0u;
+    if (!cb.dense) {
+        for (uint32_t q = lane; q < cb.cnt; q += 32) {
+            const uint32_t key = key_of(s.cand_val[cb.base + q]);
+            g += key > T ? 1u : 0u;
+            e += key == T ? 1u : 0u;
+        }
+    } else {
+        constexpr int UC = 8;   // elements per lane fetched together
+        for (uint32_t q0 = lane; q0 < cb.cnt; q0 += 32 * UC) {
+            uint32_t key[UC];
+#pragma unroll
+            for (int u = 0; u < UC; ++u)
+                key[u] = q0 + 32 * u < cb.cnt ? key_of(fetch1<GT>(s, row, cb.t, cb.seg_beg, cb.rel + q0 + 32 * u)) : 0u;
+#pragma unroll
+            for (int u = 0; u < UC; ++u) {
+                const bool in = q0 + 32 * u < cb.cnt;
+                g += in && key[u] > T ? 1u : 0u;
+                e += in && key[u] == T ? 1u : 0u;
+            }
+        }
     }
     g = __reduce_add_sync(0xffffffffu, g);
     e = __reduce_add_sync(0xffffffffu, e);
@@ -448,7 +484,6 @@ __global__ void __launch_bounds__(THREADS) topk_scan_kernel(const __grid_constan
     constexpr int PER = 4;  // consecutive tiles per thread and round
     const int t = blockIdx.x, row = blockIdx.y;
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
-    if (sel[SEL_FLAGS] & 1u) return;
     const int first = __ldg(p.tile_prefix + t), ntiles = __ldg(p.tile_prefix + t + 1) - first;
     if (ntiles == 1) return;   // selected directly by one CTA
     const uint32_t ties_wanted = sel[SEL_TIES];
@@ -494,6 +529,7 @@ __global__ void __launch_bounds__(THREADS) topk_scan_kernel(const __grid_constan
 }
 
 // write: ordered compaction of a tile's candidate block into the message (one warp per tile)
+template <typename GT>
 __global__ void __launch_bounds__(THREADS) topk_write_kernel(const __grid_constant__ Params p, const TopkSide s) {
     const int row = blockIdx.y, lane = threadIdx.x & 31;
     const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -506,56 +542,57 @@ __global__ void __launch_bounds__(THREADS) topk_write_kernel(const __grid_consta
     const int64_t obase = (int64_t)row * p.K + s.outbase[(int64_t)row * (p.TT + 1) + tile];
     const int64_t oend = (int64_t)row * p.K + __ldg(p.k_off + cb.t + 1);  // never write past the segment's slots
     const uint32_t lt_mask = (1u << lane) - 1u;
-    uint32_t run_sel = 0, run_tie = 0;
-    for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
-        const uint32_t q = c0 + lane;
-        const bool in = q < cb.cnt;
-        const float val = in ? s.cand_val[cb.base + q] : 0.0f;
-        const uint32_t idx = in ? s.cand_idx[cb.base + q] : 0u;
-        const uint32_t key = key_of(val);
-        const bool tie = in && key == T;
-        const uint32_t tb = __ballot_sync(0xffffffffu, tie);
-        const uint32_t tie_rank = run_tie + __popc(tb & lt_mask);
-        const bool take = in && (key > T || (tie && tie_rank < allowed));
-        const uint32_t sb = __ballot_sync(0xffffffffu, take);
-        if (take && obase + run_sel + __popc(sb & lt_mask) >= oend) {
-            atomicOr(p.status, STATUS_COUNT_MISMATCH);  // inconsistent selection state: drop the write
-        } else if (take) {
-            const uint32_t out = run_sel + __popc(sb & lt_mask);
-            s.idx[obase + out] = idx;
-            s.val[obase + out] = val;
-            if (s.zero_out) s.zero_out[idx] = 0.0f;
-            if (has_last && tie && tie_rank == allowed - 1) cb.sel[SEL_CUT] = idx;
+    auto walk = [&](auto &&entry_at) {   // entry_at(q, idx, val)
+        uint32_t run_sel = 0, run_tie = 0;
+        for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
+            const uint32_t q = c0 + lane;
+            const bool in = q < cb.cnt;
+            float val = 0.0f;
+            uint32_t idx = 0u;
+            if (in) entry_at(q, idx, val);
+            const uint32_t key = key_of(val);
+            const bool tie = in && key == T;
+            const uint32_t tb = __ballot_sync(0xffffffffu, tie);
+            const uint32_t tie_rank = run_tie + __popc(tb & lt_mask);
+            const bool take = in && (key > T || (tie && tie_rank < allowed));
+            const uint32_t sb = __ballot_sync(0xffffffffu, take);
+            if (take && obase + run_sel + __popc(sb & lt_mask) >= oend) {
+                atomicOr(p.status, STATUS_COUNT_MISMATCH);  // inconsistent selection state: drop the write
+            } else if (take) {
+                const uint32_t out = run_sel + __popc(sb & lt_mask);
+                s.idx[obase + out] = idx;
+                s.val[obase + out] = val;
+                if (s.zero_out) s.zero_out[idx] = 0.0f;
+                if (has_last && tie && tie_rank == allowed - 1) cb.sel[SEL_CUT] = idx;
+            }
+            run_sel += __popc(sb);
+            run_tie += __popc(tb);
         }
-        run_sel += __popc(sb);
-        run_tie += __popc(tb);
-    }
+    };
+    if (cb.dense)
+        walk([&](uint32_t q, uint32_t &idx, float &val) {
+            idx = (uint32_t)(cb.seg_beg + cb.rel + q);
+            val = fetch1<GT>(s, row, cb.t, cb.seg_beg, cb.rel + q);
+        });
+    else
+        walk([&](uint32_t q, uint32_t &idx, float &val) { idx = s.cand_idx[cb.base + q]; val = s.cand_val[cb.base + q]; });
 }
 
 // ------------------------------------------------------------------------------------------------
-// Wide form, last kernel of a side: one CTA per problem.  Runs the dense path for problems whose
-// candidates did not fit (slow_select) and closes the step's bookkeeping for every problem.
+// Wide form, last kernel of a side: closes the step's bookkeeping for every problem (one thread each).
 // ------------------------------------------------------------------------------------------------
-template <typename GT>
-__global__ void __launch_bounds__(THREADS) topk_slow_kernel(const __grid_constant__ Params p, const TopkSide s) {
-    __shared__ uint32_t bins[DIGIT1_BINS];
-    __shared__ uint32_t scratch[THREADS + 4];
-    __shared__ uint32_t wa[8], wb[8];
-    const int t = blockIdx.x, row = blockIdx.y;
-    uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
+__global__ void topk_close_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x, row = blockIdx.y;
     // the next step starts with "no problem on the regular route yet"
-    if (s.spec && t == 0 && row == 0 && threadIdx.x == 0) p.status[STATUS_ANY_REGULAR] = 0;
+    if (s.spec && t == 0 && row == 0) p.status[STATUS_ANY_REGULAR] = 0;
+    if (t >= p.T) return;
     if (__ldg(p.tile_prefix + t + 1) - __ldg(p.tile_prefix + t) == 1) return;   // selected directly by one CTA
+    uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
     const uint32_t flags = sel[SEL_FLAGS];
     const bool single = s.spec && sel[SEL_MODE] == 1u;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        sel[SEL_CAND_COUNT] = 0u;
-        sel[SEL_SPEC_FAIL] = 0u;
-        sel[SEL_ROUTE] = (single ? ROUTE_SINGLE : 0) | ((flags & 2u) ? ROUTE_REFINED : 0) | ((flags & 1u) ? ROUTE_SLOW : 0);
-    }
-    if (!(flags & 1u)) return;
-    slow_select<GT, THREADS>(p, s, t, row, sel, bins, scratch, wa, wb);
+    sel[SEL_CAND_COUNT] = 0u;
+    sel[SEL_SPEC_FAIL] = 0u;
+    sel[SEL_ROUTE] = (single ? ROUTE_SINGLE : 0) | ((flags & 2u) ? ROUTE_REFINED : 0) | ((flags & 1u) ? ROUTE_SLOW : 0);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -733,7 +770,7 @@ cudaError_t topk_first_part(const Params &p, const TopkSide &s, int src_kind, cu
         if (e != cudaSuccess) return e;
         ++*launches;
         if (!use_fused_tail(p)) {   // wide form: first digit of the single-pass problems from a global histogram
-            topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 0, cand_hist_reps(p)); CHECK_LAUNCH();
+            topk_cand_hist_kernel<float><<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 0, cand_hist_reps(p)); CHECK_LAUNCH();   // (candidates only at this level)
             topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 5); CHECK_LAUNCH();
         }
     }
@@ -759,14 +796,21 @@ cudaError_t topk_second_part(const Params &p, const TopkSide &s, int src_kind, c
     LAUNCH_BY_SOURCE(topk_filter_tma_kernel, g_filter, COMMA false);
     if (use_fused_tail(p)) return launch_topk_tail(p, s, src_kind, st, launches);
     // some segment has too many candidates or tiles for one CTA: the same steps, spread over the tile blocks
-    topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 1, cand_hist_reps(p)); CHECK_LAUNCH();
+    // (problems left without candidates - huge groups of equal keys - are walked in the dense source by
+    //  the same kernels from the last-digit histogram on: tile-parallel like everything else here)
+    const int reps = cand_hist_reps(p);
+    const dim3 g_hist = cand_hist_grid(p, s.R);
+    topk_cand_hist_kernel<float><<<g_hist, THREADS, 0, st>>>(p, s, 1, reps); CHECK_LAUNCH();
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();
-    topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 2, cand_hist_reps(p)); CHECK_LAUNCH();
+    if (src_kind == SRC_BF16) topk_cand_hist_kernel<__nv_bfloat16><<<g_hist, THREADS, 0, st>>>(p, s, 2, reps);
+    else if (src_kind == SRC_SCORES) topk_cand_hist_kernel<ScoreGen><<<g_hist, THREADS, 0, st>>>(p, s, 2, reps);
+    else topk_cand_hist_kernel<float><<<g_hist, THREADS, 0, st>>>(p, s, 2, reps);
+    CHECK_LAUNCH();
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 3); CHECK_LAUNCH();
-    topk_count_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+    LAUNCH_BY_SOURCE(topk_count_kernel, g_warp_tiles);
     topk_scan_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
-    topk_write_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
-    LAUNCH_BY_SOURCE(topk_slow_kernel, g_probs);
+    LAUNCH_BY_SOURCE(topk_write_kernel, g_warp_tiles);
+    topk_close_kernel<<<dim3((p.T + 127) / 128, s.R), 128, 0, st>>>(p, s); CHECK_LAUNCH();
     return cudaSuccess;
 }
 
