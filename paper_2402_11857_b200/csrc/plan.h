@@ -134,5 +134,6 @@ constexpr unsigned STATUS_BAD_SUBSET = 16;   // bit of the status word: a random
 constexpr unsigned STATUS_COPY_TIMEOUT = 8;  // bit of the status word: a TMA bulk copy did not land within the wait limit
 constexpr int STATUS_ANY_REGULAR = 12; // uplink: some problem takes the regular two-pass path this step
 constexpr int STATUS_ANY_REFINE = 8;  // +0 uplink, +1 downlink: some problem needs the dense second-digit pass
+constexpr int STATUS_ANY_DENSE = 16;  // +0 uplink, +1 downlink: some problem has no candidates and is finished in the dense source (wide form)
 
 }  // namespace liec

@@ -18,8 +18,9 @@
 //           compaction into (idx, val) (topk_tail_kernel).  When a segment has more candidates or
 //           tiles than one CTA is given, the same steps run as wide launches instead:
 //           cand_hist + pick (levels 2, 3), count, scan, write, close.  A problem whose candidates do
-//           not fit the buffer even under a 24-bit prefix (huge groups of equal keys) is walked in the
-//           dense source: by its one CTA in the tail, tile-parallel by the wide launches.
+//           not fit the buffer even under a 24-bit prefix (huge groups of equal keys) is finished in the
+//           dense source: by its one CTA in the tail; in the wide form by three tile-parallel kernels of
+//           its own (last-digit histogram, per-tile counts, ordered write) that leave at once otherwise.
 //
 // The uplink first tries a single-pass route: filter with a guess (a lower bound taken from the
 // previous step's threshold), check (did the guess hold?), and straight to the tail; a problem whose
@@ -146,7 +147,11 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
         sel[SEL_PREFIX] = (sel[SEL_PREFIX] << 12) | r.bin;
         sel[SEL_REMAIN] = r.rank_in_bin;
         sel[SEL_NCAND] = ncand;
-        if (ncand > cap) { sel[SEL_FLAGS] = 3u; sel[SEL_GUESS] = 0u; }  // still too many (huge groups of equal keys): slow path
+        if (ncand > cap) {  // still too many (huge groups of equal keys): no candidates, finished in the dense source
+            sel[SEL_FLAGS] = 3u;
+            sel[SEL_GUESS] = 0u;
+            p.status[STATUS_ANY_DENSE + (s.zero_out ? 1 : 0)] = 1;
+        }
     }
 }
 
@@ -334,13 +339,7 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
 // ------------------------------------------------------------------------------------------------
 // candidate passes: one CTA per (tile, row) walks that tile's block of the candidate buffer
 // ------------------------------------------------------------------------------------------------
-// A problem whose candidates did not fit the buffer even under a 24-bit prefix (huge groups of equal
-// magnitudes, e.g. a mostly-zero row whose k exceeds its non-zero count) has no candidate blocks: its
-// tiles are walked in the dense source instead (`dense`), element by element, in the same kernels.
-struct CandBlock {
-    int64_t base; uint32_t cnt; int t; uint32_t *sel; uint32_t *meta; bool skip;
-    bool dense; int64_t seg_beg, rel;   // dense: cnt = the tile's length, entry q = element rel + q of the segment
-};
+struct CandBlock { int64_t base; uint32_t cnt; int t; uint32_t *sel; uint32_t *meta; bool skip; };
 
 __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide &s, int tile, int row) {
     CandBlock cb;
@@ -348,18 +347,12 @@ __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide 
     cb.t = ti.t;
     cb.sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
     cb.meta = s.meta + ((int64_t)row * p.TT + tile) * 4;
-    cb.skip = ti.seg_tiles == 1;
-    cb.dense = !cb.skip && (cb.sel[SEL_FLAGS] & 1u) != 0u;
-    cb.cnt = cb.skip ? 0u : (cb.dense ? (uint32_t)ti.len : cb.meta[1]);
+    cb.skip = (cb.sel[SEL_FLAGS] & 1u) != 0u || ti.seg_tiles == 1;
+    cb.cnt = cb.skip ? 0u : cb.meta[1];
     cb.base = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + cb.meta[0];
-    cb.seg_beg = ti.seg_beg;
-    cb.rel = ti.rel;
     return cb;
 }
 
-// The kernels below run their loop over a tile's entries once for each kind of working set (candidate
-// block / dense tile), with the way an entry is fetched as a functor, so that the common candidate
-// path compiles to exactly the loop over the candidate arrays.
 // The candidate passes give one warp to every tile block (8 tiles per CTA): blocks are small
 // (about 1.4 % of a tile) and warps need no block-wide synchronisation.
 // Histograms over candidates, one warp per tile block; lanes holding the same digit add once
@@ -367,7 +360,6 @@ __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide 
 // the wide form of the finish step, for segments whose candidates are too many for one CTA:
 // level 1 = second digit of the candidates whose first digit is the threshold's, level 2 = last
 // 7 bits of the candidates under the 24-bit prefix.
-template <typename GT>
 __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_constant__ Params p, const TopkSide s,
                                                                   const int level, const int reps) {
     __shared__ uint32_t h[DIGIT1_BINS];
@@ -395,36 +387,31 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
         if (active) {
             cb = cand_block(p, s, tile, row);
             const uint32_t flags = cb.sel[SEL_FLAGS];
-            // (a dense problem knows its 24-bit prefix from the dense second-digit pass: level 2 only)
-            active = !cb.skip && !(cb.dense && level != 2) && !(level == 0 && cb.sel[SEL_MODE] != 1u) && !(level == 1 && flags != 0u);
+            active = !cb.skip && !(level == 0 && cb.sel[SEL_MODE] != 1u) && !(level == 1 && flags != 0u);
             prefix = cb.sel[SEL_PREFIX];
         }
         uint32_t lo = 0xffffffffu, hi = 0u;
         if (active) {
             uint32_t *gh = (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + cb.t) * DIGIT1_BINS;
-            auto walk = [&](auto &&value_at) {
-                for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
-                    const uint32_t q = c0 + lane;
-                    uint32_t digit = 0xffffffffu;  // lanes with nothing to add
-                    if (q < cb.cnt) {
-                        const uint32_t key = key_of(value_at(q));
-                        if (level == 0) digit = key >> DIGIT1_SHIFT;
-                        else if (level == 1) { if ((key >> DIGIT1_SHIFT) == prefix) digit = (key >> 7) & 0xfffu; }
-                        else if ((key >> 7) == prefix) digit = key & 0x7fu;
-                    }
-                    const uint32_t same = __match_any_sync(0xffffffffu, digit);
-                    if (digit != 0xffffffffu) {
-                        if (lane == __ffs(same) - 1) {
-                            if (gather) atomicAdd(&h[digit], (uint32_t)__popc(same));
-                            else atomicAdd(gh + digit, (uint32_t)__popc(same));
-                        }
-                        lo = min(lo, digit);
-                        hi = max(hi, digit);
-                    }
+            for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
+                const uint32_t q = c0 + lane;
+                uint32_t digit = 0xffffffffu;  // lanes with nothing to add
+                if (q < cb.cnt) {
+                    const uint32_t key = key_of(s.cand_val[cb.base + q]);
+                    if (level == 0) digit = key >> DIGIT1_SHIFT;
+                    else if (level == 1) { if ((key >> DIGIT1_SHIFT) == prefix) digit = (key >> 7) & 0xfffu; }
+                    else if ((key >> 7) == prefix) digit = key & 0x7fu;
                 }
-            };
-            if (cb.dense) walk([&](uint32_t q) { return fetch1<GT>(s, row, cb.t, cb.seg_beg, cb.rel + q); });
-            else walk([&](uint32_t q) { return s.cand_val[cb.base + q]; });
+                const uint32_t same = __match_any_sync(0xffffffffu, digit);
+                if (digit != 0xffffffffu) {
+                    if (lane == __ffs(same) - 1) {
+                        if (gather) atomicAdd(&h[digit], (uint32_t)__popc(same));
+                        else atomicAdd(gh + digit, (uint32_t)__popc(same));
+                    }
+                    lo = min(lo, digit);
+                    hi = max(hi, digit);
+                }
+            }
         }
         if (!gather && active) {  // (uniform over the warp)
             lo = __reduce_min_sync(0xffffffffu, lo);
@@ -443,7 +430,6 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
     }
 }
 
-template <typename GT>
 __global__ void __launch_bounds__(THREADS) topk_count_kernel(const __grid_constant__ Params p, const TopkSide s) {
     const int row = blockIdx.y, lane = threadIdx.x & 31;
     const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -452,26 +438,10 @@ __global__ void __launch_bounds__(THREADS) topk_count_kernel(const __grid_consta
     if (cb.skip) return;
     const uint32_t T = cb.sel[SEL_THRESH];
     uint32_t g = 0, e = 0;
-    if (!cb.dense) {
-        for (uint32_t q = lane; q < cb.cnt; q += 32) {
-            const uint32_t key = key_of(s.cand_val[cb.base + q]);
-            g += key > T ? 1u : 0u;
-            e += key == T ? 1u : 0u;
-        }
-    } else {
-        constexpr int UC = 8;   // elements per lane fetched together
-        for (uint32_t q0 = lane; q0 < cb.cnt; q0 += 32 * UC) {
-            uint32_t key[UC];
-#pragma unroll
-            for (int u = 0; u < UC; ++u)
-                key[u] = q0 + 32 * u < cb.cnt ? key_of(fetch1<GT>(s, row, cb.t, cb.seg_beg, cb.rel + q0 + 32 * u)) : 0u;
-#pragma unroll
-            for (int u = 0; u < UC; ++u) {
-                const bool in = q0 + 32 * u < cb.cnt;
-                g += in && key[u] > T ? 1u : 0u;
-                e += in && key[u] == T ? 1u : 0u;
-            }
-        }
+    for (uint32_t q = lane; q < cb.cnt; q += 32) {
+        const uint32_t key = key_of(s.cand_val[cb.base + q]);
+        g += key > T ? 1u : 0u;
+        e += key == T ? 1u : 0u;
     }
     g = __reduce_add_sync(0xffffffffu, g);
     e = __reduce_add_sync(0xffffffffu, e);
@@ -529,7 +499,6 @@ __global__ void __launch_bounds__(THREADS) topk_scan_kernel(const __grid_constan
 }
 
 // write: ordered compaction of a tile's candidate block into the message (one warp per tile)
-template <typename GT>
 __global__ void __launch_bounds__(THREADS) topk_write_kernel(const __grid_constant__ Params p, const TopkSide s) {
     const int row = blockIdx.y, lane = threadIdx.x & 31;
     const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
@@ -542,49 +511,168 @@ __global__ void __launch_bounds__(THREADS) topk_write_kernel(const __grid_consta
     const int64_t obase = (int64_t)row * p.K + s.outbase[(int64_t)row * (p.TT + 1) + tile];
     const int64_t oend = (int64_t)row * p.K + __ldg(p.k_off + cb.t + 1);  // never write past the segment's slots
     const uint32_t lt_mask = (1u << lane) - 1u;
-    auto walk = [&](auto &&entry_at) {   // entry_at(q, idx, val)
-        uint32_t run_sel = 0, run_tie = 0;
-        for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
-            const uint32_t q = c0 + lane;
-            const bool in = q < cb.cnt;
-            float val = 0.0f;
-            uint32_t idx = 0u;
-            if (in) entry_at(q, idx, val);
-            const uint32_t key = key_of(val);
-            const bool tie = in && key == T;
-            const uint32_t tb = __ballot_sync(0xffffffffu, tie);
-            const uint32_t tie_rank = run_tie + __popc(tb & lt_mask);
-            const bool take = in && (key > T || (tie && tie_rank < allowed));
-            const uint32_t sb = __ballot_sync(0xffffffffu, take);
-            if (take && obase + run_sel + __popc(sb & lt_mask) >= oend) {
-                atomicOr(p.status, STATUS_COUNT_MISMATCH);  // inconsistent selection state: drop the write
-            } else if (take) {
-                const uint32_t out = run_sel + __popc(sb & lt_mask);
-                s.idx[obase + out] = idx;
-                s.val[obase + out] = val;
-                if (s.zero_out) s.zero_out[idx] = 0.0f;
-                if (has_last && tie && tie_rank == allowed - 1) cb.sel[SEL_CUT] = idx;
-            }
-            run_sel += __popc(sb);
-            run_tie += __popc(tb);
+    uint32_t run_sel = 0, run_tie = 0;
+    for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
+        const uint32_t q = c0 + lane;
+        const bool in = q < cb.cnt;
+        const float val = in ? s.cand_val[cb.base + q] : 0.0f;
+        const uint32_t idx = in ? s.cand_idx[cb.base + q] : 0u;
+        const uint32_t key = key_of(val);
+        const bool tie = in && key == T;
+        const uint32_t tb = __ballot_sync(0xffffffffu, tie);
+        const uint32_t tie_rank = run_tie + __popc(tb & lt_mask);
+        const bool take = in && (key > T || (tie && tie_rank < allowed));
+        const uint32_t sb = __ballot_sync(0xffffffffu, take);
+        if (take && obase + run_sel + __popc(sb & lt_mask) >= oend) {
+            atomicOr(p.status, STATUS_COUNT_MISMATCH);  // inconsistent selection state: drop the write
+        } else if (take) {
+            const uint32_t out = run_sel + __popc(sb & lt_mask);
+            s.idx[obase + out] = idx;
+            s.val[obase + out] = val;
+            if (s.zero_out) s.zero_out[idx] = 0.0f;
+            if (has_last && tie && tie_rank == allowed - 1) cb.sel[SEL_CUT] = idx;
         }
-    };
-    if (cb.dense)
-        walk([&](uint32_t q, uint32_t &idx, float &val) {
-            idx = (uint32_t)(cb.seg_beg + cb.rel + q);
-            val = fetch1<GT>(s, row, cb.t, cb.seg_beg, cb.rel + q);
-        });
-    else
-        walk([&](uint32_t q, uint32_t &idx, float &val) { idx = s.cand_idx[cb.base + q]; val = s.cand_val[cb.base + q]; });
+        run_sel += __popc(sb);
+        run_tie += __popc(tb);
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
-// Wide form, last kernel of a side: closes the step's bookkeeping for every problem (one thread each).
+// Wide form, problems without candidates (SEL_FLAGS == 3: even the 24-bit prefix found by the dense
+// second-digit pass leaves more entries than the buffer holds: huge groups of equal keys, e.g. a
+// mostly-zero row whose k exceeds its non-zero count, or a vector of few distinct values).  Their
+// tiles are walked in the dense source, tile-parallel: the last-digit histogram before pick 3, the
+// per-tile counts before the scan, the ordered write after it; pick 3 and the scan treat them like
+// any other problem.  Small strided grids that leave after one load when no problem needs them.
 // ------------------------------------------------------------------------------------------------
+template <typename GT>
+__global__ void __launch_bounds__(THREADS) topk_dense_hist3_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    __shared__ uint32_t h[DIGIT1_BINS];
+    if (p.status[STATUS_ANY_DENSE + (s.zero_out ? 1 : 0)] == 0) return;
+    const int row = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int tile = blockIdx.x; tile < p.TT; tile += gridDim.x) {
+        const TileInfo ti = locate_tile(p, tile);
+        uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
+        if (sel[SEL_FLAGS] != 3u || ti.seg_tiles == 1) continue;  // uniform over the CTA
+        const uint32_t prefix = sel[SEL_PREFIX];
+        for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) h[b] = 0u;
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int pos = tile_pos(warp, lane, j);
+            float v[4];
+            fetch4<GT>(s, row, ti, pos, v);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t key = key_of(v[c]);
+                if (pos + c < ti.len && (key >> 7) == prefix) atomicAdd(&h[key & 0x7fu], 1u);
+            }
+        }
+        __syncthreads();
+        flush_hist(h, s.hist2 + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS, sel, SEL_LO2, SEL_HI2);
+        __syncthreads();
+    }
+}
+
+// entries above the threshold / equal to it per tile -> meta[2], meta[3] (what topk_count_kernel leaves)
+template <typename GT>
+__global__ void __launch_bounds__(THREADS) topk_dense_count_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    __shared__ uint32_t wg[8], we[8];
+    if (p.status[STATUS_ANY_DENSE + (s.zero_out ? 1 : 0)] == 0) return;
+    const int row = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int tile = blockIdx.x; tile < p.TT; tile += gridDim.x) {
+        const TileInfo ti = locate_tile(p, tile);
+        const uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
+        if (sel[SEL_FLAGS] != 3u || ti.seg_tiles == 1) continue;  // uniform over the CTA
+        const uint32_t T = sel[SEL_THRESH];
+        uint32_t g = 0, e = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int pos = tile_pos(warp, lane, j);
+            float v[4];
+            fetch4<GT>(s, row, ti, pos, v);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t key = key_of(v[c]);
+                const bool in = pos + c < ti.len;
+                g += in && key > T ? 1u : 0u;
+                e += in && key == T ? 1u : 0u;
+            }
+        }
+        g = __reduce_add_sync(0xffffffffu, g);
+        e = __reduce_add_sync(0xffffffffu, e);
+        if (lane == 0) { wg[warp] = g; we[warp] = e; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t *m = s.meta + ((int64_t)row * p.TT + tile) * 4;
+            m[2] = wg[0] + wg[1] + wg[2] + wg[3] + wg[4] + wg[5] + wg[6] + wg[7];
+            m[3] = we[0] + we[1] + we[2] + we[3] + we[4] + we[5] + we[6] + we[7];
+        }
+        __syncthreads();
+    }
+}
+
+// ordered write of a dense tile's selected elements: one warp per tile, 32 consecutive elements per
+// step (eight steps' elements fetched together); same rule as topk_write_kernel
+template <typename GT>
+__global__ void __launch_bounds__(THREADS) topk_dense_write_kernel(const __grid_constant__ Params p, const TopkSide s) {
+    if (p.status[STATUS_ANY_DENSE + (s.zero_out ? 1 : 0)] == 0) return;
+    const int row = blockIdx.y, lane = threadIdx.x & 31;
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    for (int tile = blockIdx.x * 8 + (threadIdx.x >> 5); tile < p.TT; tile += gridDim.x * 8) {
+        const TileInfo ti = locate_tile(p, tile);
+        uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
+        if (sel[SEL_FLAGS] != 3u || ti.seg_tiles == 1) continue;  // uniform over the warp
+        const uint32_t *m = s.meta + ((int64_t)row * p.TT + tile) * 4;
+        const uint32_t T = sel[SEL_THRESH];
+        const uint32_t allowed = m[3];
+        const bool has_last = m[2] != 0u;
+        const int64_t obase = (int64_t)row * p.K + s.outbase[(int64_t)row * (p.TT + 1) + tile];
+        const int64_t oend = (int64_t)row * p.K + __ldg(p.k_off + ti.t + 1);  // never write past the segment's slots
+        constexpr int SB = 8;
+        uint32_t run_sel = 0, run_tie = 0;
+        for (int c0 = 0; c0 < ti.len; c0 += 32 * SB) {
+            float val[SB];
+#pragma unroll
+            for (int u = 0; u < SB; ++u)
+                val[u] = c0 + 32 * u + lane < ti.len ? fetch1<GT>(s, row, ti.t, ti.seg_beg, ti.rel + c0 + 32 * u + lane) : 0.0f;
+#pragma unroll
+            for (int u = 0; u < SB; ++u) {
+                if (c0 + 32 * u >= ti.len) break;   // (uniform over the warp)
+                const int q = c0 + 32 * u + lane;
+                const bool in = q < ti.len;
+                const uint32_t idx = (uint32_t)(ti.seg_beg + ti.rel + q);
+                const uint32_t key = key_of(val[u]);
+                const bool tie = in && key == T;
+                const uint32_t tb = __ballot_sync(0xffffffffu, tie);
+                const uint32_t tie_rank = run_tie + __popc(tb & lt_mask);
+                const bool take = in && (key > T || (tie && tie_rank < allowed));
+                const uint32_t sb = __ballot_sync(0xffffffffu, take);
+                if (take && obase + run_sel + __popc(sb & lt_mask) >= oend) {
+                    atomicOr(p.status, STATUS_COUNT_MISMATCH);  // inconsistent selection state: drop the write
+                } else if (take) {
+                    const uint32_t out = run_sel + __popc(sb & lt_mask);
+                    s.idx[obase + out] = idx;
+                    s.val[obase + out] = val[u];
+                    if (s.zero_out) s.zero_out[idx] = 0.0f;
+                    if (has_last && tie && tie_rank == allowed - 1) sel[SEL_CUT] = idx;
+                }
+                run_sel += __popc(sb);
+                run_tie += __popc(tb);
+            }
+        }
+    }
+}
+
+// Wide form, last kernel of a side: closes the step's bookkeeping for every problem (one thread each).
 __global__ void topk_close_kernel(const __grid_constant__ Params p, const TopkSide s) {
     const int t = blockIdx.x * blockDim.x + threadIdx.x, row = blockIdx.y;
-    // the next step starts with "no problem on the regular route yet"
-    if (s.spec && t == 0 && row == 0) p.status[STATUS_ANY_REGULAR] = 0;
+    if (t == 0 && row == 0) {
+        if (s.spec) p.status[STATUS_ANY_REGULAR] = 0;   // the next step starts with "no problem on the regular route yet"
+        p.status[STATUS_ANY_DENSE + (s.zero_out ? 1 : 0)] = 0;
+    }
     if (t >= p.T) return;
     if (__ldg(p.tile_prefix + t + 1) - __ldg(p.tile_prefix + t) == 1) return;   // selected directly by one CTA
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
@@ -770,7 +858,7 @@ cudaError_t topk_first_part(const Params &p, const TopkSide &s, int src_kind, cu
         if (e != cudaSuccess) return e;
         ++*launches;
         if (!use_fused_tail(p)) {   // wide form: first digit of the single-pass problems from a global histogram
-            topk_cand_hist_kernel<float><<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 0, cand_hist_reps(p)); CHECK_LAUNCH();   // (candidates only at this level)
+            topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 0, cand_hist_reps(p)); CHECK_LAUNCH();
             topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 5); CHECK_LAUNCH();
         }
     }
@@ -796,20 +884,16 @@ cudaError_t topk_second_part(const Params &p, const TopkSide &s, int src_kind, c
     LAUNCH_BY_SOURCE(topk_filter_tma_kernel, g_filter, COMMA false);
     if (use_fused_tail(p)) return launch_topk_tail(p, s, src_kind, st, launches);
     // some segment has too many candidates or tiles for one CTA: the same steps, spread over the tile blocks
-    // (problems left without candidates - huge groups of equal keys - are walked in the dense source by
-    //  the same kernels from the last-digit histogram on: tile-parallel like everything else here)
-    const int reps = cand_hist_reps(p);
-    const dim3 g_hist = cand_hist_grid(p, s.R);
-    topk_cand_hist_kernel<float><<<g_hist, THREADS, 0, st>>>(p, s, 1, reps); CHECK_LAUNCH();
+    topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 1, cand_hist_reps(p)); CHECK_LAUNCH();
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();
-    if (src_kind == SRC_BF16) topk_cand_hist_kernel<__nv_bfloat16><<<g_hist, THREADS, 0, st>>>(p, s, 2, reps);
-    else if (src_kind == SRC_SCORES) topk_cand_hist_kernel<ScoreGen><<<g_hist, THREADS, 0, st>>>(p, s, 2, reps);
-    else topk_cand_hist_kernel<float><<<g_hist, THREADS, 0, st>>>(p, s, 2, reps);
-    CHECK_LAUNCH();
+    topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 2, cand_hist_reps(p)); CHECK_LAUNCH();
+    LAUNCH_BY_SOURCE(topk_dense_hist3_kernel, g_strided);
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 3); CHECK_LAUNCH();
-    LAUNCH_BY_SOURCE(topk_count_kernel, g_warp_tiles);
+    topk_count_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+    LAUNCH_BY_SOURCE(topk_dense_count_kernel, g_strided);
     topk_scan_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
-    LAUNCH_BY_SOURCE(topk_write_kernel, g_warp_tiles);
+    topk_write_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+    LAUNCH_BY_SOURCE(topk_dense_write_kernel, g_strided);
     topk_close_kernel<<<dim3((p.T + 127) / 128, s.R), 128, 0, st>>>(p, s); CHECK_LAUNCH();
     return cudaSuccess;
 }
