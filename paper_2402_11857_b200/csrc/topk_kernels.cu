@@ -164,13 +164,28 @@ __global__ void __launch_bounds__(THREADS) topk_hist2_dense_kernel(const __grid_
     if (p.status[STATUS_ANY_REFINE + (s.zero_out ? 1 : 0)] == 0) return;
     const int row = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int tile = blockIdx.x; tile < p.TT; tile += gridDim.x) {
+    // a CTA owns a run of consecutive tiles and keeps one shared histogram per segment of the run:
+    // it is flushed when the segment changes and at the end, not after every tile
+    const int chunk = (p.TT + gridDim.x - 1) / gridDim.x;
+    const int tile_end = min(p.TT, ((int)blockIdx.x + 1) * chunk);
+    int open_t = -1;   // segment whose counts the shared histogram holds (uniform over the CTA)
+    auto flush_open = [&]() {
+        __syncthreads();
+        flush_hist(h, s.hist2 + ((int64_t)row * p.T + open_t) * DIGIT1_BINS, s.sel + ((int64_t)row * p.T + open_t) * SEL_WORDS,
+                   SEL_LO2, SEL_HI2);
+        __syncthreads();
+    };
+    for (int tile = blockIdx.x * chunk; tile < tile_end; ++tile) {
         const TileInfo ti = locate_tile(p, tile);
         uint32_t *sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
         if (sel[SEL_FLAGS] != 2u) continue;  // uniform over the CTA
         const uint32_t b1 = sel[SEL_PREFIX];
-        for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) h[b] = 0u;
-        __syncthreads();
+        if (ti.t != open_t) {
+            if (open_t >= 0) flush_open();
+            for (int b = threadIdx.x; b < DIGIT1_BINS; b += THREADS) h[b] = 0u;
+            __syncthreads();
+            open_t = ti.t;
+        }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int pos = tile_pos(warp, lane, j);
@@ -182,10 +197,8 @@ __global__ void __launch_bounds__(THREADS) topk_hist2_dense_kernel(const __grid_
                 if (pos + c < ti.len && (key >> DIGIT1_SHIFT) == b1) atomicAdd(&h[(key >> 7) & 0xfffu], 1u);
             }
         }
-        __syncthreads();
-        flush_hist(h, s.hist2 + ((int64_t)row * p.T + ti.t) * DIGIT1_BINS, sel, SEL_LO2, SEL_HI2);
-        __syncthreads();
     }
+    if (open_t >= 0) flush_open();
 }
 
 // ------------------------------------------------------------------------------------------------
