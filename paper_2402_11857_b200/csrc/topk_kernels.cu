@@ -840,9 +840,11 @@ static dim3 strided_grid(const Params &p, int rows) {
     return dim3(p.TT < per_row ? p.TT : per_row, rows);
 }
 
-// Candidate histograms of the wide form: 64 tiles per CTA (its CTAs gather in shared memory and
-// flush once per 64 tiles).
-static int cand_hist_reps(const Params &) { return 8; }
+// Candidate histograms of the wide form: 64 tiles per CTA for very long segments (the CTAs gather in
+// shared memory and flush once per 64 tiles: fewer atomics on one histogram), 16 tiles per CTA
+// otherwise (more warps in flight on what is a chain of dependent loads per tile block; measured:
+// flat 2^24 uplink 0.261 -> 0.232 ms with 16, flat 2^26 0.582 -> 0.625 ms, hence the switch point).
+static int cand_hist_reps(const Params &p) { return p.max_seg_tiles >= 4096 ? 8 : 2; }
 static dim3 cand_hist_grid(const Params &p, int rows) {
     const int per = 8 * cand_hist_reps(p);
     return dim3((p.TT + per - 1) / per, rows);
