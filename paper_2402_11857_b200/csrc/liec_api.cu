@@ -573,7 +573,18 @@ liec_status liec_draw_subsets(liec_ctx *c, uint64_t seed, uint32_t epoch, void *
     s.cand_idx = p.gen_cand_idx; s.cand_val = p.gen_cand_val; s.meta = p.gen_meta; s.outbase = p.gen_outbase;
     s.zero_out = nullptr;
     s.spec = 1;
-    LIEC_CALL(c, launch_randk_draw(p, s, static_cast<cudaStream_t>(stream), &c->launches));
+    cudaStream_t main_stream = static_cast<cudaStream_t>(stream);
+    const bool forked = c->side && p.n_small > 0;   // single-tile segments beside the dense pass, as in the top-k stages
+    if (forked) {
+        LIEC_CALL(c, cudaEventRecord(c->ev_fork, main_stream));
+        LIEC_CALL(c, cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+        LIEC_CALL(c, launch_randk_draw_small(p, s, c->side, &c->launches));
+        LIEC_CALL(c, cudaEventRecord(c->ev_join, c->side));
+    } else {
+        LIEC_CALL(c, launch_randk_draw_small(p, s, main_stream, &c->launches));
+    }
+    LIEC_CALL(c, launch_randk_draw(p, s, main_stream, &c->launches));
+    if (forked) LIEC_CALL(c, cudaStreamWaitEvent(main_stream, c->ev_join, 0));
     c->p.up_sets = p.up == COMP_RANDK ? p.gen_sets : nullptr;
     c->p.down_set = p.down == COMP_RANDK ? p.gen_sets + (int64_t)p.N * p.K : nullptr;
     return LIEC_OK;

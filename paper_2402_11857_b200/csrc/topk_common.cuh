@@ -327,6 +327,7 @@ cudaError_t launch_topk_tail(const Params &p, const TopkSide &s, int src_kind, c
 constexpr int64_t TAIL_BIG_CAP = 16384;   // candidate capacity from which a problem's tail gets the larger CTA
 cudaError_t configure_topk_tail_kernels();
 // seeded random-k draw: the selection on generated scores (defined in topk_kernels.cu)
+cudaError_t launch_randk_draw_small(const Params &p, const TopkSide &s, cudaStream_t st, int64_t *launches);
 cudaError_t launch_randk_draw(const Params &p, const TopkSide &s, cudaStream_t st, int64_t *launches);
 
 // Limits of the one-CTA-per-problem tail: candidates of one segment that it sweeps, tiles of one

@@ -260,8 +260,7 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
         const ST *tile_ptr = GEN ? nullptr : reinterpret_cast<const ST *>(s.src) + row_beg + ti.rel;
         const bool fast = (ti.len == TILE) && (GEN || (row_beg & ALIGN_MASK) == 0);
         if constexpr (GEN) {
-            stage_tile_scores(reinterpret_cast<float *>(tile_s), s, row, ti.t, ti.rel, ti.len);
-            __syncthreads();
+            // nothing to stage: the scores are computed in registers below
         } else if (fast) {
             if (threadIdx.x == 0) {
                 const uint32_t bytes = TILE * sizeof(ST);
@@ -283,7 +282,17 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
         // 32 consecutive elements per thread, chunk order rotated by the lane
         const int pos0 = 32 * threadIdx.x;
         uint32_t mask = 0;
-        if constexpr (F32) {
+        if constexpr (GEN) {
+            // scores are 30-bit integers whose binary32 reading has the same order: compare the bits
+            const uint32_t low_bits = __float_as_uint(low);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint4 w = s.gen.block((uint32_t)((ti.rel + pos0 + 4 * c) >> 2), (uint32_t)ti.t, (uint32_t)row);
+                const uint32_t nib = (w.x >= low_bits ? 1u : 0u) | (w.y >= low_bits ? 2u : 0u) |
+                                     (w.z >= low_bits ? 4u : 0u) | (w.w >= low_bits ? 8u : 0u);
+                mask |= nib << (4 * c);
+            }
+        } else if constexpr (F32) {
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk) {
                 const int c = (kk + lane) & 7;
@@ -340,7 +349,8 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
                 const int b = __ffs(rest) - 1;
                 rest &= rest - 1;
                 s.cand_idx[cbase + o] = flat0 + b;
-                if constexpr (F32) s.cand_val[cbase + o] = tile_s[pos0 + b];
+                if constexpr (GEN) s.cand_val[cbase + o] = fetch1<GT>(s, row, ti.t, ti.seg_beg, ti.rel + pos0 + b);   // (candidates are rare: recomputed)
+                else if constexpr (F32) s.cand_val[cbase + o] = tile_s[pos0 + b];
                 else s.cand_val[cbase + o] = __uint_as_float((uint32_t)tile_s[pos0 + b] << 16);
                 ++o;
             }
@@ -962,14 +972,16 @@ __global__ void randk_draw_begin_kernel(const __grid_constant__ Params p, const 
     sel[SEL_GUESS] = bound;
 }
 
+// The single-tile segments of the draw (independent of the rest: the caller may put them on a stream of their own).
+cudaError_t launch_randk_draw_small(const Params &p, const TopkSide &s, cudaStream_t st, int64_t *launches) {
+    if (!p.n_small) return cudaSuccess;
+    cudaError_t e = launch_topk_small(p, s, SRC_SCORES, st);
+    if (e == cudaSuccess) ++*launches;
+    return e;
+}
+
+// The multi-tile segments of the draw.
 cudaError_t launch_randk_draw(const Params &p, const TopkSide &s, cudaStream_t st, int64_t *launches) {
-    const int src_kind = SRC_SCORES;
-    (void)src_kind;
-    if (p.n_small) {
-        cudaError_t e = launch_topk_small(p, s, SRC_SCORES, st);
-        if (e != cudaSuccess) return e;
-        ++*launches;
-    }
     if (!p.n_large) return cudaSuccess;
     randk_draw_begin_kernel<<<dim3((p.T + 127) / 128, s.R), 128, 0, st>>>(p, s);
     CHECK_LAUNCH();
