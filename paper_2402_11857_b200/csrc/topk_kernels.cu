@@ -767,10 +767,12 @@ __global__ void __launch_bounds__(THREADS, TEL ? 3 : 4) server_topk_kernel(const
         __syncthreads();
         uint32_t pidx[WG];
         float pval[WG];
+        uint32_t crowded = 0;   // workers with more than 256 entries in this tile (uniform over the CTA)
 #pragma unroll
         for (int u = 0; u < WG; ++u) {
             const uint32_t q = s_beg[u] + threadIdx.x;
             const bool have = q < s_end[u];   // (beg = end = 0 for workers beyond N)
+            crowded |= (s_end[u] - s_beg[u] > (uint32_t)THREADS ? 1u : 0u) << u;
             const int64_t at = (int64_t)(g0 + u) * p.K + q;
             pidx[u] = have ? p.up_idx[at] : 0xffffffffu;
             pval[u] = have ? p.up_val[at] : 0.0f;
@@ -780,17 +782,20 @@ __global__ void __launch_bounds__(THREADS, TEL ? 3 : 4) server_topk_kernel(const
             if (g0 + u < p.N) {  // uniform over the CTA
                 const uint32_t o = pidx[u] - tile_first;
                 if (o < (uint32_t)TILE) acc[o] = __fadd_rn(acc[o], pval[u]);  // (absent entries and those of a refused subset fall outside)
-                const uint32_t *idx = p.up_idx + (int64_t)(g0 + u) * p.K;
-                const float *val = p.up_val + (int64_t)(g0 + u) * p.K;
-                for (uint32_t q = s_beg[u] + threadIdx.x + THREADS; q < s_end[u]; q += THREADS) {  // more than 256 entries in this tile
-                    const uint32_t o2 = idx[q] - tile_first;
-                    if (o2 < (uint32_t)TILE) acc[o2] = __fadd_rn(acc[o2], val[q]);
+                if ((crowded >> u) & 1u) {
+                    const uint32_t *idx = p.up_idx + (int64_t)(g0 + u) * p.K;
+                    const float *val = p.up_val + (int64_t)(g0 + u) * p.K;
+                    for (uint32_t q = s_beg[u] + threadIdx.x + THREADS; q < s_end[u]; q += THREADS) {
+                        const uint32_t o2 = idx[q] - tile_first;
+                        if (o2 < (uint32_t)TILE) acc[o2] = __fadd_rn(acc[o2], val[q]);
+                    }
                 }
                 __syncthreads();
             }
         }
     }
     const WorkerDivisor by_n(p.N);
+    const bool with_hist = ti.seg_tiles > 1;   // (single-tile segments are selected directly from v)
     const int64_t wbase = __ldg(p.word_off + ti.t) + ti.rel / 32;
     const int nwords = (ti.len + 31) >> 5;
     double a[8];
@@ -802,13 +807,24 @@ __global__ void __launch_bounds__(THREADS, TEL ? 3 : 4) server_topk_kernel(const
         const float4 a4 = *reinterpret_cast<const float4 *>(&acc[pos]);
         const float av[4] = {a4.x, a4.y, a4.z, a4.w};
         by_n.div4(av, v);
+        if (fast) {   // one 128-bit store when any of the four changed (the others are rewritten with their own bits)
+            bool changed = false;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const bool valid = fast || pos + c < ti.len;
-            v[c] = __fadd_rn(ev[j][c], v[c]);
-            if (!valid) v[c] = 0.0f;
-            if (valid && __float_as_uint(v[c]) != __float_as_uint(ev[j][c])) e_tile[pos + c] = v[c];
-            if (DOWN == COMP_TOPK && valid && ti.seg_tiles > 1) atomicAdd(&h[key_of(v[c]) >> DIGIT1_SHIFT], 1u);
+            for (int c = 0; c < 4; ++c) {
+                v[c] = __fadd_rn(ev[j][c], v[c]);
+                changed |= __float_as_uint(v[c]) != __float_as_uint(ev[j][c]);
+                if (DOWN == COMP_TOPK && with_hist) atomicAdd(&h[key_of(v[c]) >> DIGIT1_SHIFT], 1u);
+            }
+            if (changed) *reinterpret_cast<float4 *>(e_tile + pos) = make_float4(v[0], v[1], v[2], v[3]);
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const bool valid = pos + c < ti.len;
+                v[c] = __fadd_rn(ev[j][c], v[c]);
+                if (!valid) v[c] = 0.0f;
+                if (valid && __float_as_uint(v[c]) != __float_as_uint(ev[j][c])) e_tile[pos + c] = v[c];
+                if (DOWN == COMP_TOPK && valid && with_hist) atomicAdd(&h[key_of(v[c]) >> DIGIT1_SHIFT], 1u);
+            }
         }
         if constexpr (TEL) tv[j] = leaf4_sq(v);
         if (DOWN == COMP_SIGN) {
