@@ -253,39 +253,100 @@ __global__ void __launch_bounds__(THREADS) server_dense_kernel(const __grid_cons
 // tile, i.e. exactly one word of every worker's message, so unpacking needs no shuffles
 // (shift + sign-xor + add per element and worker), the word of v is built in-thread and the
 // ||v||_1 leaf covers five tree levels in-thread.
+// Nibble k of the result is nibble k ^ m of w (m in 0..7; its own inverse).  sel = 0x3210 ^ ((m >> 1) * 0x1111).
+__device__ __forceinline__ uint32_t nibble_xor_perm(uint32_t w, uint32_t m, uint32_t sel) {
+    const uint32_t sw = ((w & 0x0f0f0f0fu) << 4) | ((w >> 4) & 0x0f0f0f0fu);
+    return __byte_perm((m & 1u) ? sw : w, 0u, sel);
+}
+
 template <bool DOWN_SIGN, bool TEL>
 __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_constant__ Params p) {
+    __shared__ __align__(128) float tile_s[TILE];  // the tile of e, then of v
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int copy_ok;
     __shared__ double warp_sums[8];
     __shared__ double tel_sums[TEL ? 16 : 1];
     constexpr int SCALE_CHUNK = 1024;              // workers whose scales are staged at once (a multiple of WG)
     __shared__ float up_scale_smem[SCALE_CHUNK];   // this segment's scales of workers c0 .. c0 + SCALE_CHUNK - 1
     const TileInfo ti = locate_tile(p, blockIdx.x);
-    const int lane = threadIdx.x & 31;
     const bool fast = (ti.len == TILE) && ((ti.seg_beg & 3) == 0);
     const int64_t wbase = __ldg(p.word_off + ti.t) + ti.rel / 32;
     const int nwords = (ti.len + 31) >> 5;
     const int my_widx = threadIdx.x;
     const bool have_word = my_widx < nwords;
+    float *e_tile = p.e + ti.seg_beg + ti.rel;
 
-    float acc[32];
+    // Thread q owns word q of the tile = elements 32q .. 32q+31, which it reads from shared memory as
+    // eight 16-byte chunks; the tile comes in by one bulk copy (or guarded loads for a ragged or
+    // misaligned tile) and v leaves by coalesced stores, so no global access is strided.  To keep the
+    // shared-memory reads free of bank conflicts the thread takes its chunks in the order k ^ (q & 7),
+    // and permutes the nibbles of every sign word the same way: slot (k, j) of its registers is then
+    // element 4 (k ^ (q & 7)) + j throughout.  The binary64 tree over a thread's eight chunks does not
+    // see the order: a XOR permutation of the leaves only swaps the operands of additions.
+    const uint32_t rot = threadIdx.x & 7u;
+    const uint32_t rot_sel = 0x3210u ^ ((rot >> 1) * 0x1111u);
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bar)));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        copy_ok = 1;
+        if (fast) {
+            const uint32_t bytes = TILE * sizeof(float);
+            bulk_copy_g2s(tile_s, e_tile, bytes, bytes + p.copy_expect_extra, &bar);
+        }
+    }
+    if (!fast) stage_tile_guarded(tile_s, e_tile, ti.len, (ti.seg_beg & 3) == 0);
+
+    // The first 8 workers' contribution to an element depends only on their 8 sign bits there: the
+    // running sum ((+0 + p^0) + p^1) + ... + p^7 is tabulated once per CTA for the 256 bit patterns (entry
+    // t by thread t, the same additions in the same order), and an element looks its pattern up.  The
+    // patterns of a thread's 32 elements come from a bit transposition of its 8 words: X[c] holds, in
+    // byte k, the pattern of slot c + 8k.  The workers after the eighth are added one by one.
+    constexpr int HEAD = 8;
+    __shared__ float head_sum[1 << HEAD];
+    static_assert(THREADS == (1 << HEAD), "one table entry per thread");
+    const uint32_t *wp = p.up_words + wbase + my_widx;
+    uint32_t hw[HEAD];
 #pragma unroll
-    for (int c = 0; c < 32; ++c) acc[c] = 0.0f;
+    for (int r = 0; r < HEAD; ++r) hw[r] = (have_word && r < p.N) ? __ldg(wp + (int64_t)r * p.W) : 0u;
     // workers four at a time: their four words are fetched together, one group ahead of use
     constexpr int WG = 4;
-    const uint32_t *wp = p.up_words + wbase + my_widx;
     uint32_t nextw[WG];
 #pragma unroll
-    for (int u = 0; u < WG; ++u) nextw[u] = (have_word && u < p.N) ? __ldg(wp + (int64_t)u * p.W) : 0u;
-    for (int i0 = 0; i0 < p.N; i0 += WG) {
+    for (int u = 0; u < WG; ++u) nextw[u] = (have_word && HEAD + u < p.N) ? __ldg(wp + (int64_t)(HEAD + u) * p.W) : 0u;
+    for (int i = threadIdx.x; i < SCALE_CHUNK && i < p.N; i += THREADS) up_scale_smem[i] = p.up_scales[(int64_t)i * p.T + ti.t];
+    __syncthreads();
+    {
+        float a = 0.0f;
+#pragma unroll
+        for (int r = 0; r < HEAD; ++r)
+            if (r < p.N) a = __fadd_rn(a, __uint_as_float(__float_as_uint(up_scale_smem[r]) ^ (((threadIdx.x >> r) & 1u) << 31)));
+        head_sum[threadIdx.x] = a;   // (bits of absent workers are zero in every pattern)
+    }
+    __syncthreads();
+    float acc[32];
+    {
+        uint32_t X[8];
+#pragma unroll
+        for (int r = 0; r < HEAD; ++r) hw[r] = nibble_xor_perm(hw[r], rot, rot_sel);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            X[c] = 0u;
+#pragma unroll
+            for (int r = 0; r < HEAD; ++r) X[c] |= (r >= c ? hw[r] << (r - c) : hw[r] >> (c - r)) & (0x01010101u << r);
+        }
+#pragma unroll
+        for (int c = 0; c < 32; ++c) acc[c] = head_sum[(X[c & 7] >> (8 * (c >> 3))) & 0xffu];
+    }
+    for (int i0 = HEAD; i0 < p.N; i0 += WG) {
         if ((i0 & (SCALE_CHUNK - 1)) == 0) {  // (uniform over the CTA) next chunk of scales
-            if (i0) __syncthreads();
+            __syncthreads();
             for (int i = threadIdx.x; i < SCALE_CHUNK && i0 + i < p.N; i += THREADS)
                 up_scale_smem[i] = p.up_scales[(int64_t)(i0 + i) * p.T + ti.t];
             __syncthreads();
         }
         uint32_t w[WG];
 #pragma unroll
-        for (int u = 0; u < WG; ++u) w[u] = nextw[u];
+        for (int u = 0; u < WG; ++u) w[u] = nibble_xor_perm(nextw[u], rot, rot_sel);
 #pragma unroll
         for (int u = 0; u < WG; ++u) {
             const int i = i0 + WG + u;
@@ -304,21 +365,27 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
         }
     }
 
+    // the tile of e must have landed by now
+    if (fast && threadIdx.x == 0 && !mbar_wait_bounded(&bar, 0u, p.copy_wait_limit)) {
+        atomicOr(p.status, STATUS_COPY_TIMEOUT);
+        mbar_drain(&bar, 0u);
+        copy_ok = 0;
+    }
+    __syncthreads();
+    if (!copy_ok) return;   // (nothing has been written)
+
     const WorkerDivisor by_n(p.N);
     const int pos0 = 32 * threadIdx.x;
-    float *e_tile = p.e + ti.seg_beg + ti.rel;
     uint32_t vword = 0u;
     double leaf[8];
     double te[TEL ? 8 : 1], tv[TEL ? 8 : 1];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-        const int pos = pos0 + 4 * k;
+        const int pos = pos0 + 4 * (k ^ (int)rot);
         float ev[4], v[4];
-        if (fast) {
-            const float4 q = *reinterpret_cast<const float4 *>(e_tile + pos);
+        {
+            const float4 q = *reinterpret_cast<const float4 *>(&tile_s[pos]);
             ev[0] = q.x; ev[1] = q.y; ev[2] = q.z; ev[3] = q.w;
-        } else {
-            load4_guarded(e_tile, pos, ti.len, ev);
         }
         if constexpr (TEL) te[k] = leaf4_sq(ev);
         {
@@ -326,20 +393,27 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
             by_n.div4(a4, v);
         }
 #pragma unroll
-        for (int c = 0; c < 4; ++c) v[c] = __fadd_rn(ev[c], v[c]);
-        if (fast) {
-            *reinterpret_cast<float4 *>(e_tile + pos) = make_float4(v[0], v[1], v[2], v[3]);
-        } else {
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                if (pos + c < ti.len) e_tile[pos + c] = v[c]; else v[c] = 0.0f;
-            }
+        for (int c = 0; c < 4; ++c) {
+            v[c] = __fadd_rn(ev[c], v[c]);
+            if (!fast && pos + c >= ti.len) v[c] = 0.0f;
         }
+        *reinterpret_cast<float4 *>(&tile_s[pos]) = make_float4(v[0], v[1], v[2], v[3]);
         if constexpr (TEL) tv[k] = leaf4_sq(v);
         if (DOWN_SIGN) {
             leaf[k] = leaf4(v);
             vword |= sign_nibble(v) << (4 * k);
         }
+    }
+    __syncthreads();
+    // v over e, coalesced
+    if (fast) {
+#pragma unroll
+        for (int c = 0; c < TILE / 4 / THREADS; ++c) {
+            const int q = c * THREADS + threadIdx.x;
+            reinterpret_cast<float4 *>(e_tile)[q] = reinterpret_cast<const float4 *>(tile_s)[q];
+        }
+    } else {
+        for (int q = threadIdx.x; q < ti.len; q += THREADS) e_tile[q] = tile_s[q];
     }
     // a thread's 32 consecutive elements: three more tree levels in-thread, five across the lanes
     auto thread_then_warp = [](const double (&l)[8]) {
@@ -350,7 +424,7 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
         return s;
     };
     if (DOWN_SIGN) {
-        if (have_word) p.down_words[wbase + my_widx] = vword;
+        if (have_word) p.down_words[wbase + my_widx] = nibble_xor_perm(vword, rot, rot_sel);
         const double s = cta_tree_reduce(thread_then_warp(leaf), warp_sums);
         if (threadIdx.x == 0) p.down_partials[blockIdx.x] = s;
     }
@@ -359,7 +433,6 @@ __global__ void __launch_bounds__(THREADS) server_sign_kernel(const __grid_const
         cta_tree_reduce_pair(thread_then_warp(te), thread_then_warp(tv), tel_sums, re, rv);
         if (threadIdx.x == 0) { p.tel_e[blockIdx.x] = re; p.tel_v[blockIdx.x] = rv; }
     }
-    (void)lane;
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -96,6 +96,33 @@ def test_bulk_copy_wait_runs_out_sign_bf16():
     _flagged_then_recovers(lambda: Pair(1, [0, 8192], SIGN, SIGN, grad_dtype=liec.BF16), G, 0.01)
 
 
+def test_bulk_copy_wait_runs_out_sign_server_pass():
+    """The sign server pass stages its tile of e by a bulk copy: when that wait runs out the pass sets
+    bit 8 and leaves e and the downlink words alone; after abort + clear the next steps match the oracle."""
+    off = [0, 2 * 8192, 2 * 8192 + 100]      # two full tiles (bulk copies) and a ragged one (guarded loads)
+    P = Pair(2, off, SIGN, SIGN)
+    P.step(make_gradients("normal", 1.0, 2, off[-1], 0, base_seed=79), 0.1)
+    ctx = P.ctx
+    G = make_gradients("normal", 1.0, 2, off[-1], 1, base_seed=79)
+    Gd = G.cuda()
+    ctx.liec_uplink_compress(Gd)
+    torch.cuda.synchronize()
+    e_before, words_before = P.ed.clone(), ctx.liec_get_messages()["down_words"].clone()
+    ctx.liec_set_copy_wait(poll_limit=1000, expect_extra_bytes=16)
+    ctx.liec_server_aggregate()
+    torch.cuda.synchronize()
+    assert ctx.liec_device_status() & 8
+    assert torch.equal(P.ed[: 2 * 8192], e_before[: 2 * 8192])      # (the ragged tile has no bulk copy and is done)
+    assert torch.equal(ctx.liec_get_messages()["down_words"][: 2 * 256], words_before[: 2 * 256])
+    P.ed.copy_(e_before)                     # the state after a flagged iteration is the caller's to restore
+    ctx.liec_abort_step()
+    ctx.liec_set_copy_wait()
+    ctx.liec_clear_status()
+    assert ctx.liec_device_status() == 0
+    for step in (1, 2):
+        P.step(make_gradients("normal", 1.0, 2, off[-1], step, base_seed=79), 0.1)
+
+
 def test_bulk_copy_wait_runs_out_topk_filter():
     """Two full tiles of one segment (a single-tile segment would be selected without any bulk copy)."""
     G = make_gradients("normal", 1.0, 1, 16384, 0, base_seed=75)
