@@ -376,6 +376,15 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
         while (p.n_big < p.n_large && cap_of(p.n_big) >= TAIL_BIG_CAP) ++p.n_big;
         for (int q = p.n_big; q < p.n_large; ++q) p.cap_rest_max = std::max<int64_t>(p.cap_rest_max, cap_of(q));
     }
+    p.n_long = 0;
+    p.cap_long_max = 0;
+    if (pl.K > 0) {
+        auto tiles_of = [&](int q) { return pl.tile_prefix[pl.large_seg[q] + 1] - pl.tile_prefix[pl.large_seg[q]]; };
+        while (p.n_long < p.n_large && tiles_of(p.n_long) >= LONG_SEG_TILES) {
+            p.cap_long_max = std::max<int64_t>(p.cap_long_max, pl.cap_off[pl.large_seg[p.n_long] + 1] - pl.cap_off[pl.large_seg[p.n_long]]);
+            ++p.n_long;
+        }
+    }
     {
         int dev = 0, sms = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms = 0;

@@ -40,6 +40,8 @@ struct Params {
     int32_t n_small, n_large;
     int32_t n_big;               // leading entries of large_seg whose candidate capacity is TAIL_BIG_CAP or more
     int64_t cap_rest_max;        // largest candidate capacity among the other entries of large_seg
+    int32_t n_long;              // leading entries of large_seg with LONG_SEG_TILES tiles or more
+    int64_t cap_long_max;        // largest candidate capacity among them
     // host side only: the context's helper stream and the events that fork / join the tail launch of
     // the big problems (cudaStream_t / cudaEvent_t; NULL = everything on the caller's stream)
     void *tail_stream, *tail_fork, *tail_join;
@@ -103,6 +105,7 @@ struct Params {
     uint32_t copy_wait_limit, copy_expect_extra;
 };
 constexpr uint32_t COPY_WAIT_LIMIT_DEFAULT = 1u << 20;
+constexpr int LONG_SEG_TILES = 1024;   // from here on a segment's candidate passes walk its candidate region as a whole, not tile block by tile block
 
 // per-problem selection state words
 constexpr int SEL_WORDS = 20;

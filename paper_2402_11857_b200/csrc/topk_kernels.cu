@@ -362,12 +362,13 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
 // ------------------------------------------------------------------------------------------------
 // candidate passes: one CTA per (tile, row) walks that tile's block of the candidate buffer
 // ------------------------------------------------------------------------------------------------
-struct CandBlock { int64_t base; uint32_t cnt; int t; uint32_t *sel; uint32_t *meta; bool skip; };
+struct CandBlock { int64_t base; uint32_t cnt; int t, seg_tiles; uint32_t *sel; uint32_t *meta; bool skip; };
 
 __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide &s, int tile, int row) {
     CandBlock cb;
     const TileInfo ti = locate_tile(p, tile);
     cb.t = ti.t;
+    cb.seg_tiles = ti.seg_tiles;
     cb.sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
     cb.meta = s.meta + ((int64_t)row * p.TT + tile) * 4;
     cb.skip = (cb.sel[SEL_FLAGS] & 1u) != 0u || ti.seg_tiles == 1;
@@ -385,22 +386,9 @@ __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide 
 // 7 bits of the candidates under the 24-bit prefix.
 __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_constant__ Params p, const TopkSide s,
                                                                   const int level, const int reps) {
-    __shared__ uint32_t h[DIGIT1_BINS];
     const int row = blockIdx.y, lane = threadIdx.x & 31;
     // a CTA owns 8 * reps consecutive tiles; warp w takes tiles tile0 + w, tile0 + 8 + w, ...
     const int tile0 = blockIdx.x * 8 * reps;
-    // When all of the CTA's tiles lie in one very large segment the counts are
-    // first gathered in shared memory, so that the segment's global histogram sees a few atomics
-    // per CTA instead of a few per warp and iteration.
-    const int tlast = min(tile0 + 8 * reps - 1, p.TT - 1);
-    const int seg0 = __ldg(p.tile_seg + tile0);
-    // (worth its fixed cost only where many CTAs hammer one histogram: segments of 1024+ tiles)
-    const bool gather = seg0 == __ldg(p.tile_seg + tlast) &&
-                        __ldg(p.tile_prefix + seg0 + 1) - __ldg(p.tile_prefix + seg0) >= 1024;
-    if (gather) {
-        for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(h)[b] = make_uint4(0u, 0u, 0u, 0u);
-        __syncthreads();
-    }
     const int lo_word = level == 0 ? SEL_LO1 : SEL_LO2, hi_word = level == 0 ? SEL_HI1 : SEL_HI2;
     for (int rep = 0; rep < reps; ++rep) {
         const int tile = tile0 + rep * 8 + (threadIdx.x >> 5);
@@ -410,7 +398,8 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
         if (active) {
             cb = cand_block(p, s, tile, row);
             const uint32_t flags = cb.sel[SEL_FLAGS];
-            active = !cb.skip && !(level == 0 && cb.sel[SEL_MODE] != 1u) && !(level == 1 && flags != 0u);
+            active = !cb.skip && cb.seg_tiles < LONG_SEG_TILES &&   // (long segments: topk_cand_hist_long_kernel)
+                     !(level == 0 && cb.sel[SEL_MODE] != 1u) && !(level == 1 && flags != 0u);
             prefix = cb.sel[SEL_PREFIX];
         }
         uint32_t lo = 0xffffffffu, hi = 0u;
@@ -427,16 +416,11 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
                 }
                 const uint32_t same = __match_any_sync(0xffffffffu, digit);
                 if (digit != 0xffffffffu) {
-                    if (lane == __ffs(same) - 1) {
-                        if (gather) atomicAdd(&h[digit], (uint32_t)__popc(same));
-                        else atomicAdd(gh + digit, (uint32_t)__popc(same));
-                    }
+                    if (lane == __ffs(same) - 1) atomicAdd(gh + digit, (uint32_t)__popc(same));
                     lo = min(lo, digit);
                     hi = max(hi, digit);
                 }
             }
-        }
-        if (!gather && active) {  // (uniform over the warp)
             lo = __reduce_min_sync(0xffffffffu, lo);
             hi = __reduce_max_sync(0xffffffffu, hi);
             if (lane == 0 && lo != 0xffffffffu) {
@@ -445,12 +429,58 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
             }
         }
     }
-    if (gather) {
-        __syncthreads();
-        // (all tiles of the CTA share the segment, hence the selection state and the histogram)
-        flush_hist(h, (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + seg0) * DIGIT1_BINS,
-                   s.sel + ((int64_t)row * p.T + seg0) * SEL_WORDS, lo_word, hi_word);
+}
+
+// The same histograms for the long segments (LONG_SEG_TILES tiles or more: flat vectors, an embedding
+// matrix).  A problem's candidates are one contiguous region of the buffer, whatever tile they came
+// from, and a histogram does not care about their order: a CTA takes 8192 consecutive candidates
+// with coalesced loads, eight in flight per thread, counts in shared memory and adds its non-empty
+// bins to the problem's histogram once.  Grid (n_long * chunks, rows); chunks past the problem's
+// candidate count leave at once.
+constexpr int CAND_CHUNK = THREADS * 32;
+__global__ void __launch_bounds__(THREADS) topk_cand_hist_long_kernel(const __grid_constant__ Params p, const TopkSide s,
+                                                                       const int level, const int chunks) {
+    __shared__ uint32_t h[DIGIT1_BINS];
+    const int t = __ldg(p.large_seg + blockIdx.x / chunks), row = blockIdx.y;
+    const uint32_t c0 = (uint32_t)(blockIdx.x % chunks) * CAND_CHUNK;
+    uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
+    const uint32_t flags = sel[SEL_FLAGS];
+    if ((flags & 1u) || (level == 0 && sel[SEL_MODE] != 1u) || (level == 1 && flags != 0u)) return;   // (uniform over the CTA)
+    const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
+    const uint32_t ncand = min(sel[SEL_CAND_COUNT], cap);
+    if (c0 >= ncand) return;
+    const uint32_t prefix = sel[SEL_PREFIX];
+    for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(h)[b] = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+    const float *cand = s.cand_val + (int64_t)row * p.CAP + __ldg(p.cap_off + t);
+    const int lane = threadIdx.x & 31;
+#pragma unroll 1
+    for (int batch = 0; batch < 4; ++batch) {
+        uint32_t key[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const uint32_t q = c0 + (uint32_t)((batch * 8 + u) * THREADS) + threadIdx.x;
+            key[u] = q < ncand ? key_of(cand[q]) : 0xffffffffu;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            uint32_t digit = 0xffffffffu;   // nothing to add
+            if (key[u] != 0xffffffffu) {
+                if (level == 0) digit = key[u] >> DIGIT1_SHIFT;
+                else if (level == 1) { if ((key[u] >> DIGIT1_SHIFT) == prefix) digit = (key[u] >> 7) & 0xfffu; }
+                else if ((key[u] >> 7) == prefix) digit = key[u] & 0x7fu;
+            }
+            if (level == 0) {   // the candidates crowd into a few first-digit bins: one atomic per distinct bin of the warp
+                const uint32_t same = __match_any_sync(0xffffffffu, digit);
+                if (digit != 0xffffffffu && lane == __ffs(same) - 1) atomicAdd(&h[digit], (uint32_t)__popc(same));
+            } else if (digit != 0xffffffffu) {
+                atomicAdd(&h[digit], 1u);
+            }
+        }
     }
+    __syncthreads();
+    flush_hist(h, (level == 0 ? s.hist : s.hist2) + ((int64_t)row * p.T + t) * DIGIT1_BINS, sel,
+               level == 0 ? SEL_LO1 : SEL_LO2, level == 0 ? SEL_HI1 : SEL_HI2);
 }
 
 __global__ void __launch_bounds__(THREADS) topk_count_kernel(const __grid_constant__ Params p, const TopkSide s) {
@@ -866,14 +896,21 @@ static dim3 strided_grid(const Params &p, int rows) {
     return dim3(p.TT < per_row ? p.TT : per_row, rows);
 }
 
-// Candidate histograms of the wide form: 64 tiles per CTA for very long segments (the CTAs gather in
-// shared memory and flush once per 64 tiles: fewer atomics on one histogram), 16 tiles per CTA
-// otherwise (more warps in flight on what is a chain of dependent loads per tile block; measured:
-// flat 2^24 uplink 0.261 -> 0.232 ms with 16, flat 2^26 0.582 -> 0.625 ms, hence the switch point).
-static int cand_hist_reps(const Params &p) { return p.max_seg_tiles >= 4096 ? 8 : 2; }
-static dim3 cand_hist_grid(const Params &p, int rows) {
-    const int per = 8 * cand_hist_reps(p);
-    return dim3((p.TT + per - 1) / per, rows);
+// Candidate histograms of the wide form.  Segments below LONG_SEG_TILES tiles: a warp per tile block,
+// 16 tiles per CTA (many warps in flight on what is a chain of dependent loads per block).  Longer
+// segments: their candidate regions as a whole, 8192 candidates per CTA.
+static cudaError_t launch_cand_hist(const Params &p, const TopkSide &s, int level, cudaStream_t st, int64_t *launches) {
+    if (p.n_long < p.n_large) {
+        constexpr int REPS = 2;
+        topk_cand_hist_kernel<<<dim3((p.TT + 8 * REPS - 1) / (8 * REPS), s.R), THREADS, 0, st>>>(p, s, level, REPS);
+        CHECK_LAUNCH();
+    }
+    if (p.n_long > 0) {
+        const int chunks = (int)((p.cap_long_max + CAND_CHUNK - 1) / CAND_CHUNK);
+        topk_cand_hist_long_kernel<<<dim3(p.n_long * chunks, s.R), THREADS, 0, st>>>(p, s, level, chunks);
+        CHECK_LAUNCH();
+    }
+    return cudaSuccess;
 }
 
 // First part of a side (multi-tile segments).  Uplink: candidates are
@@ -899,7 +936,7 @@ cudaError_t topk_first_part(const Params &p, const TopkSide &s, int src_kind, cu
         if (e != cudaSuccess) return e;
         ++*launches;
         if (!use_fused_tail(p)) {   // wide form: first digit of the single-pass problems from a global histogram
-            topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 0, cand_hist_reps(p)); CHECK_LAUNCH();
+            if ((e = launch_cand_hist(p, s, 0, st, launches)) != cudaSuccess) return e;
             topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 5); CHECK_LAUNCH();
         }
     }
@@ -925,9 +962,10 @@ cudaError_t topk_second_part(const Params &p, const TopkSide &s, int src_kind, c
     LAUNCH_BY_SOURCE(topk_filter_tma_kernel, g_filter, COMMA false);
     if (use_fused_tail(p)) return launch_topk_tail(p, s, src_kind, st, launches);
     // some segment has too many candidates or tiles for one CTA: the same steps, spread over the tile blocks
-    topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 1, cand_hist_reps(p)); CHECK_LAUNCH();
+    cudaError_t e;
+    if ((e = launch_cand_hist(p, s, 1, st, launches)) != cudaSuccess) return e;
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 2); CHECK_LAUNCH();
-    topk_cand_hist_kernel<<<cand_hist_grid(p, s.R), THREADS, 0, st>>>(p, s, 2, cand_hist_reps(p)); CHECK_LAUNCH();
+    if ((e = launch_cand_hist(p, s, 2, st, launches)) != cudaSuccess) return e;
     LAUNCH_BY_SOURCE(topk_dense_hist3_kernel, g_strided);
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 3); CHECK_LAUNCH();
     topk_count_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
