@@ -362,18 +362,22 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
 // ------------------------------------------------------------------------------------------------
 // candidate passes: one CTA per (tile, row) walks that tile's block of the candidate buffer
 // ------------------------------------------------------------------------------------------------
-struct CandBlock { int64_t base; uint32_t cnt; int t, seg_tiles; uint32_t *sel; uint32_t *meta; bool skip; };
+struct CandBlock { int64_t base; uint32_t cnt; int t, seg_tiles; uint32_t *sel; uint32_t *meta; uint4 m; bool skip; };
 
+// (the tile's metadata does not depend on its segment: it is fetched beside the segment lookup, not after it)
 __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide &s, int tile, int row) {
     CandBlock cb;
+    cb.meta = s.meta + ((int64_t)row * p.TT + tile) * 4;
+    cb.m = *reinterpret_cast<const uint4 *>(cb.meta);   // pos, cnt, and what the count / scan kernels left
     const TileInfo ti = locate_tile(p, tile);
     cb.t = ti.t;
     cb.seg_tiles = ti.seg_tiles;
     cb.sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
-    cb.meta = s.meta + ((int64_t)row * p.TT + tile) * 4;
-    cb.skip = (cb.sel[SEL_FLAGS] & 1u) != 0u || ti.seg_tiles == 1;
-    cb.cnt = cb.skip ? 0u : cb.meta[1];
-    cb.base = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + cb.meta[0];
+    const uint32_t flags = cb.sel[SEL_FLAGS];
+    const int64_t cap0 = __ldg(p.cap_off + ti.t);
+    cb.skip = (flags & 1u) != 0u || ti.seg_tiles == 1;
+    cb.cnt = cb.skip ? 0u : cb.m.y;
+    cb.base = (int64_t)row * p.CAP + cap0 + cb.m.x;
     return cb;
 }
 
@@ -433,49 +437,85 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_kernel(const __grid_co
 
 // The same histograms for the long segments (LONG_SEG_TILES tiles or more: flat vectors, an embedding
 // matrix).  A problem's candidates are one contiguous region of the buffer, whatever tile they came
-// from, and a histogram does not care about their order: a CTA takes 8192 consecutive candidates
-// with coalesced loads, eight in flight per thread, counts in shared memory and adds its non-empty
-// bins to the problem's histogram once.  Grid (n_long * chunks, rows); chunks past the problem's
-// candidate count leave at once.
-constexpr int CAND_CHUNK = THREADS * 32;
+// from, and a histogram does not care about their order: a CTA takes `batches` runs of 8192
+// consecutive candidates; a thread fetches 32 of a run with eight 128-bit loads before it uses any,
+// counts in shared memory, and the CTA adds its non-empty bins to the problem's histogram once (with
+// many small CTAs those additions, thousands of CTAs on the same 4096 words, are what the launch
+// waits for: hence several runs per CTA where there are tens of millions of candidates).
+// Grid (n_long * chunks, rows); chunks past the problem's candidate count leave at once.
+constexpr int CAND_RUN = THREADS * 32;
 __global__ void __launch_bounds__(THREADS) topk_cand_hist_long_kernel(const __grid_constant__ Params p, const TopkSide s,
-                                                                       const int level, const int chunks) {
+                                                                       const int level, const int chunks, const int batches) {
     __shared__ uint32_t h[DIGIT1_BINS];
     const int t = __ldg(p.large_seg + blockIdx.x / chunks), row = blockIdx.y;
-    const uint32_t c0 = (uint32_t)(blockIdx.x % chunks) * CAND_CHUNK;
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
     const uint32_t flags = sel[SEL_FLAGS];
     if ((flags & 1u) || (level == 0 && sel[SEL_MODE] != 1u) || (level == 1 && flags != 0u)) return;   // (uniform over the CTA)
     const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
     const uint32_t ncand = min(sel[SEL_CAND_COUNT], cap);
-    if (c0 >= ncand) return;
+    // positions are counted from the 16-byte boundary at or before the region's first candidate
+    const int64_t base = (int64_t)row * p.CAP + __ldg(p.cap_off + t);
+    const uint32_t lead = (uint32_t)(base & 3);
+    const float *al = s.cand_val + (base - lead);
+    const uint32_t end = lead + ncand;
+    const uint32_t c0 = (uint32_t)(blockIdx.x % chunks) * (uint32_t)(batches * CAND_RUN);
+    if (c0 >= end) return;
     const uint32_t prefix = sel[SEL_PREFIX];
     for (int b = threadIdx.x; b < DIGIT1_BINS / 4; b += THREADS) reinterpret_cast<uint4 *>(h)[b] = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
-    const float *cand = s.cand_val + (int64_t)row * p.CAP + __ldg(p.cap_off + t);
-    const int lane = threadIdx.x & 31;
+    // First digit: the candidates are the entries at or above the guess and crowd into the few bins
+    // from the guess's upwards, where atomics on one address would serialise; those bins are counted in
+    // registers (near[r]: first digit = guess's bin + r) and only the rare entries further up go to
+    // shared memory one by one.
+    constexpr int NEAR = 8;
+    const uint32_t gbin = sel[SEL_GUESS] >> DIGIT1_SHIFT;
+    uint32_t near[NEAR];
+#pragma unroll
+    for (int r = 0; r < NEAR; ++r) near[r] = 0u;
 #pragma unroll 1
-    for (int batch = 0; batch < 4; ++batch) {
-        uint32_t key[8];
+    for (int batch = 0; batch < batches; ++batch) {
+        const uint32_t r0 = c0 + (uint32_t)(batch * CAND_RUN);
+        if (r0 >= end) break;   // (uniform over the CTA)
+        uint32_t key[8][4];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            const uint32_t q = c0 + (uint32_t)((batch * 8 + u) * THREADS) + threadIdx.x;
-            key[u] = q < ncand ? key_of(cand[q]) : 0xffffffffu;
+            const uint32_t i = r0 + (uint32_t)(u * THREADS + threadIdx.x) * 4u;
+            if (i >= lead && i + 3u < end) {
+                const uint4 q = *reinterpret_cast<const uint4 *>(al + i);
+                key[u][0] = q.x & 0x7fffffffu; key[u][1] = q.y & 0x7fffffffu;
+                key[u][2] = q.z & 0x7fffffffu; key[u][3] = q.w & 0x7fffffffu;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) key[u][j] = (i + j >= lead && i + j < end) ? key_of(al[i + j]) : 0xffffffffu;
+            }
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-            uint32_t digit = 0xffffffffu;   // nothing to add
-            if (key[u] != 0xffffffffu) {
-                if (level == 0) digit = key[u] >> DIGIT1_SHIFT;
-                else if (level == 1) { if ((key[u] >> DIGIT1_SHIFT) == prefix) digit = (key[u] >> 7) & 0xfffu; }
-                else if ((key[u] >> 7) == prefix) digit = key[u] & 0x7fu;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t key1 = key[u][j];
+                if (key1 == 0xffffffffu) continue;
+                if (level == 0) {
+                    const uint32_t rel = (key1 >> DIGIT1_SHIFT) - gbin;
+                    if (rel < (uint32_t)NEAR) {
+#pragma unroll
+                        for (int r = 0; r < NEAR; ++r) near[r] += rel == (uint32_t)r ? 1u : 0u;
+                    } else {
+                        atomicAdd(&h[key1 >> DIGIT1_SHIFT], 1u);
+                    }
+                } else if (level == 1) {
+                    if ((key1 >> DIGIT1_SHIFT) == prefix) atomicAdd(&h[(key1 >> 7) & 0xfffu], 1u);
+                } else if ((key1 >> 7) == prefix) {
+                    atomicAdd(&h[key1 & 0x7fu], 1u);
+                }
             }
-            if (level == 0) {   // the candidates crowd into a few first-digit bins: one atomic per distinct bin of the warp
-                const uint32_t same = __match_any_sync(0xffffffffu, digit);
-                if (digit != 0xffffffffu && lane == __ffs(same) - 1) atomicAdd(&h[digit], (uint32_t)__popc(same));
-            } else if (digit != 0xffffffffu) {
-                atomicAdd(&h[digit], 1u);
-            }
+        }
+    }
+    if (level == 0) {
+#pragma unroll
+        for (int r = 0; r < NEAR; ++r) {
+            const uint32_t c = __reduce_add_sync(0xffffffffu, near[r]);
+            if ((threadIdx.x & 31) == 0 && c && gbin + r < (uint32_t)DIGIT1_BINS) atomicAdd(&h[gbin + r], c);
         }
     }
     __syncthreads();
@@ -488,13 +528,19 @@ __global__ void __launch_bounds__(THREADS) topk_count_kernel(const __grid_consta
     const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (tile >= p.TT) return;
     const CandBlock cb = cand_block(p, s, tile, row);
-    if (cb.skip) return;
     const uint32_t T = cb.sel[SEL_THRESH];
+    if (cb.skip) return;
     uint32_t g = 0, e = 0;
-    for (uint32_t q = lane; q < cb.cnt; q += 32) {
-        const uint32_t key = key_of(s.cand_val[cb.base + q]);
-        g += key > T ? 1u : 0u;
-        e += key == T ? 1u : 0u;
+    for (uint32_t q0 = lane; q0 < cb.cnt; q0 += 128) {   // four stripes of 32 candidates in flight
+        uint32_t key[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) key[u] = q0 + 32 * u < cb.cnt ? key_of(s.cand_val[cb.base + q0 + 32 * u]) : 0u;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const bool in = q0 + 32 * u < cb.cnt;
+            g += in && key[u] > T ? 1u : 0u;
+            e += in && key[u] == T ? 1u : 0u;
+        }
     }
     g = __reduce_add_sync(0xffffffffu, g);
     e = __reduce_add_sync(0xffffffffu, e);
@@ -504,7 +550,7 @@ __global__ void __launch_bounds__(THREADS) topk_count_kernel(const __grid_consta
 // scan: one CTA per (segment, row); tiles of the segment in order
 __global__ void __launch_bounds__(THREADS) topk_scan_kernel(const __grid_constant__ Params p, const TopkSide s) {
     __shared__ uint32_t warp_tot[8];
-    constexpr int PER = 4;  // consecutive tiles per thread and round
+    constexpr int PER = 16;  // consecutive tiles per thread and round (their metadata loads are in flight together)
     const int t = blockIdx.x, row = blockIdx.y;
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
     const int first = __ldg(p.tile_prefix + t), ntiles = __ldg(p.tile_prefix + t + 1) - first;
@@ -518,9 +564,9 @@ __global__ void __launch_bounds__(THREADS) topk_scan_kernel(const __grid_constan
 #pragma unroll
         for (int u = 0; u < PER; ++u) {
             const bool in = q0 + u < ntiles;
-            const uint32_t *m = s.meta + ((int64_t)row * p.TT + first + (in ? q0 + u : 0)) * 4;
-            g[u] = in ? m[2] : 0u;
-            e[u] = in ? m[3] : 0u;
+            const uint4 m = *reinterpret_cast<const uint4 *>(s.meta + ((int64_t)row * p.TT + first + (in ? q0 + u : 0)) * 4);
+            g[u] = in ? m.z : 0u;
+            e[u] = in ? m.w : 0u;
             esum += e[u];
         }
         uint32_t ties_total, sel_total;
@@ -556,20 +602,33 @@ __global__ void __launch_bounds__(THREADS) topk_write_kernel(const __grid_consta
     const int row = blockIdx.y, lane = threadIdx.x & 31;
     const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (tile >= p.TT) return;
+    const uint32_t out0 = s.outbase[(int64_t)row * (p.TT + 1) + tile];   // (fetched beside the segment lookup)
     const CandBlock cb = cand_block(p, s, tile, row);
-    if (cb.skip || cb.cnt == 0) return;
     const uint32_t T = cb.sel[SEL_THRESH];
-    const uint32_t allowed = cb.meta[3];
-    const bool has_last = cb.meta[2] != 0u;
-    const int64_t obase = (int64_t)row * p.K + s.outbase[(int64_t)row * (p.TT + 1) + tile];
     const int64_t oend = (int64_t)row * p.K + __ldg(p.k_off + cb.t + 1);  // never write past the segment's slots
+    if (cb.skip || cb.cnt == 0) return;
+    const uint32_t allowed = cb.m.w;
+    const bool has_last = cb.m.z != 0u;
+    const int64_t obase = (int64_t)row * p.K + out0;
     const uint32_t lt_mask = (1u << lane) - 1u;
     uint32_t run_sel = 0, run_tie = 0;
-    for (uint32_t c0 = 0; c0 < cb.cnt; c0 += 32) {
+    for (uint32_t c00 = 0; c00 < cb.cnt; c00 += 128) {   // four stripes of 32 candidates fetched before any is used
+      float val4[4];
+      uint32_t idx4[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+          const uint32_t q = c00 + 32 * u + lane;
+          val4[u] = q < cb.cnt ? s.cand_val[cb.base + q] : 0.0f;
+          idx4[u] = q < cb.cnt ? s.cand_idx[cb.base + q] : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t c0 = c00 + 32 * u;
+        if (c0 >= cb.cnt) break;   // (uniform over the warp)
         const uint32_t q = c0 + lane;
         const bool in = q < cb.cnt;
-        const float val = in ? s.cand_val[cb.base + q] : 0.0f;
-        const uint32_t idx = in ? s.cand_idx[cb.base + q] : 0u;
+        const float val = val4[u];
+        const uint32_t idx = idx4[u];
         const uint32_t key = key_of(val);
         const bool tie = in && key == T;
         const uint32_t tb = __ballot_sync(0xffffffffu, tie);
@@ -587,6 +646,7 @@ __global__ void __launch_bounds__(THREADS) topk_write_kernel(const __grid_consta
         }
         run_sel += __popc(sb);
         run_tie += __popc(tb);
+      }
     }
 }
 
@@ -898,7 +958,7 @@ static dim3 strided_grid(const Params &p, int rows) {
 
 // Candidate histograms of the wide form.  Segments below LONG_SEG_TILES tiles: a warp per tile block,
 // 16 tiles per CTA (many warps in flight on what is a chain of dependent loads per block).  Longer
-// segments: their candidate regions as a whole, 8192 candidates per CTA.
+// segments: their candidate regions as a whole, 8192 or 32768 candidates per CTA.
 static cudaError_t launch_cand_hist(const Params &p, const TopkSide &s, int level, cudaStream_t st, int64_t *launches) {
     if (p.n_long < p.n_large) {
         constexpr int REPS = 2;
@@ -906,8 +966,11 @@ static cudaError_t launch_cand_hist(const Params &p, const TopkSide &s, int leve
         CHECK_LAUNCH();
     }
     if (p.n_long > 0) {
-        const int chunks = (int)((p.cap_long_max + CAND_CHUNK - 1) / CAND_CHUNK);
-        topk_cand_hist_long_kernel<<<dim3(p.n_long * chunks, s.R), THREADS, 0, st>>>(p, s, level, chunks);
+        // (four runs per CTA from 2^24 candidate slots up; three more positions cover a region that starts off a 16-byte boundary)
+        const int batches = p.cap_long_max * p.n_long * s.R >= (int64_t)1 << 24 ? 4 : 1;
+        const int64_t per_cta = (int64_t)batches * CAND_RUN;
+        const int chunks = (int)((p.cap_long_max + 3 + per_cta - 1) / per_cta);
+        topk_cand_hist_long_kernel<<<dim3(p.n_long * chunks, s.R), THREADS, 0, st>>>(p, s, level, chunks, batches);
         CHECK_LAUNCH();
     }
     return cudaSuccess;
