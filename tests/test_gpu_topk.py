@@ -164,6 +164,19 @@ def test_segment_of_more_than_1024_tiles_gathers_candidate_histograms():
         P.step(G, 0.1)
 
 
+def test_long_segment_whose_candidate_region_starts_off_a_16_byte_boundary():
+    """A 9 M-element tensor behind a small one whose candidate capacity (2 k + 2048 with k = 201) is not
+    a multiple of four: the long segment's candidate histograms read its region with 128-bit loads
+    from the boundary before it, and must count neither the neighbour's slots nor anything twice."""
+    lay = Layout("offset", (20_000, 9_000_000))
+    k = np.asarray([201, 90_001], np.int64)
+    P = _pair(2, lay.seg_offsets, TOPK, TOPK, k=k)
+    for step in range(3):
+        G = make_gradients("normal", 1.0, 2, lay.dim, step, base_seed=27)
+        P.step(G, 0.1)
+    assert P.ctx.liec_topk_route_counts(True)["single_pass"] >= 2     # (the guess route, with its first-digit candidate histogram, ran)
+
+
 def test_bf16_topk():
     lay = ragged_layout()
     k = topk_counts(lay, 1, 50)
