@@ -37,12 +37,14 @@
  *   identity: no message buffer; the dense vector itself.
  *
  * Ownership: the caller owns every device buffer (params, error, gradients, workspace).
- * The library owns only the host-side context (for top-k / random-k configurations that have
- * segments of at most 8192 elements, or segments with 16384 or more selection candidates, also one
- * helper stream and four events, created by liec_init and released by liec_destroy).  The hot calls allocate nothing, never synchronise the device and only
- * enqueue work that is ordered on the given stream: a top-k stage may run part of its kernels
- * on the helper stream, forked from and joined back to the given stream by events inside the
- * same call (this also works while the given stream is being captured into a CUDA graph).
+ * The library owns only the host-side context (for configurations with a scaled-sign downlink, and
+ * for top-k / random-k configurations that have segments of at most 8192 elements or segments with
+ * 16384 or more selection candidates, also one helper stream and four events, created by liec_init
+ * and released by liec_destroy).  The hot calls allocate nothing, never synchronise the device and
+ * only enqueue work that is ordered on the given stream: a top-k stage may run part of its kernels
+ * on the helper stream, and liec_step runs the error update of a scaled-sign downlink there beside
+ * the worker update; the helper stream is forked from and joined back to the given stream by events
+ * inside the same call (this also works while the given stream is being captured into a CUDA graph).
  *
  * Errors: every call returns a liec_status; nothing throws, aborts or traps the GPU.
  * liec_last_error() gives a message for the last failing call on that context.

@@ -458,7 +458,7 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     }
     cudaError_t e = configure_topk_kernels();
     if (e == cudaSuccess) e = configure_average_kernels();
-    if (e == cudaSuccess && c->plan.K > 0 && (!c->plan.small_seg.empty() || p.n_big > 0)) {
+    if (e == cudaSuccess && ((c->plan.K > 0 && (!c->plan.small_seg.empty() || p.n_big > 0)) || p.down == COMP_SIGN)) {
         int prio_low = 0, prio_high = 0;   // the helper stream carries the longest-running CTAs of a stage: they go first
         e = cudaDeviceGetStreamPriorityRange(&prio_low, &prio_high);
         if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&c->side, cudaStreamNonBlocking, prio_high);
@@ -599,11 +599,34 @@ liec_status liec_draw_subsets(liec_ctx *c, uint64_t seed, uint32_t epoch, void *
     return LIEC_OK;
 }
 
+// Scaled-sign downlink inside liec_step: the message is complete once the scales are final; the
+// error update e <- v -/+ s (which only the next iteration reads) and the worker update (which
+// reads the message, not e) do not depend on one another, so the first runs on the helper stream
+// beside the second.  Same kernels, same bytes as the two stage calls in sequence.
+static liec_status sign_downlink_beside_update(liec_ctx *c, const void *grads, float lr, cudaStream_t s) {
+    liec_status st = check_stage(c, 2, "liec_step");
+    if (st != LIEC_OK) return st;
+    LIEC_LAUNCH(c, launch_scale_finalize(c->p, false, s));
+    LIEC_CALL(c, cudaEventRecord(c->ev_fork, s));
+    LIEC_CALL(c, cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+    LIEC_LAUNCH(c, launch_sign_error(c->p, c->side));
+    LIEC_CALL(c, cudaEventRecord(c->ev_join, c->side));
+    c->stage = 3;
+    st = liec_worker_update(c, grads, lr, s);
+    LIEC_CALL(c, cudaStreamWaitEvent(s, c->ev_join, 0));   // (also after a refused update: nothing stays forked)
+    return st;
+}
+
 liec_status liec_step(liec_ctx *c, const void *grads, float lr, void *stream) {
     liec_status st = liec_uplink_compress(c, grads, stream);
     if (st != LIEC_OK) return st;  // nothing was enqueued: the context is where it was
-    if ((st = liec_server_aggregate(c, stream)) == LIEC_OK && (st = liec_downlink_compress(c, stream)) == LIEC_OK)
-        st = liec_worker_update(c, grads, lr, stream);
+    if ((st = liec_server_aggregate(c, stream)) == LIEC_OK) {
+        if (c->p.down == COMP_SIGN && c->side) {
+            st = sign_downlink_beside_update(c, grads, lr, static_cast<cudaStream_t>(stream));
+        } else if ((st = liec_downlink_compress(c, stream)) == LIEC_OK) {
+            st = liec_worker_update(c, grads, lr, stream);
+        }
+    }
     if (st != LIEC_OK) c->stage = 0;  // a half-done iteration: back to idle, state unspecified (see liec_abort_step)
     return st;
 }
