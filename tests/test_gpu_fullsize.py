@@ -221,3 +221,128 @@ def test_c3_resnet50_seeded_randk_full_size():
                 assert np.array_equal(lists[row, koff[t]:koff[t + 1]].astype(np.int64), want), (epoch, row, t)
         # the messages carry the values found at the subsets
         assert torch.equal(m["up_val"], torch.gather(G, 1, m["up_idx"].long()))
+
+
+def _assert_is_the_topk_set(x, idx, k):
+    """idx (ascending int64, device) is THE top-k set of |x| with ties to the lower index: checked from
+    the definition with library primitives (k-th largest magnitude by torch.kthvalue)."""
+    n = x.numel()
+    mag = x.abs()
+    assert idx.numel() == k and bool((idx[1:] > idx[:-1]).all()) and int(idx[0]) >= 0 and int(idx[-1]) < n
+    thr = torch.kthvalue(mag, n - k + 1).values            # the k-th largest magnitude
+    kept = torch.zeros(n, dtype=torch.bool, device=x.device)
+    kept[idx] = True
+    assert bool((mag[kept] >= thr).all()) and bool((mag[~kept] <= thr).all())
+    ties = mag == thr
+    kept_ties, dropped_ties = torch.nonzero(ties & kept).flatten(), torch.nonzero(ties & ~kept).flatten()
+    assert int((mag > thr).sum()) + kept_ties.numel() == k
+    if dropped_ties.numel():
+        assert int(kept_ties.max()) < int(dropped_ties.min()) if kept_ties.numel() else True
+
+
+def test_c5_flat_2p28_topk_one_percent_full_size():
+    """The 2^28 point of the bandwidth sweep (N = 8, one flat vector, k = 1 %), as bench.py runs it: far
+    beyond what the oracle finishes, so every stage is checked on the device against its definition
+    written with torch's elementwise operations, kthvalue and scatter (IEEE binary32, no contraction):
+    the top-k sets of two workers and of the server, v = e + (sum in worker order) / N, e' = v off the
+    kept set, and x <- x - lr ((p - p^i) + g) for two workers, all bit for bit; two iterations, so that
+    the second one runs on a non-zero e and on the single-pass route."""
+    n, N, lr = 1 << 28, 8, 0.1
+    k = n // 100
+    off = np.asarray([0, n], np.int64)
+    X = torch.zeros(N, n, device="cuda")
+    e = torch.zeros(n, device="cuda")
+    ctx = liec.Context(X, e, off, liec.COMP_TOPK, liec.COMP_TOPK, np.asarray([k], np.int64))
+    G = torch.empty(N, n, device="cuda")
+    for step in range(2):
+        make_gradients("normal", 1.0, N, n, step, base_seed=81, device="cuda", out=G)
+        e_before = e.clone()
+        x_before = {i: X[i].clone() for i in (0, N - 1)}
+        ctx.liec_uplink_compress(G)
+        ctx.liec_server_aggregate()
+        torch.cuda.synchronize()
+        v = e.clone()
+        m = ctx.liec_get_messages()
+        up_idx = m["up_idx"].to(torch.int64) & 0xFFFFFFFF
+        for i in (0, N - 1):
+            _assert_is_the_topk_set(G[i], up_idx[i], k)
+            assert torch.equal(m["up_val"][i], G[i][up_idx[i]])
+        acc = torch.zeros(n, device="cuda")
+        for i in range(N):                       # worker order; adding an absent entry's +0 changes nothing
+            p_i = torch.zeros(n, device="cuda")
+            p_i[up_idx[i]] = m["up_val"][i]
+            acc = acc + p_i
+        want_v = e_before + acc / N
+        assert torch.equal(v.view(torch.int32), want_v.view(torch.int32)), f"v, step {step}"
+        del acc, want_v, p_i
+        ctx.liec_downlink_compress()
+        ctx.liec_worker_update(G, lr)
+        torch.cuda.synchronize()
+        assert ctx.liec_device_status() == 0
+        m = ctx.liec_get_messages()
+        down_idx = m["down_idx"].to(torch.int64) & 0xFFFFFFFF
+        _assert_is_the_topk_set(v, down_idx, k)
+        assert torch.equal(m["down_val"], v[down_idx])
+        p = torch.zeros(n, device="cuda")
+        p[down_idx] = m["down_val"]
+        want_e = v.clone()
+        want_e[down_idx] = 0.0
+        assert torch.equal(e.view(torch.int32), want_e.view(torch.int32)), f"e', step {step}"
+        del want_e
+        for i in (0, N - 1):
+            p_i = torch.zeros(n, device="cuda")
+            p_i[up_idx[i]] = m["up_val"][i]
+            u = (p - p_i) + G[i]
+            want_x = x_before[i] - u * lr
+            assert torch.equal(X[i].view(torch.int32), want_x.view(torch.int32)), f"x^{i}, step {step}"
+            del p_i, u, want_x
+        routes = ctx.liec_topk_route_counts(True)
+        assert routes["problems"] == N and routes["slow"] == 0
+        if step == 1:
+            assert routes["single_pass"] == N, routes     # the bound under the first step's thresholds held
+
+
+def test_c5_flat_2p28_sign_full_size():
+    """The 2^28 sign point of the sweep: the scales of one worker and of the server against the oracle's
+    scale of the same bytes, every sign word against the definition, v and x against the update rules
+    written with torch's elementwise operations (bit for bit)."""
+    n, N, lr = 1 << 28, 8, 0.1
+    off = np.asarray([0, n], np.int64)
+    X = torch.zeros(N, n, device="cuda")
+    e = torch.zeros(n, device="cuda")
+    ctx = liec.Context(X, e, off, liec.COMP_SCALED_SIGN, liec.COMP_SCALED_SIGN)
+    G = torch.empty(N, n, device="cuda")
+    for step in range(2):
+        make_gradients("normal", 1.0, N, n, step, base_seed=82, device="cuda", out=G)
+        e_before = e.clone()
+        x_before = X[N - 1].clone()
+        ctx.liec_uplink_compress(G)
+        ctx.liec_server_aggregate()
+        torch.cuda.synchronize()
+        v = e.clone()
+        ctx.liec_downlink_compress()
+        ctx.liec_worker_update(G, lr)
+        torch.cuda.synchronize()
+        assert ctx.liec_device_status() == 0
+        m = ctx.liec_get_messages()
+        s_up = m["up_scales"][:, 0]
+        want = oracle.scale(f32(G[N - 1]))
+        assert np.float32(f32(s_up[N - 1:N])[0]).view(np.uint32) == np.float32(want).view(np.uint32)
+        for i in range(N):
+            assert torch.equal(m["up_words"][i].to(torch.int64) & 0xFFFFFFFF, _pack_negative(G[i])), ("up words", i)
+        acc = torch.zeros(n, device="cuda")
+        for i in range(N):                       # worker order
+            acc = acc + torch.where(G[i] < 0, -s_up[i], s_up[i])
+        want_v = e_before + acc / N
+        assert torch.equal(v.view(torch.int32), want_v.view(torch.int32)), f"v, step {step}"
+        del acc, want_v
+        s_down = m["down_scales"][0]
+        want = oracle.scale(f32(v))
+        assert np.float32(f32(m["down_scales"][0:1])[0]).view(np.uint32) == np.float32(want).view(np.uint32)
+        assert torch.equal(m["down_words"].to(torch.int64) & 0xFFFFFFFF, _pack_negative(v)), "down words"
+        p = torch.where(v < 0, -s_down, s_down)
+        assert torch.equal(e.view(torch.int32), (v - p).view(torch.int32)), f"e', step {step}"
+        p_i = torch.where(G[N - 1] < 0, -s_up[N - 1], s_up[N - 1])
+        want_x = x_before - ((p - p_i) + G[N - 1]) * lr
+        assert torch.equal(X[N - 1].view(torch.int32), want_x.view(torch.int32)), f"x, step {step}"
+        del p, p_i, want_x
