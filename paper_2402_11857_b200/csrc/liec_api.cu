@@ -35,7 +35,7 @@ struct Plan {
     Region r_up_idx, r_up_val, r_down_idx, r_down_val;
     Region r_up_hist, r_down_hist, r_up_hist2, r_down_hist2, r_up_sel, r_down_sel;
     Region r_up_cand_idx, r_up_cand_val, r_down_cand_idx, r_down_cand_val;
-    Region r_up_tile_meta, r_down_tile_meta, r_up_outbase, r_down_outbase;
+    Region r_up_tile_meta, r_down_tile_meta, r_up_outbase, r_down_outbase, r_up_scan_parts, r_down_scan_parts, r_gen_scan_parts;
     Region r_gen_sets, r_gen_val, r_gen_hist, r_gen_hist2, r_gen_sel, r_gen_cand_idx, r_gen_cand_val, r_gen_meta, r_gen_outbase;
     size_t total = 0;
 };
@@ -172,8 +172,12 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
         pl.r_down_partials = c.take(sizeof(double) * pl.TT);
     }
     if (cfg->downlink == LIEC_COMP_IDENTITY) pl.r_vbuf = c.take(sizeof(float) * pl.d);
+    int max_seg_tiles = 0;
+    for (int t = 0; t < T; ++t) max_seg_tiles = std::max(max_seg_tiles, pl.tile_prefix[t + 1] - pl.tile_prefix[t]);
+    const size_t scan_parts = (size_t)(max_seg_tiles + SCAN_PART - 1) / SCAN_PART;
     auto topk_regions = [&](size_t rows, Region &idx, Region &val, Region &hist, Region &hist2, Region &sel,
-                            Region &cidx, Region &cval, Region &meta, Region &outbase) {
+                            Region &cidx, Region &cval, Region &meta, Region &outbase, Region &parts) {
+        parts = c.take(sizeof(uint32_t) * rows * T * scan_parts * 2);
         idx = c.take(sizeof(uint32_t) * rows * pl.K * 2);  // idx then val, adjacent
         idx.bytes = sizeof(uint32_t) * rows * pl.K;
         val.off = idx.off + idx.bytes;
@@ -198,13 +202,13 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     if (cfg->downlink == LIEC_COMP_RANDK) randk_regions(1, pl.r_down_idx, pl.r_down_val, pl.r_down_outbase);
     if (cfg->uplink == LIEC_COMP_RANDK || cfg->downlink == LIEC_COMP_RANDK)   // scratch of the seeded draw (liec_draw_subsets)
         topk_regions(N + 1, pl.r_gen_sets, pl.r_gen_val, pl.r_gen_hist, pl.r_gen_hist2, pl.r_gen_sel, pl.r_gen_cand_idx,
-                     pl.r_gen_cand_val, pl.r_gen_meta, pl.r_gen_outbase);
+                     pl.r_gen_cand_val, pl.r_gen_meta, pl.r_gen_outbase, pl.r_gen_scan_parts);
     if (cfg->uplink == LIEC_COMP_TOPK)
         topk_regions(N, pl.r_up_idx, pl.r_up_val, pl.r_up_hist, pl.r_up_hist2, pl.r_up_sel, pl.r_up_cand_idx,
-                     pl.r_up_cand_val, pl.r_up_tile_meta, pl.r_up_outbase);
+                     pl.r_up_cand_val, pl.r_up_tile_meta, pl.r_up_outbase, pl.r_up_scan_parts);
     if (cfg->downlink == LIEC_COMP_TOPK)
         topk_regions(1, pl.r_down_idx, pl.r_down_val, pl.r_down_hist, pl.r_down_hist2, pl.r_down_sel,
-                     pl.r_down_cand_idx, pl.r_down_cand_val, pl.r_down_tile_meta, pl.r_down_outbase);
+                     pl.r_down_cand_idx, pl.r_down_cand_val, pl.r_down_tile_meta, pl.r_down_outbase, pl.r_down_scan_parts);
     pl.total = align_up(c.cursor, 256);
     return LIEC_OK;
 }
@@ -392,6 +396,7 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     }
     p.max_seg_tiles = 0;
     for (int t = 0; t < pl.T; ++t) p.max_seg_tiles = std::max(p.max_seg_tiles, pl.tile_prefix[t + 1] - pl.tile_prefix[t]);
+    p.scan_parts = (p.max_seg_tiles + SCAN_PART - 1) / SCAN_PART;
     p.status = at<int32_t>(c, pl.r_status);
     p.X = params;
     p.e = error;
@@ -425,6 +430,8 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     p.gen_sel = at<uint32_t>(c, pl.r_gen_sel);           p.gen_meta = at<uint32_t>(c, pl.r_gen_meta);
     p.gen_cand_idx = at<uint32_t>(c, pl.r_gen_cand_idx); p.gen_cand_val = at<float>(c, pl.r_gen_cand_val);
     p.gen_outbase = at<uint32_t>(c, pl.r_gen_outbase);
+    p.up_scan_parts = at<uint32_t>(c, pl.r_up_scan_parts); p.down_scan_parts = at<uint32_t>(c, pl.r_down_scan_parts);
+    p.gen_scan_parts = at<uint32_t>(c, pl.r_gen_scan_parts);
 
     struct Up { const Region *r; const void *src; };
     const Up ups[] = {
@@ -579,7 +586,7 @@ liec_status liec_draw_subsets(liec_ctx *c, uint64_t seed, uint32_t epoch, void *
     s.src = nullptr; s.row_stride = 0; s.R = p.N + 1;
     s.gen = ScoreStream{(uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), epoch};
     s.idx = p.gen_sets; s.val = p.gen_val; s.hist = p.gen_hist; s.hist2 = p.gen_hist2; s.sel = p.gen_sel;
-    s.cand_idx = p.gen_cand_idx; s.cand_val = p.gen_cand_val; s.meta = p.gen_meta; s.outbase = p.gen_outbase;
+    s.cand_idx = p.gen_cand_idx; s.cand_val = p.gen_cand_val; s.meta = p.gen_meta; s.outbase = p.gen_outbase; s.scan_parts = p.gen_scan_parts;
     s.zero_out = nullptr;
     s.spec = 1;
     cudaStream_t main_stream = static_cast<cudaStream_t>(stream);

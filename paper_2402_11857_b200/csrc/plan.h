@@ -85,6 +85,8 @@ struct Params {
     float *up_cand_val, *down_cand_val;      // [R][CAP]
     uint32_t *up_tile_meta, *down_tile_meta; // [R][TT][4] pos, cnt, n_greater, n_ties
     uint32_t *up_outbase, *down_outbase;     // [R][TT+1] first output slot of each tile
+    uint32_t *up_scan_parts, *down_scan_parts, *gen_scan_parts;   // [R][T][scan_parts][2]: sums of a segment's per-tile counts over runs of SCAN_PART tiles (wide form)
+    int32_t scan_parts;                      // runs of SCAN_PART tiles in the longest segment
     int64_t CAP;                              // candidate capacity per row
     int64_t cap_max;                          // largest candidate capacity of one segment
 
@@ -105,6 +107,7 @@ struct Params {
     uint32_t copy_wait_limit, copy_expect_extra;
 };
 constexpr uint32_t COPY_WAIT_LIMIT_DEFAULT = 1u << 20;
+constexpr int SCAN_PART = THREADS * 16;   // tiles whose output offsets one CTA of the wide form's scan computes
 constexpr int LONG_SEG_TILES = 1024;   // from here on a segment's candidate passes walk its candidate region as a whole, not tile block by tile block
 
 // per-problem selection state words

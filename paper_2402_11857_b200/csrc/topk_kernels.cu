@@ -548,53 +548,68 @@ __global__ void __launch_bounds__(THREADS) topk_count_kernel(const __grid_consta
 }
 
 // scan: one CTA per (segment, row); tiles of the segment in order
-__global__ void __launch_bounds__(THREADS) topk_scan_kernel(const __grid_constant__ Params p, const TopkSide s) {
+// A CTA takes one run of SCAN_PART consecutive tiles of one problem (PER tiles per thread, their
+// metadata loads in flight together).  Segments longer than one run are scanned in two launches:
+// phase 0 leaves each run's sums of the per-tile counts, phase 1 starts every run from the sums of
+// the runs before it (what the ties before a run were allowed follows from their number alone: ties
+// are accepted in index order until ties_wanted are).  Grid (T * scan_parts, rows).
+__global__ void __launch_bounds__(THREADS) topk_scan_kernel(const __grid_constant__ Params p, const TopkSide s, const int phase) {
     __shared__ uint32_t warp_tot[8];
-    constexpr int PER = 16;  // consecutive tiles per thread and round (their metadata loads are in flight together)
-    const int t = blockIdx.x, row = blockIdx.y;
+    constexpr int PER = SCAN_PART / THREADS;
+    const int t = blockIdx.x / p.scan_parts, part = blockIdx.x % p.scan_parts, row = blockIdx.y;
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
     const int first = __ldg(p.tile_prefix + t), ntiles = __ldg(p.tile_prefix + t + 1) - first;
     if (ntiles == 1) return;   // selected directly by one CTA
+    const int c0 = part * SCAN_PART;
+    if (c0 >= ntiles) return;
+    uint32_t *run_sums = s.scan_parts + (((int64_t)row * p.T + t) * p.scan_parts) * 2;
+    const int q0 = c0 + threadIdx.x * PER;
+    uint32_t g[PER], e[PER], gsum = 0, esum = 0;
+#pragma unroll
+    for (int u = 0; u < PER; ++u) {
+        const bool in = q0 + u < ntiles;
+        const uint4 m = *reinterpret_cast<const uint4 *>(s.meta + ((int64_t)row * p.TT + first + (in ? q0 + u : 0)) * 4);
+        g[u] = in ? m.z : 0u;
+        e[u] = in ? m.w : 0u;
+        gsum += g[u];
+        esum += e[u];
+    }
+    if (phase == 0) {
+        uint32_t g_total, e_total;
+        block_exclusive_scan(gsum, warp_tot, g_total);
+        block_exclusive_scan(esum, warp_tot, e_total);
+        if (threadIdx.x == 0) { run_sums[2 * part] = g_total; run_sums[2 * part + 1] = e_total; }
+        return;
+    }
     const uint32_t ties_wanted = sel[SEL_TIES];
     const uint32_t kbeg = (uint32_t)__ldg(p.k_off + t), k = (uint32_t)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
-    uint32_t carry_sel = 0, carry_ties = 0;  // uniform over the CTA
-    for (int c0 = 0; c0 < ntiles; c0 += THREADS * PER) {
-        const int q0 = c0 + threadIdx.x * PER;
-        uint32_t g[PER], e[PER], esum = 0;
+    uint32_t g_before = 0, carry_ties = 0;  // over the runs before this one (uniform over the CTA)
+    for (int j = 0; j < part; ++j) { g_before += run_sums[2 * j]; carry_ties += run_sums[2 * j + 1]; }
+    const uint32_t carry_sel = g_before + min(carry_ties, ties_wanted);
+    uint32_t ties_total, sel_total;
+    uint32_t ties_before = carry_ties + block_exclusive_scan(esum, warp_tot, ties_total);
+    uint32_t allowed[PER], mine = 0;
 #pragma unroll
-        for (int u = 0; u < PER; ++u) {
-            const bool in = q0 + u < ntiles;
-            const uint4 m = *reinterpret_cast<const uint4 *>(s.meta + ((int64_t)row * p.TT + first + (in ? q0 + u : 0)) * 4);
-            g[u] = in ? m.z : 0u;
-            e[u] = in ? m.w : 0u;
-            esum += e[u];
-        }
-        uint32_t ties_total, sel_total;
-        uint32_t ties_before = carry_ties + block_exclusive_scan(esum, warp_tot, ties_total);
-        uint32_t allowed[PER], mine = 0;
-#pragma unroll
-        for (int u = 0; u < PER; ++u) {
-            allowed[u] = ties_before < ties_wanted ? min(e[u], ties_wanted - ties_before) : 0u;
-            ties_before += e[u];
-            mine += g[u] + allowed[u];
-        }
-        uint32_t out = kbeg + carry_sel + block_exclusive_scan(mine, warp_tot, sel_total);
-        uint32_t tb = ties_before - esum;  // ties before this thread's first tile
-#pragma unroll
-        for (int u = 0; u < PER; ++u) {
-            if (q0 + u < ntiles) {
-                uint32_t *m = s.meta + ((int64_t)row * p.TT + first + q0 + u) * 4;
-                s.outbase[(int64_t)row * (p.TT + 1) + first + q0 + u] = out;
-                m[3] = allowed[u];
-                m[2] = (tb + allowed[u] == ties_wanted && allowed[u] > 0) ? 1u : 0u;  // holds the last accepted tie
-            }
-            out += g[u] + allowed[u];
-            tb += e[u];
-        }
-        carry_sel += sel_total;
-        carry_ties += ties_total;
+    for (int u = 0; u < PER; ++u) {
+        allowed[u] = ties_before < ties_wanted ? min(e[u], ties_wanted - ties_before) : 0u;
+        ties_before += e[u];
+        mine += g[u] + allowed[u];
     }
-    if (threadIdx.x == 0 && carry_sel != k) atomicOr(p.status, STATUS_COUNT_MISMATCH);
+    uint32_t out = kbeg + carry_sel + block_exclusive_scan(mine, warp_tot, sel_total);
+    uint32_t tb = ties_before - esum;  // ties before this thread's first tile
+#pragma unroll
+    for (int u = 0; u < PER; ++u) {
+        if (q0 + u < ntiles) {
+            uint32_t *m = s.meta + ((int64_t)row * p.TT + first + q0 + u) * 4;
+            s.outbase[(int64_t)row * (p.TT + 1) + first + q0 + u] = out;
+            m[3] = allowed[u];
+            m[2] = (tb + allowed[u] == ties_wanted && allowed[u] > 0) ? 1u : 0u;  // holds the last accepted tie
+        }
+        out += g[u] + allowed[u];
+        tb += e[u];
+    }
+    // the last run sees the whole selection
+    if (threadIdx.x == 0 && c0 + SCAN_PART >= ntiles && carry_sel + sel_total != k) atomicOr(p.status, STATUS_COUNT_MISMATCH);
 }
 
 // write: ordered compaction of a tile's candidate block into the message (one warp per tile)
@@ -1033,7 +1048,9 @@ cudaError_t topk_second_part(const Params &p, const TopkSide &s, int src_kind, c
     topk_pick_kernel<<<g_probs, THREADS, 0, st>>>(p, s, 3); CHECK_LAUNCH();
     topk_count_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     LAUNCH_BY_SOURCE(topk_dense_count_kernel, g_strided);
-    topk_scan_kernel<<<g_probs, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
+    const dim3 g_scan(p.T * p.scan_parts, s.R);
+    if (p.scan_parts > 1) { topk_scan_kernel<<<g_scan, THREADS, 0, st>>>(p, s, 0); CHECK_LAUNCH(); }
+    topk_scan_kernel<<<g_scan, THREADS, 0, st>>>(p, s, 1); CHECK_LAUNCH();
     topk_write_kernel<<<g_warp_tiles, THREADS, 0, st>>>(p, s); CHECK_LAUNCH();
     LAUNCH_BY_SOURCE(topk_dense_write_kernel, g_strided);
     topk_close_kernel<<<dim3((p.T + 127) / 128, s.R), 128, 0, st>>>(p, s); CHECK_LAUNCH();
