@@ -26,10 +26,10 @@ struct Region {
 
 struct Plan {
     int32_t N = 0, T = 0, TT = 0, KTT = 0;
-    int64_t d = 0, W = 0, K = 0, CAP = 0, cap_max = 0;
-    std::vector<int64_t> seg_off, word_off, k_off, cap_off, topk_k;
+    int64_t d = 0, W = 0, K = 0, CAP = 0, cap_max = 0, down_CAP = 0;
+    std::vector<int64_t> seg_off, word_off, k_off, cap_off, down_cap_off, topk_k;
     std::vector<int32_t> tile_prefix, tile_seg, small_seg, large_seg, ktile_prefix, ktile_seg;
-    Region r_seg_off, r_word_off, r_k_off, r_cap_off, r_tile_prefix, r_tile_seg, r_small_seg, r_large_seg, r_status;
+    Region r_seg_off, r_word_off, r_k_off, r_cap_off, r_down_cap_off, r_tile_prefix, r_tile_seg, r_small_seg, r_large_seg, r_status;
     Region r_tel_partials, r_tel_e, r_tel_v, r_tel_g, r_tel_kept, r_ktile_prefix, r_ktile_seg;
     Region r_up_words, r_up_scales, r_up_partials, r_down_words, r_down_scales, r_down_partials, r_vbuf;
     Region r_up_idx, r_up_val, r_down_idx, r_down_val;
@@ -94,6 +94,7 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     pl.word_off.assign(T + 1, 0);
     pl.k_off.assign(T + 1, 0);
     pl.cap_off.assign(T + 1, 0);
+    pl.down_cap_off.assign(T + 1, 0);
     pl.tile_prefix.assign(T + 1, 0);
     pl.topk_k.assign(T, 0);
     int64_t tiles = 0;
@@ -111,6 +112,13 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
             if (cap > n) cap = n;
             pl.cap_off[t + 1] = pl.cap_off[t] + cap;
             if (cap > pl.cap_max) pl.cap_max = cap;
+            // The downlink has one row, and in a long segment (a flat vector, an embedding matrix) the
+            // entries of v at or above the start of the threshold's first-digit bin run to several times k
+            // (error feedback piles v up under the threshold): room for 8 k of them costs little there and
+            // saves the dense second-digit pass over the segment in most iterations.
+            int64_t down_cap = cap;
+            if ((n + TILE - 1) / TILE >= LONG_SEG_TILES) down_cap = std::min<int64_t>(n, 8 * k + 2048);
+            pl.down_cap_off[t + 1] = pl.down_cap_off[t] + down_cap;
         }
     }
     // a sparse message's values, tiled like the model (for their squared norms): segment t owns k_t entries
@@ -129,6 +137,7 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     pl.W = pl.word_off[T];
     pl.K = pl.k_off[T];
     pl.CAP = pl.cap_off[T];
+    pl.down_CAP = pl.down_cap_off[T];
     pl.TT = (int32_t)tiles;
     pl.tile_seg.resize(pl.TT);
     for (int t = 0; t < T; ++t) {
@@ -145,6 +154,7 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     pl.r_word_off = c.take(sizeof(int64_t) * (T + 1));
     pl.r_k_off = c.take(sizeof(int64_t) * (T + 1));
     pl.r_cap_off = c.take(sizeof(int64_t) * (T + 1));
+    pl.r_down_cap_off = c.take(sizeof(int64_t) * (T + 1));
     pl.r_tile_prefix = c.take(sizeof(int32_t) * (T + 1));
     pl.r_tile_seg = c.take(sizeof(int32_t) * pl.TT);
     pl.r_small_seg = c.take(sizeof(int32_t) * pl.small_seg.size());
@@ -175,7 +185,7 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     int max_seg_tiles = 0;
     for (int t = 0; t < T; ++t) max_seg_tiles = std::max(max_seg_tiles, pl.tile_prefix[t + 1] - pl.tile_prefix[t]);
     const size_t scan_parts = (size_t)(max_seg_tiles + SCAN_PART - 1) / SCAN_PART;
-    auto topk_regions = [&](size_t rows, Region &idx, Region &val, Region &hist, Region &hist2, Region &sel,
+    auto topk_regions = [&](size_t rows, int64_t cap_total, Region &idx, Region &val, Region &hist, Region &hist2, Region &sel,
                             Region &cidx, Region &cval, Region &meta, Region &outbase, Region &parts) {
         parts = c.take(sizeof(uint32_t) * rows * T * scan_parts * 2);
         idx = c.take(sizeof(uint32_t) * rows * pl.K * 2);  // idx then val, adjacent
@@ -185,8 +195,8 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
         hist = c.take(sizeof(uint32_t) * rows * T * DIGIT1_BINS);
         hist2 = c.take(sizeof(uint32_t) * rows * T * DIGIT1_BINS);
         sel = c.take(sizeof(uint32_t) * rows * T * SEL_WORDS);
-        cidx = c.take(sizeof(uint32_t) * rows * pl.CAP);
-        cval = c.take(sizeof(float) * rows * pl.CAP);
+        cidx = c.take(sizeof(uint32_t) * rows * cap_total);
+        cval = c.take(sizeof(float) * rows * cap_total);
         meta = c.take(sizeof(uint32_t) * rows * pl.TT * 4);
         outbase = c.take(sizeof(uint32_t) * rows * (pl.TT + 1));
     };
@@ -201,13 +211,13 @@ liec_status make_plan(const liec_config *cfg, Plan &pl, std::string *msg) {
     if (cfg->uplink == LIEC_COMP_RANDK) randk_regions(N, pl.r_up_idx, pl.r_up_val, pl.r_up_outbase);
     if (cfg->downlink == LIEC_COMP_RANDK) randk_regions(1, pl.r_down_idx, pl.r_down_val, pl.r_down_outbase);
     if (cfg->uplink == LIEC_COMP_RANDK || cfg->downlink == LIEC_COMP_RANDK)   // scratch of the seeded draw (liec_draw_subsets)
-        topk_regions(N + 1, pl.r_gen_sets, pl.r_gen_val, pl.r_gen_hist, pl.r_gen_hist2, pl.r_gen_sel, pl.r_gen_cand_idx,
+        topk_regions(N + 1, pl.CAP, pl.r_gen_sets, pl.r_gen_val, pl.r_gen_hist, pl.r_gen_hist2, pl.r_gen_sel, pl.r_gen_cand_idx,
                      pl.r_gen_cand_val, pl.r_gen_meta, pl.r_gen_outbase, pl.r_gen_scan_parts);
     if (cfg->uplink == LIEC_COMP_TOPK)
-        topk_regions(N, pl.r_up_idx, pl.r_up_val, pl.r_up_hist, pl.r_up_hist2, pl.r_up_sel, pl.r_up_cand_idx,
+        topk_regions(N, pl.CAP, pl.r_up_idx, pl.r_up_val, pl.r_up_hist, pl.r_up_hist2, pl.r_up_sel, pl.r_up_cand_idx,
                      pl.r_up_cand_val, pl.r_up_tile_meta, pl.r_up_outbase, pl.r_up_scan_parts);
     if (cfg->downlink == LIEC_COMP_TOPK)
-        topk_regions(1, pl.r_down_idx, pl.r_down_val, pl.r_down_hist, pl.r_down_hist2, pl.r_down_sel,
+        topk_regions(1, pl.down_CAP, pl.r_down_idx, pl.r_down_val, pl.r_down_hist, pl.r_down_hist2, pl.r_down_sel,
                      pl.r_down_cand_idx, pl.r_down_cand_val, pl.r_down_tile_meta, pl.r_down_outbase, pl.r_down_scan_parts);
     pl.total = align_up(c.cursor, 256);
     return LIEC_OK;
@@ -366,6 +376,8 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     p.word_off = at<int64_t>(c, pl.r_word_off);
     p.k_off = at<int64_t>(c, pl.r_k_off);
     p.cap_off = at<int64_t>(c, pl.r_cap_off);
+    p.down_cap_off = at<int64_t>(c, pl.r_down_cap_off);
+    p.down_CAP = pl.down_CAP;
     p.tile_prefix = at<int32_t>(c, pl.r_tile_prefix);
     p.tile_seg = at<int32_t>(c, pl.r_tile_seg);
     p.small_seg = at<int32_t>(c, pl.r_small_seg);
@@ -382,10 +394,12 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     }
     p.n_long = 0;
     p.cap_long_max = 0;
+    p.down_cap_long_max = 0;
     if (pl.K > 0) {
         auto tiles_of = [&](int q) { return pl.tile_prefix[pl.large_seg[q] + 1] - pl.tile_prefix[pl.large_seg[q]]; };
         while (p.n_long < p.n_large && tiles_of(p.n_long) >= LONG_SEG_TILES) {
             p.cap_long_max = std::max<int64_t>(p.cap_long_max, pl.cap_off[pl.large_seg[p.n_long] + 1] - pl.cap_off[pl.large_seg[p.n_long]]);
+            p.down_cap_long_max = std::max<int64_t>(p.down_cap_long_max, pl.down_cap_off[pl.large_seg[p.n_long] + 1] - pl.down_cap_off[pl.large_seg[p.n_long]]);
             ++p.n_long;
         }
     }
@@ -436,7 +450,7 @@ liec_status liec_init(const liec_config *cfg, float *params, float *error, void 
     struct Up { const Region *r; const void *src; };
     const Up ups[] = {
         {&pl.r_seg_off, pl.seg_off.data()}, {&pl.r_word_off, pl.word_off.data()}, {&pl.r_k_off, pl.k_off.data()},
-        {&pl.r_cap_off, pl.cap_off.data()}, {&pl.r_tile_prefix, pl.tile_prefix.data()},
+        {&pl.r_cap_off, pl.cap_off.data()}, {&pl.r_down_cap_off, pl.down_cap_off.data()}, {&pl.r_tile_prefix, pl.tile_prefix.data()},
         {&pl.r_tile_seg, pl.tile_seg.data()}, {&pl.r_small_seg, pl.small_seg.data()}, {&pl.r_large_seg, pl.large_seg.data()},
         {&pl.r_ktile_prefix, pl.ktile_prefix.data()}, {&pl.r_ktile_seg, pl.ktile_seg.data()},
     };
@@ -587,6 +601,7 @@ liec_status liec_draw_subsets(liec_ctx *c, uint64_t seed, uint32_t epoch, void *
     s.gen = ScoreStream{(uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32), epoch};
     s.idx = p.gen_sets; s.val = p.gen_val; s.hist = p.gen_hist; s.hist2 = p.gen_hist2; s.sel = p.gen_sel;
     s.cand_idx = p.gen_cand_idx; s.cand_val = p.gen_cand_val; s.meta = p.gen_meta; s.outbase = p.gen_outbase; s.scan_parts = p.gen_scan_parts;
+    s.cap_off = p.cap_off; s.CAP = p.CAP; s.cap_long_max = p.cap_long_max;
     s.zero_out = nullptr;
     s.spec = 1;
     cudaStream_t main_stream = static_cast<cudaStream_t>(stream);

@@ -33,6 +33,7 @@ struct Params {
     const int64_t *word_off;     // [T+1]
     const int64_t *k_off;        // [T+1] (top-k only)
     const int64_t *cap_off;      // [T+1] candidate capacity prefix (top-k only)
+    const int64_t *down_cap_off; // [T+1] the same for the downlink (its long segments get more room: see make_plan)
     const int32_t *tile_prefix;  // [T+1] tiles before segment t
     const int32_t *tile_seg;     // [TT] segment of every tile
     const int32_t *small_seg;    // [n_small] segments of one tile (top-k: selected directly by one CTA)
@@ -42,6 +43,7 @@ struct Params {
     int64_t cap_rest_max;        // largest candidate capacity among the other entries of large_seg
     int32_t n_long;              // leading entries of large_seg with LONG_SEG_TILES tiles or more
     int64_t cap_long_max;        // largest candidate capacity among them
+    int64_t down_CAP, down_cap_long_max;   // the downlink's total and largest long-segment capacity
     // host side only: the context's helper stream and the events that fork / join the tail launch of
     // the big problems (cudaStream_t / cudaEvent_t; NULL = everything on the caller's stream)
     void *tail_stream, *tail_fork, *tail_join;

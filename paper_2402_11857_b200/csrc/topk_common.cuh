@@ -20,6 +20,8 @@ struct TopkSide {
     uint32_t *idx; float *val;            // [R][K] output message
     uint32_t *hist, *hist2, *sel;         // [R][T][...]
     uint32_t *cand_idx; float *cand_val;  // [R][CAP]
+    const int64_t *cap_off;                // [T+1] candidate capacity prefix of this side
+    int64_t CAP, cap_long_max;             // its total; the largest capacity among the long segments
     uint32_t *meta;                        // [R][TT][4]: pos, cnt, n_greater -> unused, ties allowed
     uint32_t *outbase;                     // [R][TT+1]
     uint32_t *scan_parts;                  // [R][T][scan_parts][2]
@@ -34,12 +36,14 @@ inline TopkSide make_side(const Params &p, bool uplink) {
         s.src = p.G; s.row_stride = p.d; s.R = p.N;
         s.idx = p.up_idx; s.val = p.up_val; s.hist = p.up_hist; s.hist2 = p.up_hist2; s.sel = p.up_sel;
         s.cand_idx = p.up_cand_idx; s.cand_val = p.up_cand_val; s.meta = p.up_tile_meta; s.outbase = p.up_outbase; s.scan_parts = p.up_scan_parts;
+        s.cap_off = p.cap_off; s.CAP = p.CAP; s.cap_long_max = p.cap_long_max;
         s.zero_out = nullptr;
         s.spec = 1;
     } else {
         s.src = p.e; s.row_stride = 0; s.R = 1;
         s.idx = p.down_idx; s.val = p.down_val; s.hist = p.down_hist; s.hist2 = p.down_hist2; s.sel = p.down_sel;
         s.cand_idx = p.down_cand_idx; s.cand_val = p.down_cand_val; s.meta = p.down_tile_meta; s.outbase = p.down_outbase; s.scan_parts = p.down_scan_parts;
+        s.cap_off = p.down_cap_off; s.CAP = p.down_CAP; s.cap_long_max = p.down_cap_long_max;
         s.zero_out = p.e;
         s.spec = 0;
     }

@@ -121,7 +121,7 @@ __global__ void __launch_bounds__(THREADS) topk_pick_kernel(const __grid_constan
         sel[SEL_NCAND] = sel[SEL_CAND_COUNT];
         return;
     }
-    const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
+    const uint32_t cap = (uint32_t)(__ldg(s.cap_off + t + 1) - __ldg(s.cap_off + t));
     if (level == 2) {
         sel[SEL_PREFIX] = (sel[SEL_PREFIX] << 12) | r.bin;
         sel[SEL_REMAIN] = r.rank_in_bin;
@@ -323,7 +323,7 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
         uint32_t tile_cnt;
         const uint32_t before = block_exclusive_scan((uint32_t)__popc(mask), warp_tot, tile_cnt);
         if (threadIdx.x == 0) {
-            const uint32_t cap = (uint32_t)(__ldg(p.cap_off + ti.t + 1) - __ldg(p.cap_off + ti.t));
+            const uint32_t cap = (uint32_t)(__ldg(s.cap_off + ti.t + 1) - __ldg(s.cap_off + ti.t));
             uint32_t at = tile_cnt ? atomicAdd(&sel[SEL_CAND_COUNT], tile_cnt) : 0u;
             if (at + tile_cnt > cap) {
                 if (SPEC) {  // the guess lets too much through: this problem takes the regular route
@@ -342,7 +342,7 @@ __global__ void __launch_bounds__(THREADS) topk_filter_tma_kernel(const __grid_c
         __syncthreads();
         const uint32_t base_now = tile_base;
         if (base_now != 0xffffffffu && mask != 0u) {
-            const int64_t cbase = (int64_t)row * p.CAP + __ldg(p.cap_off + ti.t) + base_now + before;
+            const int64_t cbase = (int64_t)row * s.CAP + __ldg(s.cap_off + ti.t) + base_now + before;
             const uint32_t flat0 = (uint32_t)(ti.seg_beg + ti.rel) + pos0;
             uint32_t rest = mask, o = 0;
             while (rest) {  // candidates are rare: usually zero or one iteration
@@ -374,10 +374,10 @@ __device__ __forceinline__ CandBlock cand_block(const Params &p, const TopkSide 
     cb.seg_tiles = ti.seg_tiles;
     cb.sel = s.sel + ((int64_t)row * p.T + ti.t) * SEL_WORDS;
     const uint32_t flags = cb.sel[SEL_FLAGS];
-    const int64_t cap0 = __ldg(p.cap_off + ti.t);
+    const int64_t cap0 = __ldg(s.cap_off + ti.t);
     cb.skip = (flags & 1u) != 0u || ti.seg_tiles == 1;
     cb.cnt = cb.skip ? 0u : cb.m.y;
-    cb.base = (int64_t)row * p.CAP + cap0 + cb.m.x;
+    cb.base = (int64_t)row * s.CAP + cap0 + cb.m.x;
     return cb;
 }
 
@@ -451,10 +451,10 @@ __global__ void __launch_bounds__(THREADS) topk_cand_hist_long_kernel(const __gr
     uint32_t *sel = s.sel + ((int64_t)row * p.T + t) * SEL_WORDS;
     const uint32_t flags = sel[SEL_FLAGS];
     if ((flags & 1u) || (level == 0 && sel[SEL_MODE] != 1u) || (level == 1 && flags != 0u)) return;   // (uniform over the CTA)
-    const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
+    const uint32_t cap = (uint32_t)(__ldg(s.cap_off + t + 1) - __ldg(s.cap_off + t));
     const uint32_t ncand = min(sel[SEL_CAND_COUNT], cap);
     // positions are counted from the 16-byte boundary at or before the region's first candidate
-    const int64_t base = (int64_t)row * p.CAP + __ldg(p.cap_off + t);
+    const int64_t base = (int64_t)row * s.CAP + __ldg(s.cap_off + t);
     const uint32_t lead = (uint32_t)(base & 3);
     const float *al = s.cand_val + (base - lead);
     const uint32_t end = lead + ncand;
@@ -982,9 +982,9 @@ static cudaError_t launch_cand_hist(const Params &p, const TopkSide &s, int leve
     }
     if (p.n_long > 0) {
         // (four runs per CTA from 2^24 candidate slots up; three more positions cover a region that starts off a 16-byte boundary)
-        const int batches = p.cap_long_max * p.n_long * s.R >= (int64_t)1 << 24 ? 4 : 1;
+        const int batches = s.cap_long_max * p.n_long * s.R >= (int64_t)1 << 24 ? 4 : 1;
         const int64_t per_cta = (int64_t)batches * CAND_RUN;
-        const int chunks = (int)((p.cap_long_max + 3 + per_cta - 1) / per_cta);
+        const int chunks = (int)((s.cap_long_max + 3 + per_cta - 1) / per_cta);
         topk_cand_hist_long_kernel<<<dim3(p.n_long * chunks, s.R), THREADS, 0, st>>>(p, s, level, chunks, batches);
         CHECK_LAUNCH();
     }

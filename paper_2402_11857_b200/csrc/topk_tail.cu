@@ -214,7 +214,7 @@ __global__ void __launch_bounds__(NT, 1024 / NT) topk_tail_kernel(const __grid_c
     if (s.spec && blockIdx.x == 0 && row == 0 && threadIdx.x == 0) p.status[STATUS_ANY_REGULAR] = 0;
     const uint32_t flags = sel[SEL_FLAGS];
     const bool single = s.spec && sel[SEL_MODE] == 1u;
-    const uint32_t cap = (uint32_t)(__ldg(p.cap_off + t + 1) - __ldg(p.cap_off + t));
+    const uint32_t cap = (uint32_t)(__ldg(s.cap_off + t + 1) - __ldg(s.cap_off + t));
     const uint32_t k = (uint32_t)(__ldg(p.k_off + t + 1) - __ldg(p.k_off + t));
     const uint32_t kbeg = (uint32_t)__ldg(p.k_off + t);
     const uint32_t ncand = min(sel[SEL_CAND_COUNT], cap);  // (the cursor can run past the buffer when a tile was refused)
@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(NT, 1024 / NT) topk_tail_kernel(const __grid_c
         }
         return;
     }
-    const int64_t cbase = (int64_t)row * p.CAP + __ldg(p.cap_off + t);
+    const int64_t cbase = (int64_t)row * s.CAP + __ldg(s.cap_off + t);
     const float *cand = s.cand_val + cbase;
     const uint32_t *cidx = s.cand_idx + cbase;
     auto fail = [&](int bit) { if (threadIdx.x == 0) { atomicOr(p.status, bit); if (s.spec) sel[SEL_GUESS] = 0u; } };
