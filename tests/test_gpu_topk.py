@@ -177,6 +177,18 @@ def test_long_segment_whose_candidate_region_starts_off_a_16_byte_boundary():
     assert P.ctx.liec_topk_route_counts(True)["single_pass"] >= 2     # (the guess route, with its first-digit candidate histogram, ran)
 
 
+def test_segment_of_more_than_4096_tiles_between_others():
+    """A 33.6 M-element tensor (4101 tiles: two runs of the tile scan, whose second run starts from the
+    sums of the first) between a mid-size and a small one, k = 0.5 %; the second step runs on the
+    guess route."""
+    lay = Layout("runs", (300_000, 4100 * 8192 + 7, 5000))
+    k = topk_counts(lay, 1, 200)
+    P = _pair(2, lay.seg_offsets, TOPK, TOPK, k=k)
+    for step in range(2):
+        G = make_gradients("normal", 1.0, 2, lay.dim, step, base_seed=28)
+        P.step(G, 0.1)
+
+
 def test_bf16_topk():
     lay = ragged_layout()
     k = topk_counts(lay, 1, 50)
