@@ -155,7 +155,7 @@ def test_many_candidates_take_the_wide_finish():
 
 def test_segment_of_more_than_1024_tiles_gathers_candidate_histograms():
     """A 9 M-element tensor (1099 tiles) with k = 1 %: the wide finish step, with the candidate
-    histograms of 64 tiles gathered in shared memory before they reach the segment's histogram."""
+    histograms taken over the segment's whole candidate region (the long-segment form)."""
     lay = Layout("huge", (9_000_000, 3000))
     k = np.asarray([90_000, 30], np.int64)
     P = _pair(2, lay.seg_offsets, TOPK, TOPK, k=k)
