@@ -116,6 +116,15 @@ __global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK || TEL ? 3 : 0)) w
         }
         uint32_t own_nib = 0u;
         if (UP == COMP_RANDK) own_nib = own_mask[wq][pos >> 5] >> (pos & 31);  // pos is a multiple of 4: the four bits share a word
+        // top-k: entries exactly at the threshold are rare (the k-th largest itself, plus its ties): only a row
+        // of the warp that holds one compares indices with the cut
+        bool row_has_tie = false;
+        if (UP == COMP_TOPK) {
+            bool mine = false;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) mine |= (__float_as_uint(g[j][c]) & 0x7fffffffu) == up_thresh;
+            row_has_tie = __any_sync(0xffffffffu, mine);
+        }
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             float pi;
@@ -125,8 +134,11 @@ __global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK || TEL ? 3 : 0)) w
                 pi = __uint_as_float(su_bits ^ (g[j][c] < 0.0f ? 0x80000000u : 0u));
             } else if (UP == COMP_TOPK) {
                 const uint32_t key = __float_as_uint(g[j][c]) & 0x7fffffffu;
-                const uint32_t flat = (uint32_t)(ti.seg_beg + ti.rel) + pos + c;
-                const bool kept = key > up_thresh || (key == up_thresh && flat <= up_cut);
+                bool kept = key > up_thresh;
+                if (row_has_tie) {   // (uniform over the warp)
+                    const uint32_t flat = (uint32_t)(ti.seg_beg + ti.rel) + pos + c;
+                    kept = kept || (key == up_thresh && flat <= up_cut);
+                }
                 pi = kept ? g[j][c] : 0.0f;
             } else {
                 pi = g[j][c];
