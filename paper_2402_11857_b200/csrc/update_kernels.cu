@@ -18,6 +18,13 @@ __global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK || TEL ? 3 : 0)) w
     constexpr int WPC = DOWN == COMP_TOPK ? 4 : 1;
     __shared__ double tel_sums[TEL ? WPC : 1][TEL ? 8 : 1];
     __shared__ uint32_t own_mask[UP == COMP_RANDK ? WPC : 1][UP == COMP_RANDK ? TILE_WORDS : 1];  // each worker's own subset inside this tile
+    // (a sparse downlink: the tile's range in the message is fetched first, so that the entries themselves can be
+    // requested right behind the first worker's streaming loads instead of two latencies later)
+    uint32_t down_beg = 0, down_end_next = 0;
+    if (DOWN == COMP_TOPK) {
+        down_beg = p.down_outbase[blockIdx.x];
+        down_end_next = p.down_outbase[blockIdx.x + 1];   // ([TT + 1] entries; the segment's last tile ends at its k-range instead)
+    }
     const TileInfo ti = locate_tile(p, blockIdx.x);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int wq = 0; wq < WPC; ++wq) {
@@ -62,14 +69,20 @@ __global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK || TEL ? 3 : 0)) w
 
     // decode the downlink top-k message of this tile (after the streaming loads are in flight)
     if (DOWN == COMP_TOPK && wq == 0) {
+        const bool last_tile = (blockIdx.x + 1 == __ldg(p.tile_prefix + ti.t + 1));
+        const uint32_t beg = down_beg;
+        const uint32_t end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : down_end_next;
+        const uint32_t tile_first = (uint32_t)(ti.seg_beg + ti.rel);
+        // the first entry of every thread is requested before the tile is cleared
+        const uint32_t q0 = beg + threadIdx.x;
+        uint32_t o0 = 0xffffffffu;
+        float val0 = 0.0f;
+        if (q0 < end) { o0 = p.down_idx[q0] - tile_first; val0 = p.down_val[q0]; }
         for (int q = threadIdx.x; q < TILE / 4; q += THREADS)
             reinterpret_cast<float4 *>(p_tile)[q] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         __syncthreads();
-        const bool last_tile = (blockIdx.x + 1 == __ldg(p.tile_prefix + ti.t + 1));
-        const uint32_t beg = p.down_outbase[blockIdx.x];
-        const uint32_t end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : p.down_outbase[blockIdx.x + 1];
-        const uint32_t tile_first = (uint32_t)(ti.seg_beg + ti.rel);
-        for (uint32_t q = beg + threadIdx.x; q < end; q += THREADS) {
+        if (o0 < (uint32_t)TILE) p_tile[o0] = val0;
+        for (uint32_t q = q0 + THREADS; q < end; q += THREADS) {
             const uint32_t o = p.down_idx[q] - tile_first;
             if (o < (uint32_t)TILE) p_tile[o] = p.down_val[q];
         }
