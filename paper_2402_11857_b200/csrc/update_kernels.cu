@@ -51,6 +51,14 @@ __global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK || TEL ? 3 : 0)) w
         up_thresh = sel[SEL_THRESH];
         up_cut = sel[SEL_CUT];
     }
+    // element c of a quad whose first flat index is r is kept iff key > T, or key == T and r + c <= cut, i.e.
+    // ~r >= ~cut + c (which cannot wrap when cut >= c; when cut < c no index r + c can be at or below the cut and
+    // the bound asks for key > T alone)
+    unsigned long long kept_bound[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        kept_bound[c] = up_cut >= (uint32_t)c ? (((unsigned long long)up_thresh << 32) | (uint32_t)(~up_cut + (uint32_t)c))
+                                               : ((unsigned long long)(up_thresh + 1u) << 32);
     const float *v_tile = DOWN == COMP_IDENTITY ? p.vbuf + ti.seg_beg + ti.rel : nullptr;
 
     float g[8][4], x[8][4];
@@ -129,15 +137,9 @@ __global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK || TEL ? 3 : 0)) w
         }
         uint32_t own_nib = 0u;
         if (UP == COMP_RANDK) own_nib = own_mask[wq][pos >> 5] >> (pos & 31);  // pos is a multiple of 4: the four bits share a word
-        // top-k: entries exactly at the threshold are rare (the k-th largest itself, plus its ties): only a row
-        // of the warp that holds one compares indices with the cut
-        bool row_has_tie = false;
-        if (UP == COMP_TOPK) {
-            bool mine = false;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) mine |= (__float_as_uint(g[j][c]) & 0x7fffffffu) == up_thresh;
-            row_has_tie = __any_sync(0xffffffffu, mine);
-        }
+        // top-k: kept <=> (key, ~index) >= (threshold, ~cut) as one 64-bit comparison; the row's index part is
+        // formed once, the per-element offset sits in the bound (see kept_bound)
+        const uint32_t row_low = ~((uint32_t)(ti.seg_beg + ti.rel) + (uint32_t)pos);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             float pi;
@@ -147,11 +149,7 @@ __global__ void __launch_bounds__(THREADS, (DOWN == COMP_TOPK || TEL ? 3 : 0)) w
                 pi = __uint_as_float(su_bits ^ (g[j][c] < 0.0f ? 0x80000000u : 0u));
             } else if (UP == COMP_TOPK) {
                 const uint32_t key = __float_as_uint(g[j][c]) & 0x7fffffffu;
-                bool kept = key > up_thresh;
-                if (row_has_tie) {   // (uniform over the warp)
-                    const uint32_t flat = (uint32_t)(ti.seg_beg + ti.rel) + pos + c;
-                    kept = kept || (key == up_thresh && flat <= up_cut);
-                }
+                const bool kept = (((unsigned long long)key << 32) | row_low) >= kept_bound[c];
                 pi = kept ? g[j][c] : 0.0f;
             } else {
                 pi = g[j][c];

@@ -189,6 +189,20 @@ def test_segment_of_more_than_4096_tiles_between_others():
         P.step(G, 0.1)
 
 
+@pytest.mark.parametrize("k0", [1, 2, 3, 4, 5])
+def test_all_equal_magnitudes_keep_the_first_indices_of_the_vector(k0):
+    """Every entry of the first segments has the same magnitude, so the threshold ties everywhere and the
+    cut (last accepted tie) is flat index k - 1 = 0 ... 4, inside the first quad of the vector: the
+    worker update must drop the quad's other entries although they equal the threshold."""
+    lay = Layout("equal", (9000, 300, 20000))
+    k = np.asarray([k0, k0, 200], np.int64)
+    P = _pair(2, lay.seg_offsets, TOPK, TOPK, k=k)
+    for step in range(2):
+        G = make_gradients("normal", 1.0, 2, lay.dim, step, base_seed=29)
+        G[:, :9300] = torch.where(G[:, :9300] < 0, -0.5, 0.5)
+        P.step(G, 0.1)
+
+
 def test_bf16_topk():
     lay = ragged_layout()
     k = topk_counts(lay, 1, 50)
