@@ -94,7 +94,7 @@ def update_kernel_bytes(w) -> float:
 # this streaming kernel's traffic grows in proportion; c3 and c2: captured at full size (the tail
 # of the parameter writes is still in the L2 when the kernel ends, hence slightly fewer bytes than
 # the algorithmic count).  Any other workload or variant: not captured.
-UPDATE_TRAFFIC_BYTES = {"c4": (2.989412e9 + 1.934865e9) / 497759232 * 32 * 124439808, "c3": 3274351104 + 1583016704,
+UPDATE_TRAFFIC_BYTES = {"c4": (2.989412e9 + 1.934865e9) / 497759232 * 32 * 124439808, "c3": 3274712064 + 1583202304,
                         "c2": 749630720 + 322008320}
 
 
