@@ -857,40 +857,47 @@ __global__ void __launch_bounds__(THREADS, TEL ? 3 : 4) server_topk_kernel(const
     // barrier apart, so that every element sees its contributions in worker order.  Inside one
     // worker's turn the indices are distinct, so its additions do not depend on one another.
     constexpr int WG = 8;
-    for (int g0 = 0; g0 < p.N; g0 += WG) {
-        if (threadIdx.x < WG) {
-            const int i = g0 + threadIdx.x;
+    const int tid = threadIdx.x, num_workers = p.N;
+    const int64_t K = p.K;
+    const uint32_t *idx_row = p.up_idx;   // the current group's first message
+    const float *val_row = p.up_val;
+    for (int g0 = 0; g0 < num_workers; g0 += WG, idx_row += WG * K, val_row += WG * K) {
+        if (tid < WG) {
+            const int i = g0 + tid;
             uint32_t beg = 0, end = 0;
-            if (i < p.N) {
+            if (i < num_workers) {
                 const uint32_t *ob = p.up_outbase + (int64_t)i * (p.TT + 1) + blockIdx.x;
                 beg = ob[0];
                 end = last_tile ? (uint32_t)__ldg(p.k_off + ti.t + 1) : ob[1];
             }
-            s_beg[threadIdx.x] = beg;
-            s_end[threadIdx.x] = end;
+            s_beg[tid] = beg;
+            s_end[tid] = end;
         }
         __syncthreads();
         uint32_t pidx[WG];
         float pval[WG];
         uint32_t crowded = 0;   // workers with more than 256 entries in this tile (uniform over the CTA)
+        {
+            const uint32_t *ip = idx_row;
+            const float *vp = val_row;
 #pragma unroll
-        for (int u = 0; u < WG; ++u) {
-            const uint32_t q = s_beg[u] + threadIdx.x;
-            const bool have = q < s_end[u];   // (beg = end = 0 for workers beyond N)
-            crowded |= (s_end[u] - s_beg[u] > (uint32_t)THREADS ? 1u : 0u) << u;
-            const int64_t at = (int64_t)(g0 + u) * p.K + q;
-            pidx[u] = have ? p.up_idx[at] : 0xffffffffu;
-            pval[u] = have ? p.up_val[at] : 0.0f;
+            for (int u = 0; u < WG; ++u, ip += K, vp += K) {
+                const uint32_t q = s_beg[u] + tid;
+                const bool have = q < s_end[u];   // (beg = end = 0 for workers beyond N)
+                crowded |= (s_end[u] - s_beg[u] > (uint32_t)THREADS ? 1u : 0u) << u;
+                pidx[u] = have ? ip[q] : 0xffffffffu;
+                pval[u] = have ? vp[q] : 0.0f;
+            }
         }
 #pragma unroll
         for (int u = 0; u < WG; ++u) {
-            if (g0 + u < p.N) {  // uniform over the CTA
+            if (g0 + u < num_workers) {  // uniform over the CTA
                 const uint32_t o = pidx[u] - tile_first;
                 if (o < (uint32_t)TILE) acc[o] = __fadd_rn(acc[o], pval[u]);  // (absent entries and those of a refused subset fall outside)
                 if ((crowded >> u) & 1u) {
-                    const uint32_t *idx = p.up_idx + (int64_t)(g0 + u) * p.K;
-                    const float *val = p.up_val + (int64_t)(g0 + u) * p.K;
-                    for (uint32_t q = s_beg[u] + threadIdx.x + THREADS; q < s_end[u]; q += THREADS) {
+                    const uint32_t *idx = idx_row + (int64_t)u * K;
+                    const float *val = val_row + (int64_t)u * K;
+                    for (uint32_t q = s_beg[u] + tid + THREADS; q < s_end[u]; q += THREADS) {
                         const uint32_t o2 = idx[q] - tile_first;
                         if (o2 < (uint32_t)TILE) acc[o2] = __fadd_rn(acc[o2], val[q]);
                     }
