@@ -251,7 +251,7 @@ __global__ void __launch_bounds__(NT, 1024 / NT) topk_tail_kernel(const __grid_c
 
     // Sweeps over the candidates' values: a thread fetches B values (B stripes of NT consecutive
     // candidates) before it uses any, so that the loads are in flight together.
-    constexpr int B = 8;
+    constexpr int B = 16;
     auto sweep_keys = [&](auto &&use) {   // use(key) for every candidate of this thread
         for (uint32_t q0 = threadIdx.x; q0 < ncand; q0 += NT * B) {
             uint32_t key[B];
