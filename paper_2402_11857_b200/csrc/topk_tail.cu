@@ -332,7 +332,7 @@ __global__ void __launch_bounds__(NT, 1024 / NT) topk_tail_kernel(const __grid_c
     // the two bitmaps, and per tile the number of entries above the threshold and equal to it.
     // The tile of a candidate follows from its index.
     const uint32_t nwords = (ncand + 31) >> 5;
-    constexpr int BX = 4;
+    constexpr int BX = 8;
     for (uint32_t q0 = threadIdx.x & ~31u; q0 < ncand; q0 += NT * BX) {   // (bounds uniform over the warp)
         uint32_t key[BX], tile[BX];
 #pragma unroll
